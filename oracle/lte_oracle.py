@@ -1,0 +1,162 @@
+"""ctypes front end of the fp64 CPU oracle (``lte_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: imported by the tests, the smoke check and the
+benchmark's cpu_baseline / reference arm.  It shares nothing with the CUDA
+library.  Every function widens its inputs to float64 (exact for fp32 and bf16
+values) and returns float64 / int32 numpy arrays.
+"""
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "lte_oracle.c")
+_LIB = os.path.join(_HERE, "liblte_oracle.so")
+_lib = None
+
+
+def build(force=False):
+    """Compile the oracle with gcc (-O2 -fopenmp) if the .so is missing or stale."""
+    if (not force and os.path.exists(_LIB)
+            and os.path.getmtime(_LIB) >= os.path.getmtime(_SRC)):
+        return _LIB
+    tmp = _LIB + ".tmp.%d" % os.getpid()
+    subprocess.check_call(["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c99",
+                           "-o", tmp, _SRC, "-lm"])
+    os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        _lib.oracle_num_threads.restype = ctypes.c_int
+    return _lib
+
+
+def _f64(a):
+    return np.ascontiguousarray(np.asarray(a, dtype=np.float64))
+
+
+def _i32(a):
+    return np.ascontiguousarray(np.asarray(a, dtype=np.int32))
+
+
+def _p(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def num_threads():
+    return int(_load().oracle_num_threads())
+
+
+def logit(tau):
+    """Keep iff r > tau  <=>  z > logit(tau); tau <= 0 keeps every scored token."""
+    if tau <= 0.0:
+        return -np.inf
+    if tau >= 1.0:
+        return np.inf
+    return float(np.log(tau) - np.log1p(-tau))
+
+
+def scores(k, v, w, bias=None):
+    """Single-layer scorer: k, v [B,H,T,d], w [H,K,2d], bias [H] -> z [B,H,T]."""
+    k, v, w = _f64(k), _f64(v), _f64(w)
+    B, H, T, d = k.shape
+    K = w.shape[1]
+    assert w.shape == (H, K, 2 * d)
+    bias = None if bias is None else _f64(bias)
+    z = np.empty((B, H, T), np.float64)
+    _load().oracle_scores(B, H, T, d, K, _p(k), _p(v), _p(w), _p(bias), _p(z))
+    return z
+
+
+def scores_stack(k, v, wl, bl, wout, bout, ks=3, dil=2):
+    """The paper's conv stack: wl[l] [H,c_{l+1},ks,c_l], bl[l] [H,c_{l+1}] or None,
+    wout [H,c_L], bout [H] or None -> z [B,H,T]."""
+    k, v = _f64(k), _f64(v)
+    B, H, T, d = k.shape
+    L = len(wl)
+    wl = [_f64(x) for x in wl]
+    bl = [None if x is None else _f64(x) for x in bl]
+    ch = [2 * d] + [x.shape[1] for x in wl]
+    for l in range(L):
+        assert wl[l].shape == (H, ch[l + 1], ks, ch[l])
+    wout = _f64(wout)
+    bout = None if bout is None else _f64(bout)
+    ch_a = (ctypes.c_int * (L + 1))(*ch)
+    wl_a = (ctypes.c_void_p * L)(*[x.ctypes.data for x in wl])
+    bl_a = (ctypes.c_void_p * L)(*[None if x is None else x.ctypes.data for x in bl])
+    z = np.empty((B, H, T), np.float64)
+    _load().oracle_scores_stack(B, H, T, d, L, ks, dil, ch_a, wl_a, bl_a,
+                                _p(wout), _p(bout), _p(k), _p(v), _p(z))
+    return z
+
+
+def select(z, W, R, sink=0, tau=0.5):
+    """One-shot capped selection -> idx [B,H,R] ascending (-1 unused), cnt, ncand."""
+    z = _f64(z)
+    B, H, T = z.shape
+    idx = np.empty((B, H, max(R, 0)), np.int32)
+    cnt = np.empty((B, H), np.int32)
+    ncand = np.empty((B, H), np.int32)
+    _load().oracle_select(B, H, T, W, R, sink, ctypes.c_double(logit(tau)),
+                          _p(z), _p(idx), _p(cnt), _p(ncand))
+    return idx, cnt, ncand
+
+
+def attn_prefill(q, k, v, idx, cnt, W, scale=None, qpos=None):
+    """Window + retained softmax attention -> o [B,H,nq,d], lse [B,H,nq]."""
+    q, k, v = _f64(q), _f64(k), _f64(v)
+    B, H, T, d = q.shape
+    idx, cnt = _i32(idx), _i32(cnt)
+    R = idx.shape[2]
+    scale = 1.0 / np.sqrt(d) if scale is None else float(scale)
+    if qpos is None:
+        nq = T
+    else:
+        qpos = _i32(qpos)
+        nq = qpos.shape[2]
+    o = np.empty((B, H, nq, d), np.float64)
+    lse = np.empty((B, H, nq), np.float64)
+    _load().oracle_attn_prefill(B, H, T, d, W, R, ctypes.c_double(scale), _p(q), _p(k), _p(v),
+                                _p(idx), _p(cnt), _p(qpos), nq, _p(o), _p(lse))
+    return o, lse
+
+
+def stream(q, k, v, z, W, R, sink=0, tau=0.5, scale=None, n_from=0):
+    """Token-by-token simulation from an empty cache; outputs for steps >= n_from
+    and the final pool (ascending positions)."""
+    q, k, v, z = _f64(q), _f64(k), _f64(v), _f64(z)
+    B, H, T, d = q.shape
+    scale = 1.0 / np.sqrt(d) if scale is None else float(scale)
+    o = np.empty((B, H, T - n_from, d), np.float64)
+    lse = np.empty((B, H, T - n_from), np.float64)
+    pidx = np.empty((B, H, max(R, 0)), np.int32)
+    pcnt = np.empty((B, H), np.int32)
+    _load().oracle_stream(B, H, T, d, W, R, sink, ctypes.c_double(logit(tau)),
+                          ctypes.c_double(scale), n_from, _p(q), _p(k), _p(v), _p(z),
+                          _p(o), _p(lse), _p(pidx), _p(pcnt))
+    return o, lse, pidx, pcnt
+
+
+def attn_bwd(q, k, v, dO, z, idx, cnt, w, W, scale=None, tau=0.5, lam=None,
+             cnn_input_grad=True):
+    """Backward with the straight-through surrogate -> dict(dq, dk, dv, dw, dbias, dz)."""
+    q, k, v, dO, z, w = _f64(q), _f64(k), _f64(v), _f64(dO), _f64(z), _f64(w)
+    B, H, T, d = q.shape
+    idx, cnt = _i32(idx), _i32(cnt)
+    R = idx.shape[2]
+    K = w.shape[1]
+    scale = 1.0 / np.sqrt(d) if scale is None else float(scale)
+    lam = None if lam is None else _f64(lam)
+    dq = np.empty_like(q); dk = np.empty_like(q); dv = np.empty_like(q)
+    dw = np.empty_like(w); db = np.empty((H,), np.float64); dz = np.empty((B, H, T), np.float64)
+    _load().oracle_attn_bwd(B, H, T, d, W, R, K, ctypes.c_double(scale),
+                            ctypes.c_double(logit(tau)), int(bool(cnn_input_grad)),
+                            _p(q), _p(k), _p(v), _p(dO), _p(z), _p(idx), _p(cnt), _p(w), _p(lam),
+                            _p(dq), _p(dk), _p(dv), _p(dw), _p(db), _p(dz))
+    return dict(dq=dq, dk=dk, dv=dv, dw=dw, dbias=db, dz=dz)
