@@ -1,0 +1,173 @@
+/*
+ * liblte — learnable-token-eviction (LTE) sparse attention for NVIDIA B200 (sm_100a).
+ *
+ * C ABI.  Every tensor pointer is a DEVICE pointer owned by the caller, contiguous with the
+ * last index fastest and 16-byte aligned; `lte_shape` / `lte_conv` themselves are HOST structs
+ * (their `w` / `bias` members are device pointers).  Unless a function says otherwise the
+ * library allocates nothing, keeps no global state, and every call is asynchronous on `stream`
+ * (a cudaStream_t passed as void*; NULL = the legacy default stream).  Scratch memory is the
+ * caller's: ask lte_workspace_bytes() and pass at least that many bytes.
+ *
+ * Return value: LTE_OK (0) or a negative lte_status; nothing throws or aborts across the ABI.
+ * Host-side validation happens before anything is launched.
+ *
+ * Notation (0-based positions): W = sliding window, i.e. query i sees keys i-W < j <= i
+ * (W keys including itself); R = retain budget (the paper's b); sink = number of leading
+ * positions that are always kept (the paper's s); K = taps of the scorer; half = K/2;
+ * z = pre-sigmoid logit of the scorer, r = sigmoid(z) the retention score; a token is a
+ * keep candidate iff r > tau, evaluated as z > logit(tau).
+ */
+#ifndef LTE_H_
+#define LTE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum lte_status {
+    LTE_OK = 0,
+    LTE_ERR_INVALID_ARG = -1,      /* NULL pointer, misaligned pointer, non-positive size, even K, W < K ... */
+    LTE_ERR_UNSUPPORTED = -2,      /* a shape or dtype no kernel covers (see each function)                 */
+    LTE_ERR_WORKSPACE = -3,        /* ws_bytes smaller than lte_workspace_bytes() for this call             */
+    LTE_ERR_CUDA = -4,             /* a CUDA runtime / driver call failed (launch, tensor-map encode ...)   */
+    LTE_ERR_ARCH = -5,             /* current device is not compute capability 10.x                        */
+    LTE_ERR_DEVICE_STATUS = -6     /* a kernel recorded an anomaly (bounded wait expired, bad state)        */
+} lte_status;
+
+enum { LTE_F32 = 0, LTE_BF16 = 1 };
+
+typedef struct lte_shape {
+    int32_t B, H, T, d;            /* batch, heads, sequence length, head dim (32, 64 or 128)            */
+    int32_t W, R, sink;            /* window, retain budget, attention-sink size                          */
+    float   tau;                   /* keep threshold on r; 0.5 in the paper.  tau <= 0 keeps every scored token */
+    float   softmax_scale;         /* <= 0 selects 1/sqrt(d)                                               */
+    int32_t dtype;                 /* LTE_F32 or LTE_BF16: storage type of q, k, v, o and their gradients   */
+} lte_shape;
+
+typedef struct lte_conv {
+    int32_t n_layers;              /* 1: the single grouped conv layer 2d -> 1 per head                    */
+    int32_t kernel;                /* K taps, odd, centred (half past, self, half future)                   */
+    int32_t dilation;              /* 1                                                                     */
+    const float* w;                /* device, [H, K, 2d] fp32; channels [0,d) weigh k, [d,2d) weigh v       */
+    const float* bias;             /* device, [H] fp32, or NULL for zero                                    */
+} lte_conv;
+
+typedef enum lte_op {
+    LTE_OP_SCORES = 0, LTE_OP_SELECT = 1, LTE_OP_PREFILL = 2, LTE_OP_DECODE = 3, LTE_OP_BWD = 4
+} lte_op;
+
+/* Bytes of caller-supplied scratch the given entry point needs for this shape (0 if none). */
+size_t lte_workspace_bytes(int op, const lte_shape* s, const lte_conv* c);
+
+/* Static text for a status code. */
+const char* lte_strerror(int status);
+
+/*
+ * Retention logits (Section 3.1.1, "LTE module"; the single-layer width-K scorer):
+ *   z[b,h,j] = bias[h] + sum_{t<K} sum_{c<2d} w[h,t,c] * x[b,h,j+t-half,c],  x = [k ; v],
+ * with x = 0 left of position 0 and no right padding: z = -inf for j > T-1-half (that token's
+ * future context does not exist yet).  fp32 accumulation over the exact input values.
+ *   k, v      in   [B,H,T,d] of s->dtype
+ *   z         out  [B,H,T] fp32
+ *   r_or_null out  [B,H,T] fp32 sigmoid(z) (0 where z = -inf), or NULL
+ * Errors: INVALID_ARG (NULL, even K, n_layers != 1, dilation != 1, d not in {32,64,128}).
+ */
+int lte_scores(const lte_shape* s, const lte_conv* c, const void* k, const void* v,
+               float* z, float* r_or_null, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Capped retention list after a T-token prompt (Eq. 5 restricted to tokens already out of the
+ * final window; Section 3.1.3 "Capped capacity": at most R per head, top-R scores on overflow).
+ * Candidates: j <= T-1-W with (j < sink or z_j > logit(tau)).  Order: sink positions first, then
+ * z descending, ties to the older token.  The first min(R, #candidates) are kept and written in
+ * ascending position order.
+ *   z             in   [B,H,T] fp32
+ *   idx           out  [B,H,R] int32, ascending, unused entries = -1
+ *   cnt           out  [B,H]   int32, number kept (<= R)
+ *   ncand_or_null out  [B,H]   int32, number of candidates before the cap, or NULL
+ * Deterministic and exact on the given z.  Errors: INVALID_ARG; UNSUPPORTED if T-W > 2^24.
+ */
+int lte_select(const lte_shape* s, const float* z, int32_t* idx, int32_t* cnt,
+               int32_t* ncand_or_null, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Prefill attention (Section 3.1.3, "Cached prefilling and decoding"): query i attends over
+ * A_i = {max(0,i-W+1) .. i}  U  {j in idx[b,h,:cnt] : j <= i-W}:
+ *   o_i = softmax_{j in A_i}(scale * q_i.k_j) v_j,   lse_i = log sum_{j in A_i} exp(scale * q_i.k_j).
+ * bf16: tensor-core MMA with fp32 accumulation and fp32 softmax, o rounded to bf16.  fp32: fp32 throughout.
+ *   q, k, v  in   [B,H,T,d] of s->dtype
+ *   idx, cnt in   as written by lte_select (idx ascending; entries >= cnt ignored)
+ *   o        out  [B,H,T,d] of s->dtype
+ *   lse      out  [B,H,T] fp32 (natural log)
+ * Errors: INVALID_ARG, UNSUPPORTED (d not in {32,64,128}), CUDA.
+ */
+int lte_attn_prefill(const lte_shape* s, const void* q, const void* k, const void* v,
+                     const int32_t* idx, const int32_t* cnt, void* o, float* lse,
+                     void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Decode cache (Fig. 3): per (b,h) a ring of the last W keys/values (slot = position mod W) with
+ * their logits, and a pool of at most R retained keys/values with their logits and positions.
+ * The cache is one caller-owned device buffer of lte_cache_bytes() bytes; copying it is a
+ * checkpoint.  T in the shape is ignored by lte_cache_bytes.
+ */
+size_t lte_cache_bytes(const lte_shape* s);
+
+/*
+ * State after a T-token prompt: ring <- last min(T,W) rows of k, v and their logits from z (the
+ * last `half` prompt tokens are still unscored and are scored by the first decode steps), pool <-
+ * rows idx[:cnt] of k, v with their logits.  T = 0 gives the empty cache (k, v, z, idx, cnt may
+ * then be NULL).  Requires W >= K.
+ */
+int lte_cache_init(const lte_shape* s, const lte_conv* c, const void* k, const void* v,
+                   const float* z, const int32_t* idx, const int32_t* cnt, void* cache, void* stream);
+
+/*
+ * One decode step for every (b,h) (Section 3.1.3, decoding paragraph), token n = tokens seen so far:
+ *   1. the token leaving the window, p = n-W (if >= 0), is offered to the pool: ignored unless
+ *      (p < sink or z_p > logit(tau)); appended if the pool holds fewer than R entries; otherwise it
+ *      replaces the lowest-logit entry (the youngest among equals, never a sink entry) iff z_p is
+ *      strictly greater;
+ *   2. k1, v1 are written to ring slot n mod W;
+ *   3. the newest token whose receptive field is now complete, j = n-half, is scored from the ring;
+ *   4. o1, lse1 = attention of q1 over the ring (min(n+1, W) entries) and the pool.
+ *   cache        in/out
+ *   q1, k1, v1   in   [B,H,d] of s->dtype
+ *   o1           out  [B,H,d] of s->dtype;   lse1 out [B,H] fp32
+ * s->T is ignored.  Errors: INVALID_ARG, UNSUPPORTED (W + R > 4096, d not in {32,64,128}), CUDA.
+ */
+int lte_attn_decode(const lte_shape* s, const lte_conv* c, void* cache,
+                    const void* q1, const void* k1, const void* v1, void* o1, float* lse1,
+                    void* stream);
+
+/*
+ * Backward of lte_attn_prefill with the straight-through surrogate (Section 3.1.2):
+ *   delta_i = <dO_i, o_i>,  P_ij = exp(scale q_i.k_j - lse_i) on j in A_i,
+ *   dV_j = sum_i P_ij dO_i,  dS_ij = P_ij (<dO_i, v_j> - delta_i),
+ *   dQ_i = scale sum_j dS_ij k_j,  dK_j = scale sum_i dS_ij q_i;
+ *   Eq. 6:  dr_j = <v_j, dV_j>  (+ lambda[h] if z_j > logit(tau), Eq. 7),  dz_j = dr_j r_j (1 - r_j),
+ *   for every scored token j <= T-1-half;  dw[h,t,c] = sum_{b,j} dz_j x[b,h,j+t-half,c],
+ *   dbias[h] = sum_{b,j} dz_j;  with flags bit 0 the scorer's input gradient
+ *   sum_t dz[j-t+half] w[h,t,c] is added into dk (c < d) and dv (c >= d).
+ * The retained lists are constants of the backward (the cap is not differentiated).
+ *   q,k,v,o,dO in  [B,H,T,d] of s->dtype;  lse, z in [B,H,T] fp32;  idx, cnt as for prefill
+ *   lambda_or_null in [H] fp32 device, or NULL
+ *   dq,dk,dv   out [B,H,T,d] of s->dtype;  dw out [H,K,2d] fp32;  dbias_or_null out [H] fp32
+ * Deterministic (no floating-point atomics).  Errors as for prefill, plus WORKSPACE.
+ */
+int lte_attn_bwd(const lte_shape* s, const lte_conv* c,
+                 const void* q, const void* k, const void* v, const void* o, const float* lse,
+                 const void* dO, const float* z, const int32_t* idx, const int32_t* cnt,
+                 const float* lambda_or_null,
+                 void* dq, void* dk, void* dv, float* dw, float* dbias_or_null, uint32_t flags,
+                 void* ws, size_t ws_bytes, void* stream);
+
+#define LTE_BWD_CNN_INPUT_GRAD 1u
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LTE_H_ */

@@ -1,0 +1,318 @@
+// Backward of the LTE prefill attention with the straight-through surrogate (Section 3.1.2, Eq. 6, Eq. 7).
+//
+// Gather form, no floating-point atomics, so the result is deterministic:
+//   dq kernel   one warp per query i: delta_i = <dO_i, o_i>, then over A_i (visible retained prefix + window)
+//               P_ij = exp(scale q_i.k_j - lse_i), dS_ij = P_ij (<dO_i, v_j> - delta_i), dq_i = scale sum_j dS_ij k_j.
+//   dkv kernel  one warp per key j: over the queries that see j (the W window queries j..j+W-1 and, if j is in the
+//               retained list, every query >= j+W): dv_j = sum_i P_ij dO_i, dk_j = scale sum_i dS_ij q_i; then
+//               Eq. 6: dr_j = <v_j, dv_j> (+ lambda_h 1[z_j > zthr]), dz_j = dr_j r_j (1 - r_j) for scored tokens.
+//   conv kernels  dw, dbias as per-(b, chunk) partial sums reduced in a fixed order; with the input-gradient flag
+//               the scorer's share sum_t dz[p-t+half] w[h,t,c] is added to the fp32 dk, dv before the one rounding.
+// Workspace: delta, dz [B,H,T] fp32; dw/dbias partials; fp32 dk, dv [B,H,T,d] when the flag is set.
+#include "common.cuh"
+
+namespace lte {
+namespace {
+
+constexpr int CHUNK = 256;     // positions per conv-gradient partial
+
+template <typename T, int D>
+__global__ void __launch_bounds__(128) bwd_dq_kernel(const T* __restrict__ q, const T* __restrict__ k,
+                                                     const T* __restrict__ v, const T* __restrict__ o,
+                                                     const T* __restrict__ dO, const float* __restrict__ lse,
+                                                     const int32_t* __restrict__ idx, const int32_t* __restrict__ cnt,
+                                                     T* __restrict__ dq, float* __restrict__ delta, int Tlen, int W,
+                                                     int R, float scale)
+{
+    constexpr int C = D / 32;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int i = blockIdx.x * 4 + warp;
+    const int bh = blockIdx.y;
+    if (i >= Tlen) return;
+    const size_t base = (size_t)bh * Tlen * D;
+    float qv[C], gv[C], acc[C];
+    float dl = 0.f;
+#pragma unroll
+    for (int c = 0; c < C; ++c) {
+        const size_t e = base + (size_t)i * D + lane + 32 * c;
+        qv[c] = to_f(q[e]) * scale; gv[c] = to_f(dO[e]); acc[c] = 0.f;
+        dl = fmaf(gv[c], to_f(o[e]), dl);
+    }
+    dl = warp_sum(dl);
+    if (lane == 0) delta[(size_t)bh * Tlen + i] = dl;
+    const float li = lse[(size_t)bh * Tlen + i];
+    const int32_t* id = idx + (size_t)bh * R;
+    const int n_ret = cnt[bh];
+    const int lo = i - W + 1 > 0 ? i - W + 1 : 0;
+    int nvis = 0;
+    for (int m0 = 0; m0 < n_ret; m0 += 32) {
+        int e = m0 + lane < n_ret ? id[m0 + lane] : 0x7fffffff;
+        unsigned b = __ballot_sync(0xffffffffu, e <= i - W);
+        nvis += __popc(b);
+        if (b != 0xffffffffu) break;
+    }
+    const int total = nvis + (i - lo + 1);
+    for (int a = 0; a < total; ++a) {
+        const int j = a < nvis ? id[a] : lo + (a - nvis);
+        const T* kr = k + base + (size_t)j * D;
+        const T* vr = v + base + (size_t)j * D;
+        float s = 0.f, dp = 0.f, kk[C];
+#pragma unroll
+        for (int c = 0; c < C; ++c) {
+            kk[c] = to_f(kr[lane + 32 * c]);
+            s = fmaf(qv[c], kk[c], s);
+            dp = fmaf(gv[c], to_f(vr[lane + 32 * c]), dp);
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            s += __shfl_xor_sync(0xffffffffu, s, off);
+            dp += __shfl_xor_sync(0xffffffffu, dp, off);
+        }
+        const float ds = expf(s - li) * (dp - dl);
+#pragma unroll
+        for (int c = 0; c < C; ++c) acc[c] = fmaf(ds, kk[c], acc[c]);
+    }
+#pragma unroll
+    for (int c = 0; c < C; ++c) dq[base + (size_t)i * D + lane + 32 * c] = from_f<T>(acc[c] * scale);
+}
+
+template <typename T, int D, bool F32OUT>
+__global__ void __launch_bounds__(128) bwd_dkv_kernel(const T* __restrict__ q, const T* __restrict__ k,
+                                                      const T* __restrict__ v, const T* __restrict__ dO,
+                                                      const float* __restrict__ lse, const float* __restrict__ delta,
+                                                      const float* __restrict__ z, const int32_t* __restrict__ idx,
+                                                      const int32_t* __restrict__ cnt, const float* __restrict__ lambda,
+                                                      T* __restrict__ dk, T* __restrict__ dv, float* __restrict__ dk32,
+                                                      float* __restrict__ dv32, float* __restrict__ dz, int H, int Tlen,
+                                                      int W, int R, int half, float zthr, float scale)
+{
+    constexpr int C = D / 32;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int j = blockIdx.x * 4 + warp;
+    const int bh = blockIdx.y;
+    if (j >= Tlen) return;
+    const size_t base = (size_t)bh * Tlen * D;
+    float kv[C], vv[C], ak[C], av[C];
+#pragma unroll
+    for (int c = 0; c < C; ++c) {
+        const size_t e = base + (size_t)j * D + lane + 32 * c;
+        kv[c] = to_f(k[e]) * scale; vv[c] = to_f(v[e]); ak[c] = 0.f; av[c] = 0.f;
+    }
+    // is j in the retained list? (idx ascending: binary search, uniform across the warp)
+    bool kept = false;
+    {
+        const int32_t* id = idx + (size_t)bh * R;
+        int lo = 0, hi = cnt[bh];
+        while (lo < hi) { int mid = (lo + hi) >> 1; if (id[mid] < j) lo = mid + 1; else hi = mid; }
+        kept = lo < cnt[bh] && id[lo] == j;
+    }
+    const int iend = kept ? Tlen - 1 : (j + W - 1 < Tlen - 1 ? j + W - 1 : Tlen - 1);
+    for (int i = j; i <= iend; ++i) {
+        const T* qr = q + base + (size_t)i * D;
+        const T* gr = dO + base + (size_t)i * D;
+        float s = 0.f, dp = 0.f, qq[C], gg[C];
+#pragma unroll
+        for (int c = 0; c < C; ++c) {
+            qq[c] = to_f(qr[lane + 32 * c]); gg[c] = to_f(gr[lane + 32 * c]);
+            s = fmaf(qq[c], kv[c], s);
+            dp = fmaf(gg[c], vv[c], dp);
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            s += __shfl_xor_sync(0xffffffffu, s, off);
+            dp += __shfl_xor_sync(0xffffffffu, dp, off);
+        }
+        const float p = expf(s - lse[(size_t)bh * Tlen + i]);
+        const float ds = p * (dp - delta[(size_t)bh * Tlen + i]);
+#pragma unroll
+        for (int c = 0; c < C; ++c) { av[c] = fmaf(p, gg[c], av[c]); ak[c] = fmaf(ds, qq[c], ak[c]); }
+    }
+    // Eq. 6 on the attention-only dV; scored tokens only
+    float dr = 0.f;
+#pragma unroll
+    for (int c = 0; c < C; ++c) dr = fmaf(vv[c], av[c], dr);
+    dr = warp_sum(dr);
+    if (lane == 0) {
+        float g = 0.f;
+        if (j + half <= Tlen - 1) {
+            const float zz = z[(size_t)bh * Tlen + j];
+            const float r = 1.f / (1.f + expf(-zz));
+            if (lambda && zz > zthr) dr += lambda[bh % H];
+            g = dr * r * (1.f - r);
+        }
+        dz[(size_t)bh * Tlen + j] = g;
+    }
+#pragma unroll
+    for (int c = 0; c < C; ++c) {
+        const size_t e = base + (size_t)j * D + lane + 32 * c;
+        if (F32OUT) { dk32[e] = ak[c] * scale; dv32[e] = av[c]; }
+        else { dk[e] = from_f<T>(ak[c] * scale); dv[e] = from_f<T>(av[c]); }
+    }
+}
+
+// Partial dw / dbias over one (b, chunk of CHUNK positions) for head h: thread c owns channel c of x = [k ; v].
+template <typename T>
+__global__ void bwd_conv_partial_kernel(const T* __restrict__ k, const T* __restrict__ v, const float* __restrict__ dz,
+                                        float* __restrict__ part_w, float* __restrict__ part_b, int B, int H, int Tlen,
+                                        int D, int K, int nchunk)
+{
+    extern __shared__ float s_dz[];                 // CHUNK + K - 1 values: dz[j0-half .. j0+CHUNK-1+half]
+    const int half = K / 2;
+    const int h = blockIdx.y;
+    const int b = blockIdx.x / nchunk, ch = blockIdx.x % nchunk;
+    const int bh = b * H + h;
+    const int p0 = ch * CHUNK;                      // rows p0 .. p0+CHUNK-1 of x
+    // row p contributes to tap t through dz[p - t + half]
+    for (int a = threadIdx.x; a < CHUNK + K - 1; a += blockDim.x) {
+        const int j = p0 - half + a;
+        s_dz[a] = (j >= 0 && j + half <= Tlen - 1) ? dz[(size_t)bh * Tlen + j] : 0.f;
+    }
+    __syncthreads();
+    const int c = threadIdx.x;                      // 0 .. 2D-1
+    float acc[kMaxTaps];
+#pragma unroll
+    for (int t = 0; t < kMaxTaps; ++t) acc[t] = 0.f;
+    const T* src = c < D ? k : v;
+    const int cc = c < D ? c : c - D;
+    const int pend = p0 + CHUNK < Tlen ? p0 + CHUNK : Tlen;
+    for (int p = p0; p < pend; ++p) {
+        const float x = to_f(src[((size_t)bh * Tlen + p) * D + cc]);
+#pragma unroll
+        for (int t = 0; t < kMaxTaps; ++t)
+            if (t < K) acc[t] = fmaf(s_dz[(p - p0) - t + 2 * half], x, acc[t]);   // dz index j = p - t + half
+    }
+    float* out = part_w + ((size_t)h * B * nchunk + blockIdx.x) * K * 2 * D;
+#pragma unroll
+    for (int t = 0; t < kMaxTaps; ++t)
+        if (t < K) out[(size_t)t * 2 * D + c] = acc[t];
+    if (threadIdx.x == 0) {
+        // bias partial: the dz of the positions j in [p0, p0+CHUNK) themselves
+        float sb = 0.f;
+        for (int a = 0; a < CHUNK; ++a) sb += s_dz[a + half];
+        part_b[(size_t)h * B * nchunk + blockIdx.x] = sb;
+    }
+}
+
+__global__ void bwd_conv_reduce_kernel(const float* __restrict__ part_w, const float* __restrict__ part_b,
+                                       float* __restrict__ dw, float* __restrict__ dbias, int nparts, int per_head)
+{
+    const int h = blockIdx.y;
+    const int e = blockIdx.x * blockDim.x + threadIdx.x;
+    if (e < per_head) {
+        float s = 0.f;
+        for (int p = 0; p < nparts; ++p) s += part_w[((size_t)h * nparts + p) * per_head + e];
+        dw[(size_t)h * per_head + e] = s;
+    }
+    if (dbias && blockIdx.x == 0 && threadIdx.x == 0) {
+        float s = 0.f;
+        for (int p = 0; p < nparts; ++p) s += part_b[(size_t)h * nparts + p];
+        dbias[h] = s;
+    }
+}
+
+// dk, dv <- fp32 attention gradients + the scorer's input gradient, rounded once.
+template <typename T>
+__global__ void bwd_finish_kernel(const float* __restrict__ dk32, const float* __restrict__ dv32,
+                                  const float* __restrict__ dz, const float* __restrict__ w, T* __restrict__ dk,
+                                  T* __restrict__ dv, int H, int Tlen, int D, int K)
+{
+    const int half = K / 2;
+    const size_t n = (size_t)gridDim.y * Tlen * D;
+    const int bh = blockIdx.y;
+    (void)n;
+    for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < Tlen * D; e += gridDim.x * blockDim.x) {
+        const int p = e / D, c = e % D;
+        const int h = bh % H;
+        float gk = 0.f, gv = 0.f;
+        for (int t = 0; t < K; ++t) {
+            const int j = p - t + half;
+            if (j < 0 || j + half > Tlen - 1) continue;
+            const float g = dz[(size_t)bh * Tlen + j];
+            gk = fmaf(g, w[((size_t)h * K + t) * 2 * D + c], gk);
+            gv = fmaf(g, w[((size_t)h * K + t) * 2 * D + D + c], gv);
+        }
+        const size_t a = (size_t)bh * Tlen * D + e;
+        dk[a] = from_f<T>(dk32[a] + gk);
+        dv[a] = from_f<T>(dv32[a] + gv);
+    }
+}
+
+struct WsPlan { size_t delta, dz, part_w, part_b, dk32, dv32, total; int nchunk; };
+WsPlan plan(const Params& p, uint32_t flags)
+{
+    WsPlan w;
+    auto up = [](size_t x) { return (x + 255) / 256 * 256; };
+    const size_t bht = (size_t)p.B * p.H * p.T;
+    w.nchunk = (p.T + CHUNK - 1) / CHUNK;
+    size_t off = 0;
+    w.delta = off; off += up(bht * 4);
+    w.dz = off; off += up(bht * 4);
+    w.part_w = off; off += up((size_t)p.H * p.B * w.nchunk * p.K * 2 * p.d * 4);
+    w.part_b = off; off += up((size_t)p.H * p.B * w.nchunk * 4);
+    w.dk32 = w.dv32 = 0;
+    if (flags & LTE_BWD_CNN_INPUT_GRAD) {
+        w.dk32 = off; off += up(bht * p.d * 4);
+        w.dv32 = off; off += up(bht * p.d * 4);
+    }
+    w.total = off;
+    return w;
+}
+
+template <typename T, int D>
+int run(const Params& p, const void* q, const void* k, const void* v, const void* o, const float* lse, const void* dO,
+        const float* z, const int32_t* idx, const int32_t* cnt, const float* lambda, void* dq, void* dk, void* dv,
+        float* dw, float* dbias, uint32_t flags, void* ws, cudaStream_t st)
+{
+    const WsPlan w = plan(p, flags);
+    char* base = (char*)ws;
+    float* delta = (float*)(base + w.delta);
+    float* dz = (float*)(base + w.dz);
+    float* part_w = (float*)(base + w.part_w);
+    float* part_b = (float*)(base + w.part_b);
+    float* dk32 = (float*)(base + w.dk32);
+    float* dv32 = (float*)(base + w.dv32);
+    const bool f32 = flags & LTE_BWD_CNN_INPUT_GRAD;
+    dim3 grid((p.T + 3) / 4, p.B * p.H);
+    bwd_dq_kernel<T, D><<<grid, 128, 0, st>>>((const T*)q, (const T*)k, (const T*)v, (const T*)o, (const T*)dO, lse, idx,
+                                              cnt, (T*)dq, delta, p.T, p.W, p.R, p.scale);
+    if (f32)
+        bwd_dkv_kernel<T, D, true><<<grid, 128, 0, st>>>((const T*)q, (const T*)k, (const T*)v, (const T*)dO, lse, delta,
+                                                         z, idx, cnt, lambda, (T*)dk, (T*)dv, dk32, dv32, dz, p.H, p.T,
+                                                         p.W, p.R, p.half, p.zthr, p.scale);
+    else
+        bwd_dkv_kernel<T, D, false><<<grid, 128, 0, st>>>((const T*)q, (const T*)k, (const T*)v, (const T*)dO, lse, delta,
+                                                          z, idx, cnt, lambda, (T*)dk, (T*)dv, dk32, dv32, dz, p.H, p.T,
+                                                          p.W, p.R, p.half, p.zthr, p.scale);
+    dim3 gc(p.B * w.nchunk, p.H);
+    bwd_conv_partial_kernel<T><<<gc, 2 * D, (CHUNK + p.K - 1) * sizeof(float), st>>>(
+        (const T*)k, (const T*)v, dz, part_w, part_b, p.B, p.H, p.T, D, p.K, w.nchunk);
+    const int per_head = p.K * 2 * D;
+    dim3 gr((per_head + 255) / 256, p.H);
+    bwd_conv_reduce_kernel<<<gr, 256, 0, st>>>(part_w, part_b, dw, dbias, p.B * w.nchunk, per_head);
+    if (f32) {
+        dim3 gf(min((p.T * D + 255) / 256, 1024), p.B * p.H);
+        bwd_finish_kernel<T><<<gf, 256, 0, st>>>(dk32, dv32, dz, p.w, (T*)dk, (T*)dv, p.H, p.T, D, p.K);
+    }
+    return cuda_status(cudaGetLastError());
+}
+
+}  // namespace
+
+size_t bwd_workspace_bytes(const Params& p, uint32_t flags) { return plan(p, flags).total; }
+
+int launch_bwd(const Params& p, const void* q, const void* k, const void* v, const void* o, const float* lse,
+               const void* dO, const float* z, const int32_t* idx, const int32_t* cnt, const float* lambda, void* dq,
+               void* dk, void* dv, float* dw, float* dbias, uint32_t flags, void* ws, cudaStream_t st)
+{
+#define LTE_GO(T, D) \
+    return run<T, D>(p, q, k, v, o, lse, dO, z, idx, cnt, lambda, dq, dk, dv, dw, dbias, flags, ws, st)
+    if (p.dtype == LTE_BF16) {
+        switch (p.d) { case 32: LTE_GO(__nv_bfloat16, 32); case 64: LTE_GO(__nv_bfloat16, 64); case 128: LTE_GO(__nv_bfloat16, 128); }
+    } else {
+        switch (p.d) { case 32: LTE_GO(float, 32); case 64: LTE_GO(float, 64); case 128: LTE_GO(float, 128); }
+    }
+#undef LTE_GO
+    return LTE_ERR_UNSUPPORTED;
+}
+
+}  // namespace lte

@@ -1,0 +1,90 @@
+// Shared device/host helpers of liblte (CUDA side only; the CPU oracle shares nothing with this).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+
+#include "lte.h"
+
+namespace lte {
+
+constexpr int kMaxTaps = 13;          // scorer taps the kernels are instantiated for (odd, <= 13)
+
+struct Params {                       // validated, host-resolved view of lte_shape / lte_conv
+    int B, H, T, d, W, R, sink, K, half;
+    float zthr;                       // logit(tau): keep iff z > zthr
+    float scale;                      // softmax scale
+    int dtype;
+    const float* w;
+    const float* bias;
+};
+
+template <typename T> __device__ __forceinline__ float to_f(T x);
+template <> __device__ __forceinline__ float to_f<float>(float x) { return x; }
+template <> __device__ __forceinline__ float to_f<__nv_bfloat16>(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+template <typename T> __device__ __forceinline__ T from_f(float x);
+template <> __device__ __forceinline__ float from_f<float>(float x) { return x; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }
+
+__device__ __forceinline__ float warp_sum(float x) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    return x;
+}
+__device__ __forceinline__ float warp_max(float x) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, o));
+    return x;
+}
+
+// Monotone image of an fp32 logit: larger z <=> larger key.  0 is reserved for "not a candidate".
+__device__ __forceinline__ uint32_t order_key(float z) {
+    uint32_t u = __float_as_uint(z);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// ---- decode cache layout (per (b,h) block; see lte_cache_bytes) -----------------------------
+struct CacheLayout {
+    size_t esz;            // element size of k/v
+    size_t off_k, off_v;   // [(W+R), d] each: rows [0,W) ring (slot = pos mod W), rows [W,W+R) pool
+    size_t off_z;          // [(W+R)] fp32 logits, same row order
+    size_t off_pidx;       // [R] int32 positions of pool entries
+    size_t off_meta;       // int32[4]: n (tokens seen), cnt (pool entries), reserved x2
+    size_t stride;         // bytes per (b,h), multiple of 256
+    size_t header;         // bytes before the first (b,h) block (status word lives at byte 0)
+};
+__host__ __device__ inline CacheLayout cache_layout(int d, int W, int R, int dtype) {
+    CacheLayout L;
+    L.esz = dtype == LTE_BF16 ? 2 : 4;
+    size_t rows = (size_t)W + R;
+    L.off_k = 0;
+    L.off_v = L.off_k + rows * d * L.esz;
+    L.off_z = L.off_v + rows * d * L.esz;
+    L.off_pidx = L.off_z + rows * 4;
+    L.off_meta = L.off_pidx + (size_t)R * 4;
+    size_t end = L.off_meta + 16;
+    L.stride = (end + 255) / 256 * 256;
+    L.header = 256;
+    return L;
+}
+
+// kernel launchers (one translation unit each)
+int launch_scores(const Params& p, const void* k, const void* v, float* z, float* r, cudaStream_t st);
+int launch_select(const Params& p, const float* z, int32_t* idx, int32_t* cnt, int32_t* ncand, cudaStream_t st);
+int launch_prefill_simt(const Params& p, const void* q, const void* k, const void* v, const int32_t* idx,
+                        const int32_t* cnt, void* o, float* lse, cudaStream_t st);
+int launch_cache_init(const Params& p, const void* k, const void* v, const float* z, const int32_t* idx,
+                      const int32_t* cnt, void* cache, cudaStream_t st);
+int launch_decode(const Params& p, void* cache, const void* q1, const void* k1, const void* v1, void* o1,
+                  float* lse1, cudaStream_t st);
+size_t bwd_workspace_bytes(const Params& p, uint32_t flags);
+int launch_bwd(const Params& p, const void* q, const void* k, const void* v, const void* o, const float* lse,
+               const void* dO, const float* z, const int32_t* idx, const int32_t* cnt, const float* lambda,
+               void* dq, void* dk, void* dv, float* dw, float* dbias, uint32_t flags, void* ws,
+               cudaStream_t st);
+
+inline int cuda_status(cudaError_t e) { return e == cudaSuccess ? LTE_OK : LTE_ERR_CUDA; }
+
+}  // namespace lte

@@ -1,0 +1,170 @@
+// C-ABI entry points of liblte: argument validation and dispatch.  No torch types, no allocation.
+#include <math.h>
+
+#include "common.cuh"
+
+namespace lte {
+
+int launch_prefill_tc(const Params& p, const void* q, const void* k, const void* v, const int32_t* idx,
+                      const int32_t* cnt, void* o, float* lse, cudaStream_t st);
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_shape(const lte_shape* s, bool need_T)
+{
+    if (!s) return LTE_ERR_INVALID_ARG;
+    if (s->B <= 0 || s->H <= 0 || s->W <= 0 || s->R < 0 || s->sink < 0) return LTE_ERR_INVALID_ARG;
+    if (need_T ? s->T <= 0 : s->T < 0) return LTE_ERR_INVALID_ARG;
+    if (s->dtype != LTE_F32 && s->dtype != LTE_BF16) return LTE_ERR_INVALID_ARG;
+    if (s->d != 32 && s->d != 64 && s->d != 128) return LTE_ERR_UNSUPPORTED;
+    if (!(s->tau < 1.0f)) return LTE_ERR_INVALID_ARG;
+    if ((double)s->B * s->H * (double)(s->T > 0 ? s->T : 1) * s->d > 2.0e10) return LTE_ERR_UNSUPPORTED;
+    return LTE_OK;
+}
+
+int check_conv(const lte_shape* s, const lte_conv* c)
+{
+    if (!c || !c->w) return LTE_ERR_INVALID_ARG;
+    if (c->n_layers != 1 || c->dilation != 1) return LTE_ERR_UNSUPPORTED;
+    if (c->kernel < 1 || c->kernel > kMaxTaps || (c->kernel & 1) == 0) return LTE_ERR_INVALID_ARG;
+    if (s->W < c->kernel) return LTE_ERR_INVALID_ARG;     // the receptive field must fit in the window
+    return LTE_OK;
+}
+
+Params make_params(const lte_shape* s, const lte_conv* c)
+{
+    Params p;
+    p.B = s->B; p.H = s->H; p.T = s->T; p.d = s->d; p.W = s->W; p.R = s->R; p.sink = s->sink;
+    p.K = c ? c->kernel : 1; p.half = p.K / 2;
+    p.zthr = s->tau <= 0.f ? -INFINITY : (float)(log((double)s->tau) - log1p(-(double)s->tau));
+    p.scale = s->softmax_scale > 0.f ? s->softmax_scale : (float)(1.0 / sqrt((double)s->d));
+    p.dtype = s->dtype;
+    p.w = c ? c->w : nullptr;
+    p.bias = c ? c->bias : nullptr;
+    return p;
+}
+
+int check_arch()
+{
+    int dev = 0, major = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return LTE_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return LTE_ERR_CUDA;
+    return major == 10 ? LTE_OK : LTE_ERR_ARCH;
+}
+
+}  // namespace
+}  // namespace lte
+
+using namespace lte;
+
+extern "C" {
+
+const char* lte_strerror(int status)
+{
+    switch (status) {
+        case LTE_OK: return "ok";
+        case LTE_ERR_INVALID_ARG: return "invalid argument";
+        case LTE_ERR_UNSUPPORTED: return "unsupported shape or dtype";
+        case LTE_ERR_WORKSPACE: return "workspace too small";
+        case LTE_ERR_CUDA: return "CUDA call failed";
+        case LTE_ERR_ARCH: return "device is not compute capability 10.x";
+        case LTE_ERR_DEVICE_STATUS: return "a kernel recorded an anomaly";
+    }
+    return "unknown status";
+}
+
+size_t lte_workspace_bytes(int op, const lte_shape* s, const lte_conv* c)
+{
+    if (!s) return 0;
+    if (op == LTE_OP_BWD) {
+        if (check_shape(s, true) != LTE_OK || !c) return 0;
+        Params p = make_params(s, c);
+        return bwd_workspace_bytes(p, LTE_BWD_CNN_INPUT_GRAD);
+    }
+    return 0;
+}
+
+int lte_scores(const lte_shape* s, const lte_conv* c, const void* k, const void* v, float* z, float* r_or_null,
+               void* ws, size_t ws_bytes, void* stream)
+{
+    (void)ws; (void)ws_bytes;
+    int e = check_shape(s, true); if (e) return e;
+    e = check_conv(s, c); if (e) return e;
+    if (!k || !v || !z || !aligned16(k) || !aligned16(v)) return LTE_ERR_INVALID_ARG;
+    e = check_arch(); if (e) return e;
+    return launch_scores(make_params(s, c), k, v, z, r_or_null, (cudaStream_t)stream);
+}
+
+int lte_select(const lte_shape* s, const float* z, int32_t* idx, int32_t* cnt, int32_t* ncand_or_null, void* ws,
+               size_t ws_bytes, void* stream)
+{
+    (void)ws; (void)ws_bytes;
+    int e = check_shape(s, true); if (e) return e;
+    if (!z || !cnt || (s->R > 0 && !idx)) return LTE_ERR_INVALID_ARG;
+    if (s->T - s->W > (1 << 24)) return LTE_ERR_UNSUPPORTED;
+    e = check_arch(); if (e) return e;
+    return launch_select(make_params(s, nullptr), z, idx, cnt, ncand_or_null, (cudaStream_t)stream);
+}
+
+int lte_attn_prefill(const lte_shape* s, const void* q, const void* k, const void* v, const int32_t* idx,
+                     const int32_t* cnt, void* o, float* lse, void* ws, size_t ws_bytes, void* stream)
+{
+    (void)ws; (void)ws_bytes;
+    int e = check_shape(s, true); if (e) return e;
+    if (!q || !k || !v || !o || !lse || !cnt || (s->R > 0 && !idx)) return LTE_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return LTE_ERR_INVALID_ARG;
+    e = check_arch(); if (e) return e;
+    Params p = make_params(s, nullptr);
+    if (s->dtype == LTE_BF16) return launch_prefill_tc(p, q, k, v, idx, cnt, o, lse, (cudaStream_t)stream);
+    return launch_prefill_simt(p, q, k, v, idx, cnt, o, lse, (cudaStream_t)stream);
+}
+
+size_t lte_cache_bytes(const lte_shape* s)
+{
+    if (!s || s->B <= 0 || s->H <= 0 || s->W <= 0 || s->R < 0 || s->d <= 0) return 0;
+    const CacheLayout L = cache_layout(s->d, s->W, s->R, s->dtype);
+    return L.header + (size_t)s->B * s->H * L.stride;
+}
+
+int lte_cache_init(const lte_shape* s, const lte_conv* c, const void* k, const void* v, const float* z,
+                   const int32_t* idx, const int32_t* cnt, void* cache, void* stream)
+{
+    int e = check_shape(s, false); if (e) return e;
+    e = check_conv(s, c); if (e) return e;
+    if (!cache || !aligned16(cache)) return LTE_ERR_INVALID_ARG;
+    if (s->T > 0 && (!k || !v || !z || !cnt || (s->R > 0 && !idx))) return LTE_ERR_INVALID_ARG;
+    e = check_arch(); if (e) return e;
+    return launch_cache_init(make_params(s, c), k, v, z, idx, cnt, cache, (cudaStream_t)stream);
+}
+
+int lte_attn_decode(const lte_shape* s, const lte_conv* c, void* cache, const void* q1, const void* k1,
+                    const void* v1, void* o1, float* lse1, void* stream)
+{
+    int e = check_shape(s, false); if (e) return e;
+    e = check_conv(s, c); if (e) return e;
+    if (!cache || !q1 || !k1 || !v1 || !o1 || !lse1) return LTE_ERR_INVALID_ARG;
+    if (!aligned16(cache) || !aligned16(q1) || !aligned16(k1) || !aligned16(v1)) return LTE_ERR_INVALID_ARG;
+    e = check_arch(); if (e) return e;
+    return launch_decode(make_params(s, c), cache, q1, k1, v1, o1, lse1, (cudaStream_t)stream);
+}
+
+int lte_attn_bwd(const lte_shape* s, const lte_conv* c, const void* q, const void* k, const void* v, const void* o,
+                 const float* lse, const void* dO, const float* z, const int32_t* idx, const int32_t* cnt,
+                 const float* lambda_or_null, void* dq, void* dk, void* dv, float* dw, float* dbias_or_null,
+                 uint32_t flags, void* ws, size_t ws_bytes, void* stream)
+{
+    int e = check_shape(s, true); if (e) return e;
+    e = check_conv(s, c); if (e) return e;
+    if (!q || !k || !v || !o || !lse || !dO || !z || !cnt || (s->R > 0 && !idx) || !dq || !dk || !dv || !dw)
+        return LTE_ERR_INVALID_ARG;
+    if (flags & ~LTE_BWD_CNN_INPUT_GRAD) return LTE_ERR_INVALID_ARG;
+    Params p = make_params(s, c);
+    if (!ws || !aligned16(ws) || ws_bytes < bwd_workspace_bytes(p, flags)) return LTE_ERR_WORKSPACE;
+    e = check_arch(); if (e) return e;
+    return launch_bwd(p, q, k, v, o, lse, dO, z, idx, cnt, lambda_or_null, dq, dk, dv, dw, dbias_or_null, flags, ws,
+                      (cudaStream_t)stream);
+}
+
+}  // extern "C"

@@ -1,0 +1,183 @@
+"""Thin Python binding over the C-ABI library ``liblte.so`` (argument marshalling only).
+
+Every function takes CUDA ``torch`` tensors (device memory and the current stream are all PyTorch
+is used for), checks dtype / contiguity, and passes raw pointers to the entry point of the same name
+declared in ``include/lte.h``.  There is no fallback: if the library is missing or a call fails, an
+exception is raised.
+"""
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "liblte.so")
+_lib = None
+
+F32, BF16 = 0, 1
+OP_SCORES, OP_SELECT, OP_PREFILL, OP_DECODE, OP_BWD = range(5)
+BWD_CNN_INPUT_GRAD = 1
+
+EXPORTS = ["lte_workspace_bytes", "lte_strerror", "lte_scores", "lte_select", "lte_attn_prefill",
+           "lte_cache_bytes", "lte_cache_init", "lte_attn_decode", "lte_attn_bwd"]
+
+
+class LteShape(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int32), ("H", ctypes.c_int32), ("T", ctypes.c_int32), ("d", ctypes.c_int32),
+                ("W", ctypes.c_int32), ("R", ctypes.c_int32), ("sink", ctypes.c_int32),
+                ("tau", ctypes.c_float), ("softmax_scale", ctypes.c_float), ("dtype", ctypes.c_int32)]
+
+
+class LteConv(ctypes.Structure):
+    _fields_ = [("n_layers", ctypes.c_int32), ("kernel", ctypes.c_int32), ("dilation", ctypes.c_int32),
+                ("w", ctypes.c_void_p), ("bias", ctypes.c_void_p)]
+
+
+class LteError(RuntimeError):
+    def __init__(self, fn, status):
+        self.status = status
+        super().__init__("%s failed: %d (%s)" % (fn, status, lib().lte_strerror(status).decode()))
+
+
+def lib():
+    """Load ``liblte.so`` (built by ``python -m paper_2510_20787_b200.build``); raises if it is absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError("liblte.so is not built: run `python -m paper_2510_20787_b200.build`")
+        L = ctypes.CDLL(LIB_PATH)
+        L.lte_strerror.restype = ctypes.c_char_p
+        L.lte_strerror.argtypes = [ctypes.c_int]
+        L.lte_workspace_bytes.restype = ctypes.c_size_t
+        L.lte_workspace_bytes.argtypes = [ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p]
+        L.lte_cache_bytes.restype = ctypes.c_size_t
+        L.lte_cache_bytes.argtypes = [ctypes.c_void_p]
+        vp = ctypes.c_void_p
+        L.lte_scores.argtypes = [vp] * 7 + [ctypes.c_size_t, vp]
+        L.lte_select.argtypes = [vp] * 6 + [ctypes.c_size_t, vp]
+        L.lte_attn_prefill.argtypes = [vp] * 9 + [ctypes.c_size_t, vp]
+        L.lte_cache_init.argtypes = [vp] * 9
+        L.lte_attn_decode.argtypes = [vp] * 9
+        L.lte_attn_bwd.argtypes = [vp] * 17 + [ctypes.c_uint32, vp, ctypes.c_size_t, vp]
+        for name in EXPORTS:
+            if name not in ("lte_strerror", "lte_workspace_bytes", "lte_cache_bytes"):
+                getattr(L, name).restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+def _dt(t):
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError("q/k/v must be float32 or bfloat16")
+
+
+def shape(B, H, T, d, W, R, dtype, sink=0, tau=0.5, softmax_scale=0.0):
+    return LteShape(B, H, T, d, W, R, sink, tau, softmax_scale, dtype)
+
+
+def conv(w, bias=None):
+    """w: CUDA fp32 [H, K, 2d]; bias: CUDA fp32 [H] or None."""
+    assert w.is_cuda and w.dtype == torch.float32 and w.is_contiguous()
+    assert bias is None or (bias.is_cuda and bias.dtype == torch.float32 and bias.is_contiguous())
+    return LteConv(1, w.shape[1], 1, w.data_ptr(), 0 if bias is None else bias.data_ptr())
+
+
+def _ptr(t, dtype=None):
+    if t is None:
+        return None
+    assert t.is_cuda and t.is_contiguous(), "tensors must be contiguous CUDA tensors"
+    if dtype is not None:
+        assert t.dtype == dtype, "expected %s, got %s" % (dtype, t.dtype)
+    return t.data_ptr()
+
+
+def _stream():
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _check(fn, status):
+    if status != 0:
+        raise LteError(fn, status)
+
+
+def lte_workspace_bytes(op, s, c=None):
+    return int(lib().lte_workspace_bytes(op, ctypes.addressof(s), None if c is None else ctypes.addressof(c)))
+
+
+def lte_scores(s, c, k, v, z=None, r=None):
+    """k, v [B,H,T,d] -> z [B,H,T] fp32 (and r = sigmoid(z) if a tensor is given)."""
+    if z is None:
+        z = torch.empty((s.B, s.H, s.T), dtype=torch.float32, device=k.device)
+    _check("lte_scores", lib().lte_scores(ctypes.addressof(s), ctypes.addressof(c), _ptr(k), _ptr(v),
+                                          _ptr(z, torch.float32), _ptr(r, torch.float32), None, 0, _stream()))
+    return z
+
+
+def lte_select(s, z, idx=None, cnt=None, ncand=None):
+    """z [B,H,T] fp32 -> idx [B,H,R] int32 ascending (-1 unused), cnt [B,H] int32."""
+    dev = z.device
+    if idx is None:
+        idx = torch.empty((s.B, s.H, s.R), dtype=torch.int32, device=dev)
+    if cnt is None:
+        cnt = torch.empty((s.B, s.H), dtype=torch.int32, device=dev)
+    _check("lte_select", lib().lte_select(ctypes.addressof(s), _ptr(z, torch.float32), _ptr(idx, torch.int32),
+                                          _ptr(cnt, torch.int32), _ptr(ncand, torch.int32), None, 0, _stream()))
+    return idx, cnt
+
+
+def lte_attn_prefill(s, q, k, v, idx, cnt, o=None, lse=None):
+    """q, k, v [B,H,T,d], retained list -> o [B,H,T,d], lse [B,H,T] fp32."""
+    if o is None:
+        o = torch.empty_like(q)
+    if lse is None:
+        lse = torch.empty((s.B, s.H, s.T), dtype=torch.float32, device=q.device)
+    _check("lte_attn_prefill", lib().lte_attn_prefill(ctypes.addressof(s), _ptr(q), _ptr(k), _ptr(v),
+                                                      _ptr(idx, torch.int32), _ptr(cnt, torch.int32), _ptr(o),
+                                                      _ptr(lse, torch.float32), None, 0, _stream()))
+    return o, lse
+
+
+def lte_cache_bytes(s):
+    return int(lib().lte_cache_bytes(ctypes.addressof(s)))
+
+
+def lte_cache_init(s, c, k=None, v=None, z=None, idx=None, cnt=None, cache=None):
+    """Decode cache holding the state after the T-token prompt (T = 0: empty cache)."""
+    if cache is None:
+        dev = k.device if k is not None else torch.device("cuda")
+        cache = torch.empty(lte_cache_bytes(s), dtype=torch.uint8, device=dev)
+    _check("lte_cache_init", lib().lte_cache_init(ctypes.addressof(s), ctypes.addressof(c), _ptr(k), _ptr(v),
+                                                  _ptr(z), _ptr(idx), _ptr(cnt), _ptr(cache), _stream()))
+    return cache
+
+
+def lte_attn_decode(s, c, cache, q1, k1, v1, o1=None, lse1=None):
+    """One decode step: q1, k1, v1 [B,H,d] -> o1 [B,H,d], lse1 [B,H]; the cache is updated in place."""
+    if o1 is None:
+        o1 = torch.empty_like(q1)
+    if lse1 is None:
+        lse1 = torch.empty((s.B, s.H), dtype=torch.float32, device=q1.device)
+    _check("lte_attn_decode", lib().lte_attn_decode(ctypes.addressof(s), ctypes.addressof(c), _ptr(cache),
+                                                    _ptr(q1), _ptr(k1), _ptr(v1), _ptr(o1),
+                                                    _ptr(lse1, torch.float32), _stream()))
+    return o1, lse1
+
+
+def lte_attn_bwd(s, c, q, k, v, o, lse, dO, z, idx, cnt, lam=None, flags=BWD_CNN_INPUT_GRAD, want_dbias=True,
+                 ws=None):
+    """Backward with the straight-through surrogate -> dq, dk, dv, dw [H,K,2d], dbias [H] (or None)."""
+    dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+    dw = torch.empty((s.H, c.kernel, 2 * s.d), dtype=torch.float32, device=q.device)
+    db = torch.empty((s.H,), dtype=torch.float32, device=q.device) if want_dbias else None
+    need = lte_workspace_bytes(OP_BWD, s, c)
+    if ws is None:
+        ws = torch.empty(max(need, 16), dtype=torch.uint8, device=q.device)
+    _check("lte_attn_bwd", lib().lte_attn_bwd(
+        ctypes.addressof(s), ctypes.addressof(c), _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse, torch.float32),
+        _ptr(dO), _ptr(z, torch.float32), _ptr(idx, torch.int32), _ptr(cnt, torch.int32),
+        _ptr(lam, torch.float32), _ptr(dq), _ptr(dk), _ptr(dv), _ptr(dw), _ptr(db), flags, _ptr(ws),
+        ws.numel(), _stream()))
+    return dq, dk, dv, dw, db

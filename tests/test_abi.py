@@ -1,0 +1,70 @@
+"""CPU-side checks of the C-ABI library: it loads, exports every declared symbol, and validates arguments
+on the host before touching a device."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2510_20787_b200 import lte
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared():
+    names = set()
+    for fn in os.listdir(os.path.join(ROOT, "include")):
+        if not fn.endswith(".h"):
+            continue
+        text = open(os.path.join(ROOT, "include", fn)).read()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        names |= set(re.findall(r"\b(lte_[a-z0-9_]+)\s*\(", text))
+    return names
+
+
+def test_library_exports_every_declared_symbol():
+    L = lte.lib()
+    declared = _declared()
+    assert {"lte_scores", "lte_select", "lte_attn_prefill", "lte_attn_decode", "lte_attn_bwd"} <= declared
+    for name in declared:
+        assert hasattr(L, name), name
+    assert set(lte.EXPORTS) <= declared
+
+
+def test_strerror_and_sizes():
+    L = lte.lib()
+    assert L.lte_strerror(0) == b"ok"
+    assert b"workspace" in L.lte_strerror(-3)
+    s = lte.shape(128, 16, 8192, 64, 128, 128, lte.BF16)
+    per = 2 * 256 * 64 * 2 + 256 * 4 + 128 * 4 + 16
+    per = (per + 255) // 256 * 256
+    assert lte.lte_cache_bytes(s) == 256 + 128 * 16 * per
+    c = lte.LteConv(1, 7, 1, 16, 0)
+    assert lte.lte_workspace_bytes(lte.OP_BWD, s, c) > 2 * 128 * 16 * 8192 * 4
+    assert lte.lte_workspace_bytes(lte.OP_SCORES, s, c) == 0
+
+
+def test_host_side_validation_rejects_bad_arguments():
+    L = lte.lib()
+    a = ctypes.addressof
+    good = lte.shape(1, 2, 128, 32, 16, 8, lte.F32)
+    conv = lte.LteConv(1, 5, 1, 256, 0)
+    fake = 4096          # never dereferenced: validation fails first
+    assert L.lte_scores(None, a(conv), fake, fake, fake, None, None, 0, None) == -1
+    assert L.lte_scores(a(good), None, fake, fake, fake, None, None, 0, None) == -1
+    assert L.lte_scores(a(good), a(conv), None, fake, fake, None, None, 0, None) == -1
+    assert L.lte_scores(a(good), a(conv), fake + 4, fake, fake, None, None, 0, None) == -1      # misaligned
+    even = lte.LteConv(1, 4, 1, 256, 0)
+    assert L.lte_scores(a(good), a(even), fake, fake, fake, None, None, 0, None) == -1
+    deep = lte.LteConv(3, 3, 2, 256, 0)
+    assert L.lte_scores(a(good), a(deep), fake, fake, fake, None, None, 0, None) == -2
+    bad_d = lte.shape(1, 2, 128, 48, 16, 8, lte.F32)
+    assert L.lte_scores(a(bad_d), a(conv), fake, fake, fake, None, None, 0, None) == -2
+    narrow = lte.shape(1, 2, 128, 32, 3, 8, lte.F32)
+    assert L.lte_scores(a(narrow), a(conv), fake, fake, fake, None, None, 0, None) == -1        # W < K
+    assert L.lte_select(a(good), None, fake, fake, None, None, 0, None) == -1
+    assert L.lte_attn_prefill(a(good), fake, fake, fake, fake, fake, None, fake, None, 0, None) == -1
+    assert L.lte_attn_decode(a(good), a(conv), None, fake, fake, fake, fake, fake, None) == -1
+    args = [a(good), a(conv)] + [fake] * 9 + [None] + [fake] * 4 + [None, 0, fake, 16, None]
+    assert L.lte_attn_bwd(*args) == -3                                                         # workspace too small
+    assert lte.lte_cache_bytes(lte.shape(0, 2, 1, 32, 16, 8, lte.F32)) == 0

@@ -1,0 +1,68 @@
+"""GPU parity: lte_attn_bwd against the fp64 oracle gradients, through the C-ABI."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import lte_oracle as orc
+from paper_2510_20787_b200 import lte, synth
+from tests.gpu_util import check_idx, dev, rel_l2, shape_of
+
+pytestmark = pytest.mark.gpu
+
+REL = {"bf16": 5e-2, "f32": 1e-4}
+
+
+def _bwd(cfg, seed=0, batch=None, flags=lte.BWD_CNN_INPUT_GRAD, lam=None, bias=None, scale=0.0):
+    x = synth.make(cfg, seed, batch=batch, with_dO=True)
+    B = x["k"].shape[0]
+    s = shape_of(cfg, B=B, scale=scale)
+    bt = None if bias is None else torch.from_numpy(bias.astype(np.float32)).cuda()
+    c = lte.conv(torch.from_numpy(x["w"]).cuda(), bt)
+    q, k, v, dO = (dev(x[t], cfg.dtype) for t in ("q", "k", "v", "dO"))
+    z = lte.lte_scores(s, c, k, v)
+    idx, cnt = lte.lte_select(s, z)
+    o, lse = lte.lte_attn_prefill(s, q, k, v, idx, cnt)
+    lt = None if lam is None else torch.from_numpy(lam.astype(np.float32)).cuda()
+    dq, dk, dv, dw, db = lte.lte_attn_bwd(s, c, q, k, v, o, lse, dO, z, idx, cnt, lam=lt, flags=flags)
+    torch.cuda.synchronize()
+    idx_n, cnt_n = idx.cpu().numpy(), cnt.cpu().numpy()
+    z64 = orc.scores(x["k"], x["v"], x["w"], bias)
+    check_idx(idx_n, cnt_n, z64, cfg.W, cfg.R, cfg.sink)
+    g = orc.attn_bwd(x["q"], x["k"], x["v"], x["dO"], z64, idx_n, cnt_n, x["w"], cfg.W,
+                     None if scale == 0.0 else scale, lam=lam, cnn_input_grad=bool(flags & 1))
+    got = dict(dq=dq, dk=dk, dv=dv, dw=dw, dbias=db)
+    return {n: (t.float().cpu().numpy(), g[n]) for n, t in got.items()}
+
+
+def _assert(cfg, res):
+    for name, (a, b) in res.items():
+        assert np.all(np.isfinite(a)), name
+        assert rel_l2(a, b) <= REL[cfg.dtype], (name, rel_l2(a, b))
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("d,K,T,W,R,sink", [(32, 5, 128, 16, 8, 0), (64, 7, 300, 40, 25, 2), (128, 3, 130, 9, 200, 0),
+                                            (64, 7, 260, 300, 10, 0), (32, 1, 50, 4, 0, 0), (64, 13, 777, 64, 64, 0)])
+@pytest.mark.parametrize("flags", [0, 1])
+def test_small_shapes(dtype, d, K, T, W, R, sink, flags):
+    cfg = synth.Config("bwd", dtype, 2, 3, d, T, W, R, K, 0.1, sink=sink, qk_unit=(dtype == "f32"))
+    _assert(cfg, _bwd(cfg, seed=7, flags=flags, lam=np.array([0.5, 0.0, 0.1]), bias=np.array([0.1, -0.2, 0.0])))
+
+
+def test_config5_two_sequences():
+    cfg = synth.CONFIGS["C5"]
+    _assert(cfg, _bwd(cfg, seed=0, batch=[0, 6]))
+    _assert(cfg, _bwd(cfg, seed=0, batch=[3], flags=0))
+
+
+def test_config5_full_batch_weight_gradient():
+    cfg = synth.CONFIGS["C5"]
+    _assert(cfg, _bwd(cfg, seed=0))
+
+
+def test_deterministic():
+    cfg = synth.CONFIGS["C5"].with_(B=1)
+    a = _bwd(cfg, seed=1)
+    b = _bwd(cfg, seed=1)
+    for n in a:
+        assert np.array_equal(a[n][0], b[n][0])

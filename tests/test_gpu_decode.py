@@ -1,0 +1,124 @@
+"""GPU parity: lte_cache_init + lte_attn_decode against the oracle's streaming simulation."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import lte_oracle as orc
+from paper_2510_20787_b200 import lte, synth
+from tests.gpu_util import check_idx, dev, shape_of
+
+pytestmark = pytest.mark.gpu
+
+TOL = {"bf16": 2e-2, "f32": 1e-4}
+
+
+def _read_pool(cache, cfg, B):
+    """Pool positions and counts out of the raw cache buffer (layout documented in include/lte.h)."""
+    esz = 2 if cfg.dtype == "bf16" else 4
+    rows = cfg.W + cfg.R
+    off_z = 2 * rows * cfg.d * esz
+    off_pidx = off_z + rows * 4
+    off_meta = off_pidx + cfg.R * 4
+    stride = (off_meta + 16 + 255) // 256 * 256
+    raw = cache.cpu().numpy()
+    pools, ns = [], []
+    for bh in range(B * cfg.H):
+        blk = raw[256 + bh * stride: 256 + (bh + 1) * stride]
+        meta = blk[off_meta:off_meta + 16].view(np.int32)
+        pidx = blk[off_pidx:off_pidx + 4 * cfg.R].view(np.int32)
+        pools.append(np.sort(pidx[:meta[1]]))
+        ns.append(int(meta[0]))
+    return pools, ns
+
+
+def _decode_run(cfg, T0, steps, seed=0, batch=None, scale=0.0):
+    """Prefill T0 tokens on the GPU (scores -> select -> cache_init), then `steps` decode steps."""
+    Ttot = T0 + steps
+    x = synth.make(cfg, seed, batch=batch, T=Ttot)
+    B = x["k"].shape[0]
+    c = lte.conv(torch.from_numpy(x["w"]).cuda())
+    q, k, v = (dev(x[t], cfg.dtype) for t in "qkv")
+    s0 = shape_of(cfg, T=T0, B=B, scale=scale)
+    if T0 > 0:
+        kp, vp = k[:, :, :T0].contiguous(), v[:, :, :T0].contiguous()
+        z = lte.lte_scores(s0, c, kp, vp)
+        idx, cnt = lte.lte_select(s0, z)
+        cache = lte.lte_cache_init(s0, c, kp, vp, z, idx, cnt)
+    else:
+        cache = lte.lte_cache_init(s0, c)
+    outs, lses = [], []
+    for n in range(T0, Ttot):
+        o1, l1 = lte.lte_attn_decode(s0, c, cache, q[:, :, n].contiguous(), k[:, :, n].contiguous(),
+                                     v[:, :, n].contiguous())
+        outs.append(o1.float().cpu().numpy()); lses.append(l1.cpu().numpy())
+    torch.cuda.synchronize()
+    o_n = np.stack(outs, axis=2); l_n = np.stack(lses, axis=2)
+    z64 = orc.scores(x["k"], x["v"], x["w"])
+    o64, l64, pidx, pcnt = orc.stream(x["q"], x["k"], x["v"], z64, cfg.W, cfg.R, cfg.sink,
+                                      scale=None if scale == 0.0 else scale, n_from=T0)
+    pools, ns = _read_pool(cache, cfg, B)
+    return o_n, l_n, o64, l64, pools, ns, pidx, pcnt, z64
+
+
+def _assert(cfg, res, Ttot, strict_pool=True):
+    o_n, l_n, o64, l64, pools, ns, pidx, pcnt, z64 = res
+    assert all(n == Ttot for n in ns)
+    B = o_n.shape[0]
+    mism = 0
+    for bh, pool in enumerate(pools):
+        b, h = divmod(bh, cfg.H)
+        want = pidx[b, h, :pcnt[b, h]]
+        if not (len(pool) == len(want) and np.array_equal(pool, want)):
+            mism += 1
+    if strict_pool:
+        assert mism == 0
+        assert np.max(np.abs(o_n - o64)) <= TOL[cfg.dtype], np.max(np.abs(o_n - o64))
+        assert np.max(np.abs(l_n - l64)) <= TOL[cfg.dtype]
+    return mism
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("d,K,W,R,sink,T", [(32, 5, 16, 8, 0, 128), (64, 7, 24, 5, 2, 150), (128, 3, 8, 0, 0, 40),
+                                            (64, 1, 5, 3, 0, 60), (32, 7, 7, 40, 1, 90)])
+def test_decode_from_empty_cache(dtype, d, K, W, R, sink, T):
+    cfg = synth.Config("dec", dtype, 2, 2, d, T, W, R, K, 0.1, sink=sink, qk_unit=(dtype == "f32"))
+    _assert(cfg, _decode_run(cfg, 0, T, seed=1), T)
+
+
+@pytest.mark.parametrize("dtype,T0,steps", [("bf16", 300, 70), ("f32", 100, 50), ("bf16", 10, 100), ("bf16", 33, 5)])
+def test_decode_after_prefill(dtype, T0, steps):
+    cfg = synth.Config("dec", dtype, 2, 3, 64, T0, 32, 20, 7, 0.1)
+    _assert(cfg, _decode_run(cfg, T0, steps, seed=2), T0 + steps)
+
+
+def test_config4_two_sequences_all_steps():
+    cfg = synth.CONFIGS["C4"]
+    res = _decode_run(cfg, cfg.T, cfg.steps, seed=0, batch=[0, 101])
+    o_n, l_n, o64, l64, pools, ns, pidx, pcnt, z64 = res
+    # fp32-vs-fp64 logits may flip a replacement only when two logits are within the tolerance; with
+    # these inputs that does not happen, so the pools must match exactly
+    _assert(cfg, res, cfg.T + cfg.steps)
+    for pool in pools:
+        assert len(pool) == cfg.R and pool[-1] <= cfg.T + cfg.steps - 1 - cfg.W
+
+
+def test_checkpoint_replay_is_bitwise_identical():
+    cfg = synth.Config("ckpt", "bf16", 2, 2, 64, 200, 32, 16, 7, 0.1)
+    x = synth.make(cfg, 4, T=260)
+    c = lte.conv(torch.from_numpy(x["w"]).cuda())
+    q, k, v = (dev(x[t], cfg.dtype) for t in "qkv")
+    s0 = shape_of(cfg)
+    kp, vp = k[:, :, :200].contiguous(), v[:, :, :200].contiguous()
+    z = lte.lte_scores(s0, c, kp, vp)
+    idx, cnt = lte.lte_select(s0, z)
+    cache = lte.lte_cache_init(s0, c, kp, vp, z, idx, cnt)
+    for n in range(200, 230):
+        lte.lte_attn_decode(s0, c, cache, q[:, :, n].contiguous(), k[:, :, n].contiguous(), v[:, :, n].contiguous())
+    snap = cache.clone()
+    runs = []
+    for _ in range(2):
+        cc = snap.clone()
+        outs = [lte.lte_attn_decode(s0, c, cc, q[:, :, n].contiguous(), k[:, :, n].contiguous(),
+                                    v[:, :, n].contiguous())[0].clone() for n in range(230, 260)]
+        runs.append((torch.stack(outs), cc))
+    assert torch.equal(runs[0][0], runs[1][0]) and torch.equal(runs[0][1], runs[1][1])

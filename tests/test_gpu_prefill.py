@@ -1,0 +1,97 @@
+"""GPU parity: lte_attn_prefill against the fp64 oracle, through the C-ABI."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import lte_oracle as orc
+from paper_2510_20787_b200 import lte, synth
+from tests.gpu_util import check_idx, dev, shape_of
+
+pytestmark = pytest.mark.gpu
+
+TOL = {"bf16": 2e-2, "f32": 1e-4}
+
+
+def _pipeline(cfg, seed=0, scale=0.0, batch=None, qpos=None, tau=0.5):
+    """scores -> select -> prefill on the GPU; the oracle attends over the GPU's list once that list has
+    passed the retained-list rule, so a legitimate threshold difference cannot leak into the O comparison."""
+    x = synth.make(cfg, seed, batch=batch)
+    B = x["k"].shape[0]
+    s = shape_of(cfg, B=B, scale=scale, tau=tau)
+    c = lte.conv(torch.from_numpy(x["w"]).cuda())
+    q, k, v = (dev(x[t], cfg.dtype) for t in "qkv")
+    z = lte.lte_scores(s, c, k, v)
+    idx, cnt = lte.lte_select(s, z)
+    o, lse = lte.lte_attn_prefill(s, q, k, v, idx, cnt)
+    torch.cuda.synchronize()
+    idx_n, cnt_n = idx.cpu().numpy(), cnt.cpu().numpy()
+    z64 = orc.scores(x["k"], x["v"], x["w"])
+    check_idx(idx_n, cnt_n, z64, cfg.W, cfg.R, cfg.sink, tau)
+    o64, l64 = orc.attn_prefill(x["q"], x["k"], x["v"], idx_n, cnt_n, cfg.W, None if scale == 0.0 else scale, qpos)
+    o_n, l_n = o.float().cpu().numpy(), lse.cpu().numpy()
+    if qpos is not None:
+        o_n = np.take_along_axis(o_n, qpos[..., None].astype(np.int64), axis=2)
+        l_n = np.take_along_axis(l_n, qpos.astype(np.int64), axis=2)
+    return o_n, l_n, o64, l64
+
+
+def _assert_close(cfg, res):
+    o_n, l_n, o64, l64 = res
+    assert np.all(np.isfinite(o_n)) and np.all(np.isfinite(l_n))
+    assert np.max(np.abs(o_n - o64)) <= TOL[cfg.dtype], np.max(np.abs(o_n - o64))
+    assert np.max(np.abs(l_n - l64)) <= TOL[cfg.dtype], np.max(np.abs(l_n - l64))
+
+
+def test_config1_every_output():
+    cfg = synth.CONFIGS["C1"]
+    _assert_close(cfg, _pipeline(cfg, seed=0))
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("d,K,T,W,R,sink", [
+    (32, 1, 1, 1, 1, 0), (32, 3, 7, 3, 2, 0), (64, 5, 123, 16, 8, 2), (128, 7, 130, 9, 200, 0),
+    (64, 7, 517, 40, 0, 0), (32, 13, 1000, 64, 33, 4), (64, 9, 300, 400, 16, 0), (128, 11, 259, 11, 5, 7),
+    (64, 7, 700, 128, 128, 0), (128, 7, 1500, 512, 512, 0), (64, 7, 640, 64, 64, 0), (64, 7, 385, 129, 77, 1),
+])
+def test_odd_shapes(dtype, d, K, T, W, R, sink):
+    cfg = synth.Config("odd", dtype, 2, 3, d, T, W, R, K, 0.1, sink=sink)
+    _assert_close(cfg, _pipeline(cfg, seed=5))
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_sharp_softmax_and_threshold_off(dtype):
+    cfg = synth.Config("sharp", dtype, 1, 4, 64, 600, 32, 48, 7, 0.1, qk_unit=True)
+    _assert_close(cfg, _pipeline(cfg, seed=6, scale=1.0))
+    _assert_close(cfg, _pipeline(cfg.with_(R=600), seed=6, tau=0.0))       # dense causal for scored far keys
+
+
+def test_config2_full():
+    cfg = synth.CONFIGS["C2"]
+    _assert_close(cfg, _pipeline(cfg, seed=0))
+    _assert_close(cfg, _pipeline(cfg.with_(B=1), seed=1, scale=1.0))
+
+
+def test_config3_sampled_queries():
+    cfg = synth.CONFIGS["C3"]
+    qpos = synth.query_sample(cfg, 2048, seed=0)
+    _assert_close(cfg, _pipeline(cfg, seed=0, qpos=qpos))
+
+
+def test_config5_forward():
+    cfg = synth.CONFIGS["C5"]
+    _assert_close(cfg, _pipeline(cfg, seed=0, batch=[0, 7]))
+
+
+def test_zero_query_pins_set_sizes_on_gpu():
+    cfg = synth.Config("q0", "bf16", 1, 2, 64, 900, 100, 60, 7, 0.1)
+    x = synth.make(cfg, 2)
+    s = shape_of(cfg)
+    c = lte.conv(torch.from_numpy(x["w"]).cuda())
+    k, v = dev(x["k"], "bf16"), dev(x["v"], "bf16")
+    idx, cnt = lte.lte_select(s, lte.lte_scores(s, c, k, v))
+    o, lse = lte.lte_attn_prefill(s, torch.zeros_like(k), k, v, idx, cnt)
+    idx_n, cnt_n = idx.cpu().numpy(), cnt.cpu().numpy()
+    for h in range(2):
+        kept = idx_n[0, h, :cnt_n[0, h]]
+        sizes = np.array([min(i + 1, cfg.W) + np.sum(kept <= i - cfg.W) for i in range(cfg.T)])
+        np.testing.assert_allclose(np.exp(lse[0, h].cpu().numpy()), sizes, rtol=1e-5)
