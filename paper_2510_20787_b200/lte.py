@@ -82,7 +82,9 @@ def conv(w, bias=None):
     """w: CUDA fp32 [H, K, 2d]; bias: CUDA fp32 [H] or None."""
     assert w.is_cuda and w.dtype == torch.float32 and w.is_contiguous()
     assert bias is None or (bias.is_cuda and bias.dtype == torch.float32 and bias.is_contiguous())
-    return LteConv(1, w.shape[1], 1, w.data_ptr(), 0 if bias is None else bias.data_ptr())
+    c = LteConv(1, w.shape[1], 1, w.data_ptr(), 0 if bias is None else bias.data_ptr())
+    c._keep = (w, bias)          # the struct only holds raw pointers: keep the tensors alive with it
+    return c
 
 
 def _ptr(t, dtype=None):
