@@ -1,0 +1,453 @@
+#!/usr/bin/env python
+"""Benchmark of the LTE sparse-attention hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl lte|reference] [--no-extras]
+
+A step is one pass of the prefill hot path (lte_scores -> lte_select -> lte_attn_prefill) over one
+synthetic batch of the bf16 prefill configuration (B=4, H=16, d=64, T=4096, W=128, R=128, 7 taps).
+`value` is whole-job prefill tokens/s with the inputs resident in HBM; `e2e` is the same metric through
+the same calls with host buffers (pinned host -> device copies of q, k, v and the device -> host read of
+O, logsumexp and the retained lists inside the timed region).  With N > 1 every rank runs the same
+per-GPU batch on its own GPU (the (batch, head) units are independent: no data-path collective, weak
+scaling) and the slowest rank sets the time.  Extra sections time the other rows of the path on their
+own configurations: long prefill, batched decode (us per step, HBM GB/s) and forward+backward.
+
+`--impl reference` times the fp64 CPU oracle, as it stands, on the host cores for the same metric.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "LTE attn prefill tokens/s & % bf16 TC peak; decode step us & % HBM BW"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu captures (profiles/),
+# keyed by kernel family; None until a capture exists.
+NCU_TRAFFIC_BYTES = {"prefill_attn_C2": None, "decode_C4": None}
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        d["source"] = "measured"
+        return d
+    d = dict(FALLBACK_PEAKS)
+    d["source"] = "fallback"
+    return d
+
+
+class ClockSampler:
+    """nvidia-smi clocks / throttle reasons sampled every 200 ms while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------------------------------
+def device_inputs(cfg, seed, torch, T=None, with_dO=False):
+    """Seeded synthetic tensors of the configuration's distributions, drawn on the device."""
+    g = torch.Generator(device="cuda")
+    g.manual_seed(seed)
+    T = cfg.T if T is None else T
+    dt = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
+    shp = (cfg.B, cfg.H, T, cfg.d)
+    qk = 1.0 if cfg.qk_unit else cfg.d ** -0.25
+    out = {}
+    for name, sc in (("q", qk), ("k", qk), ("v", 1.0)) + ((("dO", 1.0),) if with_dO else ()):
+        out[name] = (torch.randn(shp, generator=g, device="cuda", dtype=torch.float32) * sc).to(dt)
+    out["w"] = torch.randn((cfg.H, cfg.K, 2 * cfg.d), generator=g, device="cuda", dtype=torch.float32) * cfg.sigma_w
+    return out
+
+
+def timed(torch, fn, steps, warmup, flush, sub_events=0):
+    """Run fn() warmup + steps times; returns per-step ms list and, if fn returns event lists, their deltas."""
+    for _ in range(warmup):
+        flush(); fn()
+    torch.cuda.synchronize()
+    ms, subs = [], []
+    for _ in range(steps):
+        flush()
+        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+        e0.record()
+        marks = fn()
+        e1.record()
+        ms.append((e0, e1)); subs.append(marks)
+    torch.cuda.synchronize()
+    out = [a.elapsed_time(b) for a, b in ms]
+    sub = None
+    if subs and subs[0]:
+        sub = [[m[i].elapsed_time(m[i + 1]) for i in range(len(m) - 1)] for m in subs]
+    return out, sub
+
+
+def mid3(xs):
+    """Mean of the middle values (the paper's protocol: middle three of five runs)."""
+    xs = sorted(xs)
+    if len(xs) >= 5:
+        k = (len(xs) - 3) // 2
+        xs = xs[k:k + 3]
+    return float(np.mean(xs))
+
+
+def attn_flops(idx, cnt, T, W, d, torch):
+    """Algorithmic attention FLOPs 4*d*|A_i| summed from the actual retained lists."""
+    B, H, R = idx.shape
+    i = torch.arange(T, device=idx.device)
+    win = torch.clamp(i + 1, max=W).sum().item() * B * H
+    thr = (i - W)                                               # entry visible iff idx <= i - W
+    ids = idx.reshape(B * H, R).to(torch.int64)
+    valid = torch.arange(R, device=idx.device)[None, :] < cnt.reshape(B * H, 1)
+    # number of queries that see entry j: T - (j + W) for j + W <= T - 1
+    vis = torch.where(valid, torch.clamp(T - (ids + W), min=0), torch.zeros_like(ids)).sum().item()
+    del thr
+    return 4.0 * d * (win + vis)
+
+
+def run_lte(args):
+    import torch
+    from paper_2510_20787_b200 import lte, synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    lte.lib()
+    pk = peaks()
+
+    cfg = synth.CONFIGS["C2"]
+    x = device_inputs(cfg, 1000 + rank, torch)
+    s = lte.shape(cfg.B, cfg.H, cfg.T, cfg.d, cfg.W, cfg.R, lte.BF16)
+    c = lte.conv(x["w"])
+    q, k, v = x["q"], x["k"], x["v"]
+    z = torch.empty((cfg.B, cfg.H, cfg.T), dtype=torch.float32, device="cuda")
+    idx = torch.empty((cfg.B, cfg.H, cfg.R), dtype=torch.int32, device="cuda")
+    cnt = torch.empty((cfg.B, cfg.H), dtype=torch.int32, device="cuda")
+    o = torch.empty_like(q)
+    lse = torch.empty((cfg.B, cfg.H, cfg.T), dtype=torch.float32, device="cuda")
+    flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+
+    def flush():
+        flush_buf.fill_(1)
+
+    def ev():
+        e = torch.cuda.Event(enable_timing=True); e.record(); return e
+
+    def step():
+        m = [ev()]
+        lte.lte_scores(s, c, k, v, z=z); m.append(ev())
+        lte.lte_select(s, z, idx=idx, cnt=cnt); m.append(ev())
+        lte.lte_attn_prefill(s, q, k, v, idx, cnt, o=o, lse=lse); m.append(ev())
+        return m
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(local)
+    barrier()
+    for _ in range(args.warmup):
+        flush(); step()
+    barrier()
+    if rank == 0:
+        sampler.start()
+    t_wall = time.time()
+    ms, sub = timed(torch, step, args.steps, 0, flush)
+    barrier()
+    t_wall = time.time() - t_wall
+    # keep the GPU busy long enough for a few clock samples
+    if rank == 0:
+        t0 = time.time()
+        while time.time() - t0 < 1.0:
+            step()
+        torch.cuda.synchronize()
+        clocks = sampler.stop()
+    step_ms = float(np.mean(ms))
+    if dist is not None:
+        t = torch.tensor([step_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        step_ms = float(t.item())
+    tokens = cfg.B * cfg.T * world
+    value = tokens / (step_ms * 1e-3)
+    sub = np.array(sub)                       # [steps, 3] ms: scores, select, attention
+    k_ms = sub.mean(axis=0)
+
+    # ---- end to end through the same calls, host buffers --------------------------------------
+    hq, hk, hv = (t.cpu().pin_memory() for t in (q, k, v))
+    ho = torch.empty(o.shape, dtype=o.dtype).pin_memory()
+    hl = torch.empty(lse.shape, dtype=lse.dtype).pin_memory()
+    hi = torch.empty(idx.shape, dtype=idx.dtype).pin_memory()
+    hc = torch.empty(cnt.shape, dtype=cnt.dtype).pin_memory()
+    dq_, dk_, dv_ = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+
+    def e2e_step():
+        dq_.copy_(hq, non_blocking=True); dk_.copy_(hk, non_blocking=True); dv_.copy_(hv, non_blocking=True)
+        lte.lte_scores(s, c, dk_, dv_, z=z)
+        lte.lte_select(s, z, idx=idx, cnt=cnt)
+        lte.lte_attn_prefill(s, dq_, dk_, dv_, idx, cnt, o=o, lse=lse)
+        ho.copy_(o, non_blocking=True); hl.copy_(lse, non_blocking=True)
+        hi.copy_(idx, non_blocking=True); hc.copy_(cnt, non_blocking=True)
+        return None
+
+    barrier()
+    e_ms, _ = timed(torch, e2e_step, args.steps, max(args.warmup, 3), flush)
+    barrier()
+    e2e_ms = float(np.mean(e_ms))
+    if dist is not None:
+        t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    h2d = sum(t.numel() * t.element_size() for t in (hq, hk, hv))
+    d2h = sum(t.numel() * t.element_size() for t in (ho, hl, hi, hc))
+
+    # ---- roofline of the dominant kernel -----------------------------------------------------------
+    esz = 2
+    attn_bytes = 4 * cfg.B * cfg.H * cfg.T * cfg.d * esz + cfg.B * cfg.H * cfg.T * 4 + cfg.B * cfg.H * (cfg.R + 1) * 4
+    score_bytes = 2 * cfg.B * cfg.H * cfg.T * cfg.d * esz + cfg.B * cfg.H * cfg.T * 4
+    flops = attn_flops(idx, cnt, cfg.T, cfg.W, cfg.d, torch)
+    attn_s = k_ms[2] * 1e-3
+    roof = {"bound": "hbm", "kernel": "lte_attn_prefill", "achieved": attn_bytes / attn_s / 1e9,
+            "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": attn_bytes / attn_s / 1e9 / pk["hbm_gbs"],
+            "traffic": NCU_TRAFFIC_BYTES["prefill_attn_C2"], "peak_source": pk["source"],
+            "algorithmic_bytes": attn_bytes, "algorithmic_flops": flops,
+            "tensor_tflops": flops / attn_s / 1e12, "tensor_frac": flops / attn_s / 1e12 / pk["bf16_tflops"],
+            "kernel_ms": {"lte_scores": float(k_ms[0]), "lte_select": float(k_ms[1]), "lte_attn_prefill": float(k_ms[2])},
+            "scores_gbs": score_bytes / (k_ms[0] * 1e-3) / 1e9}
+
+    line = {"metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "C2 bf16 prefill: B=4 H=16 d=64 T=4096 W=128 R=128 K=7 per GPU, "
+                                   "scores+select+attention", "l2": "flushed between timed steps (256 MB write)",
+                       "parallelism": "replicas x%d (independent (batch, head) units)" % world},
+            "e2e": {"value": tokens / (e2e_ms * 1e-3), "unit": "tokens/s", "ms_per_step": e2e_ms,
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+            "gpu_launches": 3 * args.steps, "roofline": roof, "wall_s": t_wall}
+    if rank == 0:
+        line["clocks"] = clocks
+
+    # ---- the other rows of the path on their own configurations --------------------------------
+    if not args.no_extras and rank == 0 and world == 1:
+        del hq, hk, hv, ho, dq_, dk_, dv_
+        line["extras"] = extras(torch, lte, synth, pk, flush, args)
+        line["cpu_baseline"] = cpu_baseline(synth)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(line))
+
+
+def extras(torch, lte, synth, pk, flush, args):
+    out = {}
+    n5 = 5
+
+    # long prefill (tensor-core bound)
+    cfg = synth.CONFIGS["C3"]
+    x = device_inputs(cfg, 3, torch)
+    s = lte.shape(cfg.B, cfg.H, cfg.T, cfg.d, cfg.W, cfg.R, lte.BF16)
+    c = lte.conv(x["w"])
+    z = lte.lte_scores(s, c, x["k"], x["v"])
+    idx, cnt = lte.lte_select(s, z)
+    o = torch.empty_like(x["q"]); lse = torch.empty((cfg.B, cfg.H, cfg.T), dtype=torch.float32, device="cuda")
+    def f_attn():
+        lte.lte_attn_prefill(s, x["q"], x["k"], x["v"], idx, cnt, o=o, lse=lse)
+
+    def f_scores():
+        lte.lte_scores(s, c, x["k"], x["v"], z=z)
+
+    def f_select():
+        lte.lte_select(s, z, idx=idx, cnt=cnt)
+
+    ms, _ = timed(torch, f_attn, n5, 3, flush)
+    ms_sc, _ = timed(torch, f_scores, n5, 3, flush)
+    ms_se, _ = timed(torch, f_select, n5, 3, flush)
+    fl = attn_flops(idx, cnt, cfg.T, cfg.W, cfg.d, torch)
+    t = mid3(ms) * 1e-3
+    out["C3_long_prefill"] = {"attn_ms": t * 1e3, "tokens_per_s": cfg.B * cfg.T / t, "algorithmic_tflops": fl / t / 1e12,
+                              "tensor_frac": fl / t / 1e12 / pk["bf16_tflops"], "scores_ms": mid3(ms_sc),
+                              "select_ms": mid3(ms_se)}
+    del x, o, lse, z
+
+    # forward + backward
+    cfg = synth.CONFIGS["C5"]
+    x = device_inputs(cfg, 5, torch, with_dO=True)
+    s = lte.shape(cfg.B, cfg.H, cfg.T, cfg.d, cfg.W, cfg.R, lte.BF16)
+    c = lte.conv(x["w"])
+    z = lte.lte_scores(s, c, x["k"], x["v"])
+    idx, cnt = lte.lte_select(s, z)
+    o, lse = lte.lte_attn_prefill(s, x["q"], x["k"], x["v"], idx, cnt)
+    ws = torch.empty(lte.lte_workspace_bytes(lte.OP_BWD, s, c), dtype=torch.uint8, device="cuda")
+
+    def fwd():
+        lte.lte_scores(s, c, x["k"], x["v"], z=z); lte.lte_select(s, z, idx=idx, cnt=cnt)
+        lte.lte_attn_prefill(s, x["q"], x["k"], x["v"], idx, cnt, o=o, lse=lse)
+
+    def bwd():
+        lte.lte_attn_bwd(s, c, x["q"], x["k"], x["v"], o, lse, x["dO"], z, idx, cnt, ws=ws)
+
+    ms_f, _ = timed(torch, fwd, n5, 3, flush)
+    ms_b, _ = timed(torch, bwd, n5, 3, flush)
+    fl = attn_flops(idx, cnt, cfg.T, cfg.W, cfg.d, torch)
+    tf, tb = mid3(ms_f) * 1e-3, mid3(ms_b) * 1e-3
+    nb = cfg.B * cfg.H * cfg.T * cfg.d * 2
+    out["C5_fwd_bwd"] = {"fwd_ms": tf * 1e3, "bwd_ms": tb * 1e3, "tokens_per_s": cfg.B * cfg.T / (tf + tb),
+                         "bwd_algorithmic_tflops": 2.5 * fl / tb / 1e12, "bwd_hbm_gbs": 8 * nb / tb / 1e9,
+                         "bwd_hbm_frac": 8 * nb / tb / 1e9 / pk["hbm_gbs"]}
+    del x, o, lse, z, ws
+
+    # batched decode
+    cfg = synth.CONFIGS["C4"]
+    x = device_inputs(cfg, 4, torch)
+    s = lte.shape(cfg.B, cfg.H, cfg.T, cfg.d, cfg.W, cfg.R, lte.BF16)
+    c = lte.conv(x["w"])
+    z = lte.lte_scores(s, c, x["k"], x["v"])
+    idx, cnt = lte.lte_select(s, z)
+    cache = lte.lte_cache_init(s, c, x["k"], x["v"], z, idx, cnt)
+    del x, z
+    g = torch.Generator(device="cuda"); g.manual_seed(44)
+    sc = cfg.d ** -0.25
+    qs, ks, vs = ((torch.randn((cfg.steps, cfg.B, cfg.H, cfg.d), generator=g, device="cuda") * f).to(torch.bfloat16)
+                  for f in (sc, sc, 1.0))
+    o1 = torch.empty((cfg.B, cfg.H, cfg.d), dtype=torch.bfloat16, device="cuda")
+    l1 = torch.empty((cfg.B, cfg.H), dtype=torch.float32, device="cuda")
+    for i in range(8):                                            # warm-up steps advance the cache too
+        lte.lte_attn_decode(s, c, cache, qs[i], ks[i], vs[i], o1=o1, lse1=l1)
+    torch.cuda.synchronize()
+    evs = []
+    for i in range(8, cfg.steps):
+        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+        e0.record(); lte.lte_attn_decode(s, c, cache, qs[i], ks[i], vs[i], o1=o1, lse1=l1); e1.record()
+        evs.append((e0, e1))
+    torch.cuda.synchronize()
+    us = float(np.mean([a.elapsed_time(b) for a, b in evs])) * 1e3
+    per = 2 * (cfg.W + cfg.R) * cfg.d * 2 + cfg.R * 4 + 1024 + 16      # ring+pool K,V, pool logits, q/k/v/o + row writes, meta
+    by = per * cfg.B * cfg.H
+    out["C4_decode"] = {"us_per_step": us, "steps_timed": len(evs), "algorithmic_bytes_per_step": by,
+                        "hbm_gbs": by / (us * 1e-6) / 1e9, "hbm_frac": by / (us * 1e-6) / 1e9 / pk["hbm_gbs"],
+                        "traffic": NCU_TRAFFIC_BYTES["decode_C4"],
+                        "note": "the 138 MB cache is about the size of L2: see the ncu DRAM bytes in profiles/"}
+    return out
+
+
+def oracle_step(orc, x, cfg):
+    z = orc.scores(x["k"], x["v"], x["w"])
+    idx, cnt, _ = orc.select(z, cfg.W, cfg.R)
+    orc.attn_prefill(x["q"], x["k"], x["v"], idx, cnt, cfg.W)
+
+
+def cpu_baseline(synth, reps=8):
+    """The fp64 oracle, as it stands, on the host cores: the whole C2 batch, `reps` times."""
+    from oracle import lte_oracle as orc
+    cfg = synth.CONFIGS["C2"]
+    x = synth.make(cfg, 0)
+    x = {n: np.asarray(a, np.float64) for n, a in x.items()}
+    oracle_step(orc, x, cfg)
+    t0 = time.time()
+    for _ in range(reps):
+        oracle_step(orc, x, cfg)
+    dt = (time.time() - t0) / reps
+    return {"value": cfg.B * cfg.T / dt, "unit": "tokens/s", "cores": orc.num_threads(), "kind": "oracle",
+            "sample": "the full C2 batch (B=4, 16384 tokens), scores+select+attention, mean of %d passes" % reps,
+            "ms_per_step": dt * 1e3}
+
+
+def run_reference(args):
+    """Reference arm: the oracle on the host cores, same metric and configuration; rank 0 only."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    from oracle import lte_oracle as orc
+    from paper_2510_20787_b200 import synth
+    cfg = synth.CONFIGS["C2"]
+    x = synth.make(cfg, 0)
+    x = {n: np.asarray(a, np.float64) for n, a in x.items()}
+    for _ in range(min(args.warmup, 3)):
+        oracle_step(orc, x, cfg)
+    steps = min(args.steps, 20)
+    t0 = time.time()
+    for _ in range(steps):
+        oracle_step(orc, x, cfg)
+    dt = (time.time() - t0) / steps
+    val = cfg.B * cfg.T / dt
+    sample = "each step = the full C2 batch once (B=4, 16384 tokens); %d steps timed" % steps
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": "tokens/s", "n_gpus": args.gpus,
+        "steps": steps, "warmup": min(args.warmup, 3), "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "C2 bf16 prefill: B=4 H=16 d=64 T=4096 W=128 R=128 K=7, scores+select+attention"},
+        "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": orc.num_threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="lte", choices=["lte", "reference"])
+    ap.add_argument("--no-extras", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_lte(args)
+
+
+if __name__ == "__main__":
+    main()
