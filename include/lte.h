@@ -62,6 +62,13 @@ typedef enum lte_op {
 /* Bytes of caller-supplied scratch the given entry point needs for this shape (0 if none). */
 size_t lte_workspace_bytes(int op, const lte_shape* s, const lte_conv* c);
 
+/*
+ * Sticky device-side status of the current device: LTE_OK, or LTE_ERR_DEVICE_STATUS if a kernel since the
+ * last call gave up on a bounded wait (its outputs are then undefined).  Synchronous (a 4-byte copy from
+ * the device, ordered after previously launched work on the legacy default stream's rules); reading clears it.
+ */
+int lte_device_status(void);
+
 /* Static text for a status code. */
 const char* lte_strerror(int status);
 

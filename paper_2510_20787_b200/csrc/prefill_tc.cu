@@ -1,9 +1,427 @@
-// placeholder until the tensor-core kernel lands: bf16 prefill runs on the fp32-ALU kernel
+// Prefill attention on the 5th-generation tensor cores (Section 3.1.3, "Cached prefilling and decoding").
+//
+// One CTA (128 threads) per 128-query tile of one (b,h).  Key/value tiles of 128 rows come from two
+// sources, as in the paper's two-stage loop: (1) the contiguous window span, staged by TMA
+// (cp.async.bulk.tensor, 128-byte swizzle); (2) the retained rows already out of the tile's window,
+// gathered row by row with cp.async into the same swizzled layout (idx is ascending, so the entries a
+// query may see are a prefix of the list and every mask is a column range).  Per tile:
+//   S = Q K^T      tcgen05.mma (kind::f16, bf16 in, fp32 out) into TMEM, operands from shared memory
+//   softmax        thread r owns query row r = TMEM lane r: tcgen05.ld, range mask, running max / sum in
+//                  fp32 (exp2 with the scale folded in), P written as bf16 into swizzled shared memory
+//   O_tile = P V   tcgen05.mma with V as an MN-major operand, fresh TMEM accumulator, then folded into
+//                  the fp32 register accumulator with the online-softmax rescale.
+// K/V loads of tile t+1 are in flight while tile t is computed (two stages).  Every mbarrier wait is
+// bounded; a wait that runs out records a status word and the kernel still terminates.
+#include <cuda.h>
+
 #include "common.cuh"
+
 namespace lte {
+
+__device__ int g_prefill_status = 0;          // 0 = fine; otherwise the code of the wait that gave up
+
+namespace {
+
+constexpr int BM = 128, BN = 128, NTHREADS = 128;
+constexpr uint32_t kSpinLimit = 1u << 22;
+
+// ---- PTX wrappers -----------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: gives up after kSpinLimit polls, records `code`, and lets the kernel run on to its end.
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, int code) {
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        if (mbar_try_wait(bar, parity)) return;
+        // once any wait has given up, the launch is lost: stop waiting everywhere so it ends quickly
+        if ((i & 1023u) == 1023u && *reinterpret_cast<volatile int*>(&g_prefill_status) != 0) return;
+    }
+    atomicExch(&g_prefill_status, code);
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, int x, int y, int z, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+                 ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tmem_alloc(uint32_t slot, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot), "r"(ncols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                 "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                 "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                   "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                   "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                 : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, 128-byte swizzle, 8-row atoms of 1024 bytes.
+//   K-major operand  (rows = M or N index, 128 bytes of K per row): SBO = 1024 between 8-row groups.
+//   MN-major operand (rows = K index, 128 bytes = 64 elements of N per row): SBO = 1024 between 8-row
+//   K groups, LBO = distance between consecutive 64-element N groups.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
+           (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor: fp32 accumulator, bf16 A and B, A K-major, B K-major or MN-major, M x N.
+__host__ __device__ constexpr uint32_t instr_desc(int M, int N, bool b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(N >> 3) << 17) |
+           ((uint32_t)(M >> 4) << 24);
+}
+
+template <int D> struct Smem {
+    static constexpr int SUB = D / 64;                        // 64-column (128-byte) sub-tiles per row
+    static constexpr int TILE = 128 * D * 2;                  // bytes of one [128][D] bf16 tile
+    static constexpr int OFF_Q = 0;
+    static constexpr int OFF_K = TILE;                        // 2 stages
+    static constexpr int OFF_V = OFF_K + 2 * TILE;            // 2 stages
+    static constexpr int OFF_P = OFF_V + 2 * TILE;            // [128][128] bf16 = 32 KB
+    static constexpr int OFF_BAR = OFF_P + 128 * 128 * 2;     // mbarriers + tmem slot
+    static constexpr int BYTES = OFF_BAR + 128 + 1024;        // + slack for the 1024-byte alignment
+};
+
+template <int D>
+__global__ void __launch_bounds__(NTHREADS, D == 64 ? 2 : 1)
+prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                  const __grid_constant__ CUtensorMap tmV, const __nv_bfloat16* __restrict__ kg,
+                  const __nv_bfloat16* __restrict__ vg, const int32_t* __restrict__ idx,
+                  const int32_t* __restrict__ cnt, __nv_bfloat16* __restrict__ o, float* __restrict__ lse, int Tlen,
+                  int W, int R, float scale)
+{
+    using S = Smem<D>;
+    constexpr int SUB = S::SUB;
+    constexpr uint32_t TMEM_COLS = 256;                        // S: columns [0,128), O tile: [128, 128+D)
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* gen = smem_raw + (base - smem_u32(smem_raw));     // generic pointer to the aligned base
+    const uint32_t sQ = base + S::OFF_Q, sK = base + S::OFF_K, sV = base + S::OFF_V, sP = base + S::OFF_P;
+    const uint32_t bar_q = base + S::OFF_BAR, bar_kv0 = bar_q + 8, bar_s = bar_q + 24, bar_o = bar_q + 32;
+    const uint32_t tmem_slot = bar_q + 40;
+    volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(gen + S::OFF_BAR + 40);
+    volatile int* s_nvmax = reinterpret_cast<volatile int*>(gen + S::OFF_BAR + 48);
+
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int bh = blockIdx.y;
+    const int i0 = blockIdx.x * BM;
+    const int i = i0 + tid;                                    // this thread's query row
+    const int i_hi = min(i0 + BM - 1, Tlen - 1);
+
+    if (tid == 0) {
+        mbar_init(bar_q, 1); mbar_init(bar_kv0, 1); mbar_init(bar_kv0 + 8, 1); mbar_init(bar_s, 1); mbar_init(bar_o, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) { __syncwarp(); tmem_alloc(tmem_slot, TMEM_COLS); }
+
+    // retained entries visible to this row: idx ascending => a prefix of length nvis
+    const int32_t* id = idx + (size_t)bh * R;
+    const int n_ret = cnt[bh];
+    int nvis;
+    {
+        const int lim = min(i, Tlen - 1) - W;                  // entry visible iff idx <= lim
+        int lo = 0, hi = n_ret;
+        while (lo < hi) { const int mid = (lo + hi) >> 1; if (id[mid] <= lim) lo = mid + 1; else hi = mid; }
+        nvis = lo;
+    }
+    if (i == i_hi) *s_nvmax = nvis;
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot_gen;
+    const int nv_max = *s_nvmax;
+
+    const int j_start = max(i0 - W + 1, 0);
+    const int n_win = (i_hi - j_start + 1 + BN - 1) / BN;
+    const int n_rt = (nv_max + BN - 1) / BN;
+    const int n_tiles = n_win + n_rt;
+
+    // ---- loads ---------------------------------------------------------------------------------
+    auto issue_tile = [&](int t) {
+        const int st = t & 1;
+        const uint32_t dK = sK + st * S::TILE, dV = sV + st * S::TILE;
+        if (t < n_win) {
+            if (tid == 0) {
+                const uint32_t bar = bar_kv0 + 8 * st;
+                mbar_expect_tx(bar, 2 * S::TILE);
+                const int y = j_start + t * BN;
+#pragma unroll
+                for (int sb = 0; sb < SUB; ++sb) {
+                    tma_load_3d(dK + sb * 16384, &tmK, sb * 64, y, bh, bar);
+                    tma_load_3d(dV + sb * 16384, &tmV, sb * 64, y, bh, bar);
+                }
+            }
+        } else {
+            // gather row e of the retained list into row `tid` of the stage (zero-filled past the visible prefix)
+            const int e = (t - n_win) * BN + tid;
+            const bool ok = e < nv_max;
+            const size_t row = ((size_t)bh * Tlen + (ok ? id[e] : 0)) * D;
+            const uint32_t nbytes = ok ? 16u : 0u;
+#pragma unroll
+            for (int ch = 0; ch < D / 8; ++ch) {
+                const uint32_t off = (ch >> 3) * 16384 + tid * 128 + (((ch & 7) ^ (tid & 7)) << 4);
+                cp_async16(dK + off, kg + row + ch * 8, nbytes);
+                cp_async16(dV + off, vg + row + ch * 8, nbytes);
+            }
+        }
+        cp_async_commit();                                     // one group per tile (empty for TMA tiles)
+    };
+
+    if (tid == 0) {
+        mbar_expect_tx(bar_q, S::TILE);
+#pragma unroll
+        for (int sb = 0; sb < SUB; ++sb) tma_load_3d(sQ + sb * 16384, &tmQ, sb * 64, i0, bh, bar_q);
+    }
+    issue_tile(0);
+
+    constexpr uint32_t IDESC_S = instr_desc(BM, BN, false);
+    constexpr uint32_t IDESC_O = instr_desc(BM, D, true);
+    const float c2 = scale * 1.4426950408889634f;              // logits are handled as s * scale * log2(e)
+    const uint32_t lane_base = ((uint32_t)(warp * 32)) << 16;   // this warp's TMEM lanes
+
+    float acc[D];
+#pragma unroll
+    for (int c = 0; c < D; ++c) acc[c] = 0.f;
+    float m_run = -INFINITY, l_run = 0.f;
+    uint32_t kv_phase = 0;                                     // bit st = parity of stage st's TMA barrier
+
+    for (int t = 0; t < n_tiles; ++t) {
+        const int st = t & 1;
+        if (t + 1 < n_tiles) issue_tile(t + 1);
+        // ---- wait for tile t's operands
+        if (t + 1 < n_tiles) cp_async_wait<1>(); else cp_async_wait<0>();
+        if (t >= n_win) fence_proxy_async();
+        if (t == 0 && tid == 0) mbar_wait(bar_q, 0, 1);
+        if (t < n_win) {
+            if (tid == 0) mbar_wait(bar_kv0 + 8 * st, (kv_phase >> st) & 1u, 2);
+            kv_phase ^= 1u << st;
+        }
+        tc_fence_before();
+        __syncthreads();                                       // gathered rows visible; O-tile reads of tile t-1 done
+        // ---- S = Q K^T
+        if (tid == 0) {
+            tc_fence_after();
+            const uint32_t kb = sK + st * S::TILE;
+#pragma unroll
+            for (int kk = 0; kk < D / 16; ++kk) {
+                const uint32_t off = (kk >> 2) * 16384 + (kk & 3) * 32;
+                umma(tmem, smem_desc(sQ + off, 16, 1024), smem_desc(kb + off, 16, 1024), IDESC_S, kk > 0);
+            }
+            umma_commit(bar_s);
+        }
+        // column range this row may see in the tile
+        int c_lo, c_hi;
+        if (t < n_win) {
+            const int jt0 = j_start + t * BN;
+            c_lo = max(i - W + 1, 0) - jt0;
+            c_hi = i - jt0;
+        } else {
+            c_lo = 0;
+            c_hi = nvis - (t - n_win) * BN - 1;
+        }
+        mbar_wait(bar_s, t & 1, 3);
+        tc_fence_after();
+
+        // ---- softmax over the row: pass 1 row max, pass 2 exponentials -> P (bf16, swizzled)
+        float m_tile = -INFINITY;
+#pragma unroll
+        for (int cb = 0; cb < BN / 32; ++cb) {
+            uint32_t r[32];
+            tmem_ld32(tmem + lane_base + cb * 32, r);
+            tmem_wait_ld();
+#pragma unroll
+            for (int c = 0; c < 32; ++c) {
+                const int col = cb * 32 + c;
+                if (col >= c_lo && col <= c_hi) m_tile = fmaxf(m_tile, __uint_as_float(r[c]));
+            }
+        }
+        const float m_new = fmaxf(m_run, m_tile);
+        const float m_use = m_new == -INFINITY ? 0.f : m_new;
+        const float alpha = m_run == -INFINITY ? 0.f : fast_exp2((m_run - m_use) * c2);
+        const float mb = m_use * c2;
+        float l_tile = 0.f;
+#pragma unroll
+        for (int cb = 0; cb < BN / 32; ++cb) {
+            uint32_t r[32];
+            tmem_ld32(tmem + lane_base + cb * 32, r);
+            tmem_wait_ld();
+            uint32_t pk[16];
+#pragma unroll
+            for (int c = 0; c < 32; c += 2) {
+                const int col = cb * 32 + c;
+                float p0 = (col >= c_lo && col <= c_hi) ? fast_exp2(fmaf(__uint_as_float(r[c]), c2, -mb)) : 0.f;
+                float p1 = (col + 1 >= c_lo && col + 1 <= c_hi) ? fast_exp2(fmaf(__uint_as_float(r[c + 1]), c2, -mb)) : 0.f;
+                __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
+                // the row sum uses the rounded probabilities, i.e. exactly what the PV product consumes
+                l_tile += __low2float(h) + __high2float(h);
+                pk[c >> 1] = *reinterpret_cast<uint32_t*>(&h);
+            }
+            // 32 columns = 4 chunks of 16 bytes; column block cb lives in sub-tile cb/2, chunks (cb&1)*4 ..
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+                const int ch = (cb & 1) * 4 + g;
+                const uint32_t dst = sP + (cb >> 1) * 16384 + tid * 128 + ((ch ^ (tid & 7)) << 4);
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(pk[4 * g]), "r"(pk[4 * g + 1]),
+                             "r"(pk[4 * g + 2]), "r"(pk[4 * g + 3]) : "memory");
+            }
+        }
+        l_run = l_run * alpha + l_tile;
+        m_run = m_new;
+        fence_proxy_async();                                   // P (generic proxy) -> visible to the MMA (async proxy)
+        tc_fence_before();
+        __syncthreads();
+        // ---- O_tile = P V
+        if (tid == 0) {
+            tc_fence_after();
+            const uint32_t vb = sV + st * S::TILE;
+#pragma unroll
+            for (int kk = 0; kk < BN / 16; ++kk) {
+                const uint32_t aoff = (kk >> 2) * 16384 + (kk & 3) * 32;
+                umma(tmem + 128, smem_desc(sP + aoff, 16, 1024), smem_desc(vb + kk * 2048, 16384, 1024), IDESC_O, kk > 0);
+            }
+            umma_commit(bar_o);
+        }
+        mbar_wait(bar_o, t & 1, 4);
+        tc_fence_after();
+#pragma unroll
+        for (int cb = 0; cb < D / 32; ++cb) {
+            uint32_t r[32];
+            tmem_ld32(tmem + lane_base + 128 + cb * 32, r);
+            tmem_wait_ld();
+#pragma unroll
+            for (int c = 0; c < 32; ++c) acc[cb * 32 + c] = fmaf(acc[cb * 32 + c], alpha, __uint_as_float(r[c]));
+        }
+    }
+
+    // ---- epilogue ------------------------------------------------------------------------------
+    if (i < Tlen) {
+        const float inv = 1.f / l_run;
+        __nv_bfloat16* orow = o + ((size_t)bh * Tlen + i) * D;
+#pragma unroll
+        for (int c = 0; c < D; c += 8) {
+            uint32_t w4[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                __nv_bfloat162 h = __floats2bfloat162_rn(acc[c + 2 * u] * inv, acc[c + 2 * u + 1] * inv);
+                w4[u] = *reinterpret_cast<uint32_t*>(&h);
+            }
+            *reinterpret_cast<uint4*>(orow + c) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+        }
+        lse[(size_t)bh * Tlen + i] = m_run * scale + logf(l_run);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, TMEM_COLS);
+}
+
+// ---- host side: tensor maps ---------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+// [B*H][T][d] bf16 viewed as a 3-D tensor (d fastest); box = 64 columns x 128 rows, 128-byte swizzle.
+bool make_map(CUtensorMap* m, const void* ptr, int BH, int T, int d)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)T, (cuuint64_t)BH};
+    cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)T * d * 2};
+    cuuint32_t box[3] = {64, 128, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int D>
+int run(const Params& p, const void* q, const void* k, const void* v, const int32_t* idx, const int32_t* cnt, void* o,
+        float* lse, cudaStream_t st)
+{
+    CUtensorMap tq, tk, tv;
+    const int BH = p.B * p.H;
+    if (!make_map(&tq, q, BH, p.T, D) || !make_map(&tk, k, BH, p.T, D) || !make_map(&tv, v, BH, p.T, D))
+        return LTE_ERR_CUDA;
+    static bool attr_done = false;
+    if (!attr_done) {
+        if (cudaFuncSetAttribute(prefill_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::BYTES) !=
+            cudaSuccess)
+            return LTE_ERR_CUDA;
+        attr_done = true;
+    }
+    dim3 grid((p.T + BM - 1) / BM, BH);
+    prefill_tc_kernel<D><<<grid, NTHREADS, Smem<D>::BYTES, st>>>(tq, tk, tv, (const __nv_bfloat16*)k,
+                                                                 (const __nv_bfloat16*)v, idx, cnt, (__nv_bfloat16*)o,
+                                                                 lse, p.T, p.W, p.R, p.scale);
+    return cuda_status(cudaGetLastError());
+}
+
+}  // namespace
+
 int launch_prefill_tc(const Params& p, const void* q, const void* k, const void* v, const int32_t* idx,
                       const int32_t* cnt, void* o, float* lse, cudaStream_t st)
 {
-    return launch_prefill_simt(p, q, k, v, idx, cnt, o, lse, st);
+    switch (p.d) {
+        case 64: return run<64>(p, q, k, v, idx, cnt, o, lse, st);
+        case 128: return run<128>(p, q, k, v, idx, cnt, o, lse, st);
+    }
+    return launch_prefill_simt(p, q, k, v, idx, cnt, o, lse, st);   // d = 32: rows too narrow for the 128-byte swizzle
 }
+
+int prefill_status_fetch_and_clear()
+{
+    int h = 0, zero = 0;
+    if (cudaMemcpyFromSymbol(&h, g_prefill_status, sizeof(int)) != cudaSuccess) return -1;
+    if (h != 0) cudaMemcpyToSymbol(g_prefill_status, &zero, sizeof(int));
+    return h;
+}
+
 }  // namespace lte

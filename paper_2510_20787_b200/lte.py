@@ -18,7 +18,7 @@ F32, BF16 = 0, 1
 OP_SCORES, OP_SELECT, OP_PREFILL, OP_DECODE, OP_BWD = range(5)
 BWD_CNN_INPUT_GRAD = 1
 
-EXPORTS = ["lte_workspace_bytes", "lte_strerror", "lte_scores", "lte_select", "lte_attn_prefill",
+EXPORTS = ["lte_device_status", "lte_workspace_bytes", "lte_strerror", "lte_scores", "lte_select", "lte_attn_prefill",
            "lte_cache_bytes", "lte_cache_init", "lte_attn_decode", "lte_attn_bwd"]
 
 
@@ -50,6 +50,8 @@ def lib():
         L.lte_strerror.argtypes = [ctypes.c_int]
         L.lte_workspace_bytes.restype = ctypes.c_size_t
         L.lte_workspace_bytes.argtypes = [ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p]
+        L.lte_device_status.restype = ctypes.c_int
+        L.lte_device_status.argtypes = []
         L.lte_cache_bytes.restype = ctypes.c_size_t
         L.lte_cache_bytes.argtypes = [ctypes.c_void_p]
         vp = ctypes.c_void_p
@@ -60,7 +62,7 @@ def lib():
         L.lte_attn_decode.argtypes = [vp] * 9
         L.lte_attn_bwd.argtypes = [vp] * 17 + [ctypes.c_uint32, vp, ctypes.c_size_t, vp]
         for name in EXPORTS:
-            if name not in ("lte_strerror", "lte_workspace_bytes", "lte_cache_bytes"):
+            if name not in ("lte_strerror", "lte_workspace_bytes", "lte_cache_bytes", "lte_device_status"):
                 getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -103,6 +105,11 @@ def _stream():
 def _check(fn, status):
     if status != 0:
         raise LteError(fn, status)
+
+
+def lte_device_status():
+    """0, or LTE_ERR_DEVICE_STATUS (-6) if a kernel gave up on a bounded wait since the last call."""
+    return int(lib().lte_device_status())
 
 
 def lte_workspace_bytes(op, s, c=None):

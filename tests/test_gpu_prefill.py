@@ -95,3 +95,8 @@ def test_zero_query_pins_set_sizes_on_gpu():
         kept = idx_n[0, h, :cnt_n[0, h]]
         sizes = np.array([min(i + 1, cfg.W) + np.sum(kept <= i - cfg.W) for i in range(cfg.T)])
         np.testing.assert_allclose(np.exp(lse[0, h].cpu().numpy()), sizes, rtol=1e-5)
+
+
+def test_no_bounded_wait_expired():
+    # runs after the cases above in this file: the tensor-core kernel's waits are bounded, and none gave up
+    assert lte.lte_device_status() == 0
