@@ -22,7 +22,7 @@ __device__ int g_prefill_status = 0;          // 0 = fine; otherwise the code of
 
 namespace {
 
-constexpr int BM = 128, BN = 128, NTHREADS = 128;
+constexpr int BM = 128, BN = 64, NTHREADS = 128;
 constexpr uint32_t kSpinLimit = 1u << 22;
 
 // ---- PTX wrappers -----------------------------------------------------------------------------
@@ -86,6 +86,17 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
                    "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
                  : "r"(taddr) : "memory");
 }
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+                 "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+                 "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+                 ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+                   "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+                   "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+                   "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ float fast_exp2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -109,17 +120,20 @@ __host__ __device__ constexpr uint32_t instr_desc(int M, int N, bool b_mn_major)
 
 template <int D> struct Smem {
     static constexpr int SUB = D / 64;                        // 64-column (128-byte) sub-tiles per row
-    static constexpr int TILE = 128 * D * 2;                  // bytes of one [128][D] bf16 tile
+    static constexpr int QTILE = BM * D * 2;                  // [128][D] bf16
+    static constexpr int KVTILE = BN * D * 2;                 // [64][D] bf16
     static constexpr int OFF_Q = 0;
-    static constexpr int OFF_K = TILE;                        // 2 stages
-    static constexpr int OFF_V = OFF_K + 2 * TILE;            // 2 stages
-    static constexpr int OFF_P = OFF_V + 2 * TILE;            // [128][128] bf16 = 32 KB
-    static constexpr int OFF_BAR = OFF_P + 128 * 128 * 2;     // mbarriers + tmem slot
-    static constexpr int BYTES = OFF_BAR + 128 + 1024;        // + slack for the 1024-byte alignment
+    static constexpr int OFF_K = QTILE;                       // 2 stages
+    static constexpr int OFF_V = OFF_K + 2 * KVTILE;          // 2 stages
+    static constexpr int OFF_P = OFF_V + 2 * KVTILE;          // [128][64] bf16 = 16 KB
+    static constexpr int OFF_BAR = OFF_P + BM * BN * 2;       // mbarriers, tmem slot, scratch ints
+    static constexpr int OFF_IDX = OFF_BAR + 128;             // 128 staged list entries
+    static constexpr int BYTES = OFF_IDX + 512;
+    static constexpr uint32_t TMEM_COLS = D == 64 ? 128 : 256; // S: [0,64), O: [64, 64+D)
 };
 
 template <int D>
-__global__ void __launch_bounds__(NTHREADS, D == 64 ? 2 : 1)
+__global__ void __launch_bounds__(NTHREADS, D == 64 ? 3 : 2)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                   const __grid_constant__ CUtensorMap tmV, const __nv_bfloat16* __restrict__ kg,
                   const __nv_bfloat16* __restrict__ vg, const int32_t* __restrict__ idx,
@@ -128,37 +142,59 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 {
     using S = Smem<D>;
     constexpr int SUB = S::SUB;
-    constexpr uint32_t TMEM_COLS = 256;                        // S: columns [0,128), O tile: [128, 128+D)
-    extern __shared__ uint8_t smem_raw[];
-    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    uint8_t* gen = smem_raw + (base - smem_u32(smem_raw));     // generic pointer to the aligned base
+    constexpr uint32_t TMEM_COLS = S::TMEM_COLS;
+    constexpr uint32_t O_COL = BN;
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    const uint32_t base = smem_u32(smem_raw);
+    if ((base & 1023u) != 0) {                                 // the swizzled tiles need 1024-byte alignment
+        if (threadIdx.x == 0) atomicExch(&g_prefill_status, 9);
+        return;
+    }
     const uint32_t sQ = base + S::OFF_Q, sK = base + S::OFF_K, sV = base + S::OFF_V, sP = base + S::OFF_P;
-    const uint32_t bar_q = base + S::OFF_BAR, bar_kv0 = bar_q + 8, bar_s = bar_q + 24, bar_o = bar_q + 32;
-    const uint32_t tmem_slot = bar_q + 40;
-    volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(gen + S::OFF_BAR + 40);
-    volatile int* s_nvmax = reinterpret_cast<volatile int*>(gen + S::OFF_BAR + 48);
+    const uint32_t bar_q = base + S::OFF_BAR, bar_k0 = bar_q + 8, bar_v0 = bar_q + 24, bar_s = bar_q + 40;
+    const uint32_t tmem_slot = bar_q + 48;
+    volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(smem_raw + S::OFF_BAR + 48);
+    volatile int* s_nvmax = reinterpret_cast<volatile int*>(smem_raw + S::OFF_BAR + 52);
+    volatile int* s_idx = reinterpret_cast<volatile int*>(smem_raw + S::OFF_IDX);
 
-    const int tid = threadIdx.x, warp = tid >> 5;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int bh = blockIdx.y;
     const int i0 = blockIdx.x * BM;
     const int i = i0 + tid;                                    // this thread's query row
     const int i_hi = min(i0 + BM - 1, Tlen - 1);
 
     if (tid == 0) {
-        mbar_init(bar_q, 1); mbar_init(bar_kv0, 1); mbar_init(bar_kv0 + 8, 1); mbar_init(bar_s, 1); mbar_init(bar_o, 1);
+        mbar_init(bar_q, 1); mbar_init(bar_k0, 1); mbar_init(bar_k0 + 8, 1); mbar_init(bar_v0, 1);
+        mbar_init(bar_v0 + 8, 1); mbar_init(bar_s, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 0) { __syncwarp(); tmem_alloc(tmem_slot, TMEM_COLS); }
+    __syncthreads();
+    if (tid == 0) {
+        mbar_expect_tx(bar_q, S::QTILE);
+#pragma unroll
+        for (int sb = 0; sb < SUB; ++sb) tma_load_3d(sQ + sb * 16384, &tmQ, sb * 64, i0, bh, bar_q);
+    }
 
-    // retained entries visible to this row: idx ascending => a prefix of length nvis
+    // ---- retained entries visible to this row: idx ascending => a prefix of length nvis.  The list is
+    // staged through shared memory 128 entries at a time and searched there.
     const int32_t* id = idx + (size_t)bh * R;
     const int n_ret = cnt[bh];
-    int nvis;
-    {
-        const int lim = min(i, Tlen - 1) - W;                  // entry visible iff idx <= lim
-        int lo = 0, hi = n_ret;
-        while (lo < hi) { const int mid = (lo + hi) >> 1; if (id[mid] <= lim) lo = mid + 1; else hi = mid; }
-        nvis = lo;
+    const int lim = min(i, Tlen - 1) - W;                      // entry visible iff idx <= lim
+    const int lim_max = i_hi - W;
+    int nvis = 0;
+    for (int e0 = 0; e0 < n_ret; e0 += 128) {
+        const int n_here = min(128, n_ret - e0);
+        __syncthreads();
+        if (tid < n_here) s_idx[tid] = id[e0 + tid];
+        __syncthreads();
+        if (s_idx[n_here - 1] <= lim) nvis += n_here;
+        else {
+            int lo = 0, hi = n_here;
+            while (lo < hi) { const int mid = (lo + hi) >> 1; if (s_idx[mid] <= lim) lo = mid + 1; else hi = mid; }
+            nvis += lo;
+        }
+        if (s_idx[n_here - 1] > lim_max) break;                // uniform: nothing further is visible to any row
     }
     if (i == i_hi) *s_nvmax = nvis;
     tc_fence_before();
@@ -172,79 +208,69 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     const int n_rt = (nv_max + BN - 1) / BN;
     const int n_tiles = n_win + n_rt;
 
-    // ---- loads ---------------------------------------------------------------------------------
-    auto issue_tile = [&](int t) {
+    // ---- loads: K and V of a tile are tracked separately (K runs two tiles ahead, V one) -----------------
+    auto issue_kv = [&](int t, bool is_v) {
+        if (t >= n_tiles) return;
         const int st = t & 1;
-        const uint32_t dK = sK + st * S::TILE, dV = sV + st * S::TILE;
+        const uint32_t dst = (is_v ? sV : sK) + st * S::KVTILE;
         if (t < n_win) {
             if (tid == 0) {
-                const uint32_t bar = bar_kv0 + 8 * st;
-                mbar_expect_tx(bar, 2 * S::TILE);
+                const uint32_t bar = (is_v ? bar_v0 : bar_k0) + 8 * st;
+                mbar_expect_tx(bar, S::KVTILE);
                 const int y = j_start + t * BN;
 #pragma unroll
-                for (int sb = 0; sb < SUB; ++sb) {
-                    tma_load_3d(dK + sb * 16384, &tmK, sb * 64, y, bh, bar);
-                    tma_load_3d(dV + sb * 16384, &tmV, sb * 64, y, bh, bar);
-                }
+                for (int sb = 0; sb < SUB; ++sb) tma_load_3d(dst + sb * 8192, is_v ? &tmV : &tmK, sb * 64, y, bh, bar);
             }
         } else {
-            // gather row e of the retained list into row `tid` of the stage (zero-filled past the visible prefix)
-            const int e = (t - n_win) * BN + tid;
+            // gather: two threads per row, each copies half of the row's 16-byte chunks
+            const int row = tid & 63, part = tid >> 6;
+            const int e = (t - n_win) * BN + row;
             const bool ok = e < nv_max;
-            const size_t row = ((size_t)bh * Tlen + (ok ? id[e] : 0)) * D;
-            const uint32_t nbytes = ok ? 16u : 0u;
+            const __nv_bfloat16* src = (is_v ? vg : kg) + ((size_t)bh * Tlen + (ok ? id[e] : 0)) * D;
+            const uint32_t nbytes = ok ? 16u : 0u;             // rows past the visible prefix are zero-filled
 #pragma unroll
-            for (int ch = 0; ch < D / 8; ++ch) {
-                const uint32_t off = (ch >> 3) * 16384 + tid * 128 + (((ch & 7) ^ (tid & 7)) << 4);
-                cp_async16(dK + off, kg + row + ch * 8, nbytes);
-                cp_async16(dV + off, vg + row + ch * 8, nbytes);
+            for (int c = 0; c < D / 16; ++c) {
+                const int ch = part * (D / 16) + c;
+                const uint32_t off = (ch >> 3) * 8192 + row * 128 + (((ch & 7) ^ (row & 7)) << 4);
+                cp_async16(dst + off, src + ch * 8, nbytes);
             }
         }
-        cp_async_commit();                                     // one group per tile (empty for TMA tiles)
     };
 
-    if (tid == 0) {
-        mbar_expect_tx(bar_q, S::TILE);
-#pragma unroll
-        for (int sb = 0; sb < SUB; ++sb) tma_load_3d(sQ + sb * 16384, &tmQ, sb * 64, i0, bh, bar_q);
-    }
-    issue_tile(0);
+    issue_kv(0, false); issue_kv(1, false); issue_kv(0, true);
+    cp_async_commit();
 
     constexpr uint32_t IDESC_S = instr_desc(BM, BN, false);
     constexpr uint32_t IDESC_O = instr_desc(BM, D, true);
-    const float c2 = scale * 1.4426950408889634f;              // logits are handled as s * scale * log2(e)
+    const float c2 = scale * 1.4426950408889634f;              // logits are handled in the log2 domain: x = s * c2
     const uint32_t lane_base = ((uint32_t)(warp * 32)) << 16;   // this warp's TMEM lanes
+    uint32_t k_phase = 0, v_phase = 0;                         // bit st = parity of that stage's TMA barrier
 
-    float acc[D];
+    auto mma_s = [&](int t) {                                  // thread 0 only
+        const int st = t & 1;
+        if (t < n_win) { mbar_wait(bar_k0 + 8 * st, (k_phase >> st) & 1u, 2); k_phase ^= 1u << st; }
+        const uint32_t kb = sK + st * S::KVTILE;
 #pragma unroll
-    for (int c = 0; c < D; ++c) acc[c] = 0.f;
-    float m_run = -INFINITY, l_run = 0.f;
-    uint32_t kv_phase = 0;                                     // bit st = parity of stage st's TMA barrier
+        for (int kk = 0; kk < D / 16; ++kk)
+            umma(tmem, smem_desc(sQ + (kk >> 2) * 16384 + (kk & 3) * 32, 16, 1024),
+                 smem_desc(kb + (kk >> 2) * 8192 + (kk & 3) * 32, 16, 1024), IDESC_S, kk > 0);
+        umma_commit(bar_s);
+    };
+
+    // first S: needs Q and K(0)
+    cp_async_wait<0>();
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    if (tid == 0) {
+        tc_fence_after();
+        mbar_wait(bar_q, 0, 1);
+        mma_s(0);
+    }
+
+    float m_run = -INFINITY, l_run = 0.f;                      // running max (log2 domain) and sum
 
     for (int t = 0; t < n_tiles; ++t) {
-        const int st = t & 1;
-        if (t + 1 < n_tiles) issue_tile(t + 1);
-        // ---- wait for tile t's operands
-        if (t + 1 < n_tiles) cp_async_wait<1>(); else cp_async_wait<0>();
-        if (t >= n_win) fence_proxy_async();
-        if (t == 0 && tid == 0) mbar_wait(bar_q, 0, 1);
-        if (t < n_win) {
-            if (tid == 0) mbar_wait(bar_kv0 + 8 * st, (kv_phase >> st) & 1u, 2);
-            kv_phase ^= 1u << st;
-        }
-        tc_fence_before();
-        __syncthreads();                                       // gathered rows visible; O-tile reads of tile t-1 done
-        // ---- S = Q K^T
-        if (tid == 0) {
-            tc_fence_after();
-            const uint32_t kb = sK + st * S::TILE;
-#pragma unroll
-            for (int kk = 0; kk < D / 16; ++kk) {
-                const uint32_t off = (kk >> 2) * 16384 + (kk & 3) * 32;
-                umma(tmem, smem_desc(sQ + off, 16, 1024), smem_desc(kb + off, 16, 1024), IDESC_S, kk > 0);
-            }
-            umma_commit(bar_s);
-        }
         // column range this row may see in the tile
         int c_lo, c_hi;
         if (t < n_win) {
@@ -255,95 +281,125 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             c_lo = 0;
             c_hi = nvis - (t - n_win) * BN - 1;
         }
-        mbar_wait(bar_s, t & 1, 3);
-        tc_fence_after();
+        // rows of a warp are consecutive: its union range is [c_lo of lane 0, c_hi of lane 31]
+        const int w_lo = __shfl_sync(0xffffffffu, c_lo, 0), w_hi = __shfl_sync(0xffffffffu, c_hi, 31);
+        bool act[2];
+#pragma unroll
+        for (int cb = 0; cb < 2; ++cb) act[cb] = cb * 32 <= w_hi && cb * 32 + 31 >= w_lo;
 
-        // ---- softmax over the row: pass 1 row max, pass 2 exponentials -> P (bf16, swizzled)
+        mbar_wait(bar_s, t & 1, 3);                            // S(t) is in TMEM; PV(t-1) has completed too
+        tc_fence_after();
+        issue_kv(t + 2, false); issue_kv(t + 1, true);
+        cp_async_commit();
+
+        uint32_t r[2][32];
+#pragma unroll
+        for (int cb = 0; cb < 2; ++cb)
+            if (act[cb]) tmem_ld32(tmem + lane_base + cb * 32, r[cb]);
+        tmem_wait_ld();
         float m_tile = -INFINITY;
 #pragma unroll
-        for (int cb = 0; cb < BN / 32; ++cb) {
-            uint32_t r[32];
-            tmem_ld32(tmem + lane_base + cb * 32, r);
-            tmem_wait_ld();
+        for (int cb = 0; cb < 2; ++cb) {
+            if (!act[cb]) continue;
 #pragma unroll
             for (int c = 0; c < 32; ++c) {
                 const int col = cb * 32 + c;
-                if (col >= c_lo && col <= c_hi) m_tile = fmaxf(m_tile, __uint_as_float(r[c]));
+                const float x = (col >= c_lo && col <= c_hi) ? __uint_as_float(r[cb][c]) * c2 : -INFINITY;
+                r[cb][c] = __float_as_uint(x);
+                m_tile = fmaxf(m_tile, x);
             }
         }
-        const float m_new = fmaxf(m_run, m_tile);
-        const float m_use = m_new == -INFINITY ? 0.f : m_new;
-        const float alpha = m_run == -INFINITY ? 0.f : fast_exp2((m_run - m_use) * c2);
-        const float mb = m_use * c2;
+        // lazy rescale: the running max only moves when the new one is far above it (exp2 arguments stay <= 8)
+        float alpha = 1.f;
+        bool need = false;
+        if (m_run == -INFINITY) m_run = m_tile;                 // nothing accumulated yet for this row: O row is 0
+        else if (m_tile > m_run + 8.f) { alpha = fast_exp2(m_run - m_tile); m_run = m_tile; need = true; }
+        if (__any_sync(0xffffffffu, need)) {
+#pragma unroll
+            for (int cb = 0; cb < D / 32; ++cb) {
+                uint32_t q4[32];
+                tmem_ld32(tmem + lane_base + O_COL + cb * 32, q4);
+                tmem_wait_ld();
+#pragma unroll
+                for (int c = 0; c < 32; ++c) q4[c] = __float_as_uint(__uint_as_float(q4[c]) * alpha);
+                tmem_st32(tmem + lane_base + O_COL + cb * 32, q4);
+            }
+            tmem_wait_st();
+            l_run *= alpha;
+        }
+        const float m_use = m_run == -INFINITY ? 0.f : m_run;
         float l_tile = 0.f;
 #pragma unroll
-        for (int cb = 0; cb < BN / 32; ++cb) {
-            uint32_t r[32];
-            tmem_ld32(tmem + lane_base + cb * 32, r);
-            tmem_wait_ld();
+        for (int cb = 0; cb < 2; ++cb) {
             uint32_t pk[16];
+            if (act[cb]) {
 #pragma unroll
-            for (int c = 0; c < 32; c += 2) {
-                const int col = cb * 32 + c;
-                float p0 = (col >= c_lo && col <= c_hi) ? fast_exp2(fmaf(__uint_as_float(r[c]), c2, -mb)) : 0.f;
-                float p1 = (col + 1 >= c_lo && col + 1 <= c_hi) ? fast_exp2(fmaf(__uint_as_float(r[c + 1]), c2, -mb)) : 0.f;
-                __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
-                // the row sum uses the rounded probabilities, i.e. exactly what the PV product consumes
-                l_tile += __low2float(h) + __high2float(h);
-                pk[c >> 1] = *reinterpret_cast<uint32_t*>(&h);
+                for (int c = 0; c < 32; c += 2) {
+                    const float p0 = fast_exp2(__uint_as_float(r[cb][c]) - m_use);       // exp2(-inf) = 0 when masked
+                    const float p1 = fast_exp2(__uint_as_float(r[cb][c + 1]) - m_use);
+                    __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
+                    // the row sum uses the rounded probabilities, i.e. exactly what the PV product consumes
+                    l_tile += __low2float(h) + __high2float(h);
+                    pk[c >> 1] = *reinterpret_cast<uint32_t*>(&h);
+                }
+            } else {
+#pragma unroll
+                for (int c = 0; c < 16; ++c) pk[c] = 0u;
             }
-            // 32 columns = 4 chunks of 16 bytes; column block cb lives in sub-tile cb/2, chunks (cb&1)*4 ..
 #pragma unroll
             for (int g = 0; g < 4; ++g) {
-                const int ch = (cb & 1) * 4 + g;
-                const uint32_t dst = sP + (cb >> 1) * 16384 + tid * 128 + ((ch ^ (tid & 7)) << 4);
+                const int ch = cb * 4 + g;
+                const uint32_t dst = sP + tid * 128 + ((ch ^ (tid & 7)) << 4);
                 asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(pk[4 * g]), "r"(pk[4 * g + 1]),
                              "r"(pk[4 * g + 2]), "r"(pk[4 * g + 3]) : "memory");
             }
         }
-        l_run = l_run * alpha + l_tile;
-        m_run = m_new;
-        fence_proxy_async();                                   // P (generic proxy) -> visible to the MMA (async proxy)
+        l_run += l_tile;
+
+        cp_async_wait<1>();                                    // gathered K(t+1), V(t) have landed
+        fence_proxy_async();                                   // P and gathered rows -> visible to the MMA proxy
         tc_fence_before();
         __syncthreads();
-        // ---- O_tile = P V
         if (tid == 0) {
             tc_fence_after();
-            const uint32_t vb = sV + st * S::TILE;
+            const int st = t & 1;
+            if (t < n_win) { mbar_wait(bar_v0 + 8 * st, (v_phase >> st) & 1u, 4); v_phase ^= 1u << st; }
+            const uint32_t vb = sV + st * S::KVTILE;
 #pragma unroll
-            for (int kk = 0; kk < BN / 16; ++kk) {
-                const uint32_t aoff = (kk >> 2) * 16384 + (kk & 3) * 32;
-                umma(tmem + 128, smem_desc(sP + aoff, 16, 1024), smem_desc(vb + kk * 2048, 16384, 1024), IDESC_O, kk > 0);
-            }
-            umma_commit(bar_o);
-        }
-        mbar_wait(bar_o, t & 1, 4);
-        tc_fence_after();
-#pragma unroll
-        for (int cb = 0; cb < D / 32; ++cb) {
-            uint32_t r[32];
-            tmem_ld32(tmem + lane_base + 128 + cb * 32, r);
-            tmem_wait_ld();
-#pragma unroll
-            for (int c = 0; c < 32; ++c) acc[cb * 32 + c] = fmaf(acc[cb * 32 + c], alpha, __uint_as_float(r[c]));
+            for (int kk = 0; kk < BN / 16; ++kk)
+                umma(tmem + O_COL, smem_desc(sP + kk * 32, 16, 1024), smem_desc(vb + kk * 2048, 8192, 1024), IDESC_O,
+                     (t > 0 || kk > 0) ? 1u : 0u);
+            if (t + 1 < n_tiles) mma_s(t + 1);
+            else umma_commit(bar_s);                           // final: signals that the last PV is done
         }
     }
+    mbar_wait(bar_s, n_tiles & 1, 5);
+    tc_fence_after();
 
-    // ---- epilogue ------------------------------------------------------------------------------
-    if (i < Tlen) {
+    // ---- epilogue: O / l -> bf16, logsumexp --------------------------------------------------------------
+    {
         const float inv = 1.f / l_run;
         __nv_bfloat16* orow = o + ((size_t)bh * Tlen + i) * D;
 #pragma unroll
-        for (int c = 0; c < D; c += 8) {
-            uint32_t w4[4];
+        for (int cb = 0; cb < D / 32; ++cb) {
+            uint32_t q4[32];
+            tmem_ld32(tmem + lane_base + O_COL + cb * 32, q4);
+            tmem_wait_ld();
+            if (i < Tlen) {
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                __nv_bfloat162 h = __floats2bfloat162_rn(acc[c + 2 * u] * inv, acc[c + 2 * u + 1] * inv);
-                w4[u] = *reinterpret_cast<uint32_t*>(&h);
+                for (int c = 0; c < 32; c += 8) {
+                    uint32_t w4[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(q4[c + 2 * u]) * inv,
+                                                                 __uint_as_float(q4[c + 2 * u + 1]) * inv);
+                        w4[u] = *reinterpret_cast<uint32_t*>(&h);
+                    }
+                    *reinterpret_cast<uint4*>(orow + cb * 32 + c) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+                }
             }
-            *reinterpret_cast<uint4*>(orow + c) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
         }
-        lse[(size_t)bh * Tlen + i] = m_run * scale + logf(l_run);
+        if (i < Tlen) lse[(size_t)bh * Tlen + i] = m_run * 0.6931471805599453f + logf(l_run);
     }
     tc_fence_before();
     __syncthreads();
@@ -368,14 +424,14 @@ EncodeTiledFn encode_fn()
     return fn;
 }
 
-// [B*H][T][d] bf16 viewed as a 3-D tensor (d fastest); box = 64 columns x 128 rows, 128-byte swizzle.
-bool make_map(CUtensorMap* m, const void* ptr, int BH, int T, int d)
+// [B*H][T][d] bf16 viewed as a 3-D tensor (d fastest); box = 64 columns x box_rows rows, 128-byte swizzle.
+bool make_map(CUtensorMap* m, const void* ptr, int BH, int T, int d, int box_rows)
 {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)T, (cuuint64_t)BH};
     cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)T * d * 2};
-    cuuint32_t box[3] = {64, 128, 1};
+    cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
     cuuint32_t estr[3] = {1, 1, 1};
     return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -388,7 +444,7 @@ int run(const Params& p, const void* q, const void* k, const void* v, const int3
 {
     CUtensorMap tq, tk, tv;
     const int BH = p.B * p.H;
-    if (!make_map(&tq, q, BH, p.T, D) || !make_map(&tk, k, BH, p.T, D) || !make_map(&tv, v, BH, p.T, D))
+    if (!make_map(&tq, q, BH, p.T, D, BM) || !make_map(&tk, k, BH, p.T, D, BN) || !make_map(&tv, v, BH, p.T, D, BN))
         return LTE_ERR_CUDA;
     static bool attr_done = false;
     if (!attr_done) {
