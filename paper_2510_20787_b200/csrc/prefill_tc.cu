@@ -20,6 +20,13 @@ namespace lte {
 
 __device__ int g_prefill_status = 0;          // 0 = fine; otherwise the code of the wait that gave up
 
+#ifdef LTE_PROFILE
+__device__ long long g_prof[64];
+#define PROF(slot) do { if (blockIdx.x == 5 && blockIdx.y == 3 && threadIdx.x == 64) g_prof[slot] = clock64(); } while (0)
+#else
+#define PROF(slot) do { } while (0)
+#endif
+
 namespace {
 
 constexpr int BM = 128, BN = 64, NTHREADS = 128;
@@ -150,6 +157,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         if (threadIdx.x == 0) atomicExch(&g_prefill_status, 9);
         return;
     }
+    PROF(0);
     const uint32_t sQ = base + S::OFF_Q, sK = base + S::OFF_K, sV = base + S::OFF_V, sP = base + S::OFF_P;
     const uint32_t bar_q = base + S::OFF_BAR, bar_k0 = bar_q + 8, bar_v0 = bar_q + 24, bar_s = bar_q + 40;
     const uint32_t tmem_slot = bar_q + 48;
@@ -176,6 +184,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         for (int sb = 0; sb < SUB; ++sb) tma_load_3d(sQ + sb * 16384, &tmQ, sb * 64, i0, bh, bar_q);
     }
 
+    PROF(1);
     // ---- retained entries visible to this row: idx ascending => a prefix of length nvis.  The list is
     // staged through shared memory 128 entries at a time and searched there.
     const int32_t* id = idx + (size_t)bh * R;
@@ -202,6 +211,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     tc_fence_after();
     const uint32_t tmem = *tmem_slot_gen;
     const int nv_max = *s_nvmax;
+    PROF(2);
 
     const int j_start = max(i0 - W + 1, 0);
     const int n_win = (i_hi - j_start + 1 + BN - 1) / BN;
@@ -268,6 +278,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         mma_s(0);
     }
 
+    PROF(3);
     float m_run = -INFINITY, l_run = 0.f;                      // running max (log2 domain) and sum
 
     for (int t = 0; t < n_tiles; ++t) {
@@ -281,34 +292,54 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             c_lo = 0;
             c_hi = nvis - (t - n_win) * BN - 1;
         }
-        // rows of a warp are consecutive: its union range is [c_lo of lane 0, c_hi of lane 31]
-        const int w_lo = __shfl_sync(0xffffffffu, c_lo, 0), w_hi = __shfl_sync(0xffffffffu, c_hi, 31);
-        bool act[2];
+        // rows of a warp are consecutive and both bounds grow with the row: lane 0 / lane 31 give the warp's
+        // union range (columns any row sees) and intersection range (columns every row sees)
+        const int u_lo = __shfl_sync(0xffffffffu, c_lo, 0), u_hi = __shfl_sync(0xffffffffu, c_hi, 31);
+        const int n_lo = __shfl_sync(0xffffffffu, c_lo, 31), n_hi = __shfl_sync(0xffffffffu, c_hi, 0);
+        bool act[2], full[2];
+        uint32_t vm[2];                                        // per-thread validity bits of a partial chunk
 #pragma unroll
-        for (int cb = 0; cb < 2; ++cb) act[cb] = cb * 32 <= w_hi && cb * 32 + 31 >= w_lo;
+        for (int cb = 0; cb < 2; ++cb) {
+            const int lo = cb * 32, hi = lo + 31;
+            act[cb] = lo <= u_hi && hi >= u_lo;
+            full[cb] = lo >= n_lo && hi <= n_hi;
+            const int a = min(max(c_lo - lo, 0), 32), b = min(max(c_hi - lo + 1, 0), 32);
+            const uint32_t below_b = b >= 32 ? 0xffffffffu : ((1u << b) - 1u);
+            const uint32_t below_a = a >= 32 ? 0xffffffffu : ((1u << a) - 1u);
+            vm[cb] = b > a ? (below_b & ~below_a) : 0u;
+        }
 
+        PROF(4 + 6 * t);
         mbar_wait(bar_s, t & 1, 3);                            // S(t) is in TMEM; PV(t-1) has completed too
         tc_fence_after();
+        PROF(5 + 6 * t);
         issue_kv(t + 2, false); issue_kv(t + 1, true);
         cp_async_commit();
+        PROF(6 + 6 * t);
 
         uint32_t r[2][32];
 #pragma unroll
         for (int cb = 0; cb < 2; ++cb)
             if (act[cb]) tmem_ld32(tmem + lane_base + cb * 32, r[cb]);
         tmem_wait_ld();
-        float m_tile = -INFINITY;
+        PROF(7 + 6 * t);
+        float m_raw = -INFINITY;                               // row max of the raw logits (scale applied after)
 #pragma unroll
         for (int cb = 0; cb < 2; ++cb) {
             if (!act[cb]) continue;
+            if (full[cb]) {
 #pragma unroll
-            for (int c = 0; c < 32; ++c) {
-                const int col = cb * 32 + c;
-                const float x = (col >= c_lo && col <= c_hi) ? __uint_as_float(r[cb][c]) * c2 : -INFINITY;
-                r[cb][c] = __float_as_uint(x);
-                m_tile = fmaxf(m_tile, x);
+                for (int c = 0; c < 32; ++c) m_raw = fmaxf(m_raw, __uint_as_float(r[cb][c]));
+            } else {
+#pragma unroll
+                for (int c = 0; c < 32; ++c) {
+                    const float x = (vm[cb] & (1u << c)) ? __uint_as_float(r[cb][c]) : -INFINITY;
+                    r[cb][c] = __float_as_uint(x);
+                    m_raw = fmaxf(m_raw, x);
+                }
             }
         }
+        const float m_tile = m_raw * c2;
         // lazy rescale: the running max only moves when the new one is far above it (exp2 arguments stay <= 8)
         float alpha = 1.f;
         bool need = false;
@@ -327,7 +358,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             tmem_wait_st();
             l_run *= alpha;
         }
-        const float m_use = m_run == -INFINITY ? 0.f : m_run;
+        const float neg_m = m_run == -INFINITY ? 0.f : -m_run;
         float l_tile = 0.f;
 #pragma unroll
         for (int cb = 0; cb < 2; ++cb) {
@@ -335,11 +366,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             if (act[cb]) {
 #pragma unroll
                 for (int c = 0; c < 32; c += 2) {
-                    const float p0 = fast_exp2(__uint_as_float(r[cb][c]) - m_use);       // exp2(-inf) = 0 when masked
-                    const float p1 = fast_exp2(__uint_as_float(r[cb][c + 1]) - m_use);
+                    // masked entries hold -inf: fma gives -inf and exp2(-inf) = 0
+                    const float p0 = fast_exp2(fmaf(__uint_as_float(r[cb][c]), c2, neg_m));
+                    const float p1 = fast_exp2(fmaf(__uint_as_float(r[cb][c + 1]), c2, neg_m));
+                    l_tile += p0 + p1;
                     __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
-                    // the row sum uses the rounded probabilities, i.e. exactly what the PV product consumes
-                    l_tile += __low2float(h) + __high2float(h);
                     pk[c >> 1] = *reinterpret_cast<uint32_t*>(&h);
                 }
             } else {
@@ -355,11 +386,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             }
         }
         l_run += l_tile;
+        PROF(8 + 6 * t);
 
         cp_async_wait<1>();                                    // gathered K(t+1), V(t) have landed
         fence_proxy_async();                                   // P and gathered rows -> visible to the MMA proxy
         tc_fence_before();
         __syncthreads();
+        PROF(9 + 6 * t);
         if (tid == 0) {
             tc_fence_after();
             const int st = t & 1;
@@ -373,8 +406,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             else umma_commit(bar_s);                           // final: signals that the last PV is done
         }
     }
+    PROF(50);
     mbar_wait(bar_s, n_tiles & 1, 5);
     tc_fence_after();
+    PROF(51);
 
     // ---- epilogue: O / l -> bf16, logsumexp --------------------------------------------------------------
     {
@@ -401,6 +436,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         }
         if (i < Tlen) lse[(size_t)bh * Tlen + i] = m_run * 0.6931471805599453f + logf(l_run);
     }
+    PROF(52);
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, TMEM_COLS);
@@ -471,6 +507,10 @@ int launch_prefill_tc(const Params& p, const void* q, const void* k, const void*
     }
     return launch_prefill_simt(p, q, k, v, idx, cnt, o, lse, st);   // d = 32: rows too narrow for the 128-byte swizzle
 }
+
+#ifdef LTE_PROFILE
+extern "C" int lte_prof_read(long long* out) { return cudaMemcpyFromSymbol(out, g_prof, sizeof(long long) * 64) == cudaSuccess ? 0 : -1; }
+#endif
 
 int prefill_status_fetch_and_clear()
 {
