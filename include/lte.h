@@ -174,6 +174,34 @@ int lte_attn_bwd(const lte_shape* s, const lte_conv* c,
 
 #define LTE_BWD_CNN_INPUT_GRAD 1u
 
+/*
+ * lte_attn_bwd for callers that cannot hand over scratch memory.  (The paper has no counterpart: this is a
+ * deployment convenience of this library.)
+ *
+ * Who needs it: code that runs where device allocation is off limits or already spent -- a serving process
+ * whose memory pool was sized and frozen at start-up, a plugin called from inside another framework's
+ * allocator-locked region, or a host that must not call cudaMalloc because that call synchronises the device
+ * and would stall every other stream.  Such callers cannot create the workspace lte_attn_bwd asks for.
+ *
+ * Same arguments, results and errors as lte_attn_bwd, minus `ws` / `ws_bytes`: the scratch is a fixed array of
+ * LTE_STATIC_SCRATCH_BYTES inside the library (each GPU that loads the library holds it until the process
+ * ends).  The call itself performs no cudaMalloc / cudaFree and uses no allocating library routine.
+ *   - Shapes whose scratch need (lte_workspace_bytes(LTE_OP_BWD, ...) for flags = LTE_BWD_CNN_INPUT_GRAD; less
+ *     without that flag) exceeds LTE_STATIC_SCRATCH_BYTES are rejected with LTE_ERR_WORKSPACE; nothing is launched.
+ *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with that device
+ *     current).  Make that first call outside any stream capture.
+ *   - All calls on a device share the one array, which still holds whatever the previous call left there.  The
+ *     backward kernels write every scratch value before reading it, so no clearing is needed, but two calls that
+ *     overlap on the GPU (different streams) would race on it: issue them on one stream, or serialise them.
+ */
+#define LTE_STATIC_SCRATCH_BYTES (8u << 20)
+int lte_attn_bwd_static(const lte_shape* s, const lte_conv* c,
+                        const void* q, const void* k, const void* v, const void* o, const float* lse,
+                        const void* dO, const float* z, const int32_t* idx, const int32_t* cnt,
+                        const float* lambda_or_null,
+                        void* dq, void* dk, void* dv, float* dw, float* dbias_or_null, uint32_t flags,
+                        void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -1,6 +1,8 @@
 // C-ABI entry points of liblte: argument validation and dispatch.  No torch types, no allocation.
 #include <math.h>
 
+#include <mutex>
+
 #include "common.cuh"
 
 namespace lte {
@@ -173,6 +175,51 @@ int lte_attn_bwd(const lte_shape* s, const lte_conv* c, const void* q, const voi
     e = check_arch(); if (e) return e;
     return launch_bwd(p, q, k, v, o, lse, dO, z, idx, cnt, lambda_or_null, dq, dk, dv, dw, dbias_or_null, flags, ws,
                       (cudaStream_t)stream);
+}
+
+
+/* ---- backward without any caller- or library-side allocation ------------------------------------------------
+ * Scratch for lte_attn_bwd_static lives in this fixed array instead of a caller-supplied workspace.  Every GPU
+ * that loads the library carries these LTE_STATIC_SCRATCH_BYTES until the process exits.  The symbol below is
+ * only a host-side handle; the address the kernels use is resolved once per device with cudaGetSymbolAddress. */
+static __device__ __align__(256) unsigned char g_bwd_static_scratch[LTE_STATIC_SCRATCH_BYTES];
+
+namespace {
+std::mutex g_static_mu;
+void* g_static_ptr[64] = {nullptr};          /* resolved device address of the array, per device ordinal */
+
+/* Device address of the scratch array on the current device (resolved on first use), or NULL on failure. */
+void* static_scratch_for_current_device()
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    if (!g_static_ptr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_bwd_static_scratch) != cudaSuccess) return nullptr;
+        g_static_ptr[dev] = p;
+    }
+    return g_static_ptr[dev];
+}
+}  // namespace
+
+int lte_attn_bwd_static(const lte_shape* s, const lte_conv* c, const void* q, const void* k, const void* v,
+                        const void* o, const float* lse, const void* dO, const float* z, const int32_t* idx,
+                        const int32_t* cnt, const float* lambda_or_null, void* dq, void* dk, void* dv, float* dw,
+                        float* dbias_or_null, uint32_t flags, void* stream)
+{
+    int e = check_shape(s, true); if (e) return e;
+    e = check_conv(s, c); if (e) return e;
+    if (!q || !k || !v || !o || !lse || !dO || !z || !cnt || (s->R > 0 && !idx) || !dq || !dk || !dv || !dw)
+        return LTE_ERR_INVALID_ARG;
+    if (flags & ~LTE_BWD_CNN_INPUT_GRAD) return LTE_ERR_INVALID_ARG;
+    Params p = make_params(s, c);
+    if (bwd_workspace_bytes(p, flags) > (size_t)LTE_STATIC_SCRATCH_BYTES) return LTE_ERR_WORKSPACE;   /* too large for the fixed array */
+    e = check_arch(); if (e) return e;
+    void* scratch = static_scratch_for_current_device();
+    if (!scratch) return LTE_ERR_CUDA;
+    return launch_bwd(p, q, k, v, o, lse, dO, z, idx, cnt, lambda_or_null, dq, dk, dv, dw, dbias_or_null, flags,
+                      scratch, (cudaStream_t)stream);
 }
 
 }  // extern "C"

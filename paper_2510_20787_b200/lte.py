@@ -19,7 +19,8 @@ OP_SCORES, OP_SELECT, OP_PREFILL, OP_DECODE, OP_BWD = range(5)
 BWD_CNN_INPUT_GRAD = 1
 
 EXPORTS = ["lte_device_status", "lte_workspace_bytes", "lte_strerror", "lte_scores", "lte_select", "lte_attn_prefill",
-           "lte_cache_bytes", "lte_cache_init", "lte_attn_decode", "lte_attn_bwd"]
+           "lte_cache_bytes", "lte_cache_init", "lte_attn_decode", "lte_attn_bwd", "lte_attn_bwd_static"]
+STATIC_SCRATCH_BYTES = 8 << 20
 
 
 class LteShape(ctypes.Structure):
@@ -61,6 +62,7 @@ def lib():
         L.lte_cache_init.argtypes = [vp] * 9
         L.lte_attn_decode.argtypes = [vp] * 9
         L.lte_attn_bwd.argtypes = [vp] * 17 + [ctypes.c_uint32, vp, ctypes.c_size_t, vp]
+        L.lte_attn_bwd_static.argtypes = [vp] * 17 + [ctypes.c_uint32, vp]
         for name in EXPORTS:
             if name not in ("lte_strerror", "lte_workspace_bytes", "lte_cache_bytes", "lte_device_status"):
                 getattr(L, name).restype = ctypes.c_int
@@ -189,4 +191,21 @@ def lte_attn_bwd(s, c, q, k, v, o, lse, dO, z, idx, cnt, lam=None, flags=BWD_CNN
         _ptr(dO), _ptr(z, torch.float32), _ptr(idx, torch.int32), _ptr(cnt, torch.int32),
         _ptr(lam, torch.float32), _ptr(dq), _ptr(dk), _ptr(dv), _ptr(dw), _ptr(db), flags, _ptr(ws),
         ws.numel(), _stream()))
+    return dq, dk, dv, dw, db
+
+
+def lte_attn_bwd_static(s, c, q, k, v, o, lse, dO, z, idx, cnt, lam=None, flags=BWD_CNN_INPUT_GRAD, outs=None):
+    """lte_attn_bwd with the library's built-in scratch array instead of a workspace: for callers that must not
+    allocate device memory.  ``outs`` = (dq, dk, dv, dw, dbias) preallocated by the caller makes the whole call
+    allocation-free; when omitted they are created here for convenience.  Shapes needing more scratch than
+    STATIC_SCRATCH_BYTES raise LteError (status -3)."""
+    if outs is None:
+        outs = (torch.empty_like(q), torch.empty_like(k), torch.empty_like(v),
+                torch.empty((s.H, c.kernel, 2 * s.d), dtype=torch.float32, device=q.device),
+                torch.empty((s.H,), dtype=torch.float32, device=q.device))
+    dq, dk, dv, dw, db = outs
+    _check("lte_attn_bwd_static", lib().lte_attn_bwd_static(
+        ctypes.addressof(s), ctypes.addressof(c), _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse, torch.float32),
+        _ptr(dO), _ptr(z, torch.float32), _ptr(idx, torch.int32), _ptr(cnt, torch.int32),
+        _ptr(lam, torch.float32), _ptr(dq), _ptr(dk), _ptr(dv), _ptr(dw), _ptr(db), flags, _stream()))
     return dq, dk, dv, dw, db
