@@ -277,6 +277,346 @@ __global__ void __launch_bounds__(DT) decode_kernel(unsigned char* __restrict__ 
     }
 }
 
+// ---- fast path: persistent blocks that stream whole per-head cache blocks through shared memory ------------
+// The block of one (b,h) is contiguous in HBM, so three cp.async.bulk copies (TMA, 1-D; mbarrier transaction
+// counts) bring its keys, its values and its small tail (logits, pool positions, counters) on chip.  Each CTA
+// walks a contiguous range of heads and keeps the copy engine busy: as soon as the logits of head i are done its
+// key buffer is refilled with head i+1's keys, and after the PV pass the value buffer is refilled likewise, so
+// the loads of the next head run under the softmax / PV / write-back of the current one.  Everything is computed
+// out of shared memory; only the rows that change go back to HBM.  Used when a block fits (it does at W+R = 256).
+__device__ int g_decode_status = 0;
+#ifdef LTE_PROFILE
+__device__ long long g_dprof[64];
+#define DPROF(slot) do { if (blockIdx.x == 7 && threadIdx.x == 96 && it == 2) g_dprof[slot] = clock64(); } while (0)
+#else
+#define DPROF(slot) do { } while (0)
+#endif
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+// Bounded wait; false if it ran out (the caller records it and leaves).
+__device__ __forceinline__ bool bar_wait(uint32_t bar, uint32_t parity) {
+    for (uint32_t it = 0; it < (1u << 22); ++it) {
+        uint32_t r;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(r) : "r"(bar), "r"(parity) : "memory");
+        if (r) return true;
+    }
+    return false;
+}
+
+struct BulkSmem {
+    uint32_t kv_bytes, tail_bytes, off_v, off_tail, off_log, off_bar, total;
+};
+__host__ __device__ inline BulkSmem bulk_smem_plan(const CacheLayout& L, int W, int R) {
+    BulkSmem b;
+    b.kv_bytes = (uint32_t)L.off_v;                      // bytes of the K rows (= bytes of the V rows)
+    b.tail_bytes = (uint32_t)(L.stride - L.off_z);       // logits, pool positions, counters, padding
+    b.off_v = b.kv_bytes;
+    b.off_tail = 2 * b.kv_bytes;                         // two tail buffers
+    b.off_log = b.off_tail + 2 * b.tail_bytes;
+    b.off_bar = b.off_log + (uint32_t)(((size_t)W + R + 1) * 4 + 15) / 16 * 16;
+    b.total = b.off_bar + 64;
+    return b;
+}
+
+template <typename T, int D>
+__global__ void __launch_bounds__(DT) decode_bulk_kernel(unsigned char* __restrict__ cache, CacheLayout L,
+                                                         const T* __restrict__ q1, const T* __restrict__ k1,
+                                                         const T* __restrict__ v1, T* __restrict__ o1,
+                                                         float* __restrict__ lse1, const float* __restrict__ cw,
+                                                         const float* __restrict__ cbias, int BH, int per_cta, int H,
+                                                         int W, int R, int sink, int K, float zthr, float scale)
+{
+    constexpr int EPV = V16<T>::N;
+    constexpr int LPR = D / EPV;
+    constexpr int RPP = DT / LPR;
+    constexpr int CPL = D / 32;                // channels per lane in the warp-per-row pieces
+    extern __shared__ __align__(128) unsigned char dsm[];
+    const BulkSmem P = bulk_smem_plan(L, W, R);
+    const int rows = W + R;
+    float* s_log = reinterpret_cast<float*>(dsm + P.off_log);
+    const uint32_t bar_k = smem_addr(dsm + P.off_bar), bar_v = bar_k + 8, bar_t0 = bar_k + 16;   // bar_t0, bar_t0 + 8
+    __shared__ float s_red[DT / 32][D];
+    __shared__ float s_part[DT / 32];
+    __shared__ float s_tap[kMaxTaps];
+    __shared__ float s_sum[DT / 32];
+    __shared__ int s_flag;
+
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const int seg = tid % LPR, rsub = tid / LPR;
+    const int half = K / 2;
+    const int bh_begin = blockIdx.x * per_cta;
+    const int bh_end = min(bh_begin + per_cta, BH);
+    if (bh_begin >= bh_end) return;
+    const uint32_t sK = smem_addr(dsm), sV = sK + P.off_v, sT = sK + P.off_tail;
+
+    if (tid == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_k));
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_v));
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_t0));
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_t0 + 8));
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        const unsigned char* g0 = cache + L.header + (size_t)bh_begin * L.stride;
+        bulk_load(sT, g0 + L.off_z, P.tail_bytes, bar_t0);
+        bulk_load(sK, g0 + L.off_k, P.kv_bytes, bar_k);
+        bulk_load(sV, g0 + L.off_v, P.kv_bytes, bar_v);
+    }
+    __syncthreads();                                            // barriers initialised before anyone polls them
+
+    // The step's own inputs of a head (query, new key/value, scorer weights) are fetched one head ahead, so
+    // their latency hides under the previous head's tail.
+    float qf[EPV], k1f[CPL], v1f[CPL], q1f[CPL], wk[2][CPL], wv[2][CPL], bias = 0.f, v1_mine = 0.f;
+    uint4 kv_new = make_uint4(0, 0, 0, 0);
+    auto fetch_inputs = [&](int bh) {
+        const int h = bh % H;
+        uint4 u = *reinterpret_cast<const uint4*>(q1 + (size_t)bh * D + seg * EPV);
+        unpack<T>(u, qf);
+#pragma unroll
+        for (int c = 0; c < CPL; ++c) {
+            k1f[c] = to_f(k1[(size_t)bh * D + lane + 32 * c]);
+            v1f[c] = to_f(v1[(size_t)bh * D + lane + 32 * c]);
+            q1f[c] = to_f(q1[(size_t)bh * D + lane + 32 * c]);
+        }
+#pragma unroll
+        for (int u2 = 0; u2 < 2; ++u2) {
+            const int t = wid + u2 * (DT / 32);
+#pragma unroll
+            for (int c = 0; c < CPL; ++c) {
+                wk[u2][c] = t < K ? cw[((size_t)h * K + t) * 2 * D + lane + 32 * c] : 0.f;
+                wv[u2][c] = t < K ? cw[((size_t)h * K + t) * 2 * D + D + lane + 32 * c] : 0.f;
+            }
+        }
+        bias = cbias ? cbias[h] : 0.f;
+        if (tid < D) v1_mine = to_f(v1[(size_t)bh * D + tid]);
+        if (tid >= 64 && tid < 64 + 2 * LPR) {
+            const int t2 = tid - 64;
+            kv_new = *reinterpret_cast<const uint4*>((t2 < LPR ? k1 : v1) + (size_t)bh * D + (t2 % LPR) * EPV);
+        }
+    };
+    fetch_inputs(bh_begin);
+
+    for (int bh = bh_begin, it = 0; bh < bh_end; ++bh, ++it) {
+        DPROF(0);
+        const int tb = it & 1;
+        unsigned char* gblk = cache + L.header + (size_t)bh * L.stride;
+        // one thread polls the copy barriers; the block barrier then releases everybody
+        if (tid == 0) {
+            const bool ok = bar_wait(bar_t0 + 8 * tb, (it >> 1) & 1) && bar_wait(bar_k, it & 1) && bar_wait(bar_v, it & 1);
+            s_flag = ok ? 0 : 1;
+        }
+        __syncthreads();
+        if (s_flag) {                                           // bounded wait ran out: give up, outputs undefined
+            if (tid == 0) atomicExch(&g_decode_status, 1);
+            return;
+        }
+        DPROF(1);
+        const uint4* Kc = reinterpret_cast<const uint4*>(dsm);
+        const uint4* Vc = reinterpret_cast<const uint4*>(dsm + P.off_v);
+        const unsigned char* tail = dsm + P.off_tail + (size_t)tb * P.tail_bytes;
+        const float* zc = reinterpret_cast<const float*>(tail);
+        const int32_t* pidx = reinterpret_cast<const int32_t*>(tail + (L.off_pidx - L.off_z));
+        const int32_t* meta = reinterpret_cast<const int32_t*>(tail + (L.off_meta - L.off_z));
+        const int n = meta[0], cnt_old = meta[1];
+        const int slot = n % W;
+
+        // ---- pool decision, taken redundantly by every warp so that the row masks are known before the logits --
+        int dst = -1, cnt_new = cnt_old;
+        {
+            const int p = n - W;
+            if (p >= 0 && R > 0) {
+                const float zp = zc[slot];
+                const bool is_sink = p < sink;
+                if (is_sink || zp > zthr) {
+                    if (cnt_old < R) { dst = cnt_old; cnt_new = cnt_old + 1; }
+                    else if (!is_sink) {
+                        // worst entry: lowest logit, the youngest among equals, never a sink entry
+                        float wz = INFINITY; int wpos = -1, wslot = -1;
+                        for (int m = lane; m < cnt_old; m += 32) {
+                            const int pos = pidx[m];
+                            const float zm = zc[W + m];
+                            if (pos >= sink && (zm < wz || (zm == wz && pos > wpos))) { wz = zm; wpos = pos; wslot = m; }
+                        }
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) {
+                            const float oz = __shfl_xor_sync(0xffffffffu, wz, o);
+                            const int op = __shfl_xor_sync(0xffffffffu, wpos, o);
+                            const int os = __shfl_xor_sync(0xffffffffu, wslot, o);
+                            if (os >= 0 && (wslot < 0 || oz < wz || (oz == wz && op > wpos))) { wz = oz; wpos = op; wslot = os; }
+                        }
+                        if (wslot >= 0 && zp > wz) dst = wslot;
+                    }
+                }
+            }
+        }
+        DPROF(2);
+        // ---- scorer taps (warp w owns taps w and w + 8) and the logit of the incoming token (last warp) ----
+        const int jsc = n - half;
+        if (jsc >= 0) {
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                const int t = wid + u * (DT / 32);
+                if (t >= K) continue;
+                const int pos = jsc + t - half;
+                float a = 0.f;
+                if (pos == n) {
+#pragma unroll
+                    for (int c = 0; c < CPL; ++c) a += wk[u][c] * k1f[c] + wv[u][c] * v1f[c];
+                } else if (pos >= 0) {
+                    const T* kr = reinterpret_cast<const T*>(dsm) + (size_t)(pos % W) * D;
+                    const T* vr = reinterpret_cast<const T*>(dsm + P.off_v) + (size_t)(pos % W) * D;
+#pragma unroll
+                    for (int c = 0; c < CPL; ++c) a += wk[u][c] * to_f(kr[lane + 32 * c]) + wv[u][c] * to_f(vr[lane + 32 * c]);
+                }
+                a = warp_sum(a);
+                if (lane == 0) s_tap[t] = a;
+            }
+        }
+        float m_loc = -INFINITY;
+        if (wid == DT / 32 - 1) {
+            float s = 0.f;
+#pragma unroll
+            for (int c = 0; c < CPL; ++c) s = fmaf(q1f[c], k1f[c], s);
+            s = warp_sum(s) * scale;
+            if (lane == 0) s_log[rows] = s;
+            m_loc = s;
+        }
+        DPROF(3);
+        // ---- logits of every cached row, masked, with the running max ---------------------------------------
+        // Old ring row r holds the token at slot r; valid window rows are tokens n-W+1 .. n-1.  The popped row (slot)
+        // stays in the sum iff it was accepted into the pool.  Old pool row m: valid iff m < cnt_old and m != dst.
+        for (int r0 = 0; r0 < rows; r0 += 4 * RPP) {            // uniform trip count: the shuffles need every lane
+            float sv[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int row = r0 + u * RPP + rsub;
+                float s0 = 0.f, s1 = 0.f;
+                if (row < rows) {
+                    float kf[EPV];
+                    unpack<T>(Kc[(size_t)row * LPR + seg], kf);
+#pragma unroll
+                    for (int e = 0; e < EPV; e += 2) { s0 = fmaf(qf[e], kf[e], s0); s1 = fmaf(qf[e + 1], kf[e + 1], s1); }
+                }
+                sv[u] = s0 + s1;
+            }
+#pragma unroll
+            for (int o = LPR / 2; o > 0; o >>= 1) {
+#pragma unroll
+                for (int u = 0; u < 4; ++u) sv[u] += __shfl_xor_sync(0xffffffffu, sv[u], o);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int row = r0 + u * RPP + rsub;
+                if (row < rows) {
+                    bool ok;
+                    if (row < W) ok = (n >= W) ? (row != slot || dst >= 0) : (row < n);
+                    else ok = (row - W) < cnt_old && (row - W) != dst;
+                    const float sl = ok ? sv[u] * scale : -INFINITY;
+                    m_loc = fmaxf(m_loc, sl);
+                    if (seg == 0) s_log[row] = sl;
+                }
+            }
+        }
+        m_loc = warp_max(m_loc);
+        if (lane == 0) s_part[wid] = m_loc;
+        // the popped row doubles as the new pool entry: keep it before the buffers are handed back
+        uint4 mv = make_uint4(0, 0, 0, 0);
+        if (tid < 2 * LPR) mv = (tid < LPR ? Kc : Vc)[(size_t)slot * LPR + (tid % LPR)];
+        DPROF(4);
+        __syncthreads();                                        // (A) every read of the key buffer is done
+        DPROF(5);
+        if (tid == 0 && bh + 1 < bh_end)
+            bulk_load(sK, gblk + L.stride + L.off_k, P.kv_bytes, bar_k);
+        float mx = s_part[0];
+#pragma unroll
+        for (int w2 = 1; w2 < DT / 32; ++w2) mx = fmaxf(mx, s_part[w2]);
+
+        // ---- PV with the exponentials taken in place; the row sum rides along ------------------------------
+        float acc[EPV], lsum = 0.f;
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) acc[e] = 0.f;
+        for (int r0 = 0; r0 < rows; r0 += 4 * RPP) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int row = r0 + u * RPP + rsub;
+                if (row < rows) {
+                    const float pr = __expf(s_log[row] - mx);   // exp(-inf) = 0 for masked rows
+                    if (pr != 0.f) {
+                        float vf[EPV];
+                        unpack<T>(Vc[(size_t)row * LPR + seg], vf);
+#pragma unroll
+                        for (int e = 0; e < EPV; ++e) acc[e] = fmaf(pr, vf[e], acc[e]);
+                        if (seg == 0) lsum += pr;
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int o = 16; o >= LPR; o >>= 1) {
+#pragma unroll
+            for (int e = 0; e < EPV; ++e) acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], o);
+        }
+        lsum = warp_sum(lsum);
+        if (lane < LPR) {
+#pragma unroll
+            for (int e = 0; e < EPV; ++e) s_red[wid][lane * EPV + e] = acc[e];
+        }
+        if (lane == 0) s_sum[wid] = lsum;
+        DPROF(6);
+        __syncthreads();                                        // (B) every read of the value buffer is done
+        DPROF(7);
+        if (tid == 0 && bh + 1 < bh_end) {
+            bulk_load(sV, gblk + L.stride + L.off_v, P.kv_bytes, bar_v);
+            bulk_load(sT + (tb ^ 1) * P.tail_bytes, gblk + L.stride + L.off_z, P.tail_bytes, bar_t0 + 8 * (tb ^ 1));
+        }
+        const float p_new = __expf(s_log[rows] - mx);
+        float sum = p_new;
+#pragma unroll
+        for (int w2 = 0; w2 < DT / 32; ++w2) sum += s_sum[w2];
+        if (tid < D) {
+            float o = 0.f;
+#pragma unroll
+            for (int w2 = 0; w2 < DT / 32; ++w2) o += s_red[w2][tid];
+            o = fmaf(p_new, v1_mine, o);
+            o1[(size_t)bh * D + tid] = from_f<T>(o / sum);
+        }
+        if (tid == 0) lse1[bh] = mx + logf(sum);
+
+        // ---- write-back: only what changed goes to HBM -----------------------------------------------------
+        uint4* Kw = reinterpret_cast<uint4*>(gblk + L.off_k);
+        uint4* Vw = reinterpret_cast<uint4*>(gblk + L.off_v);
+        float* zw = reinterpret_cast<float*>(gblk + L.off_z);
+        int32_t* pw = reinterpret_cast<int32_t*>(gblk + L.off_pidx);
+        int32_t* mw = reinterpret_cast<int32_t*>(gblk + L.off_meta);
+        if (dst >= 0 && tid < 2 * LPR) (tid < LPR ? Kw : Vw)[(size_t)(W + dst) * LPR + (tid % LPR)] = mv;
+        if (tid >= 64 && tid < 64 + 2 * LPR) {
+            const int t2 = tid - 64;
+            (t2 < LPR ? Kw : Vw)[(size_t)slot * LPR + (t2 % LPR)] = kv_new;
+        }
+        if (tid == 128) {
+            if (dst >= 0) { zw[W + dst] = zc[slot]; pw[dst] = n - W; }
+            float znew = -INFINITY;
+            if (jsc >= 0) {
+                znew = bias;
+                for (int t = 0; t < K; ++t) znew += s_tap[t];
+            }
+            zw[slot] = -INFINITY;
+            if (jsc >= 0) zw[jsc % W] = znew;
+            mw[0] = n + 1;
+            mw[1] = cnt_new;
+        }
+        DPROF(8);
+        __syncthreads();                                        // (C) shared scratch is reused by the next head
+        if (bh + 1 < bh_end) fetch_inputs(bh + 1);
+        DPROF(9);
+    }
+}
+
 // State after a T-token prompt.  One block per (b,h); the cache was zero-filled beforehand.
 template <typename T>
 __global__ void cache_init_kernel(unsigned char* __restrict__ cache, CacheLayout L, const T* __restrict__ k,
@@ -320,6 +660,14 @@ __global__ void cache_init_kernel(unsigned char* __restrict__ cache, CacheLayout
 
 }  // namespace
 
+int decode_status_fetch_and_clear()
+{
+    int h = 0, zero = 0;
+    if (cudaMemcpyFromSymbol(&h, g_decode_status, sizeof(int)) != cudaSuccess) return -1;
+    if (h != 0) cudaMemcpyToSymbol(g_decode_status, &zero, sizeof(int));
+    return h;
+}
+
 int launch_cache_init(const Params& p, const void* k, const void* v, const float* z, const int32_t* idx,
                       const int32_t* cnt, void* cache, cudaStream_t st)
 {
@@ -342,6 +690,51 @@ int launch_decode(const Params& p, void* cache, const void* q1, const void* k1, 
 {
     if (p.W + p.R > MAX_ROWS) return LTE_ERR_UNSUPPORTED;
     const CacheLayout L = cache_layout(p.d, p.W, p.R, p.dtype);
+    const BulkSmem bp = bulk_smem_plan(L, p.W, p.R);
+    const size_t bulk_smem = bp.total;
+    const bool bulk = bulk_smem <= 73 * 1024 && p.K <= 2 * (DT / 32);   // three blocks per SM still fit
+    static int n_sm = 0;
+    if (bulk && n_sm == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+            return LTE_ERR_CUDA;
+    }
+    // persistent grid: every CTA walks `per_cta` consecutive heads; all CTAs are resident (3 per SM)
+    const int BH = p.B * p.H;
+    const int per_cta = bulk ? (BH + 3 * n_sm - 1) / (3 * n_sm) : 1;
+    const int n_cta = bulk ? (BH + per_cta - 1) / per_cta : BH;
+#define LTE_BULK(T, D)                                                                                            \
+    do {                                                                                                          \
+        static bool attr_done = false;                                                                            \
+        if (!attr_done) {                                                                                         \
+            if (cudaFuncSetAttribute(decode_bulk_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,        \
+                                     73 * 1024) != cudaSuccess) return LTE_ERR_CUDA;                              \
+            attr_done = true;                                                                                     \
+        }                                                                                                         \
+        decode_bulk_kernel<T, D><<<n_cta, DT, bulk_smem, st>>>((unsigned char*)cache, L, (const T*)q1,             \
+            (const T*)k1, (const T*)v1, (T*)o1, lse1, p.w, p.bias, BH, per_cta, p.H, p.W, p.R, p.sink, p.K,        \
+            p.zthr, p.scale);                                                                                     \
+    } while (0)
+    if (bulk) {
+        if (p.dtype == LTE_BF16) {
+            switch (p.d) {
+                case 32: LTE_BULK(__nv_bfloat16, 32); break;
+                case 64: LTE_BULK(__nv_bfloat16, 64); break;
+                case 128: LTE_BULK(__nv_bfloat16, 128); break;
+                default: return LTE_ERR_UNSUPPORTED;
+            }
+        } else {
+            switch (p.d) {
+                case 32: LTE_BULK(float, 32); break;
+                case 64: LTE_BULK(float, 64); break;
+                case 128: LTE_BULK(float, 128); break;
+                default: return LTE_ERR_UNSUPPORTED;
+            }
+        }
+        return cuda_status(cudaGetLastError());
+    }
+#undef LTE_BULK
 #define LTE_GO(T, D)                                                                                              \
     decode_kernel<T, D><<<p.B * p.H, DT, 0, st>>>((unsigned char*)cache, L, (const T*)q1, (const T*)k1, (const T*)v1, \
                                                   (T*)o1, lse1, p.w, p.bias, p.H, p.W, p.R, p.sink, p.K, p.zthr,   \
@@ -366,3 +759,10 @@ int launch_decode(const Params& p, void* cache, const void* q1, const void* k1, 
 }
 
 }  // namespace lte
+
+#ifdef LTE_PROFILE
+extern "C" int lte_dprof_read(long long* out)
+{
+    return cudaMemcpyFromSymbol(out, lte::g_dprof, sizeof(long long) * 64) == cudaSuccess ? 0 : -1;
+}
+#endif

@@ -122,3 +122,7 @@ def test_checkpoint_replay_is_bitwise_identical():
                                     v[:, :, n].contiguous())[0].clone() for n in range(230, 260)]
         runs.append((torch.stack(outs), cc))
     assert torch.equal(runs[0][0], runs[1][0]) and torch.equal(runs[0][1], runs[1][1])
+
+
+def test_no_bounded_wait_expired():
+    assert lte.lte_device_status() == 0
