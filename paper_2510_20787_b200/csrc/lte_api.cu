@@ -11,6 +11,7 @@ int launch_prefill_tc(const Params& p, const void* q, const void* k, const void*
                       const int32_t* cnt, void* o, float* lse, cudaStream_t st);
 int prefill_status_fetch_and_clear();
 int decode_status_fetch_and_clear();
+int scores_status_fetch_and_clear();
 
 namespace {
 
@@ -83,8 +84,9 @@ int lte_device_status(void)
 {
     const int h = prefill_status_fetch_and_clear();
     const int g = decode_status_fetch_and_clear();
-    if (h < 0 || g < 0) return LTE_ERR_CUDA;
-    return (h == 0 && g == 0) ? LTE_OK : LTE_ERR_DEVICE_STATUS;
+    const int f = scores_status_fetch_and_clear();
+    if (h < 0 || g < 0 || f < 0) return LTE_ERR_CUDA;
+    return (h == 0 && g == 0 && f == 0) ? LTE_OK : LTE_ERR_DEVICE_STATUS;
 }
 
 size_t lte_workspace_bytes(int op, const lte_shape* s, const lte_conv* c)
