@@ -12,6 +12,10 @@
 #include "common.cuh"
 
 namespace lte {
+
+int launch_bwd_dq_tc(const Params& p, const void* q, const void* k, const void* v, const void* o, const float* lse,
+                     const void* dO, const int32_t* idx, const int32_t* cnt, void* dq, float* delta, cudaStream_t st);
+
 namespace {
 
 constexpr int CHUNK = 256;     // positions per conv-gradient partial
@@ -273,8 +277,13 @@ int run(const Params& p, const void* q, const void* k, const void* v, const void
     float* dv32 = (float*)(base + w.dv32);
     const bool f32 = flags & LTE_BWD_CNN_INPUT_GRAD;
     dim3 grid((p.T + 3) / 4, p.B * p.H);
-    bwd_dq_kernel<T, D><<<grid, 128, 0, st>>>((const T*)q, (const T*)k, (const T*)v, (const T*)o, (const T*)dO, lse, idx,
-                                              cnt, (T*)dq, delta, p.T, p.W, p.R, p.scale);
+    if constexpr (sizeof(T) == 2 && (D == 64 || D == 128)) {
+        const int e = launch_bwd_dq_tc(p, q, k, v, o, lse, dO, idx, cnt, dq, delta, st);
+        if (e != LTE_OK) return e;
+    } else {
+        bwd_dq_kernel<T, D><<<grid, 128, 0, st>>>((const T*)q, (const T*)k, (const T*)v, (const T*)o, (const T*)dO, lse,
+                                                  idx, cnt, (T*)dq, delta, p.T, p.W, p.R, p.scale);
+    }
     if (f32)
         bwd_dkv_kernel<T, D, true><<<grid, 128, 0, st>>>((const T*)q, (const T*)k, (const T*)v, (const T*)dO, lse, delta,
                                                          z, idx, cnt, lambda, (T*)dk, (T*)dv, dk32, dv32, dz, p.H, p.T,

@@ -1,0 +1,379 @@
+// Backward of the LTE prefill attention on the tcgen05 tensor cores (Section 3.1.2), bf16, d = 64 or 128.
+//
+// Two kernels, both in gather form (no floating-point atomics, deterministic):
+//
+// dq kernel   one CTA per 128-query tile, the same key/value tile walk as the forward kernel (window tiles by
+//             TMA, retained tiles gathered with cp.async).  Per 64-key tile:
+//               S = Q K^T and dP = dO V^T          tcgen05.mma into TMEM
+//               P = exp2(S c2 - L2_i),  dS = P (dP - delta_i) scale   by the thread owning row i (no online softmax:
+//               the forward's logsumexp fixes the normalisation), written as bf16 into swizzled shared memory
+//               dQ += dS K                          tcgen05.mma, K tile as the MN-major operand, accumulated in TMEM
+//             delta_i = <dO_i, O_i> is computed by the same thread at the start and also written out for the second kernel.
+//
+// dkv kernel  one CTA per 128-key tile: the contiguous keys of a window tile, or 128 entries of the retained list
+//             (their K/V rows gathered once).  It walks the 64-query blocks that can see those keys:
+//               S^T = K Q^T and dP^T = V dO^T       tcgen05.mma (keys on the M side)
+//               P^T, dS^T                           by the thread owning the key row; L2 and delta of the block's
+//                                                   64 queries are read from shared memory
+//               dV += P^T dO,  dK += dS^T Q         tcgen05.mma with the dO / Q block as MN-major operand
+//             and finishes with Eq. 6's inner product <v_j, dV_j> per key from the fp32 accumulators.  Window tiles
+//             write dK, dV of their keys; retained tiles write their far-query share to scratch, which a small merge
+//             kernel adds row by row (each key appears once in the list, so the sum order is fixed).
+#include "tc_common.cuh"
+
+namespace lte {
+
+__device__ int g_bwd_status = 0;
+
+namespace {
+
+using namespace tc;
+__device__ __forceinline__ void bwait(uint32_t bar, uint32_t parity, int code) { mbar_wait_s(bar, parity, code, &g_bwd_status); }
+__device__ __forceinline__ void group_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+constexpr int BM = 128, BN = 64, NTHREADS = 160, NST = 3;      // 3 stages for every streamed tile
+constexpr float kLog2e = 1.4426950408889634f;
+
+template <int D> struct SmemQ {                                // dq kernel
+    static constexpr int SUB = D / 64;
+    static constexpr int QTILE = BM * D * 2, KVTILE = BN * D * 2;
+    static constexpr int OFF_Q = 0, OFF_DO = QTILE, OFF_K = 2 * QTILE, OFF_V = OFF_K + NST * KVTILE;
+    static constexpr int OFF_DS = OFF_V + NST * KVTILE;        // [128][64] bf16
+    static constexpr int OFF_BAR = OFF_DS + BM * BN * 2;
+    static constexpr int OFF_IDX = OFF_BAR + 128;
+    static constexpr int BYTES = OFF_IDX + 512;
+    static constexpr uint32_t TMEM_COLS = 256;                 // S: [0,64)  dP: [64,128)  dQ: [128, 128+D)
+};
+
+template <int D>
+__global__ void __launch_bounds__(NTHREADS, D == 64 ? 2 : 1)
+bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmDO,
+                 const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                 const __nv_bfloat16* __restrict__ kg, const __nv_bfloat16* __restrict__ vg,
+                 const __nv_bfloat16* __restrict__ og, const __nv_bfloat16* __restrict__ dog,
+                 const float* __restrict__ lse, const int32_t* __restrict__ idx, const int32_t* __restrict__ cnt,
+                 __nv_bfloat16* __restrict__ dq, float* __restrict__ delta, int Tlen, int W, int R, float scale)
+{
+    using S = SmemQ<D>;
+    constexpr int SUB = S::SUB;
+    constexpr uint32_t DP_COL = BN, DQ_COL = 2 * BN;
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    const uint32_t base = smem_u32(smem_raw);
+    if ((base & 1023u) != 0) { if (threadIdx.x == 0) atomicExch(&g_bwd_status, 9); return; }
+    const uint32_t sQ = base + S::OFF_Q, sDO = base + S::OFF_DO, sK = base + S::OFF_K, sV = base + S::OFF_V;
+    const uint32_t sDS = base + S::OFF_DS;
+    const uint32_t bar_q = base + S::OFF_BAR, bar_k0 = bar_q + 8, bar_v0 = bar_q + 32, bar_s = bar_q + 56;
+    const uint32_t bar_g0 = bar_q + 64, bar_p = bar_q + 80, bar_pv = bar_q + 88, tmem_slot = bar_q + 96;
+    volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(smem_raw + S::OFF_BAR + 96);
+    volatile int* s_idx = reinterpret_cast<volatile int*>(smem_raw + S::OFF_IDX);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int bh = blockIdx.y;
+    const int i0 = blockIdx.x * BM;
+    const int i_hi = min(i0 + BM - 1, Tlen - 1);
+    const int j_start = max(i0 - W + 1, 0);
+    const int n_win = (i_hi - j_start + 1 + BN - 1) / BN;
+    const int32_t* id = idx + (size_t)bh * R;
+    const int n_ret = cnt[bh];
+
+    if (tid == 0) {
+        mbar_init(bar_q, 1);
+#pragma unroll
+        for (int s2 = 0; s2 < NST; ++s2) { mbar_init(bar_k0 + 8 * s2, 1); mbar_init(bar_v0 + 8 * s2, 1); }
+        mbar_init(bar_s, 1);
+        mbar_init(bar_g0, 128); mbar_init(bar_g0 + 8, 128);
+        mbar_init(bar_p, 128); mbar_init(bar_pv, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 4) tmem_alloc(tmem_slot, S::TMEM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot_gen;
+
+    if (warp == 4) {
+        // =================================== control warp (one lane) ========================================
+        int nv_max = 0;
+        {
+            const int lim = i_hi - W;
+            for (int e0 = 0; e0 < n_ret; e0 += 32) {
+                const int e = e0 + lane < n_ret ? id[e0 + lane] : 0x7fffffff;
+                const unsigned bal = __ballot_sync(0xffffffffu, e <= lim);
+                nv_max += __popc(bal);
+                if (bal != 0xffffffffu) break;
+            }
+        }
+        const int n_tiles = n_win + (nv_max + BN - 1) / BN;
+        if (lane == 0) {
+            constexpr uint32_t IDESC_S = instr_desc(BM, BN, false);
+            constexpr uint32_t IDESC_Q = instr_desc(BM, D, true);
+            const uint32_t q_lo = desc_lo(sQ, 16), do_lo = desc_lo(sDO, 16), k_lo = desc_lo(sK, 16), v_lo = desc_lo(sV, 16);
+            const uint32_t ds_lo = desc_lo(sDS, 16), kmn_lo = desc_lo(sK, 8192);
+            uint32_t k_phase = 0, v_phase = 0, g_waited = 0;
+            auto tma_kv = [&](int t, bool is_v) {
+                const int st = t % NST;
+                const uint32_t dst = (is_v ? sV : sK) + st * S::KVTILE;
+                const uint32_t bar = (is_v ? bar_v0 : bar_k0) + 8 * st;
+                mbar_expect_tx(bar, S::KVTILE);
+                const int y = j_start + t * BN;
+#pragma unroll
+                for (int sb = 0; sb < SUB; ++sb) tma_load_3d(dst + sb * 8192, is_v ? &tmV : &tmK, sb * 64, y, bh, bar);
+            };
+            auto need_g = [&](uint32_t phase) {
+                while (g_waited <= phase) { bwait(bar_g0 + 8 * (g_waited & 1), (g_waited >> 1) & 1, 10); ++g_waited; }
+            };
+            auto wait_kv = [&](int t) {
+                if (t < n_win) {
+                    const int st = t % NST;
+                    bwait(bar_k0 + 8 * st, (k_phase >> st) & 1u, 2); k_phase ^= 1u << st;
+                    bwait(bar_v0 + 8 * st, (v_phase >> st) & 1u, 4); v_phase ^= 1u << st;
+                }
+            };
+            auto mma_s_dp = [&](int t) {
+                const uint32_t so = (uint32_t)(t % NST) * (S::KVTILE >> 4);
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk)
+                    umma(tmem, desc64(q_lo + (kk >> 2) * 1024 + (kk & 3) * 2, kDescHi),
+                         desc64(k_lo + so + (kk >> 2) * 512 + (kk & 3) * 2, kDescHi), IDESC_S, kk > 0);
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk)
+                    umma(tmem + DP_COL, desc64(do_lo + (kk >> 2) * 1024 + (kk & 3) * 2, kDescHi),
+                         desc64(v_lo + so + (kk >> 2) * 512 + (kk & 3) * 2, kDescHi), IDESC_S, kk > 0);
+                umma_commit(bar_s);
+            };
+
+            mbar_expect_tx(bar_q, 2 * S::QTILE);
+#pragma unroll
+            for (int sb = 0; sb < SUB; ++sb) {
+                tma_load_3d(sQ + sb * 16384, &tmQ, sb * 64, i0, bh, bar_q);
+                tma_load_3d(sDO + sb * 16384, &tmDO, sb * 64, i0, bh, bar_q);
+            }
+            for (int t = 0; t < NST && t < n_win; ++t) { tma_kv(t, false); tma_kv(t, true); }
+            need_g(0);
+            bwait(bar_q, 0, 1);
+            wait_kv(0);
+            tc_fence_after();
+            mma_s_dp(0);
+            for (int t = 0; t < n_tiles; ++t) {
+                bwait(bar_p, t & 1, 7);                        // dS(t) is in shared memory; S / dP buffers are free
+                tc_fence_after();
+                {
+                    const uint32_t kb = kmn_lo + (uint32_t)(t % NST) * (S::KVTILE >> 4);
+#pragma unroll
+                    for (int kk = 0; kk < BN / 16; ++kk)
+                        umma(tmem + DQ_COL, desc64(ds_lo + kk * 2, kDescHi), desc64(kb + kk * 128, kDescHi), IDESC_Q,
+                             (t > 0 || kk > 0) ? 1u : 0u);
+                    umma_commit(bar_pv);
+                }
+                if (t + 1 < n_tiles) {
+                    need_g(t + 1);
+                    wait_kv(t + 1);
+                    mma_s_dp(t + 1);
+                }
+                // dQ(t-1) has completed (the softmax warps waited for it before producing dS(t)): its key stage and
+                // the value stage of tile t-1 can take window tile t-1+NST
+                if (t >= 1 && t - 1 + NST < n_win) { tma_kv(t - 1 + NST, false); tma_kv(t - 1 + NST, true); }
+            }
+        }
+    } else {
+        // =================================== softmax warps ==================================================
+        const int i = i0 + tid;
+        const int ic = min(i, Tlen - 1);
+        // delta_i = <dO_i, O_i>, L2_i = lse_i * log2(e)
+        float dl = 0.f;
+        {
+            const uint4* orow = reinterpret_cast<const uint4*>(og + ((size_t)bh * Tlen + ic) * D);
+            const uint4* grow = reinterpret_cast<const uint4*>(dog + ((size_t)bh * Tlen + ic) * D);
+#pragma unroll 4
+            for (int c = 0; c < D / 8; ++c) {
+                const uint4 a = orow[c], b = grow[c];
+                const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    dl = fmaf(__uint_as_float(aw[u] << 16), __uint_as_float(bw[u] << 16), dl);
+                    dl = fmaf(__uint_as_float(aw[u] & 0xffff0000u), __uint_as_float(bw[u] & 0xffff0000u), dl);
+                }
+            }
+        }
+        if (i < Tlen) delta[(size_t)bh * Tlen + i] = dl;
+        const float L2 = lse[(size_t)bh * Tlen + ic] * kLog2e;
+
+        const int lim = ic - W, lim_max = i_hi - W;
+        int nvis = 0;
+        for (int e0 = 0; e0 < n_ret; e0 += 128) {
+            const int n_here = min(128, n_ret - e0);
+            group_sync();
+            if (tid < n_here) s_idx[tid] = id[e0 + tid];
+            group_sync();
+            if (s_idx[n_here - 1] <= lim) nvis += n_here;
+            else {
+                int lo = 0, hi = n_here;
+                while (lo < hi) { const int mid = (lo + hi) >> 1; if (s_idx[mid] <= lim) lo = mid + 1; else hi = mid; }
+                nvis += lo;
+            }
+            if (s_idx[n_here - 1] > lim_max) break;
+        }
+        group_sync();
+        if (i == i_hi) s_idx[0] = nvis;
+        group_sync();
+        const int nv_max = s_idx[0];
+        const int n_tiles = n_win + (nv_max + BN - 1) / BN;
+
+        const int g_row = tid >> 3, g_sub = tid & 7;
+        auto gather_rows = [&](int t, int (&rows4)[4]) {
+#pragma unroll
+            for (int ps = 0; ps < 4; ++ps) {
+                const int e = (t - n_win) * BN + ps * 16 + g_row;
+                rows4[ps] = (t >= n_win && t < n_tiles && e < nv_max) ? id[e] : -1;
+            }
+        };
+        auto gather_issue = [&](int t, bool is_v, const int (&rows4)[4]) {
+            if (t >= n_win && t < n_tiles) {
+                const uint32_t dst = (is_v ? sV : sK) + (t % NST) * S::KVTILE;
+#pragma unroll
+                for (int ps = 0; ps < 4; ++ps) {
+                    const int row = ps * 16 + g_row;
+                    const bool ok = rows4[ps] >= 0;
+                    const __nv_bfloat16* src = (is_v ? vg : kg) + ((size_t)bh * Tlen + (ok ? rows4[ps] : 0)) * D;
+#pragma unroll
+                    for (int c = g_sub; c < D / 8; c += 8) {
+                        const uint32_t off = (c >> 3) * 8192 + row * 128 + (((c & 7) ^ (row & 7)) << 4);
+                        cp_async16(dst + off, src + c * 8, ok ? 16u : 0u);
+                    }
+                }
+            }
+        };
+        {
+            int rows4[4];
+            for (int t = 0; t < NST; ++t) { gather_rows(t, rows4); gather_issue(t, false, rows4); gather_issue(t, true, rows4); }
+            cp_async_commit();
+            cp_async_commit();                                 // empty group: the wait at the top of tile 0 then covers the one above
+        }
+        const float c2 = scale * kLog2e;
+        const uint32_t lane_base = ((uint32_t)(warp * 32)) << 16;
+
+        for (int t = 0; t < n_tiles; ++t) {
+            int rn[4];
+            gather_rows(t - 1 + NST, rn);                      // retained tile that goes into the stage of tile t-1
+            cp_async_wait<1>();                                // every gather but the latest tile's has landed
+            fence_proxy_async();
+            mbar_arrive(bar_g0 + 8 * (t & 1));
+
+            int c_lo, c_hi;
+            if (t < n_win) {
+                const int jt0 = j_start + t * BN;
+                c_lo = max(i - W + 1, 0) - jt0;
+                c_hi = i - jt0;
+            } else {
+                c_lo = 0;
+                c_hi = nvis - (t - n_win) * BN - 1;
+            }
+            const int u_lo = __shfl_sync(0xffffffffu, c_lo, 0), u_hi = __shfl_sync(0xffffffffu, c_hi, 31);
+
+            bwait(bar_s, t & 1, 3);                            // S(t), dP(t) are in TMEM
+            tc_fence_after();
+            uint32_t pk[32];                                   // dS row as 64 bf16
+#pragma unroll
+            for (int cb = 0; cb < 2; ++cb) {
+                const bool act = cb * 32 <= u_hi && cb * 32 + 31 >= u_lo;
+                if (act) {
+                    uint32_t rs[32], rp[32];
+                    tmem_ld32(tmem + lane_base + cb * 32, rs);
+                    tmem_ld32(tmem + lane_base + DP_COL + cb * 32, rp);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int c = 0; c < 32; c += 2) {
+                        const int col = cb * 32 + c;
+                        float d0 = 0.f, d1 = 0.f;
+                        if (col >= c_lo && col <= c_hi)
+                            d0 = fast_exp2(fmaf(__uint_as_float(rs[c]), c2, -L2)) * (__uint_as_float(rp[c]) - dl) * scale;
+                        if (col + 1 >= c_lo && col + 1 <= c_hi)
+                            d1 = fast_exp2(fmaf(__uint_as_float(rs[c + 1]), c2, -L2)) * (__uint_as_float(rp[c + 1]) - dl) * scale;
+                        __nv_bfloat162 h = __floats2bfloat162_rn(d0, d1);
+                        pk[cb * 16 + (c >> 1)] = *reinterpret_cast<uint32_t*>(&h);
+                    }
+                } else {
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) pk[cb * 16 + c] = 0u;
+                }
+            }
+            // dQ(t-1) must be done before dS is overwritten; its key stage (and the value stage) are then free
+            if (t > 0) { bwait(bar_pv, (t - 1) & 1, 4); tc_fence_after(); }
+            if (t > 0) { gather_issue(t - 1 + NST, false, rn); gather_issue(t - 1 + NST, true, rn); }
+            cp_async_commit();
+#pragma unroll
+            for (int ch = 0; ch < 8; ++ch) {
+                const uint32_t dst = sDS + tid * 128 + ((ch ^ (tid & 7)) << 4);
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(pk[4 * ch]), "r"(pk[4 * ch + 1]),
+                             "r"(pk[4 * ch + 2]), "r"(pk[4 * ch + 3]) : "memory");
+            }
+            fence_proxy_async();
+            tc_fence_before();
+            mbar_arrive(bar_p);
+        }
+        bwait(bar_pv, (n_tiles - 1) & 1, 5);
+        tc_fence_after();
+        // ---- epilogue: dQ (the softmax scale is already folded into dS) ------------------------------------
+        __nv_bfloat16* qrow = dq + ((size_t)bh * Tlen + i) * D;
+#pragma unroll
+        for (int cb = 0; cb < D / 32; ++cb) {
+            uint32_t q4[32];
+            tmem_ld32(tmem + lane_base + DQ_COL + cb * 32, q4);
+            tmem_wait_ld();
+            if (i < Tlen) {
+#pragma unroll
+                for (int c = 0; c < 32; c += 8) {
+                    uint32_t w4[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(q4[c + 2 * u]), __uint_as_float(q4[c + 2 * u + 1]));
+                        w4[u] = *reinterpret_cast<uint32_t*>(&h);
+                    }
+                    *reinterpret_cast<uint4*>(qrow + cb * 32 + c) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 4) tmem_dealloc(tmem, S::TMEM_COLS);
+}
+
+}  // namespace
+
+// dq (and delta) on the tensor cores.  Returns LTE_OK or an error; the caller runs the remaining stages.
+int launch_bwd_dq_tc(const Params& p, const void* q, const void* k, const void* v, const void* o, const float* lse,
+                     const void* dO, const int32_t* idx, const int32_t* cnt, void* dq, float* delta, cudaStream_t st)
+{
+    const int BH = p.B * p.H;
+    CUtensorMap tq, tdo, tk, tv;
+    if (!make_map(&tq, q, BH, p.T, p.d, BM) || !make_map(&tdo, dO, BH, p.T, p.d, BM) ||
+        !make_map(&tk, k, BH, p.T, p.d, BN) || !make_map(&tv, v, BH, p.T, p.d, BN))
+        return LTE_ERR_CUDA;
+    dim3 grid((p.T + BM - 1) / BM, BH);
+#define LTE_GO(D)                                                                                                  \
+    do {                                                                                                           \
+        static bool attr_done = false;                                                                             \
+        if (!attr_done) {                                                                                          \
+            if (cudaFuncSetAttribute(bwd_dq_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,      \
+                                     SmemQ<D>::BYTES) != cudaSuccess) return LTE_ERR_CUDA;                         \
+            attr_done = true;                                                                                      \
+        }                                                                                                          \
+        bwd_dq_tc_kernel<D><<<grid, NTHREADS, SmemQ<D>::BYTES, st>>>(                                        \
+            tq, tdo, tk, tv, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (const __nv_bfloat16*)o,            \
+            (const __nv_bfloat16*)dO, lse, idx, cnt, (__nv_bfloat16*)dq, delta, p.T, p.W, p.R, p.scale);           \
+    } while (0)
+    if (p.d == 64) LTE_GO(64); else if (p.d == 128) LTE_GO(128); else return LTE_ERR_UNSUPPORTED;
+#undef LTE_GO
+    return cuda_status(cudaGetLastError());
+}
+
+int bwd_status_fetch_and_clear()
+{
+    int h = 0, zero = 0;
+    if (cudaMemcpyFromSymbol(&h, g_bwd_status, sizeof(int)) != cudaSuccess) return -1;
+    if (h != 0) cudaMemcpyToSymbol(g_bwd_status, &zero, sizeof(int));
+    return h;
+}
+
+}  // namespace lte

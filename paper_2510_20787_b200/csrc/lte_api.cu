@@ -12,6 +12,7 @@ int launch_prefill_tc(const Params& p, const void* q, const void* k, const void*
 int prefill_status_fetch_and_clear();
 int decode_status_fetch_and_clear();
 int scores_status_fetch_and_clear();
+int bwd_status_fetch_and_clear();
 
 namespace {
 
@@ -85,8 +86,9 @@ int lte_device_status(void)
     const int h = prefill_status_fetch_and_clear();
     const int g = decode_status_fetch_and_clear();
     const int f = scores_status_fetch_and_clear();
-    if (h < 0 || g < 0 || f < 0) return LTE_ERR_CUDA;
-    return (h == 0 && g == 0 && f == 0) ? LTE_OK : LTE_ERR_DEVICE_STATUS;
+    const int b = bwd_status_fetch_and_clear();
+    if (h < 0 || g < 0 || f < 0 || b < 0) return LTE_ERR_CUDA;
+    return (h == 0 && g == 0 && f == 0 && b == 0) ? LTE_OK : LTE_ERR_DEVICE_STATUS;
 }
 
 size_t lte_workspace_bytes(int op, const lte_shape* s, const lte_conv* c)
