@@ -16,6 +16,11 @@ namespace lte {
 int launch_bwd_dq_tc(const Params& p, const void* q, const void* k, const void* v, const void* o, const float* lse,
                      const void* dO, const int32_t* idx, const int32_t* cnt, void* dq, float* delta, cudaStream_t st);
 
+size_t bwd_tc_ret_bytes(const Params& p);
+int launch_bwd_dkv_tc(const Params& p, const void* q, const void* k, const void* v, const float* lse, const void* dO,
+                      const float* delta, const float* z, const int32_t* idx, const int32_t* cnt, const float* lambda,
+                      void* dk, void* dv, float* dk32, float* dv32, float* dz, void* ret_ws, bool f32out, cudaStream_t st);
+
 namespace {
 
 constexpr int CHUNK = 256;     // positions per conv-gradient partial
@@ -241,7 +246,7 @@ __global__ void bwd_finish_kernel(const float* __restrict__ dk32, const float* _
     }
 }
 
-struct WsPlan { size_t delta, dz, part_w, part_b, dk32, dv32, total; int nchunk; };
+struct WsPlan { size_t delta, dz, part_w, part_b, dk32, dv32, ret, total; int nchunk; };
 WsPlan plan(const Params& p, uint32_t flags)
 {
     WsPlan w;
@@ -258,6 +263,8 @@ WsPlan plan(const Params& p, uint32_t flags)
         w.dk32 = off; off += up(bht * p.d * 4);
         w.dv32 = off; off += up(bht * p.d * 4);
     }
+    w.ret = off;
+    if (p.dtype == LTE_BF16 && (p.d == 64 || p.d == 128)) off += bwd_tc_ret_bytes(p);   // tensor-core path: retained-tile shares
     w.total = off;
     return w;
 }
@@ -284,14 +291,19 @@ int run(const Params& p, const void* q, const void* k, const void* v, const void
         bwd_dq_kernel<T, D><<<grid, 128, 0, st>>>((const T*)q, (const T*)k, (const T*)v, (const T*)o, (const T*)dO, lse,
                                                   idx, cnt, (T*)dq, delta, p.T, p.W, p.R, p.scale);
     }
-    if (f32)
+    if constexpr (sizeof(T) == 2 && (D == 64 || D == 128)) {
+        const int e = launch_bwd_dkv_tc(p, q, k, v, lse, dO, delta, z, idx, cnt, lambda, dk, dv, dk32, dv32, dz, base + w.ret,
+                                        f32, st);
+        if (e != LTE_OK) return e;
+    } else if (f32) {
         bwd_dkv_kernel<T, D, true><<<grid, 128, 0, st>>>((const T*)q, (const T*)k, (const T*)v, (const T*)dO, lse, delta,
                                                          z, idx, cnt, lambda, (T*)dk, (T*)dv, dk32, dv32, dz, p.H, p.T,
                                                          p.W, p.R, p.half, p.zthr, p.scale);
-    else
+    } else {
         bwd_dkv_kernel<T, D, false><<<grid, 128, 0, st>>>((const T*)q, (const T*)k, (const T*)v, (const T*)dO, lse, delta,
                                                           z, idx, cnt, lambda, (T*)dk, (T*)dv, dk32, dv32, dz, p.H, p.T,
                                                           p.W, p.R, p.half, p.zthr, p.scale);
+    }
     dim3 gc(p.B * w.nchunk, p.H);
     bwd_conv_partial_kernel<T><<<gc, 2 * D, (CHUNK + p.K - 1) * sizeof(float), st>>>(
         (const T*)k, (const T*)v, dz, part_w, part_b, p.B, p.H, p.T, D, p.K, w.nchunk);

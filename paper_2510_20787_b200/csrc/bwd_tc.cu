@@ -339,6 +339,342 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     if (warp == 4) tmem_dealloc(tmem, S::TMEM_COLS);
 }
 
+
+// ================================================ dkv kernel =====================================================
+template <int D> struct SmemK {
+    static constexpr int SUB = D / 64;
+    static constexpr int KTILE = 128 * D * 2, QBLK = 64 * D * 2;
+    static constexpr int OFF_K = 0, OFF_V = KTILE, OFF_Q = 2 * KTILE, OFF_DO = OFF_Q + NST * QBLK;
+    static constexpr int OFF_PT = OFF_DO + NST * QBLK;         // [128][64] bf16
+    static constexpr int OFF_DST = OFF_PT + 128 * 64 * 2;      // [128][64] bf16
+    static constexpr int OFF_COL = OFF_DST + 128 * 64 * 2;     // L2[64], delta[64] of the current query block
+    static constexpr int OFF_BAR = OFF_COL + 512;
+    static constexpr int BYTES = OFF_BAR + 128;
+    static constexpr uint32_t TMEM_COLS = D == 64 ? 256 : 512; // S^T [0,64) dP^T [64,128) dV [128,128+D) dK [128+D,128+2D)
+};
+
+template <int D, bool F32OUT>
+__global__ void __launch_bounds__(NTHREADS, D == 64 ? 2 : 1)
+bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                  const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmDO,
+                  const __nv_bfloat16* __restrict__ kg, const __nv_bfloat16* __restrict__ vg,
+                  const float* __restrict__ lse, const float* __restrict__ delta, const int32_t* __restrict__ idx,
+                  const int32_t* __restrict__ cnt, __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv,
+                  float* __restrict__ dk32, float* __restrict__ dv32, float* __restrict__ dr_win,
+                  float* __restrict__ dk_ret, float* __restrict__ dv_ret, float* __restrict__ dr_ret, int n_wt, int Tlen,
+                  int W, int R, float scale)
+{
+    using S = SmemK<D>;
+    constexpr int SUB = S::SUB;
+    constexpr uint32_t DP_COL = 64, DV_COL = 128, DK_COL = 128 + D;
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    const uint32_t base = smem_u32(smem_raw);
+    if ((base & 1023u) != 0) { if (threadIdx.x == 0) atomicExch(&g_bwd_status, 9); return; }
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int bh = blockIdx.y;
+    const bool is_ret = (int)blockIdx.x >= n_wt;
+    const int n_ret = cnt[bh];
+    const int32_t* id = idx + (size_t)bh * R;
+    const int j0 = is_ret ? 0 : blockIdx.x * 128;              // window tile: first key
+    const int e0 = is_ret ? ((int)blockIdx.x - n_wt) * 128 : 0;   // retained tile: first list entry
+    if (is_ret && e0 >= n_ret) return;                         // nothing retained in this slice of the list
+
+    // query blocks that can see the tile
+    int ib_start, n_blk;
+    if (!is_ret) {
+        ib_start = j0;
+        const int i_end = min(Tlen - 1, j0 + 127 + W - 1);
+        n_blk = (i_end - ib_start) / 64 + 1;
+    } else {
+        const int first = id[e0] + W;                          // the oldest entry's first far query
+        ib_start = (first / 64) * 64;
+        n_blk = first <= Tlen - 1 ? (Tlen - 1 - ib_start) / 64 + 1 : 0;
+    }
+
+    const uint32_t sK = base + S::OFF_K, sV = base + S::OFF_V, sQ = base + S::OFF_Q, sDO = base + S::OFF_DO;
+    const uint32_t sPT = base + S::OFF_PT, sDST = base + S::OFF_DST;
+    float* s_col = reinterpret_cast<float*>(smem_raw + S::OFF_COL);
+    const uint32_t bar_kv = base + S::OFF_BAR, bar_q0 = bar_kv + 8, bar_s = bar_kv + 32, bar_g = bar_kv + 40;
+    const uint32_t bar_p = bar_kv + 48, bar_pv = bar_kv + 56, tmem_slot = bar_kv + 64;
+    volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(smem_raw + S::OFF_BAR + 64);
+
+    if (tid == 0) {
+        mbar_init(bar_kv, 1);
+#pragma unroll
+        for (int s2 = 0; s2 < NST; ++s2) mbar_init(bar_q0 + 8 * s2, 1);
+        mbar_init(bar_s, 1); mbar_init(bar_g, 128); mbar_init(bar_p, 128); mbar_init(bar_pv, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 4) tmem_alloc(tmem_slot, S::TMEM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot_gen;
+
+    if (warp == 4) {
+        if (lane == 0 && n_blk > 0) {
+            constexpr uint32_t IDESC_S = instr_desc(128, 64, false);
+            constexpr uint32_t IDESC_O = instr_desc(128, D, true);
+            const uint32_t k_lo = desc_lo(sK, 16), v_lo = desc_lo(sV, 16), q_lo = desc_lo(sQ, 16), do_lo = desc_lo(sDO, 16);
+            const uint32_t pt_lo = desc_lo(sPT, 16), dst_lo = desc_lo(sDST, 16);
+            const uint32_t qmn_lo = desc_lo(sQ, 8192), domn_lo = desc_lo(sDO, 8192);
+            uint32_t q_phase = 0;
+            auto tma_blk = [&](int t) {
+                const int st = t % NST;
+                const uint32_t bar = bar_q0 + 8 * st;
+                mbar_expect_tx(bar, 2 * S::QBLK);
+                const int y = ib_start + t * 64;
+#pragma unroll
+                for (int sb = 0; sb < SUB; ++sb) {
+                    tma_load_3d(sQ + st * S::QBLK + sb * 8192, &tmQ, sb * 64, y, bh, bar);
+                    tma_load_3d(sDO + st * S::QBLK + sb * 8192, &tmDO, sb * 64, y, bh, bar);
+                }
+            };
+            auto wait_blk = [&](int t) {
+                const int st = t % NST;
+                bwait(bar_q0 + 8 * st, (q_phase >> st) & 1u, 2); q_phase ^= 1u << st;
+            };
+            auto mma_s_dp = [&](int t) {
+                const uint32_t so = (uint32_t)(t % NST) * (S::QBLK >> 4);
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk)
+                    umma(tmem, desc64(k_lo + (kk >> 2) * 1024 + (kk & 3) * 2, kDescHi),
+                         desc64(q_lo + so + (kk >> 2) * 512 + (kk & 3) * 2, kDescHi), IDESC_S, kk > 0);
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk)
+                    umma(tmem + DP_COL, desc64(v_lo + (kk >> 2) * 1024 + (kk & 3) * 2, kDescHi),
+                         desc64(do_lo + so + (kk >> 2) * 512 + (kk & 3) * 2, kDescHi), IDESC_S, kk > 0);
+                umma_commit(bar_s);
+            };
+            if (!is_ret) {
+                mbar_expect_tx(bar_kv, 2 * S::KTILE);
+#pragma unroll
+                for (int sb = 0; sb < SUB; ++sb) {
+                    tma_load_3d(sK + sb * 16384, &tmK, sb * 64, j0, bh, bar_kv);
+                    tma_load_3d(sV + sb * 16384, &tmV, sb * 64, j0, bh, bar_kv);
+                }
+            }
+            for (int t = 0; t < NST && t < n_blk; ++t) tma_blk(t);
+            if (!is_ret) bwait(bar_kv, 0, 1); else bwait(bar_g, 0, 10);   // the tile's own K/V rows are in shared memory
+            wait_blk(0);
+            tc_fence_after();
+            mma_s_dp(0);
+            for (int t = 0; t < n_blk; ++t) {
+                bwait(bar_p, t & 1, 7);                        // P^T(t), dS^T(t) are in shared memory
+                tc_fence_after();
+                {
+                    const uint32_t so = (uint32_t)(t % NST) * (S::QBLK >> 4);
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)
+                        umma(tmem + DV_COL, desc64(pt_lo + kk * 2, kDescHi), desc64(domn_lo + so + kk * 128, kDescHi), IDESC_O,
+                             (t > 0 || kk > 0) ? 1u : 0u);
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)
+                        umma(tmem + DK_COL, desc64(dst_lo + kk * 2, kDescHi), desc64(qmn_lo + so + kk * 128, kDescHi), IDESC_O,
+                             (t > 0 || kk > 0) ? 1u : 0u);
+                    umma_commit(bar_pv);
+                }
+                if (t + 1 < n_blk) { wait_blk(t + 1); mma_s_dp(t + 1); }
+                // the accumulations of block t-1 have completed (the key threads waited for them before producing
+                // block t's operands): its stage can take block t-1+NST
+                if (t >= 1 && t - 1 + NST < n_blk) tma_blk(t - 1 + NST);
+            }
+        }
+    } else {
+        // ==================================== key threads: thread r owns key row r ===========================
+        const int pos = is_ret ? (e0 + tid < n_ret ? id[e0 + tid] : -1) : (j0 + tid < Tlen ? j0 + tid : -1);
+        if (is_ret) {
+            // this tile's K / V rows, gathered once (zero rows past the end of the list)
+            const size_t rowoff = ((size_t)bh * Tlen + (pos >= 0 ? pos : 0)) * D;
+            const uint32_t nb = pos >= 0 ? 16u : 0u;
+#pragma unroll
+            for (int c = 0; c < D / 8; ++c) {
+                const uint32_t off = (c >> 3) * 16384 + tid * 128 + (((c & 7) ^ (tid & 7)) << 4);
+                cp_async16(sK + off, kg + rowoff + c * 8, nb);
+                cp_async16(sV + off, vg + rowoff + c * 8, nb);
+            }
+            cp_async_commit();
+            cp_async_wait<0>();
+            fence_proxy_async();
+            mbar_arrive(bar_g);
+        }
+        const float c2 = scale * kLog2e;
+        const uint32_t lane_base = ((uint32_t)(warp * 32)) << 16;
+        // per-column constants of the next block, fetched one block ahead: thread c < 64 holds L2, thread 64 + c delta
+        auto col_fetch = [&](int t) -> float {
+            const int i = ib_start + t * 64 + (tid & 63);
+            if (t >= n_blk || i >= Tlen) return tid < 64 ? INFINITY : 0.f;      // L2 = +inf makes P = 0
+            return tid < 64 ? lse[(size_t)bh * Tlen + i] * kLog2e : delta[(size_t)bh * Tlen + i];
+        };
+        float col_next = col_fetch(0);
+
+        for (int t = 0; t < n_blk; ++t) {
+            group_sync();                                      // everyone is done with the previous block's constants
+            s_col[tid] = col_next;
+            col_next = col_fetch(t + 1);
+            group_sync();
+            const int ib = ib_start + t * 64;
+            int c_lo, c_hi;                                    // query columns of the block this key row may be seen by
+            if (pos < 0) { c_lo = 1 << 20; c_hi = -(1 << 20); }
+            else if (!is_ret) { c_lo = pos - ib; c_hi = min(pos + W - 1, Tlen - 1) - ib; }
+            else { c_lo = pos + W - ib; c_hi = Tlen - 1 - ib; }
+            const int u_lo = __reduce_min_sync(0xffffffffu, c_lo), u_hi = __reduce_max_sync(0xffffffffu, c_hi);
+
+            bwait(bar_s, t & 1, 3);                            // S^T(t), dP^T(t) are in TMEM
+            tc_fence_after();
+            uint32_t pp[32], pd[32];                           // P^T and dS^T rows as 64 bf16 each
+#pragma unroll
+            for (int cb = 0; cb < 2; ++cb) {
+                const bool act = cb * 32 <= u_hi && cb * 32 + 31 >= u_lo;
+                if (act) {
+                    uint32_t rs[32], rp[32];
+                    tmem_ld32(tmem + lane_base + cb * 32, rs);
+                    tmem_ld32(tmem + lane_base + DP_COL + cb * 32, rp);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int c = 0; c < 32; c += 4) {
+                        const int col = cb * 32 + c;
+                        const float4 l4 = *reinterpret_cast<const float4*>(&s_col[col]);
+                        const float4 d4 = *reinterpret_cast<const float4*>(&s_col[64 + col]);
+                        const float lv[4] = {l4.x, l4.y, l4.z, l4.w}, dvv[4] = {d4.x, d4.y, d4.z, d4.w};
+                        float p[4], ds[4];
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const bool ok = col + u >= c_lo && col + u <= c_hi;
+                            p[u] = ok ? fast_exp2(fmaf(__uint_as_float(rs[c + u]), c2, -lv[u])) : 0.f;
+                            ds[u] = p[u] * (__uint_as_float(rp[c + u]) - dvv[u]) * scale;
+                        }
+                        __nv_bfloat162 h0 = __floats2bfloat162_rn(p[0], p[1]), h1 = __floats2bfloat162_rn(p[2], p[3]);
+                        __nv_bfloat162 g0 = __floats2bfloat162_rn(ds[0], ds[1]), g1 = __floats2bfloat162_rn(ds[2], ds[3]);
+                        pp[cb * 16 + (c >> 1)] = *reinterpret_cast<uint32_t*>(&h0);
+                        pp[cb * 16 + (c >> 1) + 1] = *reinterpret_cast<uint32_t*>(&h1);
+                        pd[cb * 16 + (c >> 1)] = *reinterpret_cast<uint32_t*>(&g0);
+                        pd[cb * 16 + (c >> 1) + 1] = *reinterpret_cast<uint32_t*>(&g1);
+                    }
+                } else {
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) { pp[cb * 16 + c] = 0u; pd[cb * 16 + c] = 0u; }
+                }
+            }
+            if (t > 0) { bwait(bar_pv, (t - 1) & 1, 4); tc_fence_after(); }   // the MMAs reading the old operands are done
+#pragma unroll
+            for (int ch = 0; ch < 8; ++ch) {
+                const uint32_t off = tid * 128 + ((ch ^ (tid & 7)) << 4);
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sPT + off), "r"(pp[4 * ch]), "r"(pp[4 * ch + 1]),
+                             "r"(pp[4 * ch + 2]), "r"(pp[4 * ch + 3]) : "memory");
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sDST + off), "r"(pd[4 * ch]), "r"(pd[4 * ch + 1]),
+                             "r"(pd[4 * ch + 2]), "r"(pd[4 * ch + 3]) : "memory");
+            }
+            fence_proxy_async();
+            tc_fence_before();
+            mbar_arrive(bar_p);
+        }
+        if (n_blk > 0) { bwait(bar_pv, (n_blk - 1) & 1, 5); tc_fence_after(); }
+
+        // ---- epilogue: dV, dK rows and Eq. 6's <v_j, dV_j> ------------------------------------------------------
+        float dr = 0.f;
+        const bool live = pos >= 0;
+        const size_t orow = is_ret ? ((size_t)bh * R + e0 + tid) * D : ((size_t)bh * Tlen + (live ? pos : 0)) * D;
+#pragma unroll
+        for (int half2 = 0; half2 < 2; ++half2) {              // 0: dV, 1: dK
+#pragma unroll
+            for (int cb = 0; cb < D / 32; ++cb) {
+                uint32_t a4[32];
+                if (n_blk > 0) {
+                    tmem_ld32(tmem + lane_base + (half2 ? DK_COL : DV_COL) + cb * 32, a4);
+                    tmem_wait_ld();
+                } else {
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) a4[c] = 0u;
+                }
+                if (half2 == 0) {
+                    // v row of this key from the swizzled tile in shared memory
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        const int ch = cb * 4 + g;             // 16-byte chunk index within the row
+                        const uint4 u = *reinterpret_cast<const uint4*>(smem_raw + S::OFF_V + (ch >> 3) * 16384 + tid * 128 +
+                                                                        (((ch & 7) ^ (tid & 7)) << 4));
+                        const uint32_t w4[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+                        for (int x = 0; x < 4; ++x) {
+                            dr = fmaf(__uint_as_float(w4[x] << 16), __uint_as_float(a4[g * 8 + 2 * x]), dr);
+                            dr = fmaf(__uint_as_float(w4[x] & 0xffff0000u), __uint_as_float(a4[g * 8 + 2 * x + 1]), dr);
+                        }
+                    }
+                }
+                if (live) {
+                    if (is_ret || F32OUT) {
+                        float* dst = (is_ret ? (half2 ? dk_ret : dv_ret) : (half2 ? dk32 : dv32)) + orow + cb * 32;
+#pragma unroll
+                        for (int c = 0; c < 32; c += 4)
+                            *reinterpret_cast<float4*>(dst + c) = make_float4(__uint_as_float(a4[c]), __uint_as_float(a4[c + 1]),
+                                                                              __uint_as_float(a4[c + 2]), __uint_as_float(a4[c + 3]));
+                    } else {
+                        __nv_bfloat16* dst = (half2 ? dk : dv) + orow + cb * 32;
+#pragma unroll
+                        for (int c = 0; c < 32; c += 8) {
+                            uint32_t w4[4];
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) {
+                                __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(a4[c + 2 * u]), __uint_as_float(a4[c + 2 * u + 1]));
+                                w4[u] = *reinterpret_cast<uint32_t*>(&h);
+                            }
+                            *reinterpret_cast<uint4*>(dst + c) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+                        }
+                    }
+                }
+            }
+        }
+        if (live) {
+            if (is_ret) dr_ret[(size_t)bh * R + e0 + tid] = dr;
+            else dr_win[(size_t)bh * Tlen + pos] = dr;
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 4) tmem_dealloc(tmem, S::TMEM_COLS);
+}
+
+// Far-query share of the retained keys added onto their rows (each key appears once in the list: fixed order).
+template <bool F32OUT>
+__global__ void bwd_merge_kernel(const int32_t* __restrict__ idx, const int32_t* __restrict__ cnt,
+                                 const float* __restrict__ dk_ret, const float* __restrict__ dv_ret,
+                                 const float* __restrict__ dr_ret, __nv_bfloat16* __restrict__ dk,
+                                 __nv_bfloat16* __restrict__ dv, float* __restrict__ dk32, float* __restrict__ dv32,
+                                 float* __restrict__ dr_win, int Tlen, int R, int D)
+{
+    const int bh = blockIdx.y, e = blockIdx.x;
+    if (e >= cnt[bh]) return;
+    const int j = idx[(size_t)bh * R + e];
+    const size_t src = ((size_t)bh * R + e) * D, dst = ((size_t)bh * Tlen + j) * D;
+    for (int c = threadIdx.x; c < D; c += blockDim.x) {
+        if (F32OUT) { dk32[dst + c] += dk_ret[src + c]; dv32[dst + c] += dv_ret[src + c]; }
+        else {
+            dk[dst + c] = __float2bfloat16_rn(__bfloat162float(dk[dst + c]) + dk_ret[src + c]);
+            dv[dst + c] = __float2bfloat16_rn(__bfloat162float(dv[dst + c]) + dv_ret[src + c]);
+        }
+    }
+    if (threadIdx.x == 0) dr_win[(size_t)bh * Tlen + j] += dr_ret[(size_t)bh * R + e];
+}
+
+// dr -> dz in place: Eq. 6 (+ Eq. 7's lambda term) through the sigmoid, for scored tokens only.
+__global__ void bwd_dz_kernel(float* __restrict__ dz, const float* __restrict__ z, const float* __restrict__ lambda, int H,
+                              int Tlen, int half, float zthr)
+{
+    const int bh = blockIdx.y;
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= Tlen) return;
+    float g = 0.f;
+    if (j + half <= Tlen - 1) {
+        const float zz = z[(size_t)bh * Tlen + j];
+        const float r = 1.f / (1.f + expf(-zz));
+        float dr = dz[(size_t)bh * Tlen + j];
+        if (lambda && zz > zthr) dr += lambda[bh % H];
+        g = dr * r * (1.f - r);
+    }
+    dz[(size_t)bh * Tlen + j] = g;
+}
+
 }  // namespace
 
 // dq (and delta) on the tensor cores.  Returns LTE_OK or an error; the caller runs the remaining stages.
@@ -365,6 +701,59 @@ int launch_bwd_dq_tc(const Params& p, const void* q, const void* k, const void* 
     } while (0)
     if (p.d == 64) LTE_GO(64); else if (p.d == 128) LTE_GO(128); else return LTE_ERR_UNSUPPORTED;
 #undef LTE_GO
+    return cuda_status(cudaGetLastError());
+}
+
+// dk, dv, dz on the tensor cores.  `ret_ws` holds dk_ret, dv_ret [B,H,R,d] and dr_ret [B,H,R] (fp32).
+size_t bwd_tc_ret_bytes(const Params& p)
+{
+    const size_t n = (size_t)p.B * p.H * (p.R > 0 ? p.R : 1);
+    return ((2 * n * p.d + n) * 4 + 255) / 256 * 256;
+}
+
+int launch_bwd_dkv_tc(const Params& p, const void* q, const void* k, const void* v, const float* lse, const void* dO,
+                      const float* delta, const float* z, const int32_t* idx, const int32_t* cnt, const float* lambda,
+                      void* dk, void* dv, float* dk32, float* dv32, float* dz, void* ret_ws, bool f32out, cudaStream_t st)
+{
+    const int BH = p.B * p.H;
+    CUtensorMap tk, tv, tq, tdo;
+    if (!make_map(&tk, k, BH, p.T, p.d, 128) || !make_map(&tv, v, BH, p.T, p.d, 128) ||
+        !make_map(&tq, q, BH, p.T, p.d, 64) || !make_map(&tdo, dO, BH, p.T, p.d, 64))
+        return LTE_ERR_CUDA;
+    const size_t n = (size_t)BH * (p.R > 0 ? p.R : 1);
+    float* dk_ret = (float*)ret_ws;
+    float* dv_ret = dk_ret + n * p.d;
+    float* dr_ret = dv_ret + n * p.d;
+    const int n_wt = (p.T + 127) / 128, n_rt = (p.R + 127) / 128;
+    dim3 grid(n_wt + n_rt, BH);
+#define LTE_GO(D, F)                                                                                               \
+    do {                                                                                                           \
+        static bool attr_done = false;                                                                             \
+        if (!attr_done) {                                                                                          \
+            if (cudaFuncSetAttribute(bwd_dkv_tc_kernel<D, F>, cudaFuncAttributeMaxDynamicSharedMemorySize,          \
+                                     SmemK<D>::BYTES) != cudaSuccess) return LTE_ERR_CUDA;                         \
+            attr_done = true;                                                                                      \
+        }                                                                                                          \
+        bwd_dkv_tc_kernel<D, F><<<grid, NTHREADS, SmemK<D>::BYTES, st>>>(                                           \
+            tk, tv, tq, tdo, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, lse, delta, idx, cnt,               \
+            (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, dk32, dv32, dz, dk_ret, dv_ret, dr_ret, n_wt, p.T, p.W, p.R,   \
+            p.scale);                                                                                              \
+    } while (0)
+    if (p.d == 64) { if (f32out) LTE_GO(64, true); else LTE_GO(64, false); }
+    else if (p.d == 128) { if (f32out) LTE_GO(128, true); else LTE_GO(128, false); }
+    else return LTE_ERR_UNSUPPORTED;
+#undef LTE_GO
+    if (p.R > 0) {
+        dim3 gm(p.R, BH);
+        if (f32out)
+            bwd_merge_kernel<true><<<gm, 64, 0, st>>>(idx, cnt, dk_ret, dv_ret, dr_ret, (__nv_bfloat16*)dk, (__nv_bfloat16*)dv,
+                                                      dk32, dv32, dz, p.T, p.R, p.d);
+        else
+            bwd_merge_kernel<false><<<gm, 64, 0, st>>>(idx, cnt, dk_ret, dv_ret, dr_ret, (__nv_bfloat16*)dk, (__nv_bfloat16*)dv,
+                                                       dk32, dv32, dz, p.T, p.R, p.d);
+    }
+    dim3 gz((p.T + 255) / 256, BH);
+    bwd_dz_kernel<<<gz, 256, 0, st>>>(dz, z, lambda, p.H, p.T, p.half, p.zthr);
     return cuda_status(cudaGetLastError());
 }
 
