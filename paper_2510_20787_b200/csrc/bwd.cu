@@ -184,6 +184,7 @@ __global__ void bwd_conv_partial_kernel(const T* __restrict__ k, const T* __rest
     const T* src = c < D ? k : v;
     const int cc = c < D ? c : c - D;
     const int pend = p0 + CHUNK < Tlen ? p0 + CHUNK : Tlen;
+#pragma unroll 8
     for (int p = p0; p < pend; ++p) {
         const float x = to_f(src[((size_t)bh * Tlen + p) * D + cc]);
 #pragma unroll
@@ -246,6 +247,63 @@ __global__ void bwd_finish_kernel(const float* __restrict__ dk32, const float* _
     }
 }
 
+// Tensor-core path: the scorer's input gradient sum_t dz[p-t+half] w[h,t,c] added in place onto the bf16 dk, dv rows.
+// A block takes ROWS consecutive positions of one (b,h); 8 channels per thread, weights and the dz window in shared memory.
+template <int D>
+__global__ void __launch_bounds__(256) bwd_finish_inplace_kernel(const float* __restrict__ dz, const float* __restrict__ w,
+                                                                 __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv,
+                                                                 int H, int Tlen, int K)
+{
+    constexpr int TPR = D / 8;                      // threads per row
+    constexpr int RPP = 256 / TPR;                  // rows per pass
+    constexpr int ROWS = 4 * RPP;
+    extern __shared__ float sm[];
+    float* ws = sm;                                 // [K][2D]
+    float* dzs = sm + K * 2 * D;                    // dz[p0-half .. p0+ROWS-1+half]
+    const int half = K / 2;
+    const int bh = blockIdx.y, h = bh % H;
+    const int p0 = blockIdx.x * ROWS;
+    for (int i = threadIdx.x; i < K * 2 * D; i += 256) ws[i] = w[(size_t)h * K * 2 * D + i];
+    for (int a = threadIdx.x; a < ROWS + K - 1; a += 256) {
+        const int j = p0 - half + a;
+        dzs[a] = (j >= 0 && j + half <= Tlen - 1) ? dz[(size_t)bh * Tlen + j] : 0.f;
+    }
+    __syncthreads();
+    const int cc = (threadIdx.x % TPR) * 8, r0 = threadIdx.x / TPR;
+#pragma unroll
+    for (int ps = 0; ps < 4; ++ps) {
+        const int rl = ps * RPP + r0, p = p0 + rl;
+        if (p >= Tlen) break;
+        float gk[8], gv[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) { gk[e] = 0.f; gv[e] = 0.f; }
+        for (int t = 0; t < K; ++t) {
+            const float g = dzs[rl - t + 2 * half];          // dz[p - t + half]
+            const float4* wk = reinterpret_cast<const float4*>(&ws[(t * 2) * D + cc]);
+            const float4* wv = reinterpret_cast<const float4*>(&ws[(t * 2 + 1) * D + cc]);
+            const float4 a = wk[0], b = wk[1], c = wv[0], d = wv[1];
+            gk[0] = fmaf(g, a.x, gk[0]); gk[1] = fmaf(g, a.y, gk[1]); gk[2] = fmaf(g, a.z, gk[2]); gk[3] = fmaf(g, a.w, gk[3]);
+            gk[4] = fmaf(g, b.x, gk[4]); gk[5] = fmaf(g, b.y, gk[5]); gk[6] = fmaf(g, b.z, gk[6]); gk[7] = fmaf(g, b.w, gk[7]);
+            gv[0] = fmaf(g, c.x, gv[0]); gv[1] = fmaf(g, c.y, gv[1]); gv[2] = fmaf(g, c.z, gv[2]); gv[3] = fmaf(g, c.w, gv[3]);
+            gv[4] = fmaf(g, d.x, gv[4]); gv[5] = fmaf(g, d.y, gv[5]); gv[6] = fmaf(g, d.z, gv[6]); gv[7] = fmaf(g, d.w, gv[7]);
+        }
+        const size_t a0 = ((size_t)bh * Tlen + p) * D + cc;
+        uint4 uk = *reinterpret_cast<const uint4*>(dk + a0), uv = *reinterpret_cast<const uint4*>(dv + a0);
+        uint32_t kw[4] = {uk.x, uk.y, uk.z, uk.w}, vw[4] = {uv.x, uv.y, uv.z, uv.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            __nv_bfloat162 hk = __floats2bfloat162_rn(__uint_as_float(kw[e] << 16) + gk[2 * e],
+                                                      __uint_as_float(kw[e] & 0xffff0000u) + gk[2 * e + 1]);
+            __nv_bfloat162 hv = __floats2bfloat162_rn(__uint_as_float(vw[e] << 16) + gv[2 * e],
+                                                      __uint_as_float(vw[e] & 0xffff0000u) + gv[2 * e + 1]);
+            kw[e] = *reinterpret_cast<uint32_t*>(&hk);
+            vw[e] = *reinterpret_cast<uint32_t*>(&hv);
+        }
+        *reinterpret_cast<uint4*>(dk + a0) = make_uint4(kw[0], kw[1], kw[2], kw[3]);
+        *reinterpret_cast<uint4*>(dv + a0) = make_uint4(vw[0], vw[1], vw[2], vw[3]);
+    }
+}
+
 struct WsPlan { size_t delta, dz, part_w, part_b, dk32, dv32, ret, total; int nchunk; };
 WsPlan plan(const Params& p, uint32_t flags)
 {
@@ -259,12 +317,13 @@ WsPlan plan(const Params& p, uint32_t flags)
     w.part_w = off; off += up((size_t)p.H * p.B * w.nchunk * p.K * 2 * p.d * 4);
     w.part_b = off; off += up((size_t)p.H * p.B * w.nchunk * 4);
     w.dk32 = w.dv32 = 0;
-    if (flags & LTE_BWD_CNN_INPUT_GRAD) {
+    const bool tc_path = p.dtype == LTE_BF16 && (p.d == 64 || p.d == 128);
+    if ((flags & LTE_BWD_CNN_INPUT_GRAD) && !tc_path) {
         w.dk32 = off; off += up(bht * p.d * 4);
         w.dv32 = off; off += up(bht * p.d * 4);
     }
     w.ret = off;
-    if (p.dtype == LTE_BF16 && (p.d == 64 || p.d == 128)) off += bwd_tc_ret_bytes(p);   // tensor-core path: retained-tile shares
+    if (tc_path) off += bwd_tc_ret_bytes(p);        // tensor-core path: retained-tile shares
     w.total = off;
     return w;
 }
@@ -293,7 +352,7 @@ int run(const Params& p, const void* q, const void* k, const void* v, const void
     }
     if constexpr (sizeof(T) == 2 && (D == 64 || D == 128)) {
         const int e = launch_bwd_dkv_tc(p, q, k, v, lse, dO, delta, z, idx, cnt, lambda, dk, dv, dk32, dv32, dz, base + w.ret,
-                                        f32, st);
+                                        false, st);
         if (e != LTE_OK) return e;
     } else if (f32) {
         bwd_dkv_kernel<T, D, true><<<grid, 128, 0, st>>>((const T*)q, (const T*)k, (const T*)v, (const T*)dO, lse, delta,
@@ -311,8 +370,15 @@ int run(const Params& p, const void* q, const void* k, const void* v, const void
     dim3 gr((per_head + 255) / 256, p.H);
     bwd_conv_reduce_kernel<<<gr, 256, 0, st>>>(part_w, part_b, dw, dbias, p.B * w.nchunk, per_head);
     if (f32) {
-        dim3 gf(min((p.T * D + 255) / 256, 1024), p.B * p.H);
-        bwd_finish_kernel<T><<<gf, 256, 0, st>>>(dk32, dv32, dz, p.w, (T*)dk, (T*)dv, p.H, p.T, D, p.K);
+        if constexpr (sizeof(T) == 2 && (D == 64 || D == 128)) {
+            constexpr int ROWS = 4 * (256 / (D / 8));
+            dim3 gf((p.T + ROWS - 1) / ROWS, p.B * p.H);
+            const size_t sm = (size_t)(p.K * 2 * D + ROWS + p.K - 1) * sizeof(float);
+            bwd_finish_inplace_kernel<D><<<gf, 256, sm, st>>>(dz, p.w, (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, p.H, p.T, p.K);
+        } else {
+            dim3 gf(min((p.T * D + 255) / 256, 1024), p.B * p.H);
+            bwd_finish_kernel<T><<<gf, 256, 0, st>>>(dk32, dv32, dz, p.w, (T*)dk, (T*)dv, p.H, p.T, D, p.K);
+        }
     }
     return cuda_status(cudaGetLastError());
 }
