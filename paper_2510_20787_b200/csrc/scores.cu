@@ -5,7 +5,7 @@
 // the logit of token j is then the shifted diagonal sum_t Y[j+t-half][t], taken from shared memory.
 // A block of NT threads covers NT rows and emits NT-(K-1) logits; the K-1 halo rows are recomputed by
 // the neighbouring block.  HBM traffic: 2*d elements read and one fp32 written per token and head.
-#include "tma_util.cuh"
+#include "tc_common.cuh"
 
 namespace lte {
 namespace {
@@ -97,101 +97,173 @@ __global__ void __launch_bounds__(NT) scores_kernel(const T* __restrict__ k, con
     }
 }
 
-// ---- bf16, d = 64 or 128: the tile of input rows is staged by TMA -----------------------------------------------
-// A block takes NT consecutive input rows of one (b,h): one cp.async.bulk.tensor box per 64-column sub-tile of k and
-// of v (128-byte swizzle, so that thread r reading row r is bank-conflict free), rows left of position 0 or right of
-// T-1 arriving as zeros, which is exactly the scorer's zero padding.  HBM is read by the copy engine only; the
-// threads spend their issue slots on the K partial dot products per row (weights broadcast from shared memory).
-__device__ __forceinline__ uint32_t s_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+// ---- bf16, d = 64 or 128: TMA-staged tiles, the K partial dot products per row on the tensor cores -----------------
+// Y[p][t] = <w_t, x_p> for a tile of 128 input rows is the small GEMM  X[128 x 2d] * Wt[2d x K]:
+//   A = the tile of k rows, then of v rows, exactly as TMA delivers them (128-byte swizzle, K-major); rows left of
+//       position 0 or right of T-1 arrive as zeros, which is the scorer's zero padding;
+//   B = the fp32 weights split into three bf16 pieces (hi + mid + lo reproduces all 24 mantissa bits, and
+//       bf16 x bf16 products are exact in the fp32 accumulator), one B row per (piece, tap), built in shared memory;
+//   D = fp32 in TMEM; the thread owning row p adds the three pieces and the block takes the shifted diagonal sum.
+// HBM is touched by the copy engine only; the kernel is bound by HBM bandwidth, not by the fp32 ALUs.
+using namespace tc;
 
+template <int D, int K> struct ScoresTc {
+    static constexpr int SUB = D / 64;
+    static constexpr int NB = (3 * K + 15) / 16 * 16;    // B rows = accumulator columns (multiple of 16)
+    static constexpr int NSTAGE = D == 64 ? 3 : 2;       // input-tile stages (each: k tile + v tile)
+    static constexpr int STAGE = 2 * SUB * 16384;
+    static constexpr int B_SLOT = NB * 128;              // bytes of one [NB][64] sub-tile of B (a multiple of 1024)
+    static constexpr int OFF_B = NSTAGE * STAGE, OFF_YS = OFF_B + 2 * SUB * B_SLOT, OFF_BAR = OFF_YS + NT * K * 4;
+    static constexpr int BYTES = OFF_BAR + 64;
+    static constexpr uint32_t ACC_COLS = NB <= 32 ? 32 : 64;   // columns of one accumulator buffer (two buffers)
+};
+
+// A CTA walks `tiles_per_cta` consecutive row tiles of one (b,h): B is built once, the input tiles stream through an
+// NSTAGE ring (TMA), the MMA of tile i+1 runs while the threads take tile i out of TMEM (two accumulator buffers).
 template <int D, int K>
-__global__ void __launch_bounds__(NT) scores_tma_kernel(const __grid_constant__ CUtensorMap tmK,
-                                                        const __grid_constant__ CUtensorMap tmV,
-                                                        const float* __restrict__ w, const float* __restrict__ bias,
-                                                        float* __restrict__ z, float* __restrict__ r, int H, int Tlen,
-                                                        int* __restrict__ status)
+__global__ void __launch_bounds__(NT) scores_tc_kernel(const __grid_constant__ CUtensorMap tmK,
+                                                       const __grid_constant__ CUtensorMap tmV,
+                                                       const float* __restrict__ w, const float* __restrict__ bias,
+                                                       float* __restrict__ z, float* __restrict__ r, int H, int Tlen,
+                                                       int tiles_per_cta, int* __restrict__ status)
 {
+    using C = ScoresTc<D, K>;
     constexpr int HALF = K / 2;
     constexpr int TJ = NT - (K - 1);
-    constexpr int SUB = D / 64;
+    constexpr int SUB = C::SUB, NB = C::NB, NSTAGE = C::NSTAGE;
+    constexpr uint32_t TMEM_COLS = 2 * C::ACC_COLS;
     extern __shared__ __align__(1024) uint8_t smem[];
-    // [k tile: SUB x 16 KB][v tile: SUB x 16 KB][weights K*2D floats][ys NT*K floats][mbarrier]
-    float* ws = reinterpret_cast<float*>(smem + 2 * SUB * 16384);
-    float* ys = ws + K * 2 * D;
-    const uint32_t bar = s_u32(ys + NT * K);
-    const uint32_t tile = s_u32(smem);
+    float* ys = reinterpret_cast<float*>(smem + C::OFF_YS);
+    const uint32_t tile0 = smem_u32(smem);
+    const uint32_t bar_ld0 = tile0 + C::OFF_BAR, bar_mma0 = bar_ld0 + 8 * NSTAGE, tmem_slot = bar_mma0 + 16;
+    volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(smem + C::OFF_BAR + 8 * NSTAGE + 16);
     const int bh = blockIdx.y, h = bh % H;
-    const int j0 = blockIdx.x * TJ;
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int n_all = (Tlen + TJ - 1) / TJ;
+    const int t_begin = blockIdx.x * tiles_per_cta;
+    const int n_tiles = min(tiles_per_cta, n_all - t_begin);
+    if (n_tiles <= 0) return;
 
-    if ((tile & 1023u) != 0) { if (tid == 0) atomicExch(status, 8); return; }
-    if (tid == 0) {
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar));
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(2 * SUB * 16384) : "memory");
+    if ((tile0 & 1023u) != 0) { if (tid == 0) atomicExch(status, 8); return; }
+    auto issue_tile = [&](int i) {                       // thread 0
+        const uint32_t dst = tile0 + (i % NSTAGE) * C::STAGE, bar = bar_ld0 + 8 * (i % NSTAGE);
+        const int y = (t_begin + i) * TJ - HALF;
+        mbar_expect_tx(bar, C::STAGE);
 #pragma unroll
         for (int sb = 0; sb < SUB; ++sb) {
-            asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-                         ::"r"(tile + sb * 16384), "l"(&tmK), "r"(sb * 64), "r"(j0 - HALF), "r"(bh), "r"(bar) : "memory");
-            asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-                         ::"r"(tile + (SUB + sb) * 16384), "l"(&tmV), "r"(sb * 64), "r"(j0 - HALF), "r"(bh), "r"(bar) : "memory");
+            tma_load_3d(dst + sb * 16384, &tmK, sb * 64, y, bh, bar);
+            tma_load_3d(dst + (SUB + sb) * 16384, &tmV, sb * 64, y, bh, bar);
         }
+    };
+    if (tid == 0) {
+#pragma unroll
+        for (int s2 = 0; s2 < NSTAGE; ++s2) mbar_init(bar_ld0 + 8 * s2, 1);
+        mbar_init(bar_mma0, 1); mbar_init(bar_mma0 + 8, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        for (int i = 0; i < NSTAGE && i < n_tiles; ++i) issue_tile(i);
     }
-    for (int i = tid; i < K * 2 * D; i += NT) ws[i] = w[(size_t)h * K * 2 * D + i];
-    __syncthreads();
-    if (tid == 0) {                                     // one thread polls (bounded), the block barrier releases the rest
-        uint32_t ok = 0;
-        for (uint32_t it = 0; it < (1u << 22) && !ok; ++it)
-            asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                         : "=r"(ok) : "r"(bar) : "memory");
-        if (!ok) atomicExch(status, 7);
-    }
-    __syncthreads();
-
-    float acc[K];
+    if (warp == 0) { __syncwarp(); tmem_alloc(tmem_slot, TMEM_COLS); }
+    // B: row n = piece * K + t, columns = the 2d input channels (k part, then v part); zero rows above 3K
+    for (int e = tid; e < NB * 2 * D / 8; e += NT) {     // one 16-byte chunk (8 channels) of one row per iteration
+        const int n = e / (2 * D / 8), c8 = e % (2 * D / 8);
+        const int piece = n / K, t = n % K;
+        uint32_t pk[4] = {0u, 0u, 0u, 0u};
+        if (n < 3 * K) {
+            const float4* src = reinterpret_cast<const float4*>(w + ((size_t)h * K + t) * 2 * D + c8 * 8);
+            const float4 f0 = src[0], f1 = src[1];
+            const float wv8[8] = {f0.x, f0.y, f0.z, f0.w, f1.x, f1.y, f1.z, f1.w};
 #pragma unroll
-    for (int t = 0; t < K; ++t) acc[t] = 0.f;
+            for (int u = 0; u < 4; ++u) {
+                float v2[2];
 #pragma unroll
-    for (int part = 0; part < 2; ++part) {
-#pragma unroll
-        for (int sb = 0; sb < SUB; ++sb) {
-            const uint8_t* rowp = smem + (part * SUB + sb) * 16384 + tid * 128;
-#pragma unroll 2
-            for (int ch = 0; ch < 8; ++ch) {
-                const uint4 u = *reinterpret_cast<const uint4*>(rowp + ((ch ^ (tid & 7)) << 4));
-                const uint32_t wd[4] = {u.x, u.y, u.z, u.w};
-                float x[8];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) { x[2 * i] = __uint_as_float(wd[i] << 16); x[2 * i + 1] = __uint_as_float(wd[i] & 0xffff0000u); }
-                const int c = sb * 64 + ch * 8;
-#pragma unroll
-                for (int t = 0; t < K; ++t) {
-                    const float4* wv = reinterpret_cast<const float4*>(&ws[(t * 2 + part) * D + c]);
-                    const float4 a = wv[0], b = wv[1];
-                    acc[t] = fmaf(x[0], a.x, acc[t]); acc[t] = fmaf(x[1], a.y, acc[t]);
-                    acc[t] = fmaf(x[2], a.z, acc[t]); acc[t] = fmaf(x[3], a.w, acc[t]);
-                    acc[t] = fmaf(x[4], b.x, acc[t]); acc[t] = fmaf(x[5], b.y, acc[t]);
-                    acc[t] = fmaf(x[6], b.z, acc[t]); acc[t] = fmaf(x[7], b.w, acc[t]);
+                for (int x = 0; x < 2; ++x) {
+                    const float wv = wv8[2 * u + x];
+                    const float hi = __bfloat162float(__float2bfloat16_rn(wv));
+                    const float mid = __bfloat162float(__float2bfloat16_rn(wv - hi));
+                    const float lo = __bfloat162float(__float2bfloat16_rn((wv - hi) - mid));
+                    v2[x] = piece == 0 ? hi : (piece == 1 ? mid : lo);
                 }
+                __nv_bfloat162 h2 = __floats2bfloat162_rn(v2[0], v2[1]);
+                pk[u] = *reinterpret_cast<uint32_t*>(&h2);
             }
         }
+        const int sub = c8 / 8, ch = c8 % 8;             // 64-column sub-tile (k: 0..SUB-1, v: SUB..2SUB-1), chunk in row
+        const uint32_t dst = tile0 + C::OFF_B + sub * C::B_SLOT + n * 128 + ((ch ^ (n & 7)) << 4);
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]) : "memory");
     }
-#pragma unroll
-    for (int t = 0; t < K; ++t) ys[tid * K + t] = acc[t];
+    fence_proxy_async();
+    tc_fence_before();
     __syncthreads();
-    const int j = j0 + tid;
-    if (tid < TJ && j < Tlen) {
-        float zz;
-        if (j + HALF > Tlen - 1) {
-            zz = -INFINITY;
-        } else {
-            zz = bias ? bias[h] : 0.f;
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot_gen;
+    constexpr uint32_t IDESC = instr_desc(128, NB, false);
+    const uint32_t b_lo = desc_lo(tile0 + C::OFF_B, 16);
+    auto mma_tile = [&](int i) {                         // thread 0: wait for the tile, issue its MMAs
+        mbar_wait_s(bar_ld0 + 8 * (i % NSTAGE), (i / NSTAGE) & 1, 7, status);
+        tc_fence_after();
+        const uint32_t a_lo = desc_lo(tile0 + (i % NSTAGE) * C::STAGE, 16);
+        const uint32_t dcol = tmem + (i & 1) * C::ACC_COLS;
 #pragma unroll
-            for (int t = 0; t < K; ++t) zz += ys[(tid + t) * K + t];
+        for (int kk = 0; kk < 2 * D / 16; ++kk)           // 2d input channels, 16 per instruction
+            umma(dcol, desc64(a_lo + (kk >> 2) * 1024 + (kk & 3) * 2, kDescHi),
+                 desc64(b_lo + (kk >> 2) * (C::B_SLOT >> 4) + (kk & 3) * 2, kDescHi), IDESC, kk > 0);
+        umma_commit(bar_mma0 + 8 * (i & 1));
+    };
+    if (tid == 0) mma_tile(0);
+    const uint32_t lane_base = ((uint32_t)(warp * 32)) << 16;
+    const float bh_bias = bias ? bias[h] : 0.f;
+
+    for (int i = 0; i < n_tiles; ++i) {
+        if (tid == 0 && i + 1 < n_tiles) mma_tile(i + 1);   // runs while tile i is taken out of TMEM below
+        mbar_wait_s(bar_mma0 + 8 * (i & 1), (i >> 1) & 1, 6, status);
+        tc_fence_after();
+        {
+            const uint32_t col = tmem + lane_base + (i & 1) * C::ACC_COLS;
+            uint32_t acc[32];
+            tmem_ld32(col, acc);
+            float y[K];
+            if constexpr (NB <= 32) {
+                tmem_wait_ld();
+#pragma unroll
+                for (int t = 0; t < K; ++t)
+                    y[t] = (__uint_as_float(acc[2 * K + t]) + __uint_as_float(acc[K + t])) + __uint_as_float(acc[t]);
+            } else {
+                uint32_t acc2[32];
+                tmem_ld32(col + 32, acc2);
+                tmem_wait_ld();
+#pragma unroll
+                for (int t = 0; t < K; ++t) {
+                    const int i0 = t, i1 = K + t, i2 = 2 * K + t;
+                    const float a0 = __uint_as_float(i0 < 32 ? acc[i0] : acc2[i0 - 32]);
+                    const float a1 = __uint_as_float(i1 < 32 ? acc[i1] : acc2[i1 - 32]);
+                    const float a2 = __uint_as_float(i2 < 32 ? acc[i2] : acc2[i2 - 32]);
+                    y[t] = (a2 + a1) + a0;
+                }
+            }
+#pragma unroll
+            for (int t = 0; t < K; ++t) ys[tid * K + t] = y[t];
         }
-        z[(size_t)bh * Tlen + j] = zz;
-        if (r) r[(size_t)bh * Tlen + j] = 1.f / (1.f + __expf(-zz));
+        tc_fence_before();
+        __syncthreads();                                 // ys complete; accumulator buffer i & 1 and stage i % NSTAGE are free
+        if (tid == 0 && i + NSTAGE < n_tiles) issue_tile(i + NSTAGE);
+        const int j = (t_begin + i) * TJ + tid;
+        if (tid < TJ && j < Tlen) {
+            float zz;
+            if (j + HALF > Tlen - 1) {
+                zz = -INFINITY;
+            } else {
+                zz = bh_bias;
+#pragma unroll
+                for (int t = 0; t < K; ++t) zz += ys[(tid + t) * K + t];
+            }
+            z[(size_t)bh * Tlen + j] = zz;
+            if (r) r[(size_t)bh * Tlen + j] = 1.f / (1.f + __expf(-zz));
+        }
+        __syncthreads();                                 // ys is rewritten by the next tile
     }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, TMEM_COLS);
 }
 
 __device__ int g_scores_status = 0;
@@ -199,20 +271,30 @@ __device__ int g_scores_status = 0;
 template <int D, int K>
 int run_tma(const Params& p, const void* k, const void* v, float* z, float* r, cudaStream_t st)
 {
+    using C = ScoresTc<D, K>;
     constexpr int TJ = NT - (K - 1);
-    constexpr int SMEM = 2 * (D / 64) * 16384 + (K * 2 * D + NT * K) * 4 + 16;
     CUtensorMap tk, tv;
     if (!make_map(&tk, k, p.B * p.H, p.T, D, NT) || !make_map(&tv, v, p.B * p.H, p.T, D, NT)) return LTE_ERR_CUDA;
     static bool attr_done = false;
     static int* status_ptr = nullptr;
+    static int n_sm = 0;
     if (!attr_done) {
-        if (cudaFuncSetAttribute(scores_tma_kernel<D, K>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess ||
-            cudaGetSymbolAddress((void**)&status_ptr, g_scores_status) != cudaSuccess)
+        int dev = 0;
+        if (cudaFuncSetAttribute(scores_tc_kernel<D, K>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::BYTES) != cudaSuccess ||
+            cudaGetSymbolAddress((void**)&status_ptr, g_scores_status) != cudaSuccess || cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
             return LTE_ERR_CUDA;
         attr_done = true;
     }
-    dim3 grid((p.T + TJ - 1) / TJ, p.B * p.H);
-    scores_tma_kernel<D, K><<<grid, NT, SMEM, st>>>(tk, tv, p.w, p.bias, z, r, p.H, p.T, status_ptr);
+    // tiles per CTA: as many CTAs as fit on the machine at once (two per SM at d = 64, one at d = 128), no second wave
+    const int n_all = (p.T + TJ - 1) / TJ, BH = p.B * p.H;
+    const int slots = n_sm * (D == 64 ? 2 : 1);
+    int per_head = slots / BH;                            // CTAs per head (rounded down: a single wave)
+    if (per_head < 1) per_head = 1;
+    if (per_head > n_all) per_head = n_all;
+    const int tiles_per_cta = (n_all + per_head - 1) / per_head;
+    dim3 grid((n_all + tiles_per_cta - 1) / tiles_per_cta, BH);
+    scores_tc_kernel<D, K><<<grid, NT, C::BYTES, st>>>(tk, tv, p.w, p.bias, z, r, p.H, p.T, tiles_per_cta, status_ptr);
     return cuda_status(cudaGetLastError());
 }
 
