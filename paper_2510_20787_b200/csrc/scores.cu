@@ -106,6 +106,12 @@ __global__ void __launch_bounds__(NT) scores_kernel(const T* __restrict__ k, con
 //   D = fp32 in TMEM; the thread owning row p adds the three pieces and the block takes the shifted diagonal sum.
 // HBM is touched by the copy engine only; the kernel is bound by HBM bandwidth, not by the fp32 ALUs.
 using namespace tc;
+#ifdef LTE_PROFILE
+__device__ long long g_sprof[64];
+#define SPROF(slot) do { if (blockIdx.x == 5 && threadIdx.x == 64 && (slot) < 64) g_sprof[slot] = clock64(); } while (0)
+#else
+#define SPROF(slot) do { } while (0)
+#endif
 
 template <int D, int K> struct ScoresTc {
     static constexpr int SUB = D / 64;
@@ -114,18 +120,18 @@ template <int D, int K> struct ScoresTc {
     static constexpr int STAGE = 2 * SUB * 16384;
     static constexpr int B_SLOT = NB * 128;              // bytes of one [NB][64] sub-tile of B (a multiple of 1024)
     static constexpr int OFF_B = NSTAGE * STAGE, OFF_YS = OFF_B + 2 * SUB * B_SLOT, OFF_BAR = OFF_YS + NT * K * 4;
-    static constexpr int BYTES = OFF_BAR + 64;
+    static constexpr int BYTES = OFF_BAR + 96;
     static constexpr uint32_t ACC_COLS = NB <= 32 ? 32 : 64;   // columns of one accumulator buffer (two buffers)
 };
 
 // A CTA walks `tiles_per_cta` consecutive row tiles of one (b,h): B is built once, the input tiles stream through an
 // NSTAGE ring (TMA), the MMA of tile i+1 runs while the threads take tile i out of TMEM (two accumulator buffers).
 template <int D, int K>
-__global__ void __launch_bounds__(NT) scores_tc_kernel(const __grid_constant__ CUtensorMap tmK,
+__global__ void __launch_bounds__(NT + 64) scores_tc_kernel(const __grid_constant__ CUtensorMap tmK,
                                                        const __grid_constant__ CUtensorMap tmV,
                                                        const float* __restrict__ w, const float* __restrict__ bias,
                                                        float* __restrict__ z, float* __restrict__ r, int H, int Tlen,
-                                                       int tiles_per_cta, int* __restrict__ status)
+                                                       int n_flat, int* __restrict__ status)
 {
     using C = ScoresTc<D, K>;
     constexpr int HALF = K / 2;
@@ -137,133 +143,170 @@ __global__ void __launch_bounds__(NT) scores_tc_kernel(const __grid_constant__ C
     const uint32_t tile0 = smem_u32(smem);
     const uint32_t bar_ld0 = tile0 + C::OFF_BAR, bar_mma0 = bar_ld0 + 8 * NSTAGE, tmem_slot = bar_mma0 + 16;
     volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(smem + C::OFF_BAR + 8 * NSTAGE + 16);
-    const int bh = blockIdx.y, h = bh % H;
     const int tid = threadIdx.x, warp = tid >> 5;
-    const int n_all = (Tlen + TJ - 1) / TJ;
-    const int t_begin = blockIdx.x * tiles_per_cta;
-    const int n_tiles = min(tiles_per_cta, n_all - t_begin);
+    const int n_all = (Tlen + TJ - 1) / TJ;              // row tiles per head
+    // this CTA's share of the flat list of (head, row tile) pairs: an even split, heads may change along the way
+    const int f_begin = (int)(((long long)blockIdx.x * n_flat) / gridDim.x);
+    const int f_end = (int)(((long long)(blockIdx.x + 1) * n_flat) / gridDim.x);
+    const int n_tiles = f_end - f_begin;
     if (n_tiles <= 0) return;
 
     if ((tile0 & 1023u) != 0) { if (tid == 0) atomicExch(status, 8); return; }
-    auto issue_tile = [&](int i) {                       // thread 0
-        const uint32_t dst = tile0 + (i % NSTAGE) * C::STAGE, bar = bar_ld0 + 8 * (i % NSTAGE);
-        const int y = (t_begin + i) * TJ - HALF;
-        mbar_expect_tx(bar, C::STAGE);
-#pragma unroll
-        for (int sb = 0; sb < SUB; ++sb) {
-            tma_load_3d(dst + sb * 16384, &tmK, sb * 64, y, bh, bar);
-            tma_load_3d(dst + (SUB + sb) * 16384, &tmV, sb * 64, y, bh, bar);
-        }
-    };
+    const uint32_t bar_free0 = tmem_slot + 8;            // 2 barriers: accumulator buffer taken out of TMEM (128 arrivals)
+    const uint32_t bar_b = bar_free0 + 16;               // B rebuilt for the next head (128 arrivals)
     if (tid == 0) {
 #pragma unroll
         for (int s2 = 0; s2 < NSTAGE; ++s2) mbar_init(bar_ld0 + 8 * s2, 1);
         mbar_init(bar_mma0, 1); mbar_init(bar_mma0 + 8, 1);
+        mbar_init(bar_free0, 128); mbar_init(bar_free0 + 8, 128); mbar_init(bar_b, 128);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        for (int i = 0; i < NSTAGE && i < n_tiles; ++i) issue_tile(i);
     }
-    if (warp == 0) { __syncwarp(); tmem_alloc(tmem_slot, TMEM_COLS); }
-    // B: row n = piece * K + t, columns = the 2d input channels (k part, then v part); zero rows above 3K
-    for (int e = tid; e < NB * 2 * D / 8; e += NT) {     // one 16-byte chunk (8 channels) of one row per iteration
-        const int n = e / (2 * D / 8), c8 = e % (2 * D / 8);
-        const int piece = n / K, t = n % K;
-        uint32_t pk[4] = {0u, 0u, 0u, 0u};
-        if (n < 3 * K) {
-            const float4* src = reinterpret_cast<const float4*>(w + ((size_t)h * K + t) * 2 * D + c8 * 8);
-            const float4 f0 = src[0], f1 = src[1];
-            const float wv8[8] = {f0.x, f0.y, f0.z, f0.w, f1.x, f1.y, f1.z, f1.w};
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                float v2[2];
-#pragma unroll
-                for (int x = 0; x < 2; ++x) {
-                    const float wv = wv8[2 * u + x];
-                    const float hi = __bfloat162float(__float2bfloat16_rn(wv));
-                    const float mid = __bfloat162float(__float2bfloat16_rn(wv - hi));
-                    const float lo = __bfloat162float(__float2bfloat16_rn((wv - hi) - mid));
-                    v2[x] = piece == 0 ? hi : (piece == 1 ? mid : lo);
-                }
-                __nv_bfloat162 h2 = __floats2bfloat162_rn(v2[0], v2[1]);
-                pk[u] = *reinterpret_cast<uint32_t*>(&h2);
-            }
-        }
-        const int sub = c8 / 8, ch = c8 % 8;             // 64-column sub-tile (k: 0..SUB-1, v: SUB..2SUB-1), chunk in row
-        const uint32_t dst = tile0 + C::OFF_B + sub * C::B_SLOT + n * 128 + ((ch ^ (n & 7)) << 4);
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]) : "memory");
-    }
-    fence_proxy_async();
+    if (warp == 4) tmem_alloc(tmem_slot, TMEM_COLS);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot_gen;
-    constexpr uint32_t IDESC = instr_desc(128, NB, false);
-    const uint32_t b_lo = desc_lo(tile0 + C::OFF_B, 16);
-    auto mma_tile = [&](int i) {                         // thread 0: wait for the tile, issue its MMAs
-        mbar_wait_s(bar_ld0 + 8 * (i % NSTAGE), (i / NSTAGE) & 1, 7, status);
-        tc_fence_after();
-        const uint32_t a_lo = desc_lo(tile0 + (i % NSTAGE) * C::STAGE, 16);
-        const uint32_t dcol = tmem + (i & 1) * C::ACC_COLS;
-#pragma unroll
-        for (int kk = 0; kk < 2 * D / 16; ++kk)           // 2d input channels, 16 per instruction
-            umma(dcol, desc64(a_lo + (kk >> 2) * 1024 + (kk & 3) * 2, kDescHi),
-                 desc64(b_lo + (kk >> 2) * (C::B_SLOT >> 4) + (kk & 3) * 2, kDescHi), IDESC, kk > 0);
-        umma_commit(bar_mma0 + 8 * (i & 1));
-    };
-    if (tid == 0) mma_tile(0);
-    const uint32_t lane_base = ((uint32_t)(warp * 32)) << 16;
-    const float bh_bias = bias ? bias[h] : 0.f;
 
-    for (int i = 0; i < n_tiles; ++i) {
-        if (tid == 0 && i + 1 < n_tiles) mma_tile(i + 1);   // runs while tile i is taken out of TMEM below
-        mbar_wait_s(bar_mma0 + 8 * (i & 1), (i >> 1) & 1, 6, status);
-        tc_fence_after();
-        {
-            const uint32_t col = tmem + lane_base + (i & 1) * C::ACC_COLS;
-            uint32_t acc[32];
-            tmem_ld32(col, acc);
-            float y[K];
-            if constexpr (NB <= 32) {
-                tmem_wait_ld();
+    if (warp == 5) {
+        // ---- load lane: streams the input tiles through the stage ring ----------------------------------------------
+        if ((tid & 31) == 0) {
+            int fb = f_begin / n_all, ft = f_begin - fb * n_all;      // (head, row tile) of the next tile to load
+            for (int i = 0; i < n_tiles; ++i) {
+                // the stage is free once the MMAs of the tile that used it have completed
+                if (i >= NSTAGE) mbar_wait_s(bar_mma0 + 8 * ((i - NSTAGE) & 1), ((i - NSTAGE) >> 1) & 1, 3, status);
+                const uint32_t dst = tile0 + (i % NSTAGE) * C::STAGE, bar = bar_ld0 + 8 * (i % NSTAGE);
+                const int y = ft * TJ - HALF;
+                mbar_expect_tx(bar, C::STAGE);
 #pragma unroll
-                for (int t = 0; t < K; ++t)
-                    y[t] = (__uint_as_float(acc[2 * K + t]) + __uint_as_float(acc[K + t])) + __uint_as_float(acc[t]);
-            } else {
-                uint32_t acc2[32];
-                tmem_ld32(col + 32, acc2);
-                tmem_wait_ld();
-#pragma unroll
-                for (int t = 0; t < K; ++t) {
-                    const int i0 = t, i1 = K + t, i2 = 2 * K + t;
-                    const float a0 = __uint_as_float(i0 < 32 ? acc[i0] : acc2[i0 - 32]);
-                    const float a1 = __uint_as_float(i1 < 32 ? acc[i1] : acc2[i1 - 32]);
-                    const float a2 = __uint_as_float(i2 < 32 ? acc[i2] : acc2[i2 - 32]);
-                    y[t] = (a2 + a1) + a0;
+                for (int sb = 0; sb < SUB; ++sb) {
+                    tma_load_3d(dst + sb * 16384, &tmK, sb * 64, y, fb, bar);
+                    tma_load_3d(dst + (SUB + sb) * 16384, &tmV, sb * 64, y, fb, bar);
                 }
+                if (++ft == n_all) { ft = 0; ++fb; }
             }
-#pragma unroll
-            for (int t = 0; t < K; ++t) ys[tid * K + t] = y[t];
         }
-        tc_fence_before();
-        __syncthreads();                                 // ys complete; accumulator buffer i & 1 and stage i % NSTAGE are free
-        if (tid == 0 && i + NSTAGE < n_tiles) issue_tile(i + NSTAGE);
-        const int j = (t_begin + i) * TJ + tid;
-        if (tid < TJ && j < Tlen) {
-            float zz;
-            if (j + HALF > Tlen - 1) {
-                zz = -INFINITY;
-            } else {
-                zz = bh_bias;
+    } else if (warp == 4) {
+        // ---- MMA lane ------------------------------------------------------------------------------------------------
+        if ((tid & 31) == 0) {
+            constexpr uint32_t IDESC = instr_desc(128, NB, false);
+            const uint32_t b_lo = desc_lo(tile0 + C::OFF_B, 16), a_lo0 = desc_lo(tile0, 16);
+            int ft = f_begin % n_all, n_heads = 0;
+            bool new_head = true;
+            for (int i = 0; i < n_tiles; ++i) {
+                if (new_head) { mbar_wait_s(bar_b, n_heads & 1, 5, status); ++n_heads; }   // B of this head is ready
+                mbar_wait_s(bar_ld0 + 8 * (i % NSTAGE), (i / NSTAGE) & 1, 7, status);
+                if (i >= 2) mbar_wait_s(bar_free0 + 8 * (i & 1), ((i - 2) >> 1) & 1, 4, status);   // its accumulator buffer is free
+                tc_fence_after();
+                const uint32_t a_lo = a_lo0 + (uint32_t)(i % NSTAGE) * (C::STAGE >> 4);
+                const uint32_t dcol = tmem + (i & 1) * C::ACC_COLS;
 #pragma unroll
-                for (int t = 0; t < K; ++t) zz += ys[(tid + t) * K + t];
+                for (int kk = 0; kk < 2 * D / 16; ++kk)   // 2d input channels, 16 per instruction
+                    umma(dcol, desc64(a_lo + (kk >> 2) * 1024 + (kk & 3) * 2, kDescHi),
+                         desc64(b_lo + (kk >> 2) * (C::B_SLOT >> 4) + (kk & 3) * 2, kDescHi), IDESC, kk > 0);
+                umma_commit(bar_mma0 + 8 * (i & 1));
+                new_head = ++ft == n_all;
+                if (new_head) ft = 0;
             }
-            z[(size_t)bh * Tlen + j] = zz;
-            if (r) r[(size_t)bh * Tlen + j] = 1.f / (1.f + __expf(-zz));
         }
-        __syncthreads();                                 // ys is rewritten by the next tile
+    } else {
+        // ---- row threads: thread p owns input row p of the tile -------------------------------------------------------
+        auto group_sync = [&]() { asm volatile("bar.sync 1, 128;" ::: "memory"); };
+        const uint32_t lane_base = ((uint32_t)(warp * 32)) << 16;
+        int cur_bh = -1;
+        float bh_bias = 0.f;
+        for (int i = 0; i < n_tiles; ++i) {
+            const int f = f_begin + i, bh = f / n_all, ti = f - bh * n_all;
+            if (bh != cur_bh) {
+                // new head: this thread has taken every earlier tile out of TMEM, and it only gets here after the others
+                // did too (the group barrier at the end of the previous tile), so no MMA is still reading the old B
+                cur_bh = bh;
+                const int h = bh % H;
+                bh_bias = bias ? bias[h] : 0.f;
+                // B: row n = piece * K + t, columns = the 2d input channels (k part, then v part); zero rows above 3K
+                for (int e = tid; e < NB * 2 * D / 8; e += NT) {   // one 16-byte chunk (8 channels) of one row
+                    const int n = e / (2 * D / 8), c8 = e % (2 * D / 8);
+                    const int piece = n / K, t = n % K;
+                    uint32_t pk[4] = {0u, 0u, 0u, 0u};
+                    if (n < 3 * K) {
+                        const float4* src = reinterpret_cast<const float4*>(w + ((size_t)h * K + t) * 2 * D + c8 * 8);
+                        const float4 f0 = src[0], f1 = src[1];
+                        const float wv8[8] = {f0.x, f0.y, f0.z, f0.w, f1.x, f1.y, f1.z, f1.w};
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            float v2[2];
+#pragma unroll
+                            for (int x = 0; x < 2; ++x) {
+                                const float wv = wv8[2 * u + x];
+                                const float hi = __bfloat162float(__float2bfloat16_rn(wv));
+                                const float mid = __bfloat162float(__float2bfloat16_rn(wv - hi));
+                                const float lo = __bfloat162float(__float2bfloat16_rn((wv - hi) - mid));
+                                v2[x] = piece == 0 ? hi : (piece == 1 ? mid : lo);
+                            }
+                            __nv_bfloat162 h2 = __floats2bfloat162_rn(v2[0], v2[1]);
+                            pk[u] = *reinterpret_cast<uint32_t*>(&h2);
+                        }
+                    }
+                    const int sub = c8 / 8, ch = c8 % 8;   // 64-column sub-tile (k: 0..SUB-1, v: SUB..2SUB-1), chunk in row
+                    const uint32_t dst = tile0 + C::OFF_B + sub * C::B_SLOT + n * 128 + ((ch ^ (n & 7)) << 4);
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]) : "memory");
+                }
+                fence_proxy_async();
+                mbar_arrive(bar_b);
+            }
+            SPROF(4 * i);
+            mbar_wait_s(bar_mma0 + 8 * (i & 1), (i >> 1) & 1, 6, status);
+            tc_fence_after();
+            SPROF(4 * i + 1);
+            {
+                const uint32_t col = tmem + lane_base + (i & 1) * C::ACC_COLS;
+                uint32_t acc[32];
+                tmem_ld32(col, acc);
+                float y[K];
+                if constexpr (NB <= 32) {
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int t = 0; t < K; ++t)
+                        y[t] = (__uint_as_float(acc[2 * K + t]) + __uint_as_float(acc[K + t])) + __uint_as_float(acc[t]);
+                } else {
+                    uint32_t acc2[32];
+                    tmem_ld32(col + 32, acc2);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int t = 0; t < K; ++t) {
+                        const int i0 = t, i1 = K + t, i2 = 2 * K + t;
+                        const float a0 = __uint_as_float(i0 < 32 ? acc[i0] : acc2[i0 - 32]);
+                        const float a1 = __uint_as_float(i1 < 32 ? acc[i1] : acc2[i1 - 32]);
+                        const float a2 = __uint_as_float(i2 < 32 ? acc[i2] : acc2[i2 - 32]);
+                        y[t] = (a2 + a1) + a0;
+                    }
+                }
+                tc_fence_before();
+                mbar_arrive(bar_free0 + 8 * (i & 1));     // the accumulator buffer can take tile i + 2
+#pragma unroll
+                for (int t = 0; t < K; ++t) ys[tid * K + t] = y[t];
+            }
+            SPROF(4 * i + 2);
+            group_sync();                                  // ys complete
+            const int j = ti * TJ + tid;
+            if (tid < TJ && j < Tlen) {
+                float zz;
+                if (j + HALF > Tlen - 1) {
+                    zz = -INFINITY;
+                } else {
+                    zz = bh_bias;
+#pragma unroll
+                    for (int t = 0; t < K; ++t) zz += ys[(tid + t) * K + t];
+                }
+                z[(size_t)bh * Tlen + j] = zz;
+                if (r) r[(size_t)bh * Tlen + j] = 1.f / (1.f + __expf(-zz));
+            }
+            group_sync();                                  // ys is rewritten by the next tile
+            SPROF(4 * i + 3);
+        }
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem, TMEM_COLS);
+    if (warp == 4) tmem_dealloc(tmem, TMEM_COLS);
 }
 
 __device__ int g_scores_status = 0;
@@ -286,15 +329,13 @@ int run_tma(const Params& p, const void* k, const void* v, float* z, float* r, c
             return LTE_ERR_CUDA;
         attr_done = true;
     }
-    // tiles per CTA: as many CTAs as fit on the machine at once (two per SM at d = 64, one at d = 128), no second wave
+    // one wave of CTAs (two per SM at d = 64, one at d = 128) shares the flat list of (head, row tile) pairs evenly
     const int n_all = (p.T + TJ - 1) / TJ, BH = p.B * p.H;
+    const long long n_flat = (long long)n_all * BH;
+    if (n_flat > 0x7fffffffLL) return LTE_ERR_UNSUPPORTED;
     const int slots = n_sm * (D == 64 ? 2 : 1);
-    int per_head = slots / BH;                            // CTAs per head (rounded down: a single wave)
-    if (per_head < 1) per_head = 1;
-    if (per_head > n_all) per_head = n_all;
-    const int tiles_per_cta = (n_all + per_head - 1) / per_head;
-    dim3 grid((n_all + tiles_per_cta - 1) / tiles_per_cta, BH);
-    scores_tc_kernel<D, K><<<grid, NT, C::BYTES, st>>>(tk, tv, p.w, p.bias, z, r, p.H, p.T, tiles_per_cta, status_ptr);
+    const int n_cta = (int)(n_flat < slots ? n_flat : slots);
+    scores_tc_kernel<D, K><<<n_cta, NT + 64, C::BYTES, st>>>(tk, tv, p.w, p.bias, z, r, p.H, p.T, (int)n_flat, status_ptr);
     return cuda_status(cudaGetLastError());
 }
 
@@ -356,3 +397,10 @@ int launch_scores(const Params& p, const void* k, const void* v, float* z, float
 }
 
 }  // namespace lte
+
+#ifdef LTE_PROFILE
+extern "C" int lte_sprof_read(long long* out)
+{
+    return cudaMemcpyFromSymbol(out, lte::g_sprof, sizeof(long long) * 64) == cudaSuccess ? 0 : -1;
+}
+#endif
