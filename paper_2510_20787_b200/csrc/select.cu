@@ -18,9 +18,13 @@ __device__ __forceinline__ uint32_t key_of(const float* zz, int j, int sink, flo
     return z > zthr ? order_key(z) : 0u;
 }
 
+// CACHED: the keys of all eligible positions are computed once and kept in dynamic shared memory, so the radix passes
+// and the compaction never go back to L2; otherwise every pass recomputes them from z.
+template <bool CACHED>
 __global__ void select_kernel(const float* __restrict__ z, int32_t* __restrict__ idx, int32_t* __restrict__ cnt,
                               int32_t* __restrict__ ncand, int T, int W, int R, int sink, float zthr)
 {
+    extern __shared__ uint32_t s_keys[];
     __shared__ uint32_t hist[256];
     __shared__ uint32_t warp_tot[2][32];
     __shared__ uint32_t sh_prefix, sh_remaining, sh_ncand;
@@ -32,12 +36,17 @@ __global__ void select_kernel(const float* __restrict__ z, int32_t* __restrict__
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int lane = tid & 31, wid = tid >> 5, nwarp = nthr >> 5;
 
-    // ---- pass 0: number of candidates
+    auto key_at = [&](int j) -> uint32_t { return CACHED ? s_keys[j] : key_of(zz, j, sink, zthr); };
+    // ---- pass 0: number of candidates (and the key cache)
     if (tid == 0) sh_ncand = 0;
     __syncthreads();
     {
         uint32_t c = 0;
-        for (int j = tid; j < N; j += nthr) c += key_of(zz, j, sink, zthr) != 0u;
+        for (int j = tid; j < N; j += nthr) {
+            const uint32_t key = key_of(zz, j, sink, zthr);
+            if (CACHED) s_keys[j] = key;
+            c += key != 0u;
+        }
         c = __reduce_add_sync(0xffffffffu, c);
         if (lane == 0 && c) atomicAdd(&sh_ncand, c);
     }
@@ -55,7 +64,7 @@ __global__ void select_kernel(const float* __restrict__ z, int32_t* __restrict__
             const uint32_t prefix = sh_prefix;
             for (int j0 = 0; j0 < N; j0 += nthr) {
                 const int j = j0 + tid;
-                uint32_t key = j < N ? key_of(zz, j, sink, zthr) : 0u;
+                uint32_t key = j < N ? key_at(j) : 0u;
                 const bool in = j < N && (key & mask) == prefix;
                 const uint32_t dig = in ? (key >> shift) & 255u : 0xFFFFFFFFu;
                 const uint32_t peers = __match_any_sync(0xffffffffu, dig);
@@ -103,7 +112,7 @@ __global__ void select_kernel(const float* __restrict__ z, int32_t* __restrict__
     int buf = 0;
     for (int j0 = 0; j0 < N && R > 0; j0 += nthr, buf ^= 1) {
         const int j = j0 + tid;
-        const uint32_t key = j < N ? key_of(zz, j, sink, zthr) : 0u;
+        const uint32_t key = j < N ? key_at(j) : 0u;
         const bool above = key > theta;
         const bool equal = need_eq > 0 && key == theta && j < N;
         const uint32_t bA = __ballot_sync(0xffffffffu, above), bE = __ballot_sync(0xffffffffu, equal);
@@ -129,13 +138,141 @@ __global__ void select_kernel(const float* __restrict__ z, int32_t* __restrict__
     if (tid == 0) cnt[bh] = (int32_t)kept;
 }
 
+
+// ---- register-resident variant: every thread keeps KPT consecutive keys in registers ---------------------------------
+// The R-th largest key is found by bisection on its 32 bits: each step counts the keys >= a candidate value (compares
+// in registers, one shared-memory atomic per warp, one block barrier), so there is no histogram and no contention
+// however concentrated the logits are.  The ordered compaction is one block-wide exclusive scan of the per-thread
+// (above, equal) counts, after which each thread writes the kept positions of its own segment.
+template <int KPT>
+__global__ void __launch_bounds__(1024) select_reg_kernel(const float* __restrict__ z, int32_t* __restrict__ idx,
+                                                          int32_t* __restrict__ cnt, int32_t* __restrict__ ncand, int T,
+                                                          int W, int R, int sink, float zthr)
+{
+    __shared__ uint32_t s_count[3];
+    __shared__ uint32_t s_wa[32], s_we[32];
+    const int bh = blockIdx.x;
+    const float* zz = z + (size_t)bh * T;
+    int32_t* out = idx + (size_t)bh * R;
+    const int N = T - W > 0 ? T - W : 0;
+    const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, wid = tid >> 5, nwarp = nthr >> 5;
+    const int p0 = tid * KPT;
+
+    uint32_t key[KPT];
+#pragma unroll
+    for (int i = 0; i < KPT; ++i) key[i] = p0 + i < N ? key_of(zz, p0 + i, sink, zthr) : 0u;
+    if (tid < 3) s_count[tid] = 0;
+    __syncthreads();
+    // block-wide sum of a per-thread count.  Three counters rotate: the one reset after this call's barrier is used two
+    // calls later, so the reset is ordered before those additions by the barrier in between (one barrier per call).
+    int slot = 0;
+    auto block_sum = [&](uint32_t c) -> uint32_t {
+        c = __reduce_add_sync(0xffffffffu, c);
+        if (lane == 0 && c) atomicAdd(&s_count[slot], c);
+        __syncthreads();
+        const uint32_t total = s_count[slot];
+        if (tid == 0) s_count[(slot + 2) % 3] = 0;
+        slot = (slot + 1) % 3;
+        return total;
+    };
+    uint32_t c0 = 0;
+#pragma unroll
+    for (int i = 0; i < KPT; ++i) c0 += key[i] != 0u;
+    const uint32_t nc = block_sum(c0);
+    if (tid == 0 && ncand) ncand[bh] = (int32_t)nc;
+
+    uint32_t theta = 0, need_eq = 0;
+    if (R > 0 && nc > (uint32_t)R) {
+        uint32_t prefix = 0;
+        for (int bit = 31; bit >= 0; --bit) {
+            const uint32_t cand = prefix | (1u << bit);
+            uint32_t c = 0;
+#pragma unroll
+            for (int i = 0; i < KPT; ++i) c += key[i] >= cand;
+            if (block_sum(c) >= (uint32_t)R) prefix = cand;  // at least R keys are >= cand: the R-th largest is too
+        }
+        theta = prefix;
+        uint32_t g = 0;
+#pragma unroll
+        for (int i = 0; i < KPT; ++i) g += key[i] > theta;
+        need_eq = (uint32_t)R - block_sum(g);
+    }
+    // ---- ordered compaction: exclusive scan of (above, equal) counts over the threads' segments
+    uint32_t a = 0, e = 0;
+    if (R > 0) {
+#pragma unroll
+        for (int i = 0; i < KPT; ++i) { a += key[i] > theta; e += (need_eq > 0 && key[i] == theta && p0 + i < N); }
+    }
+    uint32_t ia = a, ie = e;                               // inclusive warp scans
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t ta = __shfl_up_sync(0xffffffffu, ia, o), te = __shfl_up_sync(0xffffffffu, ie, o);
+        if (lane >= o) { ia += ta; ie += te; }
+    }
+    if (lane == 31) { s_wa[wid] = ia; s_we[wid] = ie; }
+    __syncthreads();
+    if (wid == 0) {
+        uint32_t wa = lane < nwarp ? s_wa[lane] : 0u, we = lane < nwarp ? s_we[lane] : 0u;
+        uint32_t xa = wa, xe = we;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t ta = __shfl_up_sync(0xffffffffu, xa, o), te = __shfl_up_sync(0xffffffffu, xe, o);
+            if (lane >= o) { xa += ta; xe += te; }
+        }
+        s_wa[lane] = xa - wa; s_we[lane] = xe - we;        // exclusive warp offsets
+    }
+    __syncthreads();
+    uint32_t a_before = s_wa[wid] + ia - a, e_before = s_we[wid] + ie - e;
+    if (R > 0) {
+#pragma unroll
+        for (int i = 0; i < KPT; ++i) {
+            const bool above = key[i] > theta;
+            const bool equal = need_eq > 0 && key[i] == theta && p0 + i < N;
+            if (above || (equal && e_before < need_eq)) {
+                const uint32_t sl = a_before + (e_before < need_eq ? e_before : need_eq);
+                if (sl < (uint32_t)R) out[sl] = p0 + i;
+            }
+            a_before += above; e_before += equal;
+        }
+    }
+    const uint32_t kept = R > 0 ? (nc < (uint32_t)R ? nc : (uint32_t)R) : 0u;
+    for (int i = (int)kept + tid; i < R; i += nthr) out[i] = -1;
+    if (tid == 0) cnt[bh] = (int32_t)kept;
+}
+
 }  // namespace
 
 int launch_select(const Params& p, const float* z, int32_t* idx, int32_t* cnt, int32_t* ncand, cudaStream_t st)
 {
-    const int N = p.T - p.W;
+    const int N = p.T - p.W > 0 ? p.T - p.W : 0;
+    {
+        // register-resident kernel: up to 64 keys per thread
+        const int nt = N <= 2048 ? 256 : 1024;
+        const int kpt = (N + nt - 1) / nt;
+        const int BH = p.B * p.H;
+#define LTE_SEL(KPT) select_reg_kernel<KPT><<<BH, nt, 0, st>>>(z, idx, cnt, ncand, p.T, p.W, p.R, p.sink, p.zthr)
+        if (kpt <= 64) {
+            if (kpt <= 1) LTE_SEL(1); else if (kpt <= 2) LTE_SEL(2); else if (kpt <= 4) LTE_SEL(4);
+            else if (kpt <= 8) LTE_SEL(8); else if (kpt <= 16) LTE_SEL(16); else if (kpt <= 32) LTE_SEL(32);
+            else LTE_SEL(64);
+            return cuda_status(cudaGetLastError());
+        }
+#undef LTE_SEL
+    }
     const int threads = N <= 1024 ? 256 : (N <= 4096 ? 512 : 1024);
-    select_kernel<<<p.B * p.H, threads, 0, st>>>(z, idx, cnt, ncand, p.T, p.W, p.R, p.sink, p.zthr);
+    const size_t key_bytes = (size_t)N * 4;
+    constexpr size_t kCacheMax = 200 * 1024;              // keys of up to 51200 positions stay on chip
+    if (key_bytes <= kCacheMax) {
+        static bool attr_done = false;
+        if (!attr_done) {
+            if (cudaFuncSetAttribute(select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCacheMax) != cudaSuccess)
+                return LTE_ERR_CUDA;
+            attr_done = true;
+        }
+        select_kernel<true><<<p.B * p.H, threads, key_bytes, st>>>(z, idx, cnt, ncand, p.T, p.W, p.R, p.sink, p.zthr);
+    } else {
+        select_kernel<false><<<p.B * p.H, threads, 0, st>>>(z, idx, cnt, ncand, p.T, p.W, p.R, p.sink, p.zthr);
+    }
     return cuda_status(cudaGetLastError());
 }
 
