@@ -31,8 +31,8 @@ METRIC = "LTE attn prefill tokens/s & % bf16 TC peak; decode step us & % HBM BW"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu captures (profiles/),
-# keyed by kernel family; None until a capture exists.
-NCU_TRAFFIC_BYTES = {"prefill_attn_C2": None, "decode_C4": None}
+# keyed by kernel family (profiles/prefill_tc_kernel_C2.md, profiles/decode_bulk_kernel_C4.md).
+NCU_TRAFFIC_BYTES = {"prefill_attn_C2": 117.1e6, "decode_C4": 142.9e6}
 
 
 def peaks():
@@ -280,6 +280,11 @@ def run_lte(args):
         line["clocks"] = clocks
 
     # ---- the other rows of the path on their own configurations --------------------------------
+    if args.section and rank == 0 and world == 1:
+        del hq, hk, hv, ho, dq_, dk_, dv_
+        print(json.dumps({"section": args.section, "extras": extras(torch, lte, synth, pk, flush, args,
+                                                                    only=(args.section,))}))
+        return
     if not args.no_extras and rank == 0 and world == 1:
         del hq, hk, hv, ho, dq_, dk_, dv_
         line["extras"] = extras(torch, lte, synth, pk, flush, args)
@@ -291,9 +296,24 @@ def run_lte(args):
         print(json.dumps(line))
 
 
-def extras(torch, lte, synth, pk, flush, args):
+def extras(torch, lte, synth, pk, flush, args, only=None):
+    """The other rows of the path on their own configurations; `only` restricts the sections run."""
+    return _extras_sections(torch, lte, synth, pk, flush, args, only if only is not None else ("C3", "C5", "C4"))
+
+
+def _extras_sections(torch, lte, synth, pk, flush, args, which):
     out = {}
     n5 = 5
+    if "C3" in which:
+        _extra_c3(out, torch, lte, synth, pk, flush, n5)
+    if "C5" in which:
+        _extra_c5(out, torch, lte, synth, pk, flush, n5)
+    if "C4" in which:
+        _extra_c4(out, torch, lte, synth, pk, flush, n5)
+    return out
+
+
+def _extra_c3(out, torch, lte, synth, pk, flush, n5):
 
     # long prefill (tensor-core bound)
     cfg = synth.CONFIGS["C3"]
@@ -322,6 +342,8 @@ def extras(torch, lte, synth, pk, flush, args):
                               "select_ms": mid3(ms_se)}
     del x, o, lse, z
 
+
+def _extra_c5(out, torch, lte, synth, pk, flush, n5):
     # forward + backward
     cfg = synth.CONFIGS["C5"]
     x = device_inputs(cfg, 5, torch, with_dO=True)
@@ -349,6 +371,8 @@ def extras(torch, lte, synth, pk, flush, args):
                          "bwd_hbm_frac": 8 * nb / tb / 1e9 / pk["hbm_gbs"]}
     del x, o, lse, z, ws
 
+
+def _extra_c4(out, torch, lte, synth, pk, flush, n5):
     # batched decode
     cfg = synth.CONFIGS["C4"]
     x = device_inputs(cfg, 4, torch)
@@ -394,7 +418,6 @@ def extras(torch, lte, synth, pk, flush, args):
                         "hbm_gbs": by / (us * 1e-6) / 1e9, "hbm_frac": by / (us * 1e-6) / 1e9 / pk["hbm_gbs"],
                         "traffic": NCU_TRAFFIC_BYTES["decode_C4"],
                         "note": "the 138 MB cache is about the size of L2: see the ncu DRAM bytes in profiles/"}
-    return out
 
 
 def oracle_step(orc, x, cfg):
@@ -455,6 +478,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="lte", choices=["lte", "reference"])
     ap.add_argument("--no-extras", action="store_true")
+    ap.add_argument("--section", default=None, choices=["C3", "C4", "C5"],
+                    help="time only this extra section (long prefill / decode / forward+backward) after the main loop")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":
