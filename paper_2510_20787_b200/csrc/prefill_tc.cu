@@ -45,10 +45,15 @@ template <int D> struct Smem {
     static constexpr int OFF_K = QTILE;
     static constexpr int OFF_V = OFF_K + KST * KVTILE;
     static constexpr int OFF_P = OFF_V + VST * KVTILE;        // [128][64] bf16 = 16 KB
-    static constexpr int OFF_BAR = OFF_P + BM * BN * 2;       // mbarriers, tmem slot
+    // d = 64: the row sums are taken by the tensor core as well: PV gets 16 extra B columns of ones, so column D of
+    // the accumulator is sum_j P_ij of exactly the (bf16-rounded) probabilities the product used.  The ones live in one
+    // more 64-column group, LBO away from the value tile.
+    static constexpr bool ONES = D == 64;
+    static constexpr int OFF_ONES = OFF_P + BM * BN * 2;      // [64][64] bf16 ones (8 KB), d = 64 only
+    static constexpr int OFF_BAR = OFF_ONES + (ONES ? BN * 128 : 0);   // mbarriers, tmem slot
     static constexpr int OFF_IDX = OFF_BAR + 128;             // 128 staged list entries
     static constexpr int BYTES = OFF_IDX + 512;
-    static constexpr uint32_t TMEM_COLS = 256;                // S0: [0,64)  S1: [64,128)  O: [128, 128+D)
+    static constexpr uint32_t TMEM_COLS = 256;                // S0: [0,64)  S1: [64,128)  O: [128, 128+D) (+16 row-sum columns)
 };
 
 __device__ __forceinline__ void softmax_group_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
@@ -132,7 +137,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         const int n_tiles = n_win + (nv_max + BN - 1) / BN;
         if (lane == 0) {
             constexpr uint32_t IDESC_S = instr_desc(BM, BN, false);
-            constexpr uint32_t IDESC_O = instr_desc(BM, D, true);
+            constexpr uint32_t IDESC_O = S::ONES ? instr_desc(BM, D + 16, true) : instr_desc(BM, D, true);
             // descriptor words: lo = (address >> 4) | LBO field, hi = SBO field | version | swizzle mode
             constexpr uint32_t HI = (1024u >> 4) | (1u << 14) | (2u << 29);
             const uint32_t q_lo = (sQ >> 4) | (1u << 16), k_lo = (sK >> 4) | (1u << 16), p_lo = (sP >> 4) | (1u << 16);
@@ -188,7 +193,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 wait_v(t);
                 tc_fence_after();
                 {
-                    const uint32_t vb = v_lo + (uint32_t)(t % VST) * (S::KVTILE >> 4);
+                    uint32_t vb = v_lo + (uint32_t)(t % VST) * (S::KVTILE >> 4);
+                    if (S::ONES)   // second 64-column group of B = the block of ones: LBO = its distance from this value tile
+                        vb = ((sV + (t % VST) * S::KVTILE) >> 4) | (((base + S::OFF_ONES - sV - (t % VST) * S::KVTILE) >> 4) << 16);
 #pragma unroll
                     for (int kk = 0; kk < BN / 16; ++kk)
                         umma(tmem + O_COL, desc64(p_lo + kk * 2, HI), desc64(vb + kk * 128, HI), IDESC_O, (t > 0 || kk > 0) ? 1u : 0u);
@@ -272,9 +279,14 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             for (int t = 0; t < VST; ++t) { gather_rows(t, rows4); gather_issue(t, true, rows4); }
         }
 
+        if (S::ONES) {                                         // 8 KB of bf16 1.0: 64 bytes per thread
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(base + S::OFF_ONES + tid * 64 + u * 16), "r"(0x3F803F80u) : "memory");
+        }
         const float c2 = scale * 1.4426950408889634f;          // logits are handled in the log2 domain: x = s * c2
         const uint32_t lane_base = ((uint32_t)(warp * 32)) << 16;   // this warp's TMEM lanes
-        float m_run = -INFINITY, l_run = 0.f;                  // running max (log2 domain) and sum
+        float m_run = -INFINITY, l_run = 0.f;                  // running max (log2 domain) and sum (sum only if !ONES)
 
         for (int t = 0; t < n_tiles; ++t) {
             // row positions for this tile's two gathers, fetched first so their latency hides under the softmax
@@ -331,7 +343,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 if (!act[cb]) continue;
                 if (full[cb]) {
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) mr[c & 3] = fmaxf(mr[c & 3], __uint_as_float(r[cb][c]));
+                    for (int c = 0; c < 32; c += 2)
+                        mr[(c >> 1) & 3] = max3(mr[(c >> 1) & 3], __uint_as_float(r[cb][c]), __uint_as_float(r[cb][c + 1]));
                 } else {
 #pragma unroll
                     for (int c = 0; c < 32; ++c) {
@@ -355,7 +368,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             else if (m_tile > m_run + 8.f) { alpha = fast_exp2(m_run - m_tile); m_run = m_tile; need = true; }
             if (__any_sync(0xffffffffu, need)) {
 #pragma unroll
-                for (int cb = 0; cb < D / 32; ++cb) {
+                for (int cb = 0; cb < D / 32 + (S::ONES ? 1 : 0); ++cb) {   // with ONES the row-sum columns are rescaled too
                     uint32_t q4[32];
                     tmem_ld32(tmem + lane_base + O_COL + cb * 32, q4);
                     tmem_wait_ld();
@@ -377,7 +390,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                         // masked entries hold -inf: fma gives -inf and exp2(-inf) = 0
                         const float p0 = fast_exp2(fmaf(__uint_as_float(r[cb][c]), c2, neg_m));
                         const float p1 = fast_exp2(fmaf(__uint_as_float(r[cb][c + 1]), c2, neg_m));
-                        ls[(c >> 1) & 3] += p0 + p1;
+                        if (!S::ONES) ls[(c >> 1) & 3] += p0 + p1;   // with ONES the tensor core sums the rounded probabilities
                         __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
                         pk[c >> 1] = *reinterpret_cast<uint32_t*>(&h);
                     }
@@ -405,6 +418,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         PROF(51);
 
         // ---- epilogue: O / l -> bf16, logsumexp ----------------------------------------------------------
+        if (S::ONES) {                                         // the row sum is column D of the accumulator
+            uint32_t q4[32];
+            tmem_ld32(tmem + lane_base + O_COL + D, q4);
+            tmem_wait_ld();
+            l_run = __uint_as_float(q4[0]);
+        }
         const float inv = 1.f / l_run;
         __nv_bfloat16* orow = o + ((size_t)bh * Tlen + i) * D;
 #pragma unroll
