@@ -120,6 +120,14 @@ int lte_attn_prefill(const lte_shape* s, const void* q, const void* k, const voi
  * their logits, and a pool of at most R retained keys/values with their logits and positions.
  * The cache is one caller-owned device buffer of lte_cache_bytes() bytes; copying it is a
  * checkpoint.  T in the shape is ignored by lte_cache_bytes.
+ *
+ * Layout: a 256-byte header, then one block per (b,h), padded to a multiple of 256 bytes:
+ *   keys    [rows_alloc][d]   rows [0,W) = ring, rows [W,W+R) = pool
+ *   values  [rows_alloc][d]
+ *   logits  [W+R] fp32, same row order          pool positions [R] int32          {n, cnt, 0, 0} int32
+ * rows_alloc = W+R, except for bf16 with d = 64 and W+R <= 256, where rows_alloc = 256 (zero rows at the end) and each
+ * key/value row is stored with the 128-byte swizzle (16-byte chunk c of row r sits at chunk position c ^ (r & 7)),
+ * which is the layout the tensor-core decode kernel consumes directly from shared memory.
  */
 size_t lte_cache_bytes(const lte_shape* s);
 

@@ -48,20 +48,26 @@ __device__ __forceinline__ uint32_t order_key(float z) {
 // ---- decode cache layout (per (b,h) block; see lte_cache_bytes) -----------------------------
 struct CacheLayout {
     size_t esz;            // element size of k/v
-    size_t off_k, off_v;   // [(W+R), d] each: rows [0,W) ring (slot = pos mod W), rows [W,W+R) pool
+    size_t off_k, off_v;   // [rows_alloc, d] each: rows [0,W) ring (slot = pos mod W), rows [W,W+R) pool
     size_t off_z;          // [(W+R)] fp32 logits, same row order
     size_t off_pidx;       // [R] int32 positions of pool entries
     size_t off_meta;       // int32[4]: n (tokens seen), cnt (pool entries), reserved x2
     size_t stride;         // bytes per (b,h), multiple of 256
     size_t header;         // bytes before the first (b,h) block (status word lives at byte 0)
+    int rows_alloc;        // key/value rows per block (W+R, or 256 with zero rows at the end in the swizzled layout)
+    int swz;               // 1: bf16, d = 64, W+R <= 256: rows are stored with the 128-byte swizzle (16-byte chunk c of
+                           //    row r sits at chunk position c ^ (r & 7)) so that the block, once copied to shared memory,
+                           //    is a valid tcgen05 operand as it stands
 };
 __host__ __device__ inline CacheLayout cache_layout(int d, int W, int R, int dtype) {
     CacheLayout L;
     L.esz = dtype == LTE_BF16 ? 2 : 4;
+    L.swz = (dtype == LTE_BF16 && d == 64 && W + R <= 256) ? 1 : 0;
+    L.rows_alloc = L.swz ? 256 : W + R;
     size_t rows = (size_t)W + R;
     L.off_k = 0;
-    L.off_v = L.off_k + rows * d * L.esz;
-    L.off_z = L.off_v + rows * d * L.esz;
+    L.off_v = L.off_k + (size_t)L.rows_alloc * d * L.esz;
+    L.off_z = L.off_v + (size_t)L.rows_alloc * d * L.esz;
     L.off_pidx = L.off_z + rows * 4;
     L.off_meta = L.off_pidx + (size_t)R * 4;
     size_t end = L.off_meta + 16;
@@ -69,6 +75,8 @@ __host__ __device__ inline CacheLayout cache_layout(int d, int W, int R, int dty
     L.header = 256;
     return L;
 }
+// chunk position of logical 16-byte chunk `c` of row `row` (bf16, d = 64: 8 chunks per row)
+__host__ __device__ inline int cache_chunk_pos(const CacheLayout& L, int row, int c) { return L.swz ? (c ^ (row & 7)) : c; }
 
 // kernel launchers (one translation unit each)
 int launch_scores(const Params& p, const void* k, const void* v, float* z, float* r, cudaStream_t st);
@@ -77,6 +85,8 @@ int launch_prefill_simt(const Params& p, const void* q, const void* k, const voi
                         const int32_t* cnt, void* o, float* lse, cudaStream_t st);
 int launch_cache_init(const Params& p, const void* k, const void* v, const float* z, const int32_t* idx,
                       const int32_t* cnt, void* cache, cudaStream_t st);
+int launch_decode_tc(const Params& p, void* cache, const void* q1, const void* k1, const void* v1, void* o1,
+                     float* lse1, cudaStream_t st);
 int launch_decode(const Params& p, void* cache, const void* q1, const void* k1, const void* v1, void* o1,
                   float* lse1, cudaStream_t st);
 size_t bwd_workspace_bytes(const Params& p, uint32_t flags);

@@ -637,8 +637,9 @@ __global__ void cache_init_kernel(unsigned char* __restrict__ cache, CacheLayout
         const int a = e / D, c = e % D;
         const int pos = a < nwin ? lo + a : idx[(size_t)bh * R + (a - nwin)];
         const int row = a < nwin ? pos % W : W + (a - nwin);
-        Kc[(size_t)row * D + c] = k[((size_t)bh * Tlen + pos) * D + c];
-        Vc[(size_t)row * D + c] = v[((size_t)bh * Tlen + pos) * D + c];
+        const int cdst = L.swz ? ((((c >> 3) ^ (row & 7)) << 3) | (c & 7)) : c;   // swizzled layout: chunk c/8 moves
+        Kc[(size_t)row * D + cdst] = k[((size_t)bh * Tlen + pos) * D + c];
+        Vc[(size_t)row * D + cdst] = v[((size_t)bh * Tlen + pos) * D + c];
     }
     for (int a = threadIdx.x; a < W + R; a += blockDim.x) {
         float zz = -INFINITY;
@@ -690,6 +691,7 @@ int launch_decode(const Params& p, void* cache, const void* q1, const void* k1, 
 {
     if (p.W + p.R > MAX_ROWS) return LTE_ERR_UNSUPPORTED;
     const CacheLayout L = cache_layout(p.d, p.W, p.R, p.dtype);
+    if (L.swz) return launch_decode_tc(p, cache, q1, k1, v1, o1, lse1, st);   // bf16, d = 64, W+R <= 256: tensor-core kernel
     const BulkSmem bp = bulk_smem_plan(L, p.W, p.R);
     const size_t bulk_smem = bp.total;
     const bool bulk = bulk_smem <= 73 * 1024 && p.K <= 2 * (DT / 32);   // three blocks per SM still fit

@@ -13,6 +13,7 @@ int prefill_status_fetch_and_clear();
 int decode_status_fetch_and_clear();
 int scores_status_fetch_and_clear();
 int bwd_status_fetch_and_clear();
+int decode_tc_status_fetch_and_clear();
 
 namespace {
 
@@ -87,8 +88,9 @@ int lte_device_status(void)
     const int g = decode_status_fetch_and_clear();
     const int f = scores_status_fetch_and_clear();
     const int b = bwd_status_fetch_and_clear();
-    if (h < 0 || g < 0 || f < 0 || b < 0) return LTE_ERR_CUDA;
-    return (h == 0 && g == 0 && f == 0 && b == 0) ? LTE_OK : LTE_ERR_DEVICE_STATUS;
+    const int d = decode_tc_status_fetch_and_clear();
+    if (h < 0 || g < 0 || f < 0 || b < 0 || d < 0) return LTE_ERR_CUDA;
+    return (h == 0 && g == 0 && f == 0 && b == 0 && d == 0) ? LTE_OK : LTE_ERR_DEVICE_STATUS;
 }
 
 size_t lte_workspace_bytes(int op, const lte_shape* s, const lte_conv* c)

@@ -36,7 +36,7 @@ def test_strerror_and_sizes():
     assert L.lte_strerror(0) == b"ok"
     assert b"workspace" in L.lte_strerror(-3)
     s = lte.shape(128, 16, 8192, 64, 128, 128, lte.BF16)
-    per = 2 * 256 * 64 * 2 + 256 * 4 + 128 * 4 + 16
+    per = 2 * 256 * 64 * 2 + 256 * 4 + 128 * 4 + 16          # W + R = 256 rows of keys and of values
     per = (per + 255) // 256 * 256
     assert lte.lte_cache_bytes(s) == 256 + 128 * 16 * per
     c = lte.LteConv(1, 7, 1, 16, 0)

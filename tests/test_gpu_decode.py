@@ -16,7 +16,9 @@ def _read_pool(cache, cfg, B):
     """Pool positions and counts out of the raw cache buffer (layout documented in include/lte.h)."""
     esz = 2 if cfg.dtype == "bf16" else 4
     rows = cfg.W + cfg.R
-    off_z = 2 * rows * cfg.d * esz
+    # bf16, d = 64, W + R <= 256: the block always holds 256 key/value rows (zero rows at the end)
+    rows_alloc = 256 if (cfg.dtype == "bf16" and cfg.d == 64 and rows <= 256) else rows
+    off_z = 2 * rows_alloc * cfg.d * esz
     off_pidx = off_z + rows * 4
     off_meta = off_pidx + cfg.R * 4
     stride = (off_meta + 16 + 255) // 256 * 256
