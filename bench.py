@@ -150,6 +150,21 @@ def attn_flops(idx, cnt, T, W, d, torch):
     return 4.0 * d * (win + vis)
 
 
+def max_over_ranks(ms, dist, device):
+    """The slowest rank sets the time: all-reduce(MAX) of a per-rank duration (no-op without a process group)."""
+    import torch
+    if dist is None:
+        return float(ms)
+    t = torch.tensor([float(ms)], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_rate(units_per_rank, world, ms):
+    """Weak scaling: every rank processes `units_per_rank` in `ms` (max over ranks) -> aggregate units per second."""
+    return units_per_rank * world / (ms * 1e-3)
+
+
 def run_lte(args):
     import torch
     from paper_2510_20787_b200 import lte, synth
@@ -215,13 +230,9 @@ def run_lte(args):
             step()
         torch.cuda.synchronize()
         clocks = sampler.stop()
-    step_ms = float(np.mean(ms))
-    if dist is not None:
-        t = torch.tensor([step_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        step_ms = float(t.item())
+    step_ms = max_over_ranks(float(np.mean(ms)), dist, "cuda")
     tokens = cfg.B * cfg.T * world
-    value = tokens / (step_ms * 1e-3)
+    value = whole_job_rate(cfg.B * cfg.T, world, step_ms)
     sub = np.array(sub)                       # [steps, 3] ms: scores, select, attention
     k_ms = sub.mean(axis=0)
 
@@ -245,11 +256,7 @@ def run_lte(args):
     barrier()
     e_ms, _ = timed(torch, e2e_step, args.steps, max(args.warmup, 3), flush)
     barrier()
-    e2e_ms = float(np.mean(e_ms))
-    if dist is not None:
-        t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = max_over_ranks(float(np.mean(e_ms)), dist, "cuda")
     h2d = sum(t.numel() * t.element_size() for t in (hq, hk, hv))
     d2h = sum(t.numel() * t.element_size() for t in (ho, hl, hi, hc))
 

@@ -128,3 +128,46 @@ def test_checkpoint_replay_is_bitwise_identical():
 
 def test_no_bounded_wait_expired():
     assert lte.lte_device_status() == 0
+
+
+def test_config4_full_batch_sampled_sequences():
+    """The benchmark's own launch configuration (B = 128: persistent CTAs walking several heads each), compared on
+    sampled sequences: those come from the shared generator, the others are seeded device noise of the same shape."""
+    cfg = synth.CONFIGS["C4"]
+    sample = [0, 63, 127]
+    steps = 24
+    g = torch.Generator(device="cuda"); g.manual_seed(7)
+    sc = cfg.d ** -0.25
+    Ttot = cfg.T + steps
+    q = (torch.randn((cfg.B, cfg.H, steps, cfg.d), generator=g, device="cuda") * sc).to(torch.bfloat16)
+    k = (torch.randn((cfg.B, cfg.H, Ttot, cfg.d), generator=g, device="cuda") * sc).to(torch.bfloat16)
+    v = torch.randn((cfg.B, cfg.H, Ttot, cfg.d), generator=g, device="cuda").to(torch.bfloat16)
+    x = synth.make(cfg, 3, batch=sample, T=Ttot)
+    for a, b in enumerate(sample):
+        k[b] = dev(x["k"][a], "bf16"); v[b] = dev(x["v"][a], "bf16")
+        q[b] = dev(x["q"][a][:, cfg.T:], "bf16")
+    w = torch.from_numpy(x["w"]).cuda()
+    c = lte.conv(w)
+    s0 = shape_of(cfg)
+    kp, vp = k[:, :, :cfg.T].contiguous(), v[:, :, :cfg.T].contiguous()
+    z = lte.lte_scores(s0, c, kp, vp)
+    idx, cnt = lte.lte_select(s0, z)
+    cache = lte.lte_cache_init(s0, c, kp, vp, z, idx, cnt)
+    del kp, vp, z
+    outs = []
+    for n in range(steps):
+        o1, _ = lte.lte_attn_decode(s0, c, cache, q[:, :, n].contiguous(), k[:, :, cfg.T + n].contiguous(),
+                                    v[:, :, cfg.T + n].contiguous())
+        outs.append(o1[sample].float().cpu().numpy())
+    torch.cuda.synchronize()
+    assert lte.lte_device_status() == 0
+    o_n = np.stack(outs, axis=2)
+    z64 = orc.scores(x["k"], x["v"], x["w"])
+    o64, _, pidx, pcnt = orc.stream(x["q"], x["k"], x["v"], z64, cfg.W, cfg.R, n_from=cfg.T)
+    assert np.max(np.abs(o_n - o64)) <= 2e-2
+    pools, ns = _read_pool(cache, cfg, cfg.B)
+    for a, b in enumerate(sample):
+        for h in range(cfg.H):
+            want = pidx[a, h, :pcnt[a, h]]
+            assert np.array_equal(pools[b * cfg.H + h], want)
+    assert all(n == Ttot for n in ns)
