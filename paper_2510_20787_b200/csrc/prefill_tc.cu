@@ -9,8 +9,9 @@
 //                  S tiles are computed while the softmax of the current one runs
 //   softmax        thread r owns query row r = TMEM lane r: tcgen05.ld, range mask (whole 32-column chunks are
 //                  skipped or taken unmasked when the warp's rows allow it), running max / sum in fp32 (exp2 with
-//                  the scale folded in), P written as bf16 into swizzled shared memory
-//   O += P V       tcgen05.mma with V as an MN-major operand, accumulated in TMEM; the accumulator is rescaled
+//                  the scale folded in), P written as bf16 back into TMEM over the S buffer it came from
+//   O += P V       tcgen05.mma with P as the TMEM A operand and V as an MN-major shared-memory operand,
+//                  accumulated in TMEM; the accumulator is rescaled
 //                  in place only when a row's maximum grows by more than 2^8 (lazy rescale)
 // Loads run two to three tiles ahead of the tensor core.  Every mbarrier wait is bounded; a wait that runs out
 // records a status word and the kernel still terminates.
@@ -37,19 +38,19 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, int cod
 
 template <int D> struct Smem {
     static constexpr int SUB = D / 64;                        // 64-column (128-byte) sub-tiles per row
-    static constexpr int KST = D == 64 ? 3 : 2;               // key stages
+    static constexpr int KST = 3;                             // key stages
     static constexpr int VST = D == 64 ? 3 : 2;               // value stages
     static constexpr int QTILE = BM * D * 2;                  // [128][D] bf16
     static constexpr int KVTILE = BN * D * 2;                 // [64][D] bf16
     static constexpr int OFF_Q = 0;
     static constexpr int OFF_K = QTILE;
     static constexpr int OFF_V = OFF_K + KST * KVTILE;
-    static constexpr int OFF_P = OFF_V + VST * KVTILE;        // [128][64] bf16 = 16 KB
+    static constexpr int OFF_P = OFF_V + VST * KVTILE;        // (P lives in TMEM; nothing here)
     // d = 64: the row sums are taken by the tensor core as well: PV gets 16 extra B columns of ones, so column D of
     // the accumulator is sum_j P_ij of exactly the (bf16-rounded) probabilities the product used.  The ones live in one
     // more 64-column group, LBO away from the value tile.
     static constexpr bool ONES = D == 64;
-    static constexpr int OFF_ONES = OFF_P + BM * BN * 2;      // [64][64] bf16 ones (8 KB), d = 64 only
+    static constexpr int OFF_ONES = OFF_P;                    // [64][64] bf16 ones (8 KB), d = 64 only
     static constexpr int OFF_BAR = OFF_ONES + (ONES ? BN * 128 : 0);   // mbarriers, tmem slot
     static constexpr int OFF_IDX = OFF_BAR + 128;             // 128 staged list entries
     static constexpr int BYTES = OFF_IDX + 512;
@@ -85,7 +86,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         return;
     }
     PROF(0);
-    const uint32_t sQ = base + S::OFF_Q, sK = base + S::OFF_K, sV = base + S::OFF_V, sP = base + S::OFF_P;
+    const uint32_t sQ = base + S::OFF_Q, sK = base + S::OFF_K, sV = base + S::OFF_V;
     const uint32_t bar_q = base + S::OFF_BAR;
     const uint32_t bar_k0 = bar_q + 8;                         // 3 slots
     const uint32_t bar_v0 = bar_q + 32;                        // 3 slots
@@ -140,7 +141,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             constexpr uint32_t IDESC_O = S::ONES ? instr_desc(BM, D + 16, true) : instr_desc(BM, D, true);
             // descriptor words: lo = (address >> 4) | LBO field, hi = SBO field | version | swizzle mode
             constexpr uint32_t HI = (1024u >> 4) | (1u << 14) | (2u << 29);
-            const uint32_t q_lo = (sQ >> 4) | (1u << 16), k_lo = (sK >> 4) | (1u << 16), p_lo = (sP >> 4) | (1u << 16);
+            const uint32_t q_lo = (sQ >> 4) | (1u << 16), k_lo = (sK >> 4) | (1u << 16);
             const uint32_t v_lo = (sV >> 4) | ((8192u >> 4) << 16);
             uint32_t k_phase = 0, v_phase = 0, g_waited = 0;   // TMA barrier parities (bit per stage); bar_g phases consumed
             auto tma_kv = [&](int t, bool is_v) {              // window tile t -> its stage
@@ -198,7 +199,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                         vb = ((sV + (t % VST) * S::KVTILE) >> 4) | (((base + S::OFF_ONES - sV - (t % VST) * S::KVTILE) >> 4) << 16);
 #pragma unroll
                     for (int kk = 0; kk < BN / 16; ++kk)
-                        umma(tmem + O_COL, desc64(p_lo + kk * 2, HI), desc64(vb + kk * 128, HI), IDESC_O, (t > 0 || kk > 0) ? 1u : 0u);
+                        umma_ts(tmem + O_COL, tmem + (t & 1) * BN + kk * 8, desc64(vb + kk * 128, HI), IDESC_O, (t > 0 || kk > 0) ? 1u : 0u);
                     umma_commit(bar_pv);
                 }
                 // B. S(t+2) into the S buffer softmax(t) has just released
@@ -381,9 +382,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             }
             const float neg_m = m_run == -INFINITY ? 0.f : -m_run;
             float ls[4] = {0.f, 0.f, 0.f, 0.f};
+            uint32_t pk[32];                                   // the row of P as 64 bf16, two per word
 #pragma unroll
             for (int cb = 0; cb < 2; ++cb) {
-                uint32_t pk[16];
                 if (act[cb]) {
 #pragma unroll
                     for (int c = 0; c < 32; c += 2) {
@@ -392,23 +393,19 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                         const float p1 = fast_exp2(fmaf(__uint_as_float(r[cb][c + 1]), c2, neg_m));
                         if (!S::ONES) ls[(c >> 1) & 3] += p0 + p1;   // with ONES the tensor core sums the rounded probabilities
                         __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
-                        pk[c >> 1] = *reinterpret_cast<uint32_t*>(&h);
+                        pk[cb * 16 + (c >> 1)] = *reinterpret_cast<uint32_t*>(&h);
                     }
                 } else {
 #pragma unroll
-                    for (int c = 0; c < 16; ++c) pk[c] = 0u;
-                }
-#pragma unroll
-                for (int g = 0; g < 4; ++g) {
-                    const int ch = cb * 4 + g;
-                    const uint32_t dst = sP + tid * 128 + ((ch ^ (tid & 7)) << 4);
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(pk[4 * g]), "r"(pk[4 * g + 1]),
-                                 "r"(pk[4 * g + 2]), "r"(pk[4 * g + 3]) : "memory");
+                    for (int c = 0; c < 16; ++c) pk[cb * 16 + c] = 0u;
                 }
             }
             l_run += (ls[0] + ls[1]) + (ls[2] + ls[3]);
-            fence_proxy_async();                               // P (generic proxy) -> visible to the MMA (async proxy)
-            tc_fence_before();                                 // our TMEM reads of S(t) are ordered before the arrive
+            // P goes back into TMEM, over the first 32 columns of the S buffer it was computed from (this thread has
+            // all of its row in registers), and feeds the PV product as the A operand: no trip through shared memory
+            tmem_st32(tmem + lane_base + s_col, pk);
+            tmem_wait_st();
+            tc_fence_before();                                 // our TMEM accesses are ordered before the arrive
             mbar_arrive(bar_p);
             PROF(9 + 6 * t);
         }
