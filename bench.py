@@ -181,6 +181,12 @@ def run_lte(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     lte.lib()
     pk = peaks()
+    if args.section and args.skip_main:
+        # only the named section (used for profiler captures of its kernels)
+        flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+        print(json.dumps({"section": args.section,
+                          "extras": extras(torch, lte, synth, pk, lambda: flush_buf.fill_(1), args, only=(args.section,))}))
+        return
 
     cfg = synth.CONFIGS["C2"]
     x = device_inputs(cfg, 1000 + rank, torch)
@@ -487,6 +493,7 @@ def main():
     ap.add_argument("--no-extras", action="store_true")
     ap.add_argument("--section", default=None, choices=["C3", "C4", "C5"],
                     help="time only this extra section (long prefill / decode / forward+backward) after the main loop")
+    ap.add_argument("--skip-main", action="store_true", help="with --section: skip the main C2 loop")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":
