@@ -1,6 +1,6 @@
 // Prefill attention on the 5th-generation tensor cores (Section 3.1.3, "Cached prefilling and decoding").
 //
-// One CTA per 128-query tile of one (b,h): four softmax warps and one control warp.  Key/value tiles of 64
+// One CTA per 128-query tile of one (b,h): four softmax warps, one MMA-issue warp and one load warp.  Key/value tiles of 64
 // rows come from two sources, as in the paper's two-stage loop: (1) the contiguous window span, staged by TMA
 // (cp.async.bulk.tensor, 128-byte swizzle); (2) the retained rows already out of the tile's window, gathered
 // row by row with cp.async into the same swizzled layout (idx is ascending, so the entries a query may see are
@@ -32,7 +32,7 @@ __device__ long long g_prof[160];
 
 namespace {
 
-constexpr int BM = 128, BN = 64, NTHREADS = 160;
+constexpr int BM = 128, BN = 64, NTHREADS = 192;
 using namespace tc;
 __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, int code) { mbar_wait_s(bar, parity, code, &g_prefill_status); }
 
@@ -52,7 +52,7 @@ template <int D> struct Smem {
     static constexpr bool ONES = D == 64;
     static constexpr int OFF_ONES = OFF_P;                    // [64][64] bf16 ones (8 KB), d = 64 only
     static constexpr int OFF_BAR = OFF_ONES + (ONES ? BN * 128 : 0);   // mbarriers, tmem slot
-    static constexpr int OFF_IDX = OFF_BAR + 128;             // 128 staged list entries
+    static constexpr int OFF_IDX = OFF_BAR + 256;             // 128 staged list entries
     static constexpr int BYTES = OFF_IDX + 512;
     static constexpr uint32_t TMEM_COLS = 256;                // S0: [0,64)  S1: [64,128)  O: [128, 128+D) (+16 row-sum columns)
 };
@@ -60,12 +60,15 @@ template <int D> struct Smem {
 __device__ __forceinline__ void softmax_group_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
 // Warps 0-3 (128 threads): softmax (thread r owns query row r) and the cp.async gathers of retained rows.
-// Warp 4, one lane: the TMA loads of Q and of the window tiles, and every tcgen05.mma.  They meet on mbarriers:
+// Warp 4, one lane: every tcgen05.mma.  Warp 5, one lane: the TMA loads of Q and of the window tiles (a single
+// lane doing both was the bottleneck: its dependent instruction stream took longer per tile than the softmax).
+// They meet on mbarriers:
 //   bar_s[b]  (commit)       S(t) is in TMEM buffer b = t & 1                     control -> softmax
 //   bar_p     (128 arrivals) P(t) is in shared memory, S buffer b is free         softmax -> control
 //   bar_pv    (commit)       PV(t) has completed                                   control -> softmax
 //   bar_g[b]  (128 arrivals) gathers issued before the top of tile t have landed   softmax -> control
 //   bar_k[s], bar_v[s]       TMA transaction barriers of the window tiles
+//   bar_kf[s], bar_vf[s]     (commit) the MMA that read stage s has completed          MMA lane -> load lane
 // S(t+1) and S(t+2) are computed while the softmax of tile t runs; loads run two to three tiles ahead.
 template <int D>
 __global__ void __launch_bounds__(NTHREADS, 2)
@@ -93,8 +96,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     const uint32_t bar_s0 = bar_q + 56;                        // 2 slots
     const uint32_t bar_g0 = bar_q + 72;                        // 2 slots
     const uint32_t bar_p = bar_q + 88, bar_pv = bar_q + 96;
-    const uint32_t tmem_slot = bar_q + 104;
-    volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(smem_raw + S::OFF_BAR + 104);
+    const uint32_t bar_kf0 = bar_q + 104;                      // 3 slots: K stage free
+    const uint32_t bar_vf0 = bar_q + 128;                      // 3 slots: V stage free
+    const uint32_t tmem_slot = bar_q + 152;
+    volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(smem_raw + S::OFF_BAR + 152);
     volatile int* s_idx = reinterpret_cast<volatile int*>(smem_raw + S::OFF_IDX);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -105,11 +110,15 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     const int n_win = (i_hi - j_start + 1 + BN - 1) / BN;
     const int32_t* id = idx + (size_t)bh * R;
     const int n_ret = cnt[bh];
+    const int g_first = max(n_win - Smem<D>::KST, 0);        // first tile whose top may have gathers in flight
 
     if (tid == 0) {
         mbar_init(bar_q, 1);
 #pragma unroll
-        for (int s2 = 0; s2 < 3; ++s2) { mbar_init(bar_k0 + 8 * s2, 1); mbar_init(bar_v0 + 8 * s2, 1); }
+        for (int s2 = 0; s2 < 3; ++s2) {
+            mbar_init(bar_k0 + 8 * s2, 1); mbar_init(bar_v0 + 8 * s2, 1);
+            mbar_init(bar_kf0 + 8 * s2, 1); mbar_init(bar_vf0 + 8 * s2, 1);
+        }
         mbar_init(bar_s0, 1); mbar_init(bar_s0 + 8, 1);
         mbar_init(bar_g0, 128); mbar_init(bar_g0 + 8, 128);
         mbar_init(bar_p, 128); mbar_init(bar_pv, 1);
@@ -122,8 +131,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     const uint32_t tmem = *tmem_slot_gen;
     PROF(1);
 
-    if (warp == 4) {
-        // =================================== control warp (one lane) ========================================
+    if (warp >= 4) {
+        // ============================ load lane (warp 5) and MMA lane (warp 4) ==============================
         // number of tiles: retained entries visible to the last row of the tile (idx ascending => a prefix)
         int nv_max = 0;
         {
@@ -136,86 +145,107 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             }
         }
         const int n_tiles = n_win + (nv_max + BN - 1) / BN;
-        if (lane == 0) {
+        if (warp == 5 && lane == 0) {
+            // ---- load lane: Q, then the window tiles, each into its stage as soon as the MMA that read the
+            //      stage's previous tile has completed (bar_kf / bar_vf, one phase per use of a stage)
+            mbar_expect_tx(bar_q, S::QTILE);
+#pragma unroll
+            for (int sb = 0; sb < SUB; ++sb) tma_load_3d(sQ + sb * 16384, &tmQ, sb * 64, i0, bh, bar_q);
+            int ks = 0, vs = 0;                                // stage of the next K / V tile to load
+            uint32_t kf_par = 0, vf_par = 0;                   // parity bit per stage of the "free" barriers
+            int tk = 0, tv = 0;                                // next window tile to load
+            int y = j_start;
+            for (; tk < KST && tk < n_win; ++tk, y += BN) {
+                mbar_expect_tx(bar_k0 + 8 * tk, S::KVTILE);
+#pragma unroll
+                for (int sb = 0; sb < SUB; ++sb) tma_load_3d(sK + tk * S::KVTILE + sb * 8192, &tmK, sb * 64, y, bh, bar_k0 + 8 * tk);
+            }
+            y = j_start;
+            for (; tv < VST && tv < n_win; ++tv, y += BN) {
+                mbar_expect_tx(bar_v0 + 8 * tv, S::KVTILE);
+#pragma unroll
+                for (int sb = 0; sb < SUB; ++sb) tma_load_3d(sV + tv * S::KVTILE + sb * 8192, &tmV, sb * 64, y, bh, bar_v0 + 8 * tv);
+            }
+            while (tk < n_win || tv < n_win) {
+                if (tk < n_win) {                              // K(tk) into the stage of K(tk - KST)
+                    mbar_wait(bar_kf0 + 8 * ks, (kf_par >> ks) & 1u, 6);
+                    kf_par ^= 1u << ks;
+                    mbar_expect_tx(bar_k0 + 8 * ks, S::KVTILE);
+#pragma unroll
+                    for (int sb = 0; sb < SUB; ++sb)
+                        tma_load_3d(sK + ks * S::KVTILE + sb * 8192, &tmK, sb * 64, j_start + tk * BN, bh, bar_k0 + 8 * ks);
+                    ++tk;
+                    ks = ks + 1 == KST ? 0 : ks + 1;
+                }
+                if (tv < n_win) {                              // V(tv) into the stage of V(tv - VST)
+                    mbar_wait(bar_vf0 + 8 * vs, (vf_par >> vs) & 1u, 8);
+                    vf_par ^= 1u << vs;
+                    mbar_expect_tx(bar_v0 + 8 * vs, S::KVTILE);
+#pragma unroll
+                    for (int sb = 0; sb < SUB; ++sb)
+                        tma_load_3d(sV + vs * S::KVTILE + sb * 8192, &tmV, sb * 64, j_start + tv * BN, bh, bar_v0 + 8 * vs);
+                    ++tv;
+                    vs = vs + 1 == VST ? 0 : vs + 1;
+                }
+            }
+        } else if (warp == 4 && lane == 0) {
+            // ---- MMA lane: nothing but barrier waits and tcgen05 issue; stage indices and parities roll
             constexpr uint32_t IDESC_S = instr_desc(BM, BN, false);
             constexpr uint32_t IDESC_O = S::ONES ? instr_desc(BM, D + 16, true) : instr_desc(BM, D, true);
             // descriptor words: lo = (address >> 4) | LBO field, hi = SBO field | version | swizzle mode
             constexpr uint32_t HI = (1024u >> 4) | (1u << 14) | (2u << 29);
             const uint32_t q_lo = (sQ >> 4) | (1u << 16), k_lo = (sK >> 4) | (1u << 16);
-            const uint32_t v_lo = (sV >> 4) | ((8192u >> 4) << 16);
-            uint32_t k_phase = 0, v_phase = 0, g_waited = 0;   // TMA barrier parities (bit per stage); bar_g phases consumed
-            auto tma_kv = [&](int t, bool is_v) {              // window tile t -> its stage
-                const int st = is_v ? (t % VST) : (t % KST);
-                const uint32_t dst = (is_v ? sV : sK) + st * S::KVTILE;
-                const uint32_t bar = (is_v ? bar_v0 : bar_k0) + 8 * st;
-                mbar_expect_tx(bar, S::KVTILE);
-                const int y = j_start + t * BN;
+            // value operand: the second 64-column group of B is the next sub-tile (d = 128) or the block of ones
+            // (d = 64, LBO = its distance from the value stage)
+            uint32_t v_desc[VST];
 #pragma unroll
-                for (int sb = 0; sb < SUB; ++sb) tma_load_3d(dst + sb * 8192, is_v ? &tmV : &tmK, sb * 64, y, bh, bar);
+            for (int st = 0; st < VST; ++st) {
+                const uint32_t va = sV + st * S::KVTILE;
+                v_desc[st] = (va >> 4) | ((S::ONES ? ((base + S::OFF_ONES - va) >> 4) : (8192u >> 4)) << 16);
+            }
+            uint32_t k_par = 0, v_par = 0, g_waited = 0;       // TMA barrier parities (bit per stage); bar_g phases consumed
+            int ks = 0, vs = 0;                                // stage of the next S / PV operand
+            int ts = 0;                                        // next S tile to issue
+            // gathers issued before the top of tile t have landed (the softmax warps signal from tile g_first on)
+            auto need_g = [&](int t) {
+                while ((int)g_waited <= t - g_first) { mbar_wait(bar_g0 + 8 * (g_waited & 1), (g_waited >> 1) & 1, 10); ++g_waited; }
             };
-            auto need_g = [&](uint32_t phase) {                // gathers issued before the top of tile `phase` have landed
-                while (g_waited <= phase) { mbar_wait(bar_g0 + 8 * (g_waited & 1), (g_waited >> 1) & 1, 10); ++g_waited; }
-            };
-            auto wait_k = [&](int t) {
-                if (t < n_win) { const int st = t % KST; mbar_wait(bar_k0 + 8 * st, (k_phase >> st) & 1u, 2); k_phase ^= 1u << st; }
-            };
-            auto wait_v = [&](int t) {
-                if (t < n_win) { const int st = t % VST; mbar_wait(bar_v0 + 8 * st, (v_phase >> st) & 1u, 4); v_phase ^= 1u << st; }
-            };
-            auto mma_s = [&](int t) {
-                const uint32_t kb = k_lo + (uint32_t)(t % KST) * (S::KVTILE >> 4);
-                const uint32_t dcol = tmem + (t & 1) * BN;
+            auto mma_s = [&]() {                               // S(ts) from K stage ks into S buffer ts & 1
+                if (ts < n_win) { mbar_wait(bar_k0 + 8 * ks, (k_par >> ks) & 1u, 2); k_par ^= 1u << ks; }
+                tc_fence_after();
+                const uint32_t kb = k_lo + (uint32_t)ks * (S::KVTILE >> 4);
+                const uint32_t dcol = tmem + (ts & 1) * BN;
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk)
                     umma(dcol, desc64(q_lo + (kk >> 2) * 1024 + (kk & 3) * 2, HI), desc64(kb + (kk >> 2) * 512 + (kk & 3) * 2, HI),
                          IDESC_S, kk > 0);
-                umma_commit(bar_s0 + 8 * (t & 1));
+                umma_commit(bar_s0 + 8 * (ts & 1));
+                umma_commit(bar_kf0 + 8 * ks);                 // the K stage is free once S(ts) has completed
+                ++ts;
+                ks = ks + 1 == KST ? 0 : ks + 1;
             };
-
-            mbar_expect_tx(bar_q, S::QTILE);
-#pragma unroll
-            for (int sb = 0; sb < SUB; ++sb) tma_load_3d(sQ + sb * 16384, &tmQ, sb * 64, i0, bh, bar_q);
-            for (int t = 0; t < KST && t < n_win; ++t) tma_kv(t, false);
-            for (int t = 0; t < VST && t < n_win; ++t) tma_kv(t, true);
 
             need_g(0);                                         // the softmax warps' prologue gathers
             mbar_wait(bar_q, 0, 1);
-            wait_k(0);
-            tc_fence_after();
-            mma_s(0);
-            if (n_tiles > 1) { wait_k(1); mma_s(1); }
-            // K(KST) reuses the stage of K(0): S(0) must have completed
-            if (KST < n_win) { mbar_wait(bar_s0, 0, 6); tma_kv(KST, false); }
-
+            mma_s();
+            if (n_tiles > 1) mma_s();
             for (int t = 0; t < n_tiles; ++t) {
-                // A. PV(t)
+                // PV(t): everything but P is normally there long before
                 need_g(t);
-                mbar_wait(bar_p, t & 1, 7);
-                wait_v(t);
-                tc_fence_after();
-                {
-                    uint32_t vb = v_lo + (uint32_t)(t % VST) * (S::KVTILE >> 4);
-                    if (S::ONES)   // second 64-column group of B = the block of ones: LBO = its distance from this value tile
-                        vb = ((sV + (t % VST) * S::KVTILE) >> 4) | (((base + S::OFF_ONES - sV - (t % VST) * S::KVTILE) >> 4) << 16);
+                if (t < n_win) { mbar_wait(bar_v0 + 8 * vs, (v_par >> vs) & 1u, 4); v_par ^= 1u << vs; }
+                uint32_t vb = v_desc[0];
 #pragma unroll
-                    for (int kk = 0; kk < BN / 16; ++kk)
-                        umma_ts(tmem + O_COL, tmem + (t & 1) * BN + kk * 8, desc64(vb + kk * 128, HI), IDESC_O, (t > 0 || kk > 0) ? 1u : 0u);
-                    umma_commit(bar_pv);
-                }
-                // B. S(t+2) into the S buffer softmax(t) has just released
-                if (t + 2 < n_tiles) {
-                    if (KST == 2) need_g(t + 1);
-                    wait_k(t + 2);
-                    mma_s(t + 2);
-                }
-                // C. window K(t+1+KST) reuses the stage of K(t+1): S(t+1) must have completed
-                if (t + 1 + KST < n_win) {
-                    mbar_wait(bar_s0 + 8 * ((t + 1) & 1), ((t + 1) >> 1) & 1, 6);
-                    tma_kv(t + 1 + KST, false);
-                }
-                // D. window V(t-1+VST) reuses the stage of V(t-1); PV(t-1) is known to be complete because the
-                //    softmax warps waited for it before they produced P(t)
-                if (t >= 1 && t - 1 + VST < n_win) tma_kv(t - 1 + VST, true);
+                for (int st = 1; st < VST; ++st) vb = vs == st ? v_desc[st] : vb;
+                mbar_wait(bar_p, t & 1, 7);
+                tc_fence_after();
+#pragma unroll
+                for (int kk = 0; kk < BN / 16; ++kk)
+                    umma_ts(tmem + O_COL, tmem + (t & 1) * BN + kk * 8, desc64(vb + kk * 128, HI), IDESC_O, (t > 0 || kk > 0) ? 1u : 0u);
+                umma_commit(bar_pv);
+                umma_commit(bar_vf0 + 8 * vs);                 // the V stage is free once PV(t) has completed
+                vs = vs + 1 == VST ? 0 : vs + 1;
+                // S(t+2) into the S buffer softmax(t) has just released
+                if (ts < n_tiles) mma_s();
             }
         }
     } else {
@@ -295,9 +325,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             gather_rows(t + KST, rk);
             gather_rows(t + VST - 1, rv);
             // gathers issued before this point have landed (all of them, or all but the latest value tile)
-            if (VST == 3) cp_async_wait<1>(); else cp_async_wait<0>();
-            fence_proxy_async();
-            mbar_arrive(bar_g0 + 8 * (t & 1));
+            if (t >= g_first) {
+                if (VST == 3) cp_async_wait<1>(); else cp_async_wait<0>();
+                fence_proxy_async();
+                mbar_arrive(bar_g0 + 8 * ((t - g_first) & 1));
+            }
 
             // column range this row may see in the tile
             int c_lo, c_hi;
@@ -357,17 +389,15 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             }
             const float m_tile = fmaxf(fmaxf(mr[0], mr[1]), fmaxf(mr[2], mr[3])) * c2;
             PROF(7 + 6 * t);
-            // PV(t-1) must be done before O is rescaled or P is overwritten
-            if (t > 0) { mbar_wait(bar_pv, (t - 1) & 1, 4); tc_fence_after(); }
             PROF(8 + 6 * t);
-            // value tile t+VST-1 goes into the stage of V(t-1), which PV(t-1) has finished reading
-            if (t > 0) gather_issue(t + VST - 1, true, rv); else cp_async_commit();
             // lazy rescale: the running max only moves when the new one is far above it (exp2 arguments stay <= 8)
             float alpha = 1.f;
             bool need = false;
             if (m_run == -INFINITY) m_run = m_tile;             // nothing accumulated yet for this row: O row is 0
             else if (m_tile > m_run + 8.f) { alpha = fast_exp2(m_run - m_tile); m_run = m_tile; need = true; }
             if (__any_sync(0xffffffffu, need)) {
+                // PV(t-1) must be done before O is rescaled
+                if (t > 0) { mbar_wait(bar_pv, (t - 1) & 1, 4); tc_fence_after(); }
 #pragma unroll
                 for (int cb = 0; cb < D / 32 + (S::ONES ? 1 : 0); ++cb) {   // with ONES the row-sum columns are rescaled too
                     uint32_t q4[32];
@@ -406,7 +436,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             tmem_st32(tmem + lane_base + s_col, pk);
             tmem_wait_st();
             tc_fence_before();                                 // our TMEM accesses are ordered before the arrive
+            // PV(t-1) has normally completed long ago; the wait sits before the arrive so that the barrier cannot
+            // run two phases ahead of this thread
+            if (t > 0) mbar_wait(bar_pv, (t - 1) & 1, 4);
             mbar_arrive(bar_p);
+            // value tile t+VST-1 goes into the stage of V(t-1), which PV(t-1) has finished reading
+            if (t > 0) gather_issue(t + VST - 1, true, rv); else cp_async_commit();
             PROF(9 + 6 * t);
         }
         PROF(50);
