@@ -371,12 +371,17 @@ bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     const uint32_t base = smem_u32(smem_raw);
     if ((base & 1023u) != 0) { if (threadIdx.x == 0) atomicExch(&g_bwd_status, 9); return; }
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int bh = blockIdx.y;
-    const bool is_ret = (int)blockIdx.x >= n_wt;
+    // the retained tiles walk many more query blocks than the window tiles: they take the lowest block numbers so
+    // that they start first and do not form the tail of the launch
+    const int n_rt = (int)gridDim.x - n_wt;
+    const int lin = blockIdx.y * gridDim.x + blockIdx.x, tot_ret = n_rt * (int)gridDim.y;
+    const bool is_ret = lin < tot_ret;
+    const int bh = is_ret ? lin / n_rt : (lin - tot_ret) / n_wt;
+    const int tile = is_ret ? lin % n_rt : (lin - tot_ret) % n_wt;
     const int n_ret = cnt[bh];
     const int32_t* id = idx + (size_t)bh * R;
-    const int j0 = is_ret ? 0 : blockIdx.x * 128;              // window tile: first key
-    const int e0 = is_ret ? ((int)blockIdx.x - n_wt) * 128 : 0;   // retained tile: first list entry
+    const int j0 = is_ret ? 0 : tile * 128;                    // window tile: first key
+    const int e0 = is_ret ? tile * 128 : 0;                    // retained tile: first list entry
     if (is_ret && e0 >= n_ret) return;                         // nothing retained in this slice of the list
 
     // query blocks that can see the tile
