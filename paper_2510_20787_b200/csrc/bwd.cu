@@ -304,162 +304,163 @@ __global__ void __launch_bounds__(256) bwd_finish_inplace_kernel(const float* __
     }
 }
 
-// Tensor-core path, K = 5 or 7: one pass over the rows of k, v, dk, dv does both scorer jobs.  A block takes TAIL_ROWS
-// consecutive positions of one (b,h); a thread owns 8 channels of k or of v (16-byte accesses) and walks the
-// block's rows: dw partials acc[t][c] += dz[p - t + half] x[p][c], and (FINISH) the scorer's input gradient
-// sum_t dz[p - t + half] w[h,t,c] added onto the bf16 dk, dv rows in place.  The partials of the threads that
-// own the same channels are added in a fixed order (shuffle, then a tree over the warps through shared memory).
-constexpr int TAIL_ROWS = 512;
+// Tensor-core path, K = 5 or 7: one pass over the rows of k, v, dk, dv does both scorer jobs.  A block takes `rows`
+// consecutive positions of one (b,h); a thread owns 4 channels of x = [k ; v] for every row it visits, so its
+// K x 4 scorer weights stay in registers, and walks the block's rows: dw partials acc[t][c] += dz[p - t + half] x[p][c],
+// and (FINISH) the scorer's input gradient sum_t dz[p - t + half] w[h,t,c] added onto the bf16 dk, dv rows in place.
+// The partials of the threads that own the same channels are added in a fixed order (a tree over the row slots
+// through shared memory).
+constexpr int TAIL_MIN_ROWS = 256, TAIL_MAX_ROWS = 1024;   // rows per block are chosen per launch to fill whole waves
 template <int D, int K, bool FINISH>
 __global__ void __launch_bounds__(256, 2)
 bwd_tail_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v, const float* __restrict__ dz,
                 const float* __restrict__ w, __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv,
-                float* __restrict__ part_w, float* __restrict__ part_b, int B, int H, int Tlen, int nchunk)
+                float* __restrict__ part_w, float* __restrict__ part_b, int B, int H, int Tlen, int nchunk, int rows)
 {
-    constexpr int TPR = 2 * D / 8;                  // threads per position: D/8 for k, D/8 for v
-    constexpr int RPP = 256 / TPR;                  // positions per pass
+    constexpr int TPR = 2 * D / 4;                  // threads per position: D/4 for k, D/4 for v
+    constexpr int RPP = 256 / TPR;                  // positions per pass (row slots)
     constexpr int half = K / 2;
-    constexpr int NDZ = (TAIL_ROWS + K - 1 + 3) & ~3;
+    const int NDZ = (rows + K - 1 + 3) & ~3;
     extern __shared__ float sm[];
-    float* ws = sm;                                 // [K][2D]
-    float* dzs = sm + K * 2 * D;                    // dz[p0-half .. p0+TAIL_ROWS-1+half]
-    float* red = dzs + NDZ;                         // [4][K][2D]
+    float* dzs = sm;                                // dz[p0-half .. p0+rows-1+half]
+    float* red = dzs + NDZ;                         // [RPP/2][K][2D]
     const int h = blockIdx.y;
     const int b = blockIdx.x / nchunk, ch = blockIdx.x % nchunk;
     const int bh = b * H + h;
-    const int p0 = ch * TAIL_ROWS;
+    const int p0 = ch * rows;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    if (FINISH)
-        for (int i = tid; i < K * 2 * D; i += 256) ws[i] = w[(size_t)h * K * 2 * D + i];
-    for (int a = tid; a < TAIL_ROWS + K - 1; a += 256) {
+    for (int a = tid; a < rows + K - 1; a += 256) {
         const int j = p0 - half + a;
         dzs[a] = (j >= 0 && j + half <= Tlen - 1) ? dz[(size_t)bh * Tlen + j] : 0.f;
     }
-    __syncthreads();
-    const int sel = tid % TPR, r0 = tid / TPR;
-    const bool isv = sel >= D / 8;
-    const int cc = (sel % (D / 8)) * 8;             // first of this thread's 8 channels within k or v
-    const int cx = (isv ? D : 0) + cc;              // the same in x = [k ; v]
+    const int cg = tid % TPR, r0 = tid / TPR;       // channel group: x channels [4 cg, 4 cg + 4); row slot
+    const bool isv = cg >= D / 4;
+    const int cc = (cg % (D / 4)) * 4;              // first of this thread's 4 channels within k or v
     const __nv_bfloat16* src = isv ? v : k;
     __nv_bfloat16* gdst = isv ? dv : dk;
-    float acc[K][8];
+    float wr[K][4];                                 // this thread's scorer weights
+    if (FINISH) {
+#pragma unroll
+        for (int t = 0; t < K; ++t) {
+            const float4 w4 = *reinterpret_cast<const float4*>(&w[((size_t)h * K + t) * 2 * D + cg * 4]);
+            wr[t][0] = w4.x; wr[t][1] = w4.y; wr[t][2] = w4.z; wr[t][3] = w4.w;
+        }
+    }
+    __syncthreads();
+    float acc[K][4];
 #pragma unroll
     for (int t = 0; t < K; ++t)
 #pragma unroll
-        for (int e = 0; e < 8; ++e) acc[t][e] = 0.f;
-#pragma unroll 2
-    for (int rl = r0; rl < TAIL_ROWS; rl += RPP) {
-        const int p = p0 + rl;
-        if (p >= Tlen) break;
-        const size_t a0 = ((size_t)bh * Tlen + p) * D + cc;
-        const uint4 ux = *reinterpret_cast<const uint4*>(src + a0);
-        uint4 ug = make_uint4(0u, 0u, 0u, 0u);
-        if (FINISH) ug = *reinterpret_cast<const uint4*>(gdst + a0);
-        const uint32_t xw[4] = {ux.x, ux.y, ux.z, ux.w};
-        float x[8], g[K];
+        for (int e = 0; e < 4; ++e) acc[t][e] = 0.f;
+    // U rows per batch: all of a batch's loads are issued before any of its arithmetic (row indices are clamped so
+    // that every load is legal; rows past the end are skipped afterwards)
+    constexpr int U = 8;
+    for (int rb = r0; rb < rows; rb += RPP * U) {
+        uint2 ux[U], ug[U];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) { x[2 * e] = __uint_as_float(xw[e] << 16); x[2 * e + 1] = __uint_as_float(xw[e] & 0xffff0000u); }
+        for (int u = 0; u < U; ++u) {
+            const int p = min(p0 + rb + u * RPP, Tlen - 1);
+            const size_t a0 = ((size_t)bh * Tlen + p) * D + cc;
+            ux[u] = *reinterpret_cast<const uint2*>(src + a0);
+            if (FINISH) ug[u] = *reinterpret_cast<const uint2*>(gdst + a0);
+        }
 #pragma unroll
-        for (int t = 0; t < K; ++t) g[t] = dzs[rl - t + 2 * half];      // dz[p - t + half]
+        for (int u = 0; u < U; ++u) {
+            const int rl = rb + u * RPP, p = p0 + rl;
+            if (rl >= rows || p >= Tlen) continue;
+            float x[4], g[K];
+            x[0] = __uint_as_float(ux[u].x << 16); x[1] = __uint_as_float(ux[u].x & 0xffff0000u);
+            x[2] = __uint_as_float(ux[u].y << 16); x[3] = __uint_as_float(ux[u].y & 0xffff0000u);
 #pragma unroll
-        for (int t = 0; t < K; ++t)
+            for (int t = 0; t < K; ++t) g[t] = dzs[rl - t + 2 * half];      // dz[p - t + half]
 #pragma unroll
-            for (int e = 0; e < 8; ++e) acc[t][e] = fmaf(g[t], x[e], acc[t][e]);
-        if (FINISH) {
-            float gi[8];
+            for (int t = 0; t < K; ++t)
 #pragma unroll
-            for (int e = 0; e < 8; ++e) gi[e] = 0.f;
+                for (int e = 0; e < 4; ++e) acc[t][e] = fmaf(g[t], x[e], acc[t][e]);
+            if (FINISH) {
+                float gi[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int t = 0; t < K; ++t) {
-                const float4 wa = *reinterpret_cast<const float4*>(&ws[t * 2 * D + cx]);
-                const float4 wb = *reinterpret_cast<const float4*>(&ws[t * 2 * D + cx + 4]);
-                gi[0] = fmaf(g[t], wa.x, gi[0]); gi[1] = fmaf(g[t], wa.y, gi[1]); gi[2] = fmaf(g[t], wa.z, gi[2]); gi[3] = fmaf(g[t], wa.w, gi[3]);
-                gi[4] = fmaf(g[t], wb.x, gi[4]); gi[5] = fmaf(g[t], wb.y, gi[5]); gi[6] = fmaf(g[t], wb.z, gi[6]); gi[7] = fmaf(g[t], wb.w, gi[7]);
+                for (int t = 0; t < K; ++t)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) gi[e] = fmaf(g[t], wr[t][e], gi[e]);
+                __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(ug[u].x << 16) + gi[0], __uint_as_float(ug[u].x & 0xffff0000u) + gi[1]);
+                __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(ug[u].y << 16) + gi[2], __uint_as_float(ug[u].y & 0xffff0000u) + gi[3]);
+                *reinterpret_cast<uint2*>(gdst + ((size_t)bh * Tlen + p) * D + cc) =
+                    make_uint2(*reinterpret_cast<uint32_t*>(&h0), *reinterpret_cast<uint32_t*>(&h1));
             }
-            uint32_t gw[4] = {ug.x, ug.y, ug.z, ug.w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                __nv_bfloat162 hh = __floats2bfloat162_rn(__uint_as_float(gw[e] << 16) + gi[2 * e],
-                                                          __uint_as_float(gw[e] & 0xffff0000u) + gi[2 * e + 1]);
-                gw[e] = *reinterpret_cast<uint32_t*>(&hh);
-            }
-            *reinterpret_cast<uint4*>(gdst + a0) = make_uint4(gw[0], gw[1], gw[2], gw[3]);
         }
     }
-    // ---- add the partials of the threads that own the same channels ---------------------------------------
-    if (TPR == 16) {                                // two positions per warp: lanes l and l + 16
+    // ---- add the partials of the row slots: slots [step, 2 step) hand their sums to slots [0, step) ---------
 #pragma unroll
-        for (int t = 0; t < K; ++t)
+    for (int step = RPP / 2; step >= 1; step >>= 1) {
+        if (r0 >= step && r0 < 2 * step) {
+            float* dst = red + (size_t)(r0 - step) * K * 2 * D;
 #pragma unroll
-            for (int e = 0; e < 8; ++e) acc[t][e] += __shfl_xor_sync(0xffffffffu, acc[t][e], 16);
-    }
-    const bool owner = TPR == 32 || lane < 16;      // one lane per channel group and warp
-    const int cg = TPR == 32 ? lane : (lane & 15);  // channel group: x channels [8 cg, 8 cg + 8)
-#pragma unroll
-    for (int step = 4; step >= 1; step >>= 1) {     // warps [step, 2 step) hand their sums to warps [0, step)
-        if (warp >= step && warp < 2 * step && owner) {
-            float* dst = red + (size_t)(warp - step) * K * 2 * D;
-#pragma unroll
-            for (int t = 0; t < K; ++t) {
-                *reinterpret_cast<float4*>(&dst[t * 2 * D + cg * 8]) = make_float4(acc[t][0], acc[t][1], acc[t][2], acc[t][3]);
-                *reinterpret_cast<float4*>(&dst[t * 2 * D + cg * 8 + 4]) = make_float4(acc[t][4], acc[t][5], acc[t][6], acc[t][7]);
-            }
+            for (int t = 0; t < K; ++t)
+                *reinterpret_cast<float4*>(&dst[t * 2 * D + cg * 4]) = make_float4(acc[t][0], acc[t][1], acc[t][2], acc[t][3]);
         }
         __syncthreads();
-        if (warp < step && owner) {
-            const float* s2 = red + (size_t)warp * K * 2 * D;
+        if (r0 < step) {
+            const float* s2 = red + (size_t)r0 * K * 2 * D;
 #pragma unroll
             for (int t = 0; t < K; ++t) {
-                const float4 a = *reinterpret_cast<const float4*>(&s2[t * 2 * D + cg * 8]);
-                const float4 c = *reinterpret_cast<const float4*>(&s2[t * 2 * D + cg * 8 + 4]);
+                const float4 a = *reinterpret_cast<const float4*>(&s2[t * 2 * D + cg * 4]);
                 acc[t][0] += a.x; acc[t][1] += a.y; acc[t][2] += a.z; acc[t][3] += a.w;
-                acc[t][4] += c.x; acc[t][5] += c.y; acc[t][6] += c.z; acc[t][7] += c.w;
             }
         }
         __syncthreads();
     }
-    if (warp == 0 && owner) {
+    if (r0 == 0) {
         float* out = part_w + ((size_t)h * B * nchunk + blockIdx.x) * K * 2 * D;
 #pragma unroll
-        for (int t = 0; t < K; ++t) {
-            *reinterpret_cast<float4*>(&out[t * 2 * D + cg * 8]) = make_float4(acc[t][0], acc[t][1], acc[t][2], acc[t][3]);
-            *reinterpret_cast<float4*>(&out[t * 2 * D + cg * 8 + 4]) = make_float4(acc[t][4], acc[t][5], acc[t][6], acc[t][7]);
-        }
+        for (int t = 0; t < K; ++t)
+            *reinterpret_cast<float4*>(&out[t * 2 * D + cg * 4]) = make_float4(acc[t][0], acc[t][1], acc[t][2], acc[t][3]);
     }
     if (warp == 7) {                                // bias partial: the dz of the block's own positions
         float sb = 0.f;
-        for (int a = lane; a < TAIL_ROWS; a += 32) sb += dzs[a + half];
+        for (int a = lane; a < rows; a += 32) sb += dzs[a + half];
 #pragma unroll
         for (int o = 16; o >= 1; o >>= 1) sb += __shfl_xor_sync(0xffffffffu, sb, o);
         if (lane == 0) part_b[(size_t)h * B * nchunk + blockIdx.x] = sb;
     }
 }
 
+// Rows per block for the fused pass: between TAIL_MIN_ROWS and TAIL_MAX_ROWS, such that the grid fills whole waves of
+// the resident-block slots as well as possible (ties: fewer, larger blocks).  Returns the chunks per sequence.
+inline int tail_chunks(const Params& p, int* rows_out)
+{
+    static int slots = 0;
+    if (slots == 0) {
+        int dev = 0, sms = 148;
+        if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        slots = 2 * sms;
+    }
+    const int lo = (p.T + TAIL_MAX_ROWS - 1) / TAIL_MAX_ROWS, hi = (p.T + TAIL_MIN_ROWS - 1) / TAIL_MIN_ROWS;
+    int best = lo;
+    double best_eff = -1.0;
+    for (int n = lo; n <= hi; ++n) {
+        const double waves = (double)p.B * p.H * n / slots;
+        const double eff = waves / (double)(long long)(waves + 0.999999);
+        if (eff > best_eff + 1e-9) { best_eff = eff; best = n; }
+    }
+    int rows = (p.T + best - 1) / best;
+    rows = (rows + 7) / 8 * 8;                      // a multiple of every kernel's rows per pass
+    *rows_out = rows;
+    return (p.T + rows - 1) / rows;
+}
+
 template <int D, int K>
 int run_tail(const Params& p, const void* k, const void* v, const float* dz, void* dk, void* dv, float* part_w,
-             float* part_b, bool finish, int nchunk, cudaStream_t st)
+             float* part_b, bool finish, int nchunk, int rows, cudaStream_t st)
 {
-    const size_t sm = (size_t)(K * 2 * D + ((TAIL_ROWS + K - 1 + 3) & ~3) + 4 * K * 2 * D) * sizeof(float);
+    const size_t sm = (size_t)(((rows + K - 1 + 3) & ~3) + (256 / (2 * D / 4) / 2) * K * 2 * D) * sizeof(float);
     dim3 grid(p.B * nchunk, p.H);
-    if (finish) {
-        static bool done = false;
-        if (!done) {
-            if (cudaFuncSetAttribute(bwd_tail_kernel<D, K, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm) != cudaSuccess)
-                return LTE_ERR_CUDA;
-            done = true;
-        }
+    if (finish)
         bwd_tail_kernel<D, K, true><<<grid, 256, sm, st>>>((const __nv_bfloat16*)k, (const __nv_bfloat16*)v, dz, p.w,
-                                                          (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, part_w, part_b, p.B, p.H, p.T, nchunk);
-    } else {
-        static bool done = false;
-        if (!done) {
-            if (cudaFuncSetAttribute(bwd_tail_kernel<D, K, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm) != cudaSuccess)
-                return LTE_ERR_CUDA;
-            done = true;
-        }
+                                                          (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, part_w, part_b, p.B, p.H, p.T, nchunk, rows);
+    else
         bwd_tail_kernel<D, K, false><<<grid, 256, sm, st>>>((const __nv_bfloat16*)k, (const __nv_bfloat16*)v, dz, p.w,
-                                                           (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, part_w, part_b, p.B, p.H, p.T, nchunk);
-    }
+                                                           (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, part_w, part_b, p.B, p.H, p.T, nchunk, rows);
     return cuda_status(cudaGetLastError());
 }
 
@@ -526,9 +527,10 @@ int run(const Params& p, const void* q, const void* k, const void* v, const void
     dim3 gr((per_head + 255) / 256, p.H);
     if constexpr (sizeof(T) == 2 && (D == 64 || D == 128)) {
         if (p.K == 5 || p.K == 7) {                   // fused pass: dw partials and the scorer's input gradient
-            const int nch = (p.T + TAIL_ROWS - 1) / TAIL_ROWS;
-            const int e = p.K == 7 ? run_tail<D, 7>(p, k, v, dz, dk, dv, part_w, part_b, f32, nch, st)
-                                   : run_tail<D, 5>(p, k, v, dz, dk, dv, part_w, part_b, f32, nch, st);
+            int rows = 0;
+            const int nch = tail_chunks(p, &rows);
+            const int e = p.K == 7 ? run_tail<D, 7>(p, k, v, dz, dk, dv, part_w, part_b, f32, nch, rows, st)
+                                   : run_tail<D, 5>(p, k, v, dz, dk, dv, part_w, part_b, f32, nch, rows, st);
             if (e != LTE_OK) return e;
             bwd_conv_reduce_kernel<<<gr, 256, 0, st>>>(part_w, part_b, dw, dbias, p.B * nch, per_head);
             return cuda_status(cudaGetLastError());
