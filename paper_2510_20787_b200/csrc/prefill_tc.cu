@@ -52,12 +52,10 @@ template <int D> struct Smem {
     static constexpr bool ONES = D == 64;
     static constexpr int OFF_ONES = OFF_P;                    // [64][64] bf16 ones (8 KB), d = 64 only
     static constexpr int OFF_BAR = OFF_ONES + (ONES ? BN * 128 : 0);   // mbarriers, tmem slot
-    static constexpr int OFF_IDX = OFF_BAR + 256;             // 128 staged list entries
-    static constexpr int BYTES = OFF_IDX + 512;
+    static constexpr int BYTES = OFF_BAR + 256;
     static constexpr uint32_t TMEM_COLS = 256;                // S0: [0,64)  S1: [64,128)  O: [128, 128+D) (+16 row-sum columns)
 };
 
-__device__ __forceinline__ void softmax_group_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
 // Warps 0-3 (128 threads): softmax (thread r owns query row r) and the cp.async gathers of retained rows.
 // Warp 4, one lane: every tcgen05.mma.  Warp 5, one lane: the TMA loads of Q and of the window tiles (a single
@@ -100,7 +98,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     const uint32_t bar_vf0 = bar_q + 128;                      // 3 slots: V stage free
     const uint32_t tmem_slot = bar_q + 152;
     volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(smem_raw + S::OFF_BAR + 152);
-    volatile int* s_idx = reinterpret_cast<volatile int*>(smem_raw + S::OFF_IDX);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int bh = blockIdx.y;
@@ -225,10 +222,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 ks = ks + 1 == KST ? 0 : ks + 1;
             };
 
-            need_g(0);                                         // the softmax warps' prologue gathers
             mbar_wait(bar_q, 0, 1);
-            mma_s();
-            if (n_tiles > 1) mma_s();
+            mma_s();                                           // tile 0 is always a window tile
+            if (n_tiles > 1) {
+                if (n_win < 2) need_g(0);                      // tile 1 is a retained tile: the prologue gathers
+                mma_s();
+            }
             for (int t = 0; t < n_tiles; ++t) {
                 // PV(t): everything but P is normally there long before
                 need_g(t);
@@ -251,27 +250,35 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     } else {
         // =================================== softmax warps ==================================================
         const int i = i0 + tid;                                // this thread's query row
-        // retained entries visible to this row: the list is staged through shared memory 128 entries at a time
+        if (S::ONES) {                                         // 8 KB of bf16 1.0: 64 bytes per thread
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(base + S::OFF_ONES + tid * 64 + u * 16), "r"(0x3F803F80u) : "memory");
+        }
+        // retained entries visible to this row.  The rows of a warp are consecutive and the list is ascending, so
+        // nvis(row) = #{idx <= lim of lane 0} + #{idx in (lim of lane 0, lim of this lane]}: a ballot count plus a
+        // 31-bit map of the entries that fall between the warp's first and last limit.  No block barrier.
         const int lim = min(i, Tlen - 1) - W;                  // entry visible iff idx <= lim
         const int lim_max = i_hi - W;
-        int nvis = 0;
-        for (int e0 = 0; e0 < n_ret; e0 += 128) {
-            const int n_here = min(128, n_ret - e0);
-            softmax_group_sync();
-            if (tid < n_here) s_idx[tid] = id[e0 + tid];
-            softmax_group_sync();
-            if (s_idx[n_here - 1] <= lim) nvis += n_here;
-            else {
-                int lo = 0, hi = n_here;
-                while (lo < hi) { const int mid = (lo + hi) >> 1; if (s_idx[mid] <= lim) lo = mid + 1; else hi = mid; }
-                nvis += lo;
+        const int lim0 = __shfl_sync(0xffffffffu, lim, 0), lim31 = __shfl_sync(0xffffffffu, lim, 31);
+        int nvis = 0, nv_max = 0;                              // nv_max: entries visible to the tile's last row
+        {
+            uint32_t bits = 0;
+            for (int e0 = 0; e0 < n_ret; e0 += 128) {
+                int e[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) e[u] = e0 + u * 32 + lane < n_ret ? id[e0 + u * 32 + lane] : 0x7fffffff;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    nvis += __popc(__ballot_sync(0xffffffffu, e[u] <= lim0));
+                    nv_max += __popc(__ballot_sync(0xffffffffu, e[u] <= lim_max));
+                    const bool in = e[u] > lim0 && e[u] <= lim31;
+                    bits |= __reduce_or_sync(0xffffffffu, in ? 1u << (e[u] - lim0 - 1) : 0u);
+                }
+                if (__shfl_sync(0xffffffffu, e[3], 31) > lim_max) break;   // nothing further is visible to any row
             }
-            if (s_idx[n_here - 1] > lim_max) break;            // uniform: nothing further is visible to any row
+            nvis += __popc(bits & ((1u << (lim - lim0)) - 1u));
         }
-        softmax_group_sync();                                  // every search in the staging buffer is done
-        if (i == i_hi) s_idx[0] = nvis;                        // the tile count follows the last valid row
-        softmax_group_sync();
-        const int nv_max = s_idx[0];
         const int n_tiles = n_win + (nv_max + BN - 1) / BN;
         PROF(2);
 
@@ -304,17 +311,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             cp_async_commit();
         };
         // prologue gathers: the first KST key tiles and VST value tiles (those that are retained tiles)
-        {
+        if (n_win < KST) {
             int rows4[4];
             for (int t = 0; t < KST; ++t) { gather_rows(t, rows4); gather_issue(t, false, rows4); }
             for (int t = 0; t < VST; ++t) { gather_rows(t, rows4); gather_issue(t, true, rows4); }
         }
 
-        if (S::ONES) {                                         // 8 KB of bf16 1.0: 64 bytes per thread
-#pragma unroll
-            for (int u = 0; u < 4; ++u)
-                asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(base + S::OFF_ONES + tid * 64 + u * 16), "r"(0x3F803F80u) : "memory");
-        }
         const float c2 = scale * 1.4426950408889634f;          // logits are handled in the log2 domain: x = s * c2
         const uint32_t lane_base = ((uint32_t)(warp * 32)) << 16;   // this warp's TMEM lanes
         float m_run = -INFINITY, l_run = 0.f;                  // running max (log2 domain) and sum (sum only if !ONES)
