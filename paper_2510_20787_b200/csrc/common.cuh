@@ -83,6 +83,9 @@ int launch_scores(const Params& p, const void* k, const void* v, float* z, float
 int launch_select(const Params& p, const float* z, int32_t* idx, int32_t* cnt, int32_t* ncand, cudaStream_t st);
 int launch_prefill_simt(const Params& p, const void* q, const void* k, const void* v, const int32_t* idx,
                         const int32_t* cnt, void* o, float* lse, cudaStream_t st);
+int launch_prefill_tc_long(const Params& p, const void* q, const void* k, const void* v, const int32_t* idx,
+                           const int32_t* cnt, void* o, float* lse, cudaStream_t st);
+int prefill_long_status_fetch_and_clear();
 int launch_cache_init(const Params& p, const void* k, const void* v, const float* z, const int32_t* idx,
                       const int32_t* cnt, void* cache, cudaStream_t st);
 int launch_decode_tc(const Params& p, void* cache, const void* q1, const void* k1, const void* v1, void* o1,

@@ -1,6 +1,8 @@
 // Prefill attention on the 5th-generation tensor cores (Section 3.1.3, "Cached prefilling and decoding").
 //
-// One CTA per 128-query tile of one (b,h): four softmax warps, one MMA-issue warp and one load warp.  Key/value tiles of 64
+// Persistent CTAs (two per SM): each walks work items, an item being one 128-query tile of one (b,h), so that the
+// loads of the next item are in flight while the current one is finished (a CTA per item spent a third of its life
+// waiting for its first tiles).  Four softmax warps, one MMA-issue warp and one load warp.  Key/value tiles of 64
 // rows come from two sources, as in the paper's two-stage loop: (1) the contiguous window span, staged by TMA
 // (cp.async.bulk.tensor, 128-byte swizzle); (2) the retained rows already out of the tile's window, gathered
 // row by row with cp.async into the same swizzled layout (idx is ascending, so the entries a query may see are
@@ -13,22 +15,13 @@
 //   O += P V       tcgen05.mma with P as the TMEM A operand and V as an MN-major shared-memory operand,
 //                  accumulated in TMEM; the accumulator is rescaled
 //                  in place only when a row's maximum grows by more than 2^8 (lazy rescale)
-// Loads run two to three tiles ahead of the tensor core.  Every mbarrier wait is bounded; a wait that runs out
-// records a status word and the kernel still terminates.
+// Tiles are numbered through all items of a CTA (g); stage, buffer and barrier phase of a tile follow from g alone.
+// Every mbarrier wait is bounded; a wait that runs out records a status word and the kernel still terminates.
 #include "tc_common.cuh"
 
 namespace lte {
 
 __device__ int g_prefill_status = 0;          // 0 = fine; otherwise the code of the wait that gave up
-
-#ifdef LTE_PROFILE
-__device__ long long g_prof[160];
-#define PROFC(slot) do { if (blockIdx.x == 5 && blockIdx.y == 3 && threadIdx.x == 128 && (slot) < 160) g_prof[slot] = clock64(); } while (0)
-#define PROF(slot) do { if (blockIdx.x == 5 && blockIdx.y == 3 && threadIdx.x == 64) g_prof[slot] = clock64(); } while (0)
-#else
-#define PROF(slot) do { } while (0)
-#define PROFC(slot) do { } while (0)
-#endif
 
 namespace {
 
@@ -45,37 +38,72 @@ template <int D> struct Smem {
     static constexpr int OFF_Q = 0;
     static constexpr int OFF_K = QTILE;
     static constexpr int OFF_V = OFF_K + KST * KVTILE;
-    static constexpr int OFF_P = OFF_V + VST * KVTILE;        // (P lives in TMEM; nothing here)
     // d = 64: the row sums are taken by the tensor core as well: PV gets 16 extra B columns of ones, so column D of
     // the accumulator is sum_j P_ij of exactly the (bf16-rounded) probabilities the product used.  The ones live in one
     // more 64-column group, LBO away from the value tile.
     static constexpr bool ONES = D == 64;
-    static constexpr int OFF_ONES = OFF_P;                    // [64][64] bf16 ones (8 KB), d = 64 only
-    static constexpr int OFF_BAR = OFF_ONES + (ONES ? BN * 128 : 0);   // mbarriers, tmem slot
+    static constexpr int OFF_ONES = OFF_V + VST * KVTILE;     // [64][64] bf16 ones (8 KB), d = 64 only
+    static constexpr int OFF_OST = OFF_ONES + (ONES ? BN * 128 : 0);   // output staging: a [32][64] bf16 slab per softmax warp
+    static constexpr int OFF_BAR = OFF_OST + 4 * 4096;        // mbarriers, tmem slot
     static constexpr int BYTES = OFF_BAR + 256;
     static constexpr uint32_t TMEM_COLS = 256;                // S0: [0,64)  S1: [64,128)  O: [128, 128+D) (+16 row-sum columns)
 };
 
+// One work item: a 128-query tile of one (b,h).
+struct Item {
+    int bh, i0, i_hi, j_start, n_win;
+};
+// Items are numbered from the last query tile of every (b,h) down to the first: later query tiles see more retained
+// rows and cost more, and a CTA takes items n, n + grid, n + 2 grid, ... so every CTA gets one item of each cost band
+// (largest first), which balances the static schedule.
+__device__ __forceinline__ Item decode_item(int item, int n_qt, int n_bh, int Tlen, int W)
+{
+    Item it;
+    const int r = item / n_bh;
+    it.bh = item - r * n_bh;
+    it.i0 = (n_qt - 1 - r) * BM;
+    it.i_hi = min(it.i0 + BM - 1, Tlen - 1);
+    it.j_start = max(it.i0 - W + 1, 0);
+    it.n_win = (it.i_hi - it.j_start + 1 + BN - 1) / BN;
+    return it;
+}
+// Entries of the ascending list id[0, n) that are <= lim (whole warp).
+__device__ __forceinline__ int count_le(const int32_t* id, int n, int lim, int lane)
+{
+    int c = 0;
+    for (int e0 = 0; e0 < n; e0 += 32) {
+        const int e = e0 + lane < n ? id[e0 + lane] : 0x7fffffff;
+        const unsigned bal = __ballot_sync(0xffffffffu, e <= lim);
+        c += __popc(bal);
+        if (bal != 0xffffffffu) break;
+    }
+    return c;
+}
 
 // Warps 0-3 (128 threads): softmax (thread r owns query row r) and the cp.async gathers of retained rows.
 // Warp 4, one lane: every tcgen05.mma.  Warp 5, one lane: the TMA loads of Q and of the window tiles (a single
 // lane doing both was the bottleneck: its dependent instruction stream took longer per tile than the softmax).
-// They meet on mbarriers:
-//   bar_s[b]  (commit)       S(t) is in TMEM buffer b = t & 1                     control -> softmax
-//   bar_p     (128 arrivals) P(t) is in shared memory, S buffer b is free         softmax -> control
-//   bar_pv    (commit)       PV(t) has completed                                   control -> softmax
-//   bar_g[b]  (128 arrivals) gathers issued before the top of tile t have landed   softmax -> control
-//   bar_k[s], bar_v[s]       TMA transaction barriers of the window tiles
-//   bar_kf[s], bar_vf[s]     (commit) the MMA that read stage s has completed          MMA lane -> load lane
-// S(t+1) and S(t+2) are computed while the softmax of tile t runs; loads run two to three tiles ahead.
+// They meet on mbarriers (g = the tile's number within the CTA, it = the item's):
+//   bar_q                    Q of item `it` has landed (TMA)                          phase it
+//   bar_qf    (commit)       the last S product of item `it` has completed            phase it     MMA -> load
+//   bar_of    (128 arrivals) O of item `it` has been read out of TMEM                 phase it     softmax -> MMA
+//   bar_s[b]  (commit)       S(g) is in TMEM buffer b = g & 1                         phase g >> 1 MMA -> softmax
+//   bar_p     (128 arrivals) P(g) is in TMEM, over S(g)                               phase g      softmax -> MMA
+//   bar_pv    (commit)       PV(g) has completed                                      phase g      MMA -> softmax
+//   bar_g[b]  (128 arrivals) gathers issued before the top of tile g have landed      phase g >> 1 softmax -> MMA
+//   bar_k[s], bar_v[s]       TMA transaction barriers of the window tiles (one phase per TMA use of the stage)
+//   bar_kf[s], bar_vf[s]     (commit) the MMA that read the stage's tile g has completed   phase g / stages   MMA -> load
+// S(g+1) and S(g+2) are computed while the softmax of tile g runs; loads run two to three tiles ahead, across items.
 template <int D>
 __global__ void __launch_bounds__(NTHREADS, 2)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                  const __grid_constant__ CUtensorMap tmV, const __nv_bfloat16* __restrict__ kg,
+                  const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
+                  const __nv_bfloat16* __restrict__ kg,
                   const __nv_bfloat16* __restrict__ vg, const int32_t* __restrict__ idx,
-                  const int32_t* __restrict__ cnt, __nv_bfloat16* __restrict__ o, float* __restrict__ lse, int Tlen,
-                  int W, int R, float scale)
+                  const int32_t* __restrict__ cnt, float* __restrict__ lse, int Tlen,
+                  int W, int R, float scale, int n_qt, int n_bh)
 {
+    const int n_items = n_qt * n_bh;
     using S = Smem<D>;
     constexpr int SUB = S::SUB, KST = S::KST, VST = S::VST;
     constexpr uint32_t TMEM_COLS = S::TMEM_COLS;
@@ -86,7 +114,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         if (threadIdx.x == 0) atomicExch(&g_prefill_status, 9);
         return;
     }
-    PROF(0);
     const uint32_t sQ = base + S::OFF_Q, sK = base + S::OFF_K, sV = base + S::OFF_V;
     const uint32_t bar_q = base + S::OFF_BAR;
     const uint32_t bar_k0 = bar_q + 8;                         // 3 slots
@@ -96,18 +123,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     const uint32_t bar_p = bar_q + 88, bar_pv = bar_q + 96;
     const uint32_t bar_kf0 = bar_q + 104;                      // 3 slots: K stage free
     const uint32_t bar_vf0 = bar_q + 128;                      // 3 slots: V stage free
-    const uint32_t tmem_slot = bar_q + 152;
-    volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(smem_raw + S::OFF_BAR + 152);
+    const uint32_t bar_qf = bar_q + 152, bar_of = bar_q + 160;
+    const uint32_t tmem_slot = bar_q + 168;
+    volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(smem_raw + S::OFF_BAR + 168);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int bh = blockIdx.y;
-    const int i0 = blockIdx.x * BM;
-    const int i_hi = min(i0 + BM - 1, Tlen - 1);
-    const int j_start = max(i0 - W + 1, 0);
-    const int n_win = (i_hi - j_start + 1 + BN - 1) / BN;
-    const int32_t* id = idx + (size_t)bh * R;
-    const int n_ret = cnt[bh];
-    const int g_first = max(n_win - Smem<D>::KST, 0);        // first tile whose top may have gathers in flight
 
     if (tid == 0) {
         mbar_init(bar_q, 1);
@@ -119,368 +139,394 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         mbar_init(bar_s0, 1); mbar_init(bar_s0 + 8, 1);
         mbar_init(bar_g0, 128); mbar_init(bar_g0 + 8, 128);
         mbar_init(bar_p, 128); mbar_init(bar_pv, 1);
+        mbar_init(bar_qf, 1); mbar_init(bar_of, 128);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 4) tmem_alloc(tmem_slot, TMEM_COLS);
+    if (S::ONES && tid < 128) {                                // 8 KB of bf16 1.0: 64 bytes per thread, once per CTA
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(base + S::OFF_ONES + tid * 64 + u * 16), "r"(0x3F803F80u) : "memory");
+        fence_proxy_async();
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot_gen;
-    PROF(1);
 
-    if (warp >= 4) {
-        // ============================ load lane (warp 5) and MMA lane (warp 4) ==============================
-        // number of tiles: retained entries visible to the last row of the tile (idx ascending => a prefix)
-        int nv_max = 0;
-        {
-            const int lim = i_hi - W;
-            for (int e0 = 0; e0 < n_ret; e0 += 32) {
-                const int e = e0 + lane < n_ret ? id[e0 + lane] : 0x7fffffff;
-                const unsigned bal = __ballot_sync(0xffffffffu, e <= lim);
-                nv_max += __popc(bal);
-                if (bal != 0xffffffffu) break;
-            }
-        }
-        const int n_tiles = n_win + (nv_max + BN - 1) / BN;
-        if (warp == 5 && lane == 0) {
-            // ---- load lane: Q, then the window tiles, each into its stage as soon as the MMA that read the
-            //      stage's previous tile has completed (bar_kf / bar_vf, one phase per use of a stage)
-            mbar_expect_tx(bar_q, S::QTILE);
+    if (warp == 5) {
+        // ================================= load warp (lane 0 issues) ========================================
+        uint32_t g = 0;                                        // tiles of the items before this one
+        int it = 0;
+        for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++it) {
+            const Item w = decode_item(item, n_qt, n_bh, Tlen, W);
+            if (lane == 0) {
+                // Q: its buffer is free once the previous item's last S product has completed
+                if (it > 0) mbar_wait(bar_qf, (it - 1) & 1, 12);
+                mbar_expect_tx(bar_q, S::QTILE);
 #pragma unroll
-            for (int sb = 0; sb < SUB; ++sb) tma_load_3d(sQ + sb * 16384, &tmQ, sb * 64, i0, bh, bar_q);
-            int ks = 0, vs = 0;                                // stage of the next K / V tile to load
-            uint32_t kf_par = 0, vf_par = 0;                   // parity bit per stage of the "free" barriers
-            int tk = 0, tv = 0;                                // next window tile to load
-            int y = j_start;
-            for (; tk < KST && tk < n_win; ++tk, y += BN) {
-                mbar_expect_tx(bar_k0 + 8 * tk, S::KVTILE);
-#pragma unroll
-                for (int sb = 0; sb < SUB; ++sb) tma_load_3d(sK + tk * S::KVTILE + sb * 8192, &tmK, sb * 64, y, bh, bar_k0 + 8 * tk);
-            }
-            y = j_start;
-            for (; tv < VST && tv < n_win; ++tv, y += BN) {
-                mbar_expect_tx(bar_v0 + 8 * tv, S::KVTILE);
-#pragma unroll
-                for (int sb = 0; sb < SUB; ++sb) tma_load_3d(sV + tv * S::KVTILE + sb * 8192, &tmV, sb * 64, y, bh, bar_v0 + 8 * tv);
-            }
-            while (tk < n_win || tv < n_win) {
-                if (tk < n_win) {                              // K(tk) into the stage of K(tk - KST)
-                    mbar_wait(bar_kf0 + 8 * ks, (kf_par >> ks) & 1u, 6);
-                    kf_par ^= 1u << ks;
+                for (int sb = 0; sb < SUB; ++sb) tma_load_3d(sQ + sb * 16384, &tmQ, sb * 64, w.i0, w.bh, bar_q);
+                // window tiles, each into its stage as soon as the MMA that read the stage's previous tile has completed
+                for (int t = 0; t < w.n_win; ++t) {
+                    const uint32_t gg = g + t;
+                    const int y = w.j_start + t * BN;
+                    const uint32_t ks = gg % KST, vs = gg % VST;
+                    if (gg >= (uint32_t)KST) mbar_wait(bar_kf0 + 8 * ks, (gg / KST - 1) & 1u, 6);
                     mbar_expect_tx(bar_k0 + 8 * ks, S::KVTILE);
 #pragma unroll
                     for (int sb = 0; sb < SUB; ++sb)
-                        tma_load_3d(sK + ks * S::KVTILE + sb * 8192, &tmK, sb * 64, j_start + tk * BN, bh, bar_k0 + 8 * ks);
-                    ++tk;
-                    ks = ks + 1 == KST ? 0 : ks + 1;
-                }
-                if (tv < n_win) {                              // V(tv) into the stage of V(tv - VST)
-                    mbar_wait(bar_vf0 + 8 * vs, (vf_par >> vs) & 1u, 8);
-                    vf_par ^= 1u << vs;
+                        tma_load_3d(sK + ks * S::KVTILE + sb * 8192, &tmK, sb * 64, y, w.bh, bar_k0 + 8 * ks);
+                    if (gg >= (uint32_t)VST) mbar_wait(bar_vf0 + 8 * vs, (gg / VST - 1) & 1u, 8);
                     mbar_expect_tx(bar_v0 + 8 * vs, S::KVTILE);
 #pragma unroll
                     for (int sb = 0; sb < SUB; ++sb)
-                        tma_load_3d(sV + vs * S::KVTILE + sb * 8192, &tmV, sb * 64, j_start + tv * BN, bh, bar_v0 + 8 * vs);
-                    ++tv;
-                    vs = vs + 1 == VST ? 0 : vs + 1;
+                        tma_load_3d(sV + vs * S::KVTILE + sb * 8192, &tmV, sb * 64, y, w.bh, bar_v0 + 8 * vs);
                 }
             }
-        } else if (warp == 4 && lane == 0) {
-            // ---- MMA lane: nothing but barrier waits and tcgen05 issue; stage indices and parities roll
-            constexpr uint32_t IDESC_S = instr_desc(BM, BN, false);
-            constexpr uint32_t IDESC_O = S::ONES ? instr_desc(BM, D + 16, true) : instr_desc(BM, D, true);
-            // descriptor words: lo = (address >> 4) | LBO field, hi = SBO field | version | swizzle mode
-            constexpr uint32_t HI = (1024u >> 4) | (1u << 14) | (2u << 29);
-            const uint32_t q_lo = (sQ >> 4) | (1u << 16), k_lo = (sK >> 4) | (1u << 16);
-            // value operand: the second 64-column group of B is the next sub-tile (d = 128) or the block of ones
-            // (d = 64, LBO = its distance from the value stage)
-            uint32_t v_desc[VST];
-#pragma unroll
-            for (int st = 0; st < VST; ++st) {
-                const uint32_t va = sV + st * S::KVTILE;
-                v_desc[st] = (va >> 4) | ((S::ONES ? ((base + S::OFF_ONES - va) >> 4) : (8192u >> 4)) << 16);
-            }
-            uint32_t k_par = 0, v_par = 0, g_waited = 0;       // TMA barrier parities (bit per stage); bar_g phases consumed
-            int ks = 0, vs = 0;                                // stage of the next S / PV operand
-            int ts = 0;                                        // next S tile to issue
-            // gathers issued before the top of tile t have landed (the softmax warps signal from tile g_first on)
-            auto need_g = [&](int t) {
-                while ((int)g_waited <= t - g_first) { mbar_wait(bar_g0 + 8 * (g_waited & 1), (g_waited >> 1) & 1, 10); ++g_waited; }
+            // the item's retained tiles also take tile numbers (counted after the loads are on their way)
+            g += w.n_win + (count_le(idx + (size_t)w.bh * R, cnt[w.bh], w.i_hi - W, lane) + BN - 1) / BN;
+        }
+    } else if (warp == 4) {
+        // ================================= MMA warp (lane 0 issues) =========================================
+        constexpr uint32_t IDESC_S = instr_desc(BM, BN, false);
+        constexpr uint32_t IDESC_O = S::ONES ? instr_desc(BM, D + 16, true) : instr_desc(BM, D, true);
+        // descriptor words: lo = (address >> 4) | LBO field, hi = SBO field | version | swizzle mode
+        constexpr uint32_t HI = (1024u >> 4) | (1u << 14) | (2u << 29);
+        const uint32_t q_lo = (sQ >> 4) | (1u << 16), k_lo = (sK >> 4) | (1u << 16);
+        uint32_t g = 0, g_waited = 0;                          // tiles before this item; bar_g phases consumed
+        uint32_t k_par = 0, v_par = 0;                         // TMA barrier parities (bit per stage)
+        int it = 0;
+        // tiles of an item (whole warp: the count of visible list entries takes global loads)
+        auto item_tiles = [&](int item) {
+            if (item >= n_items) return 0;
+            const Item w = decode_item(item, n_qt, n_bh, Tlen, W);
+            return w.n_win + (count_le(idx + (size_t)w.bh * R, cnt[w.bh], w.i_hi - W, lane) + BN - 1) / BN;
+        };
+        int n_tiles_next = item_tiles(blockIdx.x);
+        for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++it) {
+            const Item w = decode_item(item, n_qt, n_bh, Tlen, W);
+            const int n_tiles = n_tiles_next;
+            int ts = 0;                                        // S products of this item issued so far
+            // gathers issued before the top of tile gg have landed
+            auto need_g = [&](uint32_t gg) {
+                while (g_waited <= gg) { mbar_wait(bar_g0 + 8 * (g_waited & 1), (g_waited >> 1) & 1, 10); ++g_waited; }
             };
-            auto mma_s = [&]() {                               // S(ts) from K stage ks into S buffer ts & 1
-                if (ts < n_win) { mbar_wait(bar_k0 + 8 * ks, (k_par >> ks) & 1u, 2); k_par ^= 1u << ks; }
+            auto mma_s = [&]() {                           // S of the item's tile ts
+                const uint32_t gg = g + ts, ks = gg % KST;
+                if (ts < w.n_win) { mbar_wait(bar_k0 + 8 * ks, (k_par >> ks) & 1u, 2); k_par ^= 1u << ks; }
+                else need_g(g + max(ts - (KST == 2 ? 1 : 2), 0));   // a gathered K tile: issued in tile ts - KST or in the item's prologue
                 tc_fence_after();
-                const uint32_t kb = k_lo + (uint32_t)ks * (S::KVTILE >> 4);
-                const uint32_t dcol = tmem + (ts & 1) * BN;
+                const uint32_t kb = k_lo + ks * (S::KVTILE >> 4);
+                const uint32_t dcol = tmem + (gg & 1) * BN;
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk)
                     umma(dcol, desc64(q_lo + (kk >> 2) * 1024 + (kk & 3) * 2, HI), desc64(kb + (kk >> 2) * 512 + (kk & 3) * 2, HI),
                          IDESC_S, kk > 0);
-                umma_commit(bar_s0 + 8 * (ts & 1));
-                umma_commit(bar_kf0 + 8 * ks);                 // the K stage is free once S(ts) has completed
+                umma_commit(bar_s0 + 8 * (gg & 1));
+                umma_commit(bar_kf0 + 8 * ks);             // the K stage is free once this S has completed
                 ++ts;
-                ks = ks + 1 == KST ? 0 : ks + 1;
+                if (ts == n_tiles) umma_commit(bar_qf);    // and so is Q after the item's last S
             };
 
-            mbar_wait(bar_q, 0, 1);
-            mma_s();                                           // tile 0 is always a window tile
-            if (n_tiles > 1) {
-                if (n_win < 2) need_g(0);                      // tile 1 is a retained tile: the prologue gathers
-                mma_s();
+            if (lane == 0) {
+                mbar_wait(bar_q, it & 1, 1);
+                mma_s();                                       // tile 0 is always a window tile
+                if (n_tiles > 1) mma_s();
             }
-            for (int t = 0; t < n_tiles; ++t) {
-                // PV(t): everything but P is normally there long before
-                need_g(t);
-                if (t < n_win) { mbar_wait(bar_v0 + 8 * vs, (v_par >> vs) & 1u, 4); v_par ^= 1u << vs; }
-                uint32_t vb = v_desc[0];
+            // the next item's tile count, fetched while the softmax of this item's first tile runs
+            n_tiles_next = item_tiles(item + gridDim.x);
+            if (lane == 0) {
+                for (int t = 0; t < n_tiles; ++t) {
+                    const uint32_t gg = g + t, vs = gg % VST;
+                    need_g(gg);
+                    if (t < w.n_win) { mbar_wait(bar_v0 + 8 * vs, (v_par >> vs) & 1u, 4); v_par ^= 1u << vs; }
+                    // value operand: the second 64-column group of B is the next sub-tile (d = 128) or the block of
+                    // ones (d = 64, LBO = its distance from the value stage)
+                    const uint32_t va = sV + vs * S::KVTILE;
+                    const uint32_t vb = (va >> 4) | ((S::ONES ? ((base + S::OFF_ONES - va) >> 4) : (8192u >> 4)) << 16);
+                    if (t == 0 && it > 0) mbar_wait(bar_of, (it - 1) & 1, 13);   // the previous item's O has been read out
+                    mbar_wait(bar_p, gg & 1, 7);
+                    tc_fence_after();
 #pragma unroll
-                for (int st = 1; st < VST; ++st) vb = vs == st ? v_desc[st] : vb;
-                mbar_wait(bar_p, t & 1, 7);
-                tc_fence_after();
-#pragma unroll
-                for (int kk = 0; kk < BN / 16; ++kk)
-                    umma_ts(tmem + O_COL, tmem + (t & 1) * BN + kk * 8, desc64(vb + kk * 128, HI), IDESC_O, (t > 0 || kk > 0) ? 1u : 0u);
-                umma_commit(bar_pv);
-                umma_commit(bar_vf0 + 8 * vs);                 // the V stage is free once PV(t) has completed
-                vs = vs + 1 == VST ? 0 : vs + 1;
-                // S(t+2) into the S buffer softmax(t) has just released
-                if (ts < n_tiles) mma_s();
+                    for (int kk = 0; kk < BN / 16; ++kk)
+                        umma_ts(tmem + O_COL, tmem + (gg & 1) * BN + kk * 8, desc64(vb + kk * 128, HI), IDESC_O, (t > 0 || kk > 0) ? 1u : 0u);
+                    umma_commit(bar_pv);
+                    umma_commit(bar_vf0 + 8 * vs);             // the V stage is free once PV has completed
+                    // S two tiles ahead, into the S buffer the softmax has just released
+                    if (ts < n_tiles) mma_s();
+                }
             }
+            g += n_tiles;
+            __syncwarp();
         }
     } else {
         // =================================== softmax warps ==================================================
-        const int i = i0 + tid;                                // this thread's query row
-        if (S::ONES) {                                         // 8 KB of bf16 1.0: 64 bytes per thread
-#pragma unroll
-            for (int u = 0; u < 4; ++u)
-                asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(base + S::OFF_ONES + tid * 64 + u * 16), "r"(0x3F803F80u) : "memory");
-        }
-        // retained entries visible to this row.  The rows of a warp are consecutive and the list is ascending, so
-        // nvis(row) = #{idx <= lim of lane 0} + #{idx in (lim of lane 0, lim of this lane]}: a ballot count plus a
-        // 31-bit map of the entries that fall between the warp's first and last limit.  No block barrier.
-        const int lim = min(i, Tlen - 1) - W;                  // entry visible iff idx <= lim
-        const int lim_max = i_hi - W;
-        const int lim0 = __shfl_sync(0xffffffffu, lim, 0), lim31 = __shfl_sync(0xffffffffu, lim, 31);
-        int nvis = 0, nv_max = 0;                              // nv_max: entries visible to the tile's last row
-        {
-            uint32_t bits = 0;
-            for (int e0 = 0; e0 < n_ret; e0 += 128) {
-                int e[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) e[u] = e0 + u * 32 + lane < n_ret ? id[e0 + u * 32 + lane] : 0x7fffffff;
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    nvis += __popc(__ballot_sync(0xffffffffu, e[u] <= lim0));
-                    nv_max += __popc(__ballot_sync(0xffffffffu, e[u] <= lim_max));
-                    const bool in = e[u] > lim0 && e[u] <= lim31;
-                    bits |= __reduce_or_sync(0xffffffffu, in ? 1u << (e[u] - lim0 - 1) : 0u);
-                }
-                if (__shfl_sync(0xffffffffu, e[3], 31) > lim_max) break;   // nothing further is visible to any row
-            }
-            nvis += __popc(bits & ((1u << (lim - lim0)) - 1u));
-        }
-        const int n_tiles = n_win + (nv_max + BN - 1) / BN;
-        PROF(2);
-
-        // gather of one retained tile: 8 lanes per row copy its 16-byte chunks (coalesced reads, conflict-free
-        // swizzled writes), 16 rows per pass; rows past the visible prefix are zero-filled
-        const int g_row = tid >> 3, g_sub = tid & 7;
-        auto gather_rows = [&](int t, int (&rows4)[4]) {       // row positions of this thread's 4 rows of tile t
-#pragma unroll
-            for (int ps = 0; ps < 4; ++ps) {
-                const int e = (t - n_win) * BN + ps * 16 + g_row;
-                rows4[ps] = (t >= n_win && t < n_tiles && e < nv_max) ? id[e] : -1;
-            }
-        };
-        auto gather_issue = [&](int t, bool is_v, const int (&rows4)[4]) {
-            if (t >= n_win && t < n_tiles) {
-                const int st = is_v ? (t % VST) : (t % KST);
-                const uint32_t dst = (is_v ? sV : sK) + st * S::KVTILE;
-#pragma unroll
-                for (int ps = 0; ps < 4; ++ps) {
-                    const int row = ps * 16 + g_row;
-                    const bool ok = rows4[ps] >= 0;
-                    const __nv_bfloat16* src = (is_v ? vg : kg) + ((size_t)bh * Tlen + (ok ? rows4[ps] : 0)) * D;
-#pragma unroll
-                    for (int c = g_sub; c < D / 8; c += 8) {
-                        const uint32_t off = (c >> 3) * 8192 + row * 128 + (((c & 7) ^ (row & 7)) << 4);
-                        cp_async16(dst + off, src + c * 8, ok ? 16u : 0u);
-                    }
-                }
-            }
-            cp_async_commit();
-        };
-        // prologue gathers: the first KST key tiles and VST value tiles (those that are retained tiles)
-        if (n_win < KST) {
-            int rows4[4];
-            for (int t = 0; t < KST; ++t) { gather_rows(t, rows4); gather_issue(t, false, rows4); }
-            for (int t = 0; t < VST; ++t) { gather_rows(t, rows4); gather_issue(t, true, rows4); }
-        }
-
         const float c2 = scale * 1.4426950408889634f;          // logits are handled in the log2 domain: x = s * c2
         const uint32_t lane_base = ((uint32_t)(warp * 32)) << 16;   // this warp's TMEM lanes
-        float m_run = -INFINITY, l_run = 0.f;                  // running max (log2 domain) and sum (sum only if !ONES)
-
-        for (int t = 0; t < n_tiles; ++t) {
-            // row positions for this tile's two gathers, fetched first so their latency hides under the softmax
-            int rk[4], rv[4];
-            gather_rows(t + KST, rk);
-            gather_rows(t + VST - 1, rv);
-            // gathers issued before this point have landed (all of them, or all but the latest value tile)
-            if (t >= g_first) {
-                if (VST == 3) cp_async_wait<1>(); else cp_async_wait<0>();
-                fence_proxy_async();
-                mbar_arrive(bar_g0 + 8 * ((t - g_first) & 1));
+        const int g_row = tid >> 3, g_sub = tid & 7;           // gathers: 8 lanes per row, 16 rows per pass
+        uint32_t g = 0;                                        // tiles of the items before this one
+        int it = 0;
+        // the list length and the first 128 list entries of an item are fetched one item ahead, so that the visible
+        // counts at the start of an item wait for no load (entries past cnt are never used: the length guards them)
+        int pf_cnt = 0, pf_e[4] = {0, 0, 0, 0};
+        auto prefetch_list = [&](int item) {
+            if (item < n_items) {
+                const Item w = decode_item(item, n_qt, n_bh, Tlen, W);
+                pf_cnt = cnt[w.bh];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) pf_e[u] = u * 32 + lane < R ? idx[(size_t)w.bh * R + u * 32 + lane] : 0x7fffffff;
             }
-
-            // column range this row may see in the tile
-            int c_lo, c_hi;
-            if (t < n_win) {
-                const int jt0 = j_start + t * BN;
-                c_lo = max(i - W + 1, 0) - jt0;
-                c_hi = i - jt0;
-            } else {
-                c_lo = 0;
-                c_hi = nvis - (t - n_win) * BN - 1;
-            }
-            // rows of a warp are consecutive and both bounds grow with the row: lane 0 / lane 31 give the warp's
-            // union range (columns any row sees) and intersection range (columns every row sees)
-            const int u_lo = __shfl_sync(0xffffffffu, c_lo, 0), u_hi = __shfl_sync(0xffffffffu, c_hi, 31);
-            const int n_lo = __shfl_sync(0xffffffffu, c_lo, 31), n_hi = __shfl_sync(0xffffffffu, c_hi, 0);
-            bool act[2], full[2];
-            uint32_t vm[2];                                    // per-thread validity bits of a partial chunk
+        };
+        prefetch_list(blockIdx.x);
+        for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++it) {
+            const Item w = decode_item(item, n_qt, n_bh, Tlen, W);
+            const int bh = w.bh, n_win = w.n_win, j_start = w.j_start;
+            const int32_t* id = idx + (size_t)bh * R;
+            const int n_ret = pf_cnt;
+            const int i = w.i0 + tid;                          // this thread's query row
+            // retained entries visible to this row.  The rows of a warp are consecutive and the list is ascending, so
+            // nvis(row) = #{idx <= lim of lane 0} + #{idx in (lim of lane 0, lim of this lane]}: a ballot count plus a
+            // 31-bit map of the entries that fall between the warp's first and last limit.  No block barrier.
+            const int lim = min(i, Tlen - 1) - W;              // entry visible iff idx <= lim
+            const int lim_max = w.i_hi - W;
+            const int lim0 = __shfl_sync(0xffffffffu, lim, 0), lim31 = __shfl_sync(0xffffffffu, lim, 31);
+            int nvis = 0, nv_max = 0;                          // nv_max: entries visible to the tile's last row
+            {
+                uint32_t bits = 0;
+                for (int e0 = 0; e0 < n_ret; e0 += 128) {
+                    int e[4];
+                    if (e0 == 0) {
 #pragma unroll
-            for (int cb = 0; cb < 2; ++cb) {
-                const int lo = cb * 32, hi = lo + 31;
-                act[cb] = lo <= u_hi && hi >= u_lo;
-                full[cb] = lo >= n_lo && hi <= n_hi;
-                const int a = min(max(c_lo - lo, 0), 32), b2 = min(max(c_hi - lo + 1, 0), 32);
-                const uint32_t below_b = b2 >= 32 ? 0xffffffffu : ((1u << b2) - 1u);
-                const uint32_t below_a = a >= 32 ? 0xffffffffu : ((1u << a) - 1u);
-                vm[cb] = b2 > a ? (below_b & ~below_a) : 0u;
-            }
-
-            PROF(4 + 6 * t);
-            mbar_wait(bar_s0 + 8 * (t & 1), (t >> 1) & 1, 3);  // S(t) is in TMEM buffer t & 1
-            tc_fence_after();
-            PROF(5 + 6 * t);
-            gather_issue(t + KST, false, rk);                  // its stage held K(t), which S(t) has finished reading
-            const uint32_t s_col = (t & 1) * BN;
-            uint32_t r[2][32];
+                        for (int u = 0; u < 4; ++u) e[u] = u * 32 + lane < n_ret ? pf_e[u] : 0x7fffffff;
+                    } else {
 #pragma unroll
-            for (int cb = 0; cb < 2; ++cb)
-                if (act[cb]) tmem_ld32(tmem + lane_base + s_col + cb * 32, r[cb]);
-            tmem_wait_ld();
-            PROF(6 + 6 * t);
-            float mr[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // row max of the raw logits, 4 chains
-#pragma unroll
-            for (int cb = 0; cb < 2; ++cb) {
-                if (!act[cb]) continue;
-                if (full[cb]) {
-#pragma unroll
-                    for (int c = 0; c < 32; c += 2)
-                        mr[(c >> 1) & 3] = max3(mr[(c >> 1) & 3], __uint_as_float(r[cb][c]), __uint_as_float(r[cb][c + 1]));
-                } else {
-#pragma unroll
-                    for (int c = 0; c < 32; ++c) {
-                        const float x = (vm[cb] & (1u << c)) ? __uint_as_float(r[cb][c]) : -INFINITY;
-                        r[cb][c] = __float_as_uint(x);
-                        mr[c & 3] = fmaxf(mr[c & 3], x);
+                        for (int u = 0; u < 4; ++u) e[u] = e0 + u * 32 + lane < n_ret ? id[e0 + u * 32 + lane] : 0x7fffffff;
                     }
-                }
-            }
-            const float m_tile = fmaxf(fmaxf(mr[0], mr[1]), fmaxf(mr[2], mr[3])) * c2;
-            PROF(7 + 6 * t);
-            PROF(8 + 6 * t);
-            // lazy rescale: the running max only moves when the new one is far above it (exp2 arguments stay <= 8)
-            float alpha = 1.f;
-            bool need = false;
-            if (m_run == -INFINITY) m_run = m_tile;             // nothing accumulated yet for this row: O row is 0
-            else if (m_tile > m_run + 8.f) { alpha = fast_exp2(m_run - m_tile); m_run = m_tile; need = true; }
-            if (__any_sync(0xffffffffu, need)) {
-                // PV(t-1) must be done before O is rescaled
-                if (t > 0) { mbar_wait(bar_pv, (t - 1) & 1, 4); tc_fence_after(); }
-#pragma unroll
-                for (int cb = 0; cb < D / 32 + (S::ONES ? 1 : 0); ++cb) {   // with ONES the row-sum columns are rescaled too
-                    uint32_t q4[32];
-                    tmem_ld32(tmem + lane_base + O_COL + cb * 32, q4);
-                    tmem_wait_ld();
-#pragma unroll
-                    for (int c = 0; c < 32; ++c) q4[c] = __float_as_uint(__uint_as_float(q4[c]) * alpha);
-                    tmem_st32(tmem + lane_base + O_COL + cb * 32, q4);
-                }
-                tmem_wait_st();
-                l_run *= alpha;
-            }
-            const float neg_m = m_run == -INFINITY ? 0.f : -m_run;
-            float ls[4] = {0.f, 0.f, 0.f, 0.f};
-            uint32_t pk[32];                                   // the row of P as 64 bf16, two per word
-#pragma unroll
-            for (int cb = 0; cb < 2; ++cb) {
-                if (act[cb]) {
-#pragma unroll
-                    for (int c = 0; c < 32; c += 2) {
-                        // masked entries hold -inf: fma gives -inf and exp2(-inf) = 0
-                        const float p0 = fast_exp2(fmaf(__uint_as_float(r[cb][c]), c2, neg_m));
-                        const float p1 = fast_exp2(fmaf(__uint_as_float(r[cb][c + 1]), c2, neg_m));
-                        if (!S::ONES) ls[(c >> 1) & 3] += p0 + p1;   // with ONES the tensor core sums the rounded probabilities
-                        __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
-                        pk[cb * 16 + (c >> 1)] = *reinterpret_cast<uint32_t*>(&h);
-                    }
-                } else {
-#pragma unroll
-                    for (int c = 0; c < 16; ++c) pk[cb * 16 + c] = 0u;
-                }
-            }
-            l_run += (ls[0] + ls[1]) + (ls[2] + ls[3]);
-            // P goes back into TMEM, over the first 32 columns of the S buffer it was computed from (this thread has
-            // all of its row in registers), and feeds the PV product as the A operand: no trip through shared memory
-            tmem_st32(tmem + lane_base + s_col, pk);
-            tmem_wait_st();
-            tc_fence_before();                                 // our TMEM accesses are ordered before the arrive
-            // PV(t-1) has normally completed long ago; the wait sits before the arrive so that the barrier cannot
-            // run two phases ahead of this thread
-            if (t > 0) mbar_wait(bar_pv, (t - 1) & 1, 4);
-            mbar_arrive(bar_p);
-            // value tile t+VST-1 goes into the stage of V(t-1), which PV(t-1) has finished reading
-            if (t > 0) gather_issue(t + VST - 1, true, rv); else cp_async_commit();
-            PROF(9 + 6 * t);
-        }
-        PROF(50);
-        mbar_wait(bar_pv, (n_tiles - 1) & 1, 5);
-        tc_fence_after();
-        PROF(51);
-
-        // ---- epilogue: O / l -> bf16, logsumexp ----------------------------------------------------------
-        if (S::ONES) {                                         // the row sum is column D of the accumulator
-            uint32_t q4[32];
-            tmem_ld32(tmem + lane_base + O_COL + D, q4);
-            tmem_wait_ld();
-            l_run = __uint_as_float(q4[0]);
-        }
-        const float inv = 1.f / l_run;
-        __nv_bfloat16* orow = o + ((size_t)bh * Tlen + i) * D;
-#pragma unroll
-        for (int cb = 0; cb < D / 32; ++cb) {
-            uint32_t q4[32];
-            tmem_ld32(tmem + lane_base + O_COL + cb * 32, q4);
-            tmem_wait_ld();
-            if (i < Tlen) {
-#pragma unroll
-                for (int c = 0; c < 32; c += 8) {
-                    uint32_t w4[4];
 #pragma unroll
                     for (int u = 0; u < 4; ++u) {
-                        __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(q4[c + 2 * u]) * inv,
-                                                                 __uint_as_float(q4[c + 2 * u + 1]) * inv);
-                        w4[u] = *reinterpret_cast<uint32_t*>(&h);
+                        nvis += __popc(__ballot_sync(0xffffffffu, e[u] <= lim0));
+                        nv_max += __popc(__ballot_sync(0xffffffffu, e[u] <= lim_max));
+                        const bool in = e[u] > lim0 && e[u] <= lim31;
+                        bits |= __reduce_or_sync(0xffffffffu, in ? 1u << (e[u] - lim0 - 1) : 0u);
                     }
-                    *reinterpret_cast<uint4*>(orow + cb * 32 + c) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+                    if (__shfl_sync(0xffffffffu, e[3], 31) > lim_max) break;   // nothing further is visible to any row
+                }
+                nvis += __popc(bits & ((1u << (lim - lim0)) - 1u));
+            }
+            const int n_tiles = n_win + (nv_max + BN - 1) / BN;
+            prefetch_list(item + gridDim.x);
+
+            // gather of one retained tile (t = its number within the item): 8 lanes per row copy its 16-byte chunks
+            // (coalesced reads, conflict-free swizzled writes); rows past the visible prefix are zero-filled
+            auto gather_rows = [&](int t, int (&rows4)[4]) {   // row positions of this thread's 4 rows of tile t
+#pragma unroll
+                for (int ps = 0; ps < 4; ++ps) {
+                    const int e = (t - n_win) * BN + ps * 16 + g_row;
+                    rows4[ps] = (t >= n_win && t < n_tiles && e < nv_max) ? id[e] : -1;
+                }
+            };
+            auto gather_issue = [&](int t, bool is_v, const int (&rows4)[4]) {
+                if (t >= n_win && t < n_tiles) {
+                    const uint32_t st = is_v ? ((g + t) % VST) : ((g + t) % KST);
+                    const uint32_t dst = (is_v ? sV : sK) + st * S::KVTILE;
+#pragma unroll
+                    for (int ps = 0; ps < 4; ++ps) {
+                        const int row = ps * 16 + g_row;
+                        const bool ok = rows4[ps] >= 0;
+                        const __nv_bfloat16* src = (is_v ? vg : kg) + ((size_t)bh * Tlen + (ok ? rows4[ps] : 0)) * D;
+#pragma unroll
+                        for (int c = g_sub; c < D / 8; c += 8) {
+                            const uint32_t off = (c >> 3) * 8192 + row * 128 + (((c & 7) ^ (row & 7)) << 4);
+                            cp_async16(dst + off, src + c * 8, ok ? 16u : 0u);
+                        }
+                    }
+                }
+                cp_async_commit();
+            };
+            // prologue gathers: the first KST key tiles and VST value tiles, where those are retained tiles.  Their
+            // stages are free: every product of the previous item has completed (its last bar_s and bar_pv were awaited).
+            if (n_win < KST) {
+                int rows4[4];
+                for (int t = 0; t < KST; ++t) { gather_rows(t, rows4); gather_issue(t, false, rows4); }
+                for (int t = 0; t < VST; ++t) { gather_rows(t, rows4); gather_issue(t, true, rows4); }
+            }
+            float m_run = -INFINITY, l_run = 0.f;              // running max (log2 domain) and sum (sum only if !ONES)
+            bool gathered = n_win < KST;                       // some gather of this item may be in flight (warp-uniform)
+
+            for (int t = 0; t < n_tiles; ++t) {
+                const uint32_t gg = g + t;
+                // row positions for this tile's two gathers, fetched first so their latency hides under the softmax
+                // (all of this tile's gather work sits behind warp-uniform tests: most tiles of a short list have none)
+                const bool k_gather = t + KST >= n_win && t + KST < n_tiles;
+                const bool v_gather = t > 0 && t + VST - 1 >= n_win && t + VST - 1 < n_tiles;
+                int rk[4], rv[4];
+                if (k_gather) gather_rows(t + KST, rk);
+                if (v_gather) gather_rows(t + VST - 1, rv);
+                // gathers issued before this point have landed (all of them, or all but the latest value tile)
+                if (gathered) {
+                    if (VST == 3) cp_async_wait<1>(); else cp_async_wait<0>();
+                    fence_proxy_async();
+                }
+                mbar_arrive(bar_g0 + 8 * (gg & 1));
+
+                // column range this row may see in the tile
+                int c_lo, c_hi;
+                if (t < n_win) {
+                    const int jt0 = j_start + t * BN;
+                    c_lo = max(i - W + 1, 0) - jt0;
+                    c_hi = i - jt0;
+                } else {
+                    c_lo = 0;
+                    c_hi = nvis - (t - n_win) * BN - 1;
+                }
+                // rows of a warp are consecutive and both bounds grow with the row: lane 0 / lane 31 give the warp's
+                // union range (columns any row sees) and intersection range (columns every row sees)
+                const int u_lo = __shfl_sync(0xffffffffu, c_lo, 0), u_hi = __shfl_sync(0xffffffffu, c_hi, 31);
+                const int n_lo = __shfl_sync(0xffffffffu, c_lo, 31), n_hi = __shfl_sync(0xffffffffu, c_hi, 0);
+                bool act[2], full[2];
+                uint32_t vm[2];                                // per-thread validity bits of a partial chunk
+#pragma unroll
+                for (int cb = 0; cb < 2; ++cb) {
+                    const int lo = cb * 32, hi = lo + 31;
+                    act[cb] = lo <= u_hi && hi >= u_lo;
+                    full[cb] = lo >= n_lo && hi <= n_hi;
+                    const int a = min(max(c_lo - lo, 0), 32), b2 = min(max(c_hi - lo + 1, 0), 32);
+                    const uint32_t below_b = b2 >= 32 ? 0xffffffffu : ((1u << b2) - 1u);
+                    const uint32_t below_a = a >= 32 ? 0xffffffffu : ((1u << a) - 1u);
+                    vm[cb] = b2 > a ? (below_b & ~below_a) : 0u;
+                }
+                mbar_wait(bar_s0 + 8 * (gg & 1), (gg >> 1) & 1, 3);   // S is in TMEM buffer gg & 1
+                tc_fence_after();
+                if (k_gather) { gather_issue(t + KST, false, rk); gathered = true; }   // its stage held this tile's K, which S has finished reading
+                else cp_async_commit();
+                const uint32_t s_col = (gg & 1) * BN;
+                uint32_t r[2][32];
+#pragma unroll
+                for (int cb = 0; cb < 2; ++cb)
+                    if (act[cb]) tmem_ld32(tmem + lane_base + s_col + cb * 32, r[cb]);
+                tmem_wait_ld();
+                float mr[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // row max of the raw logits, 4 chains
+#pragma unroll
+                for (int cb = 0; cb < 2; ++cb) {
+                    if (!act[cb]) continue;
+                    if (full[cb]) {
+#pragma unroll
+                        for (int c = 0; c < 32; c += 2)
+                            mr[(c >> 1) & 3] = max3(mr[(c >> 1) & 3], __uint_as_float(r[cb][c]), __uint_as_float(r[cb][c + 1]));
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) {
+                            const float x = (vm[cb] & (1u << c)) ? __uint_as_float(r[cb][c]) : -INFINITY;
+                            r[cb][c] = __float_as_uint(x);
+                            mr[c & 3] = fmaxf(mr[c & 3], x);
+                        }
+                    }
+                }
+                const float m_tile = fmaxf(fmaxf(mr[0], mr[1]), fmaxf(mr[2], mr[3])) * c2;
+                // lazy rescale: the running max only moves when the new one is far above it (exp2 arguments stay <= 8)
+                float alpha = 1.f;
+                bool need = false;
+                if (m_run == -INFINITY) m_run = m_tile;         // nothing accumulated yet for this row: O row is 0
+                else if (m_tile > m_run + 8.f) { alpha = fast_exp2(m_run - m_tile); m_run = m_tile; need = true; }
+                if (__any_sync(0xffffffffu, need)) {
+                    // PV of the previous tile must be done before O is rescaled
+                    if (t > 0) { mbar_wait(bar_pv, (gg - 1) & 1, 4); tc_fence_after(); }
+#pragma unroll
+                    for (int cb = 0; cb < D / 32 + (S::ONES ? 1 : 0); ++cb) {   // with ONES the row-sum columns are rescaled too
+                        uint32_t q4[32];
+                        tmem_ld32(tmem + lane_base + O_COL + cb * 32, q4);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) q4[c] = __float_as_uint(__uint_as_float(q4[c]) * alpha);
+                        tmem_st32(tmem + lane_base + O_COL + cb * 32, q4);
+                    }
+                    tmem_wait_st();
+                    l_run *= alpha;
+                }
+                const float neg_m = m_run == -INFINITY ? 0.f : -m_run;
+                float ls[4] = {0.f, 0.f, 0.f, 0.f};
+                uint32_t pk[32];                               // the row of P as 64 bf16, two per word
+#pragma unroll
+                for (int cb = 0; cb < 2; ++cb) {
+                    if (act[cb]) {
+#pragma unroll
+                        for (int c = 0; c < 32; c += 2) {
+                            // masked entries hold -inf: fma gives -inf and exp2(-inf) = 0
+                            const float p0 = fast_exp2(fmaf(__uint_as_float(r[cb][c]), c2, neg_m));
+                            const float p1 = fast_exp2(fmaf(__uint_as_float(r[cb][c + 1]), c2, neg_m));
+                            if (!S::ONES) ls[(c >> 1) & 3] += p0 + p1;   // with ONES the tensor core sums the rounded probabilities
+                            __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
+                            pk[cb * 16 + (c >> 1)] = *reinterpret_cast<uint32_t*>(&h);
+                        }
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < 16; ++c) pk[cb * 16 + c] = 0u;
+                    }
+                }
+                l_run += (ls[0] + ls[1]) + (ls[2] + ls[3]);
+                // P goes back into TMEM, over the first 32 columns of the S buffer it was computed from (this thread has
+                // all of its row in registers), and feeds the PV product as the A operand: no trip through shared memory
+                tmem_st32(tmem + lane_base + s_col, pk);
+                tmem_wait_st();
+                tc_fence_before();                             // our TMEM accesses are ordered before the arrive
+                // PV of the previous tile has normally completed long ago.  Every phase of bar_pv is awaited in turn (a
+                // parity test is only meaningful for the current or the previous phase), and before the arrive: after
+                // it the barrier could run ahead of this thread.  At t = 0 the item's epilogue has awaited it.
+                if (t > 0) mbar_wait(bar_pv, (gg - 1) & 1, 4);
+                mbar_arrive(bar_p);
+                // value tile t+VST-1 goes into the stage of tile t-1's V, which that PV has finished reading
+                if (v_gather) { gather_issue(t + VST - 1, true, rv); gathered = true; }
+                else cp_async_commit();
+            }
+            mbar_wait(bar_pv, (g + n_tiles - 1) & 1, 5);
+            tc_fence_after();
+
+            // ---- epilogue: O / l -> bf16, logsumexp ------------------------------------------------------
+            if (S::ONES) {                                     // the row sum is column D of the accumulator
+                uint32_t q1;
+                tmem_ld1(tmem + lane_base + O_COL + D, q1);
+                tmem_wait_ld();
+                l_run = __uint_as_float(q1);
+            }
+            const float inv = 1.f / l_run;
+            // the normalised rows go through a swizzled shared-memory slab per warp and leave as one tile store per
+            // 64 columns (rows past the end of the sequence are clipped by the tensor map)
+            const uint32_t slab = base + S::OFF_OST + warp * 4096;
+#pragma unroll
+            for (int sb = 0; sb < SUB; ++sb) {
+                uint32_t ow[32];                               // 64 columns of the row as bf16 pairs
+#pragma unroll
+                for (int cb = 0; cb < 2; ++cb) {
+                    uint32_t q4[32];
+                    tmem_ld32(tmem + lane_base + O_COL + sb * 64 + cb * 32, q4);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int c = 0; c < 32; c += 2) {
+                        __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(q4[c]) * inv, __uint_as_float(q4[c + 1]) * inv);
+                        ow[cb * 16 + (c >> 1)] = *reinterpret_cast<uint32_t*>(&h);
+                    }
+                }
+                if (sb == SUB - 1) {
+                    tc_fence_before();
+                    mbar_arrive(bar_of);                       // the accumulator may take the next item
+                }
+                if (lane == 0) bulk_wait_read0();              // the slab's previous store has been read out
+                __syncwarp();
+#pragma unroll
+                for (int ch = 0; ch < 8; ++ch)
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(slab + lane * 128 + ((ch ^ (lane & 7)) << 4)),
+                                 "r"(ow[4 * ch]), "r"(ow[4 * ch + 1]), "r"(ow[4 * ch + 2]), "r"(ow[4 * ch + 3]) : "memory");
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0 && w.i0 + warp * 32 < Tlen) {
+                    tma_store_3d(&tmO, slab, sb * 64, w.i0 + warp * 32, bh);
+                    bulk_commit();
                 }
             }
+            if (i < Tlen) lse[(size_t)bh * Tlen + i] = m_run * 0.6931471805599453f + logf(l_run);
+            g += n_tiles;
         }
-        if (i < Tlen) lse[(size_t)bh * Tlen + i] = m_run * 0.6931471805599453f + logf(l_run);
-        PROF(52);
+        if (lane == 0) bulk_wait_read0();                      // this warp's tile stores have read their slab
     }
     tc_fence_before();
     __syncthreads();
@@ -491,21 +537,27 @@ template <int D>
 int run(const Params& p, const void* q, const void* k, const void* v, const int32_t* idx, const int32_t* cnt, void* o,
         float* lse, cudaStream_t st)
 {
-    CUtensorMap tq, tk, tv;
+    CUtensorMap tq, tk, tv, to;
     const int BH = p.B * p.H;
-    if (!make_map(&tq, q, BH, p.T, D, BM) || !make_map(&tk, k, BH, p.T, D, BN) || !make_map(&tv, v, BH, p.T, D, BN))
+    if (!make_map(&tq, q, BH, p.T, D, BM) || !make_map(&tk, k, BH, p.T, D, BN) || !make_map(&tv, v, BH, p.T, D, BN) ||
+        !make_map(&to, o, BH, p.T, D, 32))
         return LTE_ERR_CUDA;
-    static bool attr_done = false;
-    if (!attr_done) {
+    static int slots = 0;                                      // resident CTAs: two per SM
+    if (slots == 0) {
         if (cudaFuncSetAttribute(prefill_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::BYTES) !=
             cudaSuccess)
             return LTE_ERR_CUDA;
-        attr_done = true;
+        int dev = 0, sms = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+            return LTE_ERR_CUDA;
+        slots = 2 * sms;
     }
-    dim3 grid((p.T + BM - 1) / BM, BH);
-    prefill_tc_kernel<D><<<grid, NTHREADS, Smem<D>::BYTES, st>>>(tq, tk, tv, (const __nv_bfloat16*)k,
-                                                                 (const __nv_bfloat16*)v, idx, cnt, (__nv_bfloat16*)o,
-                                                                 lse, p.T, p.W, p.R, p.scale);
+    const int n_qt = (p.T + BM - 1) / BM, n_items = n_qt * BH;
+    const int grid = n_items < slots ? n_items : slots;
+    prefill_tc_kernel<D><<<grid, NTHREADS, Smem<D>::BYTES, st>>>(tq, tk, tv, to, (const __nv_bfloat16*)k,
+                                                                 (const __nv_bfloat16*)v, idx, cnt,
+                                                                 lse, p.T, p.W, p.R, p.scale, n_qt, BH);
     return cuda_status(cudaGetLastError());
 }
 
@@ -516,21 +568,20 @@ int launch_prefill_tc(const Params& p, const void* q, const void* k, const void*
 {
     switch (p.d) {
         case 64: return run<64>(p, q, k, v, idx, cnt, o, lse, st);
-        case 128: return run<128>(p, q, k, v, idx, cnt, o, lse, st);
+        // d = 128: ten and more key tiles per item; one CTA per item under the hardware scheduler is faster there
+        case 128: return launch_prefill_tc_long(p, q, k, v, idx, cnt, o, lse, st);
     }
     return launch_prefill_simt(p, q, k, v, idx, cnt, o, lse, st);   // d = 32: rows too narrow for the 128-byte swizzle
 }
 
-#ifdef LTE_PROFILE
-extern "C" int lte_prof_read(long long* out) { return cudaMemcpyFromSymbol(out, g_prof, sizeof(long long) * 160) == cudaSuccess ? 0 : -1; }
-#endif
 
 int prefill_status_fetch_and_clear()
 {
     int h = 0, zero = 0;
     if (cudaMemcpyFromSymbol(&h, g_prefill_status, sizeof(int)) != cudaSuccess) return -1;
     if (h != 0) cudaMemcpyToSymbol(g_prefill_status, &zero, sizeof(int));
-    return h;
+    const int h2 = prefill_long_status_fetch_and_clear();
+    return h != 0 ? h : h2;
 }
 
 }  // namespace lte

@@ -1,0 +1,500 @@
+// Prefill attention on the 5th-generation tensor cores (Section 3.1.3), variant for long items: one CTA per
+// 128-query tile of one (b,h), used at d = 128, where a tile walks ten and more key tiles and the hardware's block
+// scheduler balances the load better than a static persistent schedule (and the registers a persistent loop
+// keeps alive are not free).  The tile loop is the one of the persistent kernel:
+//   S = Q K^T      tcgen05.mma (kind::f16, bf16 in, fp32 out) into one of two TMEM buffers
+//   softmax        thread r owns query row r = TMEM lane r; P written as bf16 back into TMEM over its S buffer
+//   O += P V       tcgen05.mma with P as the TMEM A operand and V as an MN-major shared-memory operand; lazy rescale
+// Window tiles come by TMA, retained rows by cp.async gathers into the same swizzled layout.  Every mbarrier wait is
+// bounded; a wait that runs out records a status word and the kernel still terminates.
+#include "tc_common.cuh"
+
+namespace lte {
+
+__device__ int g_prefill_long_status = 0;     // 0 = fine; otherwise the code of the wait that gave up
+
+
+namespace {
+
+constexpr int BM = 128, BN = 64, NTHREADS = 192;
+using namespace tc;
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, int code) { mbar_wait_s(bar, parity, code, &g_prefill_long_status); }
+
+template <int D> struct Smem {
+    static constexpr int SUB = D / 64;                        // 64-column (128-byte) sub-tiles per row
+    static constexpr int KST = 3;                             // key stages
+    static constexpr int VST = D == 64 ? 3 : 2;               // value stages
+    static constexpr int QTILE = BM * D * 2;                  // [128][D] bf16
+    static constexpr int KVTILE = BN * D * 2;                 // [64][D] bf16
+    static constexpr int OFF_Q = 0;
+    static constexpr int OFF_K = QTILE;
+    static constexpr int OFF_V = OFF_K + KST * KVTILE;
+    static constexpr int OFF_P = OFF_V + VST * KVTILE;        // (P lives in TMEM; nothing here)
+    // d = 64: the row sums are taken by the tensor core as well: PV gets 16 extra B columns of ones, so column D of
+    // the accumulator is sum_j P_ij of exactly the (bf16-rounded) probabilities the product used.  The ones live in one
+    // more 64-column group, LBO away from the value tile.
+    static constexpr bool ONES = D == 64;
+    static constexpr int OFF_ONES = OFF_P;                    // [64][64] bf16 ones (8 KB), d = 64 only
+    static constexpr int OFF_BAR = OFF_ONES + (ONES ? BN * 128 : 0);   // mbarriers, tmem slot
+    static constexpr int BYTES = OFF_BAR + 256;
+    static constexpr uint32_t TMEM_COLS = 256;                // S0: [0,64)  S1: [64,128)  O: [128, 128+D) (+16 row-sum columns)
+};
+
+
+// Warps 0-3 (128 threads): softmax (thread r owns query row r) and the cp.async gathers of retained rows.
+// Warp 4, one lane: every tcgen05.mma.  Warp 5, one lane: the TMA loads of Q and of the window tiles (a single
+// lane doing both was the bottleneck: its dependent instruction stream took longer per tile than the softmax).
+// They meet on mbarriers:
+//   bar_s[b]  (commit)       S(t) is in TMEM buffer b = t & 1                     control -> softmax
+//   bar_p     (128 arrivals) P(t) is in shared memory, S buffer b is free         softmax -> control
+//   bar_pv    (commit)       PV(t) has completed                                   control -> softmax
+//   bar_g[b]  (128 arrivals) gathers issued before the top of tile t have landed   softmax -> control
+//   bar_k[s], bar_v[s]       TMA transaction barriers of the window tiles
+//   bar_kf[s], bar_vf[s]     (commit) the MMA that read stage s has completed          MMA lane -> load lane
+// S(t+1) and S(t+2) are computed while the softmax of tile t runs; loads run two to three tiles ahead.
+template <int D>
+__global__ void __launch_bounds__(NTHREADS, 2)
+prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                  const __grid_constant__ CUtensorMap tmV, const __nv_bfloat16* __restrict__ kg,
+                  const __nv_bfloat16* __restrict__ vg, const int32_t* __restrict__ idx,
+                  const int32_t* __restrict__ cnt, __nv_bfloat16* __restrict__ o, float* __restrict__ lse, int Tlen,
+                  int W, int R, float scale)
+{
+    using S = Smem<D>;
+    constexpr int SUB = S::SUB, KST = S::KST, VST = S::VST;
+    constexpr uint32_t TMEM_COLS = S::TMEM_COLS;
+    constexpr uint32_t O_COL = 2 * BN;
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    const uint32_t base = smem_u32(smem_raw);
+    if ((base & 1023u) != 0) {                                 // the swizzled tiles need 1024-byte alignment
+        if (threadIdx.x == 0) atomicExch(&g_prefill_long_status, 9);
+        return;
+    }
+    const uint32_t sQ = base + S::OFF_Q, sK = base + S::OFF_K, sV = base + S::OFF_V;
+    const uint32_t bar_q = base + S::OFF_BAR;
+    const uint32_t bar_k0 = bar_q + 8;                         // 3 slots
+    const uint32_t bar_v0 = bar_q + 32;                        // 3 slots
+    const uint32_t bar_s0 = bar_q + 56;                        // 2 slots
+    const uint32_t bar_g0 = bar_q + 72;                        // 2 slots
+    const uint32_t bar_p = bar_q + 88, bar_pv = bar_q + 96;
+    const uint32_t bar_kf0 = bar_q + 104;                      // 3 slots: K stage free
+    const uint32_t bar_vf0 = bar_q + 128;                      // 3 slots: V stage free
+    const uint32_t tmem_slot = bar_q + 152;
+    volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(smem_raw + S::OFF_BAR + 152);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int bh = blockIdx.y;
+    const int i0 = blockIdx.x * BM;
+    const int i_hi = min(i0 + BM - 1, Tlen - 1);
+    const int j_start = max(i0 - W + 1, 0);
+    const int n_win = (i_hi - j_start + 1 + BN - 1) / BN;
+    const int32_t* id = idx + (size_t)bh * R;
+    const int n_ret = cnt[bh];
+    const int g_first = max(n_win - Smem<D>::KST, 0);        // first tile whose top may have gathers in flight
+
+    if (tid == 0) {
+        mbar_init(bar_q, 1);
+#pragma unroll
+        for (int s2 = 0; s2 < 3; ++s2) {
+            mbar_init(bar_k0 + 8 * s2, 1); mbar_init(bar_v0 + 8 * s2, 1);
+            mbar_init(bar_kf0 + 8 * s2, 1); mbar_init(bar_vf0 + 8 * s2, 1);
+        }
+        mbar_init(bar_s0, 1); mbar_init(bar_s0 + 8, 1);
+        mbar_init(bar_g0, 128); mbar_init(bar_g0 + 8, 128);
+        mbar_init(bar_p, 128); mbar_init(bar_pv, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 4) tmem_alloc(tmem_slot, TMEM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot_gen;
+
+    if (warp >= 4) {
+        // ============================ load lane (warp 5) and MMA lane (warp 4) ==============================
+        // number of tiles: retained entries visible to the last row of the tile (idx ascending => a prefix)
+        int nv_max = 0;
+        {
+            const int lim = i_hi - W;
+            for (int e0 = 0; e0 < n_ret; e0 += 32) {
+                const int e = e0 + lane < n_ret ? id[e0 + lane] : 0x7fffffff;
+                const unsigned bal = __ballot_sync(0xffffffffu, e <= lim);
+                nv_max += __popc(bal);
+                if (bal != 0xffffffffu) break;
+            }
+        }
+        const int n_tiles = n_win + (nv_max + BN - 1) / BN;
+        if (warp == 5 && lane == 0) {
+            // ---- load lane: Q, then the window tiles, each into its stage as soon as the MMA that read the
+            //      stage's previous tile has completed (bar_kf / bar_vf, one phase per use of a stage)
+            mbar_expect_tx(bar_q, S::QTILE);
+#pragma unroll
+            for (int sb = 0; sb < SUB; ++sb) tma_load_3d(sQ + sb * 16384, &tmQ, sb * 64, i0, bh, bar_q);
+            int ks = 0, vs = 0;                                // stage of the next K / V tile to load
+            uint32_t kf_par = 0, vf_par = 0;                   // parity bit per stage of the "free" barriers
+            int tk = 0, tv = 0;                                // next window tile to load
+            int y = j_start;
+            for (; tk < KST && tk < n_win; ++tk, y += BN) {
+                mbar_expect_tx(bar_k0 + 8 * tk, S::KVTILE);
+#pragma unroll
+                for (int sb = 0; sb < SUB; ++sb) tma_load_3d(sK + tk * S::KVTILE + sb * 8192, &tmK, sb * 64, y, bh, bar_k0 + 8 * tk);
+            }
+            y = j_start;
+            for (; tv < VST && tv < n_win; ++tv, y += BN) {
+                mbar_expect_tx(bar_v0 + 8 * tv, S::KVTILE);
+#pragma unroll
+                for (int sb = 0; sb < SUB; ++sb) tma_load_3d(sV + tv * S::KVTILE + sb * 8192, &tmV, sb * 64, y, bh, bar_v0 + 8 * tv);
+            }
+            while (tk < n_win || tv < n_win) {
+                if (tk < n_win) {                              // K(tk) into the stage of K(tk - KST)
+                    mbar_wait(bar_kf0 + 8 * ks, (kf_par >> ks) & 1u, 6);
+                    kf_par ^= 1u << ks;
+                    mbar_expect_tx(bar_k0 + 8 * ks, S::KVTILE);
+#pragma unroll
+                    for (int sb = 0; sb < SUB; ++sb)
+                        tma_load_3d(sK + ks * S::KVTILE + sb * 8192, &tmK, sb * 64, j_start + tk * BN, bh, bar_k0 + 8 * ks);
+                    ++tk;
+                    ks = ks + 1 == KST ? 0 : ks + 1;
+                }
+                if (tv < n_win) {                              // V(tv) into the stage of V(tv - VST)
+                    mbar_wait(bar_vf0 + 8 * vs, (vf_par >> vs) & 1u, 8);
+                    vf_par ^= 1u << vs;
+                    mbar_expect_tx(bar_v0 + 8 * vs, S::KVTILE);
+#pragma unroll
+                    for (int sb = 0; sb < SUB; ++sb)
+                        tma_load_3d(sV + vs * S::KVTILE + sb * 8192, &tmV, sb * 64, j_start + tv * BN, bh, bar_v0 + 8 * vs);
+                    ++tv;
+                    vs = vs + 1 == VST ? 0 : vs + 1;
+                }
+            }
+        } else if (warp == 4 && lane == 0) {
+            // ---- MMA lane: nothing but barrier waits and tcgen05 issue; stage indices and parities roll
+            constexpr uint32_t IDESC_S = instr_desc(BM, BN, false);
+            constexpr uint32_t IDESC_O = S::ONES ? instr_desc(BM, D + 16, true) : instr_desc(BM, D, true);
+            // descriptor words: lo = (address >> 4) | LBO field, hi = SBO field | version | swizzle mode
+            constexpr uint32_t HI = (1024u >> 4) | (1u << 14) | (2u << 29);
+            const uint32_t q_lo = (sQ >> 4) | (1u << 16), k_lo = (sK >> 4) | (1u << 16);
+            // value operand: the second 64-column group of B is the next sub-tile (d = 128) or the block of ones
+            // (d = 64, LBO = its distance from the value stage)
+            uint32_t v_desc[VST];
+#pragma unroll
+            for (int st = 0; st < VST; ++st) {
+                const uint32_t va = sV + st * S::KVTILE;
+                v_desc[st] = (va >> 4) | ((S::ONES ? ((base + S::OFF_ONES - va) >> 4) : (8192u >> 4)) << 16);
+            }
+            uint32_t k_par = 0, v_par = 0, g_waited = 0;       // TMA barrier parities (bit per stage); bar_g phases consumed
+            int ks = 0, vs = 0;                                // stage of the next S / PV operand
+            int ts = 0;                                        // next S tile to issue
+            // gathers issued before the top of tile t have landed (the softmax warps signal from tile g_first on)
+            auto need_g = [&](int t) {
+                while ((int)g_waited <= t - g_first) { mbar_wait(bar_g0 + 8 * (g_waited & 1), (g_waited >> 1) & 1, 10); ++g_waited; }
+            };
+            auto mma_s = [&]() {                               // S(ts) from K stage ks into S buffer ts & 1
+                if (ts < n_win) { mbar_wait(bar_k0 + 8 * ks, (k_par >> ks) & 1u, 2); k_par ^= 1u << ks; }
+                tc_fence_after();
+                const uint32_t kb = k_lo + (uint32_t)ks * (S::KVTILE >> 4);
+                const uint32_t dcol = tmem + (ts & 1) * BN;
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk)
+                    umma(dcol, desc64(q_lo + (kk >> 2) * 1024 + (kk & 3) * 2, HI), desc64(kb + (kk >> 2) * 512 + (kk & 3) * 2, HI),
+                         IDESC_S, kk > 0);
+                umma_commit(bar_s0 + 8 * (ts & 1));
+                umma_commit(bar_kf0 + 8 * ks);                 // the K stage is free once S(ts) has completed
+                ++ts;
+                ks = ks + 1 == KST ? 0 : ks + 1;
+            };
+
+            mbar_wait(bar_q, 0, 1);
+            mma_s();                                           // tile 0 is always a window tile
+            if (n_tiles > 1) {
+                if (n_win < 2) need_g(0);                      // tile 1 is a retained tile: the prologue gathers
+                mma_s();
+            }
+            for (int t = 0; t < n_tiles; ++t) {
+                // PV(t): everything but P is normally there long before
+                need_g(t);
+                if (t < n_win) { mbar_wait(bar_v0 + 8 * vs, (v_par >> vs) & 1u, 4); v_par ^= 1u << vs; }
+                uint32_t vb = v_desc[0];
+#pragma unroll
+                for (int st = 1; st < VST; ++st) vb = vs == st ? v_desc[st] : vb;
+                mbar_wait(bar_p, t & 1, 7);
+                tc_fence_after();
+#pragma unroll
+                for (int kk = 0; kk < BN / 16; ++kk)
+                    umma_ts(tmem + O_COL, tmem + (t & 1) * BN + kk * 8, desc64(vb + kk * 128, HI), IDESC_O, (t > 0 || kk > 0) ? 1u : 0u);
+                umma_commit(bar_pv);
+                umma_commit(bar_vf0 + 8 * vs);                 // the V stage is free once PV(t) has completed
+                vs = vs + 1 == VST ? 0 : vs + 1;
+                // S(t+2) into the S buffer softmax(t) has just released
+                if (ts < n_tiles) mma_s();
+            }
+        }
+    } else {
+        // =================================== softmax warps ==================================================
+        const int i = i0 + tid;                                // this thread's query row
+        if (S::ONES) {                                         // 8 KB of bf16 1.0: 64 bytes per thread
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(base + S::OFF_ONES + tid * 64 + u * 16), "r"(0x3F803F80u) : "memory");
+        }
+        // retained entries visible to this row.  The rows of a warp are consecutive and the list is ascending, so
+        // nvis(row) = #{idx <= lim of lane 0} + #{idx in (lim of lane 0, lim of this lane]}: a ballot count plus a
+        // 31-bit map of the entries that fall between the warp's first and last limit.  No block barrier.
+        const int lim = min(i, Tlen - 1) - W;                  // entry visible iff idx <= lim
+        const int lim_max = i_hi - W;
+        const int lim0 = __shfl_sync(0xffffffffu, lim, 0), lim31 = __shfl_sync(0xffffffffu, lim, 31);
+        int nvis = 0, nv_max = 0;                              // nv_max: entries visible to the tile's last row
+        {
+            uint32_t bits = 0;
+            for (int e0 = 0; e0 < n_ret; e0 += 128) {
+                int e[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) e[u] = e0 + u * 32 + lane < n_ret ? id[e0 + u * 32 + lane] : 0x7fffffff;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    nvis += __popc(__ballot_sync(0xffffffffu, e[u] <= lim0));
+                    nv_max += __popc(__ballot_sync(0xffffffffu, e[u] <= lim_max));
+                    const bool in = e[u] > lim0 && e[u] <= lim31;
+                    bits |= __reduce_or_sync(0xffffffffu, in ? 1u << (e[u] - lim0 - 1) : 0u);
+                }
+                if (__shfl_sync(0xffffffffu, e[3], 31) > lim_max) break;   // nothing further is visible to any row
+            }
+            nvis += __popc(bits & ((1u << (lim - lim0)) - 1u));
+        }
+        const int n_tiles = n_win + (nv_max + BN - 1) / BN;
+
+        // gather of one retained tile: 8 lanes per row copy its 16-byte chunks (coalesced reads, conflict-free
+        // swizzled writes), 16 rows per pass; rows past the visible prefix are zero-filled
+        const int g_row = tid >> 3, g_sub = tid & 7;
+        auto gather_rows = [&](int t, int (&rows4)[4]) {       // row positions of this thread's 4 rows of tile t
+#pragma unroll
+            for (int ps = 0; ps < 4; ++ps) {
+                const int e = (t - n_win) * BN + ps * 16 + g_row;
+                rows4[ps] = (t >= n_win && t < n_tiles && e < nv_max) ? id[e] : -1;
+            }
+        };
+        auto gather_issue = [&](int t, bool is_v, const int (&rows4)[4]) {
+            if (t >= n_win && t < n_tiles) {
+                const int st = is_v ? (t % VST) : (t % KST);
+                const uint32_t dst = (is_v ? sV : sK) + st * S::KVTILE;
+#pragma unroll
+                for (int ps = 0; ps < 4; ++ps) {
+                    const int row = ps * 16 + g_row;
+                    const bool ok = rows4[ps] >= 0;
+                    const __nv_bfloat16* src = (is_v ? vg : kg) + ((size_t)bh * Tlen + (ok ? rows4[ps] : 0)) * D;
+#pragma unroll
+                    for (int c = g_sub; c < D / 8; c += 8) {
+                        const uint32_t off = (c >> 3) * 8192 + row * 128 + (((c & 7) ^ (row & 7)) << 4);
+                        cp_async16(dst + off, src + c * 8, ok ? 16u : 0u);
+                    }
+                }
+            }
+            cp_async_commit();
+        };
+        // prologue gathers: the first KST key tiles and VST value tiles (those that are retained tiles)
+        if (n_win < KST) {
+            int rows4[4];
+            for (int t = 0; t < KST; ++t) { gather_rows(t, rows4); gather_issue(t, false, rows4); }
+            for (int t = 0; t < VST; ++t) { gather_rows(t, rows4); gather_issue(t, true, rows4); }
+        }
+
+        const float c2 = scale * 1.4426950408889634f;          // logits are handled in the log2 domain: x = s * c2
+        const uint32_t lane_base = ((uint32_t)(warp * 32)) << 16;   // this warp's TMEM lanes
+        float m_run = -INFINITY, l_run = 0.f;                  // running max (log2 domain) and sum (sum only if !ONES)
+
+        for (int t = 0; t < n_tiles; ++t) {
+            // row positions for this tile's two gathers, fetched first so their latency hides under the softmax
+            int rk[4], rv[4];
+            gather_rows(t + KST, rk);
+            gather_rows(t + VST - 1, rv);
+            // gathers issued before this point have landed (all of them, or all but the latest value tile)
+            if (t >= g_first) {
+                if (VST == 3) cp_async_wait<1>(); else cp_async_wait<0>();
+                fence_proxy_async();
+                mbar_arrive(bar_g0 + 8 * ((t - g_first) & 1));
+            }
+
+            // column range this row may see in the tile
+            int c_lo, c_hi;
+            if (t < n_win) {
+                const int jt0 = j_start + t * BN;
+                c_lo = max(i - W + 1, 0) - jt0;
+                c_hi = i - jt0;
+            } else {
+                c_lo = 0;
+                c_hi = nvis - (t - n_win) * BN - 1;
+            }
+            // rows of a warp are consecutive and both bounds grow with the row: lane 0 / lane 31 give the warp's
+            // union range (columns any row sees) and intersection range (columns every row sees)
+            const int u_lo = __shfl_sync(0xffffffffu, c_lo, 0), u_hi = __shfl_sync(0xffffffffu, c_hi, 31);
+            const int n_lo = __shfl_sync(0xffffffffu, c_lo, 31), n_hi = __shfl_sync(0xffffffffu, c_hi, 0);
+            bool act[2], full[2];
+            uint32_t vm[2];                                    // per-thread validity bits of a partial chunk
+#pragma unroll
+            for (int cb = 0; cb < 2; ++cb) {
+                const int lo = cb * 32, hi = lo + 31;
+                act[cb] = lo <= u_hi && hi >= u_lo;
+                full[cb] = lo >= n_lo && hi <= n_hi;
+                const int a = min(max(c_lo - lo, 0), 32), b2 = min(max(c_hi - lo + 1, 0), 32);
+                const uint32_t below_b = b2 >= 32 ? 0xffffffffu : ((1u << b2) - 1u);
+                const uint32_t below_a = a >= 32 ? 0xffffffffu : ((1u << a) - 1u);
+                vm[cb] = b2 > a ? (below_b & ~below_a) : 0u;
+            }
+            mbar_wait(bar_s0 + 8 * (t & 1), (t >> 1) & 1, 3);  // S(t) is in TMEM buffer t & 1
+            tc_fence_after();
+            gather_issue(t + KST, false, rk);                  // its stage held K(t), which S(t) has finished reading
+            const uint32_t s_col = (t & 1) * BN;
+            uint32_t r[2][32];
+#pragma unroll
+            for (int cb = 0; cb < 2; ++cb)
+                if (act[cb]) tmem_ld32(tmem + lane_base + s_col + cb * 32, r[cb]);
+            tmem_wait_ld();
+            float mr[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // row max of the raw logits, 4 chains
+#pragma unroll
+            for (int cb = 0; cb < 2; ++cb) {
+                if (!act[cb]) continue;
+                if (full[cb]) {
+#pragma unroll
+                    for (int c = 0; c < 32; c += 2)
+                        mr[(c >> 1) & 3] = max3(mr[(c >> 1) & 3], __uint_as_float(r[cb][c]), __uint_as_float(r[cb][c + 1]));
+                } else {
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) {
+                        const float x = (vm[cb] & (1u << c)) ? __uint_as_float(r[cb][c]) : -INFINITY;
+                        r[cb][c] = __float_as_uint(x);
+                        mr[c & 3] = fmaxf(mr[c & 3], x);
+                    }
+                }
+            }
+            const float m_tile = fmaxf(fmaxf(mr[0], mr[1]), fmaxf(mr[2], mr[3])) * c2;
+            // lazy rescale: the running max only moves when the new one is far above it (exp2 arguments stay <= 8)
+            float alpha = 1.f;
+            bool need = false;
+            if (m_run == -INFINITY) m_run = m_tile;             // nothing accumulated yet for this row: O row is 0
+            else if (m_tile > m_run + 8.f) { alpha = fast_exp2(m_run - m_tile); m_run = m_tile; need = true; }
+            if (__any_sync(0xffffffffu, need)) {
+                // PV(t-1) must be done before O is rescaled
+                if (t > 0) { mbar_wait(bar_pv, (t - 1) & 1, 4); tc_fence_after(); }
+#pragma unroll
+                for (int cb = 0; cb < D / 32 + (S::ONES ? 1 : 0); ++cb) {   // with ONES the row-sum columns are rescaled too
+                    uint32_t q4[32];
+                    tmem_ld32(tmem + lane_base + O_COL + cb * 32, q4);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) q4[c] = __float_as_uint(__uint_as_float(q4[c]) * alpha);
+                    tmem_st32(tmem + lane_base + O_COL + cb * 32, q4);
+                }
+                tmem_wait_st();
+                l_run *= alpha;
+            }
+            const float neg_m = m_run == -INFINITY ? 0.f : -m_run;
+            float ls[4] = {0.f, 0.f, 0.f, 0.f};
+            uint32_t pk[32];                                   // the row of P as 64 bf16, two per word
+#pragma unroll
+            for (int cb = 0; cb < 2; ++cb) {
+                if (act[cb]) {
+#pragma unroll
+                    for (int c = 0; c < 32; c += 2) {
+                        // masked entries hold -inf: fma gives -inf and exp2(-inf) = 0
+                        const float p0 = fast_exp2(fmaf(__uint_as_float(r[cb][c]), c2, neg_m));
+                        const float p1 = fast_exp2(fmaf(__uint_as_float(r[cb][c + 1]), c2, neg_m));
+                        if (!S::ONES) ls[(c >> 1) & 3] += p0 + p1;   // with ONES the tensor core sums the rounded probabilities
+                        __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
+                        pk[cb * 16 + (c >> 1)] = *reinterpret_cast<uint32_t*>(&h);
+                    }
+                } else {
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) pk[cb * 16 + c] = 0u;
+                }
+            }
+            l_run += (ls[0] + ls[1]) + (ls[2] + ls[3]);
+            // P goes back into TMEM, over the first 32 columns of the S buffer it was computed from (this thread has
+            // all of its row in registers), and feeds the PV product as the A operand: no trip through shared memory
+            tmem_st32(tmem + lane_base + s_col, pk);
+            tmem_wait_st();
+            tc_fence_before();                                 // our TMEM accesses are ordered before the arrive
+            // PV(t-1) has normally completed long ago; the wait sits before the arrive so that the barrier cannot
+            // run two phases ahead of this thread
+            if (t > 0) mbar_wait(bar_pv, (t - 1) & 1, 4);
+            mbar_arrive(bar_p);
+            // value tile t+VST-1 goes into the stage of V(t-1), which PV(t-1) has finished reading
+            if (t > 0) gather_issue(t + VST - 1, true, rv); else cp_async_commit();
+        }
+        mbar_wait(bar_pv, (n_tiles - 1) & 1, 5);
+        tc_fence_after();
+
+        // ---- epilogue: O / l -> bf16, logsumexp ----------------------------------------------------------
+        if (S::ONES) {                                         // the row sum is column D of the accumulator
+            uint32_t q4[32];
+            tmem_ld32(tmem + lane_base + O_COL + D, q4);
+            tmem_wait_ld();
+            l_run = __uint_as_float(q4[0]);
+        }
+        const float inv = 1.f / l_run;
+        __nv_bfloat16* orow = o + ((size_t)bh * Tlen + i) * D;
+#pragma unroll
+        for (int cb = 0; cb < D / 32; ++cb) {
+            uint32_t q4[32];
+            tmem_ld32(tmem + lane_base + O_COL + cb * 32, q4);
+            tmem_wait_ld();
+            if (i < Tlen) {
+#pragma unroll
+                for (int c = 0; c < 32; c += 8) {
+                    uint32_t w4[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(q4[c + 2 * u]) * inv,
+                                                                 __uint_as_float(q4[c + 2 * u + 1]) * inv);
+                        w4[u] = *reinterpret_cast<uint32_t*>(&h);
+                    }
+                    *reinterpret_cast<uint4*>(orow + cb * 32 + c) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+                }
+            }
+        }
+        if (i < Tlen) lse[(size_t)bh * Tlen + i] = m_run * 0.6931471805599453f + logf(l_run);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 4) tmem_dealloc(tmem, TMEM_COLS);
+}
+
+template <int D>
+int run(const Params& p, const void* q, const void* k, const void* v, const int32_t* idx, const int32_t* cnt, void* o,
+        float* lse, cudaStream_t st)
+{
+    CUtensorMap tq, tk, tv;
+    const int BH = p.B * p.H;
+    if (!make_map(&tq, q, BH, p.T, D, BM) || !make_map(&tk, k, BH, p.T, D, BN) || !make_map(&tv, v, BH, p.T, D, BN))
+        return LTE_ERR_CUDA;
+    static bool attr_done = false;
+    if (!attr_done) {
+        if (cudaFuncSetAttribute(prefill_long_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::BYTES) !=
+            cudaSuccess)
+            return LTE_ERR_CUDA;
+        attr_done = true;
+    }
+    dim3 grid((p.T + BM - 1) / BM, BH);
+    prefill_long_kernel<D><<<grid, NTHREADS, Smem<D>::BYTES, st>>>(tq, tk, tv, (const __nv_bfloat16*)k,
+                                                                 (const __nv_bfloat16*)v, idx, cnt, (__nv_bfloat16*)o,
+                                                                 lse, p.T, p.W, p.R, p.scale);
+    return cuda_status(cudaGetLastError());
+}
+
+}  // namespace
+
+int launch_prefill_tc_long(const Params& p, const void* q, const void* k, const void* v, const int32_t* idx,
+                           const int32_t* cnt, void* o, float* lse, cudaStream_t st)
+{
+    if (p.d != 128) return LTE_ERR_UNSUPPORTED;
+    return run<128>(p, q, k, v, idx, cnt, o, lse, st);
+}
+
+int prefill_long_status_fetch_and_clear()
+{
+    int h = 0, zero = 0;
+    if (cudaMemcpyFromSymbol(&h, g_prefill_long_status, sizeof(int)) != cudaSuccess) return -1;
+    if (h != 0) cudaMemcpyToSymbol(g_prefill_long_status, &zero, sizeof(int));
+    return h;
+}
+
+}  // namespace lte
