@@ -100,4 +100,27 @@ int launch_bwd(const Params& p, const void* q, const void* k, const void* v, con
 
 inline int cuda_status(cudaError_t e) { return e == cudaSuccess ? LTE_OK : LTE_ERR_CUDA; }
 
+// Programmatic dependent launch: a kernel launched through launch_pdl may become resident while its predecessor in the
+// stream is still running, and does its set-up (barriers, tensor memory, index arithmetic) there.  It must execute
+// pdl_wait() before it reads anything a predecessor may have written and before its first global write; the wait
+// returns once every earlier grid of the stream has completed and its writes are visible.  pdl_launch_dependents()
+// lets the successor (if it was launched the same way) start becoming resident.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+
 }  // namespace lte

@@ -153,6 +153,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot_gen;
+    pdl_launch_dependents();
+    pdl_wait();                                                // everything above ran beside the previous kernel's tail
 
     if (warp == 5) {
         // ================================= load warp (lane 0 issues) ========================================
@@ -555,10 +557,9 @@ int run(const Params& p, const void* q, const void* k, const void* v, const int3
     }
     const int n_qt = (p.T + BM - 1) / BM, n_items = n_qt * BH;
     const int grid = n_items < slots ? n_items : slots;
-    prefill_tc_kernel<D><<<grid, NTHREADS, Smem<D>::BYTES, st>>>(tq, tk, tv, to, (const __nv_bfloat16*)k,
+    return cuda_status(launch_pdl(prefill_tc_kernel<D>, dim3(grid), dim3(NTHREADS), Smem<D>::BYTES, st, tq, tk, tv, to, (const __nv_bfloat16*)k,
                                                                  (const __nv_bfloat16*)v, idx, cnt,
-                                                                 lse, p.T, p.W, p.R, p.scale, n_qt, BH);
-    return cuda_status(cudaGetLastError());
+                                                                 lse, p.T, p.W, p.R, p.scale, n_qt, BH));
 }
 
 }  // namespace

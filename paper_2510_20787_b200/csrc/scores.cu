@@ -166,6 +166,8 @@ __global__ void __launch_bounds__(NT + 64) scores_tc_kernel(const __grid_constan
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot_gen;
+    pdl_launch_dependents();
+    pdl_wait();                                          // everything above ran beside the previous kernel's tail
 
     if (warp == 5) {
         // ---- load lane: streams the input tiles through the stage ring ----------------------------------------------
@@ -335,7 +337,9 @@ int run_tma(const Params& p, const void* k, const void* v, float* z, float* r, c
     if (n_flat > 0x7fffffffLL) return LTE_ERR_UNSUPPORTED;
     const int slots = n_sm * (D == 64 ? 2 : 1);
     const int n_cta = (int)(n_flat < slots ? n_flat : slots);
-    scores_tc_kernel<D, K><<<n_cta, NT + 64, C::BYTES, st>>>(tk, tv, p.w, p.bias, z, r, p.H, p.T, (int)n_flat, status_ptr);
+    if (launch_pdl(scores_tc_kernel<D, K>, dim3(n_cta), dim3(NT + 64), C::BYTES, st, tk, tv, p.w, p.bias, z, r, p.H, p.T,
+                   (int)n_flat, status_ptr) != cudaSuccess)
+        return LTE_ERR_CUDA;
     return cuda_status(cudaGetLastError());
 }
 

@@ -151,6 +151,8 @@ __global__ void __launch_bounds__(1024) select_reg_kernel(const float* __restric
 {
     __shared__ uint32_t s_count[3];
     __shared__ uint32_t s_wa[32], s_we[32];
+    pdl_launch_dependents();
+    pdl_wait();                                            // z comes from the previous kernel
     const int bh = blockIdx.x;
     const float* zz = z + (size_t)bh * T;
     int32_t* out = idx + (size_t)bh * R;
@@ -250,7 +252,7 @@ int launch_select(const Params& p, const float* z, int32_t* idx, int32_t* cnt, i
         const int nt = N <= 2048 ? 256 : 1024;
         const int kpt = (N + nt - 1) / nt;
         const int BH = p.B * p.H;
-#define LTE_SEL(KPT) select_reg_kernel<KPT><<<BH, nt, 0, st>>>(z, idx, cnt, ncand, p.T, p.W, p.R, p.sink, p.zthr)
+#define LTE_SEL(KPT) launch_pdl(select_reg_kernel<KPT>, dim3(BH), dim3(nt), 0, st, z, idx, cnt, ncand, p.T, p.W, p.R, p.sink, p.zthr)
         if (kpt <= 64) {
             if (kpt <= 1) LTE_SEL(1); else if (kpt <= 2) LTE_SEL(2); else if (kpt <= 4) LTE_SEL(4);
             else if (kpt <= 8) LTE_SEL(8); else if (kpt <= 16) LTE_SEL(16); else if (kpt <= 32) LTE_SEL(32);
