@@ -206,6 +206,8 @@ __global__ void bwd_conv_partial_kernel(const T* __restrict__ k, const T* __rest
 __global__ void bwd_conv_reduce_kernel(const float* __restrict__ part_w, const float* __restrict__ part_b,
                                        float* __restrict__ dw, float* __restrict__ dbias, int nparts, int per_head)
 {
+    pdl_launch_dependents();
+    pdl_wait();                                                // see launch_pdl: earlier kernels of the stream have completed
     const int h = blockIdx.y;
     const int e = blockIdx.x * blockDim.x + threadIdx.x;
     if (e < per_head) {
@@ -317,6 +319,8 @@ bwd_tail_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __rest
                 const float* __restrict__ w, __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv,
                 float* __restrict__ part_w, float* __restrict__ part_b, int B, int H, int Tlen, int nchunk, int rows)
 {
+    pdl_launch_dependents();
+    pdl_wait();                                                // see launch_pdl: earlier kernels of the stream have completed
     constexpr int TPR = 2 * D / 4;                  // threads per position: D/4 for k, D/4 for v
     constexpr int RPP = 256 / TPR;                  // positions per pass (row slots)
     constexpr int half = K / 2;
@@ -456,10 +460,10 @@ int run_tail(const Params& p, const void* k, const void* v, const float* dz, voi
     const size_t sm = (size_t)(((rows + K - 1 + 3) & ~3) + (256 / (2 * D / 4) / 2) * K * 2 * D) * sizeof(float);
     dim3 grid(p.B * nchunk, p.H);
     if (finish)
-        bwd_tail_kernel<D, K, true><<<grid, 256, sm, st>>>((const __nv_bfloat16*)k, (const __nv_bfloat16*)v, dz, p.w,
+        launch_pdl(bwd_tail_kernel<D, K, true>, grid, dim3(256), sm, st, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, dz, p.w,
                                                           (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, part_w, part_b, p.B, p.H, p.T, nchunk, rows);
     else
-        bwd_tail_kernel<D, K, false><<<grid, 256, sm, st>>>((const __nv_bfloat16*)k, (const __nv_bfloat16*)v, dz, p.w,
+        launch_pdl(bwd_tail_kernel<D, K, false>, grid, dim3(256), sm, st, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, dz, p.w,
                                                            (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, part_w, part_b, p.B, p.H, p.T, nchunk, rows);
     return cuda_status(cudaGetLastError());
 }
@@ -532,7 +536,7 @@ int run(const Params& p, const void* q, const void* k, const void* v, const void
             const int e = p.K == 7 ? run_tail<D, 7>(p, k, v, dz, dk, dv, part_w, part_b, f32, nch, rows, st)
                                    : run_tail<D, 5>(p, k, v, dz, dk, dv, part_w, part_b, f32, nch, rows, st);
             if (e != LTE_OK) return e;
-            bwd_conv_reduce_kernel<<<gr, 256, 0, st>>>(part_w, part_b, dw, dbias, p.B * nch, per_head);
+            launch_pdl(bwd_conv_reduce_kernel, gr, dim3(256), 0, st, part_w, part_b, dw, dbias, p.B * nch, per_head);
             return cuda_status(cudaGetLastError());
         }
     }

@@ -54,6 +54,8 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                  const float* __restrict__ lse, const int32_t* __restrict__ idx, const int32_t* __restrict__ cnt,
                  __nv_bfloat16* __restrict__ dq, float* __restrict__ delta, int Tlen, int W, int R, float scale)
 {
+    pdl_launch_dependents();
+    pdl_wait();                                                // see launch_pdl: earlier kernels of the stream have completed
     using S = SmemQ<D>;
     constexpr int SUB = S::SUB;
     constexpr uint32_t DP_COL = BN, DQ_COL = 2 * BN;
@@ -364,6 +366,8 @@ bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                   float* __restrict__ dk_ret, float* __restrict__ dv_ret, float* __restrict__ dr_ret, int n_wt, int Tlen,
                   int W, int R, float scale)
 {
+    pdl_launch_dependents();
+    pdl_wait();                                                // see launch_pdl: earlier kernels of the stream have completed
     using S = SmemK<D>;
     constexpr int SUB = S::SUB;
     constexpr uint32_t DP_COL = 64, DV_COL = 128, DK_COL = 128 + D;
@@ -648,6 +652,8 @@ __global__ void bwd_merge_kernel(const int32_t* __restrict__ idx, const int32_t*
                                  __nv_bfloat16* __restrict__ dv, float* __restrict__ dk32, float* __restrict__ dv32,
                                  float* __restrict__ dr_win, int Tlen, int R, int D)
 {
+    pdl_launch_dependents();
+    pdl_wait();                                                // see launch_pdl: earlier kernels of the stream have completed
     const int bh = blockIdx.y, e = blockIdx.x;
     if (e >= cnt[bh]) return;
     const int j = idx[(size_t)bh * R + e];
@@ -666,6 +672,8 @@ __global__ void bwd_merge_kernel(const int32_t* __restrict__ idx, const int32_t*
 __global__ void bwd_dz_kernel(float* __restrict__ dz, const float* __restrict__ z, const float* __restrict__ lambda, int H,
                               int Tlen, int half, float zthr)
 {
+    pdl_launch_dependents();
+    pdl_wait();                                                // see launch_pdl: earlier kernels of the stream have completed
     const int bh = blockIdx.y;
     const int j = blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= Tlen) return;
@@ -700,7 +708,7 @@ int launch_bwd_dq_tc(const Params& p, const void* q, const void* k, const void* 
                                      SmemQ<D>::BYTES) != cudaSuccess) return LTE_ERR_CUDA;                         \
             attr_done = true;                                                                                      \
         }                                                                                                          \
-        bwd_dq_tc_kernel<D><<<grid, NTHREADS, SmemQ<D>::BYTES, st>>>(                                        \
+        launch_pdl(bwd_dq_tc_kernel<D>, grid, dim3(NTHREADS), SmemQ<D>::BYTES, st,                            \
             tq, tdo, tk, tv, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (const __nv_bfloat16*)o,            \
             (const __nv_bfloat16*)dO, lse, idx, cnt, (__nv_bfloat16*)dq, delta, p.T, p.W, p.R, p.scale);           \
     } while (0)
@@ -739,7 +747,7 @@ int launch_bwd_dkv_tc(const Params& p, const void* q, const void* k, const void*
                                      SmemK<D>::BYTES) != cudaSuccess) return LTE_ERR_CUDA;                         \
             attr_done = true;                                                                                      \
         }                                                                                                          \
-        bwd_dkv_tc_kernel<D, F><<<grid, NTHREADS, SmemK<D>::BYTES, st>>>(                                           \
+        launch_pdl(bwd_dkv_tc_kernel<D, F>, grid, dim3(NTHREADS), SmemK<D>::BYTES, st,                              \
             tk, tv, tq, tdo, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, lse, delta, idx, cnt,               \
             (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, dk32, dv32, dz, dk_ret, dv_ret, dr_ret, n_wt, p.T, p.W, p.R,   \
             p.scale);                                                                                              \
@@ -751,14 +759,14 @@ int launch_bwd_dkv_tc(const Params& p, const void* q, const void* k, const void*
     if (p.R > 0) {
         dim3 gm(p.R, BH);
         if (f32out)
-            bwd_merge_kernel<true><<<gm, 64, 0, st>>>(idx, cnt, dk_ret, dv_ret, dr_ret, (__nv_bfloat16*)dk, (__nv_bfloat16*)dv,
+            launch_pdl(bwd_merge_kernel<true>, gm, dim3(64), 0, st, idx, cnt, dk_ret, dv_ret, dr_ret, (__nv_bfloat16*)dk, (__nv_bfloat16*)dv,
                                                       dk32, dv32, dz, p.T, p.R, p.d);
         else
-            bwd_merge_kernel<false><<<gm, 64, 0, st>>>(idx, cnt, dk_ret, dv_ret, dr_ret, (__nv_bfloat16*)dk, (__nv_bfloat16*)dv,
+            launch_pdl(bwd_merge_kernel<false>, gm, dim3(64), 0, st, idx, cnt, dk_ret, dv_ret, dr_ret, (__nv_bfloat16*)dk, (__nv_bfloat16*)dv,
                                                        dk32, dv32, dz, p.T, p.R, p.d);
     }
     dim3 gz((p.T + 255) / 256, BH);
-    bwd_dz_kernel<<<gz, 256, 0, st>>>(dz, z, lambda, p.H, p.T, p.half, p.zthr);
+    launch_pdl(bwd_dz_kernel, gz, dim3(256), 0, st, dz, z, lambda, p.H, p.T, p.half, p.zthr);
     return cuda_status(cudaGetLastError());
 }
 

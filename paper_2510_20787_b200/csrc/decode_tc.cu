@@ -86,6 +86,8 @@ __global__ void __launch_bounds__(NTHR) decode_tc_kernel(unsigned char* __restri
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot_gen;
+    pdl_launch_dependents();
+    pdl_wait();                                                // the previous step (or whatever wrote the cache and the inputs) has completed
 
     if (wid == 8) {
         // ======================================== control lane ==================================================
@@ -352,10 +354,9 @@ int launch_decode_tc(const Params& p, void* cache, const void* q1, const void* k
     const int slots = 3 * n_sm;                                // three CTAs per SM
     const int per_cta = (BH + slots - 1) / slots;
     const int n_cta = (BH + per_cta - 1) / per_cta;
-    decode_tc_kernel<<<n_cta, NTHR, P.total, st>>>((unsigned char*)cache, L, (const __nv_bfloat16*)q1,
+    return cuda_status(launch_pdl(decode_tc_kernel, dim3(n_cta), dim3(NTHR), P.total, st, (unsigned char*)cache, L, (const __nv_bfloat16*)q1,
                                                    (const __nv_bfloat16*)k1, (const __nv_bfloat16*)v1, (__nv_bfloat16*)o1, lse1,
-                                                   p.w, p.bias, BH, per_cta, p.H, p.W, p.R, p.sink, p.K, p.zthr, p.scale);
-    return cuda_status(cudaGetLastError());
+                                                   p.w, p.bias, BH, per_cta, p.H, p.W, p.R, p.sink, p.K, p.zthr, p.scale));
 }
 
 int decode_tc_status_fetch_and_clear()

@@ -89,7 +89,6 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const int j_start = max(i0 - W + 1, 0);
     const int n_win = (i_hi - j_start + 1 + BN - 1) / BN;
     const int32_t* id = idx + (size_t)bh * R;
-    const int n_ret = cnt[bh];
     const int g_first = max(n_win - Smem<D>::KST, 0);        // first tile whose top may have gathers in flight
 
     if (tid == 0) {
@@ -109,6 +108,9 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot_gen;
+    pdl_launch_dependents();
+    pdl_wait();                                                // everything above ran beside the previous kernel's tail
+    const int n_ret = cnt[bh];
 
     if (warp >= 4) {
         // ============================ load lane (warp 5) and MMA lane (warp 4) ==============================
@@ -474,10 +476,9 @@ int run(const Params& p, const void* q, const void* k, const void* v, const int3
         attr_done = true;
     }
     dim3 grid((p.T + BM - 1) / BM, BH);
-    prefill_long_kernel<D><<<grid, NTHREADS, Smem<D>::BYTES, st>>>(tq, tk, tv, (const __nv_bfloat16*)k,
+    return cuda_status(launch_pdl(prefill_long_kernel<D>, grid, dim3(NTHREADS), Smem<D>::BYTES, st, tq, tk, tv, (const __nv_bfloat16*)k,
                                                                  (const __nv_bfloat16*)v, idx, cnt, (__nv_bfloat16*)o,
-                                                                 lse, p.T, p.W, p.R, p.scale);
-    return cuda_status(cudaGetLastError());
+                                                                 lse, p.T, p.W, p.R, p.scale));
 }
 
 }  // namespace
