@@ -86,11 +86,11 @@ __device__ __forceinline__ int count_le(const int32_t* id, int n, int lim, int l
 // They meet on mbarriers (g = the tile's number within the CTA, it = the item's):
 //   bar_q                    Q of item `it` has landed (TMA)                          phase it
 //   bar_qf    (commit)       the last S product of item `it` has completed            phase it     MMA -> load
-//   bar_of    (128 arrivals) O of item `it` has been read out of TMEM                 phase it     softmax -> MMA
+//   bar_of    (4 arrivals)   O of item `it` has been read out of TMEM                 phase it     softmax -> MMA
 //   bar_s[b]  (commit)       S(g) is in TMEM buffer b = g & 1                         phase g >> 1 MMA -> softmax
-//   bar_p     (128 arrivals) P(g) is in TMEM, over S(g)                               phase g      softmax -> MMA
+//   bar_p     (4 arrivals)   P(g) is in TMEM, over S(g)                               phase g      softmax -> MMA
 //   bar_pv    (commit)       PV(g) has completed                                      phase g      MMA -> softmax
-//   bar_g[b]  (128 arrivals) gathers issued before the top of tile g have landed      phase g >> 1 softmax -> MMA
+//   bar_g[b]  (4 arrivals)   gathers issued before the top of tile g have landed      phase g >> 1 softmax -> MMA
 //   bar_k[s], bar_v[s]       TMA transaction barriers of the window tiles (one phase per TMA use of the stage)
 //   bar_kf[s], bar_vf[s]     (commit) the MMA that read the stage's tile g has completed   phase g / stages   MMA -> load
 // S(g+1) and S(g+2) are computed while the softmax of tile g runs; loads run two to three tiles ahead, across items.
@@ -137,9 +137,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             mbar_init(bar_kf0 + 8 * s2, 1); mbar_init(bar_vf0 + 8 * s2, 1);
         }
         mbar_init(bar_s0, 1); mbar_init(bar_s0 + 8, 1);
-        mbar_init(bar_g0, 128); mbar_init(bar_g0 + 8, 128);
-        mbar_init(bar_p, 128); mbar_init(bar_pv, 1);
-        mbar_init(bar_qf, 1); mbar_init(bar_of, 128);
+        // the softmax warps arrive once per warp (lane 0, after __syncwarp): 128 arrivals on one barrier word serialise
+        mbar_init(bar_g0, 4); mbar_init(bar_g0 + 8, 4);
+        mbar_init(bar_p, 4); mbar_init(bar_pv, 1);
+        mbar_init(bar_qf, 1); mbar_init(bar_of, 4);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 4) tmem_alloc(tmem_slot, TMEM_COLS);
@@ -369,7 +370,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     if (VST == 3) cp_async_wait<1>(); else cp_async_wait<0>();
                     fence_proxy_async();
                 }
-                mbar_arrive(bar_g0 + 8 * (gg & 1));
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_g0 + 8 * (gg & 1));
 
                 // column range this row may see in the tile
                 int c_lo, c_hi;
@@ -475,7 +477,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 // parity test is only meaningful for the current or the previous phase), and before the arrive: after
                 // it the barrier could run ahead of this thread.  At t = 0 the item's epilogue has awaited it.
                 if (t > 0) mbar_wait(bar_pv, (gg - 1) & 1, 4);
-                mbar_arrive(bar_p);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_p);
                 // value tile t+VST-1 goes into the stage of tile t-1's V, which that PV has finished reading
                 if (v_gather) { gather_issue(t + VST - 1, true, rv); gathered = true; }
                 else cp_async_commit();
@@ -510,7 +513,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 }
                 if (sb == SUB - 1) {
                     tc_fence_before();
-                    mbar_arrive(bar_of);                       // the accumulator may take the next item
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_of);        // the accumulator may take the next item
                 }
                 if (lane == 0) bulk_wait_read0();              // the slab's previous store has been read out
                 __syncwarp();
