@@ -31,8 +31,8 @@ METRIC = "LTE attn prefill tokens/s & % bf16 TC peak; decode step us & % HBM BW"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu captures (profiles/),
-# keyed by kernel family (profiles/prefill_tc_kernel_C2.md, profiles/decode_bulk_kernel_C4.md).
-NCU_TRAFFIC_BYTES = {"prefill_attn_C2": 117.1e6, "decode_C4": 142.9e6}
+# keyed by kernel family (profiles/prefill_tc_kernel_C2.md, profiles/decode_tc_kernel_C4.md).
+NCU_TRAFFIC_BYTES = {"prefill_attn_C2": 115.0e6, "decode_C4": 142.4e6}
 
 
 def peaks():
