@@ -260,13 +260,27 @@ def run_lte(args):
     hc = torch.empty(cnt.shape, dtype=cnt.dtype).pin_memory()
     dq_, dk_, dv_ = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
 
+    # One batch element per stream, round-robin over a few streams: the host->device copy of element b+1, the kernels
+    # of element b and the device->host copy of element b-1 overlap (the two copy directions use different engines).
+    s1 = lte.shape(1, cfg.H, cfg.T, cfg.d, cfg.W, cfg.R, lte.BF16)
+    side = [torch.cuda.Stream() for _ in range(min(cfg.B, 4))]
+
     def e2e_step():
-        dq_.copy_(hq, non_blocking=True); dk_.copy_(hk, non_blocking=True); dv_.copy_(hv, non_blocking=True)
-        lte.lte_scores(s, c, dk_, dv_, z=z)
-        lte.lte_select(s, z, idx=idx, cnt=cnt)
-        lte.lte_attn_prefill(s, dq_, dk_, dv_, idx, cnt, o=o, lse=lse)
-        ho.copy_(o, non_blocking=True); hl.copy_(lse, non_blocking=True)
-        hi.copy_(idx, non_blocking=True); hc.copy_(cnt, non_blocking=True)
+        cur = torch.cuda.current_stream()
+        for st in side:
+            st.wait_stream(cur)
+        for b in range(cfg.B):
+            st = side[b % len(side)]
+            with torch.cuda.stream(st):
+                sl = slice(b, b + 1)
+                dq_[sl].copy_(hq[sl], non_blocking=True); dk_[sl].copy_(hk[sl], non_blocking=True); dv_[sl].copy_(hv[sl], non_blocking=True)
+                lte.lte_scores(s1, c, dk_[sl], dv_[sl], z=z[sl])
+                lte.lte_select(s1, z[sl], idx=idx[sl], cnt=cnt[sl])
+                lte.lte_attn_prefill(s1, dq_[sl], dk_[sl], dv_[sl], idx[sl], cnt[sl], o=o[sl], lse=lse[sl])
+                ho[sl].copy_(o[sl], non_blocking=True); hl[sl].copy_(lse[sl], non_blocking=True)
+                hi[sl].copy_(idx[sl], non_blocking=True); hc[sl].copy_(cnt[sl], non_blocking=True)
+        for st in side:
+            cur.wait_stream(st)
         return None
 
     barrier()
