@@ -48,6 +48,7 @@ template <int D> struct SmemQ {                                // dq kernel
 template <int D>
 __global__ void __launch_bounds__(NTHREADS, D == 64 ? 2 : 1)
 bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmDO,
+                 const __grid_constant__ CUtensorMap tmO,
                  const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                  const __nv_bfloat16* __restrict__ kg, const __nv_bfloat16* __restrict__ vg,
                  const __nv_bfloat16* __restrict__ og, const __nv_bfloat16* __restrict__ dog,
@@ -144,15 +145,16 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                 umma_commit(bar_s);
             };
 
-            mbar_expect_tx(bar_q, 2 * S::QTILE);
+            // d = 64: the O tile rides along into the (still unused) dS buffer, for delta = <dO, O>
+            mbar_expect_tx(bar_q, (D == 64 ? 3 : 2) * S::QTILE);
 #pragma unroll
             for (int sb = 0; sb < SUB; ++sb) {
                 tma_load_3d(sQ + sb * 16384, &tmQ, sb * 64, i0, bh, bar_q);
                 tma_load_3d(sDO + sb * 16384, &tmDO, sb * 64, i0, bh, bar_q);
             }
+            if (D == 64) tma_load_3d(sDS, &tmO, 0, i0, bh, bar_q);
             for (int t = 0; t < NST && t < n_win; ++t) { tma_kv(t, false); tma_kv(t, true); }
-            need_g(0);
-            bwait(bar_q, 0, 1);
+            bwait(bar_q, 0, 1);                                // (tile 0 is always a window tile: no gather to wait for)
             wait_kv(0);
             tc_fence_after();
             mma_s_dp(0);
@@ -181,9 +183,25 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         // =================================== softmax warps ==================================================
         const int i = i0 + tid;
         const int ic = min(i, Tlen - 1);
-        // delta_i = <dO_i, O_i>, L2_i = lse_i * log2(e)
+        // delta_i = <dO_i, O_i>, L2_i = lse_i * log2(e).  d = 64: both rows are in shared memory (the TMA tiles of dO and
+        // O, 128-byte swizzle: chunk c of row r sits at chunk position c ^ (r & 7)); d = 128: from global memory.
         float dl = 0.f;
-        {
+        const float L2 = lse[(size_t)bh * Tlen + ic] * kLog2e;
+        if (D == 64) {
+            bwait(bar_q, 0, 12);
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                const uint32_t off = tid * 128 + ((c ^ (tid & 7)) << 4);
+                uint32_t aw[4], bw[4];
+                asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(aw[0]), "=r"(aw[1]), "=r"(aw[2]), "=r"(aw[3]) : "r"(sDS + off));
+                asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(bw[0]), "=r"(bw[1]), "=r"(bw[2]), "=r"(bw[3]) : "r"(sDO + off));
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    dl = fmaf(__uint_as_float(aw[u] << 16), __uint_as_float(bw[u] << 16), dl);
+                    dl = fmaf(__uint_as_float(aw[u] & 0xffff0000u), __uint_as_float(bw[u] & 0xffff0000u), dl);
+                }
+            }
+        } else {
             const uint4* orow = reinterpret_cast<const uint4*>(og + ((size_t)bh * Tlen + ic) * D);
             const uint4* grow = reinterpret_cast<const uint4*>(dog + ((size_t)bh * Tlen + ic) * D);
 #pragma unroll 4
@@ -198,27 +216,29 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             }
         }
         if (i < Tlen) delta[(size_t)bh * Tlen + i] = dl;
-        const float L2 = lse[(size_t)bh * Tlen + ic] * kLog2e;
 
+        // retained entries visible to this row: rows of a warp are consecutive and the list is ascending, so the count is
+        // #{idx <= lim of lane 0} plus the entries between the warp's first limit and this lane's (a 31-bit map)
         const int lim = ic - W, lim_max = i_hi - W;
-        int nvis = 0;
-        for (int e0 = 0; e0 < n_ret; e0 += 128) {
-            const int n_here = min(128, n_ret - e0);
-            group_sync();
-            if (tid < n_here) s_idx[tid] = id[e0 + tid];
-            group_sync();
-            if (s_idx[n_here - 1] <= lim) nvis += n_here;
-            else {
-                int lo = 0, hi = n_here;
-                while (lo < hi) { const int mid = (lo + hi) >> 1; if (s_idx[mid] <= lim) lo = mid + 1; else hi = mid; }
-                nvis += lo;
+        const int lim0 = __shfl_sync(0xffffffffu, lim, 0), lim31 = __shfl_sync(0xffffffffu, lim, 31);
+        int nvis = 0, nv_max = 0;
+        {
+            uint32_t bits = 0;
+            for (int e0 = 0; e0 < n_ret; e0 += 128) {
+                int e[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) e[u] = e0 + u * 32 + lane < n_ret ? id[e0 + u * 32 + lane] : 0x7fffffff;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    nvis += __popc(__ballot_sync(0xffffffffu, e[u] <= lim0));
+                    nv_max += __popc(__ballot_sync(0xffffffffu, e[u] <= lim_max));
+                    const bool in = e[u] > lim0 && e[u] <= lim31;
+                    bits |= __reduce_or_sync(0xffffffffu, in ? 1u << (e[u] - lim0 - 1) : 0u);
+                }
+                if (__shfl_sync(0xffffffffu, e[3], 31) > lim_max) break;
             }
-            if (s_idx[n_here - 1] > lim_max) break;
+            nvis += __popc(bits & ((1u << (lim - lim0)) - 1u));
         }
-        group_sync();
-        if (i == i_hi) s_idx[0] = nvis;
-        group_sync();
-        const int nv_max = s_idx[0];
         const int n_tiles = n_win + (nv_max + BN - 1) / BN;
 
         const int g_row = tid >> 3, g_sub = tid & 7;
@@ -695,8 +715,8 @@ int launch_bwd_dq_tc(const Params& p, const void* q, const void* k, const void* 
                      const void* dO, const int32_t* idx, const int32_t* cnt, void* dq, float* delta, cudaStream_t st)
 {
     const int BH = p.B * p.H;
-    CUtensorMap tq, tdo, tk, tv;
-    if (!make_map(&tq, q, BH, p.T, p.d, BM) || !make_map(&tdo, dO, BH, p.T, p.d, BM) ||
+    CUtensorMap tq, tdo, to, tk, tv;
+    if (!make_map(&tq, q, BH, p.T, p.d, BM) || !make_map(&tdo, dO, BH, p.T, p.d, BM) || !make_map(&to, o, BH, p.T, p.d, BM) ||
         !make_map(&tk, k, BH, p.T, p.d, BN) || !make_map(&tv, v, BH, p.T, p.d, BN))
         return LTE_ERR_CUDA;
     dim3 grid((p.T + BM - 1) / BM, BH);
@@ -709,7 +729,7 @@ int launch_bwd_dq_tc(const Params& p, const void* q, const void* k, const void* 
             attr_done = true;                                                                                      \
         }                                                                                                          \
         launch_pdl(bwd_dq_tc_kernel<D>, grid, dim3(NTHREADS), SmemQ<D>::BYTES, st,                            \
-            tq, tdo, tk, tv, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (const __nv_bfloat16*)o,            \
+            tq, tdo, to, tk, tv, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (const __nv_bfloat16*)o,        \
             (const __nv_bfloat16*)dO, lse, idx, cnt, (__nv_bfloat16*)dq, delta, p.T, p.W, p.R, p.scale);           \
     } while (0)
     if (p.d == 64) LTE_GO(64); else if (p.d == 128) LTE_GO(128); else return LTE_ERR_UNSUPPORTED;
