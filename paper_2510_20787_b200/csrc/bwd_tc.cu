@@ -379,6 +379,7 @@ template <int D, bool F32OUT>
 __global__ void __launch_bounds__(NTHREADS, D == 64 ? 2 : 1)
 bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                   const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmDO,
+                  const __grid_constant__ CUtensorMap tmDK, const __grid_constant__ CUtensorMap tmDV,
                   const __nv_bfloat16* __restrict__ kg, const __nv_bfloat16* __restrict__ vg,
                   const float* __restrict__ lse, const float* __restrict__ delta, const int32_t* __restrict__ idx,
                   const int32_t* __restrict__ cnt, __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv,
@@ -631,14 +632,14 @@ bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                         }
                     }
                 }
-                if (live) {
+                if (live && (is_ret || F32OUT || D != 64)) {
                     if (is_ret || F32OUT) {
                         float* dst = (is_ret ? (half2 ? dk_ret : dv_ret) : (half2 ? dk32 : dv32)) + orow + cb * 32;
 #pragma unroll
                         for (int c = 0; c < 32; c += 4)
                             *reinterpret_cast<float4*>(dst + c) = make_float4(__uint_as_float(a4[c]), __uint_as_float(a4[c + 1]),
                                                                               __uint_as_float(a4[c + 2]), __uint_as_float(a4[c + 3]));
-                    } else {
+                    } else if (D != 64) {
                         __nv_bfloat16* dst = (half2 ? dk : dv) + orow + cb * 32;
 #pragma unroll
                         for (int c = 0; c < 32; c += 8) {
@@ -652,6 +653,33 @@ bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                         }
                     }
                 }
+                if (D == 64 && !is_ret && !F32OUT) {
+                    // window tile, bf16 out: the rows go into the (now idle) P^T / dS^T operand buffers in the swizzled
+                    // layout and leave as one tile store per warp (a 128-byte store per thread stalls the load/store unit)
+                    const uint32_t buf = half2 ? sDST : sPT;
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        uint32_t w4[4];
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(a4[g * 8 + 2 * u]), __uint_as_float(a4[g * 8 + 2 * u + 1]));
+                            w4[u] = *reinterpret_cast<uint32_t*>(&h);
+                        }
+                        const int ch = cb * 4 + g;
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(buf + tid * 128 + ((ch ^ (tid & 7)) << 4)),
+                                     "r"(w4[0]), "r"(w4[1]), "r"(w4[2]), "r"(w4[3]) : "memory");
+                    }
+                }
+            }
+        }
+        if (D == 64 && !is_ret && !F32OUT) {
+            fence_proxy_async();
+            __syncwarp();
+            if (lane == 0 && j0 + warp * 32 < Tlen) {
+                tma_store_3d(&tmDV, sPT + warp * 4096, 0, j0 + warp * 32, bh);
+                tma_store_3d(&tmDK, sDST + warp * 4096, 0, j0 + warp * 32, bh);
+                bulk_commit();
+                bulk_wait_read0();                             // the buffers are released with the CTA
             }
         }
         if (live) {
@@ -749,9 +777,10 @@ int launch_bwd_dkv_tc(const Params& p, const void* q, const void* k, const void*
                       void* dk, void* dv, float* dk32, float* dv32, float* dz, void* ret_ws, bool f32out, cudaStream_t st)
 {
     const int BH = p.B * p.H;
-    CUtensorMap tk, tv, tq, tdo;
+    CUtensorMap tk, tv, tq, tdo, tdk, tdv;
     if (!make_map(&tk, k, BH, p.T, p.d, 128) || !make_map(&tv, v, BH, p.T, p.d, 128) ||
-        !make_map(&tq, q, BH, p.T, p.d, 64) || !make_map(&tdo, dO, BH, p.T, p.d, 64))
+        !make_map(&tq, q, BH, p.T, p.d, 64) || !make_map(&tdo, dO, BH, p.T, p.d, 64) ||
+        !make_map(&tdk, dk, BH, p.T, p.d, 32) || !make_map(&tdv, dv, BH, p.T, p.d, 32))
         return LTE_ERR_CUDA;
     const size_t n = (size_t)BH * (p.R > 0 ? p.R : 1);
     float* dk_ret = (float*)ret_ws;
@@ -768,7 +797,7 @@ int launch_bwd_dkv_tc(const Params& p, const void* q, const void* k, const void*
             attr_done = true;                                                                                      \
         }                                                                                                          \
         launch_pdl(bwd_dkv_tc_kernel<D, F>, grid, dim3(NTHREADS), SmemK<D>::BYTES, st,                              \
-            tk, tv, tq, tdo, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, lse, delta, idx, cnt,               \
+            tk, tv, tq, tdo, tdk, tdv, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, lse, delta, idx, cnt,     \
             (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, dk32, dv32, dz, dk_ret, dv_ret, dr_ret, n_wt, p.T, p.W, p.R,   \
             p.scale);                                                                                              \
     } while (0)
