@@ -48,7 +48,7 @@ template <int D> struct SmemQ {                                // dq kernel
 template <int D>
 __global__ void __launch_bounds__(NTHREADS, D == 64 ? 2 : 1)
 bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmDO,
-                 const __grid_constant__ CUtensorMap tmO,
+                 const __grid_constant__ CUtensorMap tmO, const __grid_constant__ CUtensorMap tmDQ,
                  const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                  const __nv_bfloat16* __restrict__ kg, const __nv_bfloat16* __restrict__ vg,
                  const __nv_bfloat16* __restrict__ og, const __nv_bfloat16* __restrict__ dog,
@@ -336,22 +336,51 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         bwait(bar_pv, (n_tiles - 1) & 1, 5);
         tc_fence_after();
         // ---- epilogue: dQ (the softmax scale is already folded into dS) ------------------------------------
-        __nv_bfloat16* qrow = dq + ((size_t)bh * Tlen + i) * D;
+        if (D == 64) {
+            // the rows go into the (now idle) dS buffer in the swizzled layout and leave as one tile store per warp
 #pragma unroll
-        for (int cb = 0; cb < D / 32; ++cb) {
-            uint32_t q4[32];
-            tmem_ld32(tmem + lane_base + DQ_COL + cb * 32, q4);
-            tmem_wait_ld();
-            if (i < Tlen) {
+            for (int cb = 0; cb < 2; ++cb) {
+                uint32_t q4[32];
+                tmem_ld32(tmem + lane_base + DQ_COL + cb * 32, q4);
+                tmem_wait_ld();
 #pragma unroll
-                for (int c = 0; c < 32; c += 8) {
+                for (int g = 0; g < 4; ++g) {
                     uint32_t w4[4];
 #pragma unroll
                     for (int u = 0; u < 4; ++u) {
-                        __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(q4[c + 2 * u]), __uint_as_float(q4[c + 2 * u + 1]));
+                        __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(q4[g * 8 + 2 * u]), __uint_as_float(q4[g * 8 + 2 * u + 1]));
                         w4[u] = *reinterpret_cast<uint32_t*>(&h);
                     }
-                    *reinterpret_cast<uint4*>(qrow + cb * 32 + c) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+                    const int ch = cb * 4 + g;
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sDS + tid * 128 + ((ch ^ (tid & 7)) << 4)),
+                                 "r"(w4[0]), "r"(w4[1]), "r"(w4[2]), "r"(w4[3]) : "memory");
+                }
+            }
+            fence_proxy_async();
+            __syncwarp();
+            if (lane == 0 && i0 + warp * 32 < Tlen) {
+                tma_store_3d(&tmDQ, sDS + warp * 4096, 0, i0 + warp * 32, bh);
+                bulk_commit();
+                bulk_wait_read0();                             // the buffer is released with the CTA
+            }
+        } else {
+            __nv_bfloat16* qrow = dq + ((size_t)bh * Tlen + i) * D;
+#pragma unroll
+            for (int cb = 0; cb < D / 32; ++cb) {
+                uint32_t q4[32];
+                tmem_ld32(tmem + lane_base + DQ_COL + cb * 32, q4);
+                tmem_wait_ld();
+                if (i < Tlen) {
+#pragma unroll
+                    for (int c = 0; c < 32; c += 8) {
+                        uint32_t w4[4];
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(q4[c + 2 * u]), __uint_as_float(q4[c + 2 * u + 1]));
+                            w4[u] = *reinterpret_cast<uint32_t*>(&h);
+                        }
+                        *reinterpret_cast<uint4*>(qrow + cb * 32 + c) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+                    }
                 }
             }
         }
@@ -743,8 +772,9 @@ int launch_bwd_dq_tc(const Params& p, const void* q, const void* k, const void* 
                      const void* dO, const int32_t* idx, const int32_t* cnt, void* dq, float* delta, cudaStream_t st)
 {
     const int BH = p.B * p.H;
-    CUtensorMap tq, tdo, to, tk, tv;
+    CUtensorMap tq, tdo, to, tdq, tk, tv;
     if (!make_map(&tq, q, BH, p.T, p.d, BM) || !make_map(&tdo, dO, BH, p.T, p.d, BM) || !make_map(&to, o, BH, p.T, p.d, BM) ||
+        !make_map(&tdq, dq, BH, p.T, p.d, 32) ||
         !make_map(&tk, k, BH, p.T, p.d, BN) || !make_map(&tv, v, BH, p.T, p.d, BN))
         return LTE_ERR_CUDA;
     dim3 grid((p.T + BM - 1) / BM, BH);
@@ -757,7 +787,7 @@ int launch_bwd_dq_tc(const Params& p, const void* q, const void* k, const void* 
             attr_done = true;                                                                                      \
         }                                                                                                          \
         launch_pdl(bwd_dq_tc_kernel<D>, grid, dim3(NTHREADS), SmemQ<D>::BYTES, st,                            \
-            tq, tdo, to, tk, tv, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (const __nv_bfloat16*)o,        \
+            tq, tdo, to, tdq, tk, tv, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (const __nv_bfloat16*)o,        \
             (const __nv_bfloat16*)dO, lse, idx, cnt, (__nv_bfloat16*)dq, delta, p.T, p.W, p.R, p.scale);           \
     } while (0)
     if (p.d == 64) LTE_GO(64); else if (p.d == 128) LTE_GO(128); else return LTE_ERR_UNSUPPORTED;
