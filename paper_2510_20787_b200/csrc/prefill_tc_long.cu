@@ -55,7 +55,7 @@ template <int D> struct Smem {
 template <int D>
 __global__ void __launch_bounds__(NTHREADS, 2)
 prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                  const __grid_constant__ CUtensorMap tmV, const __nv_bfloat16* __restrict__ kg,
+                  const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO, const __nv_bfloat16* __restrict__ kg,
                   const __nv_bfloat16* __restrict__ vg, const int32_t* __restrict__ idx,
                   const int32_t* __restrict__ cnt, __nv_bfloat16* __restrict__ o, float* __restrict__ lse, int Tlen,
                   int W, int R, float scale)
@@ -433,25 +433,35 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             l_run = __uint_as_float(q4[0]);
         }
         const float inv = 1.f / l_run;
-        __nv_bfloat16* orow = o + ((size_t)bh * Tlen + i) * D;
+        // the normalised rows go into the Q tile's buffer (idle: every product of the CTA has completed) in the swizzled
+        // layout and leave as one tile store per warp and 64 columns (rows past the end are clipped by the tensor map;
+        // a 256-byte store per thread kept the load/store unit busy for thousands of cycles)
 #pragma unroll
         for (int cb = 0; cb < D / 32; ++cb) {
             uint32_t q4[32];
             tmem_ld32(tmem + lane_base + O_COL + cb * 32, q4);
             tmem_wait_ld();
-            if (i < Tlen) {
 #pragma unroll
-                for (int c = 0; c < 32; c += 8) {
-                    uint32_t w4[4];
+            for (int g = 0; g < 4; ++g) {
+                uint32_t w4[4];
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(q4[c + 2 * u]) * inv,
-                                                                 __uint_as_float(q4[c + 2 * u + 1]) * inv);
-                        w4[u] = *reinterpret_cast<uint32_t*>(&h);
-                    }
-                    *reinterpret_cast<uint4*>(orow + cb * 32 + c) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+                for (int u = 0; u < 4; ++u) {
+                    __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(q4[g * 8 + 2 * u]) * inv,
+                                                             __uint_as_float(q4[g * 8 + 2 * u + 1]) * inv);
+                    w4[u] = *reinterpret_cast<uint32_t*>(&h);
                 }
+                const int ch = (cb & 1) * 4 + g;               // 16-byte chunk within the 64-column sub-tile cb >> 1
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sQ + (cb >> 1) * 16384 + tid * 128 + ((ch ^ (tid & 7)) << 4)),
+                             "r"(w4[0]), "r"(w4[1]), "r"(w4[2]), "r"(w4[3]) : "memory");
             }
+        }
+        fence_proxy_async();
+        __syncwarp();
+        if (lane == 0 && i0 + warp * 32 < Tlen) {
+#pragma unroll
+            for (int sb = 0; sb < SUB; ++sb) tma_store_3d(&tmO, sQ + sb * 16384 + warp * 4096, sb * 64, i0 + warp * 32, bh);
+            bulk_commit();
+            bulk_wait_read0();                                 // the buffer is released with the CTA
         }
         if (i < Tlen) lse[(size_t)bh * Tlen + i] = m_run * 0.6931471805599453f + logf(l_run);
     }
@@ -464,9 +474,10 @@ template <int D>
 int run(const Params& p, const void* q, const void* k, const void* v, const int32_t* idx, const int32_t* cnt, void* o,
         float* lse, cudaStream_t st)
 {
-    CUtensorMap tq, tk, tv;
+    CUtensorMap tq, tk, tv, to;
     const int BH = p.B * p.H;
-    if (!make_map(&tq, q, BH, p.T, D, BM) || !make_map(&tk, k, BH, p.T, D, BN) || !make_map(&tv, v, BH, p.T, D, BN))
+    if (!make_map(&tq, q, BH, p.T, D, BM) || !make_map(&tk, k, BH, p.T, D, BN) || !make_map(&tv, v, BH, p.T, D, BN) ||
+        !make_map(&to, o, BH, p.T, D, 32))
         return LTE_ERR_CUDA;
     static bool attr_done = false;
     if (!attr_done) {
@@ -476,7 +487,7 @@ int run(const Params& p, const void* q, const void* k, const void* v, const int3
         attr_done = true;
     }
     dim3 grid((p.T + BM - 1) / BM, BH);
-    return cuda_status(launch_pdl(prefill_long_kernel<D>, grid, dim3(NTHREADS), Smem<D>::BYTES, st, tq, tk, tv, (const __nv_bfloat16*)k,
+    return cuda_status(launch_pdl(prefill_long_kernel<D>, grid, dim3(NTHREADS), Smem<D>::BYTES, st, tq, tk, tv, to, (const __nv_bfloat16*)k,
                                                                  (const __nv_bfloat16*)v, idx, cnt, (__nv_bfloat16*)o,
                                                                  lse, p.T, p.W, p.R, p.scale));
 }
