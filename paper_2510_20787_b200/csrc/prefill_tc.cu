@@ -191,6 +191,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         }
     } else if (warp == 4) {
         // ================================= MMA warp (lane 0 issues) =========================================
+        // The whole warp walks the loop and waits on the barriers; only the tcgen05 instructions are guarded by the lane
+        // test.  Descriptors and addresses are then computed in convergent code (the compiler can keep them in uniform
+        // registers), which roughly halves the issue cost of an MMA compared with a loop run by one lane alone.
         constexpr uint32_t IDESC_S = instr_desc(BM, BN, false);
         constexpr uint32_t IDESC_O = S::ONES ? instr_desc(BM, D + 16, true) : instr_desc(BM, D, true);
         // descriptor words: lo = (address >> 4) | LBO field, hi = SBO field | version | swizzle mode
@@ -221,24 +224,25 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 tc_fence_after();
                 const uint32_t kb = k_lo + ks * (S::KVTILE >> 4);
                 const uint32_t dcol = tmem + (gg & 1) * BN;
-#pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk)
-                    umma(dcol, desc64(q_lo + (kk >> 2) * 1024 + (kk & 3) * 2, HI), desc64(kb + (kk >> 2) * 512 + (kk & 3) * 2, HI),
-                         IDESC_S, kk > 0);
-                umma_commit(bar_s0 + 8 * (gg & 1));
-                umma_commit(bar_kf0 + 8 * ks);             // the K stage is free once this S has completed
                 ++ts;
-                if (ts == n_tiles) umma_commit(bar_qf);    // and so is Q after the item's last S
+                if (lane == 0) {
+#pragma unroll
+                    for (int kk = 0; kk < D / 16; ++kk)
+                        umma(dcol, desc64(q_lo + (kk >> 2) * 1024 + (kk & 3) * 2, HI), desc64(kb + (kk >> 2) * 512 + (kk & 3) * 2, HI),
+                             IDESC_S, kk > 0);
+                    umma_commit(bar_s0 + 8 * (gg & 1));
+                    umma_commit(bar_kf0 + 8 * ks);             // the K stage is free once this S has completed
+                    if (ts == n_tiles) umma_commit(bar_qf);    // and so is Q after the item's last S
+                }
+                __syncwarp();
             };
 
-            if (lane == 0) {
-                mbar_wait(bar_q, it & 1, 1);
-                mma_s();                                       // tile 0 is always a window tile
-                if (n_tiles > 1) mma_s();
-            }
+            mbar_wait(bar_q, it & 1, 1);
+            mma_s();                                           // tile 0 is always a window tile
+            if (n_tiles > 1) mma_s();
             // the next item's tile count, fetched while the softmax of this item's first tile runs
             n_tiles_next = item_tiles(item + gridDim.x);
-            if (lane == 0) {
+            {
                 for (int t = 0; t < n_tiles; ++t) {
                     const uint32_t gg = g + t, vs = gg % VST;
                     need_g(gg);
@@ -250,11 +254,14 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     if (t == 0 && it > 0) mbar_wait(bar_of, (it - 1) & 1, 13);   // the previous item's O has been read out
                     mbar_wait(bar_p, gg & 1, 7);
                     tc_fence_after();
+                    if (lane == 0) {
 #pragma unroll
-                    for (int kk = 0; kk < BN / 16; ++kk)
-                        umma_ts(tmem + O_COL, tmem + (gg & 1) * BN + kk * 8, desc64(vb + kk * 128, HI), IDESC_O, (t > 0 || kk > 0) ? 1u : 0u);
-                    umma_commit(bar_pv);
-                    umma_commit(bar_vf0 + 8 * vs);             // the V stage is free once PV has completed
+                        for (int kk = 0; kk < BN / 16; ++kk)
+                            umma_ts(tmem + O_COL, tmem + (gg & 1) * BN + kk * 8, desc64(vb + kk * 128, HI), IDESC_O, (t > 0 || kk > 0) ? 1u : 0u);
+                        umma_commit(bar_pv);
+                        umma_commit(bar_vf0 + 8 * vs);         // the V stage is free once PV has completed
+                    }
+                    __syncwarp();
                     // S two tiles ahead, into the S buffer the softmax has just released
                     if (ts < n_tiles) mma_s();
                 }
