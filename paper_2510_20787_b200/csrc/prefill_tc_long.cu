@@ -169,8 +169,10 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     vs = vs + 1 == VST ? 0 : vs + 1;
                 }
             }
-        } else if (warp == 4 && lane == 0) {
-            // ---- MMA lane: nothing but barrier waits and tcgen05 issue; stage indices and parities roll
+        } else if (warp == 4) {
+            // ---- MMA warp: nothing but barrier waits and tcgen05 issue; stage indices and parities roll.  The whole warp
+            //      walks the loop and waits; only the tcgen05 instructions are guarded by the lane test, so that addresses
+            //      and descriptors are computed in convergent code (cheaper to issue than from a loop run by one lane).
             constexpr uint32_t IDESC_S = instr_desc(BM, BN, false);
             constexpr uint32_t IDESC_O = S::ONES ? instr_desc(BM, D + 16, true) : instr_desc(BM, D, true);
             // descriptor words: lo = (address >> 4) | LBO field, hi = SBO field | version | swizzle mode
@@ -196,12 +198,15 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 tc_fence_after();
                 const uint32_t kb = k_lo + (uint32_t)ks * (S::KVTILE >> 4);
                 const uint32_t dcol = tmem + (ts & 1) * BN;
+                if (lane == 0) {
 #pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk)
-                    umma(dcol, desc64(q_lo + (kk >> 2) * 1024 + (kk & 3) * 2, HI), desc64(kb + (kk >> 2) * 512 + (kk & 3) * 2, HI),
-                         IDESC_S, kk > 0);
-                umma_commit(bar_s0 + 8 * (ts & 1));
-                umma_commit(bar_kf0 + 8 * ks);                 // the K stage is free once S(ts) has completed
+                    for (int kk = 0; kk < D / 16; ++kk)
+                        umma(dcol, desc64(q_lo + (kk >> 2) * 1024 + (kk & 3) * 2, HI), desc64(kb + (kk >> 2) * 512 + (kk & 3) * 2, HI),
+                             IDESC_S, kk > 0);
+                    umma_commit(bar_s0 + 8 * (ts & 1));
+                    umma_commit(bar_kf0 + 8 * ks);             // the K stage is free once S(ts) has completed
+                }
+                __syncwarp();
                 ++ts;
                 ks = ks + 1 == KST ? 0 : ks + 1;
             };
@@ -221,11 +226,14 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 for (int st = 1; st < VST; ++st) vb = vs == st ? v_desc[st] : vb;
                 mbar_wait(bar_p, t & 1, 7);
                 tc_fence_after();
+                if (lane == 0) {
 #pragma unroll
-                for (int kk = 0; kk < BN / 16; ++kk)
-                    umma_ts(tmem + O_COL, tmem + (t & 1) * BN + kk * 8, desc64(vb + kk * 128, HI), IDESC_O, (t > 0 || kk > 0) ? 1u : 0u);
-                umma_commit(bar_pv);
-                umma_commit(bar_vf0 + 8 * vs);                 // the V stage is free once PV(t) has completed
+                    for (int kk = 0; kk < BN / 16; ++kk)
+                        umma_ts(tmem + O_COL, tmem + (t & 1) * BN + kk * 8, desc64(vb + kk * 128, HI), IDESC_O, (t > 0 || kk > 0) ? 1u : 0u);
+                    umma_commit(bar_pv);
+                    umma_commit(bar_vf0 + 8 * vs);             // the V stage is free once PV(t) has completed
+                }
+                __syncwarp();
                 vs = vs + 1 == VST ? 0 : vs + 1;
                 // S(t+2) into the S buffer softmax(t) has just released
                 if (ts < n_tiles) mma_s();
