@@ -107,7 +107,10 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             }
         }
         const int n_tiles = n_win + (nv_max + BN - 1) / BN;
-        if (lane == 0) {
+        // The whole warp walks the loop and waits on the barriers; only the TMA / tcgen05 instructions are guarded by the
+        // lane test, so that addresses and descriptors are computed in convergent code (cheaper to issue).
+        const bool leader = lane == 0;
+        {
             constexpr uint32_t IDESC_S = instr_desc(BM, BN, false);
             constexpr uint32_t IDESC_Q = instr_desc(BM, D, true);
             const uint32_t q_lo = desc_lo(sQ, 16), do_lo = desc_lo(sDO, 16), k_lo = desc_lo(sK, 16), v_lo = desc_lo(sV, 16);
@@ -117,10 +120,12 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                 const int st = t % NST;
                 const uint32_t dst = (is_v ? sV : sK) + st * S::KVTILE;
                 const uint32_t bar = (is_v ? bar_v0 : bar_k0) + 8 * st;
-                mbar_expect_tx(bar, S::KVTILE);
                 const int y = j_start + t * BN;
+                if (leader) {
+                    mbar_expect_tx(bar, S::KVTILE);
 #pragma unroll
-                for (int sb = 0; sb < SUB; ++sb) tma_load_3d(dst + sb * 8192, is_v ? &tmV : &tmK, sb * 64, y, bh, bar);
+                    for (int sb = 0; sb < SUB; ++sb) tma_load_3d(dst + sb * 8192, is_v ? &tmV : &tmK, sb * 64, y, bh, bar);
+                }
             };
             auto need_g = [&](uint32_t phase) {
                 while (g_waited <= phase) { bwait(bar_g0 + 8 * (g_waited & 1), (g_waited >> 1) & 1, 10); ++g_waited; }
@@ -134,25 +139,30 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             };
             auto mma_s_dp = [&](int t) {
                 const uint32_t so = (uint32_t)(t % NST) * (S::KVTILE >> 4);
+                if (leader) {
 #pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk)
-                    umma(tmem, desc64(q_lo + (kk >> 2) * 1024 + (kk & 3) * 2, kDescHi),
-                         desc64(k_lo + so + (kk >> 2) * 512 + (kk & 3) * 2, kDescHi), IDESC_S, kk > 0);
+                    for (int kk = 0; kk < D / 16; ++kk)
+                        umma(tmem, desc64(q_lo + (kk >> 2) * 1024 + (kk & 3) * 2, kDescHi),
+                             desc64(k_lo + so + (kk >> 2) * 512 + (kk & 3) * 2, kDescHi), IDESC_S, kk > 0);
 #pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk)
-                    umma(tmem + DP_COL, desc64(do_lo + (kk >> 2) * 1024 + (kk & 3) * 2, kDescHi),
-                         desc64(v_lo + so + (kk >> 2) * 512 + (kk & 3) * 2, kDescHi), IDESC_S, kk > 0);
-                umma_commit(bar_s);
+                    for (int kk = 0; kk < D / 16; ++kk)
+                        umma(tmem + DP_COL, desc64(do_lo + (kk >> 2) * 1024 + (kk & 3) * 2, kDescHi),
+                             desc64(v_lo + so + (kk >> 2) * 512 + (kk & 3) * 2, kDescHi), IDESC_S, kk > 0);
+                    umma_commit(bar_s);
+                }
+                __syncwarp();
             };
 
             // d = 64: the O tile rides along into the (still unused) dS buffer, for delta = <dO, O>
-            mbar_expect_tx(bar_q, (D == 64 ? 3 : 2) * S::QTILE);
+            if (leader) {
+                mbar_expect_tx(bar_q, (D == 64 ? 3 : 2) * S::QTILE);
 #pragma unroll
-            for (int sb = 0; sb < SUB; ++sb) {
-                tma_load_3d(sQ + sb * 16384, &tmQ, sb * 64, i0, bh, bar_q);
-                tma_load_3d(sDO + sb * 16384, &tmDO, sb * 64, i0, bh, bar_q);
+                for (int sb = 0; sb < SUB; ++sb) {
+                    tma_load_3d(sQ + sb * 16384, &tmQ, sb * 64, i0, bh, bar_q);
+                    tma_load_3d(sDO + sb * 16384, &tmDO, sb * 64, i0, bh, bar_q);
+                }
+                if (D == 64) tma_load_3d(sDS, &tmO, 0, i0, bh, bar_q);
             }
-            if (D == 64) tma_load_3d(sDS, &tmO, 0, i0, bh, bar_q);
             for (int t = 0; t < NST && t < n_win; ++t) { tma_kv(t, false); tma_kv(t, true); }
             bwait(bar_q, 0, 1);                                // (tile 0 is always a window tile: no gather to wait for)
             wait_kv(0);
@@ -163,11 +173,14 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                 tc_fence_after();
                 {
                     const uint32_t kb = kmn_lo + (uint32_t)(t % NST) * (S::KVTILE >> 4);
+                    if (leader) {
 #pragma unroll
-                    for (int kk = 0; kk < BN / 16; ++kk)
-                        umma(tmem + DQ_COL, desc64(ds_lo + kk * 2, kDescHi), desc64(kb + kk * 128, kDescHi), IDESC_Q,
-                             (t > 0 || kk > 0) ? 1u : 0u);
-                    umma_commit(bar_pv);
+                        for (int kk = 0; kk < BN / 16; ++kk)
+                            umma(tmem + DQ_COL, desc64(ds_lo + kk * 2, kDescHi), desc64(kb + kk * 128, kDescHi), IDESC_Q,
+                                 (t > 0 || kk > 0) ? 1u : 0u);
+                        umma_commit(bar_pv);
+                    }
+                    __syncwarp();
                 }
                 if (t + 1 < n_tiles) {
                     need_g(t + 1);
