@@ -484,7 +484,9 @@ bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     const uint32_t tmem = *tmem_slot_gen;
 
     if (warp == 4) {
-        if (lane == 0 && n_blk > 0) {
+        // (the whole warp walks the loop and waits; only the TMA / tcgen05 instructions are guarded by the lane test)
+        const bool leader = lane == 0;
+        if (n_blk > 0) {
             constexpr uint32_t IDESC_S = instr_desc(128, 64, false);
             constexpr uint32_t IDESC_O = instr_desc(128, D, true);
             const uint32_t k_lo = desc_lo(sK, 16), v_lo = desc_lo(sV, 16), q_lo = desc_lo(sQ, 16), do_lo = desc_lo(sDO, 16);
@@ -494,12 +496,14 @@ bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
             auto tma_blk = [&](int t) {
                 const int st = t % NST;
                 const uint32_t bar = bar_q0 + 8 * st;
-                mbar_expect_tx(bar, 2 * S::QBLK);
                 const int y = ib_start + t * 64;
+                if (leader) {
+                    mbar_expect_tx(bar, 2 * S::QBLK);
 #pragma unroll
-                for (int sb = 0; sb < SUB; ++sb) {
-                    tma_load_3d(sQ + st * S::QBLK + sb * 8192, &tmQ, sb * 64, y, bh, bar);
-                    tma_load_3d(sDO + st * S::QBLK + sb * 8192, &tmDO, sb * 64, y, bh, bar);
+                    for (int sb = 0; sb < SUB; ++sb) {
+                        tma_load_3d(sQ + st * S::QBLK + sb * 8192, &tmQ, sb * 64, y, bh, bar);
+                        tma_load_3d(sDO + st * S::QBLK + sb * 8192, &tmDO, sb * 64, y, bh, bar);
+                    }
                 }
             };
             auto wait_blk = [&](int t) {
@@ -508,17 +512,20 @@ bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
             };
             auto mma_s_dp = [&](int t) {
                 const uint32_t so = (uint32_t)(t % NST) * (S::QBLK >> 4);
+                if (leader) {
 #pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk)
-                    umma(tmem, desc64(k_lo + (kk >> 2) * 1024 + (kk & 3) * 2, kDescHi),
-                         desc64(q_lo + so + (kk >> 2) * 512 + (kk & 3) * 2, kDescHi), IDESC_S, kk > 0);
+                    for (int kk = 0; kk < D / 16; ++kk)
+                        umma(tmem, desc64(k_lo + (kk >> 2) * 1024 + (kk & 3) * 2, kDescHi),
+                             desc64(q_lo + so + (kk >> 2) * 512 + (kk & 3) * 2, kDescHi), IDESC_S, kk > 0);
 #pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk)
-                    umma(tmem + DP_COL, desc64(v_lo + (kk >> 2) * 1024 + (kk & 3) * 2, kDescHi),
-                         desc64(do_lo + so + (kk >> 2) * 512 + (kk & 3) * 2, kDescHi), IDESC_S, kk > 0);
-                umma_commit(bar_s);
+                    for (int kk = 0; kk < D / 16; ++kk)
+                        umma(tmem + DP_COL, desc64(v_lo + (kk >> 2) * 1024 + (kk & 3) * 2, kDescHi),
+                             desc64(do_lo + so + (kk >> 2) * 512 + (kk & 3) * 2, kDescHi), IDESC_S, kk > 0);
+                    umma_commit(bar_s);
+                }
+                __syncwarp();
             };
-            if (!is_ret) {
+            if (!is_ret && leader) {
                 mbar_expect_tx(bar_kv, 2 * S::KTILE);
 #pragma unroll
                 for (int sb = 0; sb < SUB; ++sb) {
@@ -536,15 +543,18 @@ bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                 tc_fence_after();
                 {
                     const uint32_t so = (uint32_t)(t % NST) * (S::QBLK >> 4);
+                    if (leader) {
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk)
-                        umma(tmem + DV_COL, desc64(pt_lo + kk * 2, kDescHi), desc64(domn_lo + so + kk * 128, kDescHi), IDESC_O,
-                             (t > 0 || kk > 0) ? 1u : 0u);
+                        for (int kk = 0; kk < 4; ++kk)
+                            umma(tmem + DV_COL, desc64(pt_lo + kk * 2, kDescHi), desc64(domn_lo + so + kk * 128, kDescHi), IDESC_O,
+                                 (t > 0 || kk > 0) ? 1u : 0u);
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk)
-                        umma(tmem + DK_COL, desc64(dst_lo + kk * 2, kDescHi), desc64(qmn_lo + so + kk * 128, kDescHi), IDESC_O,
-                             (t > 0 || kk > 0) ? 1u : 0u);
-                    umma_commit(bar_pv);
+                        for (int kk = 0; kk < 4; ++kk)
+                            umma(tmem + DK_COL, desc64(dst_lo + kk * 2, kDescHi), desc64(qmn_lo + so + kk * 128, kDescHi), IDESC_O,
+                                 (t > 0 || kk > 0) ? 1u : 0u);
+                        umma_commit(bar_pv);
+                    }
+                    __syncwarp();
                 }
                 if (t + 1 < n_blk) { wait_blk(t + 1); mma_s_dp(t + 1); }
                 // the accumulations of block t-1 have completed (the key threads waited for them before producing
