@@ -82,6 +82,15 @@ def test_config5_forward():
     _assert_close(cfg, _pipeline(cfg, seed=0, batch=[0, 7]))
 
 
+def test_persistent_schedule_ragged_many_items():
+    """More work items than resident CTAs (each CTA walks several items), a last query tile that is ragged, lists
+    longer than the prefetched 128 entries and sink tokens: covers the item-to-item hand-over of the persistent
+    d = 64 kernel (Q buffer, accumulator, stage ring, prefetched list) on a shape unlike the benchmark's."""
+    cfg = synth.Config("ragged", "bf16", 3, 8, 64, 2075, 96, 200, 7, 0.1, sink=3)
+    assert 3 * 8 * ((2075 + 127) // 128) > 2 * 148
+    _assert_close(cfg, _pipeline(cfg, seed=11))
+
+
 def test_zero_query_pins_set_sizes_on_gpu():
     cfg = synth.Config("q0", "bf16", 1, 2, 64, 900, 100, 60, 7, 0.1)
     x = synth.make(cfg, 2)
