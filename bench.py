@@ -351,7 +351,40 @@ def _extras_sections(torch, lte, synth, pk, flush, args, which):
         _extra_c4(out, torch, lte, synth, pk, flush, n5)
     if "P" in which:
         _extra_p(out, torch, lte, synth, pk, flush, n5)
+    if "S" in which:
+        _extra_s(out, torch, lte, synth, pk, flush, n5)
     return out
+
+
+def _extra_s(out, torch, lte, synth, pk, flush, n5):
+    """The paper's three-layer scorer (kernel 3, dilation 2, channels 2d -> d -> d/2 -> d/4 -> 1) at the C2 shape.
+    fp32 on the ordinary ALUs; the bound is their FMA rate: 148 SMs x 128 lanes x 2 FLOP x the SM clock."""
+    cfg = synth.CONFIGS["C2"]
+    x = device_inputs(cfg, 7, torch)
+    d, H = cfg.d, cfg.H
+    g = torch.Generator(device="cuda"); g.manual_seed(70)
+    ch = [2 * d, d, d // 2, d // 4]
+    wl = [torch.randn((H, ch[l + 1], 3, ch[l]), generator=g, device="cuda") * (1.5 / (3 * ch[l]) ** 0.5) for l in range(3)]
+    wout = torch.randn((H, ch[3]), generator=g, device="cuda") * (2.0 / ch[3] ** 0.5)
+    c = lte.conv_stack(wl, wout)
+    s = lte.shape(cfg.B, cfg.H, cfg.T, cfg.d, cfg.W, cfg.R, lte.BF16)
+    z = torch.empty((cfg.B, cfg.H, cfg.T), dtype=torch.float32, device="cuda")
+
+    def f():
+        lte.lte_scores(s, c, x["k"], x["v"], z=z)
+
+    ms, _ = timed(torch, f, n5, 3, flush)
+    t = mid3(ms) * 1e-3
+    macs = 3 * (ch[0] * ch[1] + ch[1] * ch[2] + ch[2] * ch[3]) + ch[3]
+    fl = 2.0 * macs * cfg.B * cfg.H * cfg.T
+    props = torch.cuda.get_device_properties(0)
+    alu_peak = props.multi_processor_count * 128 * 2 * 1.965e9
+    out["S_scorer_stack"] = {"workload": "C2 shape, 3 conv layers k=3 dil=2, channels 128 -> 64 -> 32 -> 16 -> 1",
+                             "scores_ms": t * 1e3, "tokens_per_s": cfg.B * cfg.T / t, "algorithmic_tflops": fl / t / 1e12,
+                             "roofline": {"bound": "alu", "achieved": fl / t / 1e12, "peak": alu_peak / 1e12, "unit": "TFLOP/s",
+                                          "frac": fl / t / alu_peak, "peak_source": "SMs x 128 fp32 lanes x 2 x 1.965 GHz"},
+                             "fraction_kept": float((z[:, :, : cfg.T - 6] > 0).float().mean())}
+    del x, z
 
 
 def _extra_p(out, torch, lte, synth, pk, flush, n5):
@@ -555,7 +588,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="lte", choices=["lte", "reference"])
     ap.add_argument("--no-extras", action="store_true")
-    ap.add_argument("--section", default=None, choices=["C3", "C4", "C5", "P"],
+    ap.add_argument("--section", default=None, choices=["C3", "C4", "C5", "P", "S"],
                     help="time only this extra section (long prefill / decode / forward+backward) after the main loop")
     ap.add_argument("--skip-main", action="store_true", help="with --section: skip the main C2 loop")
     args = ap.parse_args()

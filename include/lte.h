@@ -48,12 +48,22 @@ typedef struct lte_shape {
 } lte_shape;
 
 typedef struct lte_conv {
-    int32_t n_layers;              /* 1: the single grouped conv layer 2d -> 1 per head                    */
+    int32_t n_layers;              /* 1: the single grouped conv layer 2d -> 1 per head; 3: the paper's stack (below) */
     int32_t kernel;                /* K taps, odd, centred (half past, self, half future)                   */
     int32_t dilation;              /* 1                                                                     */
     const float* w;                /* device, [H, K, 2d] fp32; channels [0,d) weigh k, [d,2d) weigh v       */
     const float* bias;             /* device, [H] fp32, or NULL for zero                                    */
 } lte_conv;
+/*
+ * n_layers = 3 (accepted by lte_scores only; d = 32 or 64): the scorer of Section 3.1.1 with the hyper-parameters of
+ * Appendix A: three grouped conv layers of kernel = 3, dilation = 2, channels 2d -> d -> d/2 -> d/4, Swish after each,
+ * then a per-head linear map to the logit; receptive field 13, the logit of token j is the output at time j + 6
+ * (z_j = -inf for j > T-1-6).  Every layer's input is zero at negative times, hidden activations included.
+ *   w    = wl0 [H, d, 3, 2d] | wl1 [H, d/2, 3, d] | wl2 [H, d/4, 3, d/2] | wout [H, d/4]    (one fp32 buffer, 16-byte aligned;
+ *          wl[o][tau][c] multiplies channel c of the input at time t - (2 - tau) * 2)
+ *   bias = bl0 [H, d] | bl1 [H, d/2] | bl2 [H, d/4] | bout [H], or NULL for zero.
+ * The other entry points (decode, backward, cache_init) take the single layer only and answer LTE_ERR_UNSUPPORTED.
+ */
 
 typedef enum lte_op {
     LTE_OP_SCORES = 0, LTE_OP_SELECT = 1, LTE_OP_PREFILL = 2, LTE_OP_DECODE = 3, LTE_OP_BWD = 4

@@ -109,6 +109,17 @@ int lte_scores(const lte_shape* s, const lte_conv* c, const void* k, const void*
 {
     (void)ws; (void)ws_bytes;
     int e = check_shape(s, true); if (e) return e;
+    if (c && c->w && c->n_layers == 3) {
+        // the paper's stack: kernel 3, dilation 2, channels 2d -> d -> d/2 -> d/4 -> 1 (packed parameters, see lte.h)
+        if (c->kernel != 3 || c->dilation != 2) return LTE_ERR_UNSUPPORTED;
+        if (s->d != 32 && s->d != 64) return LTE_ERR_UNSUPPORTED;
+        if (s->W < 7) return LTE_ERR_INVALID_ARG;            // tokens must be scored before they leave the window
+        if (!k || !v || !z || !aligned16(k) || !aligned16(v) || !aligned16(c->w)) return LTE_ERR_INVALID_ARG;
+        e = check_arch(); if (e) return e;
+        Params p = make_params(s, c);
+        p.K = 13; p.half = 6;
+        return launch_scores_stack(p, k, v, z, r_or_null, (cudaStream_t)stream);
+    }
     e = check_conv(s, c); if (e) return e;
     if (!k || !v || !z || !aligned16(k) || !aligned16(v)) return LTE_ERR_INVALID_ARG;
     e = check_arch(); if (e) return e;

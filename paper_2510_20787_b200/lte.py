@@ -91,6 +91,24 @@ def conv(w, bias=None):
     return c
 
 
+def conv_stack(wl, wout, bl=None, bout=None):
+    """The paper's three-layer scorer for lte_scores: wl = [wl0 [H,d,3,2d], wl1 [H,d/2,3,d], wl2 [H,d/4,3,d/2]],
+    wout [H,d/4]; bl = three bias tensors [H,c] or None, bout [H] or None.  All CUDA fp32.  The tensors are packed
+    into the two buffers the C struct carries."""
+    assert len(wl) == 3 and all(t.is_cuda and t.dtype == torch.float32 for t in list(wl) + [wout])
+    w = torch.cat([t.contiguous().reshape(-1) for t in list(wl) + [wout]]).contiguous()
+    b = None
+    if bl is not None or bout is not None:
+        H = wout.shape[0]
+        parts = [(bl[i] if bl is not None and bl[i] is not None else torch.zeros((H, wl[i].shape[1]), device=w.device))
+                 for i in range(3)]
+        parts.append(bout if bout is not None else torch.zeros((H,), device=w.device))
+        b = torch.cat([t.to(torch.float32).contiguous().reshape(-1) for t in parts]).contiguous()
+    c = LteConv(3, 3, 2, w.data_ptr(), 0 if b is None else b.data_ptr())
+    c._keep = (w, b)
+    return c
+
+
 def _ptr(t, dtype=None):
     if t is None:
         return None

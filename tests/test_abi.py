@@ -56,8 +56,13 @@ def test_host_side_validation_rejects_bad_arguments():
     assert L.lte_scores(a(good), a(conv), fake + 4, fake, fake, None, None, 0, None) == -1      # misaligned
     even = lte.LteConv(1, 4, 1, 256, 0)
     assert L.lte_scores(a(good), a(even), fake, fake, fake, None, None, 0, None) == -1
-    deep = lte.LteConv(3, 3, 2, 256, 0)
-    assert L.lte_scores(a(good), a(deep), fake, fake, fake, None, None, 0, None) == -2
+    # stacks other than the paper's (3 layers, kernel 3, dilation 2, d = 32 or 64) are unsupported
+    for deep in (lte.LteConv(2, 3, 2, 256, 0), lte.LteConv(3, 5, 2, 256, 0), lte.LteConv(3, 3, 1, 256, 0)):
+        assert L.lte_scores(a(good), a(deep), fake, fake, fake, None, None, 0, None) == -2
+    wide = lte.shape(1, 2, 128, 128, 16, 8, lte.F32)
+    assert L.lte_scores(a(wide), a(lte.LteConv(3, 3, 2, 256, 0)), fake, fake, fake, None, None, 0, None) == -2
+    narrow = lte.shape(1, 2, 128, 32, 6, 8, lte.F32)          # window shorter than the stack's look-ahead + 1
+    assert L.lte_scores(a(narrow), a(lte.LteConv(3, 3, 2, 256, 0)), fake, fake, fake, None, None, 0, None) == -1
     bad_d = lte.shape(1, 2, 128, 48, 16, 8, lte.F32)
     assert L.lte_scores(a(bad_d), a(conv), fake, fake, fake, None, None, 0, None) == -2
     narrow = lte.shape(1, 2, 128, 32, 3, 8, lte.F32)
