@@ -188,8 +188,10 @@ __global__ void __launch_bounds__(NT + 64) scores_tc_kernel(const __grid_constan
             }
         }
     } else if (warp == 4) {
-        // ---- MMA lane ------------------------------------------------------------------------------------------------
-        if ((tid & 31) == 0) {
+        // ---- MMA warp: the whole warp walks the loop and waits; only the tcgen05 instructions are guarded by the lane test
+        //      (descriptors computed in convergent code are cheaper to issue than from a loop run by one lane alone)
+        {
+            const bool leader = (tid & 31) == 0;
             constexpr uint32_t IDESC = instr_desc(128, NB, false);
             const uint32_t b_lo = desc_lo(tile0 + C::OFF_B, 16), a_lo0 = desc_lo(tile0, 16);
             int ft = f_begin % n_all, n_heads = 0;
@@ -201,11 +203,14 @@ __global__ void __launch_bounds__(NT + 64) scores_tc_kernel(const __grid_constan
                 tc_fence_after();
                 const uint32_t a_lo = a_lo0 + (uint32_t)(i % NSTAGE) * (C::STAGE >> 4);
                 const uint32_t dcol = tmem + (i & 1) * C::ACC_COLS;
+                if (leader) {
 #pragma unroll
-                for (int kk = 0; kk < 2 * D / 16; ++kk)   // 2d input channels, 16 per instruction
-                    umma(dcol, desc64(a_lo + (kk >> 2) * 1024 + (kk & 3) * 2, kDescHi),
-                         desc64(b_lo + (kk >> 2) * (C::B_SLOT >> 4) + (kk & 3) * 2, kDescHi), IDESC, kk > 0);
-                umma_commit(bar_mma0 + 8 * (i & 1));
+                    for (int kk = 0; kk < 2 * D / 16; ++kk)   // 2d input channels, 16 per instruction
+                        umma(dcol, desc64(a_lo + (kk >> 2) * 1024 + (kk & 3) * 2, kDescHi),
+                             desc64(b_lo + (kk >> 2) * (C::B_SLOT >> 4) + (kk & 3) * 2, kDescHi), IDESC, kk > 0);
+                    umma_commit(bar_mma0 + 8 * (i & 1));
+                }
+                __syncwarp();
                 new_head = ++ft == n_all;
                 if (new_head) ft = 0;
             }
