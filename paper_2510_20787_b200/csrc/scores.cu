@@ -230,14 +230,27 @@ __global__ void __launch_bounds__(NT + 64) scores_tc_kernel(const __grid_constan
                 const int h = bh % H;
                 bh_bias = bias ? bias[h] : 0.f;
                 // B: row n = piece * K + t, columns = the 2d input channels (k part, then v part); zero rows above 3K
-                for (int e = tid; e < NB * 2 * D / 8; e += NT) {   // one 16-byte chunk (8 channels) of one row
-                    const int n = e / (2 * D / 8), c8 = e % (2 * D / 8);
-                    const int piece = n / K, t = n % K;
+                // (one 16-byte chunk = 8 channels of one row per step; all of a thread's weights are fetched before any is
+                // converted: the shared-memory stores below are compiler barriers and would serialise the load latencies)
+                constexpr int NCH = NB * 2 * D / 8 / NT;        // chunks per thread
+                static_assert(NB * 2 * D / 8 % NT == 0, "B chunks must divide evenly over the row threads");
+                float4 wf[NCH][2];
+#pragma unroll
+                for (int q = 0; q < NCH; ++q) {
+                    const int e = tid + q * NT, n = e / (2 * D / 8), c8 = e % (2 * D / 8);
+                    wf[q][0] = wf[q][1] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (n < 3 * K) {
+                        const float4* src = reinterpret_cast<const float4*>(w + ((size_t)h * K + n % K) * 2 * D + c8 * 8);
+                        wf[q][0] = src[0]; wf[q][1] = src[1];
+                    }
+                }
+#pragma unroll
+                for (int q = 0; q < NCH; ++q) {
+                    const int e = tid + q * NT, n = e / (2 * D / 8), c8 = e % (2 * D / 8);
+                    const int piece = n / K;
                     uint32_t pk[4] = {0u, 0u, 0u, 0u};
                     if (n < 3 * K) {
-                        const float4* src = reinterpret_cast<const float4*>(w + ((size_t)h * K + t) * 2 * D + c8 * 8);
-                        const float4 f0 = src[0], f1 = src[1];
-                        const float wv8[8] = {f0.x, f0.y, f0.z, f0.w, f1.x, f1.y, f1.z, f1.w};
+                        const float wv8[8] = {wf[q][0].x, wf[q][0].y, wf[q][0].z, wf[q][0].w, wf[q][1].x, wf[q][1].y, wf[q][1].z, wf[q][1].w};
 #pragma unroll
                         for (int u = 0; u < 4; ++u) {
                             float v2[2];
