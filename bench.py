@@ -416,11 +416,37 @@ def _extra_p(out, torch, lte, synth, pk, flush, n5):
     ms_a, _ = timed(torch, f_attn, n5, 3, flush)
     fl = attn_flops(idx, cnt, cfg.T, cfg.W, cfg.d, torch)
     t, ta = mid3(ms) * 1e-3, mid3(ms_a) * 1e-3
+    # decode from that prompt: 32 steps in a CUDA graph after 8 warm-up steps
+    cache = lte.lte_cache_init(s, c, x["k"], x["v"], z, idx, cnt)
+    n_dec = 40
+    g = torch.Generator(device="cuda"); g.manual_seed(61)
+    sc = cfg.d ** -0.25
+    qs, ks, vs = ((torch.randn((n_dec, cfg.B, cfg.H, cfg.d), generator=g, device="cuda") * f).to(torch.bfloat16)
+                  for f in (sc, sc, 1.0))
+    o1 = torch.empty((cfg.B, cfg.H, cfg.d), dtype=torch.bfloat16, device="cuda")
+    l1 = torch.empty((cfg.B, cfg.H), dtype=torch.float32, device="cuda")
+    for i in range(8):
+        lte.lte_attn_decode(s, c, cache, qs[i], ks[i], vs[i], o1=o1, lse1=l1)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        for i in range(8, n_dec):
+            lte.lte_attn_decode(s, c, cache, qs[i], ks[i], vs[i], o1=o1, lse1=l1)
+    reps = []
+    for _ in range(5):
+        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+        e0.record(); graph.replay(); e1.record()
+        torch.cuda.synchronize()
+        reps.append(e0.elapsed_time(e1) * 1e3 / (n_dec - 8))
+    dec_us = mid3(reps)
+    dec_bytes = (2 * (cfg.W + cfg.R) * cfg.d * 2 + cfg.R * 4 + 1024 + 16) * cfg.B * cfg.H
     out["P_paper_like"] = {"workload": "B=32 H=16 d=64 T=4096 W=768 R=512 sink=4 K=7, bias set for ~R/2 retained per head",
                            "step_ms": t * 1e3, "tokens_per_s": cfg.B * cfg.T / t, "attn_ms": ta * 1e3,
                            "attn_algorithmic_tflops": fl / ta / 1e12, "attn_tensor_frac": fl / ta / 1e12 / pk["bf16_tflops"],
-                           "mean_retained": float(cnt.float().mean()), "max_retained": int(cnt.max())}
-    del x, o, lse, z, z0
+                           "mean_retained": float(cnt.float().mean()), "max_retained": int(cnt.max()),
+                           "decode_us_per_step": dec_us, "decode_hbm_gbs": dec_bytes / dec_us / 1e3,
+                           "decode_hbm_frac": dec_bytes / dec_us / 1e3 / pk["hbm_gbs"]}
+    del x, o, lse, z, z0, cache
 
 
 def _extra_c3(out, torch, lte, synth, pk, flush, n5):
