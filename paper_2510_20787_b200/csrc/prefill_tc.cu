@@ -324,6 +324,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 nvis += __popc(bits & ((1u << (lim - lim0)) - 1u));
             }
             const int n_tiles = n_win + (nv_max + BN - 1) / BN;
+            const int nvis_first = __shfl_sync(0xffffffffu, nvis, 0), nvis_last = __shfl_sync(0xffffffffu, nvis, 31);
             prefetch_list(item + gridDim.x);
 
             // gather of one retained tile (t = its number within the item): 8 lanes per row copy its 16-byte chunks
@@ -390,10 +391,18 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     c_lo = 0;
                     c_hi = nvis - (t - n_win) * BN - 1;
                 }
-                // rows of a warp are consecutive and both bounds grow with the row: lane 0 / lane 31 give the warp's
-                // union range (columns any row sees) and intersection range (columns every row sees)
-                const int u_lo = __shfl_sync(0xffffffffu, c_lo, 0), u_hi = __shfl_sync(0xffffffffu, c_hi, 31);
-                const int n_lo = __shfl_sync(0xffffffffu, c_lo, 31), n_hi = __shfl_sync(0xffffffffu, c_hi, 0);
+                // rows of a warp are consecutive and both bounds grow with the row: the bounds of its first and last row
+                // give the warp's union range (columns any row sees) and intersection range (columns every row sees).
+                // They follow from the warp's first row alone (no shuffles on the per-tile path).
+                int u_lo, u_hi, n_lo, n_hi;
+                if (t < n_win) {
+                    const int jt0 = j_start + t * BN, ia = i - lane, ib = ia + 31;
+                    u_lo = max(ia - W + 1, 0) - jt0; n_lo = max(ib - W + 1, 0) - jt0;
+                    n_hi = ia - jt0; u_hi = ib - jt0;
+                } else {
+                    u_lo = n_lo = 0;
+                    n_hi = nvis_first - (t - n_win) * BN - 1; u_hi = nvis_last - (t - n_win) * BN - 1;
+                }
                 bool act[2], full[2];
                 uint32_t vm[2];                                // per-thread validity bits of a partial chunk
 #pragma unroll
