@@ -149,7 +149,7 @@ __global__ void __launch_bounds__(1024) select_reg_kernel(const float* __restric
                                                           int32_t* __restrict__ cnt, int32_t* __restrict__ ncand, int T,
                                                           int W, int R, int sink, float zthr)
 {
-    __shared__ uint32_t s_count[3];
+    __shared__ uint32_t s_part[2][32];
     __shared__ uint32_t s_wa[32], s_we[32];
     pdl_launch_dependents();
     pdl_wait();                                            // z comes from the previous kernel
@@ -163,18 +163,16 @@ __global__ void __launch_bounds__(1024) select_reg_kernel(const float* __restric
     uint32_t key[KPT];
 #pragma unroll
     for (int i = 0; i < KPT; ++i) key[i] = p0 + i < N ? key_of(zz, p0 + i, sink, zthr) : 0u;
-    if (tid < 3) s_count[tid] = 0;
-    __syncthreads();
-    // block-wide sum of a per-thread count.  Three counters rotate: the one reset after this call's barrier is used two
-    // calls later, so the reset is ordered before those additions by the barrier in between (one barrier per call).
+    // block-wide sum of a per-thread count, one barrier per call and no atomics: every warp leaves its sum in one of two
+    // alternating rows of partials, and after the barrier every warp adds the row up itself.  A row is rewritten two calls
+    // later, when every warp has passed the barrier of the call in between and so has finished reading it.
     int slot = 0;
     auto block_sum = [&](uint32_t c) -> uint32_t {
         c = __reduce_add_sync(0xffffffffu, c);
-        if (lane == 0 && c) atomicAdd(&s_count[slot], c);
+        if (lane == 0) s_part[slot][wid] = c;
         __syncthreads();
-        const uint32_t total = s_count[slot];
-        if (tid == 0) s_count[(slot + 2) % 3] = 0;
-        slot = (slot + 1) % 3;
+        const uint32_t total = __reduce_add_sync(0xffffffffu, lane < nwarp ? s_part[slot][lane] : 0u);
+        slot ^= 1;
         return total;
     };
     uint32_t c0 = 0;
