@@ -91,6 +91,19 @@ def test_persistent_schedule_ragged_many_items():
     _assert_close(cfg, _pipeline(cfg, seed=11))
 
 
+def test_random_shapes_many_items():
+    """Seeded random shapes with more work items than resident CTAs (d = 64: the persistent schedule; d = 128: one CTA
+    per tile), windows and budgets of every relation to the tile sizes, with and without sink tokens."""
+    rng = np.random.default_rng(77)
+    for n in range(6):
+        d = 64 if n % 3 else 128
+        T = int(rng.integers(1500, 4200)) if d == 64 else int(rng.integers(300, 1400))
+        cfg = synth.Config("rnd", "bf16", int(rng.integers(2, 5)), int(rng.integers(6, 13)), d, T,
+                           int(rng.integers(16, 400)), int(rng.integers(0, 520)), 7, 0.1, sink=int(rng.integers(0, 5)))
+        _assert_close(cfg, _pipeline(cfg, seed=100 + n))
+    assert lte.lte_device_status() == 0
+
+
 def test_zero_query_pins_set_sizes_on_gpu():
     cfg = synth.Config("q0", "bf16", 1, 2, 64, 900, 100, 60, 7, 0.1)
     x = synth.make(cfg, 2)
