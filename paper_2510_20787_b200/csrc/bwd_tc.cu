@@ -541,6 +541,9 @@ bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
             for (int t = 0; t < n_blk; ++t) {
                 bwait(bar_p, t & 1, 7);                        // P^T(t), dS^T(t) are in shared memory
                 tc_fence_after();
+                // the next block's S^T, dP^T first: the key threads wait for those, while dV, dK of this block are only
+                // needed before the operand buffers are rewritten a block later
+                if (t + 1 < n_blk) { wait_blk(t + 1); mma_s_dp(t + 1); }
                 {
                     const uint32_t so = (uint32_t)(t % NST) * (S::QBLK >> 4);
                     if (leader) {
@@ -556,7 +559,6 @@ bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                     }
                     __syncwarp();
                 }
-                if (t + 1 < n_blk) { wait_blk(t + 1); mma_s_dp(t + 1); }
                 // the accumulations of block t-1 have completed (the key threads waited for them before producing
                 // block t's operands): its stage can take block t-1+NST
                 if (t >= 1 && t - 1 + NST < n_blk) tma_blk(t - 1 + NST);
