@@ -171,6 +171,13 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             for (int t = 0; t < n_tiles; ++t) {
                 bwait(bar_p, t & 1, 7);                        // dS(t) is in shared memory; S / dP buffers are free
                 tc_fence_after();
+                // the next tile's S, dP first: the row threads wait for those, while dQ of this tile is only needed before
+                // the dS buffer is rewritten a tile later
+                if (t + 1 < n_tiles) {
+                    need_g(t + 1);
+                    wait_kv(t + 1);
+                    mma_s_dp(t + 1);
+                }
                 {
                     const uint32_t kb = kmn_lo + (uint32_t)(t % NST) * (S::KVTILE >> 4);
                     if (leader) {
@@ -181,11 +188,6 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                         umma_commit(bar_pv);
                     }
                     __syncwarp();
-                }
-                if (t + 1 < n_tiles) {
-                    need_g(t + 1);
-                    wait_kv(t + 1);
-                    mma_s_dp(t + 1);
                 }
                 // dQ(t-1) has completed (the softmax warps waited for it before producing dS(t)): its key stage and
                 // the value stage of tile t-1 can take window tile t-1+NST
