@@ -8,6 +8,7 @@
 // order "z descending, ties to the older token".  A final ordered compaction (ballot prefix sums,
 // positions visited in ascending order) writes idx.  Nothing here rounds: the result is exact on z.
 #include "common.cuh"
+#include "select_body.cuh"
 
 namespace lte {
 namespace {
@@ -154,90 +155,8 @@ __global__ void __launch_bounds__(1024) select_reg_kernel(const float* __restric
     pdl_launch_dependents();
     pdl_wait();                                            // z comes from the previous kernel
     const int bh = blockIdx.x;
-    const float* zz = z + (size_t)bh * T;
-    int32_t* out = idx + (size_t)bh * R;
-    const int N = T - W > 0 ? T - W : 0;
-    const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, wid = tid >> 5, nwarp = nthr >> 5;
-    const int p0 = tid * KPT;
-
-    uint32_t key[KPT];
-#pragma unroll
-    for (int i = 0; i < KPT; ++i) key[i] = p0 + i < N ? key_of(zz, p0 + i, sink, zthr) : 0u;
-    // block-wide sum of a per-thread count, one barrier per call and no atomics: every warp leaves its sum in one of two
-    // alternating rows of partials, and after the barrier every warp adds the row up itself.  A row is rewritten two calls
-    // later, when every warp has passed the barrier of the call in between and so has finished reading it.
-    int slot = 0;
-    auto block_sum = [&](uint32_t c) -> uint32_t {
-        c = __reduce_add_sync(0xffffffffu, c);
-        if (lane == 0) s_part[slot][wid] = c;
-        __syncthreads();
-        const uint32_t total = __reduce_add_sync(0xffffffffu, lane < nwarp ? s_part[slot][lane] : 0u);
-        slot ^= 1;
-        return total;
-    };
-    uint32_t c0 = 0;
-#pragma unroll
-    for (int i = 0; i < KPT; ++i) c0 += key[i] != 0u;
-    const uint32_t nc = block_sum(c0);
-    if (tid == 0 && ncand) ncand[bh] = (int32_t)nc;
-
-    uint32_t theta = 0, need_eq = 0;
-    if (R > 0 && nc > (uint32_t)R) {
-        uint32_t prefix = 0;
-        for (int bit = 31; bit >= 0; --bit) {
-            const uint32_t cand = prefix | (1u << bit);
-            uint32_t c = 0;
-#pragma unroll
-            for (int i = 0; i < KPT; ++i) c += key[i] >= cand;
-            if (block_sum(c) >= (uint32_t)R) prefix = cand;  // at least R keys are >= cand: the R-th largest is too
-        }
-        theta = prefix;
-        uint32_t g = 0;
-#pragma unroll
-        for (int i = 0; i < KPT; ++i) g += key[i] > theta;
-        need_eq = (uint32_t)R - block_sum(g);
-    }
-    // ---- ordered compaction: exclusive scan of (above, equal) counts over the threads' segments
-    uint32_t a = 0, e = 0;
-    if (R > 0) {
-#pragma unroll
-        for (int i = 0; i < KPT; ++i) { a += key[i] > theta; e += (need_eq > 0 && key[i] == theta && p0 + i < N); }
-    }
-    uint32_t ia = a, ie = e;                               // inclusive warp scans
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t ta = __shfl_up_sync(0xffffffffu, ia, o), te = __shfl_up_sync(0xffffffffu, ie, o);
-        if (lane >= o) { ia += ta; ie += te; }
-    }
-    if (lane == 31) { s_wa[wid] = ia; s_we[wid] = ie; }
-    __syncthreads();
-    if (wid == 0) {
-        uint32_t wa = lane < nwarp ? s_wa[lane] : 0u, we = lane < nwarp ? s_we[lane] : 0u;
-        uint32_t xa = wa, xe = we;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const uint32_t ta = __shfl_up_sync(0xffffffffu, xa, o), te = __shfl_up_sync(0xffffffffu, xe, o);
-            if (lane >= o) { xa += ta; xe += te; }
-        }
-        s_wa[lane] = xa - wa; s_we[lane] = xe - we;        // exclusive warp offsets
-    }
-    __syncthreads();
-    uint32_t a_before = s_wa[wid] + ia - a, e_before = s_we[wid] + ie - e;
-    if (R > 0) {
-#pragma unroll
-        for (int i = 0; i < KPT; ++i) {
-            const bool above = key[i] > theta;
-            const bool equal = need_eq > 0 && key[i] == theta && p0 + i < N;
-            if (above || (equal && e_before < need_eq)) {
-                const uint32_t sl = a_before + (e_before < need_eq ? e_before : need_eq);
-                if (sl < (uint32_t)R) out[sl] = p0 + i;
-            }
-            a_before += above; e_before += equal;
-        }
-    }
-    const uint32_t kept = R > 0 ? (nc < (uint32_t)R ? nc : (uint32_t)R) : 0u;
-    for (int i = (int)kept + tid; i < R; i += nthr) out[i] = -1;
-    if (tid == 0) cnt[bh] = (int32_t)kept;
+    select_group<KPT>(z + (size_t)bh * T, idx + (size_t)bh * R, cnt + bh, ncand ? ncand + bh : nullptr, T, W, R, sink, zthr,
+                      (int)threadIdx.x, (int)blockDim.x, s_part, s_wa, s_we, [] { __syncthreads(); });
 }
 
 }  // namespace

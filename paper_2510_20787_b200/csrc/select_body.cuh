@@ -1,0 +1,112 @@
+// Capped selection of one (b,h) by a group of threads that keep their keys in registers (Section 3.1.3, "Capped
+// capacity"): shared by the select kernel (a whole block) and by the scorer kernel, whose CTA that completes a head's
+// last logits selects that head on the spot.
+//
+// Thread `tid` of `nthr` owns KPT consecutive positions.  The R-th largest key is found by bisection on its 32 bits:
+// each step counts the keys >= a candidate value (compares in registers, a warp reduction, one group barrier), so
+// there is no histogram and no contention however concentrated the logits are.  The ordered compaction is one
+// group-wide exclusive scan of the per-thread (above, equal) counts, after which each thread writes the kept
+// positions of its own segment.  `sync` is the group's barrier; s_part [2][32], s_wa [32], s_we [32] are its scratch.
+#pragma once
+#include "common.cuh"
+
+namespace lte {
+
+// key of position j: 0xFFFFFFFF for sink positions, the monotone image of z_j for candidates (z_j > zthr), 0 otherwise.
+// The logit is read past L1: in the fused path other SMs wrote it during the same launch.
+__device__ __forceinline__ uint32_t select_key_of(const float* zz, int j, int sink, float zthr) {
+    if (j < sink) return 0xFFFFFFFFu;
+    const float z = __ldcg(zz + j);
+    return z > zthr ? order_key(z) : 0u;
+}
+
+template <int KPT, typename Sync>
+__device__ __forceinline__ void select_group(const float* __restrict__ zz, int32_t* __restrict__ out, int32_t* cnt_out,
+                                             int32_t* ncand_out, int T, int W, int R, int sink, float zthr, int tid,
+                                             int nthr, uint32_t (*s_part)[32], uint32_t* s_wa, uint32_t* s_we, Sync sync)
+{
+    const int lane = tid & 31, wid = tid >> 5, nwarp = nthr >> 5;
+    const int N = T - W > 0 ? T - W : 0;
+    const int p0 = tid * KPT;
+
+    uint32_t key[KPT];
+#pragma unroll
+    for (int i = 0; i < KPT; ++i) key[i] = p0 + i < N ? select_key_of(zz, p0 + i, sink, zthr) : 0u;
+    // block-wide sum of a per-thread count, one barrier per call and no atomics: every warp leaves its sum in one of two
+    // alternating rows of partials, and after the barrier every warp adds the row up itself.  A row is rewritten two calls
+    // later, when every warp has passed the barrier of the call in between and so has finished reading it.
+    int slot = 0;
+    auto block_sum = [&](uint32_t c) -> uint32_t {
+        c = __reduce_add_sync(0xffffffffu, c);
+        if (lane == 0) s_part[slot][wid] = c;
+        sync();
+        const uint32_t total = __reduce_add_sync(0xffffffffu, lane < nwarp ? s_part[slot][lane] : 0u);
+        slot ^= 1;
+        return total;
+    };
+    uint32_t c0 = 0;
+#pragma unroll
+    for (int i = 0; i < KPT; ++i) c0 += key[i] != 0u;
+    const uint32_t nc = block_sum(c0);
+    if (tid == 0 && ncand_out) *ncand_out = (int32_t)nc;
+
+    uint32_t theta = 0, need_eq = 0;
+    if (R > 0 && nc > (uint32_t)R) {
+        uint32_t prefix = 0;
+        for (int bit = 31; bit >= 0; --bit) {
+            const uint32_t cand = prefix | (1u << bit);
+            uint32_t c = 0;
+#pragma unroll
+            for (int i = 0; i < KPT; ++i) c += key[i] >= cand;
+            if (block_sum(c) >= (uint32_t)R) prefix = cand;  // at least R keys are >= cand: the R-th largest is too
+        }
+        theta = prefix;
+        uint32_t g = 0;
+#pragma unroll
+        for (int i = 0; i < KPT; ++i) g += key[i] > theta;
+        need_eq = (uint32_t)R - block_sum(g);
+    }
+    // ---- ordered compaction: exclusive scan of (above, equal) counts over the threads' segments
+    uint32_t a = 0, e = 0;
+    if (R > 0) {
+#pragma unroll
+        for (int i = 0; i < KPT; ++i) { a += key[i] > theta; e += (need_eq > 0 && key[i] == theta && p0 + i < N); }
+    }
+    uint32_t ia = a, ie = e;                               // inclusive warp scans
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t ta = __shfl_up_sync(0xffffffffu, ia, o), te = __shfl_up_sync(0xffffffffu, ie, o);
+        if (lane >= o) { ia += ta; ie += te; }
+    }
+    if (lane == 31) { s_wa[wid] = ia; s_we[wid] = ie; }
+    sync();
+    if (wid == 0) {
+        uint32_t wa = lane < nwarp ? s_wa[lane] : 0u, we = lane < nwarp ? s_we[lane] : 0u;
+        uint32_t xa = wa, xe = we;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t ta = __shfl_up_sync(0xffffffffu, xa, o), te = __shfl_up_sync(0xffffffffu, xe, o);
+            if (lane >= o) { xa += ta; xe += te; }
+        }
+        s_wa[lane] = xa - wa; s_we[lane] = xe - we;        // exclusive warp offsets
+    }
+    sync();
+    uint32_t a_before = s_wa[wid] + ia - a, e_before = s_we[wid] + ie - e;
+    if (R > 0) {
+#pragma unroll
+        for (int i = 0; i < KPT; ++i) {
+            const bool above = key[i] > theta;
+            const bool equal = need_eq > 0 && key[i] == theta && p0 + i < N;
+            if (above || (equal && e_before < need_eq)) {
+                const uint32_t sl = a_before + (e_before < need_eq ? e_before : need_eq);
+                if (sl < (uint32_t)R) out[sl] = p0 + i;
+            }
+            a_before += above; e_before += equal;
+        }
+    }
+    const uint32_t kept = R > 0 ? (nc < (uint32_t)R ? nc : (uint32_t)R) : 0u;
+    for (int i = (int)kept + tid; i < R; i += nthr) out[i] = -1;
+    if (tid == 0) *cnt_out = (int32_t)kept;
+}
+
+}  // namespace lte
