@@ -82,6 +82,9 @@ __host__ __device__ inline int cache_chunk_pos(const CacheLayout& L, int row, in
 int launch_scores(const Params& p, const void* k, const void* v, float* z, float* r, cudaStream_t st);
 int launch_scores_stack(const Params& p, const void* k, const void* v, float* z, float* r, cudaStream_t st);
 size_t scores_stack_weight_floats(int d, int H);
+size_t scores_stack_tc_workspace(const Params& p);
+int launch_scores_stack_tc(const Params& p, const void* k, const void* v, float* z, float* r, void* ws, size_t ws_bytes,
+                           cudaStream_t st);
 int launch_select(const Params& p, const float* z, int32_t* idx, int32_t* cnt, int32_t* ncand, cudaStream_t st);
 int launch_prefill_simt(const Params& p, const void* q, const void* k, const void* v, const int32_t* idx,
                         const int32_t* cnt, void* o, float* lse, cudaStream_t st);

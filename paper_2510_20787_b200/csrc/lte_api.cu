@@ -12,6 +12,7 @@ int launch_prefill_tc(const Params& p, const void* q, const void* k, const void*
 int prefill_status_fetch_and_clear();
 int decode_status_fetch_and_clear();
 int scores_status_fetch_and_clear();
+int stack_tc_status_fetch_and_clear();
 int bwd_status_fetch_and_clear();
 int decode_tc_status_fetch_and_clear();
 
@@ -89,8 +90,9 @@ int lte_device_status(void)
     const int f = scores_status_fetch_and_clear();
     const int b = bwd_status_fetch_and_clear();
     const int d = decode_tc_status_fetch_and_clear();
-    if (h < 0 || g < 0 || f < 0 || b < 0 || d < 0) return LTE_ERR_CUDA;
-    return (h == 0 && g == 0 && f == 0 && b == 0 && d == 0) ? LTE_OK : LTE_ERR_DEVICE_STATUS;
+    const int t = stack_tc_status_fetch_and_clear();
+    if (h < 0 || g < 0 || f < 0 || b < 0 || d < 0 || t < 0) return LTE_ERR_CUDA;
+    return (h == 0 && g == 0 && f == 0 && b == 0 && d == 0 && t == 0) ? LTE_OK : LTE_ERR_DEVICE_STATUS;
 }
 
 size_t lte_workspace_bytes(int op, const lte_shape* s, const lte_conv* c)
@@ -101,13 +103,16 @@ size_t lte_workspace_bytes(int op, const lte_shape* s, const lte_conv* c)
         Params p = make_params(s, c);
         return bwd_workspace_bytes(p, LTE_BWD_CNN_INPUT_GRAD);
     }
+    if (op == LTE_OP_SCORES && c && c->n_layers == 3) {
+        if (check_shape(s, true) != LTE_OK) return 0;
+        return scores_stack_tc_workspace(make_params(s, c));
+    }
     return 0;
 }
 
 int lte_scores(const lte_shape* s, const lte_conv* c, const void* k, const void* v, float* z, float* r_or_null,
                void* ws, size_t ws_bytes, void* stream)
 {
-    (void)ws; (void)ws_bytes;
     int e = check_shape(s, true); if (e) return e;
     if (c && c->w && c->n_layers == 3) {
         // the paper's stack: kernel 3, dilation 2, channels 2d -> d -> d/2 -> d/4 -> 1 (packed parameters, see lte.h)
@@ -118,6 +123,9 @@ int lte_scores(const lte_shape* s, const lte_conv* c, const void* k, const void*
         e = check_arch(); if (e) return e;
         Params p = make_params(s, c);
         p.K = 13; p.half = 6;
+        // tensor cores where the shape allows and the caller brought the workspace for the split weight image
+        e = launch_scores_stack_tc(p, k, v, z, r_or_null, ws, ws_bytes, (cudaStream_t)stream);
+        if (e != LTE_ERR_UNSUPPORTED) return e;
         return launch_scores_stack(p, k, v, z, r_or_null, (cudaStream_t)stream);
     }
     e = check_conv(s, c); if (e) return e;

@@ -136,12 +136,17 @@ def lte_workspace_bytes(op, s, c=None):
     return int(lib().lte_workspace_bytes(op, ctypes.addressof(s), None if c is None else ctypes.addressof(c)))
 
 
-def lte_scores(s, c, k, v, z=None, r=None):
-    """k, v [B,H,T,d] -> z [B,H,T] fp32 (and r = sigmoid(z) if a tensor is given)."""
+def lte_scores(s, c, k, v, z=None, r=None, ws=None):
+    """k, v [B,H,T,d] -> z [B,H,T] fp32 (and r = sigmoid(z) if a tensor is given).  ws: a uint8 workspace tensor of
+    lte_workspace_bytes(OP_SCORES, s, c) bytes (allocated here when None and the call wants one; False = none)."""
     if z is None:
         z = torch.empty((s.B, s.H, s.T), dtype=torch.float32, device=k.device)
+    if ws is None:
+        n = lte_workspace_bytes(OP_SCORES, s, c)
+        ws = torch.empty(n, dtype=torch.uint8, device=k.device) if n > 0 else False
+    wp, wn = (None, 0) if ws is False else (_ptr(ws, torch.uint8), ws.numel())
     _check("lte_scores", lib().lte_scores(ctypes.addressof(s), ctypes.addressof(c), _ptr(k), _ptr(v),
-                                          _ptr(z, torch.float32), _ptr(r, torch.float32), None, 0, _stream()))
+                                          _ptr(z, torch.float32), _ptr(r, torch.float32), wp, wn, _stream()))
     return z
 
 

@@ -45,6 +45,42 @@ def test_stack_logits_and_selection(dtype, d, T, W, R, bias):
     check_idx(idx.cpu().numpy(), cnt.cpu().numpy(), z64, W, R, 0, 0.5)
 
 
+@pytest.mark.parametrize("B,H,T,bias", [(1, 1, 13, True), (2, 2, 126, False), (1, 2, 127, True), (2, 1, 246, True), (1, 3, 247, False),
+                                        (3, 20, 500, True), (4, 16, 4096, True)])
+def test_stack_tensor_core_path(B, H, T, bias):
+    """bf16, d = 64 with a workspace: the tensor-core kernel (three-way split operands).  Tile edges (120 logits per
+    tile), several heads per thread block and several thread blocks per head; the same call without a workspace runs
+    the fp32 kernel, and both have to agree with the oracle."""
+    cfg = synth.Config("stack", "bf16", B, H, 64, T, 8, 12, 7, 0.1)
+    x = synth.make(cfg, 5)
+    wl, wout, bl, bout = _stack_params(H, 64, 5, bias)
+    z64 = orc.scores_stack(x["k"], x["v"], wl, bl, wout, bout)
+    s = shape_of(cfg, B=B)
+    t = lambda a: None if a is None else torch.from_numpy(a).cuda()
+    c = lte.conv_stack([t(w) for w in wl], t(wout), [t(b) for b in bl] if bias else None, t(bout))
+    k, v = dev(x["k"], "bf16"), dev(x["v"], "bf16")
+    need = lte.lte_workspace_bytes(lte.OP_SCORES, s, c)
+    assert need == H * 194176
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    r = torch.empty((B, H, T), dtype=torch.float32, device="cuda")
+    fin = np.isfinite(z64)
+    tol = 2e-5 * max(1.0, np.max(np.abs(z64[fin])))
+    for rep in range(2):                                             # twice: the kernel's barriers and the workspace are reusable
+        z = lte.lte_scores(s, c, k, v, r=r, ws=ws)
+        torch.cuda.synchronize()
+        assert lte.lib().lte_device_status() == 0
+        zn = z.cpu().numpy().astype(np.float64)
+        assert np.array_equal(np.isfinite(zn), fin) and np.all(np.isneginf(zn[~fin]))
+        assert np.max(np.abs(zn[fin] - z64[fin])) <= tol
+        rn = r.cpu().numpy()
+        assert np.max(np.abs(rn[fin] - 1 / (1 + np.exp(-z64[fin])))) < 1e-5 and np.all(rn[~fin] == 0)
+    z32 = lte.lte_scores(s, c, k, v, ws=False).cpu().numpy().astype(np.float64)     # no workspace: the fp32 kernel
+    assert np.max(np.abs(z32[fin] - z64[fin])) <= tol
+    idx, cnt = lte.lte_select(s, z)
+    torch.cuda.synchronize()
+    check_idx(idx.cpu().numpy(), cnt.cpu().numpy(), z64, cfg.W, cfg.R, 0, 0.5)
+
+
 def test_stack_rejected_elsewhere():
     """decode, cache_init and the backward take the single layer only."""
     cfg = synth.Config("stack", "bf16", 1, 2, 64, 64, 16, 8, 7, 0.1)
