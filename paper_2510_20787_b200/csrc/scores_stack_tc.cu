@@ -14,8 +14,8 @@
 // start address.  Row m of a tile is time tb - 8 + m: the input tile carries 4 more rows above, the first 4 rows of
 // the second layer and the first 8 of the third are not used, so a tile yields 120 logits.
 //
-// One CTA per SM walks consecutive tiles of (head, batch) rows.  Warp 9 feeds shared memory: the input rows by TMA
-// (16-byte-wide boxes, one per chunk column; rows before time 0 arrive as zeros), the first layer's weights tap by
+// One CTA per SM walks consecutive tiles of (head, batch) rows.  Warp 9 feeds shared memory: the input rows by
+// 16-byte asynchronous copies into their chunk columns (rows before time 0 zero-filled), the first layer's weights tap by
 // tap through a two-slot ring (their split image, 144 KB per head, does not fit beside the rest), the small layers'
 // weights once per head.  Warp 8 issues the MMAs.  Warps 0-7 are the epilogues: TMEM -> bias, Swish -> three bf16
 // pieces -> the next layer's operand in shared memory; the last one takes the dot product with the output vector.
@@ -25,6 +25,12 @@
 namespace lte {
 
 __device__ int g_stack_tc_status = 0;
+#ifdef ST_PROFILE
+__device__ long long g_stprof[64];
+#define STP(i) do { if (blockIdx.x == 3 && it == 5 && lane == 0) g_stprof[i] = clock64(); } while (0)
+#else
+#define STP(i) do {} while (0)
+#endif
 
 namespace {
 
@@ -36,7 +42,7 @@ constexpr int ST_COL = ST_ROWS * 16;                           // bytes of a chu
 constexpr int ST_XROWS = 132;                                  // input rows per tile: times tb-12 .. tb+119
 constexpr int ST_VALID = 120;                                  // logits per tile
 constexpr int ST_HALF = 6;
-constexpr int ST_THREADS = 320;
+constexpr int ST_THREADS = 352;                                // 8 epilogue warps, first-layer MMA warp, producer, later-layers MMA warp
 
 // per-head image in the workspace (bytes): first-layer weights per tap, then what stays resident for the head
 constexpr int IMG_W0_TAP = 16 * 192 * 16;                      // [chunk 16][n = piece * 64 + c_out][8 channels] bf16
@@ -55,15 +61,27 @@ constexpr int OFF_W1 = OFF_HID + 24 * ST_COL;
 constexpr int OFF_W2 = OFF_W1 + IMG_W1;
 constexpr int OFF_PAR = OFF_W2 + IMG_W2;
 constexpr int OFF_BAR = OFF_PAR + IMG_PAR;
-constexpr int ST_SMEM = OFF_BAR + 128;
+constexpr int ST_SMEM = OFF_BAR + 192;
 static_assert(ST_SMEM <= 232448, "shared memory");
-constexpr uint32_t D0_COL = 0, D1_COL = 192, D2_COL = 288, ST_TMEM = 512;
+constexpr uint32_t D0_COL = 0, D1_COL = 384, D2_COL = 384, ST_TMEM = 512;   // two first-layer accumulators; the third layer's takes the second's columns
 
 // unswizzled K-major descriptor: 8 rows x 16 bytes per core matrix, SBO = 128 bytes between 8-row groups, LBO = the
 // distance between the two 8-channel chunk columns of a K = 16 step
 constexpr uint32_t kDescHiFlat = (128u >> 4) | (1u << 14);
 
-__device__ __forceinline__ void swait(uint32_t bar, uint32_t parity, int code) { mbar_wait_s(bar, parity, code, &g_stack_tc_status); }
+// Bounded wait.  The phases of this kernel are long (thousands of cycles) and at any time most warps are waiting, so the
+// wait must not poll: try_wait is given a suspend-time hint and the thread sleeps in hardware until the phase
+// completes (polling warps kept the shared-memory pipeline busy and slowed the working warps several times over).
+__device__ __forceinline__ void swait(uint32_t bar, uint32_t parity, int code) {
+    for (uint32_t i = 0; i < (1u << 20); ++i) {
+        uint32_t ok;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(ok) : "r"(bar), "r"(parity), "r"(20000u) : "memory");
+        if (ok) return;
+        if ((i & 255u) == 255u && *reinterpret_cast<volatile int*>(&g_stack_tc_status) != 0) return;
+    }
+    atomicExch(&g_stack_tc_status, code);
+}
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
@@ -141,7 +159,7 @@ __device__ __forceinline__ StackWork stack_work(int f, int n_t, int B, int H) {
 }
 
 __global__ void __launch_bounds__(ST_THREADS, 1)
-scores_stack_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+scores_stack_tc_kernel(const __nv_bfloat16* __restrict__ kg, const __nv_bfloat16* __restrict__ vg,
                        const uint8_t* __restrict__ img, float* __restrict__ z, float* __restrict__ r_out, int B, int H,
                        int Tlen, int n_t, int n_flat, int per_cta)
 {
@@ -154,8 +172,10 @@ scores_stack_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
     const float* par = reinterpret_cast<const float*>(smem_raw + OFF_PAR);
     const uint32_t bar0 = base + OFF_BAR;
     const uint32_t bar_x = bar0, bar_rf = bar0 + 8, bar_re = bar0 + 24, bar_d0 = bar0 + 40, bar_d1 = bar0 + 48, bar_d2 = bar0 + 56;
-    const uint32_t bar_h0 = bar0 + 64, bar_h1 = bar0 + 72, bar_ed = bar0 + 80, bar_w = bar0 + 88, tmem_slot = bar0 + 96;
-    volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(smem_raw + OFF_BAR + 96);
+    const uint32_t bar_h0 = bar0 + 64, bar_h1 = bar0 + 72, bar_w = bar0 + 88, bar_d0b = bar0 + 96, bar_f0 = bar0 + 104;
+    const uint32_t bar_ed4 = bar0 + 128;                       // four barriers, one per tile modulo 4 (see the producer)
+    const uint32_t tmem_slot = bar0 + 120;
+    volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(smem_raw + OFF_BAR + 120);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int f_begin = blockIdx.x * per_cta, f_end = min(f_begin + per_cta, n_flat);
@@ -168,8 +188,11 @@ scores_stack_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
     if (tid == 0) {
         mbar_init(bar_x, 1);
         mbar_init(bar_rf, 1); mbar_init(bar_rf + 8, 1); mbar_init(bar_re, 1); mbar_init(bar_re + 8, 1);
-        mbar_init(bar_d0, 1); mbar_init(bar_d1, 1); mbar_init(bar_d2, 1);
-        mbar_init(bar_h0, 8); mbar_init(bar_h1, 8); mbar_init(bar_ed, 4); mbar_init(bar_w, 1);
+        mbar_init(bar_d0, 1); mbar_init(bar_d0b, 1); mbar_init(bar_d1, 1); mbar_init(bar_d2, 1);
+        mbar_init(bar_f0, 8); mbar_init(bar_f0 + 8, 8);
+        mbar_init(bar_h0, 8); mbar_init(bar_h1, 8); mbar_init(bar_w, 1);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) mbar_init(bar_ed4 + 8 * e, 4);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 8) tmem_alloc(tmem_slot, ST_TMEM);
@@ -182,15 +205,31 @@ scores_stack_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
     if (warp == 9) {
         // =================================== producer ======================================================
         const bool leader = lane == 0;
+        // input rows tb-12 .. tb+119 into their chunk columns, 16 bytes per copy: a lane takes row (l & 7) of a block of 8
+        // rows and one of 4 chunks, so a quarter warp writes 128 contiguous bytes and reads full 32-byte sectors.  Rows
+        // outside [0, T) are zero-filled.  (Tensor-map copies with 16-byte boxes needed about 3,600 cycles per tile.)
         auto load_x = [&](const StackWork& w) {
-            if (leader) {
-                mbar_expect_tx(bar_x, 16 * ST_XROWS * 16);
+            const __nv_bfloat16* kb = kg + (size_t)w.bh * Tlen * ST_D;
+            const __nv_bfloat16* vb = vg + (size_t)w.bh * Tlen * ST_D;
+            const int t0 = w.tb - 12, r_in = lane & 7, cq = lane >> 3;
+#pragma unroll 1
+            for (int rb = 0; rb < (ST_XROWS + 7) / 8; ++rb) {
+                const int r = rb * 8 + r_in, t = t0 + r;
+                const bool ok = r < ST_XROWS && t >= 0 && t < Tlen;
+                if (r < ST_XROWS) {
 #pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    tma_load_3d(sX + c * ST_COL, &tmK, c * 8, w.tb - 12, w.bh, bar_x);
-                    tma_load_3d(sX + (8 + c) * ST_COL, &tmV, c * 8, w.tb - 12, w.bh, bar_x);
+                    for (int cg = 0; cg < 4; ++cg) {
+                        const int c = cg * 4 + cq;
+                        const __nv_bfloat16* src = (cg < 2 ? kb : vb) + (size_t)(ok ? t : 0) * ST_D + (c & 7) * 8;
+                        cp_async16(sX + c * ST_COL + r * 16, src, ok ? 16u : 0u);
+                    }
                 }
             }
+            cp_async_commit();
+            cp_async_wait<0>();
+            fence_proxy_async();                               // the tensor core reads these rows through the async proxy
+            __syncwarp();
+            if (leader) mbar_arrive(bar_x);
         };
         auto load_tap = [&](int n, int h) {                    // n: taps since the start of this CTA's walk (3 per tile)
             if (leader) {
@@ -209,93 +248,125 @@ scores_stack_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
         auto wait_tap_done = [&](int n) { swait(bar_re + 8 * (n & 1), (n >> 1) & 1, 20); };
         if (n_my > 0) {
             StackWork w = stack_work(f_begin, n_t, B, H);
+            int h_loaded = w.h;
             load_head(w.h);
-            load_x(w);
             load_tap(0, w.h); load_tap(1, w.h);
+            load_x(w);
             wait_tap_done(0);
             load_tap(2, w.h);
             for (int it = 0; it < n_my; ++it) {
                 const bool more = it + 1 < n_my;
                 StackWork wn = w;
                 if (more) wn = stack_work(f_begin + it + 1, n_t, B, H);
-                wait_tap_done(3 * it + 1);
-                if (more) load_tap(3 * it + 3, wn.h);
-                wait_tap_done(3 * it + 2);                     // the first layer is done: the input buffer takes the next tile
-                if (more) { load_x(wn); load_tap(3 * it + 4, wn.h); }
-                swait(bar_ed, it & 1, 22);                     // every reader of this head's resident weights is done with this tile
-                if (more && wn.h != w.h) load_head(wn.h);
                 if (more) {
+                    wait_tap_done(3 * it + 1);
+                    load_tap(3 * it + 3, wn.h);
+                    wait_tap_done(3 * it + 2);                 // the first layer of tile it is done: the input buffer takes the next tile
+                    load_tap(3 * it + 4, wn.h);
+                    load_x(wn);
                     wait_tap_done(3 * it + 3);
                     load_tap(3 * it + 5, wn.h);
+                } else {
+                    wait_tap_done(3 * it + 1);
+                    wait_tap_done(3 * it + 2);
+                }
+                // The resident weights change with the head, once every reader of the old ones is done with the previous
+                // tile.  That tile's end is awaited here, one tile late, where it no longer holds up the loads above; the
+                // epilogue of a head's first tile waits for the new weights.  While this warp waits for the end of tile
+                // it-1, the epilogues can get as far as the end of tile it+1 (whose loads are out), so the barrier is one
+                // of four by tile number: with fewer, a late waiter would take a later completion for the one it wants.
+                if (it >= 1) {
+                    swait(bar_ed4 + 8 * ((it - 1) & 3), ((it - 1) >> 2) & 1, 22);
+                    if (w.h != h_loaded) { load_head(w.h); h_loaded = w.h; }
                 }
                 w = wn;
             }
         }
     } else if (warp == 8) {
-        // =================================== MMA issue =====================================================
+        // =================================== MMA issue, first layer ========================================
+        // Two warps issue MMAs (an issue costs some 50 cycles, more than the small products of the later layers take):
+        // this one the first layer, one tile ahead of the epilogues and into the other of two accumulators; warp 10 the
+        // second and third layers.  The whole warp walks the schedule; only the tcgen05 instructions are issued by lane 0.
         const bool leader = lane == 0;
-        constexpr uint32_t LBO_X = ST_COL, LBO_W0 = 192 * 16, LBO_W1 = 96 * 16, LBO_W2 = 48 * 16;
-        int heads_seen = 0, h_prev = -1;
+        constexpr uint32_t LBO_X = ST_COL, LBO_W0 = 192 * 16;
         for (int it = 0; it < n_my; ++it) {
-            const StackWork w = stack_work(f_begin + it, n_t, B, H);
+            // this accumulator was last used by tile it-2: its epilogue has loaded it.  (Barriers per accumulator: this
+            // warp runs up to two tiles ahead of the epilogues, and a barrier must never get two phases ahead of a waiter.)
+            if (it >= 2) swait(bar_f0 + 8 * (it & 1), ((it >> 1) - 1) & 1, 6);
             swait(bar_x, it & 1, 1);
-            // ---- layer 0: 3 taps x 8 K steps, N = 192 (three weight pieces of 64 channels) ----
+            STP(0);
             for (int tau = 0; tau < 3; ++tau) {
                 const int n = 3 * it + tau;
                 swait(bar_rf + 8 * (n & 1), (n >> 1) & 1, 2);
                 tc_fence_after();
                 const uint32_t a0 = desc_lo(sX + 2 * tau * 16, LBO_X), b0 = desc_lo(sRing + (n & 1) * IMG_W0_TAP, LBO_W0);
-                if (leader) {
+                const uint32_t d = tmem + D0_COL + (it & 1) * 192;
 #pragma unroll
-                    for (int kk = 0; kk < 8; ++kk)
-                        umma(tmem + D0_COL, desc64(a0 + ((2 * kk * ST_COL) >> 4), kDescHiFlat),
-                             desc64(b0 + ((2 * kk * 192 * 16) >> 4), kDescHiFlat), instr_desc(128, 192, false), (tau > 0 || kk > 0) ? 1u : 0u);
+                for (int kk = 0; kk < 8; ++kk) {
+                    const uint64_t ad = desc64(a0 + ((2 * kk * ST_COL) >> 4), kDescHiFlat), bd = desc64(b0 + ((2 * kk * 192 * 16) >> 4), kDescHiFlat);
+                    if (leader) umma(d, ad, bd, instr_desc(128, 192, false), (tau > 0 || kk > 0) ? 1u : 0u);
+                }
+                if (leader) {
                     umma_commit(bar_re + 8 * (n & 1));
-                    if (tau == 2) umma_commit(bar_d0);
+                    if (tau == 2) umma_commit((it & 1) ? bar_d0b : bar_d0);
                 }
                 __syncwarp();
             }
+            STP(2);
+        }
+    } else if (warp == 10) {
+        // =================================== MMA issue, second and third layers ============================
+        const bool leader = lane == 0;
+        constexpr uint32_t LBO_X = ST_COL, LBO_W1 = 96 * 16, LBO_W2 = 48 * 16;
+        int heads_seen = 0, h_prev = -1;
+        for (int it = 0; it < n_my; ++it) {
+            const StackWork w = stack_work(f_begin + it, n_t, B, H);
             if (w.h != h_prev) { swait(bar_w, heads_seen & 1, 3); ++heads_seen; h_prev = w.h; }   // this head's small layers are in
             // ---- layer 1: taps x activation pieces (N = 96, 64, 32: the weight pieces each one meets) x 4 K steps ----
             swait(bar_h0, it & 1, 4);
+            STP(3);
             tc_fence_after();
+#pragma unroll
             for (int tau = 0; tau < 3; ++tau) {
 #pragma unroll
                 for (int p = 0; p < 3; ++p) {
                     const uint32_t a1 = desc_lo(sH0 + p * 8 * ST_COL + (4 + 2 * tau) * 16, LBO_X);
                     const uint32_t b1 = desc_lo(sW1 + tau * 8 * 96 * 16, LBO_W1);
                     const uint32_t idesc = p == 0 ? instr_desc(128, 96, false) : p == 1 ? instr_desc(128, 64, false) : instr_desc(128, 32, false);
-                    if (leader) {
 #pragma unroll
-                        for (int kk = 0; kk < 4; ++kk)
-                            umma(tmem + D1_COL, desc64(a1 + ((2 * kk * ST_COL) >> 4), kDescHiFlat),
-                                 desc64(b1 + ((2 * kk * 96 * 16) >> 4), kDescHiFlat), idesc, (tau > 0 || p > 0 || kk > 0) ? 1u : 0u);
+                    for (int kk = 0; kk < 4; ++kk) {
+                        const uint64_t ad = desc64(a1 + ((2 * kk * ST_COL) >> 4), kDescHiFlat), bd = desc64(b1 + ((2 * kk * 96 * 16) >> 4), kDescHiFlat);
+                        if (leader) umma(tmem + D1_COL, ad, bd, idesc, (tau > 0 || p > 0 || kk > 0) ? 1u : 0u);
                     }
                 }
             }
             if (leader) umma_commit(bar_d1);
             __syncwarp();
-            // ---- layer 2: N = 48, 32, 16, 2 K steps ----
+            STP(4);
+            // ---- layer 2: N = 48, 32, 16, 2 K steps; its accumulator takes the columns of the second layer's, which the
+            // epilogue has read before it publishes h1 ----
             swait(bar_h1, it & 1, 5);
+            STP(5);
             tc_fence_after();
+#pragma unroll
             for (int tau = 0; tau < 3; ++tau) {
 #pragma unroll
                 for (int p = 0; p < 3; ++p) {
                     const uint32_t a2 = desc_lo(sH1 + p * 4 * ST_COL + (4 + 2 * tau) * 16, LBO_X);
                     const uint32_t b2 = desc_lo(sW2 + tau * 4 * 48 * 16, LBO_W2);
                     const uint32_t idesc = p == 0 ? instr_desc(128, 48, false) : p == 1 ? instr_desc(128, 32, false) : instr_desc(128, 16, false);
-                    if (leader) {
 #pragma unroll
-                        for (int kk = 0; kk < 2; ++kk)
-                            umma(tmem + D2_COL, desc64(a2 + ((2 * kk * ST_COL) >> 4), kDescHiFlat),
-                                 desc64(b2 + ((2 * kk * 48 * 16) >> 4), kDescHiFlat), idesc, (tau > 0 || p > 0 || kk > 0) ? 1u : 0u);
+                    for (int kk = 0; kk < 2; ++kk) {
+                        const uint64_t ad = desc64(a2 + ((2 * kk * ST_COL) >> 4), kDescHiFlat), bd = desc64(b2 + ((2 * kk * 48 * 16) >> 4), kDescHiFlat);
+                        if (leader) umma(tmem + D2_COL, ad, bd, idesc, (tau > 0 || p > 0 || kk > 0) ? 1u : 0u);
                     }
                 }
             }
             if (leader) umma_commit(bar_d2);
             __syncwarp();
+            STP(6);
         }
-    } else {
+    } else if (warp < 8) {
         // =================================== epilogue warps ================================================
         // warp w owns TMEM lanes 32 (w & 3) .. +31 (row m of the tile) and, where a layer is split, half (w >> 2) of its channels
         const int q = warp & 3, half = warp >> 2;
@@ -311,19 +382,28 @@ scores_stack_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
             const int ff = f_begin + it;
             const StackWork w = stack_work(ff, n_t, B, H);
             const int time = w.tb - 8 + m;
-            const bool live = time >= 0;                       // every layer's output is zero at negative times
+            // every layer's output is zero at negative times (a mask, not a branch: the channels' chains must interleave)
+            const uint32_t live_mask = time >= 0 ? 0xffffffffu : 0u;
             if (w.h != h_prev) { swait(bar_w, heads_seen & 1, 10); ++heads_seen; h_prev = w.h; }
 
             // ---- layer 0 -> h0: 32 of the 64 channels per warp ----
-            swait(bar_d0, it & 1, 11);
+            if (warp == 0) STP(10);
+            swait((it & 1) ? bar_d0b : bar_d0, (it >> 1) & 1, 11);
+            if (warp == 0) STP(11);
             tc_fence_after();
             {
                 uint32_t a[32], b[32], c[32];
-                tmem_ld32(tmem + lane_base + D0_COL + half * 32, a);
-                tmem_ld32(tmem + lane_base + D0_COL + 64 + half * 32, b);
-                tmem_ld32(tmem + lane_base + D0_COL + 128 + half * 32, c);
+                tmem_ld32(tmem + lane_base + D0_COL + (it & 1) * 192 + half * 32, a);
+                tmem_ld32(tmem + lane_base + D0_COL + (it & 1) * 192 + 64 + half * 32, b);
+                tmem_ld32(tmem + lane_base + D0_COL + (it & 1) * 192 + 128 + half * 32, c);
                 tmem_wait_ld();
-                const float* bias = par + half * 32;
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_f0 + 8 * (it & 1));   // the accumulator may take tile it + 2
+                if (warp == 0) STP(20);
+                float bias[32];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) *reinterpret_cast<float4*>(&bias[4 * e]) = *reinterpret_cast<const float4*>(par + half * 32 + 4 * e);
 #pragma unroll
                 for (int ch = 0; ch < 4; ++ch) {
                     uint32_t hi[4], mid[4], lo[4];
@@ -332,21 +412,24 @@ scores_stack_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
                         const int c0 = ch * 8 + 2 * e;
                         float y0 = (f(a[c0]) + f(b[c0])) + f(c[c0]) + bias[c0];
                         float y1 = (f(a[c0 + 1]) + f(b[c0 + 1])) + f(c[c0 + 1]) + bias[c0 + 1];
-                        y0 = live ? swish(y0) : 0.f;
-                        y1 = live ? swish(y1) : 0.f;
+                        y0 = __uint_as_float(__float_as_uint(swish(y0)) & live_mask);
+                        y1 = __uint_as_float(__float_as_uint(swish(y1)) & live_mask);
                         split3(y0, y1, hi[e], mid[e], lo[e]);
                     }
                     const uint32_t dst = sH0 + (uint32_t)(half * 4 + ch) * ST_COL + row_off;
                     store_chunk(dst, hi); store_chunk(dst + 8 * ST_COL, mid); store_chunk(dst + 16 * ST_COL, lo);
                 }
             }
+            if (warp == 0) STP(21);
             fence_proxy_async();                               // the tensor core reads these rows through the async proxy
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_h0);
+            if (warp == 0) STP(12);
 
             // ---- layer 1 -> h1: 16 of the 32 channels per warp ----
             swait(bar_d1, it & 1, 12);
+            if (warp == 0) STP(13);
             tc_fence_after();
             {
                 uint32_t a[16], b[16], c[16];
@@ -354,7 +437,9 @@ scores_stack_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
                 tmem_ld16(tmem + lane_base + D1_COL + 32 + half * 16, b);
                 tmem_ld16(tmem + lane_base + D1_COL + 64 + half * 16, c);
                 tmem_wait_ld();
-                const float* bias = par + 64 + half * 16;
+                float bias[16];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) *reinterpret_cast<float4*>(&bias[4 * e]) = *reinterpret_cast<const float4*>(par + 64 + half * 16 + 4 * e);
 #pragma unroll
                 for (int ch = 0; ch < 2; ++ch) {
                     uint32_t hi[4], mid[4], lo[4];
@@ -363,8 +448,8 @@ scores_stack_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
                         const int c0 = ch * 8 + 2 * e;
                         float y0 = (f(a[c0]) + f(b[c0])) + f(c[c0]) + bias[c0];
                         float y1 = (f(a[c0 + 1]) + f(b[c0 + 1])) + f(c[c0 + 1]) + bias[c0 + 1];
-                        y0 = live ? swish(y0) : 0.f;
-                        y1 = live ? swish(y1) : 0.f;
+                        y0 = __uint_as_float(__float_as_uint(swish(y0)) & live_mask);
+                        y1 = __uint_as_float(__float_as_uint(swish(y1)) & live_mask);
                         split3(y0, y1, hi[e], mid[e], lo[e]);
                     }
                     const uint32_t dst = sH1 + (uint32_t)(half * 2 + ch) * ST_COL + row_off;
@@ -375,23 +460,32 @@ scores_stack_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_h1);
+            if (warp == 0) STP(14);
 
-            // ---- layer 2 and the output map: warps 0-3, one logit per row ----
+            // ---- layer 2 and the output map: warps 0-3, one logit per row.  Every warp waits for the third layer: it reads
+            // h1 from the columns that the next tile's h0 goes to ----
+            swait(bar_d2, it & 1, 13);
             if (half == 0) {
-                swait(bar_d2, it & 1, 13);
+                if (warp == 0) STP(15);
                 tc_fence_after();
                 uint32_t a[16], b[16], c[16];
                 tmem_ld16(tmem + lane_base + D2_COL, a);
                 tmem_ld16(tmem + lane_base + D2_COL + 16, b);
                 tmem_ld16(tmem + lane_base + D2_COL + 32, c);
                 tmem_wait_ld();
-                float zz = par[128];
+                if (warp == 0) STP(17);
+                float pv[32];                                  // b2[16] | wout[16]
+#pragma unroll
+                for (int e = 0; e < 8; ++e) *reinterpret_cast<float4*>(&pv[4 * e]) = *reinterpret_cast<const float4*>(par + 96 + 4 * e);
+                float zq[4] = {par[128], 0.f, 0.f, 0.f};
 #pragma unroll
                 for (int c0 = 0; c0 < 16; ++c0) {
-                    float y = (f(a[c0]) + f(b[c0])) + f(c[c0]) + par[96 + c0];
-                    y = live ? swish(y) : 0.f;
-                    zz = fmaf(par[112 + c0], y, zz);
+                    float y = (f(a[c0]) + f(b[c0])) + f(c[c0]) + pv[c0];
+                    y = __uint_as_float(__float_as_uint(swish(y)) & live_mask);
+                    zq[c0 & 3] = fmaf(pv[16 + c0], y, zq[c0 & 3]);
                 }
+                const float zz = (zq[0] + zq[1]) + (zq[2] + zq[3]);
+                if (warp == 0) STP(18);
                 const int j = time - ST_HALF;                  // the logit of token j is the output at time j + 6
                 if (m >= 8 && time < Tlen) {
                     z[(size_t)w.bh * Tlen + j] = zz;
@@ -402,29 +496,17 @@ scores_stack_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
                     z[(size_t)w.bh * Tlen + Tlen - ST_HALF + lane] = -INFINITY;
                     if (r_out) r_out[(size_t)w.bh * Tlen + Tlen - ST_HALF + lane] = 0.f;
                 }
+                if (warp == 0) STP(19);
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar_ed);
+                if (lane == 0) mbar_arrive(bar_ed4 + 8 * (it & 3));
+                if (warp == 0) STP(16);
             }
         }
     }
     tc_fence_before();
     __syncthreads();
     if (warp == 8) tmem_dealloc(tmem, ST_TMEM);
-}
-
-// [B*H][T][d] bf16 as a 3-D tensor; box = 8 channels (16 bytes) x ST_XROWS rows, no swizzle: one chunk column per load.
-bool make_chunk_map(CUtensorMap* m, const void* ptr, int BH, int T, int d)
-{
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)T, (cuuint64_t)BH};
-    cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)T * d * 2};
-    cuuint32_t box[3] = {8, (cuuint32_t)ST_XROWS, 1};
-    cuuint32_t estr[3] = {1, 1, 1};
-    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 }  // namespace
@@ -459,9 +541,7 @@ int launch_scores_stack_tc(const Params& p, const void* k, const void* v, float*
             return LTE_ERR_CUDA;
         attr_done = true;
     }
-    CUtensorMap tk, tv;
     const int BH = p.B * p.H;
-    if (!make_chunk_map(&tk, k, BH, p.T, p.d) || !make_chunk_map(&tv, v, BH, p.T, p.d)) return LTE_ERR_CUDA;
     if (launch_pdl(stack_image_kernel, dim3(p.H, 32), dim3(256), 0, st, p.w, p.bias, (uint8_t*)ws, p.H) != cudaSuccess) return LTE_ERR_CUDA;
     const int n_t = (p.T - ST_HALF + ST_VALID - 1) / ST_VALID;
     const long long n_flat = (long long)BH * n_t;
@@ -469,10 +549,22 @@ int launch_scores_stack_tc(const Params& p, const void* k, const void* v, float*
     const int grid = (int)(n_flat < n_sm ? n_flat : n_sm);
     const int per = (int)((n_flat + grid - 1) / grid);
     const int n_cta = (int)((n_flat + per - 1) / per);
-    if (launch_pdl(scores_stack_tc_kernel, dim3(n_cta), dim3(ST_THREADS), ST_SMEM, st, tk, tv, (const uint8_t*)ws, z, r, p.B, p.H,
+    if (launch_pdl(scores_stack_tc_kernel, dim3(n_cta), dim3(ST_THREADS), ST_SMEM, st, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (const uint8_t*)ws, z, r, p.B, p.H,
                    p.T, n_t, (int)n_flat, per) != cudaSuccess)
         return LTE_ERR_CUDA;
     return cuda_status(cudaGetLastError());
 }
 
 }  // namespace lte
+
+#if defined(ST_PROFILE) || defined(ST_RAW)
+namespace lte { int prefill_status_fetch_and_clear(); int decode_status_fetch_and_clear(); int scores_status_fetch_and_clear(); int bwd_status_fetch_and_clear(); int decode_tc_status_fetch_and_clear(); }
+extern "C" void lte_status_all(int* o) { o[0] = lte::prefill_status_fetch_and_clear(); o[1] = lte::decode_status_fetch_and_clear(); o[2] = lte::scores_status_fetch_and_clear(); o[3] = lte::bwd_status_fetch_and_clear(); o[4] = lte::decode_tc_status_fetch_and_clear(); o[5] = lte::stack_tc_status_fetch_and_clear(); }
+extern "C" int lte_stack_status_raw() { return lte::stack_tc_status_fetch_and_clear(); }
+#endif
+#ifdef ST_PROFILE
+extern "C" int lte_stprof_read(long long* out)
+{
+    return cudaMemcpyFromSymbol(out, lte::g_stprof, sizeof(long long) * 64) == cudaSuccess ? 0 : -1;
+}
+#endif
