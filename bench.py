@@ -358,7 +358,8 @@ def _extras_sections(torch, lte, synth, pk, flush, args, which):
 
 def _extra_s(out, torch, lte, synth, pk, flush, n5):
     """The paper's three-layer scorer (kernel 3, dilation 2, channels 2d -> d -> d/2 -> d/4 -> 1) at the C2 shape.
-    fp32 on the ordinary ALUs; the bound is their FMA rate: 148 SMs x 128 lanes x 2 FLOP x the SM clock."""
+    With a workspace: the tensor-core kernel (three-way split bf16 operands, so 3x to 6x the algorithmic products are
+    executed); without: the fp32 kernel on the ordinary ALUs, bounded by 148 SMs x 128 lanes x 2 FLOP x the SM clock."""
     cfg = synth.CONFIGS["C2"]
     x = device_inputs(cfg, 7, torch)
     d, H = cfg.d, cfg.H
@@ -369,21 +370,35 @@ def _extra_s(out, torch, lte, synth, pk, flush, n5):
     c = lte.conv_stack(wl, wout)
     s = lte.shape(cfg.B, cfg.H, cfg.T, cfg.d, cfg.W, cfg.R, lte.BF16)
     z = torch.empty((cfg.B, cfg.H, cfg.T), dtype=torch.float32, device="cuda")
+    ws = torch.empty(lte.lte_workspace_bytes(lte.OP_SCORES, s, c), dtype=torch.uint8, device="cuda")
 
-    def f():
-        lte.lte_scores(s, c, x["k"], x["v"], z=z)
+    def f_tc():
+        lte.lte_scores(s, c, x["k"], x["v"], z=z, ws=ws)
 
-    ms, _ = timed(torch, f, n5, 3, flush)
-    t = mid3(ms) * 1e-3
+    def f_alu():
+        lte.lte_scores(s, c, x["k"], x["v"], z=z, ws=False)
+
+    t_tc = mid3(timed(torch, f_tc, n5, 3, flush)[0]) * 1e-3
+    kept = float((z[:, :, : cfg.T - 6] > 0).float().mean())
+    z_tc = z.clone()
+    t_alu = mid3(timed(torch, f_alu, n5, 3, flush)[0]) * 1e-3
+    dz = (z_tc - z)[:, :, : cfg.T - 6].abs().max()
     macs = 3 * (ch[0] * ch[1] + ch[1] * ch[2] + ch[2] * ch[3]) + ch[3]
+    macs_exec = 3 * (3 * ch[0] * ch[1] + 6 * ch[1] * ch[2] + 6 * ch[2] * ch[3])      # weight pieces x activation pieces
     fl = 2.0 * macs * cfg.B * cfg.H * cfg.T
     props = torch.cuda.get_device_properties(0)
     alu_peak = props.multi_processor_count * 128 * 2 * 1.965e9
-    out["S_scorer_stack"] = {"workload": "C2 shape, 3 conv layers k=3 dil=2, channels 128 -> 64 -> 32 -> 16 -> 1",
-                             "scores_ms": t * 1e3, "tokens_per_s": cfg.B * cfg.T / t, "algorithmic_tflops": fl / t / 1e12,
-                             "roofline": {"bound": "alu", "achieved": fl / t / 1e12, "peak": alu_peak / 1e12, "unit": "TFLOP/s",
-                                          "frac": fl / t / alu_peak, "peak_source": "SMs x 128 fp32 lanes x 2 x 1.965 GHz"},
-                             "fraction_kept": float((z[:, :, : cfg.T - 6] > 0).float().mean())}
+    out["S_scorer_stack"] = {
+        "workload": "C2 shape, 3 conv layers k=3 dil=2, channels 128 -> 64 -> 32 -> 16 -> 1",
+        "scores_ms": t_tc * 1e3, "tokens_per_s": cfg.B * cfg.T / t_tc, "algorithmic_tflops": fl / t_tc / 1e12,
+        "executed_tflops": fl / t_tc / 1e12 * macs_exec / macs,
+        "roofline": {"bound": "tensor", "achieved": fl / t_tc / 1e12, "peak": pk["bf16_tflops"], "unit": "TFLOP/s",
+                     "frac": fl / t_tc / 1e12 / pk["bf16_tflops"], "peak_source": pk["source"],
+                     "note": "algorithmic products; every one is executed 3 to 6 times over (split operands)"},
+        "fp32_alu_kernel": {"scores_ms": t_alu * 1e3,
+                            "roofline": {"bound": "alu", "achieved": fl / t_alu / 1e12, "peak": alu_peak / 1e12, "unit": "TFLOP/s",
+                                         "frac": fl / t_alu / alu_peak, "peak_source": "SMs x 128 fp32 lanes x 2 x 1.965 GHz"}},
+        "max_abs_z_difference_between_kernels": float(dz), "fraction_kept": kept}
     del x, z
 
 

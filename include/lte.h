@@ -62,6 +62,10 @@ typedef struct lte_conv {
  *   w    = wl0 [H, d, 3, 2d] | wl1 [H, d/2, 3, d] | wl2 [H, d/4, 3, d/2] | wout [H, d/4]    (one fp32 buffer, 16-byte aligned;
  *          wl[o][tau][c] multiplies channel c of the input at time t - (2 - tau) * 2)
  *   bias = bl0 [H, d] | bl1 [H, d/2] | bl2 [H, d/4] | bout [H], or NULL for zero.
+ * With bf16 inputs, d = 64, T > 12 and a workspace of lte_workspace_bytes(LTE_OP_SCORES, s, c) bytes (128-byte
+ * aligned; it receives the weights split into bf16 pieces, rebuilt by every call) the stack runs on the tensor cores
+ * with exact products and fp32 accumulation; without the workspace, and for every other accepted shape, on the fp32
+ * ALUs.  Both agree with an fp64 evaluation to about 1e-5 at |z| of a few units.
  * The other entry points (decode, backward, cache_init) take the single layer only and answer LTE_ERR_UNSUPPORTED.
  */
 
@@ -90,6 +94,7 @@ const char* lte_strerror(int status);
  *   k, v      in   [B,H,T,d] of s->dtype
  *   z         out  [B,H,T] fp32
  *   r_or_null out  [B,H,T] fp32 sigmoid(z) (0 where z = -inf), or NULL
+ *   ws, ws_bytes   device scratch, used by the three-layer stack only (see lte_conv); may be NULL, 0
  * Errors: INVALID_ARG (NULL, even K, n_layers != 1, dilation != 1, d not in {32,64,128}).
  */
 int lte_scores(const lte_shape* s, const lte_conv* c, const void* k, const void* v,

@@ -25,7 +25,7 @@
 namespace lte {
 
 __device__ int g_stack_tc_status = 0;
-#ifdef ST_PROFILE
+#ifdef LTE_PROFILE
 __device__ long long g_stprof[64];
 #define STP(i) do { if (blockIdx.x == 3 && it == 5 && lane == 0) g_stprof[i] = clock64(); } while (0)
 #else
@@ -557,12 +557,8 @@ int launch_scores_stack_tc(const Params& p, const void* k, const void* v, float*
 
 }  // namespace lte
 
-#if defined(ST_PROFILE) || defined(ST_RAW)
-namespace lte { int prefill_status_fetch_and_clear(); int decode_status_fetch_and_clear(); int scores_status_fetch_and_clear(); int bwd_status_fetch_and_clear(); int decode_tc_status_fetch_and_clear(); }
-extern "C" void lte_status_all(int* o) { o[0] = lte::prefill_status_fetch_and_clear(); o[1] = lte::decode_status_fetch_and_clear(); o[2] = lte::scores_status_fetch_and_clear(); o[3] = lte::bwd_status_fetch_and_clear(); o[4] = lte::decode_tc_status_fetch_and_clear(); o[5] = lte::stack_tc_status_fetch_and_clear(); }
+#ifdef LTE_PROFILE
 extern "C" int lte_stack_status_raw() { return lte::stack_tc_status_fetch_and_clear(); }
-#endif
-#ifdef ST_PROFILE
 extern "C" int lte_stprof_read(long long* out)
 {
     return cudaMemcpyFromSymbol(out, lte::g_stprof, sizeof(long long) * 64) == cudaSuccess ? 0 : -1;
