@@ -461,7 +461,54 @@ def _extra_p(out, torch, lte, synth, pk, flush, n5):
                            "mean_retained": float(cnt.float().mean()), "max_retained": int(cnt.max()),
                            "decode_us_per_step": dec_us, "decode_hbm_gbs": dec_bytes / dec_us / 1e3,
                            "decode_hbm_frac": dec_bytes / dec_us / 1e3 / pk["hbm_gbs"]}
-    del x, o, lse, z, z0, cache
+    del o, lse, z, z0, cache
+    # the same serving shape with grouped queries as in the paper's models: 32 query heads on 8 key/value heads
+    G, Hk = 4, 8
+    sg = lte.shape(cfg.B, Hk, cfg.T, cfg.d, cfg.W, cfg.R, lte.BF16, sink=cfg.sink, group=G)
+    kg, vg = x["k"][:, :Hk].contiguous(), x["v"][:, :Hk].contiguous()
+    cg = lte.conv(x["w"][:Hk].contiguous(), beta[:Hk].contiguous())
+    gq = torch.Generator(device="cuda"); gq.manual_seed(62)
+    qg = (torch.randn((cfg.B, Hk * G, cfg.T, cfg.d), generator=gq, device="cuda") * sc).to(torch.bfloat16)
+    del x
+    zg = lte.lte_scores(sg, cg, kg, vg)
+    idxg, cntg = lte.lte_select(sg, zg)
+    og = torch.empty_like(qg); lseg = torch.empty((cfg.B, Hk * G, cfg.T), dtype=torch.float32, device="cuda")
+
+    def step_g():
+        lte.lte_scores(sg, cg, kg, vg, z=zg)
+        lte.lte_select(sg, zg, idx=idxg, cnt=cntg)
+        lte.lte_attn_prefill(sg, qg, kg, vg, idxg, cntg, o=og, lse=lseg)
+
+    def attn_g():
+        lte.lte_attn_prefill(sg, qg, kg, vg, idxg, cntg, o=og, lse=lseg)
+
+    tg, tag = mid3(timed(torch, step_g, n5, 3, flush)[0]) * 1e-3, mid3(timed(torch, attn_g, n5, 3, flush)[0]) * 1e-3
+    flg = attn_flops(idxg, cntg, cfg.T, cfg.W, cfg.d, torch) * G
+    cache = lte.lte_cache_init(sg, cg, kg, vg, zg, idxg, cntg)
+    qs = (torch.randn((n_dec, cfg.B, Hk * G, cfg.d), generator=gq, device="cuda") * sc).to(torch.bfloat16)
+    o1 = torch.empty((cfg.B, Hk * G, cfg.d), dtype=torch.bfloat16, device="cuda")
+    l1 = torch.empty((cfg.B, Hk * G), dtype=torch.float32, device="cuda")
+    ks8, vs8 = ks[:, :, :Hk].contiguous(), vs[:, :, :Hk].contiguous()
+    for i in range(8):
+        lte.lte_attn_decode(sg, cg, cache, qs[i], ks8[i], vs8[i], o1=o1, lse1=l1)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        for i in range(8, n_dec):
+            lte.lte_attn_decode(sg, cg, cache, qs[i], ks8[i], vs8[i], o1=o1, lse1=l1)
+    reps = []
+    for _ in range(5):
+        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+        e0.record(); graph.replay(); e1.record()
+        torch.cuda.synchronize()
+        reps.append(e0.elapsed_time(e1) * 1e3 / (n_dec - 8))
+    out["P_paper_like"]["grouped_queries"] = {
+        "workload": "the same with 32 query heads on 8 key/value heads (group = 4)",
+        "step_ms": tg * 1e3, "tokens_per_s": cfg.B * cfg.T / tg, "attn_ms": tag * 1e3,
+        "attn_algorithmic_tflops": flg / tag / 1e12, "attn_tensor_frac": flg / tag / 1e12 / pk["bf16_tflops"],
+        "decode_us_per_step": mid3(reps),
+        "note": "decode: the step kernel serves the first query head of a group, a second kernel the other three"}
+    del og, lseg, zg, cache, qg
 
 
 def _extra_c3(out, torch, lte, synth, pk, flush, n5):

@@ -45,6 +45,10 @@ typedef struct lte_shape {
     float   tau;                   /* keep threshold on r; 0.5 in the paper.  tau <= 0 keeps every scored token */
     float   softmax_scale;         /* <= 0 selects 1/sqrt(d)                                               */
     int32_t dtype;                 /* LTE_F32 or LTE_BF16: storage type of q, k, v, o and their gradients   */
+    int32_t group;                 /* grouped-query attention: query heads per key/value head; 0 or 1 = one.
+                                      H counts key/value heads (k, v, z, idx, cnt, the cache); q, o, lse have
+                                      H * group heads, those of one key/value head adjacent: [B, H, group, ...].
+                                      lte_attn_prefill and lte_attn_decode; the backward answers UNSUPPORTED      */
 } lte_shape;
 
 typedef struct lte_conv {
@@ -120,10 +124,12 @@ int lte_select(const lte_shape* s, const float* z, int32_t* idx, int32_t* cnt,
  * A_i = {max(0,i-W+1) .. i}  U  {j in idx[b,h,:cnt] : j <= i-W}:
  *   o_i = softmax_{j in A_i}(scale * q_i.k_j) v_j,   lse_i = log sum_{j in A_i} exp(scale * q_i.k_j).
  * bf16: tensor-core MMA with fp32 accumulation and fp32 softmax, o rounded to bf16.  fp32: fp32 throughout.
- *   q, k, v  in   [B,H,T,d] of s->dtype
+ *   q        in   [B,H*group,T,d] of s->dtype (group = 1 unless s->group says otherwise: query heads
+ *                 h*group .. h*group+group-1 attend over key/value head h and its list)
+ *   k, v     in   [B,H,T,d] of s->dtype
  *   idx, cnt in   as written by lte_select (idx ascending; entries >= cnt ignored)
- *   o        out  [B,H,T,d] of s->dtype
- *   lse      out  [B,H,T] fp32 (natural log)
+ *   o        out  [B,H*group,T,d] of s->dtype
+ *   lse      out  [B,H*group,T] fp32 (natural log)
  * Errors: INVALID_ARG, UNSUPPORTED (d not in {32,64,128}), CUDA.
  */
 int lte_attn_prefill(const lte_shape* s, const void* q, const void* k, const void* v,
@@ -165,8 +171,10 @@ int lte_cache_init(const lte_shape* s, const lte_conv* c, const void* k, const v
  *   3. the newest token whose receptive field is now complete, j = n-half, is scored from the ring;
  *   4. o1, lse1 = attention of q1 over the ring (min(n+1, W) entries) and the pool.
  *   cache        in/out
- *   q1, k1, v1   in   [B,H,d] of s->dtype
- *   o1           out  [B,H,d] of s->dtype;   lse1 out [B,H] fp32
+ *   q1           in   [B,H*group,d] of s->dtype;   k1, v1 in [B,H,d]
+ *   o1           out  [B,H*group,d] of s->dtype;   lse1 out [B,H*group] fp32
+ *   With group > 1 the cache update and the first query head of every group run in the step kernel, the other
+ *   query heads in a second kernel over the updated cache.
  * s->T is ignored.  Errors: INVALID_ARG, UNSUPPORTED (W + R > 4096, d not in {32,64,128}), CUDA.
  */
 int lte_attn_decode(const lte_shape* s, const lte_conv* c, void* cache,

@@ -13,6 +13,7 @@ constexpr int kMaxTaps = 13;          // scorer taps the kernels are instantiate
 
 struct Params {                       // validated, host-resolved view of lte_shape / lte_conv
     int B, H, T, d, W, R, sink, K, half;
+    int G;                            // query heads per key/value head (q, o, lse have H * G heads)
     float zthr;                       // logit(tau): keep iff z > zthr
     float scale;                      // softmax scale
     int dtype;

@@ -36,7 +36,7 @@ __global__ void __launch_bounds__(DT) decode_kernel(unsigned char* __restrict__ 
                                                     const T* __restrict__ v1, T* __restrict__ o1,
                                                     float* __restrict__ lse1, const float* __restrict__ cw,
                                                     const float* __restrict__ cbias, int H, int W, int R, int sink,
-                                                    int K, float zthr, float scale)
+                                                    int K, float zthr, float scale, int G)
 {
     constexpr int EPV = V16<T>::N;            // elements per 16-byte vector
     constexpr int LPR = D / EPV;              // lanes per row
@@ -63,7 +63,7 @@ __global__ void __launch_bounds__(DT) decode_kernel(unsigned char* __restrict__ 
     // query segment of this thread (pre-scaled)
     float qf[EPV];
     {
-        uint4 u = *reinterpret_cast<const uint4*>(q1 + (size_t)bh * D + seg * EPV);
+        uint4 u = *reinterpret_cast<const uint4*>(q1 + (size_t)bh * G * D + seg * EPV);
         unpack<T>(u, qf);
 #pragma unroll
         for (int e = 0; e < EPV; ++e) qf[e] *= scale;
@@ -141,7 +141,7 @@ __global__ void __launch_bounds__(DT) decode_kernel(unsigned char* __restrict__ 
     // logit of the incoming token (row index `rows`)
     if (wid == 1) {
         float s = 0.f;
-        for (int c = lane; c < D; c += 32) s = fmaf(to_f(q1[(size_t)bh * D + c]) * scale, to_f(k1[(size_t)bh * D + c]), s);
+        for (int c = lane; c < D; c += 32) s = fmaf(to_f(q1[(size_t)bh * G * D + c]) * scale, to_f(k1[(size_t)bh * D + c]), s);
         s = warp_sum(s);
         if (lane == 0) s_log[rows] = s;
     }
@@ -250,9 +250,9 @@ __global__ void __launch_bounds__(DT) decode_kernel(unsigned char* __restrict__ 
 #pragma unroll
         for (int w2 = 0; w2 < DT / 32; ++w2) o += s_red[w2][tid];
         o = fmaf(s_log[rows], to_f(v1[(size_t)bh * D + tid]), o);
-        o1[(size_t)bh * D + tid] = from_f<T>(o * inv);
+        o1[(size_t)bh * G * D + tid] = from_f<T>(o * inv);
     }
-    if (tid == 0) lse1[bh] = mx + logf(sum);
+    if (tid == 0) lse1[(size_t)bh * G] = mx + logf(sum);
 
     // ---- write-back ---------------------------------------------------------------------------
     uint4* Kw = reinterpret_cast<uint4*>(blk + L.off_k);
@@ -331,7 +331,7 @@ __global__ void __launch_bounds__(DT) decode_bulk_kernel(unsigned char* __restri
                                                          const T* __restrict__ v1, T* __restrict__ o1,
                                                          float* __restrict__ lse1, const float* __restrict__ cw,
                                                          const float* __restrict__ cbias, int BH, int per_cta, int H,
-                                                         int W, int R, int sink, int K, float zthr, float scale)
+                                                         int W, int R, int sink, int K, float zthr, float scale, int G)
 {
     constexpr int EPV = V16<T>::N;
     constexpr int LPR = D / EPV;
@@ -375,13 +375,13 @@ __global__ void __launch_bounds__(DT) decode_bulk_kernel(unsigned char* __restri
     uint4 kv_new = make_uint4(0, 0, 0, 0);
     auto fetch_inputs = [&](int bh) {
         const int h = bh % H;
-        uint4 u = *reinterpret_cast<const uint4*>(q1 + (size_t)bh * D + seg * EPV);
+        uint4 u = *reinterpret_cast<const uint4*>(q1 + (size_t)bh * G * D + seg * EPV);
         unpack<T>(u, qf);
 #pragma unroll
         for (int c = 0; c < CPL; ++c) {
             k1f[c] = to_f(k1[(size_t)bh * D + lane + 32 * c]);
             v1f[c] = to_f(v1[(size_t)bh * D + lane + 32 * c]);
-            q1f[c] = to_f(q1[(size_t)bh * D + lane + 32 * c]);
+            q1f[c] = to_f(q1[(size_t)bh * G * D + lane + 32 * c]);
         }
 #pragma unroll
         for (int u2 = 0; u2 < 2; ++u2) {
@@ -583,9 +583,9 @@ __global__ void __launch_bounds__(DT) decode_bulk_kernel(unsigned char* __restri
 #pragma unroll
             for (int w2 = 0; w2 < DT / 32; ++w2) o += s_red[w2][tid];
             o = fmaf(p_new, v1_mine, o);
-            o1[(size_t)bh * D + tid] = from_f<T>(o / sum);
+            o1[(size_t)bh * G * D + tid] = from_f<T>(o / sum);
         }
-        if (tid == 0) lse1[bh] = mx + logf(sum);
+        if (tid == 0) lse1[(size_t)bh * G] = mx + logf(sum);
 
         // ---- write-back: only what changed goes to HBM -----------------------------------------------------
         uint4* Kw = reinterpret_cast<uint4*>(gblk + L.off_k);
@@ -686,8 +686,128 @@ int launch_cache_init(const Params& p, const void* k, const void* v, const float
     return cuda_status(cudaGetLastError());
 }
 
-int launch_decode(const Params& p, void* cache, const void* q1, const void* k1, const void* v1, void* o1, float* lse1,
-                  cudaStream_t st)
+// ---- grouped-query attention: the other query heads of a key/value head -------------------------------------------
+// The step kernels above update the cache of a key/value head and attend for its first query head.  The remaining
+// G - 1 query heads attend over the updated block (ring rows of the min(n, W) newest tokens, cnt pool rows) here:
+// one block per key/value head, up to ATT_Q query heads per pass.  The warps take the rows in turn (lanes over the d
+// channels): logits into shared memory, block max and sum per query head, then the value rows weighted per query
+// head in registers and a reduction over the warps.
+constexpr int ATT_Q = 4;
+template <typename T, int D>
+__global__ void __launch_bounds__(DT) decode_attend_kernel(const unsigned char* __restrict__ cache, CacheLayout L,
+                                                           const T* __restrict__ q1, T* __restrict__ o1,
+                                                           float* __restrict__ lse1, int W, int G, float scale)
+{
+    constexpr int C = D / 32, NW = DT / 32;
+    extern __shared__ float att_sm[];                          // logits [ATT_Q][rows], then partial outputs [NW][ATT_Q][D]
+    __shared__ float s_red[NW][ATT_Q];
+    __shared__ float s_mx[ATT_Q], s_sum[ATT_Q];
+    const int bh = blockIdx.x, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const unsigned char* blk = cache + L.header + (size_t)bh * L.stride;
+    const T* Kc = reinterpret_cast<const T*>(blk + L.off_k);
+    const T* Vc = reinterpret_cast<const T*>(blk + L.off_v);
+    const int32_t* meta = reinterpret_cast<const int32_t*>(blk + L.off_meta);
+    const int n = meta[0], cnt = meta[1];
+    const int n_ring = n < W ? n : W, rows = n_ring + cnt;
+    float* s_log = att_sm;
+    float* s_out = att_sm + (size_t)ATT_Q * rows;
+    // element (r, ch): in the swizzled layout (bf16, d = 64) 16-byte chunk ch / 8 of row r sits at position (ch / 8) ^ (r & 7)
+    auto pos_of = [&](int r, int ch) { return L.swz ? ((((ch >> 3) ^ (r & 7)) << 3) | (ch & 7)) : ch; };
+    for (int g0 = 1; g0 < G; g0 += ATT_Q) {
+        const int nq = G - g0 < ATT_Q ? G - g0 : ATT_Q;
+        float qv[ATT_Q][C];
+#pragma unroll
+        for (int u = 0; u < ATT_Q; ++u)
+#pragma unroll
+            for (int c = 0; c < C; ++c)
+                qv[u][c] = u < nq ? to_f(q1[((size_t)bh * G + g0 + u) * D + lane + 32 * c]) * scale : 0.f;
+        // ---- logits ----
+        float mx[ATT_Q];
+#pragma unroll
+        for (int u = 0; u < ATT_Q; ++u) mx[u] = -INFINITY;
+        for (int a = wid; a < rows; a += NW) {
+            const int r = a < n_ring ? a : W + (a - n_ring);
+            float kk[C];
+#pragma unroll
+            for (int c = 0; c < C; ++c) kk[c] = to_f(Kc[(size_t)r * D + pos_of(r, lane + 32 * c)]);
+#pragma unroll
+            for (int u = 0; u < ATT_Q; ++u) {
+                float sdot = 0.f;
+#pragma unroll
+                for (int c = 0; c < C; ++c) sdot = fmaf(qv[u][c], kk[c], sdot);
+                sdot = warp_sum(sdot);
+                mx[u] = fmaxf(mx[u], sdot);
+                if (lane == 0) s_log[(size_t)u * rows + a] = sdot;
+            }
+        }
+        if (lane == 0)
+#pragma unroll
+            for (int u = 0; u < ATT_Q; ++u) s_red[wid][u] = mx[u];
+        __syncthreads();
+        if (tid < ATT_Q) {
+            float m = -INFINITY;
+            for (int w2 = 0; w2 < NW; ++w2) m = fmaxf(m, s_red[w2][tid]);
+            s_mx[tid] = m;
+        }
+        __syncthreads();
+        // ---- probabilities in place, their sums ----
+        float ps[ATT_Q];
+#pragma unroll
+        for (int u = 0; u < ATT_Q; ++u) {
+            ps[u] = 0.f;
+            const float m = s_mx[u];
+            for (int a = tid; a < rows; a += DT) {
+                const float pj = expf(s_log[(size_t)u * rows + a] - m);
+                s_log[(size_t)u * rows + a] = pj;
+                ps[u] += pj;
+            }
+            ps[u] = warp_sum(ps[u]);
+        }
+        if (lane == 0)
+#pragma unroll
+            for (int u = 0; u < ATT_Q; ++u) s_red[wid][u] = ps[u];
+        __syncthreads();
+        if (tid < ATT_Q) {
+            float t = 0.f;
+            for (int w2 = 0; w2 < NW; ++w2) t += s_red[w2][tid];
+            s_sum[tid] = t;
+        }
+        // ---- weighted value rows ----
+        float acc[ATT_Q][C];
+#pragma unroll
+        for (int u = 0; u < ATT_Q; ++u)
+#pragma unroll
+            for (int c = 0; c < C; ++c) acc[u][c] = 0.f;
+        for (int a = wid; a < rows; a += NW) {
+            const int r = a < n_ring ? a : W + (a - n_ring);
+            float vv[C];
+#pragma unroll
+            for (int c = 0; c < C; ++c) vv[c] = to_f(Vc[(size_t)r * D + pos_of(r, lane + 32 * c)]);
+#pragma unroll
+            for (int u = 0; u < ATT_Q; ++u) {
+                const float pj = s_log[(size_t)u * rows + a];
+#pragma unroll
+                for (int c = 0; c < C; ++c) acc[u][c] = fmaf(pj, vv[c], acc[u][c]);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < ATT_Q; ++u)
+#pragma unroll
+            for (int c = 0; c < C; ++c) s_out[((size_t)wid * ATT_Q + u) * D + lane + 32 * c] = acc[u][c];
+        __syncthreads();
+        for (int e = tid; e < nq * D; e += DT) {
+            const int u = e / D, ch = e - u * D;
+            float t = 0.f;
+            for (int w2 = 0; w2 < NW; ++w2) t += s_out[((size_t)w2 * ATT_Q + u) * D + ch];
+            o1[((size_t)bh * G + g0 + u) * D + ch] = from_f<T>(t / s_sum[u]);
+        }
+        if (tid < nq) lse1[(size_t)bh * G + g0 + tid] = s_mx[tid] + logf(s_sum[tid]);
+        __syncthreads();                                       // the buffers are rewritten by the next pass
+    }
+}
+
+static int launch_decode_step(const Params& p, void* cache, const void* q1, const void* k1, const void* v1, void* o1, float* lse1,
+                              cudaStream_t st)
 {
     if (p.W + p.R > MAX_ROWS) return LTE_ERR_UNSUPPORTED;
     const CacheLayout L = cache_layout(p.d, p.W, p.R, p.dtype);
@@ -716,7 +836,7 @@ int launch_decode(const Params& p, void* cache, const void* q1, const void* k1, 
         }                                                                                                         \
         decode_bulk_kernel<T, D><<<n_cta, DT, bulk_smem, st>>>((unsigned char*)cache, L, (const T*)q1,             \
             (const T*)k1, (const T*)v1, (T*)o1, lse1, p.w, p.bias, BH, per_cta, p.H, p.W, p.R, p.sink, p.K,        \
-            p.zthr, p.scale);                                                                                     \
+            p.zthr, p.scale, p.G);                                                                                     \
     } while (0)
     if (bulk) {
         if (p.dtype == LTE_BF16) {
@@ -740,7 +860,7 @@ int launch_decode(const Params& p, void* cache, const void* q1, const void* k1, 
 #define LTE_GO(T, D)                                                                                              \
     decode_kernel<T, D><<<p.B * p.H, DT, 0, st>>>((unsigned char*)cache, L, (const T*)q1, (const T*)k1, (const T*)v1, \
                                                   (T*)o1, lse1, p.w, p.bias, p.H, p.W, p.R, p.sink, p.K, p.zthr,   \
-                                                  p.scale)
+                                                  p.scale, p.G)
     if (p.dtype == LTE_BF16) {
         switch (p.d) {
             case 32: LTE_GO(__nv_bfloat16, 32); break;
@@ -757,6 +877,44 @@ int launch_decode(const Params& p, void* cache, const void* q1, const void* k1, 
         }
     }
 #undef LTE_GO
+    return cuda_status(cudaGetLastError());
+}
+
+int launch_decode(const Params& p, void* cache, const void* q1, const void* k1, const void* v1, void* o1, float* lse1,
+                  cudaStream_t st)
+{
+    int e = launch_decode_step(p, cache, q1, k1, v1, o1, lse1, st);
+    if (e != LTE_OK || p.G <= 1) return e;
+    const CacheLayout L = cache_layout(p.d, p.W, p.R, p.dtype);
+    const size_t att_smem = sizeof(float) * ((size_t)ATT_Q * (p.W + p.R) + (size_t)(DT / 32) * ATT_Q * p.d);
+#define LTE_ATT(T, D)                                                                                                  \
+    do {                                                                                                               \
+        static bool attr_done = false;                                                                                 \
+        if (!attr_done) {                                                                                              \
+            if (cudaFuncSetAttribute(decode_attend_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,           \
+                                     (int)(sizeof(float) * ((size_t)ATT_Q * MAX_ROWS + (DT / 32) * ATT_Q * 128))) != cudaSuccess) \
+                return LTE_ERR_CUDA;                                                                                   \
+            attr_done = true;                                                                                          \
+        }                                                                                                              \
+        decode_attend_kernel<T, D><<<p.B * p.H, DT, att_smem, st>>>((const unsigned char*)cache, L, (const T*)q1,       \
+                                                                    (T*)o1, lse1, p.W, p.G, p.scale);                  \
+    } while (0)
+    if (p.dtype == LTE_BF16) {
+        switch (p.d) {
+            case 32: LTE_ATT(__nv_bfloat16, 32); break;
+            case 64: LTE_ATT(__nv_bfloat16, 64); break;
+            case 128: LTE_ATT(__nv_bfloat16, 128); break;
+            default: return LTE_ERR_UNSUPPORTED;
+        }
+    } else {
+        switch (p.d) {
+            case 32: LTE_ATT(float, 32); break;
+            case 64: LTE_ATT(float, 64); break;
+            case 128: LTE_ATT(float, 128); break;
+            default: return LTE_ERR_UNSUPPORTED;
+        }
+    }
+#undef LTE_ATT
     return cuda_status(cudaGetLastError());
 }
 

@@ -54,7 +54,7 @@ __global__ void __launch_bounds__(NTHR) decode_tc_kernel(unsigned char* __restri
                                                          __nv_bfloat16* __restrict__ o1, float* __restrict__ lse1,
                                                          const float* __restrict__ cw, const float* __restrict__ cbias,
                                                          int BH, int per_cta, int H, int W, int R, int sink, int K,
-                                                         float zthr, float scale)
+                                                         float zthr, float scale, int G)
 {
     extern __shared__ __align__(1024) unsigned char dsm[];
     const Plan P = plan_of(L);
@@ -138,7 +138,7 @@ __global__ void __launch_bounds__(NTHR) decode_tc_kernel(unsigned char* __restri
             for (int c = 0; c < CPL; ++c) {
                 k1f[c] = __bfloat162float(k1[(size_t)bh * D + lane + 32 * c]);
                 v1f[c] = __bfloat162float(v1[(size_t)bh * D + lane + 32 * c]);
-                q1f[c] = __bfloat162float(q1[(size_t)bh * D + lane + 32 * c]);
+                q1f[c] = __bfloat162float(q1[(size_t)bh * G * D + lane + 32 * c]);
             }
 #pragma unroll
             for (int u2 = 0; u2 < 2; ++u2) {
@@ -151,7 +151,7 @@ __global__ void __launch_bounds__(NTHR) decode_tc_kernel(unsigned char* __restri
             }
             bias = cbias ? cbias[h] : 0.f;
             if (tid < D) v1_mine = __bfloat162float(v1[(size_t)bh * D + tid]);
-            if (tid < 8) q_chunk = *reinterpret_cast<const uint4*>(q1 + (size_t)bh * D + tid * 8);
+            if (tid < 8) q_chunk = *reinterpret_cast<const uint4*>(q1 + (size_t)bh * G * D + tid * 8);
             if (tid >= 64 && tid < 80) {
                 const int t2 = tid - 64;
                 kv_new = *reinterpret_cast<const uint4*>((t2 < 8 ? k1 : v1) + (size_t)bh * D + (t2 & 7) * 8);
@@ -292,9 +292,9 @@ __global__ void __launch_bounds__(NTHR) decode_tc_kernel(unsigned char* __restri
             for (int w2 = 0; w2 < 8; ++w2) sum += s_sum[w2];
             if (tid < D) {
                 const float o = s_o[tid] + s_o[64 + tid] + p_new * v1_mine;
-                o1[(size_t)bh * D + tid] = __float2bfloat16_rn(o / sum);
+                o1[(size_t)bh * G * D + tid] = __float2bfloat16_rn(o / sum);
             }
-            if (tid == 0) lse1[bh] = mx + logf(sum);
+            if (tid == 0) lse1[(size_t)bh * G] = mx + logf(sum);
 
             // ---- write-back: only what changed goes to HBM (rows are stored swizzled) ----------------------------
             uint4* Kw = reinterpret_cast<uint4*>(gblk + L.off_k);
@@ -356,7 +356,7 @@ int launch_decode_tc(const Params& p, void* cache, const void* q1, const void* k
     const int n_cta = (BH + per_cta - 1) / per_cta;
     return cuda_status(launch_pdl(decode_tc_kernel, dim3(n_cta), dim3(NTHR), P.total, st, (unsigned char*)cache, L, (const __nv_bfloat16*)q1,
                                                    (const __nv_bfloat16*)k1, (const __nv_bfloat16*)v1, (__nv_bfloat16*)o1, lse1,
-                                                   p.w, p.bias, BH, per_cta, p.H, p.W, p.R, p.sink, p.K, p.zthr, p.scale));
+                                                   p.w, p.bias, BH, per_cta, p.H, p.W, p.R, p.sink, p.K, p.zthr, p.scale, p.G));
 }
 
 int decode_tc_status_fetch_and_clear()

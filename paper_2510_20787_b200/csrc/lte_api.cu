@@ -23,12 +23,12 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 int check_shape(const lte_shape* s, bool need_T)
 {
     if (!s) return LTE_ERR_INVALID_ARG;
-    if (s->B <= 0 || s->H <= 0 || s->W <= 0 || s->R < 0 || s->sink < 0) return LTE_ERR_INVALID_ARG;
+    if (s->B <= 0 || s->H <= 0 || s->W <= 0 || s->R < 0 || s->sink < 0 || s->group < 0) return LTE_ERR_INVALID_ARG;
     if (need_T ? s->T <= 0 : s->T < 0) return LTE_ERR_INVALID_ARG;
     if (s->dtype != LTE_F32 && s->dtype != LTE_BF16) return LTE_ERR_INVALID_ARG;
     if (s->d != 32 && s->d != 64 && s->d != 128) return LTE_ERR_UNSUPPORTED;
     if (!(s->tau < 1.0f)) return LTE_ERR_INVALID_ARG;
-    if ((double)s->B * s->H * (double)(s->T > 0 ? s->T : 1) * s->d > 2.0e10) return LTE_ERR_UNSUPPORTED;
+    if ((double)s->B * s->H * (s->group > 1 ? s->group : 1) * (double)(s->T > 0 ? s->T : 1) * s->d > 2.0e10) return LTE_ERR_UNSUPPORTED;
     return LTE_OK;
 }
 
@@ -45,6 +45,7 @@ Params make_params(const lte_shape* s, const lte_conv* c)
 {
     Params p;
     p.B = s->B; p.H = s->H; p.T = s->T; p.d = s->d; p.W = s->W; p.R = s->R; p.sink = s->sink;
+    p.G = s->group > 1 ? s->group : 1;
     p.K = c ? c->kernel : 1; p.half = p.K / 2;
     p.zthr = s->tau <= 0.f ? -INFINITY : (float)(log((double)s->tau) - log1p(-(double)s->tau));
     p.scale = s->softmax_scale > 0.f ? s->softmax_scale : (float)(1.0 / sqrt((double)s->d));
@@ -197,6 +198,7 @@ int lte_attn_bwd(const lte_shape* s, const lte_conv* c, const void* q, const voi
     if (!q || !k || !v || !o || !lse || !dO || !z || !cnt || (s->R > 0 && !idx) || !dq || !dk || !dv || !dw)
         return LTE_ERR_INVALID_ARG;
     if (flags & ~LTE_BWD_CNN_INPUT_GRAD) return LTE_ERR_INVALID_ARG;
+    if (s->group > 1) return LTE_ERR_UNSUPPORTED;          // grouped-query attention: forward and decode only
     Params p = make_params(s, c);
     if (!ws || !aligned16(ws) || ws_bytes < bwd_workspace_bytes(p, flags)) return LTE_ERR_WORKSPACE;
     e = check_arch(); if (e) return e;
@@ -240,6 +242,7 @@ int lte_attn_bwd_static(const lte_shape* s, const lte_conv* c, const void* q, co
     if (!q || !k || !v || !o || !lse || !dO || !z || !cnt || (s->R > 0 && !idx) || !dq || !dk || !dv || !dw)
         return LTE_ERR_INVALID_ARG;
     if (flags & ~LTE_BWD_CNN_INPUT_GRAD) return LTE_ERR_INVALID_ARG;
+    if (s->group > 1) return LTE_ERR_UNSUPPORTED;
     Params p = make_params(s, c);
     if (bwd_workspace_bytes(p, flags) > (size_t)LTE_STATIC_SCRATCH_BYTES) return LTE_ERR_WORKSPACE;   /* too large for the fixed array */
     e = check_arch(); if (e) return e;

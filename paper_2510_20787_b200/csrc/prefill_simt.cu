@@ -11,20 +11,20 @@ template <typename T, int D>
 __global__ void __launch_bounds__(128) prefill_simt_kernel(const T* __restrict__ q, const T* __restrict__ k,
                                                            const T* __restrict__ v, const int32_t* __restrict__ idx,
                                                            const int32_t* __restrict__ cnt, T* __restrict__ o,
-                                                           float* __restrict__ lse, int Tlen, int W, int R, float scale)
+                                                           float* __restrict__ lse, int Tlen, int W, int R, float scale, int G)
 {
     constexpr int C = D / 32;                  // channels per lane
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int i = blockIdx.x * 4 + warp;
-    const int bh = blockIdx.y;
+    const int bh = blockIdx.y, bhk = bh / G;   // query head and its key/value head
     if (i >= Tlen) return;
-    const size_t base = (size_t)bh * Tlen * D;
+    const size_t base = (size_t)bh * Tlen * D, kbase = (size_t)bhk * Tlen * D;
     float qv[C], acc[C];
 #pragma unroll
     for (int c = 0; c < C; ++c) { qv[c] = to_f(q[base + (size_t)i * D + lane + 32 * c]) * scale; acc[c] = 0.f; }
     float m = -INFINITY, l = 0.f;
-    const int32_t* id = idx + (size_t)bh * R;
-    const int n_ret = cnt[bh];
+    const int32_t* id = idx + (size_t)bhk * R;
+    const int n_ret = cnt[bhk];
     const int lo = i - W + 1 > 0 ? i - W + 1 : 0;
     // number of retained entries visible to this query: idx ascending => a prefix
     int nvis = 0;
@@ -37,8 +37,8 @@ __global__ void __launch_bounds__(128) prefill_simt_kernel(const T* __restrict__
     const int total = nvis + (i - lo + 1);
     for (int a = 0; a < total; ++a) {
         const int j = a < nvis ? id[a] : lo + (a - nvis);
-        const T* kr = k + base + (size_t)j * D;
-        const T* vr = v + base + (size_t)j * D;
+        const T* kr = k + kbase + (size_t)j * D;
+        const T* vr = v + kbase + (size_t)j * D;
         float s = 0.f;
 #pragma unroll
         for (int c = 0; c < C; ++c) s = fmaf(qv[c], to_f(kr[lane + 32 * c]), s);
@@ -60,10 +60,10 @@ template <typename T>
 int run(const Params& p, const void* q, const void* k, const void* v, const int32_t* idx, const int32_t* cnt,
         void* o, float* lse, cudaStream_t st)
 {
-    dim3 grid((p.T + 3) / 4, p.B * p.H);
+    dim3 grid((p.T + 3) / 4, p.B * p.H * p.G);
 #define LTE_GO(D)                                                                                          \
     prefill_simt_kernel<T, D><<<grid, 128, 0, st>>>((const T*)q, (const T*)k, (const T*)v, idx, cnt, (T*)o, \
-                                                    lse, p.T, p.W, p.R, p.scale)
+                                                    lse, p.T, p.W, p.R, p.scale, p.G)
     switch (p.d) {
         case 32: LTE_GO(32); break;
         case 64: LTE_GO(64); break;

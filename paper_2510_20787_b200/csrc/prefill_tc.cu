@@ -51,16 +51,17 @@ template <int D> struct Smem {
 
 // One work item: a 128-query tile of one (b,h).
 struct Item {
-    int bh, i0, i_hi, j_start, n_win;
+    int bh, bhk, i0, i_hi, j_start, n_win;              // bh: query head (b, h, g); bhk: its key/value head (b, h)
 };
 // Items are numbered from the last query tile of every (b,h) down to the first: later query tiles see more retained
 // rows and cost more, and a CTA takes items n, n + grid, n + 2 grid, ... so every CTA gets one item of each cost band
 // (largest first), which balances the static schedule.
-__device__ __forceinline__ Item decode_item(int item, int n_qt, int n_bh, int Tlen, int W)
+__device__ __forceinline__ Item decode_item(int item, int n_qt, int n_bh, int Tlen, int W, int G)
 {
     Item it;
     const int r = item / n_bh;
     it.bh = item - r * n_bh;
+    it.bhk = it.bh / G;                                 // the G query heads of a key/value head are adjacent
     it.i0 = (n_qt - 1 - r) * BM;
     it.i_hi = min(it.i0 + BM - 1, Tlen - 1);
     it.j_start = max(it.i0 - W + 1, 0);
@@ -101,7 +102,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                   const __nv_bfloat16* __restrict__ kg,
                   const __nv_bfloat16* __restrict__ vg, const int32_t* __restrict__ idx,
                   const int32_t* __restrict__ cnt, float* __restrict__ lse, int Tlen,
-                  int W, int R, float scale, int n_qt, int n_bh)
+                  int W, int R, float scale, int n_qt, int n_bh, int G)
 {
     const int n_items = n_qt * n_bh;
     using S = Smem<D>;
@@ -162,7 +163,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         uint32_t g = 0;                                        // tiles of the items before this one
         int it = 0;
         for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++it) {
-            const Item w = decode_item(item, n_qt, n_bh, Tlen, W);
+            const Item w = decode_item(item, n_qt, n_bh, Tlen, W, G);
             if (lane == 0) {
                 // Q: its buffer is free once the previous item's last S product has completed
                 if (it > 0) mbar_wait(bar_qf, (it - 1) & 1, 12);
@@ -178,16 +179,16 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     mbar_expect_tx(bar_k0 + 8 * ks, S::KVTILE);
 #pragma unroll
                     for (int sb = 0; sb < SUB; ++sb)
-                        tma_load_3d(sK + ks * S::KVTILE + sb * 8192, &tmK, sb * 64, y, w.bh, bar_k0 + 8 * ks);
+                        tma_load_3d(sK + ks * S::KVTILE + sb * 8192, &tmK, sb * 64, y, w.bhk, bar_k0 + 8 * ks);
                     if (gg >= (uint32_t)VST) mbar_wait(bar_vf0 + 8 * vs, (gg / VST - 1) & 1u, 8);
                     mbar_expect_tx(bar_v0 + 8 * vs, S::KVTILE);
 #pragma unroll
                     for (int sb = 0; sb < SUB; ++sb)
-                        tma_load_3d(sV + vs * S::KVTILE + sb * 8192, &tmV, sb * 64, y, w.bh, bar_v0 + 8 * vs);
+                        tma_load_3d(sV + vs * S::KVTILE + sb * 8192, &tmV, sb * 64, y, w.bhk, bar_v0 + 8 * vs);
                 }
             }
             // the item's retained tiles also take tile numbers (counted after the loads are on their way)
-            g += w.n_win + (count_le(idx + (size_t)w.bh * R, cnt[w.bh], w.i_hi - W, lane) + BN - 1) / BN;
+            g += w.n_win + (count_le(idx + (size_t)w.bhk * R, cnt[w.bhk], w.i_hi - W, lane) + BN - 1) / BN;
         }
     } else if (warp == 4) {
         // ================================= MMA warp (lane 0 issues) =========================================
@@ -205,12 +206,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         // tiles of an item (whole warp: the count of visible list entries takes global loads)
         auto item_tiles = [&](int item) {
             if (item >= n_items) return 0;
-            const Item w = decode_item(item, n_qt, n_bh, Tlen, W);
-            return w.n_win + (count_le(idx + (size_t)w.bh * R, cnt[w.bh], w.i_hi - W, lane) + BN - 1) / BN;
+            const Item w = decode_item(item, n_qt, n_bh, Tlen, W, G);
+            return w.n_win + (count_le(idx + (size_t)w.bhk * R, cnt[w.bhk], w.i_hi - W, lane) + BN - 1) / BN;
         };
         int n_tiles_next = item_tiles(blockIdx.x);
         for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++it) {
-            const Item w = decode_item(item, n_qt, n_bh, Tlen, W);
+            const Item w = decode_item(item, n_qt, n_bh, Tlen, W, G);
             const int n_tiles = n_tiles_next;
             int ts = 0;                                        // S products of this item issued so far
             // gathers issued before the top of tile gg have landed
@@ -281,17 +282,17 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         int pf_cnt = 0, pf_e[4] = {0, 0, 0, 0};
         auto prefetch_list = [&](int item) {
             if (item < n_items) {
-                const Item w = decode_item(item, n_qt, n_bh, Tlen, W);
-                pf_cnt = cnt[w.bh];
+                const Item w = decode_item(item, n_qt, n_bh, Tlen, W, G);
+                pf_cnt = cnt[w.bhk];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) pf_e[u] = u * 32 + lane < R ? idx[(size_t)w.bh * R + u * 32 + lane] : 0x7fffffff;
+                for (int u = 0; u < 4; ++u) pf_e[u] = u * 32 + lane < R ? idx[(size_t)w.bhk * R + u * 32 + lane] : 0x7fffffff;
             }
         };
         prefetch_list(blockIdx.x);
         for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++it) {
-            const Item w = decode_item(item, n_qt, n_bh, Tlen, W);
-            const int bh = w.bh, n_win = w.n_win, j_start = w.j_start;
-            const int32_t* id = idx + (size_t)bh * R;
+            const Item w = decode_item(item, n_qt, n_bh, Tlen, W, G);
+            const int bh = w.bh, bhk = w.bhk, n_win = w.n_win, j_start = w.j_start;
+            const int32_t* id = idx + (size_t)bhk * R;
             const int n_ret = pf_cnt;
             const int i = w.i0 + tid;                          // this thread's query row
             // retained entries visible to this row.  The rows of a warp are consecutive and the list is ascending, so
@@ -344,7 +345,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     for (int ps = 0; ps < 4; ++ps) {
                         const int row = ps * 16 + g_row;
                         const bool ok = rows4[ps] >= 0;
-                        const __nv_bfloat16* src = (is_v ? vg : kg) + ((size_t)bh * Tlen + (ok ? rows4[ps] : 0)) * D;
+                        const __nv_bfloat16* src = (is_v ? vg : kg) + ((size_t)bhk * Tlen + (ok ? rows4[ps] : 0)) * D;
 #pragma unroll
                         for (int c = g_sub; c < D / 8; c += 8) {
                             const uint32_t off = (c >> 3) * 8192 + row * 128 + (((c & 7) ^ (row & 7)) << 4);
@@ -560,8 +561,8 @@ int run(const Params& p, const void* q, const void* k, const void* v, const int3
         float* lse, cudaStream_t st)
 {
     CUtensorMap tq, tk, tv, to;
-    const int BH = p.B * p.H;
-    if (!make_map(&tq, q, BH, p.T, D, BM) || !make_map(&tk, k, BH, p.T, D, BN) || !make_map(&tv, v, BH, p.T, D, BN) ||
+    const int BHK = p.B * p.H, BH = BHK * p.G;                 // key/value heads, query heads
+    if (!make_map(&tq, q, BH, p.T, D, BM) || !make_map(&tk, k, BHK, p.T, D, BN) || !make_map(&tv, v, BHK, p.T, D, BN) ||
         !make_map(&to, o, BH, p.T, D, 32))
         return LTE_ERR_CUDA;
     static int slots = 0;                                      // resident CTAs: two per SM
@@ -579,7 +580,7 @@ int run(const Params& p, const void* q, const void* k, const void* v, const int3
     const int grid = n_items < slots ? n_items : slots;
     return cuda_status(launch_pdl(prefill_tc_kernel<D>, dim3(grid), dim3(NTHREADS), Smem<D>::BYTES, st, tq, tk, tv, to, (const __nv_bfloat16*)k,
                                                                  (const __nv_bfloat16*)v, idx, cnt,
-                                                                 lse, p.T, p.W, p.R, p.scale, n_qt, BH));
+                                                                 lse, p.T, p.W, p.R, p.scale, n_qt, BH, p.G));
 }
 
 }  // namespace

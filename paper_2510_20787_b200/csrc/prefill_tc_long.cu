@@ -58,7 +58,7 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                   const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO, const __nv_bfloat16* __restrict__ kg,
                   const __nv_bfloat16* __restrict__ vg, const int32_t* __restrict__ idx,
                   const int32_t* __restrict__ cnt, __nv_bfloat16* __restrict__ o, float* __restrict__ lse, int Tlen,
-                  int W, int R, float scale)
+                  int W, int R, float scale, int G)
 {
     using S = Smem<D>;
     constexpr int SUB = S::SUB, KST = S::KST, VST = S::VST;
@@ -83,12 +83,12 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(smem_raw + S::OFF_BAR + 152);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int bh = blockIdx.y;
+    const int bh = blockIdx.y, bhk = bh / G;                   // query head and its key/value head (the G query heads of one are adjacent)
     const int i0 = blockIdx.x * BM;
     const int i_hi = min(i0 + BM - 1, Tlen - 1);
     const int j_start = max(i0 - W + 1, 0);
     const int n_win = (i_hi - j_start + 1 + BN - 1) / BN;
-    const int32_t* id = idx + (size_t)bh * R;
+    const int32_t* id = idx + (size_t)bhk * R;
     const int g_first = max(n_win - Smem<D>::KST, 0);        // first tile whose top may have gathers in flight
 
     if (tid == 0) {
@@ -110,7 +110,7 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const uint32_t tmem = *tmem_slot_gen;
     pdl_launch_dependents();
     pdl_wait();                                                // everything above ran beside the previous kernel's tail
-    const int n_ret = cnt[bh];
+    const int n_ret = cnt[bhk];
 
     if (warp >= 4) {
         // ============================ load lane (warp 5) and MMA lane (warp 4) ==============================
@@ -139,13 +139,13 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             for (; tk < KST && tk < n_win; ++tk, y += BN) {
                 mbar_expect_tx(bar_k0 + 8 * tk, S::KVTILE);
 #pragma unroll
-                for (int sb = 0; sb < SUB; ++sb) tma_load_3d(sK + tk * S::KVTILE + sb * 8192, &tmK, sb * 64, y, bh, bar_k0 + 8 * tk);
+                for (int sb = 0; sb < SUB; ++sb) tma_load_3d(sK + tk * S::KVTILE + sb * 8192, &tmK, sb * 64, y, bhk, bar_k0 + 8 * tk);
             }
             y = j_start;
             for (; tv < VST && tv < n_win; ++tv, y += BN) {
                 mbar_expect_tx(bar_v0 + 8 * tv, S::KVTILE);
 #pragma unroll
-                for (int sb = 0; sb < SUB; ++sb) tma_load_3d(sV + tv * S::KVTILE + sb * 8192, &tmV, sb * 64, y, bh, bar_v0 + 8 * tv);
+                for (int sb = 0; sb < SUB; ++sb) tma_load_3d(sV + tv * S::KVTILE + sb * 8192, &tmV, sb * 64, y, bhk, bar_v0 + 8 * tv);
             }
             while (tk < n_win || tv < n_win) {
                 if (tk < n_win) {                              // K(tk) into the stage of K(tk - KST)
@@ -154,7 +154,7 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     mbar_expect_tx(bar_k0 + 8 * ks, S::KVTILE);
 #pragma unroll
                     for (int sb = 0; sb < SUB; ++sb)
-                        tma_load_3d(sK + ks * S::KVTILE + sb * 8192, &tmK, sb * 64, j_start + tk * BN, bh, bar_k0 + 8 * ks);
+                        tma_load_3d(sK + ks * S::KVTILE + sb * 8192, &tmK, sb * 64, j_start + tk * BN, bhk, bar_k0 + 8 * ks);
                     ++tk;
                     ks = ks + 1 == KST ? 0 : ks + 1;
                 }
@@ -164,7 +164,7 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     mbar_expect_tx(bar_v0 + 8 * vs, S::KVTILE);
 #pragma unroll
                     for (int sb = 0; sb < SUB; ++sb)
-                        tma_load_3d(sV + vs * S::KVTILE + sb * 8192, &tmV, sb * 64, j_start + tv * BN, bh, bar_v0 + 8 * vs);
+                        tma_load_3d(sV + vs * S::KVTILE + sb * 8192, &tmV, sb * 64, j_start + tv * BN, bhk, bar_v0 + 8 * vs);
                     ++tv;
                     vs = vs + 1 == VST ? 0 : vs + 1;
                 }
@@ -291,7 +291,7 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 for (int ps = 0; ps < 4; ++ps) {
                     const int row = ps * 16 + g_row;
                     const bool ok = rows4[ps] >= 0;
-                    const __nv_bfloat16* src = (is_v ? vg : kg) + ((size_t)bh * Tlen + (ok ? rows4[ps] : 0)) * D;
+                    const __nv_bfloat16* src = (is_v ? vg : kg) + ((size_t)bhk * Tlen + (ok ? rows4[ps] : 0)) * D;
 #pragma unroll
                     for (int c = g_sub; c < D / 8; c += 8) {
                         const uint32_t off = (c >> 3) * 8192 + row * 128 + (((c & 7) ^ (row & 7)) << 4);
@@ -483,8 +483,8 @@ int run(const Params& p, const void* q, const void* k, const void* v, const int3
         float* lse, cudaStream_t st)
 {
     CUtensorMap tq, tk, tv, to;
-    const int BH = p.B * p.H;
-    if (!make_map(&tq, q, BH, p.T, D, BM) || !make_map(&tk, k, BH, p.T, D, BN) || !make_map(&tv, v, BH, p.T, D, BN) ||
+    const int BHK = p.B * p.H, BH = BHK * p.G;                 // key/value heads, query heads
+    if (!make_map(&tq, q, BH, p.T, D, BM) || !make_map(&tk, k, BHK, p.T, D, BN) || !make_map(&tv, v, BHK, p.T, D, BN) ||
         !make_map(&to, o, BH, p.T, D, 32))
         return LTE_ERR_CUDA;
     static bool attr_done = false;
@@ -497,7 +497,7 @@ int run(const Params& p, const void* q, const void* k, const void* v, const int3
     dim3 grid((p.T + BM - 1) / BM, BH);
     return cuda_status(launch_pdl(prefill_long_kernel<D>, grid, dim3(NTHREADS), Smem<D>::BYTES, st, tq, tk, tv, to, (const __nv_bfloat16*)k,
                                                                  (const __nv_bfloat16*)v, idx, cnt, (__nv_bfloat16*)o,
-                                                                 lse, p.T, p.W, p.R, p.scale));
+                                                                 lse, p.T, p.W, p.R, p.scale, p.G));
 }
 
 }  // namespace

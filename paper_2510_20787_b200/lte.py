@@ -26,7 +26,8 @@ STATIC_SCRATCH_BYTES = 8 << 20
 class LteShape(ctypes.Structure):
     _fields_ = [("B", ctypes.c_int32), ("H", ctypes.c_int32), ("T", ctypes.c_int32), ("d", ctypes.c_int32),
                 ("W", ctypes.c_int32), ("R", ctypes.c_int32), ("sink", ctypes.c_int32),
-                ("tau", ctypes.c_float), ("softmax_scale", ctypes.c_float), ("dtype", ctypes.c_int32)]
+                ("tau", ctypes.c_float), ("softmax_scale", ctypes.c_float), ("dtype", ctypes.c_int32),
+                ("group", ctypes.c_int32)]
 
 
 class LteConv(ctypes.Structure):
@@ -78,8 +79,9 @@ def _dt(t):
     raise TypeError("q/k/v must be float32 or bfloat16")
 
 
-def shape(B, H, T, d, W, R, dtype, sink=0, tau=0.5, softmax_scale=0.0):
-    return LteShape(B, H, T, d, W, R, sink, tau, softmax_scale, dtype)
+def shape(B, H, T, d, W, R, dtype, sink=0, tau=0.5, softmax_scale=0.0, group=1):
+    """H key/value heads; with group > 1 (grouped-query attention) q, o and lse have H * group heads."""
+    return LteShape(B, H, T, d, W, R, sink, tau, softmax_scale, dtype, group)
 
 
 def conv(w, bias=None):
@@ -163,11 +165,11 @@ def lte_select(s, z, idx=None, cnt=None, ncand=None):
 
 
 def lte_attn_prefill(s, q, k, v, idx, cnt, o=None, lse=None):
-    """q, k, v [B,H,T,d], retained list -> o [B,H,T,d], lse [B,H,T] fp32."""
+    """q [B,H*group,T,d], k, v [B,H,T,d], retained list -> o [B,H*group,T,d], lse [B,H*group,T] fp32."""
     if o is None:
         o = torch.empty_like(q)
     if lse is None:
-        lse = torch.empty((s.B, s.H, s.T), dtype=torch.float32, device=q.device)
+        lse = torch.empty((s.B, s.H * max(s.group, 1), s.T), dtype=torch.float32, device=q.device)
     _check("lte_attn_prefill", lib().lte_attn_prefill(ctypes.addressof(s), _ptr(q), _ptr(k), _ptr(v),
                                                       _ptr(idx, torch.int32), _ptr(cnt, torch.int32), _ptr(o),
                                                       _ptr(lse, torch.float32), None, 0, _stream()))
@@ -189,11 +191,12 @@ def lte_cache_init(s, c, k=None, v=None, z=None, idx=None, cnt=None, cache=None)
 
 
 def lte_attn_decode(s, c, cache, q1, k1, v1, o1=None, lse1=None):
-    """One decode step: q1, k1, v1 [B,H,d] -> o1 [B,H,d], lse1 [B,H]; the cache is updated in place."""
+    """One decode step: q1 [B,H*group,d], k1, v1 [B,H,d] -> o1 [B,H*group,d], lse1 [B,H*group]; the cache is
+    updated in place."""
     if o1 is None:
         o1 = torch.empty_like(q1)
     if lse1 is None:
-        lse1 = torch.empty((s.B, s.H), dtype=torch.float32, device=q1.device)
+        lse1 = torch.empty((s.B, s.H * max(s.group, 1)), dtype=torch.float32, device=q1.device)
     _check("lte_attn_decode", lib().lte_attn_decode(ctypes.addressof(s), ctypes.addressof(c), _ptr(cache),
                                                     _ptr(q1), _ptr(k1), _ptr(v1), _ptr(o1),
                                                     _ptr(lse1, torch.float32), _stream()))

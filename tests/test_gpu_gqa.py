@@ -1,0 +1,89 @@
+"""GPU parity with grouped-query attention (several query heads share a key/value head, its retained list and its
+decode cache): lte_attn_prefill and lte_attn_decode against the oracle run per query head on repeated keys/values."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import lte_oracle as orc
+from paper_2510_20787_b200 import lte, synth
+from tests.gpu_util import dev, tdtype
+
+pytestmark = pytest.mark.gpu
+
+TOL = {"bf16": 2e-2, "f32": 1e-4}
+
+
+def _inputs(cfg, G, seed, T=None):
+    """k, v, w for cfg.H key/value heads; q for cfg.H * G query heads (query heads of one key/value head adjacent)."""
+    x = synth.make(cfg, seed, T=T)
+    xq = synth.make(cfg.with_(H=cfg.H * G), seed + 100, T=T)
+    return x, xq["q"]
+
+
+@pytest.mark.parametrize("dtype,d,T,W,R,G", [("bf16", 64, 700, 64, 48, 4), ("bf16", 64, 300, 32, 16, 2), ("bf16", 128, 520, 96, 64, 4),
+                                             ("f32", 32, 200, 16, 12, 3), ("bf16", 32, 260, 24, 10, 2)])
+def test_prefill_gqa(dtype, d, T, W, R, G):
+    cfg = synth.Config("gqa", dtype, 2, 3, d, T, W, R, 7, 0.1, sink=1)
+    x, q = _inputs(cfg, G, 11)
+    s = lte.shape(cfg.B, cfg.H, T, d, W, R, tdtype(cfg), sink=cfg.sink, group=G)
+    c = lte.conv(torch.from_numpy(x["w"]).cuda())
+    k, v = dev(x["k"], dtype), dev(x["v"], dtype)
+    z = lte.lte_scores(s, c, k, v)
+    idx, cnt = lte.lte_select(s, z)
+    o, lse = lte.lte_attn_prefill(s, dev(q, dtype), k, v, idx, cnt)
+    torch.cuda.synchronize()
+    assert lte.lib().lte_device_status() == 0
+    assert o.shape == (cfg.B, cfg.H * G, T, d) and lse.shape == (cfg.B, cfg.H * G, T)
+    rep = lambda a: np.repeat(a, G, axis=1)
+    o64, l64 = orc.attn_prefill(q, rep(x["k"]), rep(x["v"]), rep(idx.cpu().numpy()), rep(cnt.cpu().numpy()), W)
+    assert np.max(np.abs(o.float().cpu().numpy() - o64)) <= TOL[dtype]
+    assert np.max(np.abs(lse.cpu().numpy() - l64)) <= TOL[dtype]
+    # group = 1 through the same entry point gives the plain result for the first query head of every group
+    s1 = lte.shape(cfg.B, cfg.H, T, d, W, R, tdtype(cfg), sink=cfg.sink)
+    o1, _ = lte.lte_attn_prefill(s1, dev(np.ascontiguousarray(q[:, ::G]), dtype), k, v, idx, cnt)
+    assert torch.equal(o1, o[:, ::G].contiguous())
+
+
+@pytest.mark.parametrize("dtype,d,W,R,G,T0,steps", [("bf16", 64, 32, 24, 4, 100, 40), ("bf16", 64, 16, 8, 2, 0, 60), ("bf16", 128, 24, 16, 4, 64, 30),
+                                                    ("f32", 32, 16, 12, 3, 40, 30), ("bf16", 64, 200, 150, 2, 260, 20)])
+def test_decode_gqa(dtype, d, W, R, G, T0, steps):
+    cfg = synth.Config("gqa", dtype, 2, 2, d, T0 + steps, W, R, 7, 0.1)
+    Ttot = T0 + steps
+    x, q = _inputs(cfg, G, 5, T=Ttot)
+    c = lte.conv(torch.from_numpy(x["w"]).cuda())
+    k, v, qd = dev(x["k"], dtype), dev(x["v"], dtype), dev(q, dtype)
+    s0 = lte.shape(cfg.B, cfg.H, T0, d, W, R, tdtype(cfg), group=G)
+    if T0 > 0:
+        kp, vp = k[:, :, :T0].contiguous(), v[:, :, :T0].contiguous()
+        z = lte.lte_scores(s0, c, kp, vp)
+        idx, cnt = lte.lte_select(s0, z)
+        cache = lte.lte_cache_init(s0, c, kp, vp, z, idx, cnt)
+    else:
+        cache = lte.lte_cache_init(s0, c)
+    outs, lses = [], []
+    for n in range(T0, Ttot):
+        o1, l1 = lte.lte_attn_decode(s0, c, cache, qd[:, :, n].contiguous(), k[:, :, n].contiguous(), v[:, :, n].contiguous())
+        outs.append(o1.float().cpu().numpy()); lses.append(l1.cpu().numpy())
+    torch.cuda.synchronize()
+    assert lte.lib().lte_device_status() == 0
+    o_n, l_n = np.stack(outs, axis=2), np.stack(lses, axis=2)
+    assert o_n.shape == (cfg.B, cfg.H * G, steps, d)
+    rep = lambda a: np.repeat(a, G, axis=1)
+    z64 = orc.scores(x["k"], x["v"], x["w"])
+    o64, l64, _, _ = orc.stream(q, rep(x["k"]), rep(x["v"]), rep(z64), W, R, 0, n_from=T0)
+    assert np.max(np.abs(o_n - o64)) <= TOL[dtype], np.max(np.abs(o_n - o64))
+    assert np.max(np.abs(l_n - l64)) <= TOL[dtype]
+
+
+def test_backward_rejects_groups():
+    cfg = synth.Config("gqa", "bf16", 1, 2, 64, 128, 16, 8, 7, 0.1)
+    x, q = _inputs(cfg, 2, 0)
+    s = lte.shape(1, 2, 128, 64, 16, 8, lte.BF16, group=2)
+    c = lte.conv(torch.from_numpy(x["w"]).cuda())
+    k, v, qd = dev(x["k"], "bf16"), dev(x["v"], "bf16"), dev(q, "bf16")
+    z = lte.lte_scores(s, c, k, v)
+    idx, cnt = lte.lte_select(s, z)
+    o, lse = lte.lte_attn_prefill(s, qd, k, v, idx, cnt)
+    with pytest.raises(lte.LteError) as e:
+        lte.lte_attn_bwd(s, c, qd, k, v, o, lse, torch.ones_like(o), z, idx, cnt)
+    assert e.value.status == -2
