@@ -130,6 +130,115 @@ void oracle_scores_stack(int B, int H, int T, int d, int L, int ks, int dil,
 }
 
 /* ------------------------------------------------------------------------- */
+/* Backward of the stack above (Section 3.1.1's scorer under the gradient of
+ * Section 3.1.2): given dL/dz [B,H,T] (zero where the logit is undefined), the
+ * gradients of every layer's weights and biases (summed over the batch), of the
+ * output map, and of the inputs k, v [B,H,T,d].  Plain chain rule, layer by
+ * layer: Swish'(y) = s + y s (1 - s) with s = sigmoid(y); a layer's input at
+ * negative time is the constant zero and receives nothing.                   */
+void oracle_scores_stack_bwd(int B, int H, int T, int d, int L, int ks, int dil,
+                             const int* ch, const double* const* wl, const double* const* bl,
+                             const double* wout, const double* bout,
+                             const double* k, const double* v, const double* dz,
+                             double* const* dwl, double* const* dbl, double* dwout, double* dbout,
+                             double* dk, double* dv)
+{
+    const int half = L * (ks - 1) * dil / 2;
+    int cmax = 0;
+    for (int l = 0; l <= L; ++l) if (ch[l] > cmax) cmax = ch[l];
+    (void)bout;
+    for (int l = 0; l < L; ++l) {
+        memset(dwl[l], 0, sizeof(double) * (size_t)H * ch[l + 1] * ks * ch[l]);
+        memset(dbl[l], 0, sizeof(double) * (size_t)H * ch[l + 1]);
+    }
+    memset(dwout, 0, sizeof(double) * (size_t)H * ch[L]);
+    memset(dbout, 0, sizeof(double) * (size_t)H);
+    /* heads in parallel, the batch in order inside: the sums over b have a fixed order */
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int h = 0; h < H; ++h) {
+        /* act[l]: input of layer l (act[0] = x), pre[l]: pre-activation of layer l */
+        double** act = (double**)malloc(sizeof(double*) * (size_t)(L + 1));
+        double** pre = (double**)malloc(sizeof(double*) * (size_t)L);
+        for (int l = 0; l <= L; ++l) act[l] = (double*)malloc(sizeof(double) * (size_t)T * cmax);
+        for (int l = 0; l < L; ++l) pre[l] = (double*)malloc(sizeof(double) * (size_t)T * cmax);
+        double* g = (double*)malloc(sizeof(double) * (size_t)T * cmax);
+        double* gp = (double*)malloc(sizeof(double) * (size_t)T * cmax);
+        for (int b = 0; b < B; ++b) {
+            const size_t bh = (size_t)b * H + h;
+            const double* kk = k + bh * T * d;
+            const double* vv = v + bh * T * d;
+            const double* dzz = dz + bh * T;
+            for (int t = 0; t < T; ++t) {
+                for (int c = 0; c < d; ++c) act[0][(size_t)t * cmax + c] = kk[(size_t)t * d + c];
+                for (int c = 0; c < d; ++c) act[0][(size_t)t * cmax + d + c] = vv[(size_t)t * d + c];
+            }
+            for (int l = 0; l < L; ++l) {
+                const int cin = ch[l], cout = ch[l + 1];
+                const double* Wl = wl[l] + (size_t)h * cout * ks * cin;
+                const double* Bl = bl[l] ? bl[l] + (size_t)h * cout : NULL;
+                for (int t = 0; t < T; ++t)
+                    for (int o = 0; o < cout; ++o) {
+                        double acc = Bl ? Bl[o] : 0.0;
+                        for (int tau = 0; tau < ks; ++tau) {
+                            int p = t - (ks - 1 - tau) * dil;
+                            if (p < 0) continue;
+                            const double* wv = Wl + ((size_t)o * ks + tau) * cin;
+                            for (int c = 0; c < cin; ++c) acc += wv[c] * act[l][(size_t)p * cmax + c];
+                        }
+                        pre[l][(size_t)t * cmax + o] = acc;
+                        act[l + 1][(size_t)t * cmax + o] = acc * sigmoid(acc);
+                    }
+            }
+            /* output map: z_j = bout + <wout, act[L][j + half]> */
+            memset(g, 0, sizeof(double) * (size_t)T * cmax);
+            for (int j = 0; j + half <= T - 1; ++j) {
+                const int t = j + half;
+                const double dzt = dzz[j];
+                dbout[h] += dzt;
+                for (int c = 0; c < ch[L]; ++c) {
+                    dwout[(size_t)h * ch[L] + c] += dzt * act[L][(size_t)t * cmax + c];
+                    g[(size_t)t * cmax + c] = dzt * wout[(size_t)h * ch[L] + c];
+                }
+            }
+            for (int l = L - 1; l >= 0; --l) {
+                const int cin = ch[l], cout = ch[l + 1];
+                const double* Wl = wl[l] + (size_t)h * cout * ks * cin;
+                double* dW = dwl[l] + (size_t)h * cout * ks * cin;
+                double* dBl = dbl[l] + (size_t)h * cout;
+                memset(gp, 0, sizeof(double) * (size_t)T * cmax);
+                for (int t = 0; t < T; ++t)
+                    for (int o = 0; o < cout; ++o) {
+                        const double y = pre[l][(size_t)t * cmax + o], sg = sigmoid(y);
+                        const double delta = g[(size_t)t * cmax + o] * (sg + y * sg * (1.0 - sg));
+                        if (delta == 0.0) continue;
+                        dBl[o] += delta;
+                        for (int tau = 0; tau < ks; ++tau) {
+                            int p = t - (ks - 1 - tau) * dil;
+                            if (p < 0) continue;
+                            const double* wv = Wl + ((size_t)o * ks + tau) * cin;
+                            double* dwv = dW + ((size_t)o * ks + tau) * cin;
+                            for (int c = 0; c < cin; ++c) {
+                                dwv[c] += delta * act[l][(size_t)p * cmax + c];
+                                gp[(size_t)p * cmax + c] += delta * wv[c];
+                            }
+                        }
+                    }
+                double* tmp = g; g = gp; gp = tmp;
+            }
+            double* dkk = dk + bh * T * d;
+            double* dvv = dv + bh * T * d;
+            for (int t = 0; t < T; ++t) {
+                for (int c = 0; c < d; ++c) dkk[(size_t)t * d + c] = g[(size_t)t * cmax + c];
+                for (int c = 0; c < d; ++c) dvv[(size_t)t * d + c] = g[(size_t)t * cmax + d + c];
+            }
+        }
+        for (int l = 0; l <= L; ++l) free(act[l]);
+        for (int l = 0; l < L; ++l) free(pre[l]);
+        free(act); free(pre); free(g); free(gp);
+    }
+}
+
+/* ------------------------------------------------------------------------- */
 /* One-shot selection after a T-token prompt (Eq. 5 restricted to tokens already
  * out of the final window, plus the capped capacity of Section 3.1.3).
  * Candidates: j <= T-1-W with (j < sink or z_j > zthr).  Keep the first

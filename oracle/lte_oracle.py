@@ -96,6 +96,31 @@ def scores_stack(k, v, wl, bl, wout, bout, ks=3, dil=2):
     return z
 
 
+def scores_stack_bwd(k, v, wl, bl, wout, bout, dz, ks=3, dil=2):
+    """Gradients of the conv stack for a given dL/dz [B,H,T] (taken as zero where the logit is undefined):
+    dict(dwl [list], dbl [list], dwout, dbout, dk, dv)."""
+    k, v, dz = _f64(k), _f64(v), _f64(dz)
+    B, H, T, d = k.shape
+    L = len(wl)
+    half = L * (ks - 1) * dil // 2
+    dz = dz.copy()
+    dz[:, :, max(T - half, 0):] = 0.0
+    wl = [_f64(x) for x in wl]
+    bl = [None if x is None else _f64(x) for x in bl]
+    ch = [2 * d] + [x.shape[1] for x in wl]
+    wout = _f64(wout)
+    bout = None if bout is None else _f64(bout)
+    dwl = [np.empty_like(x) for x in wl]
+    dbl = [np.empty((H, ch[l + 1]), np.float64) for l in range(L)]
+    dwout = np.empty_like(wout); dbout = np.empty((H,), np.float64)
+    dk = np.empty_like(k); dv = np.empty_like(v)
+    ch_a = (ctypes.c_int * (L + 1))(*ch)
+    arr = lambda xs: (ctypes.c_void_p * L)(*[None if x is None else x.ctypes.data for x in xs])
+    _load().oracle_scores_stack_bwd(B, H, T, d, L, ks, dil, ch_a, arr(wl), arr(bl), _p(wout), _p(bout),
+                                    _p(k), _p(v), _p(dz), arr(dwl), arr(dbl), _p(dwout), _p(dbout), _p(dk), _p(dv))
+    return dict(dwl=dwl, dbl=dbl, dwout=dwout, dbout=dbout, dk=dk, dv=dv)
+
+
 def select(z, W, R, sink=0, tau=0.5):
     """One-shot capped selection -> idx [B,H,R] ascending (-1 unused), cnt, ncand."""
     z = _f64(z)

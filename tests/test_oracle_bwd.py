@@ -119,3 +119,64 @@ def test_row_sums_and_constant_upstream():
     vc = np.broadcast_to(np.random.default_rng(1).standard_normal(d), v.shape).copy()
     g = orc.attn_bwd(q, k, vc, dO, z, idx, cnt, w, 5, 0.5, cnn_input_grad=False)
     assert np.abs(g["dq"]).max() < 1e-12 and np.abs(g["dk"]).max() < 1e-12
+
+
+# ---- the three-layer scorer stack: its backward against central finite differences ------------------------------------
+def _stack_case(seed, B=2, H=2, T=37, d=8, bias=True):
+    rng = np.random.default_rng(seed)
+    ch = [2 * d, d, d // 2, d // 4]
+    k = rng.standard_normal((B, H, T, d)); v = rng.standard_normal((B, H, T, d))
+    wl = [rng.standard_normal((H, ch[l + 1], 3, ch[l])) * 0.4 for l in range(3)]
+    bl = [rng.standard_normal((H, ch[l + 1])) * 0.2 for l in range(3)] if bias else [None] * 3
+    wout = rng.standard_normal((H, ch[3])); bout = rng.standard_normal((H,)) if bias else None
+    g = rng.standard_normal((B, H, T))
+    return rng, k, v, wl, bl, wout, bout, g
+
+
+@pytest.mark.parametrize("seed,bias", [(0, True), (1, False)])
+def test_stack_backward_matches_finite_differences(seed, bias):
+    """L = sum_j g_j z_j over the defined logits; every gradient of the stack's backward is dL/d(parameter or input),
+    checked entry by entry with central differences in fp64 (the definition, independent of the chain rule used)."""
+    rng, k, v, wl, bl, wout, bout, g = _stack_case(seed, bias=bias)
+    T = k.shape[2]
+
+    def loss():
+        z = orc.scores_stack(k, v, wl, bl, wout, bout)
+        return float((g[:, :, : T - 6] * z[:, :, : T - 6]).sum())
+
+    r = orc.scores_stack_bwd(k, v, wl, bl, wout, bout, g)        # g at the undefined tail is ignored
+    groups = [("wl0", wl[0], r["dwl"][0]), ("wl1", wl[1], r["dwl"][1]), ("wl2", wl[2], r["dwl"][2]),
+              ("wout", wout, r["dwout"]), ("k", k, r["dk"]), ("v", v, r["dv"])]
+    if bias:
+        groups += [("bl0", bl[0], r["dbl"][0]), ("bl1", bl[1], r["dbl"][1]), ("bl2", bl[2], r["dbl"][2]), ("bout", bout, r["dbout"])]
+    eps = 1e-6
+    for name, arr, grad in groups:
+        picks = [tuple(rng.integers(0, n) for n in arr.shape) for _ in range(6)]
+        if name in ("k", "v"):                                   # early and late times: the zero padding and the open right end
+            picks += [(0, 0, 0, 1), (1, 1, 3, 2), (0, 1, T - 1, 0), (1, 0, T - 7, 3)]
+        for ix in picks:
+            old = arr[ix]
+            arr[ix] = old + eps; a = loss()
+            arr[ix] = old - eps; b = loss()
+            arr[ix] = old
+            fd = (a - b) / (2 * eps)
+            assert abs(fd - grad[ix]) <= 1e-6 * max(1.0, abs(fd)), (name, ix, fd, grad[ix])
+
+
+def test_stack_backward_structure():
+    """Linearity in the upstream gradient, no gradient from the undefined tail, and the last inputs that cannot reach a
+    defined logit (a token's receptive field reaches 6 positions to either side) get exactly zero."""
+    rng, k, v, wl, bl, wout, bout, g = _stack_case(2)
+    T = k.shape[2]
+    r1 = orc.scores_stack_bwd(k, v, wl, bl, wout, bout, g)
+    r2 = orc.scores_stack_bwd(k, v, wl, bl, wout, bout, 2.0 * g)
+    assert np.allclose(r2["dwl"][0], 2 * r1["dwl"][0]) and np.allclose(r2["dk"], 2 * r1["dk"])
+    g_tail = np.zeros_like(g); g_tail[:, :, T - 6:] = 1.0
+    r0 = orc.scores_stack_bwd(k, v, wl, bl, wout, bout, g_tail)
+    assert all(np.all(a == 0) for a in r0["dwl"]) and np.all(r0["dk"] == 0) and np.all(r0["dbout"] == 0)
+    g_one = np.zeros_like(g); g_one[0, 0, 10] = 1.0                # one logit: inputs outside [10-6, 10+6] are untouched
+    r3 = orc.scores_stack_bwd(k, v, wl, bl, wout, bout, g_one)
+    live = np.abs(r3["dk"][0, 0]).sum(axis=1) > 0
+    # dilation 2: the logit of token 10 is the output at time 16 and sees times 16, 14, ..., 4 only
+    assert live[4:17:2].all() and not live[5:17:2].any() and not live[:4].any() and not live[17:].any()
+    assert np.all(r3["dk"][1] == 0) and np.all(r3["dk"][0, 1] == 0)
