@@ -478,11 +478,16 @@ WsPlan plan(const Params& p, uint32_t flags)
     size_t off = 0;
     w.delta = off; off += up(bht * 4);
     w.dz = off; off += up(bht * 4);
-    w.part_w = off; off += up((size_t)p.H * p.B * w.nchunk * p.K * 2 * p.d * 4);
-    w.part_b = off; off += up((size_t)p.H * p.B * w.nchunk * 4);
+    if (p.stack) {                                  // the stack's backward keeps one packed partial gradient per CTA
+        w.part_w = off; off += up(stack_bwd_workspace(p));
+        w.part_b = off;
+    } else {
+        w.part_w = off; off += up((size_t)p.H * p.B * w.nchunk * p.K * 2 * p.d * 4);
+        w.part_b = off; off += up((size_t)p.H * p.B * w.nchunk * 4);
+    }
     w.dk32 = w.dv32 = 0;
     const bool tc_path = p.dtype == LTE_BF16 && (p.d == 64 || p.d == 128);
-    if ((flags & LTE_BWD_CNN_INPUT_GRAD) && !tc_path) {
+    if ((flags & LTE_BWD_CNN_INPUT_GRAD) && !tc_path && !p.stack) {
         w.dk32 = off; off += up(bht * p.d * 4);
         w.dv32 = off; off += up(bht * p.d * 4);
     }
@@ -505,7 +510,8 @@ int run(const Params& p, const void* q, const void* k, const void* v, const void
     float* part_b = (float*)(base + w.part_b);
     float* dk32 = (float*)(base + w.dk32);
     float* dv32 = (float*)(base + w.dv32);
-    const bool f32 = flags & LTE_BWD_CNN_INPUT_GRAD;
+    const bool want_in = flags & LTE_BWD_CNN_INPUT_GRAD;
+    const bool f32 = want_in && !p.stack;             // the stack's backward adds its input gradient to dk, dv in place
     dim3 grid((p.T + 3) / 4, p.B * p.H);
     if constexpr (sizeof(T) == 2 && (D == 64 || D == 128)) {
         const int e = launch_bwd_dq_tc(p, q, k, v, o, lse, dO, idx, cnt, dq, delta, st);
@@ -527,6 +533,7 @@ int run(const Params& p, const void* q, const void* k, const void* v, const void
                                                           z, idx, cnt, lambda, (T*)dk, (T*)dv, dk32, dv32, dz, p.H, p.T,
                                                           p.W, p.R, p.half, p.zthr, p.scale);
     }
+    if (p.stack) return launch_stack_bwd(p, k, v, dz, dk, dv, dw, dbias, want_in, part_w, st);
     const int per_head = p.K * 2 * D;
     dim3 gr((per_head + 255) / 256, p.H);
     if constexpr (sizeof(T) == 2 && (D == 64 || D == 128)) {

@@ -14,6 +14,7 @@ constexpr int kMaxTaps = 13;          // scorer taps the kernels are instantiate
 struct Params {                       // validated, host-resolved view of lte_shape / lte_conv
     int B, H, T, d, W, R, sink, K, half;
     int G;                            // query heads per key/value head (q, o, lse have H * G heads)
+    int stack;                        // 1: the three-layer scorer stack (w, bias packed as lte.h describes; K = 13, half = 6)
     float zthr;                       // logit(tau): keep iff z > zthr
     float scale;                      // softmax scale
     int dtype;
@@ -84,6 +85,9 @@ int launch_scores(const Params& p, const void* k, const void* v, float* z, float
 int launch_scores_stack(const Params& p, const void* k, const void* v, float* z, float* r, cudaStream_t st);
 size_t scores_stack_weight_floats(int d, int H);
 size_t scores_stack_tc_workspace(const Params& p);
+size_t stack_bwd_workspace(const Params& p);
+int launch_stack_bwd(const Params& p, const void* k, const void* v, const float* dz, void* dk, void* dv, float* dw,
+                     float* dbias, bool input_grad, void* part, cudaStream_t st);
 int launch_scores_stack_tc(const Params& p, const void* k, const void* v, float* z, float* r, void* ws, size_t ws_bytes,
                            cudaStream_t st);
 int launch_select(const Params& p, const float* z, int32_t* idx, int32_t* cnt, int32_t* ncand, cudaStream_t st);

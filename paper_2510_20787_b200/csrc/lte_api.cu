@@ -46,6 +46,8 @@ Params make_params(const lte_shape* s, const lte_conv* c)
     Params p;
     p.B = s->B; p.H = s->H; p.T = s->T; p.d = s->d; p.W = s->W; p.R = s->R; p.sink = s->sink;
     p.G = s->group > 1 ? s->group : 1;
+    p.stack = 0;
+    if (c && c->n_layers == 3) { p.stack = 1; p.K = 13; p.half = 6; }   // the paper's stack: receptive field 13
     p.K = c ? c->kernel : 1; p.half = p.K / 2;
     p.zthr = s->tau <= 0.f ? -INFINITY : (float)(log((double)s->tau) - log1p(-(double)s->tau));
     p.scale = s->softmax_scale > 0.f ? s->softmax_scale : (float)(1.0 / sqrt((double)s->d));
@@ -123,7 +125,6 @@ int lte_scores(const lte_shape* s, const lte_conv* c, const void* k, const void*
         if (!k || !v || !z || !aligned16(k) || !aligned16(v) || !aligned16(c->w)) return LTE_ERR_INVALID_ARG;
         e = check_arch(); if (e) return e;
         Params p = make_params(s, c);
-        p.K = 13; p.half = 6;
         // tensor cores where the shape allows and the caller brought the workspace for the split weight image
         e = launch_scores_stack_tc(p, k, v, z, r_or_null, ws, ws_bytes, (cudaStream_t)stream);
         if (e != LTE_ERR_UNSUPPORTED) return e;
@@ -194,7 +195,12 @@ int lte_attn_bwd(const lte_shape* s, const lte_conv* c, const void* q, const voi
                  uint32_t flags, void* ws, size_t ws_bytes, void* stream)
 {
     int e = check_shape(s, true); if (e) return e;
-    e = check_conv(s, c); if (e) return e;
+    if (c && c->w && c->n_layers == 3) {                   // the paper's stack: d = 64, gradients packed like the parameters
+        if (c->kernel != 3 || c->dilation != 2 || s->d != 64) return LTE_ERR_UNSUPPORTED;
+        if (s->W < 7 || !aligned16(c->w)) return LTE_ERR_INVALID_ARG;
+    } else {
+        e = check_conv(s, c); if (e) return e;
+    }
     if (!q || !k || !v || !o || !lse || !dO || !z || !cnt || (s->R > 0 && !idx) || !dq || !dk || !dv || !dw)
         return LTE_ERR_INVALID_ARG;
     if (flags & ~LTE_BWD_CNN_INPUT_GRAD) return LTE_ERR_INVALID_ARG;

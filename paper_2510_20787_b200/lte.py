@@ -205,10 +205,16 @@ def lte_attn_decode(s, c, cache, q1, k1, v1, o1=None, lse1=None):
 
 def lte_attn_bwd(s, c, q, k, v, o, lse, dO, z, idx, cnt, lam=None, flags=BWD_CNN_INPUT_GRAD, want_dbias=True,
                  ws=None):
-    """Backward with the straight-through surrogate -> dq, dk, dv, dw [H,K,2d], dbias [H] (or None)."""
+    """Backward with the straight-through surrogate -> dq, dk, dv, dw [H,K,2d], dbias [H] (or None).  With the
+    three-layer stack (conv_stack) dw and dbias are flat, packed like the parameters: use unpack_stack_grads."""
     dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
-    dw = torch.empty((s.H, c.kernel, 2 * s.d), dtype=torch.float32, device=q.device)
-    db = torch.empty((s.H,), dtype=torch.float32, device=q.device) if want_dbias else None
+    if c.n_layers == 3:
+        d = s.d
+        dw = torch.empty((s.H * (d * 3 * 2 * d + (d // 2) * 3 * d + (d // 4) * 3 * (d // 2) + d // 4),), dtype=torch.float32, device=q.device)
+        db = torch.empty((s.H * (d + d // 2 + d // 4 + 1),), dtype=torch.float32, device=q.device) if want_dbias else None
+    else:
+        dw = torch.empty((s.H, c.kernel, 2 * s.d), dtype=torch.float32, device=q.device)
+        db = torch.empty((s.H,), dtype=torch.float32, device=q.device) if want_dbias else None
     need = lte_workspace_bytes(OP_BWD, s, c)
     if ws is None:
         ws = torch.empty(max(need, 16), dtype=torch.uint8, device=q.device)
@@ -218,6 +224,23 @@ def lte_attn_bwd(s, c, q, k, v, o, lse, dO, z, idx, cnt, lam=None, flags=BWD_CNN
         _ptr(lam, torch.float32), _ptr(dq), _ptr(dk), _ptr(dv), _ptr(dw), _ptr(db), flags, _ptr(ws),
         ws.numel(), _stream()))
     return dq, dk, dv, dw, db
+
+
+def unpack_stack_grads(H, d, dw, db=None):
+    """Flat gradients of the three-layer stack -> (dwl [3 tensors [H,c_out,3,c_in]], dwout [H,d/4], dbl [3] or None,
+    dbout [H] or None), the shapes conv_stack takes."""
+    ch = [2 * d, d, d // 2, d // 4]
+    dwl, off = [], 0
+    for l in range(3):
+        n = H * ch[l + 1] * 3 * ch[l]
+        dwl.append(dw[off:off + n].view(H, ch[l + 1], 3, ch[l])); off += n
+    dwout = dw[off:off + H * ch[3]].view(H, ch[3])
+    if db is None:
+        return dwl, dwout, None, None
+    dbl, off = [], 0
+    for l in range(3):
+        dbl.append(db[off:off + H * ch[l + 1]].view(H, ch[l + 1])); off += H * ch[l + 1]
+    return dwl, dwout, dbl, db[off:off + H]
 
 
 def lte_attn_bwd_static(s, c, q, k, v, o, lse, dO, z, idx, cnt, lam=None, flags=BWD_CNN_INPUT_GRAD, outs=None):

@@ -82,7 +82,7 @@ def test_stack_tensor_core_path(B, H, T, bias):
 
 
 def test_stack_rejected_elsewhere():
-    """decode, cache_init and the backward take the single layer only."""
+    """decode and cache_init take the single layer only."""
     cfg = synth.Config("stack", "bf16", 1, 2, 64, 64, 16, 8, 7, 0.1)
     wl, wout, bl, bout = _stack_params(cfg.H, 64, 1, False)
     c = lte.conv_stack([torch.from_numpy(w).cuda() for w in wl], torch.from_numpy(wout).cuda())
@@ -93,3 +93,49 @@ def test_stack_rejected_elsewhere():
     idx, cnt = lte.lte_select(s, z)
     with pytest.raises(Exception):
         lte.lte_cache_init(s, c, k, v, z, idx, cnt)
+
+
+# ---- backward through the stack (lte_attn_bwd with the three-layer scorer) ---------------------------------------------
+def _rel(a, b):
+    return float(np.linalg.norm(np.asarray(a, np.float64) - b) / (np.linalg.norm(b) + 1e-30))
+
+
+@pytest.mark.parametrize("dtype,T,W,R,bias,in_grad", [("bf16", 200, 16, 12, True, True), ("bf16", 333, 24, 40, False, True),
+                                                      ("f32", 150, 16, 10, True, True), ("bf16", 260, 32, 16, True, False)])
+def test_stack_backward(dtype, T, W, R, bias, in_grad):
+    """dq, dk, dv and the gradients of every parameter of the stack against the oracle: the attention backward and the
+    straight-through surrogate give dz, the stack's backward (pinned by finite differences on the CPU) the rest."""
+    d = 64
+    cfg = synth.Config("stackbwd", dtype, 2, 2, d, T, W, R, 7, 0.1)
+    x = synth.make(cfg, 8, with_dO=True)
+    wl, wout, bl, bout = _stack_params(cfg.H, d, 8, bias)
+    t = lambda a: None if a is None else torch.from_numpy(a).cuda()
+    c = lte.conv_stack([t(w) for w in wl], t(wout), [t(b) for b in bl] if bias else None, t(bout))
+    s = shape_of(cfg, B=cfg.B)
+    q, k, v, dO = (dev(x[n], dtype) for n in ("q", "k", "v", "dO"))
+    z = lte.lte_scores(s, c, k, v, ws=False)
+    idx, cnt = lte.lte_select(s, z)
+    o, lse = lte.lte_attn_prefill(s, q, k, v, idx, cnt)
+    flags = lte.BWD_CNN_INPUT_GRAD if in_grad else 0
+    dq, dk, dv, dw, db = lte.lte_attn_bwd(s, c, q, k, v, o, lse, dO, z, idx, cnt, flags=flags)
+    torch.cuda.synchronize()
+    assert lte.lib().lte_device_status() == 0
+    # oracle: same logits, same list; the single-layer weight argument only sets the width of the undefined tail (13 taps)
+    z64 = z.cpu().numpy().astype(np.float64)
+    w13 = np.zeros((cfg.H, 13, 2 * d))
+    ra = orc.attn_bwd(x["q"], x["k"], x["v"], x["dO"], z64, idx.cpu().numpy(), cnt.cpu().numpy(), w13, W, cnn_input_grad=False)
+    rs = orc.scores_stack_bwd(x["k"], x["v"], wl, bl, wout, bout, ra["dz"])
+    dk64 = ra["dk"] + (rs["dk"] if in_grad else 0.0)
+    dv64 = ra["dv"] + (rs["dv"] if in_grad else 0.0)
+    assert _rel(dq.float().cpu().numpy(), ra["dq"]) < 5e-2
+    assert _rel(dk.float().cpu().numpy(), dk64) < 5e-2
+    assert _rel(dv.float().cpu().numpy(), dv64) < 5e-2
+    dwl, dwout, dbl, dbout = lte.unpack_stack_grads(cfg.H, d, dw, db)
+    for l in range(3):
+        assert _rel(dwl[l].cpu().numpy(), rs["dwl"][l]) < 5e-2, l
+        assert _rel(dbl[l].cpu().numpy(), rs["dbl"][l]) < 5e-2, l
+    assert _rel(dwout.cpu().numpy(), rs["dwout"]) < 5e-2
+    assert _rel(dbout.cpu().numpy(), rs["dbout"]) < 5e-2
+    if dtype == "f32":                                               # fp32 storage: the scorer's part is exact to rounding
+        for l in range(3):
+            assert _rel(dwl[l].cpu().numpy(), rs["dwl"][l]) < 1e-4
