@@ -400,6 +400,35 @@ def _extra_s(out, torch, lte, synth, pk, flush, n5):
                                          "frac": fl / t_alu / alu_peak, "peak_source": "SMs x 128 fp32 lanes x 2 x 1.965 GHz"}},
         "max_abs_z_difference_between_kernels": float(dz), "fraction_kept": kept}
     del x, z
+    # backward through the stack at the training shape (C5): the attention backward is the same as with the single layer,
+    # the scorer's part is the fp32 kernel
+    cfg5 = synth.CONFIGS["C5"]
+    x5 = device_inputs(cfg5, 8, torch, with_dO=True)
+    s5 = lte.shape(cfg5.B, cfg5.H, cfg5.T, cfg5.d, cfg5.W, cfg5.R, lte.BF16)
+    z5 = lte.lte_scores(s5, c, x5["k"], x5["v"])
+    idx5, cnt5 = lte.lte_select(s5, z5)
+    o5, lse5 = lte.lte_attn_prefill(s5, x5["q"], x5["k"], x5["v"], idx5, cnt5)
+    ws5 = torch.empty(lte.lte_workspace_bytes(lte.OP_BWD, s5, c), dtype=torch.uint8, device="cuda")
+    c1 = lte.conv(x5["w"])
+    ws1 = torch.empty(lte.lte_workspace_bytes(lte.OP_BWD, s5, c1), dtype=torch.uint8, device="cuda")
+
+    def b_stack():
+        lte.lte_attn_bwd(s5, c, x5["q"], x5["k"], x5["v"], o5, lse5, x5["dO"], z5, idx5, cnt5, ws=ws5)
+
+    def b_single():
+        lte.lte_attn_bwd(s5, c1, x5["q"], x5["k"], x5["v"], o5, lse5, x5["dO"], z5, idx5, cnt5, ws=ws1)
+
+    t_bs = mid3(timed(torch, b_stack, n5, 3, flush)[0]) * 1e-3
+    t_b1 = mid3(timed(torch, b_single, n5, 3, flush)[0]) * 1e-3
+    fl5 = 2.0 * macs * cfg5.B * cfg5.H * cfg5.T
+    out["S_scorer_stack"]["backward_C5"] = {
+        "workload": "C5 shape, lte_attn_bwd with the stack (weight, bias and input gradients)",
+        "bwd_ms": t_bs * 1e3, "bwd_ms_single_layer_scorer": t_b1 * 1e3,
+        "stack_part_ms": (t_bs - t_b1) * 1e3 if t_bs > t_b1 else None,
+        "roofline": {"bound": "alu", "achieved": 3 * fl5 / max(t_bs - t_b1, 1e-9) / 1e12, "peak": alu_peak / 1e12, "unit": "TFLOP/s",
+                     "frac": 3 * fl5 / max(t_bs - t_b1, 1e-9) / alu_peak,
+                     "note": "3 x the forward's products (forward again, transposed products, weight gradients) over the time the stack adds"}}
+    del x5, o5, lse5, z5
 
 
 def _extra_p(out, torch, lte, synth, pk, flush, n5):

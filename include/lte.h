@@ -70,7 +70,8 @@ typedef struct lte_conv {
  * aligned; it receives the weights split into bf16 pieces, rebuilt by every call) the stack runs on the tensor cores
  * with exact products and fp32 accumulation; without the workspace, and for every other accepted shape, on the fp32
  * ALUs.  Both agree with an fp64 evaluation to about 1e-5 at |z| of a few units.
- * The other entry points (decode, backward, cache_init) take the single layer only and answer LTE_ERR_UNSUPPORTED.
+ * lte_attn_bwd takes the stack for d = 64: dw and dbias then have the packed layouts of w and bias above.
+ * lte_attn_decode, lte_cache_init and lte_attn_bwd_static take the single layer only and answer LTE_ERR_UNSUPPORTED.
  */
 
 typedef enum lte_op {

@@ -100,13 +100,14 @@ def _rel(a, b):
     return float(np.linalg.norm(np.asarray(a, np.float64) - b) / (np.linalg.norm(b) + 1e-30))
 
 
-@pytest.mark.parametrize("dtype,T,W,R,bias,in_grad", [("bf16", 200, 16, 12, True, True), ("bf16", 333, 24, 40, False, True),
-                                                      ("f32", 150, 16, 10, True, True), ("bf16", 260, 32, 16, True, False)])
-def test_stack_backward(dtype, T, W, R, bias, in_grad):
+@pytest.mark.parametrize("dtype,T,W,R,bias,in_grad,B,H", [("bf16", 200, 16, 12, True, True, 2, 2), ("bf16", 333, 24, 40, False, True, 2, 2),
+                                                          ("f32", 150, 16, 10, True, True, 2, 2), ("bf16", 260, 32, 16, True, False, 2, 2),
+                                                          ("bf16", 2048, 64, 64, True, True, 5, 8), ("bf16", 700, 64, 32, True, True, 40, 8)])
+def test_stack_backward(dtype, T, W, R, bias, in_grad, B, H):
     """dq, dk, dv and the gradients of every parameter of the stack against the oracle: the attention backward and the
     straight-through surrogate give dz, the stack's backward (pinned by finite differences on the CPU) the rest."""
     d = 64
-    cfg = synth.Config("stackbwd", dtype, 2, 2, d, T, W, R, 7, 0.1)
+    cfg = synth.Config("stackbwd", dtype, B, H, d, T, W, R, 7, 0.1)   # the last two: several tiles per thread block
     x = synth.make(cfg, 8, with_dO=True)
     wl, wout, bl, bout = _stack_params(cfg.H, d, 8, bias)
     t = lambda a: None if a is None else torch.from_numpy(a).cuda()
