@@ -429,6 +429,33 @@ def _extra_s(out, torch, lte, synth, pk, flush, n5):
                      "frac": 3 * fl5 / max(t_bs - t_b1, 1e-9) / alu_peak,
                      "note": "3 x the forward's products (forward again, transposed products, weight gradients) over the time the stack adds"}}
     del x5, o5, lse5, z5
+    # the stack in decode at the C4 cache shape (prompt of 1024 tokens): the step scores nothing, lte_cache_score runs once per
+    # W - 13 steps over the whole ring (lazy batches)
+    cfg4 = synth.CONFIGS["C4"].with_(T=1024)
+    x4 = device_inputs(cfg4, 9, torch)
+    s4 = lte.shape(cfg4.B, cfg4.H, cfg4.T, cfg4.d, cfg4.W, cfg4.R, lte.BF16)
+    z4 = lte.lte_scores(s4, c, x4["k"], x4["v"])
+    idx4, cnt4 = lte.lte_select(s4, z4)
+    cache = lte.lte_cache_init(s4, c, x4["k"], x4["v"], z4, idx4, cnt4)
+    wsd = torch.empty(lte.lte_workspace_bytes(lte.OP_DECODE, s4, c), dtype=torch.uint8, device="cuda")
+    g4 = torch.Generator(device="cuda"); g4.manual_seed(91)
+    q1, k1, v1 = ((torch.randn((cfg4.B, cfg4.H, cfg4.d), generator=g4, device="cuda") * f).to(torch.bfloat16) for f in (0.35, 0.35, 1.0))
+    o1 = torch.empty_like(q1); l1 = torch.empty((cfg4.B, cfg4.H), dtype=torch.float32, device="cuda")
+
+    def f_score():
+        lte.lte_cache_score(s4, c, cache, ws=wsd)
+
+    def f_step():
+        lte.lte_attn_decode(s4, c, cache, q1, k1, v1, o1=o1, lse1=l1)
+
+    t_sc = mid3(timed(torch, f_score, n5, 3, flush)[0]) * 1e-3
+    t_st = mid3(timed(torch, f_step, n5, 3, flush)[0]) * 1e-3
+    out["S_scorer_stack"]["decode_C4_cache"] = {
+        "workload": "B=128 H=16 d=64 W=128 R=128, stack scorer: lte_cache_score every W - 13 = 115 steps",
+        "cache_score_ms": t_sc * 1e3, "amortised_us_per_step": t_sc * 1e6 / (cfg4.W - 13),
+        "decode_step_us_single_launch": t_st * 1e6,
+        "note": "single launches with the L2 flushed in between (the C4 section times the step in a CUDA graph)"}
+    del x4, cache, wsd
 
 
 def _extra_p(out, torch, lte, synth, pk, flush, n5):

@@ -71,7 +71,8 @@ typedef struct lte_conv {
  * with exact products and fp32 accumulation; without the workspace, and for every other accepted shape, on the fp32
  * ALUs.  Both agree with an fp64 evaluation to about 1e-5 at |z| of a few units.
  * lte_attn_bwd takes the stack for d = 64: dw and dbias then have the packed layouts of w and bias above.
- * lte_attn_decode, lte_cache_init and lte_attn_bwd_static take the single layer only and answer LTE_ERR_UNSUPPORTED.
+ * lte_cache_init and lte_attn_decode take the stack for d = 32 or 64 and W >= 20; the step then scores nothing and
+ * lte_cache_score has to be called periodically.  lte_attn_bwd_static takes the single layer only.
  */
 
 typedef enum lte_op {
@@ -181,6 +182,19 @@ int lte_cache_init(const lte_shape* s, const lte_conv* c, const void* k, const v
 int lte_attn_decode(const lte_shape* s, const lte_conv* c, void* cache,
                     const void* q1, const void* k1, const void* v1, void* o1, float* lse1,
                     void* stream);
+
+/*
+ * Lazy scoring of the ring (Section 3.1.3, "Cached prefilling and decoding": scores are computed in batches, each
+ * before its tokens leave the window), for the three-layer stack (lte_conv.n_layers = 3), which lte_attn_decode does
+ * not evaluate inside the step: every token in the ring whose receptive field (6 tokens to either side) lies inside
+ * the ring, or left of time 0, receives its logit.  A token that is n tokens old can be scored while 7 <= n <= W - 6,
+ * and its logit is read when it leaves the window (n = W): call this at least every W - 13 steps; a token that leaves
+ * the window unscored is evicted.  Scoring a token again rewrites the same value.
+ *   cache      in/out  the state lte_cache_init / lte_attn_decode maintain
+ *   ws         device scratch of lte_workspace_bytes(LTE_OP_DECODE, s, c) bytes, 256-byte aligned
+ * Errors: UNSUPPORTED for the single layer (it is scored inside the step), INVALID_ARG, WORKSPACE.
+ */
+int lte_cache_score(const lte_shape* s, const lte_conv* c, void* cache, void* ws, size_t ws_bytes, void* stream);
 
 /*
  * Backward of lte_attn_prefill with the straight-through surrogate (Section 3.1.2):

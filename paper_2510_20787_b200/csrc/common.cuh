@@ -98,6 +98,8 @@ int launch_prefill_tc_long(const Params& p, const void* q, const void* k, const 
 int prefill_long_status_fetch_and_clear();
 int launch_cache_init(const Params& p, const void* k, const void* v, const float* z, const int32_t* idx,
                       const int32_t* cnt, void* cache, cudaStream_t st);
+int launch_ring_linearize(const Params& p, const void* cache, void* klin, void* vlin, cudaStream_t st);
+int launch_ring_scatter_z(const Params& p, void* cache, const float* zlin, cudaStream_t st);
 int launch_decode_tc(const Params& p, void* cache, const void* q1, const void* k1, const void* v1, void* o1,
                      float* lse1, cudaStream_t st);
 int launch_decode(const Params& p, void* cache, const void* q1, const void* k1, const void* v1, void* o1,

@@ -151,7 +151,7 @@ __global__ void __launch_bounds__(DT) decode_kernel(unsigned char* __restrict__ 
     const int slot = n % W;
 
     // ---- scorer for token j = n - half, from the old ring rows and the incoming row -------------
-    const int jsc = n - half;
+    const int jsc = K > 0 ? n - half : -1;   // K = 0: the scorer runs outside (lte_cache_score), nothing is scored here
     if (jsc >= 0) {
         for (int t = wid; t < K; t += DT / 32) {
             const int pos = jsc + t - half;
@@ -456,7 +456,7 @@ __global__ void __launch_bounds__(DT) decode_bulk_kernel(unsigned char* __restri
         }
         DPROF(2);
         // ---- scorer taps (warp w owns taps w and w + 8) and the logit of the incoming token (last warp) ----
-        const int jsc = n - half;
+        const int jsc = K > 0 ? n - half : -1;   // K = 0: the scorer runs outside (lte_cache_score)
         if (jsc >= 0) {
 #pragma unroll
             for (int u = 0; u < 2; ++u) {
@@ -686,6 +686,64 @@ int launch_cache_init(const Params& p, const void* k, const void* v, const float
     return cuda_status(cudaGetLastError());
 }
 
+// ---- lazy scoring of the ring for scorers that do not run inside the step (the three-layer stack) -------------------
+// The ring's rows in time order: row r of the copy is token base + r, base = max(n - W, 0); rows past the newest token are
+// zero.  The scorer then runs over the copy as over a W-token sequence, and the logits whose receptive field lies inside
+// the ring (or left of time 0) go back to the ring's logit slots: rows r >= half unless the ring starts at time 0, and
+// r <= min(n, W) - 1 - half.
+template <typename T>
+__global__ void ring_linearize_kernel(const unsigned char* __restrict__ cache, CacheLayout L, T* __restrict__ klin,
+                                      T* __restrict__ vlin, int D, int W)
+{
+    const int bh = blockIdx.x;
+    const unsigned char* blk = cache + L.header + (size_t)bh * L.stride;
+    const T* Kc = reinterpret_cast<const T*>(blk + L.off_k);
+    const T* Vc = reinterpret_cast<const T*>(blk + L.off_v);
+    const int n = reinterpret_cast<const int32_t*>(blk + L.off_meta)[0];
+    const int base = n > W ? n - W : 0, n_eff = n < W ? n : W;
+    for (int e = threadIdx.x; e < W * D; e += blockDim.x) {
+        const int r = e / D, c = e % D;
+        T kx = from_f<T>(0.f), vx = from_f<T>(0.f);
+        if (r < n_eff) {
+            const int row = (base + r) % W;
+            const int cs = L.swz ? ((((c >> 3) ^ (row & 7)) << 3) | (c & 7)) : c;
+            kx = Kc[(size_t)row * D + cs]; vx = Vc[(size_t)row * D + cs];
+        }
+        klin[((size_t)bh * W + r) * D + c] = kx;
+        vlin[((size_t)bh * W + r) * D + c] = vx;
+    }
+}
+
+__global__ void ring_scatter_z_kernel(unsigned char* __restrict__ cache, CacheLayout L, const float* __restrict__ zlin, int W,
+                                      int half)
+{
+    const int bh = blockIdx.x;
+    unsigned char* blk = cache + L.header + (size_t)bh * L.stride;
+    float* zc = reinterpret_cast<float*>(blk + L.off_z);
+    const int n = reinterpret_cast<const int32_t*>(blk + L.off_meta)[0];
+    const int base = n > W ? n - W : 0, n_eff = n < W ? n : W;
+    const int r_lo = base > 0 ? half : 0, r_hi = n_eff - 1 - half;
+    for (int r = r_lo + threadIdx.x; r <= r_hi; r += blockDim.x) zc[(base + r) % W] = zlin[(size_t)bh * W + r];
+}
+
+int launch_ring_linearize(const Params& p, const void* cache, void* klin, void* vlin, cudaStream_t st)
+{
+    const CacheLayout L = cache_layout(p.d, p.W, p.R, p.dtype);
+    if (p.dtype == LTE_BF16)
+        ring_linearize_kernel<__nv_bfloat16><<<p.B * p.H, 256, 0, st>>>((const unsigned char*)cache, L, (__nv_bfloat16*)klin,
+                                                                        (__nv_bfloat16*)vlin, p.d, p.W);
+    else
+        ring_linearize_kernel<float><<<p.B * p.H, 256, 0, st>>>((const unsigned char*)cache, L, (float*)klin, (float*)vlin, p.d, p.W);
+    return cuda_status(cudaGetLastError());
+}
+
+int launch_ring_scatter_z(const Params& p, void* cache, const float* zlin, cudaStream_t st)
+{
+    const CacheLayout L = cache_layout(p.d, p.W, p.R, p.dtype);
+    ring_scatter_z_kernel<<<p.B * p.H, 128, 0, st>>>((unsigned char*)cache, L, zlin, p.W, p.half);
+    return cuda_status(cudaGetLastError());
+}
+
 // ---- grouped-query attention: the other query heads of a key/value head -------------------------------------------
 // The step kernels above update the cache of a key/value head and attend for its first query head.  The remaining
 // G - 1 query heads attend over the updated block (ring rows of the min(n, W) newest tokens, cnt pool rows) here:
@@ -883,7 +941,9 @@ static int launch_decode_step(const Params& p, void* cache, const void* q1, cons
 int launch_decode(const Params& p, void* cache, const void* q1, const void* k1, const void* v1, void* o1, float* lse1,
                   cudaStream_t st)
 {
-    int e = launch_decode_step(p, cache, q1, k1, v1, o1, lse1, st);
+    Params ps = p;
+    if (p.stack) ps.K = 0;                               // the stack is scored outside the step (lte_cache_score)
+    int e = launch_decode_step(ps, cache, q1, k1, v1, o1, lse1, st);
     if (e != LTE_OK || p.G <= 1) return e;
     const CacheLayout L = cache_layout(p.d, p.W, p.R, p.dtype);
     const size_t att_smem = sizeof(float) * ((size_t)ATT_Q * (p.W + p.R) + (size_t)(DT / 32) * ATT_Q * p.d);

@@ -209,7 +209,7 @@ __global__ void __launch_bounds__(NTHR) decode_tc_kernel(unsigned char* __restri
             // ---- direct reads of the key / value blocks: scorer taps and the popped row ----------------------
             dwait(bar_k, it & 1, 7);
             dwait(bar_v, it & 1, 8);
-            const int jsc = n - half;
+            const int jsc = K > 0 ? n - half : -1;   // K = 0: the scorer runs outside (lte_cache_score)
             if (jsc >= 0) {
 #pragma unroll
                 for (int u = 0; u < 2; ++u) {

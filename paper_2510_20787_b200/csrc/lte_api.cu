@@ -46,9 +46,9 @@ Params make_params(const lte_shape* s, const lte_conv* c)
     Params p;
     p.B = s->B; p.H = s->H; p.T = s->T; p.d = s->d; p.W = s->W; p.R = s->R; p.sink = s->sink;
     p.G = s->group > 1 ? s->group : 1;
+    p.K = c ? c->kernel : 1; p.half = p.K / 2;
     p.stack = 0;
     if (c && c->n_layers == 3) { p.stack = 1; p.K = 13; p.half = 6; }   // the paper's stack: receptive field 13
-    p.K = c ? c->kernel : 1; p.half = p.K / 2;
     p.zthr = s->tau <= 0.f ? -INFINITY : (float)(log((double)s->tau) - log1p(-(double)s->tau));
     p.scale = s->softmax_scale > 0.f ? s->softmax_scale : (float)(1.0 / sqrt((double)s->d));
     p.dtype = s->dtype;
@@ -57,12 +57,42 @@ Params make_params(const lte_shape* s, const lte_conv* c)
     return p;
 }
 
+// the single layer, or the paper's stack where the decode cache takes it (d = 32 or 64, window at least 20 tokens: the
+// ring has to hold a token's receptive field of 13 with room for a scoring period)
+int check_conv_or_stack(const lte_shape* s, const lte_conv* c)
+{
+    if (c && c->w && c->n_layers == 3) {
+        if (c->kernel != 3 || c->dilation != 2 || (s->d != 32 && s->d != 64)) return LTE_ERR_UNSUPPORTED;
+        if (s->W < 20 || !aligned16(c->w)) return LTE_ERR_INVALID_ARG;
+        return LTE_OK;
+    }
+    return check_conv(s, c);
+}
+
 int check_arch()
 {
     int dev = 0, major = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return LTE_ERR_CUDA;
     if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return LTE_ERR_CUDA;
     return major == 10 ? LTE_OK : LTE_ERR_ARCH;
+}
+
+// scratch of lte_cache_score: the ring in time order (keys, values), its logits, the tensor-core scorer's weight image
+struct CacheScorePlan { size_t klin, vlin, zlin, tc, total; };
+CacheScorePlan cache_score_plan(const lte_shape* s, const lte_conv* c)
+{
+    auto up = [](size_t x) { return (x + 255) / 256 * 256; };
+    CacheScorePlan w;
+    const size_t rows = (size_t)s->B * s->H * s->W, esz = s->dtype == LTE_BF16 ? 2 : 4;
+    size_t off = 0;
+    w.klin = off; off += up(rows * s->d * esz);
+    w.vlin = off; off += up(rows * s->d * esz);
+    w.zlin = off; off += up(rows * 4);
+    w.tc = off;
+    lte_shape s2 = *s; s2.T = s->W;
+    off += up(scores_stack_tc_workspace(make_params(&s2, c)));
+    w.total = off;
+    return w;
 }
 
 }  // namespace
@@ -105,6 +135,10 @@ size_t lte_workspace_bytes(int op, const lte_shape* s, const lte_conv* c)
         if (check_shape(s, true) != LTE_OK || !c) return 0;
         Params p = make_params(s, c);
         return bwd_workspace_bytes(p, LTE_BWD_CNN_INPUT_GRAD);
+    }
+    if (op == LTE_OP_DECODE && c && c->n_layers == 3) {
+        if (check_shape(s, false) != LTE_OK) return 0;
+        return cache_score_plan(s, c).total;
     }
     if (op == LTE_OP_SCORES && c && c->n_layers == 3) {
         if (check_shape(s, true) != LTE_OK) return 0;
@@ -171,18 +205,39 @@ int lte_cache_init(const lte_shape* s, const lte_conv* c, const void* k, const v
                    const int32_t* idx, const int32_t* cnt, void* cache, void* stream)
 {
     int e = check_shape(s, false); if (e) return e;
-    e = check_conv(s, c); if (e) return e;
+    e = check_conv_or_stack(s, c); if (e) return e;
     if (!cache || !aligned16(cache)) return LTE_ERR_INVALID_ARG;
     if (s->T > 0 && (!k || !v || !z || !cnt || (s->R > 0 && !idx))) return LTE_ERR_INVALID_ARG;
     e = check_arch(); if (e) return e;
     return launch_cache_init(make_params(s, c), k, v, z, idx, cnt, cache, (cudaStream_t)stream);
 }
 
+int lte_cache_score(const lte_shape* s, const lte_conv* c, void* cache, void* ws, size_t ws_bytes, void* stream)
+{
+    int e = check_shape(s, false); if (e) return e;
+    if (!c || !c->w || c->n_layers != 3) return LTE_ERR_UNSUPPORTED;       // the single layer is scored inside the step
+    e = check_conv_or_stack(s, c); if (e) return e;
+    if (!cache || !aligned16(cache)) return LTE_ERR_INVALID_ARG;
+    const CacheScorePlan w = cache_score_plan(s, c);
+    if (!ws || ((uintptr_t)ws & 255u) != 0 || ws_bytes < w.total) return LTE_ERR_WORKSPACE;
+    e = check_arch(); if (e) return e;
+    cudaStream_t st = (cudaStream_t)stream;
+    char* base = (char*)ws;
+    lte_shape s2 = *s; s2.T = s->W;                                         // the ring as a W-token sequence
+    Params p = make_params(&s2, c);
+    e = launch_ring_linearize(p, cache, base + w.klin, base + w.vlin, st); if (e) return e;
+    float* zlin = (float*)(base + w.zlin);
+    e = launch_scores_stack_tc(p, base + w.klin, base + w.vlin, zlin, nullptr, base + w.tc, w.total - w.tc, st);
+    if (e == LTE_ERR_UNSUPPORTED) e = launch_scores_stack(p, base + w.klin, base + w.vlin, zlin, nullptr, st);
+    if (e) return e;
+    return launch_ring_scatter_z(p, cache, zlin, st);
+}
+
 int lte_attn_decode(const lte_shape* s, const lte_conv* c, void* cache, const void* q1, const void* k1,
                     const void* v1, void* o1, float* lse1, void* stream)
 {
     int e = check_shape(s, false); if (e) return e;
-    e = check_conv(s, c); if (e) return e;
+    e = check_conv_or_stack(s, c); if (e) return e;
     if (!cache || !q1 || !k1 || !v1 || !o1 || !lse1) return LTE_ERR_INVALID_ARG;
     if (!aligned16(cache) || !aligned16(q1) || !aligned16(k1) || !aligned16(v1)) return LTE_ERR_INVALID_ARG;
     e = check_arch(); if (e) return e;

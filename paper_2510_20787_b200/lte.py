@@ -18,7 +18,7 @@ F32, BF16 = 0, 1
 OP_SCORES, OP_SELECT, OP_PREFILL, OP_DECODE, OP_BWD = range(5)
 BWD_CNN_INPUT_GRAD = 1
 
-EXPORTS = ["lte_device_status", "lte_workspace_bytes", "lte_strerror", "lte_scores", "lte_select", "lte_attn_prefill",
+EXPORTS = ["lte_device_status", "lte_workspace_bytes", "lte_strerror", "lte_scores", "lte_select", "lte_cache_score", "lte_attn_prefill",
            "lte_cache_bytes", "lte_cache_init", "lte_attn_decode", "lte_attn_bwd", "lte_attn_bwd_static"]
 STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -62,6 +62,7 @@ def lib():
         L.lte_attn_prefill.argtypes = [vp] * 9 + [ctypes.c_size_t, vp]
         L.lte_cache_init.argtypes = [vp] * 9
         L.lte_attn_decode.argtypes = [vp] * 9
+        L.lte_cache_score.argtypes = [vp] * 4 + [ctypes.c_size_t, vp]
         L.lte_attn_bwd.argtypes = [vp] * 17 + [ctypes.c_uint32, vp, ctypes.c_size_t, vp]
         L.lte_attn_bwd_static.argtypes = [vp] * 17 + [ctypes.c_uint32, vp]
         for name in EXPORTS:
@@ -201,6 +202,15 @@ def lte_attn_decode(s, c, cache, q1, k1, v1, o1=None, lse1=None):
                                                     _ptr(q1), _ptr(k1), _ptr(v1), _ptr(o1),
                                                     _ptr(lse1, torch.float32), _stream()))
     return o1, lse1
+
+
+def lte_cache_score(s, c, cache, ws=None):
+    """Three-layer stack only: score the ring tokens whose receptive field is complete (call at least every W - 13
+    decode steps).  ws: uint8 tensor of lte_workspace_bytes(OP_DECODE, s, c) bytes, allocated here when None."""
+    if ws is None:
+        ws = torch.empty(max(lte_workspace_bytes(OP_DECODE, s, c), 256), dtype=torch.uint8, device=cache.device)
+    _check("lte_cache_score", lib().lte_cache_score(ctypes.addressof(s), ctypes.addressof(c), _ptr(cache), _ptr(ws),
+                                                    ws.numel(), _stream()))
 
 
 def lte_attn_bwd(s, c, q, k, v, o, lse, dO, z, idx, cnt, lam=None, flags=BWD_CNN_INPUT_GRAD, want_dbias=True,

@@ -81,18 +81,45 @@ def test_stack_tensor_core_path(B, H, T, bias):
     check_idx(idx.cpu().numpy(), cnt.cpu().numpy(), z64, cfg.W, cfg.R, 0, 0.5)
 
 
-def test_stack_rejected_elsewhere():
-    """decode and cache_init take the single layer only."""
-    cfg = synth.Config("stack", "bf16", 1, 2, 64, 64, 16, 8, 7, 0.1)
-    wl, wout, bl, bout = _stack_params(cfg.H, 64, 1, False)
-    c = lte.conv_stack([torch.from_numpy(w).cuda() for w in wl], torch.from_numpy(wout).cuda())
-    s = shape_of(cfg, B=1)
-    x = synth.make(cfg, 0)
-    k, v = dev(x["k"], "bf16"), dev(x["v"], "bf16")
-    z = lte.lte_scores(s, c, k, v)
-    idx, cnt = lte.lte_select(s, z)
-    with pytest.raises(Exception):
-        lte.lte_cache_init(s, c, k, v, z, idx, cnt)
+@pytest.mark.parametrize("dtype,d,W,R,T0,steps,period", [("bf16", 64, 32, 24, 100, 90, 19), ("bf16", 64, 40, 16, 0, 120, 27),
+                                                         ("f32", 32, 24, 12, 30, 70, 5), ("bf16", 64, 128, 64, 300, 150, 115)])
+def test_stack_in_decode(dtype, d, W, R, T0, steps, period):
+    """Prefill with the stack, then decode: the step scores nothing, lte_cache_score runs every `period` <= W - 13 steps
+    (lazy batches), and outputs and the final pool equal the oracle's streaming simulation on the stack's logits."""
+    cfg = synth.Config("stackdec", dtype, 2, 2, d, T0 + steps, W, R, 7, 0.1)
+    Ttot = T0 + steps
+    x = synth.make(cfg, 4, T=Ttot)
+    wl, wout, bl, bout = _stack_params(cfg.H, d, 4, True)
+    t = lambda a: torch.from_numpy(a).cuda()
+    c = lte.conv_stack([t(w) for w in wl], t(wout), [t(b) for b in bl], t(bout))
+    q, k, v = (dev(x[n], dtype) for n in "qkv")
+    s0 = shape_of(cfg, T=T0, B=cfg.B)
+    if T0 > 0:
+        kp, vp = k[:, :, :T0].contiguous(), v[:, :, :T0].contiguous()
+        z = lte.lte_scores(s0, c, kp, vp)
+        idx, cnt = lte.lte_select(s0, z)
+        cache = lte.lte_cache_init(s0, c, kp, vp, z, idx, cnt)
+    else:
+        cache = lte.lte_cache_init(s0, c)
+    outs, lses = [], []
+    for i, n in enumerate(range(T0, Ttot)):
+        if i % period == 0:
+            lte.lte_cache_score(s0, c, cache)
+        o1, l1 = lte.lte_attn_decode(s0, c, cache, q[:, :, n].contiguous(), k[:, :, n].contiguous(), v[:, :, n].contiguous())
+        outs.append(o1.float().cpu().numpy()); lses.append(l1.cpu().numpy())
+    torch.cuda.synchronize()
+    assert lte.lib().lte_device_status() == 0
+    z64 = orc.scores_stack(x["k"], x["v"], wl, bl, wout, bout)
+    o64, l64, pidx, pcnt = orc.stream(x["q"], x["k"], x["v"], z64, W, R, 0, n_from=T0)
+    tol = 2e-2 if dtype == "bf16" else 1e-4
+    assert np.max(np.abs(np.stack(outs, axis=2) - o64)) <= tol
+    assert np.max(np.abs(np.stack(lses, axis=2) - l64)) <= tol
+    from tests.test_gpu_decode import _read_pool
+    pools, ns = _read_pool(cache, cfg, cfg.B)
+    assert all(n == Ttot for n in ns)
+    for bh, pool in enumerate(pools):
+        b, h = divmod(bh, cfg.H)
+        assert np.array_equal(pool, pidx[b, h, :pcnt[b, h]])
 
 
 # ---- backward through the stack (lte_attn_bwd with the three-layer scorer) ---------------------------------------------
