@@ -479,7 +479,8 @@ WsPlan plan(const Params& p, uint32_t flags)
     w.delta = off; off += up(bht * 4);
     w.dz = off; off += up(bht * 4);
     if (p.stack) {                                  // the stack's backward keeps one packed partial gradient per CTA
-        w.part_w = off; off += up(stack_bwd_workspace(p));
+        const size_t a = stack_bwd_workspace(p), b = stack_bwd_tc_workspace(p);
+        w.part_w = off; off += up(a > b ? a : b);
         w.part_b = off;
     } else {
         w.part_w = off; off += up((size_t)p.H * p.B * w.nchunk * p.K * 2 * p.d * 4);
@@ -533,7 +534,10 @@ int run(const Params& p, const void* q, const void* k, const void* v, const void
                                                           z, idx, cnt, lambda, (T*)dk, (T*)dv, dk32, dv32, dz, p.H, p.T,
                                                           p.W, p.R, p.half, p.zthr, p.scale);
     }
-    if (p.stack) return launch_stack_bwd(p, k, v, dz, dk, dv, dw, dbias, want_in, part_w, st);
+    if (p.stack) {                                  // bf16: tensor cores; fp32 storage: the fp32 kernel
+        if (stack_bwd_tc_workspace(p) > 0) return launch_stack_bwd_tc(p, k, v, dz, dk, dv, dw, dbias, want_in, part_w, st);
+        return launch_stack_bwd(p, k, v, dz, dk, dv, dw, dbias, want_in, part_w, st);
+    }
     const int per_head = p.K * 2 * D;
     dim3 gr((per_head + 255) / 256, p.H);
     if constexpr (sizeof(T) == 2 && (D == 64 || D == 128)) {

@@ -86,6 +86,9 @@ int launch_scores_stack(const Params& p, const void* k, const void* v, float* z,
 size_t scores_stack_weight_floats(int d, int H);
 size_t scores_stack_tc_workspace(const Params& p);
 size_t stack_bwd_workspace(const Params& p);
+size_t stack_bwd_tc_workspace(const Params& p);
+int launch_stack_bwd_tc(const Params& p, const void* k, const void* v, const float* dz, void* dk, void* dv, float* dw,
+                        float* dbias, bool input_grad, void* ws, cudaStream_t st);
 int launch_stack_bwd(const Params& p, const void* k, const void* v, const float* dz, void* dk, void* dv, float* dw,
                      float* dbias, bool input_grad, void* part, cudaStream_t st);
 int launch_scores_stack_tc(const Params& p, const void* k, const void* v, float* z, float* r, void* ws, size_t ws_bytes,

@@ -13,6 +13,7 @@ int prefill_status_fetch_and_clear();
 int decode_status_fetch_and_clear();
 int scores_status_fetch_and_clear();
 int stack_tc_status_fetch_and_clear();
+int stack_bwd_tc_status_fetch_and_clear();
 int bwd_status_fetch_and_clear();
 int decode_tc_status_fetch_and_clear();
 
@@ -124,8 +125,9 @@ int lte_device_status(void)
     const int b = bwd_status_fetch_and_clear();
     const int d = decode_tc_status_fetch_and_clear();
     const int t = stack_tc_status_fetch_and_clear();
-    if (h < 0 || g < 0 || f < 0 || b < 0 || d < 0 || t < 0) return LTE_ERR_CUDA;
-    return (h == 0 && g == 0 && f == 0 && b == 0 && d == 0 && t == 0) ? LTE_OK : LTE_ERR_DEVICE_STATUS;
+    const int u = stack_bwd_tc_status_fetch_and_clear();
+    if (h < 0 || g < 0 || f < 0 || b < 0 || d < 0 || t < 0 || u < 0) return LTE_ERR_CUDA;
+    return (h == 0 && g == 0 && f == 0 && b == 0 && d == 0 && t == 0 && u == 0) ? LTE_OK : LTE_ERR_DEVICE_STATUS;
 }
 
 size_t lte_workspace_bytes(int op, const lte_shape* s, const lte_conv* c)
