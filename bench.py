@@ -401,7 +401,7 @@ def _extra_s(out, torch, lte, synth, pk, flush, n5):
         "max_abs_z_difference_between_kernels": float(dz), "fraction_kept": kept}
     del x, z
     # backward through the stack at the training shape (C5): the attention backward is the same as with the single layer,
-    # the scorer's part is the fp32 kernel
+    # the scorer's part runs on the tensor cores (plain bf16 operands)
     cfg5 = synth.CONFIGS["C5"]
     x5 = device_inputs(cfg5, 8, torch, with_dO=True)
     s5 = lte.shape(cfg5.B, cfg5.H, cfg5.T, cfg5.d, cfg5.W, cfg5.R, lte.BF16)
@@ -425,8 +425,8 @@ def _extra_s(out, torch, lte, synth, pk, flush, n5):
         "workload": "C5 shape, lte_attn_bwd with the stack (weight, bias and input gradients)",
         "bwd_ms": t_bs * 1e3, "bwd_ms_single_layer_scorer": t_b1 * 1e3,
         "stack_part_ms": (t_bs - t_b1) * 1e3 if t_bs > t_b1 else None,
-        "roofline": {"bound": "alu", "achieved": 3 * fl5 / max(t_bs - t_b1, 1e-9) / 1e12, "peak": alu_peak / 1e12, "unit": "TFLOP/s",
-                     "frac": 3 * fl5 / max(t_bs - t_b1, 1e-9) / alu_peak,
+        "roofline": {"bound": "tensor", "achieved": 3 * fl5 / max(t_bs - t_b1, 1e-9) / 1e12, "peak": pk["bf16_tflops"], "unit": "TFLOP/s",
+                     "frac": 3 * fl5 / max(t_bs - t_b1, 1e-9) / 1e12 / pk["bf16_tflops"], "peak_source": pk["source"],
                      "note": "3 x the forward's products (forward again, transposed products, weight gradients) over the time the stack adds"}}
     del x5, o5, lse5, z5
     # the stack in decode at the C4 cache shape (prompt of 1024 tokens): the step scores nothing, lte_cache_score runs once per

@@ -575,11 +575,15 @@ int bt_chunks(const Params& p)
     int dev = 0, sms = 148;
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int BH = p.B * p.H, n_tiles = (p.T + BT_OWN - 1) / BT_OWN;
-    int chunks = (sms + BH - 1) / BH;
-    if (chunks < 1) chunks = 1;
-    if (chunks > n_tiles) chunks = n_tiles;
-    const int per = (n_tiles + chunks - 1) / chunks;
-    return (n_tiles + per - 1) / per;
+    // row chunks per (b,h): the split that minimises waves x (tiles per CTA + about one tile of set-up and write-out)
+    int best = 1;
+    long best_cost = -1;
+    for (int chunks = 1; chunks <= n_tiles && chunks <= 64; ++chunks) {
+        const int per = (n_tiles + chunks - 1) / chunks, eff = (n_tiles + per - 1) / per;
+        const long waves = ((long)BH * eff + sms - 1) / sms, cost = waves * (per + 1);
+        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = eff; }
+    }
+    return best;
 }
 
 }  // namespace
