@@ -747,9 +747,9 @@ int launch_ring_scatter_z(const Params& p, void* cache, const float* zlin, cudaS
 // ---- grouped-query attention: the other query heads of a key/value head -------------------------------------------
 // The step kernels above update the cache of a key/value head and attend for its first query head.  The remaining
 // G - 1 query heads attend over the updated block (ring rows of the min(n, W) newest tokens, cnt pool rows) here:
-// one block per key/value head, up to ATT_Q query heads per pass.  The warps take the rows in turn (lanes over the d
-// channels): logits into shared memory, block max and sum per query head, then the value rows weighted per query
-// head in registers and a reduction over the warps.
+// one block per key/value head, up to ATT_Q query heads per pass: logits by one thread per row (the queries in shared
+// memory, no reductions across lanes), block max and sum per query head, then the warps take the value rows in turn
+// (lanes over the d channels), weight them per query head in registers, and a reduction over the warps closes.
 constexpr int ATT_Q = 4;
 template <typename T, int D>
 __global__ void __launch_bounds__(DT) decode_attend_kernel(const unsigned char* __restrict__ cache, CacheLayout L,
@@ -759,6 +759,7 @@ __global__ void __launch_bounds__(DT) decode_attend_kernel(const unsigned char* 
     constexpr int C = D / 32, NW = DT / 32;
     extern __shared__ float att_sm[];                          // logits [ATT_Q][rows], then partial outputs [NW][ATT_Q][D]
     __shared__ float s_red[NW][ATT_Q];
+    __shared__ __align__(16) float s_q[ATT_Q][D];              // the pass's queries, pre-scaled
     __shared__ float s_mx[ATT_Q], s_sum[ATT_Q];
     const int bh = blockIdx.x, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     const unsigned char* blk = cache + L.header + (size_t)bh * L.stride;
@@ -771,6 +772,22 @@ __global__ void __launch_bounds__(DT) decode_attend_kernel(const unsigned char* 
     float* s_out = att_sm + (size_t)ATT_Q * rows;
     // element (r, ch): in the swizzled layout (bf16, d = 64) 16-byte chunk ch / 8 of row r sits at position (ch / 8) ^ (r & 7)
     auto pos_of = [&](int r, int ch) { return L.swz ? ((((ch >> 3) ^ (r & 7)) << 3) | (ch & 7)) : ch; };
+    // a lane owns the channel pairs (2 lane, 2 lane + 1) + 64 j: one 4- or 8-byte load per pair, a row of d = 64 per warp load
+    auto ch_of = [&](int c) { return C == 1 ? lane : 2 * lane + (c & 1) + 64 * (c >> 1); };   // d = 32: one channel per lane
+    auto load_row = [&](const T* base, int r, float (&out)[C]) {
+        if constexpr (C == 1) out[0] = to_f(base[(size_t)r * D + pos_of(r, lane)]);
+#pragma unroll
+        for (int j = 0; j < C / 2; ++j) {
+            const T* p2 = base + (size_t)r * D + pos_of(r, 2 * lane + 64 * j);
+            if constexpr (sizeof(T) == 2) {
+                const uint32_t u = *reinterpret_cast<const uint32_t*>(p2);
+                out[2 * j] = __uint_as_float(u << 16); out[2 * j + 1] = __uint_as_float(u & 0xffff0000u);
+            } else {
+                const float2 u = *reinterpret_cast<const float2*>(p2);
+                out[2 * j] = u.x; out[2 * j + 1] = u.y;
+            }
+        }
+    };
     for (int g0 = 1; g0 < G; g0 += ATT_Q) {
         const int nq = G - g0 < ATT_Q ? G - g0 : ATT_Q;
         float qv[ATT_Q][C];
@@ -778,26 +795,51 @@ __global__ void __launch_bounds__(DT) decode_attend_kernel(const unsigned char* 
         for (int u = 0; u < ATT_Q; ++u)
 #pragma unroll
             for (int c = 0; c < C; ++c)
-                qv[u][c] = u < nq ? to_f(q1[((size_t)bh * G + g0 + u) * D + lane + 32 * c]) * scale : 0.f;
-        // ---- logits ----
+                qv[u][c] = u < nq ? to_f(q1[((size_t)bh * G + g0 + u) * D + ch_of(c)]) * scale : 0.f;
+        // ---- logits: a thread takes whole rows (no reductions across lanes), the queries come from shared memory ----
+        __syncthreads();                                       // s_q of the previous pass has been read
+#pragma unroll
+        for (int u = 0; u < ATT_Q; ++u)
+#pragma unroll
+            for (int c = 0; c < C; ++c) s_q[u][ch_of(c)] = qv[u][c];
+        __syncthreads();
         float mx[ATT_Q];
 #pragma unroll
         for (int u = 0; u < ATT_Q; ++u) mx[u] = -INFINITY;
-        for (int a = wid; a < rows; a += NW) {
+        for (int a = tid; a < rows; a += DT) {
             const int r = a < n_ring ? a : W + (a - n_ring);
-            float kk[C];
+            constexpr int EPV = 16 / sizeof(T);                // elements per 16-byte vector
+            float dot[ATT_Q];
 #pragma unroll
-            for (int c = 0; c < C; ++c) kk[c] = to_f(Kc[(size_t)r * D + pos_of(r, lane + 32 * c)]);
+            for (int u = 0; u < ATT_Q; ++u) dot[u] = 0.f;
+#pragma unroll 2
+            for (int cv = 0; cv < D / EPV; ++cv) {
+                const int pos = L.swz ? (cv ^ (r & 7)) : cv;
+                const uint4 raw = *reinterpret_cast<const uint4*>(Kc + (size_t)r * D + pos * EPV);
+                float kf[EPV];
+                if constexpr (sizeof(T) == 2) {
+                    const uint32_t wv[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) { kf[2 * e] = __uint_as_float(wv[e] << 16); kf[2 * e + 1] = __uint_as_float(wv[e] & 0xffff0000u); }
+                } else {
+                    kf[0] = __uint_as_float(raw.x); kf[1] = __uint_as_float(raw.y); kf[2] = __uint_as_float(raw.z); kf[3] = __uint_as_float(raw.w);
+                }
+#pragma unroll
+                for (int u = 0; u < ATT_Q; ++u)
+#pragma unroll
+                    for (int e = 0; e < EPV; e += 4) {
+                        const float4 q4 = *reinterpret_cast<const float4*>(&s_q[u][cv * EPV + e]);
+                        dot[u] = fmaf(kf[e], q4.x, fmaf(kf[e + 1], q4.y, fmaf(kf[e + 2], q4.z, fmaf(kf[e + 3], q4.w, dot[u]))));
+                    }
+            }
 #pragma unroll
             for (int u = 0; u < ATT_Q; ++u) {
-                float sdot = 0.f;
-#pragma unroll
-                for (int c = 0; c < C; ++c) sdot = fmaf(qv[u][c], kk[c], sdot);
-                sdot = warp_sum(sdot);
-                mx[u] = fmaxf(mx[u], sdot);
-                if (lane == 0) s_log[(size_t)u * rows + a] = sdot;
+                mx[u] = fmaxf(mx[u], dot[u]);
+                s_log[(size_t)u * rows + a] = dot[u];
             }
         }
+#pragma unroll
+        for (int u = 0; u < ATT_Q; ++u) mx[u] = warp_max(mx[u]);
         if (lane == 0)
 #pragma unroll
             for (int u = 0; u < ATT_Q; ++u) s_red[wid][u] = mx[u];
@@ -839,8 +881,7 @@ __global__ void __launch_bounds__(DT) decode_attend_kernel(const unsigned char* 
         for (int a = wid; a < rows; a += NW) {
             const int r = a < n_ring ? a : W + (a - n_ring);
             float vv[C];
-#pragma unroll
-            for (int c = 0; c < C; ++c) vv[c] = to_f(Vc[(size_t)r * D + pos_of(r, lane + 32 * c)]);
+            load_row(Vc, r, vv);
 #pragma unroll
             for (int u = 0; u < ATT_Q; ++u) {
                 const float pj = s_log[(size_t)u * rows + a];
@@ -851,7 +892,7 @@ __global__ void __launch_bounds__(DT) decode_attend_kernel(const unsigned char* 
 #pragma unroll
         for (int u = 0; u < ATT_Q; ++u)
 #pragma unroll
-            for (int c = 0; c < C; ++c) s_out[((size_t)wid * ATT_Q + u) * D + lane + 32 * c] = acc[u][c];
+            for (int c = 0; c < C; ++c) s_out[((size_t)wid * ATT_Q + u) * D + ch_of(c)] = acc[u][c];
         __syncthreads();
         for (int e = tid; e < nq * D; e += DT) {
             const int u = e / D, ch = e - u * D;
