@@ -48,7 +48,7 @@ typedef struct lte_shape {
     int32_t group;                 /* grouped-query attention: query heads per key/value head; 0 or 1 = one.
                                       H counts key/value heads (k, v, z, idx, cnt, the cache); q, o, lse have
                                       H * group heads, those of one key/value head adjacent: [B, H, group, ...].
-                                      lte_attn_prefill and lte_attn_decode; the backward answers UNSUPPORTED      */
+                                      dq has H * group heads too; dk, dv, dw, dbias are summed over a group          */
 } lte_shape;
 
 typedef struct lte_conv {

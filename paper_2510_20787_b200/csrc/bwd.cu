@@ -31,14 +31,14 @@ __global__ void __launch_bounds__(128) bwd_dq_kernel(const T* __restrict__ q, co
                                                      const T* __restrict__ dO, const float* __restrict__ lse,
                                                      const int32_t* __restrict__ idx, const int32_t* __restrict__ cnt,
                                                      T* __restrict__ dq, float* __restrict__ delta, int Tlen, int W,
-                                                     int R, float scale)
+                                                     int R, float scale, int G)
 {
     constexpr int C = D / 32;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int i = blockIdx.x * 4 + warp;
-    const int bh = blockIdx.y;
+    const int bh = blockIdx.y, bhk = bh / G;                   // query head; its key/value head
     if (i >= Tlen) return;
-    const size_t base = (size_t)bh * Tlen * D;
+    const size_t base = (size_t)bh * Tlen * D, kbase = (size_t)bhk * Tlen * D;
     float qv[C], gv[C], acc[C];
     float dl = 0.f;
 #pragma unroll
@@ -50,8 +50,8 @@ __global__ void __launch_bounds__(128) bwd_dq_kernel(const T* __restrict__ q, co
     dl = warp_sum(dl);
     if (lane == 0) delta[(size_t)bh * Tlen + i] = dl;
     const float li = lse[(size_t)bh * Tlen + i];
-    const int32_t* id = idx + (size_t)bh * R;
-    const int n_ret = cnt[bh];
+    const int32_t* id = idx + (size_t)bhk * R;
+    const int n_ret = cnt[bhk];
     const int lo = i - W + 1 > 0 ? i - W + 1 : 0;
     int nvis = 0;
     for (int m0 = 0; m0 < n_ret; m0 += 32) {
@@ -63,8 +63,8 @@ __global__ void __launch_bounds__(128) bwd_dq_kernel(const T* __restrict__ q, co
     const int total = nvis + (i - lo + 1);
     for (int a = 0; a < total; ++a) {
         const int j = a < nvis ? id[a] : lo + (a - nvis);
-        const T* kr = k + base + (size_t)j * D;
-        const T* vr = v + base + (size_t)j * D;
+        const T* kr = k + kbase + (size_t)j * D;
+        const T* vr = v + kbase + (size_t)j * D;
         float s = 0.f, dp = 0.f, kk[C];
 #pragma unroll
         for (int c = 0; c < C; ++c) {
@@ -93,7 +93,7 @@ __global__ void __launch_bounds__(128) bwd_dkv_kernel(const T* __restrict__ q, c
                                                       const int32_t* __restrict__ cnt, const float* __restrict__ lambda,
                                                       T* __restrict__ dk, T* __restrict__ dv, float* __restrict__ dk32,
                                                       float* __restrict__ dv32, float* __restrict__ dz, int H, int Tlen,
-                                                      int W, int R, int half, float zthr, float scale)
+                                                      int W, int R, int half, float zthr, float scale, int G)
 {
     constexpr int C = D / 32;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -116,9 +116,11 @@ __global__ void __launch_bounds__(128) bwd_dkv_kernel(const T* __restrict__ q, c
         kept = lo < cnt[bh] && id[lo] == j;
     }
     const int iend = kept ? Tlen - 1 : (j + W - 1 < Tlen - 1 ? j + W - 1 : Tlen - 1);
-    for (int i = j; i <= iend; ++i) {
-        const T* qr = q + base + (size_t)i * D;
-        const T* gr = dO + base + (size_t)i * D;
+    for (int gi = 0; gi < G * (iend - j + 1); ++gi) {          // the group's query heads in turn, each over its queries
+        const int g = gi / (iend - j + 1), i = j + gi % (iend - j + 1);
+        const size_t qbase = ((size_t)bh * G + g) * Tlen;
+        const T* qr = q + (qbase + i) * D;
+        const T* gr = dO + (qbase + i) * D;
         float s = 0.f, dp = 0.f, qq[C], gg[C];
 #pragma unroll
         for (int c = 0; c < C; ++c) {
@@ -131,8 +133,8 @@ __global__ void __launch_bounds__(128) bwd_dkv_kernel(const T* __restrict__ q, c
             s += __shfl_xor_sync(0xffffffffu, s, off);
             dp += __shfl_xor_sync(0xffffffffu, dp, off);
         }
-        const float p = expf(s - lse[(size_t)bh * Tlen + i]);
-        const float ds = p * (dp - delta[(size_t)bh * Tlen + i]);
+        const float p = expf(s - lse[qbase + i]);
+        const float ds = p * (dp - delta[qbase + i]);
 #pragma unroll
         for (int c = 0; c < C; ++c) { av[c] = fmaf(p, gg[c], av[c]); ak[c] = fmaf(ds, qq[c], ak[c]); }
     }
@@ -476,7 +478,7 @@ WsPlan plan(const Params& p, uint32_t flags)
     const size_t bht = (size_t)p.B * p.H * p.T;
     w.nchunk = (p.T + CHUNK - 1) / CHUNK;
     size_t off = 0;
-    w.delta = off; off += up(bht * 4);
+    w.delta = off; off += up(bht * p.G * 4);        // one per query head
     w.dz = off; off += up(bht * 4);
     if (p.stack) {                                  // the stack's backward keeps one packed partial gradient per CTA
         const size_t a = stack_bwd_workspace(p), b = stack_bwd_tc_workspace(p);
@@ -513,13 +515,13 @@ int run(const Params& p, const void* q, const void* k, const void* v, const void
     float* dv32 = (float*)(base + w.dv32);
     const bool want_in = flags & LTE_BWD_CNN_INPUT_GRAD;
     const bool f32 = want_in && !p.stack;             // the stack's backward adds its input gradient to dk, dv in place
-    dim3 grid((p.T + 3) / 4, p.B * p.H);
+    dim3 grid((p.T + 3) / 4, p.B * p.H), gridq((p.T + 3) / 4, p.B * p.H * p.G);
     if constexpr (sizeof(T) == 2 && (D == 64 || D == 128)) {
         const int e = launch_bwd_dq_tc(p, q, k, v, o, lse, dO, idx, cnt, dq, delta, st);
         if (e != LTE_OK) return e;
     } else {
-        bwd_dq_kernel<T, D><<<grid, 128, 0, st>>>((const T*)q, (const T*)k, (const T*)v, (const T*)o, (const T*)dO, lse,
-                                                  idx, cnt, (T*)dq, delta, p.T, p.W, p.R, p.scale);
+        bwd_dq_kernel<T, D><<<gridq, 128, 0, st>>>((const T*)q, (const T*)k, (const T*)v, (const T*)o, (const T*)dO, lse,
+                                                   idx, cnt, (T*)dq, delta, p.T, p.W, p.R, p.scale, p.G);
     }
     if constexpr (sizeof(T) == 2 && (D == 64 || D == 128)) {
         const int e = launch_bwd_dkv_tc(p, q, k, v, lse, dO, delta, z, idx, cnt, lambda, dk, dv, dk32, dv32, dz, base + w.ret,
@@ -528,11 +530,11 @@ int run(const Params& p, const void* q, const void* k, const void* v, const void
     } else if (f32) {
         bwd_dkv_kernel<T, D, true><<<grid, 128, 0, st>>>((const T*)q, (const T*)k, (const T*)v, (const T*)dO, lse, delta,
                                                          z, idx, cnt, lambda, (T*)dk, (T*)dv, dk32, dv32, dz, p.H, p.T,
-                                                         p.W, p.R, p.half, p.zthr, p.scale);
+                                                         p.W, p.R, p.half, p.zthr, p.scale, p.G);
     } else {
         bwd_dkv_kernel<T, D, false><<<grid, 128, 0, st>>>((const T*)q, (const T*)k, (const T*)v, (const T*)dO, lse, delta,
                                                           z, idx, cnt, lambda, (T*)dk, (T*)dv, dk32, dv32, dz, p.H, p.T,
-                                                          p.W, p.R, p.half, p.zthr, p.scale);
+                                                          p.W, p.R, p.half, p.zthr, p.scale, p.G);
     }
     if (p.stack) {                                  // bf16: tensor cores; fp32 storage: the fp32 kernel
         if (stack_bwd_tc_workspace(p) > 0) return launch_stack_bwd_tc(p, k, v, dz, dk, dv, dw, dbias, want_in, part_w, st);

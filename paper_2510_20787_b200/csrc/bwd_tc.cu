@@ -53,7 +53,7 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                  const __nv_bfloat16* __restrict__ kg, const __nv_bfloat16* __restrict__ vg,
                  const __nv_bfloat16* __restrict__ og, const __nv_bfloat16* __restrict__ dog,
                  const float* __restrict__ lse, const int32_t* __restrict__ idx, const int32_t* __restrict__ cnt,
-                 __nv_bfloat16* __restrict__ dq, float* __restrict__ delta, int Tlen, int W, int R, float scale)
+                 __nv_bfloat16* __restrict__ dq, float* __restrict__ delta, int Tlen, int W, int R, float scale, int G)
 {
     pdl_launch_dependents();
     pdl_wait();                                                // see launch_pdl: earlier kernels of the stream have completed
@@ -71,13 +71,13 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     volatile int* s_idx = reinterpret_cast<volatile int*>(smem_raw + S::OFF_IDX);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int bh = blockIdx.y;
+    const int bh = blockIdx.y, bhk = bh / G;                   // query head; its key/value head (grouped queries: G per head)
     const int i0 = blockIdx.x * BM;
     const int i_hi = min(i0 + BM - 1, Tlen - 1);
     const int j_start = max(i0 - W + 1, 0);
     const int n_win = (i_hi - j_start + 1 + BN - 1) / BN;
-    const int32_t* id = idx + (size_t)bh * R;
-    const int n_ret = cnt[bh];
+    const int32_t* id = idx + (size_t)bhk * R;
+    const int n_ret = cnt[bhk];
 
     if (tid == 0) {
         mbar_init(bar_q, 1);
@@ -124,7 +124,7 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                 if (leader) {
                     mbar_expect_tx(bar, S::KVTILE);
 #pragma unroll
-                    for (int sb = 0; sb < SUB; ++sb) tma_load_3d(dst + sb * 8192, is_v ? &tmV : &tmK, sb * 64, y, bh, bar);
+                    for (int sb = 0; sb < SUB; ++sb) tma_load_3d(dst + sb * 8192, is_v ? &tmV : &tmK, sb * 64, y, bhk, bar);
                 }
             };
             auto need_g = [&](uint32_t phase) {
@@ -271,7 +271,7 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                 for (int ps = 0; ps < 4; ++ps) {
                     const int row = ps * 16 + g_row;
                     const bool ok = rows4[ps] >= 0;
-                    const __nv_bfloat16* src = (is_v ? vg : kg) + ((size_t)bh * Tlen + (ok ? rows4[ps] : 0)) * D;
+                    const __nv_bfloat16* src = (is_v ? vg : kg) + ((size_t)bhk * Tlen + (ok ? rows4[ps] : 0)) * D;
 #pragma unroll
                     for (int c = g_sub; c < D / 8; c += 8) {
                         const uint32_t off = (c >> 3) * 8192 + row * 128 + (((c & 7) ^ (row & 7)) << 4);
@@ -429,7 +429,7 @@ bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                   const int32_t* __restrict__ cnt, __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv,
                   float* __restrict__ dk32, float* __restrict__ dv32, float* __restrict__ dr_win,
                   float* __restrict__ dk_ret, float* __restrict__ dv_ret, float* __restrict__ dr_ret, int n_wt, int Tlen,
-                  int W, int R, float scale)
+                  int W, int R, float scale, int G)
 {
     pdl_launch_dependents();
     pdl_wait();                                                // see launch_pdl: earlier kernels of the stream have completed
@@ -464,6 +464,10 @@ bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         ib_start = (first / 64) * 64;
         n_blk = first <= Tlen - 1 ? (Tlen - 1 - ib_start) / 64 + 1 : 0;
     }
+    // grouped queries: the G query heads of this key/value head walk the same query blocks one after the other and
+    // accumulate into the same dK, dV; walk step t is block t % n_pos of query head bh G + t / n_pos
+    const int n_pos = n_blk;
+    n_blk *= G;
 
     const uint32_t sK = base + S::OFF_K, sV = base + S::OFF_V, sQ = base + S::OFF_Q, sDO = base + S::OFF_DO;
     const uint32_t sPT = base + S::OFF_PT, sDST = base + S::OFF_DST;
@@ -498,13 +502,13 @@ bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
             auto tma_blk = [&](int t) {
                 const int st = t % NST;
                 const uint32_t bar = bar_q0 + 8 * st;
-                const int y = ib_start + t * 64;
+                const int y = ib_start + (t % n_pos) * 64, bhq = bh * G + t / n_pos;
                 if (leader) {
                     mbar_expect_tx(bar, 2 * S::QBLK);
 #pragma unroll
                     for (int sb = 0; sb < SUB; ++sb) {
-                        tma_load_3d(sQ + st * S::QBLK + sb * 8192, &tmQ, sb * 64, y, bh, bar);
-                        tma_load_3d(sDO + st * S::QBLK + sb * 8192, &tmDO, sb * 64, y, bh, bar);
+                        tma_load_3d(sQ + st * S::QBLK + sb * 8192, &tmQ, sb * 64, y, bhq, bar);
+                        tma_load_3d(sDO + st * S::QBLK + sb * 8192, &tmDO, sb * 64, y, bhq, bar);
                     }
                 }
             };
@@ -588,9 +592,11 @@ bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         const uint32_t lane_base = ((uint32_t)(warp * 32)) << 16;
         // per-column constants of the next block, fetched one block ahead: thread c < 64 holds L2, thread 64 + c delta
         auto col_fetch = [&](int t) -> float {
-            const int i = ib_start + t * 64 + (tid & 63);
-            if (t >= n_blk || i >= Tlen) return tid < 64 ? INFINITY : 0.f;      // L2 = +inf makes P = 0
-            return tid < 64 ? lse[(size_t)bh * Tlen + i] * kLog2e : delta[(size_t)bh * Tlen + i];
+            if (t >= n_blk) return 0.f;
+            const int i = ib_start + (t % n_pos) * 64 + (tid & 63);
+            if (i >= Tlen) return tid < 64 ? INFINITY : 0.f;                    // L2 = +inf makes P = 0
+            const size_t bhq = (size_t)bh * G + t / n_pos;
+            return tid < 64 ? lse[bhq * Tlen + i] * kLog2e : delta[bhq * Tlen + i];
         };
         float col_next = col_fetch(0);
 
@@ -599,7 +605,7 @@ bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
             s_col[tid] = col_next;
             col_next = col_fetch(t + 1);
             group_sync();
-            const int ib = ib_start + t * 64;
+            const int ib = ib_start + (t % n_pos) * 64;
             int c_lo, c_hi;                                    // query columns of the block this key row may be seen by
             if (pos < 0) { c_lo = 1 << 20; c_hi = -(1 << 20); }
             else if (!is_ret) { c_lo = pos - ib; c_hi = min(pos + W - 1, Tlen - 1) - ib; }
@@ -798,11 +804,11 @@ __global__ void bwd_dz_kernel(float* __restrict__ dz, const float* __restrict__ 
 int launch_bwd_dq_tc(const Params& p, const void* q, const void* k, const void* v, const void* o, const float* lse,
                      const void* dO, const int32_t* idx, const int32_t* cnt, void* dq, float* delta, cudaStream_t st)
 {
-    const int BH = p.B * p.H;
+    const int BHK = p.B * p.H, BH = BHK * p.G;                 // key/value heads, query heads
     CUtensorMap tq, tdo, to, tdq, tk, tv;
     if (!make_map(&tq, q, BH, p.T, p.d, BM) || !make_map(&tdo, dO, BH, p.T, p.d, BM) || !make_map(&to, o, BH, p.T, p.d, BM) ||
         !make_map(&tdq, dq, BH, p.T, p.d, 32) ||
-        !make_map(&tk, k, BH, p.T, p.d, BN) || !make_map(&tv, v, BH, p.T, p.d, BN))
+        !make_map(&tk, k, BHK, p.T, p.d, BN) || !make_map(&tv, v, BHK, p.T, p.d, BN))
         return LTE_ERR_CUDA;
     dim3 grid((p.T + BM - 1) / BM, BH);
 #define LTE_GO(D)                                                                                                  \
@@ -815,7 +821,7 @@ int launch_bwd_dq_tc(const Params& p, const void* q, const void* k, const void* 
         }                                                                                                          \
         launch_pdl(bwd_dq_tc_kernel<D>, grid, dim3(NTHREADS), SmemQ<D>::BYTES, st,                            \
             tq, tdo, to, tdq, tk, tv, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (const __nv_bfloat16*)o,        \
-            (const __nv_bfloat16*)dO, lse, idx, cnt, (__nv_bfloat16*)dq, delta, p.T, p.W, p.R, p.scale);           \
+            (const __nv_bfloat16*)dO, lse, idx, cnt, (__nv_bfloat16*)dq, delta, p.T, p.W, p.R, p.scale, p.G);      \
     } while (0)
     if (p.d == 64) LTE_GO(64); else if (p.d == 128) LTE_GO(128); else return LTE_ERR_UNSUPPORTED;
 #undef LTE_GO
@@ -836,7 +842,7 @@ int launch_bwd_dkv_tc(const Params& p, const void* q, const void* k, const void*
     const int BH = p.B * p.H;
     CUtensorMap tk, tv, tq, tdo, tdk, tdv;
     if (!make_map(&tk, k, BH, p.T, p.d, 128) || !make_map(&tv, v, BH, p.T, p.d, 128) ||
-        !make_map(&tq, q, BH, p.T, p.d, 64) || !make_map(&tdo, dO, BH, p.T, p.d, 64) ||
+        !make_map(&tq, q, BH * p.G, p.T, p.d, 64) || !make_map(&tdo, dO, BH * p.G, p.T, p.d, 64) ||
         !make_map(&tdk, dk, BH, p.T, p.d, 32) || !make_map(&tdv, dv, BH, p.T, p.d, 32))
         return LTE_ERR_CUDA;
     const size_t n = (size_t)BH * (p.R > 0 ? p.R : 1);
@@ -856,7 +862,7 @@ int launch_bwd_dkv_tc(const Params& p, const void* q, const void* k, const void*
         launch_pdl(bwd_dkv_tc_kernel<D, F>, grid, dim3(NTHREADS), SmemK<D>::BYTES, st,                              \
             tk, tv, tq, tdo, tdk, tdv, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, lse, delta, idx, cnt,     \
             (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, dk32, dv32, dz, dk_ret, dv_ret, dr_ret, n_wt, p.T, p.W, p.R,   \
-            p.scale);                                                                                              \
+            p.scale, p.G);                                                                                         \
     } while (0)
     if (p.d == 64) { if (f32out) LTE_GO(64, true); else LTE_GO(64, false); }
     else if (p.d == 128) { if (f32out) LTE_GO(128, true); else LTE_GO(128, false); }

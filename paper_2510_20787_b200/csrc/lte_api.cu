@@ -261,7 +261,6 @@ int lte_attn_bwd(const lte_shape* s, const lte_conv* c, const void* q, const voi
     if (!q || !k || !v || !o || !lse || !dO || !z || !cnt || (s->R > 0 && !idx) || !dq || !dk || !dv || !dw)
         return LTE_ERR_INVALID_ARG;
     if (flags & ~LTE_BWD_CNN_INPUT_GRAD) return LTE_ERR_INVALID_ARG;
-    if (s->group > 1) return LTE_ERR_UNSUPPORTED;          // grouped-query attention: forward and decode only
     Params p = make_params(s, c);
     if (!ws || !aligned16(ws) || ws_bytes < bwd_workspace_bytes(p, flags)) return LTE_ERR_WORKSPACE;
     e = check_arch(); if (e) return e;

@@ -75,15 +75,32 @@ def test_decode_gqa(dtype, d, W, R, G, T0, steps):
     assert np.max(np.abs(l_n - l64)) <= TOL[dtype]
 
 
-def test_backward_rejects_groups():
-    cfg = synth.Config("gqa", "bf16", 1, 2, 64, 128, 16, 8, 7, 0.1)
-    x, q = _inputs(cfg, 2, 0)
-    s = lte.shape(1, 2, 128, 64, 16, 8, lte.BF16, group=2)
+@pytest.mark.parametrize("dtype,d,T,W,R,G,in_grad", [("bf16", 64, 300, 32, 24, 4, True), ("bf16", 128, 260, 48, 32, 2, True),
+                                                     ("f32", 32, 150, 16, 10, 3, True), ("bf16", 64, 520, 64, 64, 2, False)])
+def test_backward_gqa(dtype, d, T, W, R, G, in_grad):
+    """dq per query head; dk, dv, dw, dbias summed over the query heads of a group.  Everything downstream of dV is linear
+    in it (no Eq. 7 term here), so the reference is the oracle run per query head on repeated keys/values, summed."""
+    cfg = synth.Config("gqa", dtype, 2, 2, d, T, W, R, 7, 0.1)
+    x, q = _inputs(cfg, G, 21)
+    dO = synth.make(cfg.with_(H=cfg.H * G), 321, with_dO=True)["dO"]
+    s = lte.shape(cfg.B, cfg.H, T, d, W, R, tdtype(cfg), group=G)
     c = lte.conv(torch.from_numpy(x["w"]).cuda())
-    k, v, qd = dev(x["k"], "bf16"), dev(x["v"], "bf16"), dev(q, "bf16")
+    k, v, qd, gd = dev(x["k"], dtype), dev(x["v"], dtype), dev(q, dtype), dev(dO, dtype)
     z = lte.lte_scores(s, c, k, v)
     idx, cnt = lte.lte_select(s, z)
     o, lse = lte.lte_attn_prefill(s, qd, k, v, idx, cnt)
-    with pytest.raises(lte.LteError) as e:
-        lte.lte_attn_bwd(s, c, qd, k, v, o, lse, torch.ones_like(o), z, idx, cnt)
-    assert e.value.status == -2
+    flags = lte.BWD_CNN_INPUT_GRAD if in_grad else 0
+    dq, dk, dv, dw, db = lte.lte_attn_bwd(s, c, qd, k, v, o, lse, gd, z, idx, cnt, flags=flags)
+    torch.cuda.synchronize()
+    assert lte.lib().lte_device_status() == 0
+    rep = lambda a: np.repeat(a, G, axis=1)
+    z64 = z.cpu().numpy().astype(np.float64)
+    r = orc.attn_bwd(q, rep(x["k"]), rep(x["v"]), dO, rep(z64), rep(idx.cpu().numpy()), rep(cnt.cpu().numpy()),
+                     np.repeat(x["w"], G, axis=0), W, cnn_input_grad=in_grad)
+    grp = lambda a: a.reshape(a.shape[0], cfg.H, G, *a.shape[2:]).sum(axis=2)          # [B, H*G, ...] -> sum over the group
+    rel = lambda a, b: float(np.linalg.norm(np.asarray(a, np.float64) - b) / (np.linalg.norm(b) + 1e-30))
+    assert rel(dq.float().cpu().numpy(), r["dq"]) < 5e-2
+    assert rel(dk.float().cpu().numpy(), grp(r["dk"])) < 5e-2
+    assert rel(dv.float().cpu().numpy(), grp(r["dv"])) < 5e-2
+    assert rel(dw.cpu().numpy(), r["dw"].reshape(cfg.H, G, *r["dw"].shape[1:]).sum(axis=1)) < 5e-2
+    assert rel(db.cpu().numpy(), r["dbias"].reshape(cfg.H, G).sum(axis=1)) < 5e-2
