@@ -73,3 +73,38 @@ def test_host_side_validation_rejects_bad_arguments():
     args = [a(good), a(conv)] + [fake] * 9 + [None] + [fake] * 4 + [None, 0, fake, 16, None]
     assert L.lte_attn_bwd(*args) == -3                                                         # workspace too small
     assert lte.lte_cache_bytes(lte.shape(0, 2, 1, 32, 16, 8, lte.F32)) == 0
+
+
+def test_three_layer_stack_and_groups_host_side():
+    """Workspace sizes and argument checks of the entry points that take the three-layer stack or grouped queries
+    (no kernel is launched: validation fails first, or only sizes are asked for)."""
+    L = lte.lib()
+    a = ctypes.addressof
+    fake = 4096
+    stack = lte.LteConv(3, 3, 2, 256, 0)
+    single = lte.LteConv(1, 7, 1, 256, 0)
+    s = lte.shape(4, 16, 4096, 64, 128, 128, lte.BF16)
+    assert lte.lte_workspace_bytes(lte.OP_SCORES, s, stack) == 16 * 194176            # the split weight image per head
+    assert lte.lte_workspace_bytes(lte.OP_SCORES, lte.shape(4, 16, 4096, 64, 128, 128, lte.F32), stack) == 0
+    assert lte.lte_workspace_bytes(lte.OP_SCORES, lte.shape(4, 16, 4096, 32, 128, 128, lte.BF16), stack) == 0
+    dec = lte.lte_workspace_bytes(lte.OP_DECODE, s, stack)                             # ring copy (k, v), its logits, the image
+    assert dec >= 2 * 4 * 16 * 128 * 64 * 2 + 4 * 16 * 128 * 4 + 16 * 194176
+    assert lte.lte_workspace_bytes(lte.OP_DECODE, s, single) == 0
+    assert lte.lte_workspace_bytes(lte.OP_BWD, s, stack) > 16 * 129664                 # weight image + per-CTA partial gradients
+    # lte_cache_score: the stack only, a window of at least 20, an aligned and large enough workspace
+    assert L.lte_cache_score(a(s), a(single), fake, fake, 1 << 30, None) == -2
+    assert L.lte_cache_score(a(s), a(stack), None, fake, 1 << 30, None) == -1
+    assert L.lte_cache_score(a(s), a(stack), fake, None, 0, None) == -3
+    assert L.lte_cache_score(a(s), a(stack), fake, fake, 16, None) == -3
+    assert L.lte_cache_score(a(s), a(stack), fake, fake + 16, 1 << 30, None) == -3     # not 256-byte aligned
+    short = lte.shape(4, 16, 4096, 64, 16, 8, lte.BF16)
+    assert L.lte_cache_score(a(short), a(stack), fake, fake, 1 << 30, None) == -1
+    assert L.lte_attn_decode(a(short), a(stack), fake, fake, fake, fake, fake, fake, None) == -1
+    # the stack's backward: d = 64 only; negative group counts are rejected everywhere
+    s32 = lte.shape(1, 2, 128, 32, 16, 8, lte.BF16)
+    args = [a(s32), a(stack)] + [fake] * 9 + [None] + [fake] * 4 + [None, 0, fake, 1 << 30, None]
+    assert L.lte_attn_bwd(*args) == -2
+    neg = lte.shape(1, 2, 128, 64, 16, 8, lte.BF16, group=-1)
+    assert L.lte_attn_prefill(a(neg), fake, fake, fake, fake, fake, fake, fake, None, 0, None) == -1
+    # the shape struct ends with the group field (the binding and the header agree on the layout)
+    assert ctypes.sizeof(lte.LteShape) == 11 * 4 and lte.LteShape.group.offset == 40
