@@ -152,11 +152,12 @@ __global__ void __launch_bounds__(1024) select_reg_kernel(const float* __restric
 {
     __shared__ uint32_t s_part[2][32];
     __shared__ uint32_t s_wa[32], s_we[32];
+    __shared__ uint32_t s_list[kSelList + 2];
     pdl_launch_dependents();
     pdl_wait();                                            // z comes from the previous kernel
     const int bh = blockIdx.x;
     select_group<KPT>(z + (size_t)bh * T, idx + (size_t)bh * R, cnt + bh, ncand ? ncand + bh : nullptr, T, W, R, sink, zthr,
-                      (int)threadIdx.x, (int)blockDim.x, s_part, s_wa, s_we, [] { __syncthreads(); });
+                      (int)threadIdx.x, (int)blockDim.x, s_part, s_wa, s_we, [] { __syncthreads(); }, s_list);
 }
 
 }  // namespace

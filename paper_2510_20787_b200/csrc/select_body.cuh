@@ -20,10 +20,13 @@ __device__ __forceinline__ uint32_t select_key_of(const float* zz, int j, int si
     return z > zthr ? order_key(z) : 0u;
 }
 
+constexpr int kSelList = 1024;      // keys that share the upper half of the threshold: up to this many are settled by one warp
+
 template <int KPT, typename Sync>
 __device__ __forceinline__ void select_group(const float* __restrict__ zz, int32_t* __restrict__ out, int32_t* cnt_out,
                                              int32_t* ncand_out, int T, int W, int R, int sink, float zthr, int tid,
-                                             int nthr, uint32_t (*s_part)[32], uint32_t* s_wa, uint32_t* s_we, Sync sync)
+                                             int nthr, uint32_t (*s_part)[32], uint32_t* s_wa, uint32_t* s_we, Sync sync,
+                                             uint32_t* s_list = nullptr)
 {
     const int lane = tid & 31, wid = tid >> 5, nwarp = nthr >> 5;
     const int N = T - W > 0 ? T - W : 0;
@@ -53,12 +56,55 @@ __device__ __forceinline__ void select_group(const float* __restrict__ zz, int32
     uint32_t theta = 0, need_eq = 0;
     if (R > 0 && nc > (uint32_t)R) {
         uint32_t prefix = 0;
-        for (int bit = 31; bit >= 0; --bit) {
+        int bit = 31;
+        for (; bit >= 16; --bit) {
             const uint32_t cand = prefix | (1u << bit);
             uint32_t c = 0;
 #pragma unroll
             for (int i = 0; i < KPT; ++i) c += key[i] >= cand;
             if (block_sum(c) >= (uint32_t)R) prefix = cand;  // at least R keys are >= cand: the R-th largest is too
+        }
+        // The upper half of the R-th largest key is known.  Only the keys that share it can still move a count, and with
+        // spread-out logits they are few: they go into a short list, and one warp settles the lower 16 bits on it without
+        // any group barrier.  (s_list: kSelList entries, then the list length, then the result.)
+        bool done = false;
+        if (s_list != nullptr) {
+            const uint32_t hi = prefix >> 16;
+            uint32_t ca = 0, cm = 0;
+#pragma unroll
+            for (int i = 0; i < KPT; ++i) { ca += (key[i] >> 16) > hi; cm += (key[i] >> 16) == hi; }
+            const uint32_t above = block_sum(ca), match = block_sum(cm);
+            if (match <= (uint32_t)kSelList) {
+                if (tid == 0) s_list[kSelList] = 0u;
+                sync();
+#pragma unroll
+                for (int i = 0; i < KPT; ++i)
+                    if ((key[i] >> 16) == hi) s_list[atomicAdd(&s_list[kSelList], 1u)] = key[i];
+                sync();
+                if (wid == 0) {
+                    uint32_t pf = prefix;
+                    for (int b2 = 15; b2 >= 0; --b2) {
+                        const uint32_t cand = pf | (1u << b2);
+                        uint32_t c = 0;
+                        for (uint32_t l = lane; l < match; l += 32) c += s_list[l] >= cand;
+                        c = __reduce_add_sync(0xffffffffu, c);
+                        if (above + c >= (uint32_t)R) pf = cand;
+                    }
+                    if (lane == 0) s_list[kSelList + 1] = pf;
+                }
+                sync();
+                prefix = s_list[kSelList + 1];
+                done = true;
+            }
+        }
+        if (!done) {
+            for (; bit >= 0; --bit) {
+                const uint32_t cand = prefix | (1u << bit);
+                uint32_t c = 0;
+#pragma unroll
+                for (int i = 0; i < KPT; ++i) c += key[i] >= cand;
+                if (block_sum(c) >= (uint32_t)R) prefix = cand;
+            }
         }
         theta = prefix;
         uint32_t g = 0;
