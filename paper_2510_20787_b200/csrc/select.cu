@@ -152,9 +152,12 @@ __global__ void __launch_bounds__(1024) select_reg_kernel(const float* __restric
 {
     __shared__ uint32_t s_part[2][32];
     __shared__ uint32_t s_wa[32], s_we[32];
-    __shared__ uint32_t s_list[kSelList + 2];
+    __shared__ uint32_t s_list[kSelList + 3];
+    const int tid = threadIdx.x;
+    SELP(0);
     pdl_launch_dependents();
     pdl_wait();                                            // z comes from the previous kernel
+    SELP(1);
     const int bh = blockIdx.x;
     select_group<KPT>(z + (size_t)bh * T, idx + (size_t)bh * R, cnt + bh, ncand ? ncand + bh : nullptr, T, W, R, sink, zthr,
                       (int)threadIdx.x, (int)blockDim.x, s_part, s_wa, s_we, [] { __syncthreads(); }, s_list);
@@ -197,3 +200,10 @@ int launch_select(const Params& p, const float* z, int32_t* idx, int32_t* cnt, i
 }
 
 }  // namespace lte
+
+#ifdef LTE_PROFILE
+extern "C" int lte_selprof_read(long long* out)
+{
+    return cudaMemcpyFromSymbol(out, lte::g_selprof, sizeof(long long) * 16) == cudaSuccess ? 0 : -1;
+}
+#endif

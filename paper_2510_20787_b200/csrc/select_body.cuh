@@ -12,6 +12,13 @@
 
 namespace lte {
 
+#ifdef LTE_PROFILE
+__device__ long long g_selprof[16];
+#define SELP(i) do { if (blockIdx.x == 0 && tid == 0) g_selprof[i] = clock64(); } while (0)
+#else
+#define SELP(i) do {} while (0)
+#endif
+
 // key of position j: 0xFFFFFFFF for sink positions, the monotone image of z_j for candidates (z_j > zthr), 0 otherwise.
 // The logit is read past L1: in the fused path other SMs wrote it during the same launch.
 __device__ __forceinline__ uint32_t select_key_of(const float* zz, int j, int sink, float zthr) {
@@ -47,12 +54,15 @@ __device__ __forceinline__ void select_group(const float* __restrict__ zz, int32
         slot ^= 1;
         return total;
     };
+    SELP(2);
+    if (tid == 0 && s_list != nullptr) s_list[kSelList] = 0u;   // the first group barrier below publishes it
     uint32_t c0 = 0;
 #pragma unroll
     for (int i = 0; i < KPT; ++i) c0 += key[i] != 0u;
     const uint32_t nc = block_sum(c0);
     if (tid == 0 && ncand_out) *ncand_out = (int32_t)nc;
 
+    SELP(3);
     uint32_t theta = 0, need_eq = 0;
     if (R > 0 && nc > (uint32_t)R) {
         uint32_t prefix = 0;
@@ -66,35 +76,53 @@ __device__ __forceinline__ void select_group(const float* __restrict__ zz, int32
         }
         // The upper half of the R-th largest key is known.  Only the keys that share it can still move a count, and with
         // spread-out logits they are few: they go into a short list, and one warp settles the lower 16 bits on it without
-        // any group barrier.  (s_list: kSelList entries, then the list length, then the result.)
+        // any group barrier.  (s_list: kSelList entries, then the list length, the threshold and the number of keys equal to it to keep.)
+        SELP(4);
         bool done = false;
-        if (s_list != nullptr) {
+        bool have_need = false;
+        if (s_list != nullptr && N < 65536) {
             const uint32_t hi = prefix >> 16;
-            uint32_t ca = 0, cm = 0;
+            uint32_t cam = 0;                                  // keys above the upper half (low 16 bits of the sum), keys sharing it (high)
 #pragma unroll
-            for (int i = 0; i < KPT; ++i) { ca += (key[i] >> 16) > hi; cm += (key[i] >> 16) == hi; }
-            const uint32_t above = block_sum(ca), match = block_sum(cm);
+            for (int i = 0; i < KPT; ++i) cam += ((key[i] >> 16) > hi ? 1u : 0u) + ((key[i] >> 16) == hi ? 65536u : 0u);
+            const uint32_t both = block_sum(cam);
+            const uint32_t above = both & 0xffffu, match = both >> 16;
+            SELP(7);
             if (match <= (uint32_t)kSelList) {
-                if (tid == 0) s_list[kSelList] = 0u;
-                sync();
+                // (the list length was zeroed before the first group barrier of this function)
 #pragma unroll
                 for (int i = 0; i < KPT; ++i)
                     if ((key[i] >> 16) == hi) s_list[atomicAdd(&s_list[kSelList], 1u)] = key[i];
                 sync();
+                SELP(8);
                 if (wid == 0) {
-                    uint32_t pf = prefix;
-                    for (int b2 = 15; b2 >= 0; --b2) {
-                        const uint32_t cand = pf | (1u << b2);
-                        uint32_t c = 0;
-                        for (uint32_t l = lane; l < match; l += 32) c += s_list[l] >= cand;
-                        c = __reduce_add_sync(0xffffffffu, c);
-                        if (above + c >= (uint32_t)R) pf = cand;
+                    uint32_t pf = prefix, g;
+                    if (match <= 32u) {
+                        // the usual case: one key per lane, a vote per bit
+                        const uint32_t mine = (uint32_t)lane < match ? s_list[lane] : 0u;   // 0 never counts: candidates are > 0
+                        for (int b2 = 15; b2 >= 0; --b2) {
+                            const uint32_t cand = pf | (1u << b2);
+                            if (above + (uint32_t)__popc(__ballot_sync(0xffffffffu, mine >= cand)) >= (uint32_t)R) pf = cand;
+                        }
+                        g = above + (uint32_t)__popc(__ballot_sync(0xffffffffu, mine > pf));
+                    } else {
+                        for (int b2 = 15; b2 >= 0; --b2) {
+                            const uint32_t cand = pf | (1u << b2);
+                            uint32_t c = 0;
+                            for (uint32_t l = lane; l < match; l += 32) c += s_list[l] >= cand;
+                            if (above + __reduce_add_sync(0xffffffffu, c) >= (uint32_t)R) pf = cand;
+                        }
+                        uint32_t c = 0;                        // keys strictly above the threshold: all of them are in `above` or the list
+                        for (uint32_t l = lane; l < match; l += 32) c += s_list[l] > pf;
+                        g = above + __reduce_add_sync(0xffffffffu, c);
                     }
-                    if (lane == 0) s_list[kSelList + 1] = pf;
+                    if (lane == 0) { s_list[kSelList + 1] = pf; s_list[kSelList + 2] = (uint32_t)R - g; }
                 }
                 sync();
+                SELP(9);
                 prefix = s_list[kSelList + 1];
-                done = true;
+                need_eq = s_list[kSelList + 2];
+                done = true; have_need = true;
             }
         }
         if (!done) {
@@ -107,11 +135,14 @@ __device__ __forceinline__ void select_group(const float* __restrict__ zz, int32
             }
         }
         theta = prefix;
-        uint32_t g = 0;
+        if (!have_need) {
+            uint32_t g = 0;
 #pragma unroll
-        for (int i = 0; i < KPT; ++i) g += key[i] > theta;
-        need_eq = (uint32_t)R - block_sum(g);
+            for (int i = 0; i < KPT; ++i) g += key[i] > theta;
+            need_eq = (uint32_t)R - block_sum(g);
+        }
     }
+    SELP(5);
     // ---- ordered compaction: exclusive scan of (above, equal) counts over the threads' segments
     uint32_t a = 0, e = 0;
     if (R > 0) {
@@ -153,6 +184,7 @@ __device__ __forceinline__ void select_group(const float* __restrict__ zz, int32
     const uint32_t kept = R > 0 ? (nc < (uint32_t)R ? nc : (uint32_t)R) : 0u;
     for (int i = (int)kept + tid; i < R; i += nthr) out[i] = -1;
     if (tid == 0) *cnt_out = (int32_t)kept;
+    SELP(6);
 }
 
 }  // namespace lte
