@@ -594,7 +594,19 @@ def _extra_c3(out, torch, lte, synth, pk, flush, n5):
     out["C3_long_prefill"] = {"attn_ms": t * 1e3, "tokens_per_s": cfg.B * cfg.T / t, "algorithmic_tflops": fl / t / 1e12,
                               "tensor_frac": fl / t / 1e12 / pk["bf16_tflops"], "scores_ms": mid3(ms_sc),
                               "select_ms": mid3(ms_se)}
-    del x, o, lse, z
+    # backward at the same shape: the only configuration whose backward is tensor-core bound (2.5 x the forward's FLOPs)
+    g = torch.Generator(device="cuda"); g.manual_seed(3)
+    dO = torch.randn(x["q"].shape, device="cuda", generator=g).to(x["q"].dtype)
+    ws = torch.empty(lte.lte_workspace_bytes(lte.OP_BWD, s, c), dtype=torch.uint8, device="cuda")
+
+    def f_bwd():
+        lte.lte_attn_bwd(s, c, x["q"], x["k"], x["v"], o, lse, dO, z, idx, cnt, ws=ws)
+
+    ms_b, _ = timed(torch, f_bwd, n5, 3, flush)
+    tb = mid3(ms_b) * 1e-3
+    out["C3_long_prefill"].update({"bwd_ms": tb * 1e3, "bwd_algorithmic_tflops": 2.5 * fl / tb / 1e12,
+                                   "bwd_tensor_frac": 2.5 * fl / tb / 1e12 / pk["bf16_tflops"]})
+    del x, o, lse, z, dO, ws
 
 
 def _extra_c5(out, torch, lte, synth, pk, flush, n5):

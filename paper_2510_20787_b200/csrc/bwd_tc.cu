@@ -36,13 +36,18 @@ constexpr float kLog2e = 1.4426950408889634f;
 
 template <int D> struct SmemQ {                                // dq kernel
     static constexpr int SUB = D / 64;
+    // d = 128 runs one CTA per SM (shared memory), so tensor memory has room for two S / dP buffers: the products of tile
+    // t+1 are in flight while the row threads work on tile t, which needs a fourth key / value stage
+    static constexpr bool DB = D == 128;
+    static constexpr int NS = DB ? 4 : 3;
     static constexpr int QTILE = BM * D * 2, KVTILE = BN * D * 2;
-    static constexpr int OFF_Q = 0, OFF_DO = QTILE, OFF_K = 2 * QTILE, OFF_V = OFF_K + NST * KVTILE;
-    static constexpr int OFF_DS = OFF_V + NST * KVTILE;        // [128][64] bf16
+    static constexpr int OFF_Q = 0, OFF_DO = QTILE, OFF_K = 2 * QTILE, OFF_V = OFF_K + NS * KVTILE;
+    static constexpr int OFF_DS = OFF_V + NS * KVTILE;         // [128][64] bf16
     static constexpr int OFF_BAR = OFF_DS + BM * BN * 2;
     static constexpr int OFF_IDX = OFF_BAR + 128;
     static constexpr int BYTES = OFF_IDX + 512;
-    static constexpr uint32_t TMEM_COLS = 256;                 // S: [0,64)  dP: [64,128)  dQ: [128, 128+D)
+    // d = 64:  S [0,64)  dP [64,128)  dQ [128,192);   d = 128:  S, dP of buffer b at 128 b, 128 b + 64;  dQ [256,384)
+    static constexpr uint32_t TMEM_COLS = DB ? 512 : 256;
 };
 
 template <int D>
@@ -59,15 +64,17 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     pdl_wait();                                                // see launch_pdl: earlier kernels of the stream have completed
     using S = SmemQ<D>;
     constexpr int SUB = S::SUB;
-    constexpr uint32_t DP_COL = BN, DQ_COL = 2 * BN;
+    constexpr bool DB = S::DB;
+    constexpr int NS = S::NS;
+    constexpr uint32_t DP_COL = BN, DQ_COL = DB ? 4 * BN : 2 * BN;
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     const uint32_t base = smem_u32(smem_raw);
     if ((base & 1023u) != 0) { if (threadIdx.x == 0) atomicExch(&g_bwd_status, 9); return; }
     const uint32_t sQ = base + S::OFF_Q, sDO = base + S::OFF_DO, sK = base + S::OFF_K, sV = base + S::OFF_V;
     const uint32_t sDS = base + S::OFF_DS;
-    const uint32_t bar_q = base + S::OFF_BAR, bar_k0 = bar_q + 8, bar_v0 = bar_q + 32, bar_s = bar_q + 56;
-    const uint32_t bar_g0 = bar_q + 64, bar_p = bar_q + 80, bar_pv = bar_q + 88, tmem_slot = bar_q + 96;
-    volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(smem_raw + S::OFF_BAR + 96);
+    const uint32_t bar_q = base + S::OFF_BAR, bar_k0 = bar_q + 8, bar_v0 = bar_q + 40, bar_s0 = bar_q + 72;   // 4, 4, 2 slots
+    const uint32_t bar_g0 = bar_q + 88, bar_p = bar_q + 104, bar_pv = bar_q + 112, tmem_slot = bar_q + 120;
+    volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(smem_raw + S::OFF_BAR + 120);
     volatile int* s_idx = reinterpret_cast<volatile int*>(smem_raw + S::OFF_IDX);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -82,8 +89,8 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     if (tid == 0) {
         mbar_init(bar_q, 1);
 #pragma unroll
-        for (int s2 = 0; s2 < NST; ++s2) { mbar_init(bar_k0 + 8 * s2, 1); mbar_init(bar_v0 + 8 * s2, 1); }
-        mbar_init(bar_s, 1);
+        for (int s2 = 0; s2 < NS; ++s2) { mbar_init(bar_k0 + 8 * s2, 1); mbar_init(bar_v0 + 8 * s2, 1); }
+        mbar_init(bar_s0, 1); mbar_init(bar_s0 + 8, 1);
         mbar_init(bar_g0, 128); mbar_init(bar_g0 + 8, 128);
         mbar_init(bar_p, 128); mbar_init(bar_pv, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -117,7 +124,7 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             const uint32_t ds_lo = desc_lo(sDS, 16), kmn_lo = desc_lo(sK, 8192);
             uint32_t k_phase = 0, v_phase = 0, g_waited = 0;
             auto tma_kv = [&](int t, bool is_v) {
-                const int st = t % NST;
+                const int st = t % NS;
                 const uint32_t dst = (is_v ? sV : sK) + st * S::KVTILE;
                 const uint32_t bar = (is_v ? bar_v0 : bar_k0) + 8 * st;
                 const int y = j_start + t * BN;
@@ -132,23 +139,24 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             };
             auto wait_kv = [&](int t) {
                 if (t < n_win) {
-                    const int st = t % NST;
+                    const int st = t % NS;
                     bwait(bar_k0 + 8 * st, (k_phase >> st) & 1u, 2); k_phase ^= 1u << st;
                     bwait(bar_v0 + 8 * st, (v_phase >> st) & 1u, 4); v_phase ^= 1u << st;
                 }
             };
             auto mma_s_dp = [&](int t) {
-                const uint32_t so = (uint32_t)(t % NST) * (S::KVTILE >> 4);
+                const uint32_t so = (uint32_t)(t % NS) * (S::KVTILE >> 4);
+                const uint32_t sbuf = DB ? (uint32_t)(t & 1) * (2 * BN) : 0u;
                 if (leader) {
 #pragma unroll
                     for (int kk = 0; kk < D / 16; ++kk)
-                        umma(tmem, desc64(q_lo + (kk >> 2) * 1024 + (kk & 3) * 2, kDescHi),
+                        umma(tmem + sbuf, desc64(q_lo + (kk >> 2) * 1024 + (kk & 3) * 2, kDescHi),
                              desc64(k_lo + so + (kk >> 2) * 512 + (kk & 3) * 2, kDescHi), IDESC_S, kk > 0);
 #pragma unroll
                     for (int kk = 0; kk < D / 16; ++kk)
-                        umma(tmem + DP_COL, desc64(do_lo + (kk >> 2) * 1024 + (kk & 3) * 2, kDescHi),
+                        umma(tmem + sbuf + DP_COL, desc64(do_lo + (kk >> 2) * 1024 + (kk & 3) * 2, kDescHi),
                              desc64(v_lo + so + (kk >> 2) * 512 + (kk & 3) * 2, kDescHi), IDESC_S, kk > 0);
-                    umma_commit(bar_s);
+                    umma_commit(bar_s0 + (DB ? 8 * (t & 1) : 0));
                 }
                 __syncwarp();
             };
@@ -163,23 +171,29 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                 }
                 if (D == 64) tma_load_3d(sDS, &tmO, 0, i0, bh, bar_q);
             }
-            for (int t = 0; t < NST && t < n_win; ++t) { tma_kv(t, false); tma_kv(t, true); }
+            for (int t = 0; t < NS && t < n_win; ++t) { tma_kv(t, false); tma_kv(t, true); }
             bwait(bar_q, 0, 1);                                // (tile 0 is always a window tile: no gather to wait for)
             wait_kv(0);
             tc_fence_after();
             mma_s_dp(0);
-            for (int t = 0; t < n_tiles; ++t) {
-                bwait(bar_p, t & 1, 7);                        // dS(t) is in shared memory; S / dP buffers are free
+            if (DB && n_tiles > 1) {                           // two buffers: tile 1 follows at once (prologue gathers: phase 0)
+                need_g(0);
+                wait_kv(1);
                 tc_fence_after();
-                // the next tile's S, dP first: the row threads wait for those, while dQ of this tile is only needed before
-                // the dS buffer is rewritten a tile later
-                if (t + 1 < n_tiles) {
+                mma_s_dp(1);
+            }
+            for (int t = 0; t < n_tiles; ++t) {
+                bwait(bar_p, t & 1, 7);                        // dS(t) is in shared memory; its S / dP buffer is free
+                tc_fence_after();
+                // one buffer: the next tile's S, dP first: the row threads wait for those, while dQ of this tile is only
+                // needed before the dS buffer is rewritten a tile later
+                if (!DB && t + 1 < n_tiles) {
                     need_g(t + 1);
                     wait_kv(t + 1);
                     mma_s_dp(t + 1);
                 }
                 {
-                    const uint32_t kb = kmn_lo + (uint32_t)(t % NST) * (S::KVTILE >> 4);
+                    const uint32_t kb = kmn_lo + (uint32_t)(t % NS) * (S::KVTILE >> 4);
                     if (leader) {
 #pragma unroll
                         for (int kk = 0; kk < BN / 16; ++kk)
@@ -189,9 +203,17 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     }
                     __syncwarp();
                 }
+                // two buffers: the row threads are already on tile t+1; S, dP of tile t+2 go into the buffer tile t has left.
+                // Its gathers were committed in tile t-1 and are covered by the arrival at the top of tile t+1.
+                if (DB && t + 2 < n_tiles) {
+                    need_g(t + 1);
+                    wait_kv(t + 2);
+                    tc_fence_after();
+                    mma_s_dp(t + 2);
+                }
                 // dQ(t-1) has completed (the softmax warps waited for it before producing dS(t)): its key stage and
-                // the value stage of tile t-1 can take window tile t-1+NST
-                if (t >= 1 && t - 1 + NST < n_win) { tma_kv(t - 1 + NST, false); tma_kv(t - 1 + NST, true); }
+                // the value stage of tile t-1 can take window tile t-1+NS
+                if (t >= 1 && t - 1 + NS < n_win) { tma_kv(t - 1 + NS, false); tma_kv(t - 1 + NS, true); }
             }
         }
     } else {
@@ -266,7 +288,7 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         };
         auto gather_issue = [&](int t, bool is_v, const int (&rows4)[4]) {
             if (t >= n_win && t < n_tiles) {
-                const uint32_t dst = (is_v ? sV : sK) + (t % NST) * S::KVTILE;
+                const uint32_t dst = (is_v ? sV : sK) + (t % NS) * S::KVTILE;
 #pragma unroll
                 for (int ps = 0; ps < 4; ++ps) {
                     const int row = ps * 16 + g_row;
@@ -282,7 +304,7 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         };
         {
             int rows4[4];
-            for (int t = 0; t < NST; ++t) { gather_rows(t, rows4); gather_issue(t, false, rows4); gather_issue(t, true, rows4); }
+            for (int t = 0; t < NS; ++t) { gather_rows(t, rows4); gather_issue(t, false, rows4); gather_issue(t, true, rows4); }
             cp_async_commit();
             cp_async_commit();                                 // empty group: the wait at the top of tile 0 then covers the one above
         }
@@ -291,7 +313,7 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 
         for (int t = 0; t < n_tiles; ++t) {
             int rn[4];
-            gather_rows(t - 1 + NST, rn);                      // retained tile that goes into the stage of tile t-1
+            gather_rows(t - 1 + NS, rn);                       // retained tile that goes into the stage of tile t-1
             cp_async_wait<1>();                                // every gather but the latest tile's has landed
             fence_proxy_async();
             mbar_arrive(bar_g0 + 8 * (t & 1));
@@ -307,16 +329,17 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             }
             const int u_lo = __shfl_sync(0xffffffffu, c_lo, 0), u_hi = __shfl_sync(0xffffffffu, c_hi, 31);
 
-            bwait(bar_s, t & 1, 3);                            // S(t), dP(t) are in TMEM
+            bwait(bar_s0 + (DB ? 8 * (t & 1) : 0), DB ? (t >> 1) & 1 : t & 1, 3);   // S(t), dP(t) are in TMEM
             tc_fence_after();
+            const uint32_t sbuf = DB ? (uint32_t)(t & 1) * (2 * BN) : 0u;
             uint32_t pk[32];                                   // dS row as 64 bf16
 #pragma unroll
             for (int cb = 0; cb < 2; ++cb) {
                 const bool act = cb * 32 <= u_hi && cb * 32 + 31 >= u_lo;
                 if (act) {
                     uint32_t rs[32], rp[32];
-                    tmem_ld32(tmem + lane_base + cb * 32, rs);
-                    tmem_ld32(tmem + lane_base + DP_COL + cb * 32, rp);
+                    tmem_ld32(tmem + lane_base + sbuf + cb * 32, rs);
+                    tmem_ld32(tmem + lane_base + sbuf + DP_COL + cb * 32, rp);
                     tmem_wait_ld();
 #pragma unroll
                     for (int c = 0; c < 32; c += 2) {
@@ -336,7 +359,7 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             }
             // dQ(t-1) must be done before dS is overwritten; its key stage (and the value stage) are then free
             if (t > 0) { bwait(bar_pv, (t - 1) & 1, 4); tc_fence_after(); }
-            if (t > 0) { gather_issue(t - 1 + NST, false, rn); gather_issue(t - 1 + NST, true, rn); }
+            if (t > 0) { gather_issue(t - 1 + NS, false, rn); gather_issue(t - 1 + NS, true, rn); }
             cp_async_commit();
 #pragma unroll
             for (int ch = 0; ch < 8; ++ch) {
@@ -590,13 +613,14 @@ bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         }
         const float c2 = scale * kLog2e;
         const uint32_t lane_base = ((uint32_t)(warp * 32)) << 16;
-        // per-column constants of the next block, fetched one block ahead: thread c < 64 holds L2, thread 64 + c delta
+        // per-column constants of the next block, fetched one block ahead: thread c < 64 holds -L2, thread 64 + c
+        // -delta scale (the forms the fused multiply-adds below take)
         auto col_fetch = [&](int t) -> float {
             if (t >= n_blk) return 0.f;
             const int i = ib_start + (t % n_pos) * 64 + (tid & 63);
-            if (i >= Tlen) return tid < 64 ? INFINITY : 0.f;                    // L2 = +inf makes P = 0
+            if (i >= Tlen) return tid < 64 ? -INFINITY : 0.f;                   // -L2 = -inf makes P = 0
             const size_t bhq = (size_t)bh * G + t / n_pos;
-            return tid < 64 ? lse[bhq * Tlen + i] * kLog2e : delta[bhq * Tlen + i];
+            return tid < 64 ? -lse[bhq * Tlen + i] * kLog2e : -delta[bhq * Tlen + i] * scale;
         };
         float col_next = col_fetch(0);
 
@@ -633,8 +657,8 @@ bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
 #pragma unroll
                         for (int u = 0; u < 4; ++u) {
                             const bool ok = col + u >= c_lo && col + u <= c_hi;
-                            p[u] = ok ? fast_exp2(fmaf(__uint_as_float(rs[c + u]), c2, -lv[u])) : 0.f;
-                            ds[u] = p[u] * (__uint_as_float(rp[c + u]) - dvv[u]) * scale;
+                            p[u] = ok ? fast_exp2(fmaf(__uint_as_float(rs[c + u]), c2, lv[u])) : 0.f;
+                            ds[u] = p[u] * fmaf(__uint_as_float(rp[c + u]), scale, dvv[u]);
                         }
                         __nv_bfloat162 h0 = __floats2bfloat162_rn(p[0], p[1]), h1 = __floats2bfloat162_rn(p[2], p[3]);
                         __nv_bfloat162 g0 = __floats2bfloat162_rn(ds[0], ds[1]), g1 = __floats2bfloat162_rn(ds[2], ds[3]);

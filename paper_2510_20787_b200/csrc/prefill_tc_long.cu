@@ -14,6 +14,21 @@ namespace lte {
 __device__ int g_prefill_long_status = 0;     // 0 = fine; otherwise the code of the wait that gave up
 
 
+#ifdef LTE_PROFILE
+// cycles per phase, summed over all CTAs: [0,16) softmax thread 0, [16,32) the MMA warp's lane 0
+__device__ unsigned long long g_plprof[64];
+// (accumulated in shared memory and flushed once per CTA: global atomics in the loop slowed the fences down)
+#define PLM(k) do { if (prof_on) { const long long now_ = clock64(); prof_[(k) + pofs_] += (unsigned long long)(now_ - tprev_); tprev_ = now_; } } while (0)
+#define PLM_INIT(cond) const bool prof_on = (cond); long long tprev_ = clock64(); int pofs_ = 0
+#define PLM_TILE(t) pofs_ = (t) >= n_win ? 32 : 0
+#define PLM_FLUSH(lo, hi) do { if (prof_on) for (int k_ = lo; k_ < hi; ++k_) { atomicAdd(&g_plprof[k_], prof_[k_]); atomicAdd(&g_plprof[k_ + 32], prof_[k_ + 32]); } } while (0)
+#else
+#define PLM(k) do { } while (0)
+#define PLM_INIT(cond) do { } while (0)
+#define PLM_TILE(t) do { } while (0)
+#define PLM_FLUSH(lo, hi) do { } while (0)
+#endif
+
 namespace {
 
 constexpr int BM = 128, BN = 64, NTHREADS = 192;
@@ -36,7 +51,11 @@ template <int D> struct Smem {
     static constexpr bool ONES = D == 64;
     static constexpr int OFF_ONES = OFF_P;                    // [64][64] bf16 ones (8 KB), d = 64 only
     static constexpr int OFF_BAR = OFF_ONES + (ONES ? BN * 128 : 0);   // mbarriers, tmem slot
+#ifdef LTE_PROFILE
+    static constexpr int BYTES = OFF_BAR + 768;
+#else
     static constexpr int BYTES = OFF_BAR + 256;
+#endif
     static constexpr uint32_t TMEM_COLS = 256;                // S0: [0,64)  S1: [64,128)  O: [128, 128+D) (+16 row-sum columns)
 };
 
@@ -83,6 +102,10 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(smem_raw + S::OFF_BAR + 152);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+#ifdef LTE_PROFILE
+    volatile unsigned long long* prof_ = reinterpret_cast<volatile unsigned long long*>(smem_raw + S::OFF_BAR + 256);
+    if (tid < 64) prof_[tid] = 0ull;
+#endif
     const int bh = blockIdx.y, bhk = bh / G;                   // query head and its key/value head (the G query heads of one are adjacent)
     const int i0 = blockIdx.x * BM;
     const int i_hi = min(i0 + BM - 1, Tlen - 1);
@@ -99,6 +122,8 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             mbar_init(bar_kf0 + 8 * s2, 1); mbar_init(bar_vf0 + 8 * s2, 1);
         }
         mbar_init(bar_s0, 1); mbar_init(bar_s0 + 8, 1);
+        // every softmax thread arrives itself: one arrival per warp behind a __syncwarp() lengthened the hand-over of P
+        // to the MMA warp and cost 3 % at d = 128, T = 32768
         mbar_init(bar_g0, 128); mbar_init(bar_g0 + 8, 128);
         mbar_init(bar_p, 128); mbar_init(bar_pv, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -211,7 +236,9 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 ks = ks + 1 == KST ? 0 : ks + 1;
             };
 
+            PLM_INIT(lane == 0);
             mbar_wait(bar_q, 0, 1);
+            PLM(16);
             mma_s();                                           // tile 0 is always a window tile
             if (n_tiles > 1) {
                 if (n_win < 2) need_g(0);                      // tile 1 is a retained tile: the prologue gathers
@@ -219,12 +246,16 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             }
             for (int t = 0; t < n_tiles; ++t) {
                 // PV(t): everything but P is normally there long before
+                PLM(17);
+                PLM_TILE(t);
                 need_g(t);
                 if (t < n_win) { mbar_wait(bar_v0 + 8 * vs, (v_par >> vs) & 1u, 4); v_par ^= 1u << vs; }
+                PLM(18);
                 uint32_t vb = v_desc[0];
 #pragma unroll
                 for (int st = 1; st < VST; ++st) vb = vs == st ? v_desc[st] : vb;
                 mbar_wait(bar_p, t & 1, 7);
+                PLM(19);
                 tc_fence_after();
                 if (lane == 0) {
 #pragma unroll
@@ -235,9 +266,12 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 }
                 __syncwarp();
                 vs = vs + 1 == VST ? 0 : vs + 1;
+                PLM(20);
                 // S(t+2) into the S buffer softmax(t) has just released
                 if (ts < n_tiles) mma_s();
+                PLM(21);
             }
+            PLM_FLUSH(16, 22);
         }
     } else {
         // =================================== softmax warps ==================================================
@@ -272,6 +306,8 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             nvis += __popc(bits & ((1u << (lim - lim0)) - 1u));
         }
         const int n_tiles = n_win + (nv_max + BN - 1) / BN;
+        const int iw0 = i0 + warp * 32;                        // the warp's first row
+        const int nvis0 = __shfl_sync(0xffffffffu, nvis, 0), nvis31 = __shfl_sync(0xffffffffu, nvis, 31);
 
         // gather of one retained tile: 8 lanes per row copy its 16-byte chunks (coalesced reads, conflict-free
         // swizzled writes), 16 rows per pass; rows past the visible prefix are zero-filled
@@ -312,7 +348,10 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         const uint32_t lane_base = ((uint32_t)(warp * 32)) << 16;   // this warp's TMEM lanes
         float m_run = -INFINITY, l_run = 0.f;                  // running max (log2 domain) and sum (sum only if !ONES)
 
+        PLM_INIT(tid == 0);
+        PLM(0);
         for (int t = 0; t < n_tiles; ++t) {
+            PLM_TILE(t);
             // row positions for this tile's two gathers, fetched first so their latency hides under the softmax
             int rk[4], rv[4];
             gather_rows(t + KST, rk);
@@ -325,40 +364,51 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             }
 
             // column range this row may see in the tile
-            int c_lo, c_hi;
+            // rows of a warp are consecutive and both bounds grow with the row: its first / last row give the warp's
+            // union range (columns any row sees) and intersection range (columns every row sees)
+            int c_lo, c_hi, u_lo, u_hi, n_lo, n_hi;
             if (t < n_win) {
                 const int jt0 = j_start + t * BN;
                 c_lo = max(i - W + 1, 0) - jt0;
                 c_hi = i - jt0;
+                u_lo = max(iw0 - W + 1, 0) - jt0; n_lo = max(iw0 + 31 - W + 1, 0) - jt0;
+                n_hi = iw0 - jt0; u_hi = iw0 + 31 - jt0;
             } else {
-                c_lo = 0;
-                c_hi = nvis - (t - n_win) * BN - 1;
+                const int off = (t - n_win) * BN + 1;
+                c_lo = 0; u_lo = 0; n_lo = 0;
+                c_hi = nvis - off; n_hi = nvis0 - off; u_hi = nvis31 - off;
             }
-            // rows of a warp are consecutive and both bounds grow with the row: lane 0 / lane 31 give the warp's
-            // union range (columns any row sees) and intersection range (columns every row sees)
-            const int u_lo = __shfl_sync(0xffffffffu, c_lo, 0), u_hi = __shfl_sync(0xffffffffu, c_hi, 31);
-            const int n_lo = __shfl_sync(0xffffffffu, c_lo, 31), n_hi = __shfl_sync(0xffffffffu, c_hi, 0);
+            PLM(1);
             bool act[2], full[2];
             uint32_t vm[2];                                    // per-thread validity bits of a partial chunk
+            if (n_lo <= 0 && n_hi >= BN - 1) {                 // most tiles: every row of the warp sees every column
+                act[0] = act[1] = full[0] = full[1] = true;
+                vm[0] = vm[1] = 0xffffffffu;
+            } else {
 #pragma unroll
-            for (int cb = 0; cb < 2; ++cb) {
-                const int lo = cb * 32, hi = lo + 31;
-                act[cb] = lo <= u_hi && hi >= u_lo;
-                full[cb] = lo >= n_lo && hi <= n_hi;
-                const int a = min(max(c_lo - lo, 0), 32), b2 = min(max(c_hi - lo + 1, 0), 32);
-                const uint32_t below_b = b2 >= 32 ? 0xffffffffu : ((1u << b2) - 1u);
-                const uint32_t below_a = a >= 32 ? 0xffffffffu : ((1u << a) - 1u);
-                vm[cb] = b2 > a ? (below_b & ~below_a) : 0u;
+                for (int cb = 0; cb < 2; ++cb) {
+                    const int lo = cb * 32, hi = lo + 31;
+                    act[cb] = lo <= u_hi && hi >= u_lo;
+                    full[cb] = lo >= n_lo && hi <= n_hi;
+                    const int a = min(max(c_lo - lo, 0), 32), b2 = min(max(c_hi - lo + 1, 0), 32);
+                    const uint32_t below_b = b2 >= 32 ? 0xffffffffu : ((1u << b2) - 1u);
+                    const uint32_t below_a = a >= 32 ? 0xffffffffu : ((1u << a) - 1u);
+                    vm[cb] = b2 > a ? (below_b & ~below_a) : 0u;
+                }
             }
+            PLM(2);
             mbar_wait(bar_s0 + 8 * (t & 1), (t >> 1) & 1, 3);  // S(t) is in TMEM buffer t & 1
             tc_fence_after();
+            PLM(3);
             gather_issue(t + KST, false, rk);                  // its stage held K(t), which S(t) has finished reading
+            PLM(4);
             const uint32_t s_col = (t & 1) * BN;
             uint32_t r[2][32];
 #pragma unroll
             for (int cb = 0; cb < 2; ++cb)
                 if (act[cb]) tmem_ld32(tmem + lane_base + s_col + cb * 32, r[cb]);
             tmem_wait_ld();
+            PLM(5);
             float mr[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // row max of the raw logits, 4 chains
 #pragma unroll
             for (int cb = 0; cb < 2; ++cb) {
@@ -378,6 +428,7 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             }
             const float m_tile = fmaxf(fmaxf(mr[0], mr[1]), fmaxf(mr[2], mr[3])) * c2;
             // lazy rescale: the running max only moves when the new one is far above it (exp2 arguments stay <= 8)
+            PLM(6);
             float alpha = 1.f;
             bool need = false;
             if (m_run == -INFINITY) m_run = m_tile;             // nothing accumulated yet for this row: O row is 0
@@ -397,18 +448,22 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 tmem_wait_st();
                 l_run *= alpha;
             }
+            PLM(7);
             const float neg_m = m_run == -INFINITY ? 0.f : -m_run;
-            float ls[4] = {0.f, 0.f, 0.f, 0.f};
+            uint64_t ls2[2] = {0ull, 0ull};                    // two chains of packed pairs
+            const uint64_t c2p = pack2(c2, c2), nmp = pack2(neg_m, neg_m);
             uint32_t pk[32];                                   // the row of P as 64 bf16, two per word
 #pragma unroll
             for (int cb = 0; cb < 2; ++cb) {
                 if (act[cb]) {
 #pragma unroll
                     for (int c = 0; c < 32; c += 2) {
-                        // masked entries hold -inf: fma gives -inf and exp2(-inf) = 0
-                        const float p0 = fast_exp2(fmaf(__uint_as_float(r[cb][c]), c2, neg_m));
-                        const float p1 = fast_exp2(fmaf(__uint_as_float(r[cb][c + 1]), c2, neg_m));
-                        if (!S::ONES) ls[(c >> 1) & 3] += p0 + p1;   // with ONES the tensor core sums the rounded probabilities
+                        // masked entries hold -inf: fma gives -inf and exp2(-inf) = 0.  Scale and shift of two columns
+                        // are one packed fma, their contribution to the row sum one packed add
+                        float a0, a1;
+                        unpack2(fma2(pack2(__uint_as_float(r[cb][c]), __uint_as_float(r[cb][c + 1])), c2p, nmp), a0, a1);
+                        const float p0 = fast_exp2(a0), p1 = fast_exp2(a1);
+                        if (!S::ONES) ls2[(c >> 1) & 1] = add2(ls2[(c >> 1) & 1], pack2(p0, p1));   // with ONES the tensor core sums the rounded probabilities
                         __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
                         pk[cb * 16 + (c >> 1)] = *reinterpret_cast<uint32_t*>(&h);
                     }
@@ -417,20 +472,30 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     for (int c = 0; c < 16; ++c) pk[cb * 16 + c] = 0u;
                 }
             }
-            l_run += (ls[0] + ls[1]) + (ls[2] + ls[3]);
+            {
+                float s0, s1, s2, s3;
+                unpack2(ls2[0], s0, s1); unpack2(ls2[1], s2, s3);
+                l_run += (s0 + s1) + (s2 + s3);
+            }
             // P goes back into TMEM, over the first 32 columns of the S buffer it was computed from (this thread has
             // all of its row in registers), and feeds the PV product as the A operand: no trip through shared memory
+            PLM(8);
             tmem_st32(tmem + lane_base + s_col, pk);
             tmem_wait_st();
             tc_fence_before();                                 // our TMEM accesses are ordered before the arrive
+            PLM(9);
             // PV(t-1) has normally completed long ago; the wait sits before the arrive so that the barrier cannot
             // run two phases ahead of this thread
             if (t > 0) mbar_wait(bar_pv, (t - 1) & 1, 4);
             mbar_arrive(bar_p);
+            PLM(10);
             // value tile t+VST-1 goes into the stage of V(t-1), which PV(t-1) has finished reading
             if (t > 0) gather_issue(t + VST - 1, true, rv); else cp_async_commit();
+            PLM(11);
         }
         mbar_wait(bar_pv, (n_tiles - 1) & 1, 5);
+        PLM_TILE(0);
+        PLM(12);
         tc_fence_after();
 
         // ---- epilogue: O / l -> bf16, logsumexp ----------------------------------------------------------
@@ -472,6 +537,8 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             bulk_wait_read0();                                 // the buffer is released with the CTA
         }
         if (i < Tlen) lse[(size_t)bh * Tlen + i] = m_run * 0.6931471805599453f + logf(l_run);
+        PLM(13);
+        PLM_FLUSH(0, 14);
     }
     tc_fence_before();
     __syncthreads();
@@ -508,6 +575,14 @@ int launch_prefill_tc_long(const Params& p, const void* q, const void* k, const 
     if (p.d != 128) return LTE_ERR_UNSUPPORTED;
     return run<128>(p, q, k, v, idx, cnt, o, lse, st);
 }
+
+#ifdef LTE_PROFILE
+extern "C" void lte_plprof_read(unsigned long long* out, int clear)
+{
+    cudaMemcpyFromSymbol(out, g_plprof, sizeof(unsigned long long) * 64);
+    if (clear) { unsigned long long z[64] = {}; cudaMemcpyToSymbol(g_plprof, z, sizeof(z)); }
+}
+#endif
 
 int prefill_long_status_fetch_and_clear()
 {
