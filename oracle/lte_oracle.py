@@ -152,6 +152,42 @@ def attn_prefill(q, k, v, idx, cnt, W, scale=None, qpos=None):
     return o, lse
 
 
+def chunk_select(z, n0, n1, W, R, pool_idx, pool_cnt, sink=0, tau=0.5):
+    """Retained list after a chunk of tokens [n0, n1) arrives on top of a cache that holds n0 tokens
+    (Section 3.1.3, cached prefilling): the pool entries pool_idx[:pool_cnt] compete with the tokens that leave
+    the window during the chunk, positions max(n0 - W, 0) .. n1 - 1 - W, of which only sink tokens and tokens
+    with z > logit(tau) are candidates; the best R stay (sink first, then z descending, then position ascending).
+    z [B,H,>=n1-W] are the logits of the whole sequence.  -> idx [B,H,R] ascending (-1 unused), cnt [B,H]."""
+    z = _f64(z)
+    B, H = z.shape[:2]
+    thr = logit(tau)
+    idx = np.full((B, H, max(R, 0)), -1, np.int32)
+    cnt = np.zeros((B, H), np.int32)
+    for b in range(B):
+        for h in range(H):
+            cand = [int(j) for j in pool_idx[b, h, :pool_cnt[b, h]]]
+            for j in range(max(n0 - W, 0), n1 - W):
+                if j < sink or z[b, h, j] > thr:
+                    cand.append(j)
+            assert len(set(cand)) == len(cand), "a pool entry is still inside the window"
+            cand.sort(key=lambda j: (0 if j < sink else 1, 0.0 if j < sink else -z[b, h, j], j))
+            keep = sorted(cand[:max(R, 0)])
+            idx[b, h, :len(keep)] = keep
+            cnt[b, h] = len(keep)
+    return idx, cnt
+
+
+def prefill_chunk(q, k, v, z, n0, W, R, pool_idx, pool_cnt, sink=0, tau=0.5, scale=None):
+    """Attention of the chunk's queries [n0, n1) (n1 = sequence length of q, k, v) under the chunk-end reading:
+    query i sees its window and the entries of the list after the chunk that are older than its window.
+    -> o [B,H,n1-n0,d], lse [B,H,n1-n0], idx, cnt (the new pool)."""
+    B, H, n1, d = np.asarray(q).shape
+    idx, cnt = chunk_select(z, n0, n1, W, R, pool_idx, pool_cnt, sink, tau)
+    qpos = np.broadcast_to(np.arange(n0, n1, dtype=np.int32), (B, H, n1 - n0)).copy()
+    o, lse = attn_prefill(q, k, v, idx, cnt, W, scale, qpos=qpos)
+    return o, lse, idx, cnt
+
+
 def stream(q, k, v, z, W, R, sink=0, tau=0.5, scale=None, n_from=0):
     """Token-by-token simulation from an empty cache; outputs for steps >= n_from
     and the final pool (ascending positions)."""
