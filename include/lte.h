@@ -76,7 +76,7 @@ typedef struct lte_conv {
  */
 
 typedef enum lte_op {
-    LTE_OP_SCORES = 0, LTE_OP_SELECT = 1, LTE_OP_PREFILL = 2, LTE_OP_DECODE = 3, LTE_OP_BWD = 4
+    LTE_OP_SCORES = 0, LTE_OP_SELECT = 1, LTE_OP_PREFILL = 2, LTE_OP_DECODE = 3, LTE_OP_BWD = 4, LTE_OP_CHUNK = 5
 } lte_op;
 
 /* Bytes of caller-supplied scratch the given entry point needs for this shape (0 if none). */
@@ -195,6 +195,30 @@ int lte_attn_decode(const lte_shape* s, const lte_conv* c, void* cache,
  * Errors: UNSUPPORTED for the single layer (it is scored inside the step), INVALID_ARG, WORKSPACE.
  */
 int lte_cache_score(const lte_shape* s, const lte_conv* c, void* cache, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Chunked (continued) prefill on top of a cache (Section 3.1.3, "Cached prefilling and decoding"): T = s->T new tokens
+ * arrive at a cache that holds n_past tokens (from lte_cache_init, lte_attn_decode or an earlier chunk).  Chunk-end
+ * reading: the pool's entries compete with the tokens that leave the window while the chunk arrives (positions
+ * max(n_past - W, 0) .. n_past + T - 1 - W; sink tokens and tokens with z > logit(tau) are candidates); the best R (sink
+ * first, then z descending) form the new pool; query i of the chunk sees its window of W keys and the new pool's entries
+ * at positions <= i - W.  On top of a one-shot prefill of the first n_past tokens this is exactly the one-shot prefill
+ * of the n_past + T tokens, restricted to the chunk's queries; where the cap R never binds it is also what T decode steps
+ * compute.  A ring token the cache has not scored yet (the newest K/2 tokens, or whatever lte_cache_score has not
+ * reached for the stack) is scored with the chunk as its right context; the chunk's last K/2 tokens stay unscored.
+ *   cache    in/out  state for n_past tokens -> state for n_past + T tokens (lte_attn_decode may follow)
+ *   n_past   tokens the cache holds, the same for every (b,h); a cache that holds another count is left unchanged and
+ *            lte_device_status() reports it
+ *   q        in   [B,H*group,T,d];   k, v in [B,H,T,d] of s->dtype
+ *   o        out  [B,H*group,T,d];   lse out [B,H*group,T] fp32
+ *   ws       device scratch of lte_workspace_bytes(LTE_OP_CHUNK, s, c) bytes, 256-byte aligned: the pool, the ring in
+ *            time order and the chunk are laid out as one local sequence of at most R + W + T rows, which the scorer, the
+ *            selection and the prefill attention kernels then process (queries padded to that length)
+ * Errors: INVALID_ARG, UNSUPPORTED (as lte_cache_init; local sequence too long), WORKSPACE, CUDA.
+ */
+int lte_attn_prefill_chunk(const lte_shape* s, const lte_conv* c, void* cache, int32_t n_past,
+                           const void* q, const void* k, const void* v, void* o, float* lse,
+                           void* ws, size_t ws_bytes, void* stream);
 
 /*
  * Backward of lte_attn_prefill with the straight-through surrogate (Section 3.1.2):

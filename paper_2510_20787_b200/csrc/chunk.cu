@@ -1,0 +1,183 @@
+// Chunked (continued) prefill on top of a decode cache (Section 3.1.3, "Cached prefilling and decoding"): glue kernels.
+//
+// The cache holds n0 tokens: a ring with the last min(n0, W) of them and a pool of retained ones.  A chunk of Tc tokens
+// arrives.  The chunk-end reading: the pool entries compete with the tokens that leave the window while the chunk
+// arrives, the best R form the new list, and query i of the chunk sees its window plus the list entries older than its
+// window.  This is what the one-shot prefill computes over the "local sequence"
+//     rows [0, R0)            the pool rows, slot order      (R0 = R once anything has left the window, else 0)
+//     rows [R0, R0 + Wn)      the ring in time order         (Wn = min(n0, W))
+//     rows [R0 + Wn, T_loc)   the chunk
+// because every pool row is older than every chunk query's window and the window of a chunk query never reaches below
+// row R0.  So the path is: gather the local sequence (here), score it (the scorer kernels), merge the logits the cache
+// already holds (here), select, attend (the prefill kernels, queries padded to the local length), and write the new
+// cache (here).  Local row r stands for position pos(r) = old pool position (r < R0) or n0 - Wn + (r - R0).
+#include "common.cuh"
+
+namespace lte {
+
+__device__ int g_chunk_status = 0;            // 0 = fine; 31: the cache does not hold n_past tokens
+
+namespace {
+
+// one 16-byte piece of a cache row -> the same piece of a plain row (the swizzled layout permutes the pieces of a row)
+__device__ __forceinline__ int piece_src(const CacheLayout& L, int row, int c) { return L.swz ? (c ^ (row & 7)) : c; }
+
+// Block per (b,h): pool rows and ring rows (time order) into the local sequence, their logits into zsrc [R0 + Wn], the
+// pool's positions into oldpos [R].
+__global__ void chunk_gather_kernel(const unsigned char* __restrict__ cache, CacheLayout L, unsigned char* __restrict__ klin,
+                                    unsigned char* __restrict__ vlin, float* __restrict__ zsrc, int32_t* __restrict__ oldpos,
+                                    int D, int W, int R, int n0, int R0, int Wn, int Tloc)
+{
+    const int bh = blockIdx.x;
+    const unsigned char* blk = cache + L.header + (size_t)bh * L.stride;
+    const uint4* Kc = reinterpret_cast<const uint4*>(blk + L.off_k);
+    const uint4* Vc = reinterpret_cast<const uint4*>(blk + L.off_v);
+    const float* zc = reinterpret_cast<const float*>(blk + L.off_z);
+    const int32_t* pidx = reinterpret_cast<const int32_t*>(blk + L.off_pidx);
+    const int32_t* meta = reinterpret_cast<const int32_t*>(blk + L.off_meta);
+    if (meta[0] != n0) { if (threadIdx.x == 0) atomicExch(&g_chunk_status, 31); return; }
+    const int cnt = meta[1];
+    const int pieces = D * (int)L.esz / 16;                    // 16-byte pieces per row
+    uint4* kd = reinterpret_cast<uint4*>(klin) + (size_t)bh * Tloc * pieces;
+    uint4* vd = reinterpret_cast<uint4*>(vlin) + (size_t)bh * Tloc * pieces;
+    const int rows = R0 + Wn;
+    for (int e = threadIdx.x; e < rows * pieces; e += blockDim.x) {
+        const int r = e / pieces, c = e % pieces;
+        uint4 kx = make_uint4(0, 0, 0, 0), vx = kx;
+        int src = -1;
+        if (r < R0) { if (r < cnt) src = W + r; }
+        else src = (n0 - Wn + (r - R0)) % W;
+        if (src >= 0) {
+            const int cs = piece_src(L, src, c);
+            kx = Kc[(size_t)src * pieces + cs];
+            vx = Vc[(size_t)src * pieces + cs];
+        }
+        kd[(size_t)r * pieces + c] = kx;
+        vd[(size_t)r * pieces + c] = vx;
+    }
+    for (int r = threadIdx.x; r < rows; r += blockDim.x) {
+        float zz = -INFINITY;
+        if (r < R0) { if (r < cnt) zz = zc[W + r]; }
+        else zz = zc[(n0 - Wn + (r - R0)) % W];
+        zsrc[(size_t)bh * (R + W) + r] = zz;
+    }
+    for (int r = threadIdx.x; r < R; r += blockDim.x) oldpos[(size_t)bh * R + r] = r < cnt ? pidx[r] : -1;
+}
+
+// Logits of the local sequence.  In: z = the scorer's output over the local sequence (wrong where the receptive field
+// reaches below row R0 + half, undefined for the pool rows).  Out: z = the logit of each row's token (the cache's own where
+// it holds one), zrank = the same with sink tokens lifted to +inf, which is what the selection ranks by.
+__global__ void chunk_merge_z_kernel(float* __restrict__ z, float* __restrict__ zrank, const float* __restrict__ zsrc,
+                                     const int32_t* __restrict__ oldpos, int R, int W, int n0, int R0, int Wn, int Tloc,
+                                     int half, int sink)
+{
+    const int bh = blockIdx.y;
+    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= Tloc) return;
+    float zt;
+    int pos;
+    if (r < R0) {
+        pos = oldpos[(size_t)bh * R + r];
+        zt = zsrc[(size_t)bh * (R + W) + r];
+        if (pos < 0) zt = -INFINITY;
+    } else {
+        pos = n0 - Wn + (r - R0);
+        zt = z[(size_t)bh * Tloc + r];
+        if (r < R0 + Wn) {
+            const float zc = zsrc[(size_t)bh * (R + W) + r];
+            // a ring token keeps the logit the cache holds; one the cache has not scored yet is scored now, unless its
+            // left neighbours are no longer there (then it stays unscored, as in the decode step)
+            if (zc > -INFINITY) zt = zc;
+            else if (R0 > 0 && r < R0 + half) zt = -INFINITY;
+        }
+    }
+    z[(size_t)bh * Tloc + r] = zt;
+    zrank[(size_t)bh * Tloc + r] = (pos >= 0 && pos < sink) ? INFINITY : zt;
+}
+
+// Block per (b,h): the cache after the chunk.  Ring <- the last min(n1, W) rows of the local sequence, pool <- the rows the
+// selection kept, with their logits and positions.  Reads only the scratch copies, so the old block can be overwritten.
+__global__ void chunk_commit_kernel(unsigned char* __restrict__ cache, CacheLayout L, const unsigned char* __restrict__ klin,
+                                    const unsigned char* __restrict__ vlin, const float* __restrict__ z,
+                                    const int32_t* __restrict__ idx, const int32_t* __restrict__ cntp,
+                                    const int32_t* __restrict__ oldpos, int D, int W, int R, int n0, int n1, int R0, int Wn,
+                                    int Tloc, int half)
+{
+    if (*reinterpret_cast<volatile int*>(&g_chunk_status) != 0) return;   // the gather found another state: leave the cache alone
+    const int bh = blockIdx.x;
+    unsigned char* blk = cache + L.header + (size_t)bh * L.stride;
+    uint4* Kc = reinterpret_cast<uint4*>(blk + L.off_k);
+    uint4* Vc = reinterpret_cast<uint4*>(blk + L.off_v);
+    float* zc = reinterpret_cast<float*>(blk + L.off_z);
+    int32_t* pidx = reinterpret_cast<int32_t*>(blk + L.off_pidx);
+    int32_t* meta = reinterpret_cast<int32_t*>(blk + L.off_meta);
+    const int pieces = D * (int)L.esz / 16;
+    const uint4* ks = reinterpret_cast<const uint4*>(klin) + (size_t)bh * Tloc * pieces;
+    const uint4* vs = reinterpret_cast<const uint4*>(vlin) + (size_t)bh * Tloc * pieces;
+    const float* zl = z + (size_t)bh * Tloc;
+    const int Wnew = n1 < W ? n1 : W;
+    const int cnt = R > 0 ? cntp[bh] : 0;
+    for (int e = threadIdx.x; e < (Wnew + cnt) * pieces; e += blockDim.x) {
+        const int a = e / pieces, c = e % pieces;
+        int r, row;
+        if (a < Wnew) { r = Tloc - Wnew + a; row = (n1 - Wnew + a) % W; }
+        else { r = idx[(size_t)bh * R + (a - Wnew)]; row = W + (a - Wnew); }
+        const int cd = piece_src(L, row, c);
+        Kc[(size_t)row * pieces + cd] = ks[(size_t)r * pieces + c];
+        Vc[(size_t)row * pieces + cd] = vs[(size_t)r * pieces + c];
+    }
+    for (int a = threadIdx.x; a < W + R; a += blockDim.x) {
+        float zz = -INFINITY;
+        if (a < W) {
+            // slot a holds the newest position congruent to a (mod W), if there is one yet
+            const int lo = n1 - Wnew;
+            const int pos = lo + ((a - lo % W) + W) % W;
+            if (pos < n1 && pos <= n1 - 1 - half) zz = zl[Tloc - (n1 - pos)];
+        } else if (a - W < cnt) {
+            const int r = idx[(size_t)bh * R + (a - W)];
+            zz = zl[r];
+            pidx[a - W] = r < R0 ? oldpos[(size_t)bh * R + r] : n0 - Wn + (r - R0);
+        }
+        zc[a] = zz;
+    }
+    if (threadIdx.x == 0) { meta[0] = n1; meta[1] = cnt; }
+}
+
+}  // namespace
+
+int chunk_status_fetch_and_clear()
+{
+    int h = 0, zero = 0;
+    if (cudaMemcpyFromSymbol(&h, g_chunk_status, sizeof(int)) != cudaSuccess) return -1;
+    if (h != 0) cudaMemcpyToSymbol(g_chunk_status, &zero, sizeof(int));
+    return h;
+}
+
+// p.T = local length; the three launchers run on the same stream in the order gather, (scores), merge, (select, attention), commit
+int launch_chunk_gather(const Params& p, const void* cache, void* klin, void* vlin, float* zsrc, int32_t* oldpos, int n0, int R0,
+                        int Wn, cudaStream_t st)
+{
+    const CacheLayout L = cache_layout(p.d, p.W, p.R, p.dtype);
+    chunk_gather_kernel<<<p.B * p.H, 256, 0, st>>>((const unsigned char*)cache, L, (unsigned char*)klin, (unsigned char*)vlin, zsrc,
+                                                   oldpos, p.d, p.W, p.R, n0, R0, Wn, p.T);
+    return cuda_status(cudaGetLastError());
+}
+
+int launch_chunk_merge_z(const Params& p, float* z, float* zrank, const float* zsrc, const int32_t* oldpos, int n0, int R0, int Wn,
+                         cudaStream_t st)
+{
+    dim3 grid((p.T + 255) / 256, p.B * p.H);
+    chunk_merge_z_kernel<<<grid, 256, 0, st>>>(z, zrank, zsrc, oldpos, p.R, p.W, n0, R0, Wn, p.T, p.half, p.sink);
+    return cuda_status(cudaGetLastError());
+}
+
+int launch_chunk_commit(const Params& p, void* cache, const void* klin, const void* vlin, const float* z, const int32_t* idx,
+                        const int32_t* cnt, const int32_t* oldpos, int n0, int n1, int R0, int Wn, cudaStream_t st)
+{
+    const CacheLayout L = cache_layout(p.d, p.W, p.R, p.dtype);
+    chunk_commit_kernel<<<p.B * p.H, 256, 0, st>>>((unsigned char*)cache, L, (const unsigned char*)klin, (const unsigned char*)vlin, z,
+                                                   idx, cnt, oldpos, p.d, p.W, p.R, n0, n1, R0, Wn, p.T, p.half);
+    return cuda_status(cudaGetLastError());
+}
+
+}  // namespace lte

@@ -103,6 +103,13 @@ int launch_cache_init(const Params& p, const void* k, const void* v, const float
                       const int32_t* cnt, void* cache, cudaStream_t st);
 int launch_ring_linearize(const Params& p, const void* cache, void* klin, void* vlin, cudaStream_t st);
 int launch_ring_scatter_z(const Params& p, void* cache, const float* zlin, cudaStream_t st);
+int launch_chunk_gather(const Params& p, const void* cache, void* klin, void* vlin, float* zsrc, int32_t* oldpos, int n0, int R0,
+                        int Wn, cudaStream_t st);
+int launch_chunk_merge_z(const Params& p, float* z, float* zrank, const float* zsrc, const int32_t* oldpos, int n0, int R0, int Wn,
+                         cudaStream_t st);
+int launch_chunk_commit(const Params& p, void* cache, const void* klin, const void* vlin, const float* z, const int32_t* idx,
+                        const int32_t* cnt, const int32_t* oldpos, int n0, int n1, int R0, int Wn, cudaStream_t st);
+int chunk_status_fetch_and_clear();
 int launch_decode_tc(const Params& p, void* cache, const void* q1, const void* k1, const void* v1, void* o1,
                      float* lse1, cudaStream_t st);
 int launch_decode(const Params& p, void* cache, const void* q1, const void* k1, const void* v1, void* o1,

@@ -96,6 +96,35 @@ CacheScorePlan cache_score_plan(const lte_shape* s, const lte_conv* c)
     return w;
 }
 
+// scratch of lte_attn_prefill_chunk, sized for the longest local sequence (pool rows + full ring + chunk)
+struct ChunkPlan { size_t klin, vlin, qloc, oloc, lseloc, z, zrank, zsrc, oldpos, idx, cnt, sub, total; };
+ChunkPlan chunk_plan(const lte_shape* s, const lte_conv* c)
+{
+    auto up = [](size_t x) { return (x + 255) / 256 * 256; };
+    ChunkPlan w;
+    const size_t G = s->group > 1 ? s->group : 1, bhk = (size_t)s->B * s->H, bhq = bhk * G;
+    const size_t Tm = (size_t)s->R + s->W + s->T, esz = s->dtype == LTE_BF16 ? 2 : 4;
+    size_t off = 0;
+    w.klin = off; off += up(bhk * Tm * s->d * esz);
+    w.vlin = off; off += up(bhk * Tm * s->d * esz);
+    w.qloc = off; off += up(bhq * Tm * s->d * esz);
+    w.oloc = off; off += up(bhq * Tm * s->d * esz);
+    w.lseloc = off; off += up(bhq * Tm * 4);
+    w.z = off; off += up(bhk * Tm * 4);
+    w.zrank = off; off += up(bhk * Tm * 4);
+    w.zsrc = off; off += up(bhk * ((size_t)s->R + s->W) * 4);
+    w.oldpos = off; off += up(bhk * (size_t)(s->R > 0 ? s->R : 1) * 4);
+    w.idx = off; off += up(bhk * (size_t)(s->R > 0 ? s->R : 1) * 4);
+    w.cnt = off; off += up(bhk * 4);
+    w.sub = off;
+    if (c && c->n_layers == 3) {
+        lte_shape s2 = *s; s2.T = (int32_t)Tm;
+        off += up(scores_stack_tc_workspace(make_params(&s2, c)));
+    }
+    w.total = off;
+    return w;
+}
+
 }  // namespace
 }  // namespace lte
 
@@ -126,8 +155,9 @@ int lte_device_status(void)
     const int d = decode_tc_status_fetch_and_clear();
     const int t = stack_tc_status_fetch_and_clear();
     const int u = stack_bwd_tc_status_fetch_and_clear();
-    if (h < 0 || g < 0 || f < 0 || b < 0 || d < 0 || t < 0 || u < 0) return LTE_ERR_CUDA;
-    return (h == 0 && g == 0 && f == 0 && b == 0 && d == 0 && t == 0 && u == 0) ? LTE_OK : LTE_ERR_DEVICE_STATUS;
+    const int k = chunk_status_fetch_and_clear();
+    if (h < 0 || g < 0 || f < 0 || b < 0 || d < 0 || t < 0 || u < 0 || k < 0) return LTE_ERR_CUDA;
+    return (h == 0 && g == 0 && f == 0 && b == 0 && d == 0 && t == 0 && u == 0 && k == 0) ? LTE_OK : LTE_ERR_DEVICE_STATUS;
 }
 
 size_t lte_workspace_bytes(int op, const lte_shape* s, const lte_conv* c)
@@ -141,6 +171,11 @@ size_t lte_workspace_bytes(int op, const lte_shape* s, const lte_conv* c)
     if (op == LTE_OP_DECODE && c && c->n_layers == 3) {
         if (check_shape(s, false) != LTE_OK) return 0;
         return cache_score_plan(s, c).total;
+    }
+    if (op == LTE_OP_CHUNK) {
+        if (check_shape(s, true) != LTE_OK || !c) return 0;
+        if ((double)s->B * s->H * (s->group > 1 ? s->group : 1) * ((double)s->R + s->W + s->T) * s->d > 2.0e10) return 0;
+        return chunk_plan(s, c).total;
     }
     if (op == LTE_OP_SCORES && c && c->n_layers == 3) {
         if (check_shape(s, true) != LTE_OK) return 0;
@@ -233,6 +268,55 @@ int lte_cache_score(const lte_shape* s, const lte_conv* c, void* cache, void* ws
     if (e == LTE_ERR_UNSUPPORTED) e = launch_scores_stack(p, base + w.klin, base + w.vlin, zlin, nullptr, st);
     if (e) return e;
     return launch_ring_scatter_z(p, cache, zlin, st);
+}
+
+int lte_attn_prefill_chunk(const lte_shape* s, const lte_conv* c, void* cache, int32_t n_past, const void* q, const void* k,
+                           const void* v, void* o, float* lse, void* ws, size_t ws_bytes, void* stream)
+{
+    int e = check_shape(s, true); if (e) return e;
+    e = check_conv_or_stack(s, c); if (e) return e;
+    if (!cache || !q || !k || !v || !o || !lse || n_past < 0) return LTE_ERR_INVALID_ARG;
+    if (!aligned16(cache) || !aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return LTE_ERR_INVALID_ARG;
+    const size_t G = s->group > 1 ? s->group : 1, bhk = (size_t)s->B * s->H, bhq = bhk * G;
+    if ((double)bhq * ((double)s->R + s->W + s->T) * s->d > 2.0e10 || (double)n_past + s->T > 2.0e9) return LTE_ERR_UNSUPPORTED;
+    const ChunkPlan w = chunk_plan(s, c);
+    if (!ws || ((uintptr_t)ws & 255u) != 0 || ws_bytes < w.total) return LTE_ERR_WORKSPACE;
+    e = check_arch(); if (e) return e;
+    cudaStream_t st = (cudaStream_t)stream;
+    char* base = (char*)ws;
+    // the local sequence: pool rows (once anything has left the window), the ring in time order, the chunk
+    const int Tc = s->T, Wn = n_past < s->W ? n_past : s->W, R0 = n_past > s->W ? s->R : 0, qoff = R0 + Wn, Tloc = qoff + Tc;
+    lte_shape sl = *s; sl.T = Tloc;
+    Params p = make_params(&sl, c);                          // p.sink: positions of the whole sequence (the logit merge)
+    Params psel = p; psel.sink = 0;                          // the selection sees sink tokens as +inf logits instead
+    const size_t rowb = (size_t)s->d * (s->dtype == LTE_BF16 ? 2 : 4);
+    float* z = (float*)(base + w.z); float* zrank = (float*)(base + w.zrank); float* zsrc = (float*)(base + w.zsrc);
+    int32_t* oldpos = (int32_t*)(base + w.oldpos); int32_t* idx = (int32_t*)(base + w.idx); int32_t* cnt = (int32_t*)(base + w.cnt);
+    e = launch_chunk_gather(p, cache, base + w.klin, base + w.vlin, zsrc, oldpos, n_past, R0, Wn, st); if (e) return e;
+    if (cudaMemcpy2DAsync(base + w.klin + qoff * rowb, Tloc * rowb, k, Tc * rowb, Tc * rowb, bhk, cudaMemcpyDeviceToDevice, st) != cudaSuccess ||
+        cudaMemcpy2DAsync(base + w.vlin + qoff * rowb, Tloc * rowb, v, Tc * rowb, Tc * rowb, bhk, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+        return LTE_ERR_CUDA;
+    if (p.stack) {
+        e = launch_scores_stack_tc(p, base + w.klin, base + w.vlin, z, nullptr, base + w.sub, w.total - w.sub, st);
+        if (e == LTE_ERR_UNSUPPORTED) e = launch_scores_stack(p, base + w.klin, base + w.vlin, z, nullptr, st);
+    } else {
+        e = launch_scores(p, base + w.klin, base + w.vlin, z, nullptr, st);
+    }
+    if (e) return e;
+    e = launch_chunk_merge_z(p, z, zrank, zsrc, oldpos, n_past, R0, Wn, st); if (e) return e;
+    e = launch_select(psel, zrank, idx, cnt, nullptr, st); if (e) return e;
+    // queries padded to the local length (the rows below the chunk are zero and their outputs unused)
+    if (cudaMemsetAsync(base + w.qloc, 0, bhq * Tloc * rowb, st) != cudaSuccess ||
+        cudaMemcpy2DAsync(base + w.qloc + qoff * rowb, Tloc * rowb, q, Tc * rowb, Tc * rowb, bhq, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+        return LTE_ERR_CUDA;
+    float* lsel = (float*)(base + w.lseloc);
+    if (s->dtype == LTE_BF16) e = launch_prefill_tc(p, base + w.qloc, base + w.klin, base + w.vlin, idx, cnt, base + w.oloc, lsel, st);
+    else e = launch_prefill_simt(p, base + w.qloc, base + w.klin, base + w.vlin, idx, cnt, base + w.oloc, lsel, st);
+    if (e) return e;
+    if (cudaMemcpy2DAsync(o, Tc * rowb, base + w.oloc + qoff * rowb, Tloc * rowb, Tc * rowb, bhq, cudaMemcpyDeviceToDevice, st) != cudaSuccess ||
+        cudaMemcpy2DAsync(lse, (size_t)Tc * 4, lsel + qoff, (size_t)Tloc * 4, (size_t)Tc * 4, bhq, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+        return LTE_ERR_CUDA;
+    return launch_chunk_commit(p, cache, base + w.klin, base + w.vlin, z, idx, cnt, oldpos, n_past, n_past + Tc, R0, Wn, st);
 }
 
 int lte_attn_decode(const lte_shape* s, const lte_conv* c, void* cache, const void* q1, const void* k1,
