@@ -353,7 +353,58 @@ def _extras_sections(torch, lte, synth, pk, flush, args, which):
         _extra_p(out, torch, lte, synth, pk, flush, n5)
     if "S" in which:
         _extra_s(out, torch, lte, synth, pk, flush, n5)
+    if "K" in which:
+        _extra_k(out, torch, lte, synth, pk, flush, n5)
     return out
+
+
+def _extra_k(out, torch, lte, synth, pk, flush, n5):
+    """Chunked prefill on top of a cache (lte_attn_prefill_chunk): a prompt of T tokens is prefilled in one shot and cached,
+    then a chunk of Tc more tokens arrives.  Two shapes: C2's (chunk = another 4096 tokens) and a serving-like one with the
+    paper's window and budget (W = 768, R = 512; chunk of 512 tokens), where the local sequence is mostly cache rows."""
+    import dataclasses
+    res = {}
+    for tag, cfg, Tc in (("C2_shape", synth.CONFIGS["C2"], 4096),
+                         ("serving_like", dataclasses.replace(synth.CONFIGS["C2"], B=8, W=768, R=512), 512)):
+        x = device_inputs(cfg, 11, torch, T=cfg.T + Tc)
+        s0 = lte.shape(cfg.B, cfg.H, cfg.T, cfg.d, cfg.W, cfg.R, lte.BF16)
+        sc = lte.shape(cfg.B, cfg.H, Tc, cfg.d, cfg.W, cfg.R, lte.BF16)
+        c = lte.conv(x["w"])
+        kp, vp = x["k"][:, :, :cfg.T].contiguous(), x["v"][:, :, :cfg.T].contiguous()
+        z = lte.lte_scores(s0, c, kp, vp)
+        idx, cnt = lte.lte_select(s0, z)
+        cache0 = lte.lte_cache_init(s0, c, kp, vp, z, idx, cnt)
+        cache = cache0.clone()
+        qc, kc, vc = (x[t][:, :, cfg.T:].contiguous() for t in "qkv")
+        o = torch.empty_like(qc); lse = torch.empty((cfg.B, cfg.H, Tc), dtype=torch.float32, device="cuda")
+        ws = torch.empty(lte.lte_workspace_bytes(lte.OP_CHUNK, sc, c), dtype=torch.uint8, device="cuda")
+        ms = []
+        for it in range(3 + n5):
+            cache.copy_(cache0)
+            flush()
+            e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+            e0.record()
+            lte.lte_attn_prefill_chunk(sc, c, cache, cfg.T, qc, kc, vc, o=o, lse=lse, ws=ws)
+            e1.record(); torch.cuda.synchronize()
+            if it >= 3:
+                ms.append(e0.elapsed_time(e1))
+        # the one-shot path over a prompt of the chunk's length, for scale
+        s1 = lte.shape(cfg.B, cfg.H, Tc, cfg.d, cfg.W, cfg.R, lte.BF16)
+        z1 = torch.empty((cfg.B, cfg.H, Tc), dtype=torch.float32, device="cuda")
+        i1 = torch.empty((cfg.B, cfg.H, cfg.R), dtype=torch.int32, device="cuda"); c1 = torch.empty((cfg.B, cfg.H), dtype=torch.int32, device="cuda")
+
+        def one_shot():
+            lte.lte_scores(s1, c, kc, vc, z=z1); lte.lte_select(s1, z1, idx=i1, cnt=c1)
+            lte.lte_attn_prefill(s1, qc, kc, vc, i1, c1, o=o, lse=lse)
+
+        ms1, _ = timed(torch, one_shot, n5, 3, flush)
+        t = mid3(ms) * 1e-3
+        res[tag] = {"workload": "B=%d H=%d d=%d, cache after %d tokens (W=%d, R=%d), chunk of %d tokens" % (cfg.B, cfg.H, cfg.d, cfg.T, cfg.W, cfg.R, Tc),
+                    "chunk_ms": t * 1e3, "tokens_per_s": cfg.B * Tc / t, "local_rows": cfg.R + cfg.W + Tc,
+                    "one_shot_prefill_of_a_prompt_of_the_chunks_length_ms": mid3(ms1),
+                    "workspace_bytes": int(ws.numel())}
+        del x, cache, cache0, ws, o, lse, qc, kc, vc
+    out["K_chunked_prefill"] = res
 
 
 def _extra_s(out, torch, lte, synth, pk, flush, n5):
@@ -744,7 +795,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="lte", choices=["lte", "reference"])
     ap.add_argument("--no-extras", action="store_true")
-    ap.add_argument("--section", default=None, choices=["C3", "C4", "C5", "P", "S"],
+    ap.add_argument("--section", default=None, choices=["C3", "C4", "C5", "P", "S", "K"],
                     help="time only this extra section (long prefill / decode / forward+backward) after the main loop")
     ap.add_argument("--skip-main", action="store_true", help="with --section: skip the main C2 loop")
     args = ap.parse_args()

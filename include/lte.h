@@ -213,7 +213,7 @@ int lte_cache_score(const lte_shape* s, const lte_conv* c, void* cache, void* ws
  *   o        out  [B,H*group,T,d];   lse out [B,H*group,T] fp32
  *   ws       device scratch of lte_workspace_bytes(LTE_OP_CHUNK, s, c) bytes, 256-byte aligned: the pool, the ring in
  *            time order and the chunk are laid out as one local sequence of at most R + W + T rows, which the scorer, the
- *            selection and the prefill attention kernels then process (queries padded to that length)
+ *            selection and the prefill attention kernels then process (q, o and lse are used in place)
  * Errors: INVALID_ARG, UNSUPPORTED (as lte_cache_init; local sequence too long), WORKSPACE, CUDA.
  */
 int lte_attn_prefill_chunk(const lte_shape* s, const lte_conv* c, void* cache, int32_t n_past,

@@ -9,8 +9,8 @@
 //     rows [R0 + Wn, T_loc)   the chunk
 // because every pool row is older than every chunk query's window and the window of a chunk query never reaches below
 // row R0.  So the path is: gather the local sequence (here), score it (the scorer kernels), merge the logits the cache
-// already holds (here), select, attend (the prefill kernels, queries padded to the local length), and write the new
-// cache (here).  Local row r stands for position pos(r) = old pool position (r < R0) or n0 - Wn + (r - R0).
+// already holds (here), select, attend (the prefill kernels, told that their queries start at row R0 + Wn), and write the
+// new cache (here).  Local row r stands for position pos(r) = old pool position (r < R0) or n0 - Wn + (r - R0).
 #include "common.cuh"
 
 namespace lte {
@@ -22,13 +22,17 @@ namespace {
 // one 16-byte piece of a cache row -> the same piece of a plain row (the swizzled layout permutes the pieces of a row)
 __device__ __forceinline__ int piece_src(const CacheLayout& L, int row, int c) { return L.swz ? (c ^ (row & 7)) : c; }
 
-// Block per (b,h): pool rows and ring rows (time order) into the local sequence, their logits into zsrc [R0 + Wn], the
-// pool's positions into oldpos [R].
-__global__ void chunk_gather_kernel(const unsigned char* __restrict__ cache, CacheLayout L, unsigned char* __restrict__ klin,
+constexpr int kRowsPerBlock = 128;
+
+// Block (part, (b,h)): rows [part 128, part 128 + 128) of the local sequence: pool rows, ring rows (time order) and the
+// chunk's rows of k, v.  Part 0 also copies the logits of the pool and the ring into zsrc [R0 + Wn] and the pool's
+// positions into oldpos [R].
+__global__ void chunk_gather_kernel(const unsigned char* __restrict__ cache, CacheLayout L, const unsigned char* __restrict__ kc,
+                                    const unsigned char* __restrict__ vc, unsigned char* __restrict__ klin,
                                     unsigned char* __restrict__ vlin, float* __restrict__ zsrc, int32_t* __restrict__ oldpos,
                                     int D, int W, int R, int n0, int R0, int Wn, int Tloc)
 {
-    const int bh = blockIdx.x;
+    const int bh = blockIdx.y;
     const unsigned char* blk = cache + L.header + (size_t)bh * L.stride;
     const uint4* Kc = reinterpret_cast<const uint4*>(blk + L.off_k);
     const uint4* Vc = reinterpret_cast<const uint4*>(blk + L.off_v);
@@ -40,21 +44,30 @@ __global__ void chunk_gather_kernel(const unsigned char* __restrict__ cache, Cac
     const int pieces = D * (int)L.esz / 16;                    // 16-byte pieces per row
     uint4* kd = reinterpret_cast<uint4*>(klin) + (size_t)bh * Tloc * pieces;
     uint4* vd = reinterpret_cast<uint4*>(vlin) + (size_t)bh * Tloc * pieces;
-    const int rows = R0 + Wn;
-    for (int e = threadIdx.x; e < rows * pieces; e += blockDim.x) {
+    const int rows = R0 + Wn, Tc = Tloc - rows;
+    const uint4* kq = reinterpret_cast<const uint4*>(kc) + (size_t)bh * Tc * pieces;
+    const uint4* vq = reinterpret_cast<const uint4*>(vc) + (size_t)bh * Tc * pieces;
+    const int r_lo = blockIdx.x * kRowsPerBlock, r_hi = min(r_lo + kRowsPerBlock, Tloc);
+    for (int e = r_lo * pieces + threadIdx.x; e < r_hi * pieces; e += blockDim.x) {
         const int r = e / pieces, c = e % pieces;
         uint4 kx = make_uint4(0, 0, 0, 0), vx = kx;
-        int src = -1;
-        if (r < R0) { if (r < cnt) src = W + r; }
-        else src = (n0 - Wn + (r - R0)) % W;
-        if (src >= 0) {
-            const int cs = piece_src(L, src, c);
-            kx = Kc[(size_t)src * pieces + cs];
-            vx = Vc[(size_t)src * pieces + cs];
+        if (r >= rows) {
+            kx = kq[(size_t)(r - rows) * pieces + c];
+            vx = vq[(size_t)(r - rows) * pieces + c];
+        } else {
+            int src = -1;
+            if (r < R0) { if (r < cnt) src = W + r; }
+            else src = (n0 - Wn + (r - R0)) % W;
+            if (src >= 0) {
+                const int cs = piece_src(L, src, c);
+                kx = Kc[(size_t)src * pieces + cs];
+                vx = Vc[(size_t)src * pieces + cs];
+            }
         }
         kd[(size_t)r * pieces + c] = kx;
         vd[(size_t)r * pieces + c] = vx;
     }
+    if (blockIdx.x != 0) return;
     for (int r = threadIdx.x; r < rows; r += blockDim.x) {
         float zz = -INFINITY;
         if (r < R0) { if (r < cnt) zz = zc[W + r]; }
@@ -95,7 +108,8 @@ __global__ void chunk_merge_z_kernel(float* __restrict__ z, float* __restrict__ 
     zrank[(size_t)bh * Tloc + r] = (pos >= 0 && pos < sink) ? INFINITY : zt;
 }
 
-// Block per (b,h): the cache after the chunk.  Ring <- the last min(n1, W) rows of the local sequence, pool <- the rows the
+// Block (part, (b,h)): the cache after the chunk, 128 of its key/value rows per part; part 0 also writes the logits, the
+// positions and the counters.  Ring <- the last min(n1, W) rows of the local sequence, pool <- the rows the
 // selection kept, with their logits and positions.  Reads only the scratch copies, so the old block can be overwritten.
 __global__ void chunk_commit_kernel(unsigned char* __restrict__ cache, CacheLayout L, const unsigned char* __restrict__ klin,
                                     const unsigned char* __restrict__ vlin, const float* __restrict__ z,
@@ -104,7 +118,7 @@ __global__ void chunk_commit_kernel(unsigned char* __restrict__ cache, CacheLayo
                                     int Tloc, int half)
 {
     if (*reinterpret_cast<volatile int*>(&g_chunk_status) != 0) return;   // the gather found another state: leave the cache alone
-    const int bh = blockIdx.x;
+    const int bh = blockIdx.y;
     unsigned char* blk = cache + L.header + (size_t)bh * L.stride;
     uint4* Kc = reinterpret_cast<uint4*>(blk + L.off_k);
     uint4* Vc = reinterpret_cast<uint4*>(blk + L.off_v);
@@ -117,7 +131,8 @@ __global__ void chunk_commit_kernel(unsigned char* __restrict__ cache, CacheLayo
     const float* zl = z + (size_t)bh * Tloc;
     const int Wnew = n1 < W ? n1 : W;
     const int cnt = R > 0 ? cntp[bh] : 0;
-    for (int e = threadIdx.x; e < (Wnew + cnt) * pieces; e += blockDim.x) {
+    const int a_lo = blockIdx.x * kRowsPerBlock, a_hi = min(a_lo + kRowsPerBlock, Wnew + cnt);
+    for (int e = a_lo * pieces + threadIdx.x; e < a_hi * pieces; e += blockDim.x) {
         const int a = e / pieces, c = e % pieces;
         int r, row;
         if (a < Wnew) { r = Tloc - Wnew + a; row = (n1 - Wnew + a) % W; }
@@ -126,6 +141,7 @@ __global__ void chunk_commit_kernel(unsigned char* __restrict__ cache, CacheLayo
         Kc[(size_t)row * pieces + cd] = ks[(size_t)r * pieces + c];
         Vc[(size_t)row * pieces + cd] = vs[(size_t)r * pieces + c];
     }
+    if (blockIdx.x != 0) return;
     for (int a = threadIdx.x; a < W + R; a += blockDim.x) {
         float zz = -INFINITY;
         if (a < W) {
@@ -153,13 +169,14 @@ int chunk_status_fetch_and_clear()
     return h;
 }
 
-// p.T = local length; the three launchers run on the same stream in the order gather, (scores), merge, (select, attention), commit
-int launch_chunk_gather(const Params& p, const void* cache, void* klin, void* vlin, float* zsrc, int32_t* oldpos, int n0, int R0,
-                        int Wn, cudaStream_t st)
+// p.T = local length; the launchers run on one stream in the order gather, (scores), merge, (select, attention), commit
+int launch_chunk_gather(const Params& p, const void* cache, const void* k, const void* v, void* klin, void* vlin, float* zsrc,
+                        int32_t* oldpos, int n0, int R0, int Wn, cudaStream_t st)
 {
     const CacheLayout L = cache_layout(p.d, p.W, p.R, p.dtype);
-    chunk_gather_kernel<<<p.B * p.H, 256, 0, st>>>((const unsigned char*)cache, L, (unsigned char*)klin, (unsigned char*)vlin, zsrc,
-                                                   oldpos, p.d, p.W, p.R, n0, R0, Wn, p.T);
+    dim3 grid((p.T + kRowsPerBlock - 1) / kRowsPerBlock, p.B * p.H);
+    chunk_gather_kernel<<<grid, 256, 0, st>>>((const unsigned char*)cache, L, (const unsigned char*)k, (const unsigned char*)v,
+                                              (unsigned char*)klin, (unsigned char*)vlin, zsrc, oldpos, p.d, p.W, p.R, n0, R0, Wn, p.T);
     return cuda_status(cudaGetLastError());
 }
 
@@ -175,7 +192,8 @@ int launch_chunk_commit(const Params& p, void* cache, const void* klin, const vo
                         const int32_t* cnt, const int32_t* oldpos, int n0, int n1, int R0, int Wn, cudaStream_t st)
 {
     const CacheLayout L = cache_layout(p.d, p.W, p.R, p.dtype);
-    chunk_commit_kernel<<<p.B * p.H, 256, 0, st>>>((unsigned char*)cache, L, (const unsigned char*)klin, (const unsigned char*)vlin, z,
+    dim3 grid((p.W + p.R + kRowsPerBlock - 1) / kRowsPerBlock, p.B * p.H);
+    chunk_commit_kernel<<<grid, 256, 0, st>>>((unsigned char*)cache, L, (const unsigned char*)klin, (const unsigned char*)vlin, z,
                                                    idx, cnt, oldpos, p.d, p.W, p.R, n0, n1, R0, Wn, p.T, p.half);
     return cuda_status(cudaGetLastError());
 }

@@ -14,6 +14,7 @@ constexpr int kMaxTaps = 13;          // scorer taps the kernels are instantiate
 struct Params {                       // validated, host-resolved view of lte_shape / lte_conv
     int B, H, T, d, W, R, sink, K, half;
     int G;                            // query heads per key/value head (q, o, lse have H * G heads)
+    int qoff;                         // prefill attention: q, o, lse hold the queries at positions qoff .. T-1 only (chunked prefill; else 0)
     int stack;                        // 1: the three-layer scorer stack (w, bias packed as lte.h describes; K = 13, half = 6)
     float zthr;                       // logit(tau): keep iff z > zthr
     float scale;                      // softmax scale
@@ -103,8 +104,8 @@ int launch_cache_init(const Params& p, const void* k, const void* v, const float
                       const int32_t* cnt, void* cache, cudaStream_t st);
 int launch_ring_linearize(const Params& p, const void* cache, void* klin, void* vlin, cudaStream_t st);
 int launch_ring_scatter_z(const Params& p, void* cache, const float* zlin, cudaStream_t st);
-int launch_chunk_gather(const Params& p, const void* cache, void* klin, void* vlin, float* zsrc, int32_t* oldpos, int n0, int R0,
-                        int Wn, cudaStream_t st);
+int launch_chunk_gather(const Params& p, const void* cache, const void* k, const void* v, void* klin, void* vlin, float* zsrc,
+                        int32_t* oldpos, int n0, int R0, int Wn, cudaStream_t st);
 int launch_chunk_merge_z(const Params& p, float* z, float* zrank, const float* zsrc, const int32_t* oldpos, int n0, int R0, int Wn,
                          cudaStream_t st);
 int launch_chunk_commit(const Params& p, void* cache, const void* klin, const void* vlin, const float* z, const int32_t* idx,

@@ -49,6 +49,7 @@ Params make_params(const lte_shape* s, const lte_conv* c)
     p.G = s->group > 1 ? s->group : 1;
     p.K = c ? c->kernel : 1; p.half = p.K / 2;
     p.stack = 0;
+    p.qoff = 0;
     if (c && c->n_layers == 3) { p.stack = 1; p.K = 13; p.half = 6; }   // the paper's stack: receptive field 13
     p.zthr = s->tau <= 0.f ? -INFINITY : (float)(log((double)s->tau) - log1p(-(double)s->tau));
     p.scale = s->softmax_scale > 0.f ? s->softmax_scale : (float)(1.0 / sqrt((double)s->d));
@@ -97,19 +98,16 @@ CacheScorePlan cache_score_plan(const lte_shape* s, const lte_conv* c)
 }
 
 // scratch of lte_attn_prefill_chunk, sized for the longest local sequence (pool rows + full ring + chunk)
-struct ChunkPlan { size_t klin, vlin, qloc, oloc, lseloc, z, zrank, zsrc, oldpos, idx, cnt, sub, total; };
+struct ChunkPlan { size_t klin, vlin, z, zrank, zsrc, oldpos, idx, cnt, sub, total; };
 ChunkPlan chunk_plan(const lte_shape* s, const lte_conv* c)
 {
     auto up = [](size_t x) { return (x + 255) / 256 * 256; };
     ChunkPlan w;
-    const size_t G = s->group > 1 ? s->group : 1, bhk = (size_t)s->B * s->H, bhq = bhk * G;
+    const size_t bhk = (size_t)s->B * s->H;
     const size_t Tm = (size_t)s->R + s->W + s->T, esz = s->dtype == LTE_BF16 ? 2 : 4;
     size_t off = 0;
     w.klin = off; off += up(bhk * Tm * s->d * esz);
     w.vlin = off; off += up(bhk * Tm * s->d * esz);
-    w.qloc = off; off += up(bhq * Tm * s->d * esz);
-    w.oloc = off; off += up(bhq * Tm * s->d * esz);
-    w.lseloc = off; off += up(bhq * Tm * 4);
     w.z = off; off += up(bhk * Tm * 4);
     w.zrank = off; off += up(bhk * Tm * 4);
     w.zsrc = off; off += up(bhk * ((size_t)s->R + s->W) * 4);
@@ -277,7 +275,7 @@ int lte_attn_prefill_chunk(const lte_shape* s, const lte_conv* c, void* cache, i
     e = check_conv_or_stack(s, c); if (e) return e;
     if (!cache || !q || !k || !v || !o || !lse || n_past < 0) return LTE_ERR_INVALID_ARG;
     if (!aligned16(cache) || !aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return LTE_ERR_INVALID_ARG;
-    const size_t G = s->group > 1 ? s->group : 1, bhk = (size_t)s->B * s->H, bhq = bhk * G;
+    const size_t G = s->group > 1 ? s->group : 1, bhq = (size_t)s->B * s->H * G;
     if ((double)bhq * ((double)s->R + s->W + s->T) * s->d > 2.0e10 || (double)n_past + s->T > 2.0e9) return LTE_ERR_UNSUPPORTED;
     const ChunkPlan w = chunk_plan(s, c);
     if (!ws || ((uintptr_t)ws & 255u) != 0 || ws_bytes < w.total) return LTE_ERR_WORKSPACE;
@@ -289,13 +287,10 @@ int lte_attn_prefill_chunk(const lte_shape* s, const lte_conv* c, void* cache, i
     lte_shape sl = *s; sl.T = Tloc;
     Params p = make_params(&sl, c);                          // p.sink: positions of the whole sequence (the logit merge)
     Params psel = p; psel.sink = 0;                          // the selection sees sink tokens as +inf logits instead
-    const size_t rowb = (size_t)s->d * (s->dtype == LTE_BF16 ? 2 : 4);
+    Params patt = p; patt.qoff = qoff;                       // the queries are the chunk's: positions qoff .. Tloc-1
     float* z = (float*)(base + w.z); float* zrank = (float*)(base + w.zrank); float* zsrc = (float*)(base + w.zsrc);
     int32_t* oldpos = (int32_t*)(base + w.oldpos); int32_t* idx = (int32_t*)(base + w.idx); int32_t* cnt = (int32_t*)(base + w.cnt);
-    e = launch_chunk_gather(p, cache, base + w.klin, base + w.vlin, zsrc, oldpos, n_past, R0, Wn, st); if (e) return e;
-    if (cudaMemcpy2DAsync(base + w.klin + qoff * rowb, Tloc * rowb, k, Tc * rowb, Tc * rowb, bhk, cudaMemcpyDeviceToDevice, st) != cudaSuccess ||
-        cudaMemcpy2DAsync(base + w.vlin + qoff * rowb, Tloc * rowb, v, Tc * rowb, Tc * rowb, bhk, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
-        return LTE_ERR_CUDA;
+    e = launch_chunk_gather(p, cache, k, v, base + w.klin, base + w.vlin, zsrc, oldpos, n_past, R0, Wn, st); if (e) return e;
     if (p.stack) {
         e = launch_scores_stack_tc(p, base + w.klin, base + w.vlin, z, nullptr, base + w.sub, w.total - w.sub, st);
         if (e == LTE_ERR_UNSUPPORTED) e = launch_scores_stack(p, base + w.klin, base + w.vlin, z, nullptr, st);
@@ -305,17 +300,10 @@ int lte_attn_prefill_chunk(const lte_shape* s, const lte_conv* c, void* cache, i
     if (e) return e;
     e = launch_chunk_merge_z(p, z, zrank, zsrc, oldpos, n_past, R0, Wn, st); if (e) return e;
     e = launch_select(psel, zrank, idx, cnt, nullptr, st); if (e) return e;
-    // queries padded to the local length (the rows below the chunk are zero and their outputs unused)
-    if (cudaMemsetAsync(base + w.qloc, 0, bhq * Tloc * rowb, st) != cudaSuccess ||
-        cudaMemcpy2DAsync(base + w.qloc + qoff * rowb, Tloc * rowb, q, Tc * rowb, Tc * rowb, bhq, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
-        return LTE_ERR_CUDA;
-    float* lsel = (float*)(base + w.lseloc);
-    if (s->dtype == LTE_BF16) e = launch_prefill_tc(p, base + w.qloc, base + w.klin, base + w.vlin, idx, cnt, base + w.oloc, lsel, st);
-    else e = launch_prefill_simt(p, base + w.qloc, base + w.klin, base + w.vlin, idx, cnt, base + w.oloc, lsel, st);
+    // the attention kernels take the chunk's q, o, lse as they are: query row r stands at position qoff + r
+    if (s->dtype == LTE_BF16) e = launch_prefill_tc(patt, q, base + w.klin, base + w.vlin, idx, cnt, o, lse, st);
+    else e = launch_prefill_simt(patt, q, base + w.klin, base + w.vlin, idx, cnt, o, lse, st);
     if (e) return e;
-    if (cudaMemcpy2DAsync(o, Tc * rowb, base + w.oloc + qoff * rowb, Tloc * rowb, Tc * rowb, bhq, cudaMemcpyDeviceToDevice, st) != cudaSuccess ||
-        cudaMemcpy2DAsync(lse, (size_t)Tc * 4, lsel + qoff, (size_t)Tloc * 4, (size_t)Tc * 4, bhq, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
-        return LTE_ERR_CUDA;
     return launch_chunk_commit(p, cache, base + w.klin, base + w.vlin, z, idx, cnt, oldpos, n_past, n_past + Tc, R0, Wn, st);
 }
 

@@ -11,17 +11,17 @@ template <typename T, int D>
 __global__ void __launch_bounds__(128) prefill_simt_kernel(const T* __restrict__ q, const T* __restrict__ k,
                                                            const T* __restrict__ v, const int32_t* __restrict__ idx,
                                                            const int32_t* __restrict__ cnt, T* __restrict__ o,
-                                                           float* __restrict__ lse, int Tlen, int W, int R, float scale, int G)
+                                                           float* __restrict__ lse, int Tlen, int W, int R, float scale, int G, int qoff)
 {
     constexpr int C = D / 32;                  // channels per lane
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int i = blockIdx.x * 4 + warp;
+    const int i = qoff + blockIdx.x * 4 + warp;     // position; q, o, lse hold the queries from position qoff on
     const int bh = blockIdx.y, bhk = bh / G;   // query head and its key/value head
     if (i >= Tlen) return;
-    const size_t base = (size_t)bh * Tlen * D, kbase = (size_t)bhk * Tlen * D;
+    const size_t base = ((size_t)bh * (Tlen - qoff) + (i - qoff)) * D, kbase = (size_t)bhk * Tlen * D;   // this query's row of q and o
     float qv[C], acc[C];
 #pragma unroll
-    for (int c = 0; c < C; ++c) { qv[c] = to_f(q[base + (size_t)i * D + lane + 32 * c]) * scale; acc[c] = 0.f; }
+    for (int c = 0; c < C; ++c) { qv[c] = to_f(q[base + lane + 32 * c]) * scale; acc[c] = 0.f; }
     float m = -INFINITY, l = 0.f;
     const int32_t* id = idx + (size_t)bhk * R;
     const int n_ret = cnt[bhk];
@@ -52,18 +52,18 @@ __global__ void __launch_bounds__(128) prefill_simt_kernel(const T* __restrict__
     }
     const float inv = 1.f / l;
 #pragma unroll
-    for (int c = 0; c < C; ++c) o[base + (size_t)i * D + lane + 32 * c] = from_f<T>(acc[c] * inv);
-    if (lane == 0) lse[(size_t)bh * Tlen + i] = m + logf(l);
+    for (int c = 0; c < C; ++c) o[base + lane + 32 * c] = from_f<T>(acc[c] * inv);
+    if (lane == 0) lse[(size_t)bh * (Tlen - qoff) + (i - qoff)] = m + logf(l);
 }
 
 template <typename T>
 int run(const Params& p, const void* q, const void* k, const void* v, const int32_t* idx, const int32_t* cnt,
         void* o, float* lse, cudaStream_t st)
 {
-    dim3 grid((p.T + 3) / 4, p.B * p.H * p.G);
+    dim3 grid((p.T - p.qoff + 3) / 4, p.B * p.H * p.G);
 #define LTE_GO(D)                                                                                          \
     prefill_simt_kernel<T, D><<<grid, 128, 0, st>>>((const T*)q, (const T*)k, (const T*)v, idx, cnt, (T*)o, \
-                                                    lse, p.T, p.W, p.R, p.scale, p.G)
+                                                    lse, p.T, p.W, p.R, p.scale, p.G, p.qoff)
     switch (p.d) {
         case 32: LTE_GO(32); break;
         case 64: LTE_GO(64); break;

@@ -56,13 +56,13 @@ struct Item {
 // Items are numbered from the last query tile of every (b,h) down to the first: later query tiles see more retained
 // rows and cost more, and a CTA takes items n, n + grid, n + 2 grid, ... so every CTA gets one item of each cost band
 // (largest first), which balances the static schedule.
-__device__ __forceinline__ Item decode_item(int item, int n_qt, int n_bh, int Tlen, int W, int G)
+__device__ __forceinline__ Item decode_item(int item, int n_qt, int n_bh, int Tlen, int W, int G, int qoff)
 {
     Item it;
     const int r = item / n_bh;
     it.bh = item - r * n_bh;
     it.bhk = it.bh / G;                                 // the G query heads of a key/value head are adjacent
-    it.i0 = (n_qt - 1 - r) * BM;
+    it.i0 = qoff + (n_qt - 1 - r) * BM;                 // positions; the query tensors start at position qoff
     it.i_hi = min(it.i0 + BM - 1, Tlen - 1);
     it.j_start = max(it.i0 - W + 1, 0);
     it.n_win = (it.i_hi - it.j_start + 1 + BN - 1) / BN;
@@ -102,7 +102,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                   const __nv_bfloat16* __restrict__ kg,
                   const __nv_bfloat16* __restrict__ vg, const int32_t* __restrict__ idx,
                   const int32_t* __restrict__ cnt, float* __restrict__ lse, int Tlen,
-                  int W, int R, float scale, int n_qt, int n_bh, int G)
+                  int W, int R, float scale, int n_qt, int n_bh, int G, int qoff)
 {
     const int n_items = n_qt * n_bh;
     using S = Smem<D>;
@@ -163,13 +163,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         uint32_t g = 0;                                        // tiles of the items before this one
         int it = 0;
         for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++it) {
-            const Item w = decode_item(item, n_qt, n_bh, Tlen, W, G);
+            const Item w = decode_item(item, n_qt, n_bh, Tlen, W, G, qoff);
             if (lane == 0) {
                 // Q: its buffer is free once the previous item's last S product has completed
                 if (it > 0) mbar_wait(bar_qf, (it - 1) & 1, 12);
                 mbar_expect_tx(bar_q, S::QTILE);
 #pragma unroll
-                for (int sb = 0; sb < SUB; ++sb) tma_load_3d(sQ + sb * 16384, &tmQ, sb * 64, w.i0, w.bh, bar_q);
+                for (int sb = 0; sb < SUB; ++sb) tma_load_3d(sQ + sb * 16384, &tmQ, sb * 64, w.i0 - qoff, w.bh, bar_q);
                 // window tiles, each into its stage as soon as the MMA that read the stage's previous tile has completed
                 for (int t = 0; t < w.n_win; ++t) {
                     const uint32_t gg = g + t;
@@ -206,12 +206,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         // tiles of an item (whole warp: the count of visible list entries takes global loads)
         auto item_tiles = [&](int item) {
             if (item >= n_items) return 0;
-            const Item w = decode_item(item, n_qt, n_bh, Tlen, W, G);
+            const Item w = decode_item(item, n_qt, n_bh, Tlen, W, G, qoff);
             return w.n_win + (count_le(idx + (size_t)w.bhk * R, cnt[w.bhk], w.i_hi - W, lane) + BN - 1) / BN;
         };
         int n_tiles_next = item_tiles(blockIdx.x);
         for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++it) {
-            const Item w = decode_item(item, n_qt, n_bh, Tlen, W, G);
+            const Item w = decode_item(item, n_qt, n_bh, Tlen, W, G, qoff);
             const int n_tiles = n_tiles_next;
             int ts = 0;                                        // S products of this item issued so far
             // gathers issued before the top of tile gg have landed
@@ -282,7 +282,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         int pf_cnt = 0, pf_e[4] = {0, 0, 0, 0};
         auto prefetch_list = [&](int item) {
             if (item < n_items) {
-                const Item w = decode_item(item, n_qt, n_bh, Tlen, W, G);
+                const Item w = decode_item(item, n_qt, n_bh, Tlen, W, G, qoff);
                 pf_cnt = cnt[w.bhk];
 #pragma unroll
                 for (int u = 0; u < 4; ++u) pf_e[u] = u * 32 + lane < R ? idx[(size_t)w.bhk * R + u * 32 + lane] : 0x7fffffff;
@@ -290,7 +290,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         };
         prefetch_list(blockIdx.x);
         for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++it) {
-            const Item w = decode_item(item, n_qt, n_bh, Tlen, W, G);
+            const Item w = decode_item(item, n_qt, n_bh, Tlen, W, G, qoff);
             const int bh = w.bh, bhk = w.bhk, n_win = w.n_win, j_start = w.j_start;
             const int32_t* id = idx + (size_t)bhk * R;
             const int n_ret = pf_cnt;
@@ -542,11 +542,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 fence_proxy_async();
                 __syncwarp();
                 if (lane == 0 && w.i0 + warp * 32 < Tlen) {
-                    tma_store_3d(&tmO, slab, sb * 64, w.i0 + warp * 32, bh);
+                    tma_store_3d(&tmO, slab, sb * 64, w.i0 - qoff + warp * 32, bh);
                     bulk_commit();
                 }
             }
-            if (i < Tlen) lse[(size_t)bh * Tlen + i] = m_run * 0.6931471805599453f + logf(l_run);
+            if (i < Tlen) lse[(size_t)bh * (Tlen - qoff) + (i - qoff)] = m_run * 0.6931471805599453f + logf(l_run);
             g += n_tiles;
         }
         if (lane == 0) bulk_wait_read0();                      // this warp's tile stores have read their slab
@@ -562,8 +562,9 @@ int run(const Params& p, const void* q, const void* k, const void* v, const int3
 {
     CUtensorMap tq, tk, tv, to;
     const int BHK = p.B * p.H, BH = BHK * p.G;                 // key/value heads, query heads
-    if (!make_map(&tq, q, BH, p.T, D, BM) || !make_map(&tk, k, BHK, p.T, D, BN) || !make_map(&tv, v, BHK, p.T, D, BN) ||
-        !make_map(&to, o, BH, p.T, D, 32))
+    const int Tq = p.T - p.qoff;                               // query rows (the whole sequence unless a chunk is prefilled)
+    if (!make_map(&tq, q, BH, Tq, D, BM) || !make_map(&tk, k, BHK, p.T, D, BN) || !make_map(&tv, v, BHK, p.T, D, BN) ||
+        !make_map(&to, o, BH, Tq, D, 32))
         return LTE_ERR_CUDA;
     static int slots = 0;                                      // resident CTAs: two per SM
     if (slots == 0) {
@@ -576,11 +577,11 @@ int run(const Params& p, const void* q, const void* k, const void* v, const int3
             return LTE_ERR_CUDA;
         slots = 2 * sms;
     }
-    const int n_qt = (p.T + BM - 1) / BM, n_items = n_qt * BH;
+    const int n_qt = (Tq + BM - 1) / BM, n_items = n_qt * BH;
     const int grid = n_items < slots ? n_items : slots;
     return cuda_status(launch_pdl(prefill_tc_kernel<D>, dim3(grid), dim3(NTHREADS), Smem<D>::BYTES, st, tq, tk, tv, to, (const __nv_bfloat16*)k,
                                                                  (const __nv_bfloat16*)v, idx, cnt,
-                                                                 lse, p.T, p.W, p.R, p.scale, n_qt, BH, p.G));
+                                                                 lse, p.T, p.W, p.R, p.scale, n_qt, BH, p.G, p.qoff));
 }
 
 }  // namespace

@@ -77,7 +77,7 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                   const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO, const __nv_bfloat16* __restrict__ kg,
                   const __nv_bfloat16* __restrict__ vg, const int32_t* __restrict__ idx,
                   const int32_t* __restrict__ cnt, __nv_bfloat16* __restrict__ o, float* __restrict__ lse, int Tlen,
-                  int W, int R, float scale, int G)
+                  int W, int R, float scale, int G, int qoff)
 {
     using S = Smem<D>;
     constexpr int SUB = S::SUB, KST = S::KST, VST = S::VST;
@@ -107,7 +107,7 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     if (tid < 64) prof_[tid] = 0ull;
 #endif
     const int bh = blockIdx.y, bhk = bh / G;                   // query head and its key/value head (the G query heads of one are adjacent)
-    const int i0 = blockIdx.x * BM;
+    const int i0 = qoff + blockIdx.x * BM;                     // positions; the query tensors start at position qoff
     const int i_hi = min(i0 + BM - 1, Tlen - 1);
     const int j_start = max(i0 - W + 1, 0);
     const int n_win = (i_hi - j_start + 1 + BN - 1) / BN;
@@ -156,7 +156,7 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             //      stage's previous tile has completed (bar_kf / bar_vf, one phase per use of a stage)
             mbar_expect_tx(bar_q, S::QTILE);
 #pragma unroll
-            for (int sb = 0; sb < SUB; ++sb) tma_load_3d(sQ + sb * 16384, &tmQ, sb * 64, i0, bh, bar_q);
+            for (int sb = 0; sb < SUB; ++sb) tma_load_3d(sQ + sb * 16384, &tmQ, sb * 64, i0 - qoff, bh, bar_q);
             int ks = 0, vs = 0;                                // stage of the next K / V tile to load
             uint32_t kf_par = 0, vf_par = 0;                   // parity bit per stage of the "free" barriers
             int tk = 0, tv = 0;                                // next window tile to load
@@ -532,11 +532,11 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         __syncwarp();
         if (lane == 0 && i0 + warp * 32 < Tlen) {
 #pragma unroll
-            for (int sb = 0; sb < SUB; ++sb) tma_store_3d(&tmO, sQ + sb * 16384 + warp * 4096, sb * 64, i0 + warp * 32, bh);
+            for (int sb = 0; sb < SUB; ++sb) tma_store_3d(&tmO, sQ + sb * 16384 + warp * 4096, sb * 64, i0 - qoff + warp * 32, bh);
             bulk_commit();
             bulk_wait_read0();                                 // the buffer is released with the CTA
         }
-        if (i < Tlen) lse[(size_t)bh * Tlen + i] = m_run * 0.6931471805599453f + logf(l_run);
+        if (i < Tlen) lse[(size_t)bh * (Tlen - qoff) + (i - qoff)] = m_run * 0.6931471805599453f + logf(l_run);
         PLM(13);
         PLM_FLUSH(0, 14);
     }
@@ -551,8 +551,9 @@ int run(const Params& p, const void* q, const void* k, const void* v, const int3
 {
     CUtensorMap tq, tk, tv, to;
     const int BHK = p.B * p.H, BH = BHK * p.G;                 // key/value heads, query heads
-    if (!make_map(&tq, q, BH, p.T, D, BM) || !make_map(&tk, k, BHK, p.T, D, BN) || !make_map(&tv, v, BHK, p.T, D, BN) ||
-        !make_map(&to, o, BH, p.T, D, 32))
+    const int Tq = p.T - p.qoff;                               // query rows
+    if (!make_map(&tq, q, BH, Tq, D, BM) || !make_map(&tk, k, BHK, p.T, D, BN) || !make_map(&tv, v, BHK, p.T, D, BN) ||
+        !make_map(&to, o, BH, Tq, D, 32))
         return LTE_ERR_CUDA;
     static bool attr_done = false;
     if (!attr_done) {
@@ -561,10 +562,10 @@ int run(const Params& p, const void* q, const void* k, const void* v, const int3
             return LTE_ERR_CUDA;
         attr_done = true;
     }
-    dim3 grid((p.T + BM - 1) / BM, BH);
+    dim3 grid((Tq + BM - 1) / BM, BH);
     return cuda_status(launch_pdl(prefill_long_kernel<D>, grid, dim3(NTHREADS), Smem<D>::BYTES, st, tq, tk, tv, to, (const __nv_bfloat16*)k,
                                                                  (const __nv_bfloat16*)v, idx, cnt, (__nv_bfloat16*)o,
-                                                                 lse, p.T, p.W, p.R, p.scale, p.G));
+                                                                 lse, p.T, p.W, p.R, p.scale, p.G, p.qoff));
 }
 
 }  // namespace

@@ -122,6 +122,63 @@ def test_stack_in_decode(dtype, d, W, R, T0, steps, period):
         assert np.array_equal(pool, pidx[b, h, :pcnt[b, h]])
 
 
+@pytest.mark.parametrize("dtype,d,W,R,T0,dec,Tc", [("bf16", 64, 32, 24, 100, 20, 90), ("f32", 32, 24, 12, 0, 0, 70), ("bf16", 64, 64, 40, 30, 50, 200)])
+def test_stack_in_chunked_prefill(dtype, d, W, R, T0, dec, Tc):
+    """Prefill with the stack, decode with lazy scoring, then a chunk on top of the cache: ring tokens the lazy scoring has
+    not reached are scored with the chunk as right context; outputs equal the oracle's chunk-end reading on the stack's
+    logits, and decode steps continue from the cache the chunk leaves."""
+    cfg = synth.Config("stackchunk", dtype, 2, 2, d, 0, W, R, 7, 0.1)
+    n0, Ttot = T0 + dec, T0 + dec + Tc + 8
+    x = synth.make(cfg, 6, T=Ttot)
+    wl, wout, bl, bout = _stack_params(cfg.H, d, 6, True)
+    t = lambda a: torch.from_numpy(a).cuda()
+    c = lte.conv_stack([t(w) for w in wl], t(wout), [t(b) for b in bl], t(bout))
+    q, k, v = (dev(x[n], dtype) for n in "qkv")
+    s0 = shape_of(cfg, T=T0, B=cfg.B)
+    if T0 > 0:
+        kp, vp = k[:, :, :T0].contiguous(), v[:, :, :T0].contiguous()
+        z = lte.lte_scores(s0, c, kp, vp)
+        idx, cnt = lte.lte_select(s0, z)
+        cache = lte.lte_cache_init(s0, c, kp, vp, z, idx, cnt)
+    else:
+        cache = lte.lte_cache_init(s0, c)
+    period = W - 13
+    for i, n in enumerate(range(T0, n0)):
+        if i % period == 0:
+            lte.lte_cache_score(s0, c, cache)
+        lte.lte_attn_decode(s0, c, cache, q[:, :, n].contiguous(), k[:, :, n].contiguous(), v[:, :, n].contiguous())
+    sc = shape_of(cfg, T=Tc, B=cfg.B)
+    o, l = lte.lte_attn_prefill_chunk(sc, c, cache, n0, q[:, :, n0:n0 + Tc].contiguous(), k[:, :, n0:n0 + Tc].contiguous(),
+                                      v[:, :, n0:n0 + Tc].contiguous())
+    outs, lses = [], []
+    for i, n in enumerate(range(n0 + Tc, Ttot)):
+        if i % period == 0:
+            lte.lte_cache_score(s0, c, cache)
+        o1, l1 = lte.lte_attn_decode(s0, c, cache, q[:, :, n].contiguous(), k[:, :, n].contiguous(), v[:, :, n].contiguous())
+        outs.append(o1.float().cpu().numpy()); lses.append(l1.cpu().numpy())
+    torch.cuda.synchronize()
+    assert lte.lib().lte_device_status() == 0
+    z64 = orc.scores_stack(x["k"], x["v"], wl, bl, wout, bout)
+    if n0 > 0:
+        p_idx, p_cnt, _ = orc.select(z64[:, :, :n0], W, R)
+    else:
+        p_idx, p_cnt = np.full((cfg.B, cfg.H, R), -1, np.int32), np.zeros((cfg.B, cfg.H), np.int32)
+    n1 = n0 + Tc
+    o64, l64, _, _ = orc.prefill_chunk(x["q"][:, :, :n1], x["k"][:, :, :n1], x["v"][:, :, :n1], z64, n0, W, R, p_idx, p_cnt)
+    tol = 2e-2 if dtype == "bf16" else 1e-4
+    assert np.max(np.abs(o.float().cpu().numpy() - o64)) <= tol
+    assert np.max(np.abs(l.cpu().numpy() - l64)) <= tol
+    od, ld, pidx, pcnt = orc.stream(x["q"], x["k"], x["v"], z64, W, R, 0, n_from=n1)
+    assert np.max(np.abs(np.stack(outs, axis=2) - od)) <= tol
+    assert np.max(np.abs(np.stack(lses, axis=2) - ld)) <= tol
+    from tests.test_gpu_decode import _read_pool
+    pools, ns = _read_pool(cache, cfg, cfg.B)
+    assert all(n == Ttot for n in ns)
+    for bh, pool in enumerate(pools):
+        b, h = divmod(bh, cfg.H)
+        assert np.array_equal(pool, pidx[b, h, :pcnt[b, h]])
+
+
 # ---- backward through the stack (lte_attn_bwd with the three-layer scorer) ---------------------------------------------
 def _rel(a, b):
     return float(np.linalg.norm(np.asarray(a, np.float64) - b) / (np.linalg.norm(b) + 1e-30))
