@@ -108,3 +108,32 @@ def test_three_layer_stack_and_groups_host_side():
     assert L.lte_attn_prefill(a(neg), fake, fake, fake, fake, fake, fake, fake, None, 0, None) == -1
     # the shape struct ends with the group field (the binding and the header agree on the layout)
     assert ctypes.sizeof(lte.LteShape) == 11 * 4 and lte.LteShape.group.offset == 40
+
+
+def test_chunked_prefill_host_side():
+    """Workspace size and argument checks of lte_attn_prefill_chunk (validation fails before anything is launched)."""
+    L = lte.lib()
+    a = ctypes.addressof
+    fake = 4096
+    single = lte.LteConv(1, 7, 1, 256, 0)
+    s = lte.shape(4, 16, 1024, 64, 128, 128, lte.BF16)
+    ws = lte.lte_workspace_bytes(lte.OP_CHUNK, s, single)
+    rows = 128 + 128 + 1024                                                   # pool + ring + chunk: the longest local sequence
+    assert ws >= 2 * 64 * rows * 64 * 2 + 2 * 64 * rows * 4                   # its keys and values, two logit arrays
+    assert ws % 256 == 0
+    stack = lte.LteConv(3, 3, 2, 256, 0)
+    assert lte.lte_workspace_bytes(lte.OP_CHUNK, s, stack) >= ws + 16 * 194176   # plus the stack's weight image
+    assert lte.lte_workspace_bytes(lte.OP_CHUNK, s, None) == 0
+    ok = [a(s), a(single), fake, 0, fake, fake, fake, fake, fake, fake, 1 << 40, None]
+    def call(**kw):
+        args = list(ok)
+        for i, v in kw.items():
+            args[int(i[1:])] = v
+        return L.lte_attn_prefill_chunk(*args)
+    assert call(_2=None) == -1                                                 # no cache
+    assert call(_3=-1) == -1                                                   # negative token count
+    assert call(_4=None) == -1 and call(_7=None) == -1 and call(_8=None) == -1
+    assert call(_4=fake + 2) == -1                                             # misaligned q
+    assert call(_9=None) == -3 and call(_10=16) == -3 and call(_9=fake + 16) == -3
+    assert call(_1=a(lte.LteConv(1, 6, 1, 256, 0))) == -1                      # even tap count
+    assert call(_0=a(lte.shape(4, 16, 0, 64, 128, 128, lte.BF16))) == -1       # empty chunk
