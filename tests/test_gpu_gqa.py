@@ -45,7 +45,9 @@ def test_prefill_gqa(dtype, d, T, W, R, G):
 
 
 @pytest.mark.parametrize("dtype,d,W,R,G,T0,steps", [("bf16", 64, 32, 24, 4, 100, 40), ("bf16", 64, 16, 8, 2, 0, 60), ("bf16", 128, 24, 16, 4, 64, 30),
-                                                    ("f32", 32, 16, 12, 3, 40, 30), ("bf16", 64, 200, 150, 2, 260, 20)])
+                                                    ("f32", 32, 16, 12, 3, 40, 30), ("bf16", 64, 200, 150, 2, 260, 20),
+                                                    # few heads, long blocks: a cluster of blocks shares a head (2 x 320, 4 x 260 rows), 5 query heads = two passes
+                                                    ("bf16", 64, 384, 256, 5, 700, 12), ("f32", 32, 600, 440, 2, 1300, 8), ("bf16", 128, 300, 220, 6, 10, 14)])
 def test_decode_gqa(dtype, d, W, R, G, T0, steps):
     cfg = synth.Config("gqa", dtype, 2, 2, d, T0 + steps, W, R, 7, 0.1)
     Ttot = T0 + steps
