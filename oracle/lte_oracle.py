@@ -188,6 +188,36 @@ def prefill_chunk(q, k, v, z, n0, W, R, pool_idx, pool_cnt, sink=0, tau=0.5, sca
     return o, lse, idx, cnt
 
 
+def sparsity_stats(z, lam=None, tau=0.5):
+    """Eq. 7 and the retention count it is steered by: count[h] = mean over the batch of #{i : r_i > tau} per sequence,
+    penalty = sum_h lam[h] sum_{b,i} ReLU(r_i - tau), r = sigmoid(z), over the scored positions (z > -inf)."""
+    z = _f64(z)
+    B, H, T = z.shape
+    r = 1.0 / (1.0 + np.exp(-z))                       # sigmoid(-inf) = 0: unscored positions drop out of both sums
+    count = (r > tau).sum(axis=2).mean(axis=0)
+    pen = np.maximum(r - tau, 0.0).sum(axis=(0, 2))
+    lam = np.ones(H) if lam is None else _f64(lam)
+    return count, float((lam * pen).sum())
+
+
+def lambda_update(lam, cbar, count, step, u=32, cap=512.0, alpha=1.2, band=0.95, lam_floor=1e-9, lam_max=1.0):
+    """One step of Algorithm 1's feedback loop for the penalty weights (arrays over heads, returned as new arrays).
+    Every step: cbar <- (1 - a) cbar + a count with a = 2 / (1 + u / 2) (the new sample takes the weight a: the
+    listing prints the two weights the other way round, which would freeze cbar).  Every u-th step (step mod u == 0):
+    lam <- lam alpha^s with s = [cbar > cap] - [cbar < band cap]; lam <- min(lam, lam_max); lam below lam_floor -> 0;
+    a head whose cbar exceeds the cap with lam = 0 is re-enabled at lam_floor."""
+    lam, cbar, count = _f64(lam).copy(), _f64(cbar).copy(), _f64(count)
+    a = 2.0 / (1.0 + u / 2.0)
+    cbar = (1.0 - a) * cbar + a * count
+    if step % u == 0:
+        s = (cbar > cap).astype(np.float64) - (cbar < band * cap).astype(np.float64)
+        lam = lam * np.power(alpha, s)
+        lam = np.minimum(lam, lam_max)
+        lam[lam < lam_floor] = 0.0
+        lam[(cbar > cap) & (lam == 0.0)] = lam_floor
+    return lam, cbar
+
+
 def stream(q, k, v, z, W, R, sink=0, tau=0.5, scale=None, n_from=0):
     """Token-by-token simulation from an empty cache; outputs for steps >= n_from
     and the final pool (ascending positions)."""
