@@ -76,7 +76,7 @@ typedef struct lte_conv {
  */
 
 typedef enum lte_op {
-    LTE_OP_SCORES = 0, LTE_OP_SELECT = 1, LTE_OP_PREFILL = 2, LTE_OP_DECODE = 3, LTE_OP_BWD = 4, LTE_OP_CHUNK = 5
+    LTE_OP_SCORES = 0, LTE_OP_SELECT = 1, LTE_OP_PREFILL = 2, LTE_OP_DECODE = 3, LTE_OP_BWD = 4, LTE_OP_CHUNK = 5, LTE_OP_STATS = 6
 } lte_op;
 
 /* Bytes of caller-supplied scratch the given entry point needs for this shape (0 if none). */
@@ -219,6 +219,36 @@ int lte_cache_score(const lte_shape* s, const lte_conv* c, void* cache, void* ws
 int lte_attn_prefill_chunk(const lte_shape* s, const lte_conv* c, void* cache, int32_t n_past,
                            const void* q, const void* k, const void* v, void* o, float* lse,
                            void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Training-side statistics of the scorer (Section 3.1.2, Eq. 7, and the retention count that Algorithm 1 steers):
+ *   count[h]  = mean over the batch of #{i : r_i > tau} per sequence          (r = sigmoid(z); the test is z > logit(tau))
+ *   penalty   = sum_h lambda[h] sum_{b,i} ReLU(r_i - tau)                     (lambda = 1 when NULL)
+ * over the scored positions (z > -inf).  The gradient of the penalty is what lte_attn_bwd adds when given lambda.
+ *   z        in   [B,H,T] fp32 device;   lambda_or_null in [H] fp32 device
+ *   count    out  [H] fp32 device;       penalty out [1] fp32 device
+ *   ws       device scratch of lte_workspace_bytes(LTE_OP_STATS, s, NULL) bytes, 16-byte aligned
+ * Fixed summation order (no floating-point atomics).  Errors: INVALID_ARG, UNSUPPORTED (H > 8192), WORKSPACE, CUDA.
+ */
+int lte_sparsity_stats(const lte_shape* s, const float* z, const float* lambda_or_null, float* count, float* penalty,
+                       void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * The feedback loop for the penalty weights (Algorithm 1), one call per training step, on HOST arrays of n entries
+ * (heads, or layers x heads).  Every call: cbar <- (1 - a) cbar + a count with a = 2 / (1 + period / 2) (the weight of
+ * the new sample; the listing prints the two weights the other way round).  When step is a multiple of period:
+ * lambda <- lambda alpha if cbar > cap, lambda / alpha if cbar < band cap; lambda <- min(lambda, max); lambda below
+ * floor -> 0; cbar > cap with lambda = 0 -> floor.  The listing leaves alpha undefined: 1.2 by default.
+ * With several ranks the caller averages `count` (or cbar) over the ranks first, so that every rank takes the same
+ * decision ("synchronize" in the listing).  cfg = NULL: period 32, cap 512, alpha 1.2, band 0.95, floor 1e-9, max 1.
+ * Pure host arithmetic: no CUDA call, usable without a GPU.  Errors: INVALID_ARG.
+ */
+typedef struct lte_lambda_cfg {
+    int32_t period;                /* u: steps between adjustments                       */
+    float cap, alpha, band;        /* retention cap b, adjustment factor, lower band     */
+    float floor, max;              /* smallest non-zero weight, upper clamp              */
+} lte_lambda_cfg;
+int lte_lambda_update(int32_t n, float* lambda, float* cbar, const float* count, int64_t step, const lte_lambda_cfg* cfg);
 
 /*
  * Backward of lte_attn_prefill with the straight-through surrogate (Section 3.1.2):

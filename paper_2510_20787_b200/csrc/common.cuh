@@ -111,6 +111,8 @@ int launch_chunk_merge_z(const Params& p, float* z, float* zrank, const float* z
 int launch_chunk_commit(const Params& p, void* cache, const void* klin, const void* vlin, const float* z, const int32_t* idx,
                         const int32_t* cnt, const int32_t* oldpos, int n0, int n1, int R0, int Wn, cudaStream_t st);
 int chunk_status_fetch_and_clear();
+int launch_sparsity_stats(const Params& p, const float* z, const float* lambda, float* count, float* penalty, float* part, float tau,
+                          cudaStream_t st);
 int launch_decode_tc(const Params& p, void* cache, const void* q1, const void* k1, const void* v1, void* o1,
                      float* lse1, cudaStream_t st);
 int launch_decode(const Params& p, void* cache, const void* q1, const void* k1, const void* v1, void* o1,

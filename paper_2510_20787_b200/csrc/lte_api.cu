@@ -170,6 +170,10 @@ size_t lte_workspace_bytes(int op, const lte_shape* s, const lte_conv* c)
         if (check_shape(s, false) != LTE_OK) return 0;
         return cache_score_plan(s, c).total;
     }
+    if (op == LTE_OP_STATS) {
+        if (check_shape(s, true) != LTE_OK) return 0;
+        return ((size_t)s->B * s->H * 2 * sizeof(float) + 255) / 256 * 256;
+    }
     if (op == LTE_OP_CHUNK) {
         if (check_shape(s, true) != LTE_OK || !c) return 0;
         if ((double)s->B * s->H * (s->group > 1 ? s->group : 1) * ((double)s->R + s->W + s->T) * s->d > 2.0e10) return 0;
@@ -316,6 +320,42 @@ int lte_attn_decode(const lte_shape* s, const lte_conv* c, void* cache, const vo
     if (!aligned16(cache) || !aligned16(q1) || !aligned16(k1) || !aligned16(v1)) return LTE_ERR_INVALID_ARG;
     e = check_arch(); if (e) return e;
     return launch_decode(make_params(s, c), cache, q1, k1, v1, o1, lse1, (cudaStream_t)stream);
+}
+
+int lte_sparsity_stats(const lte_shape* s, const float* z, const float* lambda_or_null, float* count, float* penalty,
+                       void* ws, size_t ws_bytes, void* stream)
+{
+    int e = check_shape(s, true); if (e) return e;
+    if (!z || !count || !penalty) return LTE_ERR_INVALID_ARG;
+    if (s->H > 8192) return LTE_ERR_UNSUPPORTED;
+    if (!ws || ((uintptr_t)ws & 15u) != 0 || ws_bytes < (size_t)s->B * s->H * 2 * sizeof(float)) return LTE_ERR_WORKSPACE;
+    e = check_arch(); if (e) return e;
+    return launch_sparsity_stats(make_params(s, nullptr), z, lambda_or_null, count, penalty, (float*)ws, s->tau, (cudaStream_t)stream);
+}
+
+int lte_lambda_update(int32_t n, float* lambda, float* cbar, const float* count, int64_t step, const lte_lambda_cfg* cfg)
+{
+    if (n < 0 || (n > 0 && (!lambda || !cbar || !count)) || step < 0) return LTE_ERR_INVALID_ARG;
+    lte_lambda_cfg d;
+    d.period = 32; d.cap = 512.f; d.alpha = 1.2f; d.band = 0.95f; d.floor = 1e-9f; d.max = 1.f;
+    if (cfg) d = *cfg;
+    if (d.period <= 0 || !(d.alpha > 1.f) || !(d.cap > 0.f) || !(d.band > 0.f && d.band <= 1.f) || !(d.floor > 0.f) || !(d.max >= d.floor))
+        return LTE_ERR_INVALID_ARG;
+    const double a = 2.0 / (1.0 + d.period / 2.0);          // the new sample's weight in the moving average
+    const bool adjust = step % d.period == 0;
+    for (int32_t i = 0; i < n; ++i) {
+        const double cb = (1.0 - a) * (double)cbar[i] + a * (double)count[i];
+        cbar[i] = (float)cb;
+        if (!adjust) continue;
+        double l = lambda[i];
+        if (cb > d.cap) l *= d.alpha;
+        else if (cb < (double)d.band * d.cap) l /= d.alpha;
+        if (l > d.max) l = d.max;
+        if (l < d.floor) l = 0.0;
+        if (cb > d.cap && l == 0.0) l = d.floor;
+        lambda[i] = (float)l;
+    }
+    return LTE_OK;
 }
 
 int lte_attn_bwd(const lte_shape* s, const lte_conv* c, const void* q, const void* k, const void* v, const void* o,

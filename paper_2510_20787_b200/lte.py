@@ -15,11 +15,12 @@ LIB_PATH = os.path.join(_HERE, "liblte.so")
 _lib = None
 
 F32, BF16 = 0, 1
-OP_SCORES, OP_SELECT, OP_PREFILL, OP_DECODE, OP_BWD, OP_CHUNK = range(6)
+OP_SCORES, OP_SELECT, OP_PREFILL, OP_DECODE, OP_BWD, OP_CHUNK, OP_STATS = range(7)
 BWD_CNN_INPUT_GRAD = 1
 
 EXPORTS = ["lte_device_status", "lte_workspace_bytes", "lte_strerror", "lte_scores", "lte_select", "lte_cache_score", "lte_attn_prefill",
-           "lte_cache_bytes", "lte_cache_init", "lte_attn_decode", "lte_attn_prefill_chunk", "lte_attn_bwd", "lte_attn_bwd_static"]
+           "lte_cache_bytes", "lte_cache_init", "lte_attn_decode", "lte_attn_prefill_chunk", "lte_attn_bwd", "lte_attn_bwd_static",
+           "lte_sparsity_stats", "lte_lambda_update"]
 STATIC_SCRATCH_BYTES = 8 << 20
 
 
@@ -63,6 +64,8 @@ def lib():
         L.lte_cache_init.argtypes = [vp] * 9
         L.lte_attn_decode.argtypes = [vp] * 9
         L.lte_cache_score.argtypes = [vp] * 4 + [ctypes.c_size_t, vp]
+        L.lte_sparsity_stats.argtypes = [vp] * 6 + [ctypes.c_size_t, vp]
+        L.lte_lambda_update.argtypes = [ctypes.c_int32, vp, vp, vp, ctypes.c_int64, vp]
         L.lte_attn_prefill_chunk.argtypes = [vp] * 3 + [ctypes.c_int32] + [vp] * 6 + [ctypes.c_size_t, vp]
         L.lte_attn_bwd.argtypes = [vp] * 17 + [ctypes.c_uint32, vp, ctypes.c_size_t, vp]
         L.lte_attn_bwd_static.argtypes = [vp] * 17 + [ctypes.c_uint32, vp]
@@ -220,6 +223,36 @@ def lte_attn_prefill_chunk(s, c, cache, n_past, q, k, v, o=None, lse=None, ws=No
                                                                   _ptr(o), _ptr(lse, torch.float32), _ptr(ws), ws.numel(),
                                                                   _stream()))
     return o, lse
+
+
+class LteLambdaCfg(ctypes.Structure):
+    _fields_ = [("period", ctypes.c_int32), ("cap", ctypes.c_float), ("alpha", ctypes.c_float), ("band", ctypes.c_float),
+                ("floor", ctypes.c_float), ("max", ctypes.c_float)]
+
+
+def lte_sparsity_stats(s, z, lam=None, ws=None):
+    """Eq. 7 statistics: z [B,H,T] -> count [H] (batch mean of tokens above the threshold), penalty [1]."""
+    count = torch.empty((s.H,), dtype=torch.float32, device=z.device)
+    penalty = torch.empty((1,), dtype=torch.float32, device=z.device)
+    if ws is None:
+        ws = torch.empty(max(lte_workspace_bytes(OP_STATS, s, None), 256), dtype=torch.uint8, device=z.device)
+    _check("lte_sparsity_stats", lib().lte_sparsity_stats(ctypes.addressof(s), _ptr(z, torch.float32), _ptr(lam, torch.float32),
+                                                          _ptr(count), _ptr(penalty), _ptr(ws), ws.numel(), _stream()))
+    return count, penalty
+
+
+def lte_lambda_update(lam, cbar, count, step, cfg=None, group=None):
+    """Algorithm 1's feedback step on host tensors (float32, contiguous, updated in place).  When torch.distributed is
+    initialised the counts are averaged over the ranks of `group` first, so that all ranks take the same decision."""
+    import torch.distributed as dist
+    assert lam.device.type == "cpu" and cbar.device.type == "cpu" and lam.dtype == torch.float32 and cbar.dtype == torch.float32
+    count = count.detach().to("cpu", torch.float32).contiguous().clone()
+    if dist.is_available() and dist.is_initialized():
+        dist.all_reduce(count, group=group)
+        count /= dist.get_world_size(group)
+    _check("lte_lambda_update", lib().lte_lambda_update(lam.numel(), lam.data_ptr(), cbar.data_ptr(), count.data_ptr(), int(step),
+                                                        ctypes.addressof(cfg) if cfg is not None else None))
+    return lam, cbar
 
 
 def lte_cache_score(s, c, cache, ws=None):

@@ -137,3 +137,18 @@ def test_chunked_prefill_host_side():
     assert call(_9=None) == -3 and call(_10=16) == -3 and call(_9=fake + 16) == -3
     assert call(_1=a(lte.LteConv(1, 6, 1, 256, 0))) == -1                      # even tap count
     assert call(_0=a(lte.shape(4, 16, 0, 64, 128, 128, lte.BF16))) == -1       # empty chunk
+
+
+def test_training_pieces_host_side():
+    """Argument checks of lte_sparsity_stats (nothing is launched) and its workspace size."""
+    L = lte.lib()
+    a = ctypes.addressof
+    fake = 4096
+    s = lte.shape(8, 16, 2048, 64, 64, 64, lte.BF16)
+    assert lte.lte_workspace_bytes(lte.OP_STATS, s, None) == 8 * 16 * 2 * 4
+    assert L.lte_sparsity_stats(a(s), None, None, fake, fake, fake, 1 << 20, None) == -1
+    assert L.lte_sparsity_stats(a(s), fake, None, None, fake, fake, 1 << 20, None) == -1
+    assert L.lte_sparsity_stats(a(s), fake, None, fake, fake, None, 0, None) == -3
+    assert L.lte_sparsity_stats(a(s), fake, None, fake, fake, fake, 8, None) == -3
+    wide = lte.shape(1, 9000, 16, 64, 8, 4, lte.BF16)
+    assert L.lte_sparsity_stats(a(wide), fake, None, fake, fake, fake, 1 << 20, None) == -2
