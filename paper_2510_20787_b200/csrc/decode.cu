@@ -860,19 +860,23 @@ __global__ void __launch_bounds__(DTU) decode_update_kernel(unsigned char* __res
 }
 
 // The attend kernel: query heads g_first .. G-1 of a key/value head over its block (ring rows of the min(n, W) newest
-// tokens, cnt pool rows), after the update.  One block per key/value head, up to ATT_Q query heads per pass: logits by one thread per row (the queries in shared
-// memory, no reductions across lanes), block max and sum per query head, then the warps take the value rows in turn
-// (lanes over the d channels), weight them per query head in registers, and a reduction over the warps closes.
+// tokens, cnt pool rows), after the update.  One block (or a cluster of blocks) per key/value head, up to ATT_Q query heads
+// per pass.  Rows are spread as in the step kernels: LPR lanes share a row, each with one 16-byte piece of it, so a warp's
+// load covers whole consecutive rows; four rows per thread are in flight.  Logits: partial dots per lane against the
+// lane's slice of every query, reduced over the LPR lanes by shuffles; block maxima and sums per query head; value rows
+// the same way, weighted per query head in registers, reduced over lanes sharing a slice and then over the warps.
 constexpr int ATT_Q = 4;
 template <typename T, int D>
 __global__ void __launch_bounds__(DT) decode_attend_kernel(const unsigned char* __restrict__ cache, CacheLayout L,
                                                            const T* __restrict__ q1, T* __restrict__ o1,
                                                            float* __restrict__ lse1, int W, int G, float scale, int g_first)
 {
-    constexpr int C = D / 32, NW = DT / 32;
+    constexpr int EPV = V16<T>::N;                             // elements per 16-byte piece
+    constexpr int LPR = D / EPV;                               // lanes per row
+    constexpr int RPP = DT / LPR;                              // rows per pass of the block
+    constexpr int NW = DT / 32, UNR = 4;
     extern __shared__ float att_sm[];                          // logits [ATT_Q][rows], then partial outputs [NW][ATT_Q][D]
     __shared__ float s_red[NW][ATT_Q];
-    __shared__ __align__(16) float s_q[ATT_Q][D];              // the pass's queries, pre-scaled
     __shared__ float s_mx[ATT_Q], s_sum[ATT_Q];
     __shared__ float s_fin[ATT_Q][D];                          // this block's unnormalised outputs (read by the cluster's first block)
     // A thread-block cluster shares one key/value head: block `rank` of `nsplit` takes a contiguous share of the rows,
@@ -880,9 +884,10 @@ __global__ void __launch_bounds__(DT) decode_attend_kernel(const unsigned char* 
     cg::cluster_group cluster = cg::this_cluster();
     const int nsplit = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
     const int bh = blockIdx.x / nsplit, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const int seg = tid % LPR, rsub = tid / LPR;
     const unsigned char* blk = cache + L.header + (size_t)bh * L.stride;
-    const T* Kc = reinterpret_cast<const T*>(blk + L.off_k);
-    const T* Vc = reinterpret_cast<const T*>(blk + L.off_v);
+    const uint4* Kc = reinterpret_cast<const uint4*>(blk + L.off_k);
+    const uint4* Vc = reinterpret_cast<const uint4*>(blk + L.off_v);
     const int32_t* meta = reinterpret_cast<const int32_t*>(blk + L.off_meta);
     const int n = meta[0], cnt = meta[1];
     const int n_ring = n < W ? n : W, rows_all = n_ring + cnt;
@@ -890,72 +895,60 @@ __global__ void __launch_bounds__(DT) decode_attend_kernel(const unsigned char* 
     const int a_lo = min(rank * share, rows_all), rows = min(a_lo + share, rows_all) - a_lo;   // this block's rows: a_lo + [0, rows)
     float* s_log = att_sm;
     float* s_out = att_sm + (size_t)ATT_Q * rows;
-    // element (r, ch): in the swizzled layout (bf16, d = 64) 16-byte chunk ch / 8 of row r sits at position (ch / 8) ^ (r & 7)
-    auto pos_of = [&](int r, int ch) { return L.swz ? ((((ch >> 3) ^ (r & 7)) << 3) | (ch & 7)) : ch; };
-    // a lane owns the channel pairs (2 lane, 2 lane + 1) + 64 j: one 4- or 8-byte load per pair, a row of d = 64 per warp load
-    auto ch_of = [&](int c) { return C == 1 ? lane : 2 * lane + (c & 1) + 64 * (c >> 1); };   // d = 32: one channel per lane
-    auto load_row = [&](const T* base, int r, float (&out)[C]) {
-        if constexpr (C == 1) out[0] = to_f(base[(size_t)r * D + pos_of(r, lane)]);
-#pragma unroll
-        for (int j = 0; j < C / 2; ++j) {
-            const T* p2 = base + (size_t)r * D + pos_of(r, 2 * lane + 64 * j);
-            if constexpr (sizeof(T) == 2) {
-                const uint32_t u = *reinterpret_cast<const uint32_t*>(p2);
-                out[2 * j] = __uint_as_float(u << 16); out[2 * j + 1] = __uint_as_float(u & 0xffff0000u);
-            } else {
-                const float2 u = *reinterpret_cast<const float2*>(p2);
-                out[2 * j] = u.x; out[2 * j + 1] = u.y;
-            }
-        }
+    // this thread's piece of list entry a: cache row (ring rows first, then pool rows) and the piece's place in it (the
+    // swizzled layout permutes the pieces of a row)
+    auto piece_of = [&](int a) {
+        const int r = a_lo + a < n_ring ? a_lo + a : W + (a_lo + a - n_ring);
+        return (size_t)r * LPR + (L.swz ? (seg ^ (r & 7)) : seg);
     };
     for (int g0 = g_first; g0 < G; g0 += ATT_Q) {
         const int nq = G - g0 < ATT_Q ? G - g0 : ATT_Q;
-        float qv[ATT_Q][C];
+        float qv[ATT_Q][EPV];                                  // this lane's slice of the pass's queries, pre-scaled
 #pragma unroll
         for (int u = 0; u < ATT_Q; ++u)
 #pragma unroll
-            for (int c = 0; c < C; ++c)
-                qv[u][c] = u < nq ? to_f(q1[((size_t)bh * G + g0 + u) * D + ch_of(c)]) * scale : 0.f;
-        // ---- logits: a thread takes whole rows (no reductions across lanes), the queries come from shared memory ----
-        __syncthreads();                                       // s_q of the previous pass has been read
-#pragma unroll
-        for (int u = 0; u < ATT_Q; ++u)
-#pragma unroll
-            for (int c = 0; c < C; ++c) s_q[u][ch_of(c)] = qv[u][c];
-        __syncthreads();
+            for (int e = 0; e < EPV; ++e)
+                qv[u][e] = u < nq ? to_f(q1[((size_t)bh * G + g0 + u) * D + seg * EPV + e]) * scale : 0.f;
+        // ---- logits ----
         float mx[ATT_Q];
 #pragma unroll
         for (int u = 0; u < ATT_Q; ++u) mx[u] = -INFINITY;
-        for (int a = tid; a < rows; a += DT) {
-            const int r = a_lo + a < n_ring ? a_lo + a : W + (a_lo + a - n_ring);
-            constexpr int EPV = 16 / sizeof(T);                // elements per 16-byte vector
-            float dot[ATT_Q];
+        for (int a0 = 0; a0 < rows; a0 += UNR * RPP) {         // uniform trip count: the shuffles need every lane
+            uint4 raw[UNR];
 #pragma unroll
-            for (int u = 0; u < ATT_Q; ++u) dot[u] = 0.f;
-#pragma unroll 2
-            for (int cv = 0; cv < D / EPV; ++cv) {             // (deeper unrolling measured slower: 43 us against 36 us per step)
-                const int pos = L.swz ? (cv ^ (r & 7)) : cv;
-                const uint4 raw = *reinterpret_cast<const uint4*>(Kc + (size_t)r * D + pos * EPV);
+            for (int j = 0; j < UNR; ++j) {
+                const int a = a0 + j * RPP + rsub;
+                raw[j] = a < rows ? Kc[piece_of(a)] : make_uint4(0, 0, 0, 0);
+            }
+            float dot[UNR][ATT_Q];
+#pragma unroll
+            for (int j = 0; j < UNR; ++j) {
                 float kf[EPV];
-                if constexpr (sizeof(T) == 2) {
-                    const uint32_t wv[4] = {raw.x, raw.y, raw.z, raw.w};
+                unpack<T>(raw[j], kf);
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) { kf[2 * e] = __uint_as_float(wv[e] << 16); kf[2 * e + 1] = __uint_as_float(wv[e] & 0xffff0000u); }
-                } else {
-                    kf[0] = __uint_as_float(raw.x); kf[1] = __uint_as_float(raw.y); kf[2] = __uint_as_float(raw.z); kf[3] = __uint_as_float(raw.w);
+                for (int u = 0; u < ATT_Q; ++u) {
+                    float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+                    for (int e = 0; e < EPV; e += 2) { s0 = fmaf(qv[u][e], kf[e], s0); s1 = fmaf(qv[u][e + 1], kf[e + 1], s1); }
+                    dot[j][u] = s0 + s1;
                 }
-#pragma unroll
-                for (int u = 0; u < ATT_Q; ++u)
-#pragma unroll
-                    for (int e = 0; e < EPV; e += 4) {
-                        const float4 q4 = *reinterpret_cast<const float4*>(&s_q[u][cv * EPV + e]);
-                        dot[u] = fmaf(kf[e], q4.x, fmaf(kf[e + 1], q4.y, fmaf(kf[e + 2], q4.z, fmaf(kf[e + 3], q4.w, dot[u]))));
-                    }
             }
 #pragma unroll
-            for (int u = 0; u < ATT_Q; ++u) {
-                mx[u] = fmaxf(mx[u], dot[u]);
-                s_log[(size_t)u * rows + a] = dot[u];
+            for (int o = LPR / 2; o > 0; o >>= 1)
+#pragma unroll
+                for (int j = 0; j < UNR; ++j)
+#pragma unroll
+                    for (int u = 0; u < ATT_Q; ++u) dot[j][u] += __shfl_xor_sync(0xffffffffu, dot[j][u], o);
+#pragma unroll
+            for (int j = 0; j < UNR; ++j) {
+                const int a = a0 + j * RPP + rsub;
+                if (a < rows) {
+#pragma unroll
+                    for (int u = 0; u < ATT_Q; ++u) {
+                        mx[u] = fmaxf(mx[u], dot[j][u]);
+                        if (seg == u % LPR) s_log[(size_t)u * rows + a] = dot[j][u];   // (the LPR lanes hold the same sums: spread the stores)
+                    }
+                }
             }
         }
 #pragma unroll
@@ -977,7 +970,7 @@ __global__ void __launch_bounds__(DT) decode_attend_kernel(const unsigned char* 
             ps[u] = 0.f;
             const float m = s_mx[u];
             for (int a = tid; a < rows; a += DT) {
-                const float pj = expf(s_log[(size_t)u * rows + a] - m);
+                const float pj = __expf(s_log[(size_t)u * rows + a] - m);
                 s_log[(size_t)u * rows + a] = pj;
                 ps[u] += pj;
             }
@@ -993,26 +986,44 @@ __global__ void __launch_bounds__(DT) decode_attend_kernel(const unsigned char* 
             s_sum[tid] = t;
         }
         // ---- weighted value rows ----
-        float acc[ATT_Q][C];
+        float acc[ATT_Q][EPV];
 #pragma unroll
         for (int u = 0; u < ATT_Q; ++u)
 #pragma unroll
-            for (int c = 0; c < C; ++c) acc[u][c] = 0.f;
-        for (int a = wid; a < rows; a += NW) {
-            const int r = a_lo + a < n_ring ? a_lo + a : W + (a_lo + a - n_ring);
-            float vv[C];
-            load_row(Vc, r, vv);
+            for (int e = 0; e < EPV; ++e) acc[u][e] = 0.f;
+        for (int a0 = 0; a0 < rows; a0 += UNR * RPP) {
+            uint4 raw[UNR];
 #pragma unroll
-            for (int u = 0; u < ATT_Q; ++u) {
-                const float pj = s_log[(size_t)u * rows + a];
+            for (int j = 0; j < UNR; ++j) {
+                const int a = a0 + j * RPP + rsub;
+                raw[j] = a < rows ? Vc[piece_of(a)] : make_uint4(0, 0, 0, 0);
+            }
 #pragma unroll
-                for (int c = 0; c < C; ++c) acc[u][c] = fmaf(pj, vv[c], acc[u][c]);
+            for (int j = 0; j < UNR; ++j) {
+                const int a = min(a0 + j * RPP + rsub, rows - 1);   // (rows past the end carry zero values)
+                float vf[EPV];
+                unpack<T>(raw[j], vf);
+#pragma unroll
+                for (int u = 0; u < ATT_Q; ++u) {
+                    const float pj = s_log[(size_t)u * rows + a];
+#pragma unroll
+                    for (int e = 0; e < EPV; ++e) acc[u][e] = fmaf(pj, vf[e], acc[u][e]);
+                }
             }
         }
+        // lanes that share a slice of the row (same seg) add up, then the warps
 #pragma unroll
-        for (int u = 0; u < ATT_Q; ++u)
+        for (int o = 16; o >= LPR; o >>= 1)
 #pragma unroll
-            for (int c = 0; c < C; ++c) s_out[((size_t)wid * ATT_Q + u) * D + ch_of(c)] = acc[u][c];
+            for (int u = 0; u < ATT_Q; ++u)
+#pragma unroll
+                for (int e = 0; e < EPV; ++e) acc[u][e] += __shfl_xor_sync(0xffffffffu, acc[u][e], o);
+        if (lane < LPR) {
+#pragma unroll
+            for (int u = 0; u < ATT_Q; ++u)
+#pragma unroll
+                for (int e = 0; e < EPV; ++e) s_out[((size_t)wid * ATT_Q + u) * D + lane * EPV + e] = acc[u][e];
+        }
         __syncthreads();
         for (int e = tid; e < nq * D; e += DT) {
             const int u = e / D, ch = e - u * D;
@@ -1145,7 +1156,7 @@ int launch_decode(const Params& p, void* cache, const void* q1, const void* k1, 
     if (cudaGetLastError() != cudaSuccess) return LTE_ERR_CUDA;
     const size_t att_smem = sizeof(float) * ((size_t)ATT_Q * (p.W + p.R) + (size_t)(DT / 32) * ATT_Q * p.d);
     // blocks per key/value head (a cluster): more than one only while there are fewer blocks than SMs and a share keeps 256 rows
-    // (with 256 heads of 1280 rows, four blocks per head measured 41 us per step against 36 us for one)
+    // (with 256 heads of 1280 rows, two blocks per head measured 41 us per step against 29 us for one)
     static int n_sm_att = 0;
     if (n_sm_att == 0) {
         int dev = 0;
