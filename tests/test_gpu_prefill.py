@@ -122,3 +122,24 @@ def test_zero_query_pins_set_sizes_on_gpu():
 def test_no_bounded_wait_expired():
     # runs after the cases above in this file: the tensor-core kernel's waits are bounded, and none gave up
     assert lte.lte_device_status() == 0
+
+
+@pytest.mark.parametrize("dtype,d,T,W,R", [("bf16", 64, 1500, 96, 80, ), ("bf16", 128, 900, 64, 50), ("f32", 32, 400, 24, 30)])
+def test_caller_made_list_uniform_stride(dtype, d, T, W, R):
+    """The attention takes any ascending list: the training-free "uniform stride + sliding window" rule of the paper's
+    ablation (Section 4, ablation paragraph) needs no scorer, the caller writes the list; heads may hold different counts."""
+    cfg = synth.Config("unif", dtype, 2, 3, d, T, W, R, 7, 0.1)
+    x = synth.make(cfg, 9)
+    q, k, v = (dev(x[t], dtype) for t in "qkv")
+    idx = np.full((cfg.B, cfg.H, R), -1, np.int32); cnt = np.zeros((cfg.B, cfg.H), np.int32)
+    for b in range(cfg.B):
+        for h in range(cfg.H):
+            n = R - (b * cfg.H + h) * 3                                       # a different budget per head
+            stride = max((T - W + n - 1) // n, 1)
+            pos = np.arange(h % stride, T - W, stride, dtype=np.int32)[:n]    # out-of-window tokens at a uniform stride
+            idx[b, h, :len(pos)] = pos; cnt[b, h] = len(pos)
+    s = shape_of(cfg)
+    o, lse = lte.lte_attn_prefill(s, q, k, v, torch.from_numpy(idx).cuda(), torch.from_numpy(cnt).cuda())
+    torch.cuda.synchronize()
+    o64, l64 = orc.attn_prefill(x["q"], x["k"], x["v"], idx, cnt, W)
+    _assert_close(cfg, (o.float().cpu().numpy(), lse.cpu().numpy(), o64, l64))
