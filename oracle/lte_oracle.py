@@ -188,6 +188,27 @@ def prefill_chunk(q, k, v, z, n0, W, R, pool_idx, pool_cnt, sink=0, tau=0.5, sca
     return o, lse, idx, cnt
 
 
+def rope_tables(n_pos, d, base=10000.0):
+    """cos, sin [n_pos, d/2] of the rotary position embedding: angle(p, c) = p base^(-2c/d)."""
+    inv = base ** (-np.arange(0, d, 2, dtype=np.float64) / d)
+    ang = np.arange(n_pos, dtype=np.float64)[:, None] * inv[None, :]
+    return np.cos(ang), np.sin(ang)
+
+
+def rope(x, cos, sin, pos0=0, inverse=False):
+    """Rotary embedding of x [..., T, d] at positions pos0 .. pos0+T-1, half-split pairing: channels c and c + d/2 form
+    the pair that is rotated by angle(p, c): (x1, x2) -> (x1 cos - x2 sin, x2 cos + x1 sin).  inverse=True rotates back
+    (the same with the sine negated), which is what the scorer needs when the cache holds rotated keys
+    (Section 3.1.3, lazy scoring paragraph)."""
+    x = _f64(x)
+    T, d = x.shape[-2], x.shape[-1]
+    c, s = _f64(cos)[pos0:pos0 + T], _f64(sin)[pos0:pos0 + T]
+    if inverse:
+        s = -s
+    x1, x2 = x[..., :d // 2], x[..., d // 2:]
+    return np.concatenate([x1 * c - x2 * s, x2 * c + x1 * s], axis=-1)
+
+
 def sparsity_stats(z, lam=None, tau=0.5):
     """Eq. 7 and the retention count it is steered by: count[h] = mean over the batch of #{i : r_i > tau} per sequence,
     penalty = sum_h lam[h] sum_{b,i} ReLU(r_i - tau), r = sigmoid(z), over the scored positions (z > -inf)."""

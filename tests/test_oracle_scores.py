@@ -121,3 +121,21 @@ def test_stack_parameter_share_at_0p4b():
     per_head = sum(ch[l + 1] * 3 * ch[l] + ch[l + 1] for l in range(3)) + ch[3] + 1
     total = per_head * heads * lte_layers
     assert 0.012 < total / 0.4e9 < 0.02
+
+
+def test_rope_is_a_rotation_of_channel_pairs_and_inverts():
+    """Pins for the rotary embedding the lazy scoring undoes on cached keys (Section 3.1.3): each pair (c, c + d/2) is
+    multiplied by exp(i angle) as a complex number; position 0 is the identity; norms are kept; the inverse undoes it."""
+    rng = np.random.default_rng(0)
+    d, T = 16, 40
+    x = rng.standard_normal((2, 3, T, d))
+    cos, sin = orc.rope_tables(100, d)
+    assert np.allclose(cos[0], 1.0) and np.allclose(sin[0], 0.0)
+    assert np.allclose(cos[5, 0], np.cos(5.0)) and np.allclose(sin[7, d // 2 - 1], np.sin(7.0 * 10000.0 ** (-(d - 2) / d)))
+    y = orc.rope(x, cos, sin, pos0=11)
+    zc = (x[..., :d // 2] + 1j * x[..., d // 2:]) * np.exp(1j * np.arange(11, 11 + T)[:, None] * 10000.0 ** (-np.arange(0, d, 2) / d))
+    np.testing.assert_allclose(y[..., :d // 2], zc.real, atol=1e-12)
+    np.testing.assert_allclose(y[..., d // 2:], zc.imag, atol=1e-12)
+    np.testing.assert_allclose(np.linalg.norm(y, axis=-1), np.linalg.norm(x, axis=-1), rtol=1e-12)
+    np.testing.assert_allclose(orc.rope(y, cos, sin, pos0=11, inverse=True), x, atol=1e-12)
+    np.testing.assert_allclose(orc.rope(x[..., :1, :], cos, sin, pos0=0), x[..., :1, :], atol=0)
