@@ -197,6 +197,22 @@ int lte_attn_decode(const lte_shape* s, const lte_conv* c, void* cache,
 int lte_cache_score(const lte_shape* s, const lte_conv* c, void* cache, void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * The same for a cache whose keys carry a rotary position embedding (Section 3.1.3, lazy scoring paragraph: the scorer
+ * consumes keys as they were before the embedding, the cache stores them after it): the ring's keys are rotated back
+ * (the rotation with the sine negated, at each token's own position) on their way into the scorer's input.  Prefill
+ * needs nothing of the kind: lte_scores is simply given the un-rotated keys, lte_attn_prefill and lte_cache_init the
+ * rotated ones.
+ *   rope_cos, rope_sin   in  [rope_len, d/2] fp32 device: cos / sin of the angle of channel pair (c, c + d/2) at position p
+ *                        (half-split pairing: (x1, x2) -> (x1 cos - x2 sin, x2 cos + x1 sin) is the embedding);
+ *                        both NULL = lte_cache_score
+ *   rope_len             positions the tables cover; a ring token at a position >= rope_len keeps its rotated key and
+ *                        lte_device_status() reports it
+ * Errors: as lte_cache_score; INVALID_ARG for one NULL table or rope_len <= 0.
+ */
+int lte_cache_score_unrope(const lte_shape* s, const lte_conv* c, void* cache, const float* rope_cos, const float* rope_sin,
+                           int32_t rope_len, void* ws, size_t ws_bytes, void* stream);
+
+/*
  * Chunked (continued) prefill on top of a cache (Section 3.1.3, "Cached prefilling and decoding"): T = s->T new tokens
  * arrive at a cache that holds n_past tokens (from lte_cache_init, lte_attn_decode or an earlier chunk).  Chunk-end
  * reading: the pool's entries compete with the tokens that leave the window while the chunk arrives (positions

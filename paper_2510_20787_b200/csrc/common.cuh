@@ -102,7 +102,8 @@ int launch_prefill_tc_long(const Params& p, const void* q, const void* k, const 
 int prefill_long_status_fetch_and_clear();
 int launch_cache_init(const Params& p, const void* k, const void* v, const float* z, const int32_t* idx,
                       const int32_t* cnt, void* cache, cudaStream_t st);
-int launch_ring_linearize(const Params& p, const void* cache, void* klin, void* vlin, cudaStream_t st);
+int launch_ring_linearize(const Params& p, const void* cache, void* klin, void* vlin, const float* rope_cos, const float* rope_sin,
+                          int rope_len, cudaStream_t st);
 int launch_ring_scatter_z(const Params& p, void* cache, const float* zlin, cudaStream_t st);
 int launch_chunk_gather(const Params& p, const void* cache, const void* k, const void* v, void* klin, void* vlin, float* zsrc,
                         int32_t* oldpos, int n0, int R0, int Wn, cudaStream_t st);

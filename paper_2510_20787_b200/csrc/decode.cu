@@ -694,9 +694,13 @@ int launch_cache_init(const Params& p, const void* k, const void* v, const float
 // zero.  The scorer then runs over the copy as over a W-token sequence, and the logits whose receptive field lies inside
 // the ring (or left of time 0) go back to the ring's logit slots: rows r >= half unless the ring starts at time 0, and
 // r <= min(n, W) - 1 - half.
+// With rotary tables (cos, sin [rope_len, D/2], half-split pairing: channels c and c + D/2 form a pair) the keys are
+// rotated back to their un-rotated form on the way: the scorer consumes keys as they were before the position embedding,
+// the cache holds them after it (Section 3.1.3, lazy scoring paragraph).  Row r is the token at position base + r.
 template <typename T>
 __global__ void ring_linearize_kernel(const unsigned char* __restrict__ cache, CacheLayout L, T* __restrict__ klin,
-                                      T* __restrict__ vlin, int D, int W)
+                                      T* __restrict__ vlin, int D, int W, const float* __restrict__ rope_cos,
+                                      const float* __restrict__ rope_sin, int rope_len)
 {
     const int bh = blockIdx.x;
     const unsigned char* blk = cache + L.header + (size_t)bh * L.stride;
@@ -711,6 +715,19 @@ __global__ void ring_linearize_kernel(const unsigned char* __restrict__ cache, C
             const int row = (base + r) % W;
             const int cs = L.swz ? ((((c >> 3) ^ (row & 7)) << 3) | (c & 7)) : c;
             kx = Kc[(size_t)row * D + cs]; vx = Vc[(size_t)row * D + cs];
+            if (rope_cos) {
+                const int pos = base + r, hd = D / 2;
+                if (pos < rope_len) {
+                    const int cp = c < hd ? c + hd : c - hd;       // the channel this one is paired with
+                    const int cps = L.swz ? ((((cp >> 3) ^ (row & 7)) << 3) | (cp & 7)) : cp;
+                    const float co = rope_cos[(size_t)pos * hd + (c % hd)], si = rope_sin[(size_t)pos * hd + (c % hd)];
+                    const float a = to_f(kx), b = to_f(Kc[(size_t)row * D + cps]);
+                    // inverse rotation: (x1, x2) -> (x1 cos + x2 sin, x2 cos - x1 sin)
+                    kx = from_f<T>(c < hd ? a * co + b * si : a * co - b * si);
+                } else if (c == 0) {
+                    atomicExch(&g_decode_status, 32);              // the tables do not reach this position: key left rotated
+                }
+            }
         }
         klin[((size_t)bh * W + r) * D + c] = kx;
         vlin[((size_t)bh * W + r) * D + c] = vx;
@@ -729,14 +746,16 @@ __global__ void ring_scatter_z_kernel(unsigned char* __restrict__ cache, CacheLa
     for (int r = r_lo + threadIdx.x; r <= r_hi; r += blockDim.x) zc[(base + r) % W] = zlin[(size_t)bh * W + r];
 }
 
-int launch_ring_linearize(const Params& p, const void* cache, void* klin, void* vlin, cudaStream_t st)
+int launch_ring_linearize(const Params& p, const void* cache, void* klin, void* vlin, const float* rope_cos, const float* rope_sin,
+                          int rope_len, cudaStream_t st)
 {
     const CacheLayout L = cache_layout(p.d, p.W, p.R, p.dtype);
     if (p.dtype == LTE_BF16)
         ring_linearize_kernel<__nv_bfloat16><<<p.B * p.H, 256, 0, st>>>((const unsigned char*)cache, L, (__nv_bfloat16*)klin,
-                                                                        (__nv_bfloat16*)vlin, p.d, p.W);
+                                                                        (__nv_bfloat16*)vlin, p.d, p.W, rope_cos, rope_sin, rope_len);
     else
-        ring_linearize_kernel<float><<<p.B * p.H, 256, 0, st>>>((const unsigned char*)cache, L, (float*)klin, (float*)vlin, p.d, p.W);
+        ring_linearize_kernel<float><<<p.B * p.H, 256, 0, st>>>((const unsigned char*)cache, L, (float*)klin, (float*)vlin, p.d, p.W,
+                                                                rope_cos, rope_sin, rope_len);
     return cuda_status(cudaGetLastError());
 }
 

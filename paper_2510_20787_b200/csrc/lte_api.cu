@@ -253,7 +253,14 @@ int lte_cache_init(const lte_shape* s, const lte_conv* c, const void* k, const v
 
 int lte_cache_score(const lte_shape* s, const lte_conv* c, void* cache, void* ws, size_t ws_bytes, void* stream)
 {
+    return lte_cache_score_unrope(s, c, cache, nullptr, nullptr, 0, ws, ws_bytes, stream);
+}
+
+int lte_cache_score_unrope(const lte_shape* s, const lte_conv* c, void* cache, const float* rope_cos, const float* rope_sin,
+                           int32_t rope_len, void* ws, size_t ws_bytes, void* stream)
+{
     int e = check_shape(s, false); if (e) return e;
+    if ((rope_cos == nullptr) != (rope_sin == nullptr) || (rope_cos && rope_len <= 0)) return LTE_ERR_INVALID_ARG;
     if (!c || !c->w || c->n_layers != 3) return LTE_ERR_UNSUPPORTED;       // the single layer is scored inside the step
     e = check_conv_or_stack(s, c); if (e) return e;
     if (!cache || !aligned16(cache)) return LTE_ERR_INVALID_ARG;
@@ -264,7 +271,7 @@ int lte_cache_score(const lte_shape* s, const lte_conv* c, void* cache, void* ws
     char* base = (char*)ws;
     lte_shape s2 = *s; s2.T = s->W;                                         // the ring as a W-token sequence
     Params p = make_params(&s2, c);
-    e = launch_ring_linearize(p, cache, base + w.klin, base + w.vlin, st); if (e) return e;
+    e = launch_ring_linearize(p, cache, base + w.klin, base + w.vlin, rope_cos, rope_sin, rope_len, st); if (e) return e;
     float* zlin = (float*)(base + w.zlin);
     e = launch_scores_stack_tc(p, base + w.klin, base + w.vlin, zlin, nullptr, base + w.tc, w.total - w.tc, st);
     if (e == LTE_ERR_UNSUPPORTED) e = launch_scores_stack(p, base + w.klin, base + w.vlin, zlin, nullptr, st);

@@ -20,7 +20,7 @@ BWD_CNN_INPUT_GRAD = 1
 
 EXPORTS = ["lte_device_status", "lte_workspace_bytes", "lte_strerror", "lte_scores", "lte_select", "lte_cache_score", "lte_attn_prefill",
            "lte_cache_bytes", "lte_cache_init", "lte_attn_decode", "lte_attn_prefill_chunk", "lte_attn_bwd", "lte_attn_bwd_static",
-           "lte_sparsity_stats", "lte_lambda_update"]
+           "lte_sparsity_stats", "lte_lambda_update", "lte_cache_score_unrope"]
 STATIC_SCRATCH_BYTES = 8 << 20
 
 
@@ -64,6 +64,7 @@ def lib():
         L.lte_cache_init.argtypes = [vp] * 9
         L.lte_attn_decode.argtypes = [vp] * 9
         L.lte_cache_score.argtypes = [vp] * 4 + [ctypes.c_size_t, vp]
+        L.lte_cache_score_unrope.argtypes = [vp] * 5 + [ctypes.c_int32, vp, ctypes.c_size_t, vp]
         L.lte_sparsity_stats.argtypes = [vp] * 6 + [ctypes.c_size_t, vp]
         L.lte_lambda_update.argtypes = [ctypes.c_int32, vp, vp, vp, ctypes.c_int64, vp]
         L.lte_attn_prefill_chunk.argtypes = [vp] * 3 + [ctypes.c_int32] + [vp] * 6 + [ctypes.c_size_t, vp]
@@ -262,6 +263,15 @@ def lte_cache_score(s, c, cache, ws=None):
         ws = torch.empty(max(lte_workspace_bytes(OP_DECODE, s, c), 256), dtype=torch.uint8, device=cache.device)
     _check("lte_cache_score", lib().lte_cache_score(ctypes.addressof(s), ctypes.addressof(c), _ptr(cache), _ptr(ws),
                                                     ws.numel(), _stream()))
+
+
+def lte_cache_score_unrope(s, c, cache, rope_cos, rope_sin, ws=None):
+    """lte_cache_score for a cache that holds rotated keys: rope_cos, rope_sin [positions, d/2] fp32 on the device."""
+    if ws is None:
+        ws = torch.empty(max(lte_workspace_bytes(OP_DECODE, s, c), 256), dtype=torch.uint8, device=cache.device)
+    _check("lte_cache_score_unrope", lib().lte_cache_score_unrope(ctypes.addressof(s), ctypes.addressof(c), _ptr(cache),
+                                                                  _ptr(rope_cos, torch.float32), _ptr(rope_sin, torch.float32),
+                                                                  int(rope_cos.shape[0]), _ptr(ws), ws.numel(), _stream()))
 
 
 def lte_attn_bwd(s, c, q, k, v, o, lse, dO, z, idx, cnt, lam=None, flags=BWD_CNN_INPUT_GRAD, want_dbias=True,

@@ -179,6 +179,54 @@ def test_stack_in_chunked_prefill(dtype, d, W, R, T0, dec, Tc):
         assert np.array_equal(pool, pidx[b, h, :pcnt[b, h]])
 
 
+@pytest.mark.parametrize("dtype,d,W,R,T0,steps,period", [("bf16", 64, 32, 24, 100, 60, 19), ("f32", 32, 24, 12, 0, 70, 11), ("bf16", 64, 64, 30, 200, 90, 40)])
+def test_stack_decode_with_rotated_keys(dtype, d, W, R, T0, steps, period):
+    """The cache holds keys with a rotary position embedding, the scorer wants them without: the prompt is scored on the
+    un-rotated keys, and lte_cache_score_unrope rotates the ring's keys back before the lazy batches of the decode."""
+    cfg = synth.Config("stackrope", dtype, 2, 2, d, T0 + steps, W, R, 7, 0.1)
+    Ttot = T0 + steps
+    x = synth.make(cfg, 8, T=Ttot)
+    wl, wout, bl, bout = _stack_params(cfg.H, d, 8, True)
+    t = lambda a: torch.from_numpy(a).cuda()
+    c = lte.conv_stack([t(w) for w in wl], t(wout), [t(b) for b in bl], t(bout))
+    cos, sin = (a.astype(np.float32) for a in orc.rope_tables(Ttot, d))
+    rnd = synth.round_bf16 if dtype == "bf16" else (lambda a: a.astype(np.float32))
+    kr = rnd(orc.rope(x["k"], cos, sin).astype(np.float32))                 # what the cache holds
+    q, k0, krd, v = dev(x["q"], dtype), dev(x["k"], dtype), dev(kr, dtype), dev(x["v"], dtype)
+    s0 = shape_of(cfg, T=T0, B=cfg.B)
+    if T0 > 0:
+        z = lte.lte_scores(s0, c, k0[:, :, :T0].contiguous(), v[:, :, :T0].contiguous())      # the prompt: un-rotated keys
+        idx, cnt = lte.lte_select(s0, z)
+        cache = lte.lte_cache_init(s0, c, krd[:, :, :T0].contiguous(), v[:, :, :T0].contiguous(), z, idx, cnt)
+    else:
+        cache = lte.lte_cache_init(s0, c)
+    outs, lses = [], []
+    for i, n in enumerate(range(T0, Ttot)):
+        if i % period == 0:
+            lte.lte_cache_score_unrope(s0, c, cache, t(cos), t(sin))
+        o1, l1 = lte.lte_attn_decode(s0, c, cache, q[:, :, n].contiguous(), krd[:, :, n].contiguous(), v[:, :, n].contiguous())
+        outs.append(o1.float().cpu().numpy()); lses.append(l1.cpu().numpy())
+    torch.cuda.synchronize()
+    assert lte.lib().lte_device_status() == 0
+    ku = rnd(orc.rope(kr, cos, sin, inverse=True).astype(np.float32))        # the keys the lazy batches see (storage precision)
+    za = orc.scores_stack(x["k"], x["v"], wl, bl, wout, bout)
+    zb = orc.scores_stack(ku, x["v"], wl, bl, wout, bout)
+    z64 = np.where(np.arange(Ttot)[None, None, :] <= T0 - 1 - 6, za, zb)
+    o64, l64, pidx, pcnt = orc.stream(x["q"], kr, x["v"], z64, W, R, 0, n_from=T0)
+    tol = 2e-2 if dtype == "bf16" else 1e-4
+    assert np.max(np.abs(np.stack(outs, axis=2) - o64)) <= tol
+    assert np.max(np.abs(np.stack(lses, axis=2) - l64)) <= tol
+    from tests.test_gpu_decode import _read_pool
+    pools, ns = _read_pool(cache, cfg, cfg.B)
+    for bh, pool in enumerate(pools):
+        b, h = divmod(bh, cfg.H)
+        assert np.array_equal(pool, pidx[b, h, :pcnt[b, h]])
+    # tables that do not reach the newest position are reported, not silently applied
+    lte.lte_cache_score_unrope(s0, c, cache, t(cos[:Ttot - 5]), t(sin[:Ttot - 5]))
+    torch.cuda.synchronize()
+    assert lte.lib().lte_device_status() != 0
+
+
 # ---- backward through the stack (lte_attn_bwd with the three-layer scorer) ---------------------------------------------
 def _rel(a, b):
     return float(np.linalg.norm(np.asarray(a, np.float64) - b) / (np.linalg.norm(b) + 1e-30))
