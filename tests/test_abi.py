@@ -152,3 +152,17 @@ def test_training_pieces_host_side():
     assert L.lte_sparsity_stats(a(s), fake, None, fake, fake, fake, 8, None) == -3
     wide = lte.shape(1, 9000, 16, 64, 8, 4, lte.BF16)
     assert L.lte_sparsity_stats(a(wide), fake, None, fake, fake, fake, 1 << 20, None) == -2
+
+
+def test_unrope_scoring_host_side():
+    """lte_cache_score_unrope: both tables or none, a positive length (validation fails before anything is launched)."""
+    L = lte.lib()
+    a = ctypes.addressof
+    fake = 4096
+    stack = lte.LteConv(3, 3, 2, 256, 0)
+    s = lte.shape(4, 16, 0, 64, 128, 128, lte.BF16)
+    assert L.lte_cache_score_unrope(a(s), a(stack), fake, fake, None, 100, fake, 1 << 30, None) == -1
+    assert L.lte_cache_score_unrope(a(s), a(stack), fake, None, fake, 100, fake, 1 << 30, None) == -1
+    assert L.lte_cache_score_unrope(a(s), a(stack), fake, fake, fake, 0, fake, 1 << 30, None) == -1
+    assert L.lte_cache_score_unrope(a(s), a(stack), fake, fake, fake, 100, fake, 16, None) == -3
+    assert L.lte_cache_score_unrope(a(s), a(lte.LteConv(1, 7, 1, 256, 0)), fake, fake, fake, 100, fake, 1 << 30, None) == -2
