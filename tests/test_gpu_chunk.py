@@ -122,6 +122,8 @@ def test_chunk_plans_bf16(plan):
     (dict(sink=2, W=8, R=5), [("prefill", 0), ("chunk", 9), ("chunk", 40)], 1.0, 1),
     (dict(W=64, R=64, B=1, H=2), [("prefill", 300), ("chunk", 200), ("decode", 6)], 0.0, 4),
     (dict(W=128, R=128, B=2, H=4), [("prefill", 700), ("chunk", 650)], 0.0, 1),      # several tiles, ragged tail
+    (dict(W=32, R=0), [("prefill", 50), ("chunk", 90), ("decode", 5)], 0.0, 1),           # no pool at all: sliding window only
+    (dict(dtype="f32", d=64, W=20, R=10, K=3, B=1, H=2), [("prefill", 0), ("chunk", 45), ("decode", 3), ("chunk", 30)], 0.0, 3),
 ])
 def test_chunk_dtypes_sinks_groups(kw, plan, scale, group):
     _compare(_cfg(**kw), plan, seed=1, scale=scale, group=group)
