@@ -614,7 +614,7 @@ def _extra_p(out, torch, lte, synth, pk, flush, n5):
         "step_ms": tg * 1e3, "tokens_per_s": cfg.B * cfg.T / tg, "attn_ms": tag * 1e3,
         "attn_algorithmic_tflops": flg / tag / 1e12, "attn_tensor_frac": flg / tag / 1e12 / pk["bf16_tflops"],
         "decode_us_per_step": mid3(reps),
-        "note": "decode: one kernel updates the cache, one attends for the four query heads of a group over the updated block"}
+        "note": "decode: one kernel updates the cache block of a key/value head and attends for the four query heads of its group"}
     del og, lseg, zg, cache, qg
 
 

@@ -175,7 +175,7 @@ int lte_cache_init(const lte_shape* s, const lte_conv* c, const void* k, const v
  *   cache        in/out
  *   q1           in   [B,H*group,d] of s->dtype;   k1, v1 in [B,H,d]
  *   o1           out  [B,H*group,d] of s->dtype;   lse1 out [B,H*group] fp32
- *   With group > 1 the step is two kernels: one updates the cache (steps 1-3), one attends for all query heads of a
+ *   With group > 1 the head's thread block updates the cache (steps 1-3) and then attends for all query heads of the
  *   group over the updated block, which is read once.
  * s->T is ignored.  Errors: INVALID_ARG, UNSUPPORTED (W + R > 4096, d not in {32,64,128}), CUDA.
  */

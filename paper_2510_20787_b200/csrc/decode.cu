@@ -767,21 +767,22 @@ int launch_ring_scatter_z(const Params& p, void* cache, const float* zlin, cudaS
 }
 
 // ---- grouped-query attention -----------------------------------------------------------------------------------------
-// With G > 1 query heads per key/value head the step is split so that the cache block is read once: an update kernel
-// applies the replacement rule, scores the newest complete token and writes the new key/value into the ring (it touches a
-// handful of rows), and the attend kernel below serves all G query heads over the updated block.
-constexpr int DTU = 128;
-template <typename T, int D>
-__global__ void __launch_bounds__(DTU) decode_update_kernel(unsigned char* __restrict__ cache, CacheLayout L,
-                                                            const T* __restrict__ k1, const T* __restrict__ v1,
-                                                            const float* __restrict__ cw, const float* __restrict__ cbias, int H,
-                                                            int W, int R, int sink, int K, float zthr)
+// With G > 1 query heads per key/value head the cache block is read once per step: the head's thread block first applies
+// the replacement rule, scores the newest complete token and writes the new key/value into the ring (a handful of rows),
+// then serves all G query heads over the updated block (the attend kernel below).
+// The update of one key/value head's block by the DTU threads of a thread block (every thread of the block calls it; it
+// ends with the block's writes issued, not yet ordered: the caller synchronises).
+template <typename T, int D, int DTU>
+__device__ __forceinline__ void cache_update_block(unsigned char* __restrict__ cache, const CacheLayout& L, int bh,
+                                                   const T* __restrict__ k1, const T* __restrict__ v1,
+                                                   const float* __restrict__ cw, const float* __restrict__ cbias, int H,
+                                                   int W, int R, int sink, int K, float zthr)
 {
     constexpr int CPL = D / 32, NWU = DTU / 32, PIECES = D * (int)sizeof(T) / 16;
     __shared__ float s_tap[kMaxTaps];
     __shared__ float s_wz[NWU];
     __shared__ int s_wpos[NWU], s_wslot[NWU];
-    const int bh = blockIdx.x, h = bh % H, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const int h = bh % H, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     unsigned char* blk = cache + L.header + (size_t)bh * L.stride;
     T* Kc = reinterpret_cast<T*>(blk + L.off_k);
     T* Vc = reinterpret_cast<T*>(blk + L.off_v);
@@ -886,9 +887,12 @@ __global__ void __launch_bounds__(DTU) decode_update_kernel(unsigned char* __res
 // the same way, weighted per query head in registers, reduced over lanes sharing a slice and then over the warps.
 constexpr int ATT_Q = 4;
 template <typename T, int D>
-__global__ void __launch_bounds__(DT) decode_attend_kernel(const unsigned char* __restrict__ cache, CacheLayout L,
+__global__ void __launch_bounds__(DT) decode_attend_kernel(unsigned char* __restrict__ cache, CacheLayout L,
                                                            const T* __restrict__ q1, T* __restrict__ o1,
-                                                           float* __restrict__ lse1, int W, int G, float scale, int g_first)
+                                                           float* __restrict__ lse1, int W, int G, float scale, int g_first,
+                                                           const T* __restrict__ k1, const T* __restrict__ v1,
+                                                           const float* __restrict__ cw, const float* __restrict__ cbias, int H,
+                                                           int R, int sink, int K, float zthr)
 {
     constexpr int EPV = V16<T>::N;                             // elements per 16-byte piece
     constexpr int LPR = D / EPV;                               // lanes per row
@@ -904,6 +908,15 @@ __global__ void __launch_bounds__(DT) decode_attend_kernel(const unsigned char* 
     const int nsplit = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
     const int bh = blockIdx.x / nsplit, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     const int seg = tid % LPR, rsub = tid / LPR;
+    // the step's cache update first (k1 != NULL), by the head's (first) block: a handful of rows, then everybody reads the
+    // updated block
+    if (k1 != nullptr) {
+        if (rank == 0) {
+            cache_update_block<T, D, DT>(cache, L, bh, k1, v1, cw, cbias, H, W, R, sink, K, zthr);
+            __threadfence();
+        }
+        if (nsplit > 1) cluster.sync(); else __syncthreads();
+    }
     const unsigned char* blk = cache + L.header + (size_t)bh * L.stride;
     const uint4* Kc = reinterpret_cast<const uint4*>(blk + L.off_k);
     const uint4* Vc = reinterpret_cast<const uint4*>(blk + L.off_v);
@@ -1150,29 +1163,9 @@ int launch_decode(const Params& p, void* cache, const void* q1, const void* k1, 
     Params ps = p;
     if (p.stack) ps.K = 0;                               // the stack is scored outside the step (lte_cache_score)
     if (p.G <= 1) return launch_decode_step(ps, cache, q1, k1, v1, o1, lse1, st);
-    // grouped queries: update the cache, then one pass over the updated block for all query heads of the group
+    // grouped queries: one kernel updates the head's cache block and then serves all query heads of the group from it
     if (p.W + p.R > MAX_ROWS) return LTE_ERR_UNSUPPORTED;
     const CacheLayout L = cache_layout(p.d, p.W, p.R, p.dtype);
-#define LTE_UPD(T, D)                                                                                                  \
-    decode_update_kernel<T, D><<<p.B * p.H, DTU, 0, st>>>((unsigned char*)cache, L, (const T*)k1, (const T*)v1, p.w,    \
-                                                          p.bias, p.H, p.W, p.R, p.sink, ps.K, p.zthr)
-    if (p.dtype == LTE_BF16) {
-        switch (p.d) {
-            case 32: LTE_UPD(__nv_bfloat16, 32); break;
-            case 64: LTE_UPD(__nv_bfloat16, 64); break;
-            case 128: LTE_UPD(__nv_bfloat16, 128); break;
-            default: return LTE_ERR_UNSUPPORTED;
-        }
-    } else {
-        switch (p.d) {
-            case 32: LTE_UPD(float, 32); break;
-            case 64: LTE_UPD(float, 64); break;
-            case 128: LTE_UPD(float, 128); break;
-            default: return LTE_ERR_UNSUPPORTED;
-        }
-    }
-#undef LTE_UPD
-    if (cudaGetLastError() != cudaSuccess) return LTE_ERR_CUDA;
     const size_t att_smem = sizeof(float) * ((size_t)ATT_Q * (p.W + p.R) + (size_t)(DT / 32) * ATT_Q * p.d);
     // blocks per key/value head (a cluster): more than one only while there are fewer blocks than SMs and a share keeps 256 rows
     // (with 256 heads of 1280 rows, two blocks per head measured 41 us per step against 29 us for one)
@@ -1199,8 +1192,9 @@ int launch_decode(const Params& p, void* cache, const void* q1, const void* k1, 
                 return LTE_ERR_CUDA;                                                                                   \
             attr_done = true;                                                                                          \
         }                                                                                                              \
-        if (cudaLaunchKernelEx(&acfg, decode_attend_kernel<T, D>, (const unsigned char*)cache, L, (const T*)q1, (T*)o1, lse1,  \
-                               p.W, p.G, p.scale, 0) != cudaSuccess) return LTE_ERR_CUDA;                               \
+        if (cudaLaunchKernelEx(&acfg, decode_attend_kernel<T, D>, (unsigned char*)cache, L, (const T*)q1, (T*)o1, lse1,        \
+                               p.W, p.G, p.scale, 0, (const T*)k1, (const T*)v1, p.w, p.bias, p.H, p.R, p.sink, ps.K,    \
+                               p.zthr) != cudaSuccess) return LTE_ERR_CUDA;                                             \
     } while (0)
     if (p.dtype == LTE_BF16) {
         switch (p.d) {
