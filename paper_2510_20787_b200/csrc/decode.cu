@@ -882,7 +882,7 @@ __device__ __forceinline__ void cache_update_block(unsigned char* __restrict__ c
 // The attend kernel: query heads g_first .. G-1 of a key/value head over its block (ring rows of the min(n, W) newest
 // tokens, cnt pool rows), after the update.  One block (or a cluster of blocks) per key/value head, up to ATT_Q query heads
 // per pass.  Rows are spread as in the step kernels: LPR lanes share a row, each with one 16-byte piece of it, so a warp's
-// load covers whole consecutive rows; four rows per thread are in flight.  Logits: partial dots per lane against the
+// load covers whole consecutive rows; eight rows per thread are in flight.  Logits: partial dots per lane against the
 // lane's slice of every query, reduced over the LPR lanes by shuffles; block maxima and sums per query head; value rows
 // the same way, weighted per query head in registers, reduced over lanes sharing a slice and then over the warps.
 constexpr int ATT_Q = 4;
@@ -897,7 +897,7 @@ __global__ void __launch_bounds__(DT) decode_attend_kernel(unsigned char* __rest
     constexpr int EPV = V16<T>::N;                             // elements per 16-byte piece
     constexpr int LPR = D / EPV;                               // lanes per row
     constexpr int RPP = DT / LPR;                              // rows per pass of the block
-    constexpr int NW = DT / 32, UNR = 4;
+    constexpr int NW = DT / 32, UNR = 8;
     extern __shared__ float att_sm[];                          // logits [ATT_Q][rows], then partial outputs [NW][ATT_Q][D]
     __shared__ float s_red[NW][ATT_Q];
     __shared__ float s_mx[ATT_Q], s_sum[ATT_Q];
