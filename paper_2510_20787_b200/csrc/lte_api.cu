@@ -295,6 +295,7 @@ int lte_attn_prefill_chunk(const lte_shape* s, const lte_conv* c, void* cache, i
     char* base = (char*)ws;
     // the local sequence: pool rows (once anything has left the window), the ring in time order, the chunk
     const int Tc = s->T, Wn = n_past < s->W ? n_past : s->W, R0 = n_past > s->W ? s->R : 0, qoff = R0 + Wn, Tloc = qoff + Tc;
+    if (Tloc - s->W > (1 << 24)) return LTE_ERR_UNSUPPORTED;   // the selection's limit on candidates per head
     lte_shape sl = *s; sl.T = Tloc;
     Params p = make_params(&sl, c);                          // p.sink: positions of the whole sequence (the logit merge)
     Params psel = p; psel.sink = 0;                          // the selection sees sink tokens as +inf logits instead
