@@ -260,27 +260,39 @@ def run_lte(args):
     hc = torch.empty(cnt.shape, dtype=cnt.dtype).pin_memory()
     dq_, dk_, dv_ = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
 
-    # One batch element per stream, round-robin over a few streams: the host->device copy of element b+1, the kernels
-    # of element b and the device->host copy of element b-1 overlap (the two copy directions use different engines).
+    # Three streams: all host->device copies in order on one (k, v of an element first, then its q), the kernels of the
+    # elements on the current stream as their inputs arrive, all device->host copies on a third: the copy of element b+1, the
+    # kernels of element b and the read-back of element b-1 overlap (the two copy directions use different engines), and
+    # each engine sees one queue of large copies.
     s1 = lte.shape(1, cfg.H, cfg.T, cfg.d, cfg.W, cfg.R, lte.BF16)
-    side = [torch.cuda.Stream() for _ in range(min(cfg.B, 4))]
+    st_in, st_out = torch.cuda.Stream(), torch.cuda.Stream()
+    ev_kv = [torch.cuda.Event() for _ in range(cfg.B)]
+    ev_q = [torch.cuda.Event() for _ in range(cfg.B)]
+    ev_done = [torch.cuda.Event() for _ in range(cfg.B)]
 
     def e2e_step():
         cur = torch.cuda.current_stream()
-        for st in side:
-            st.wait_stream(cur)
-        for b in range(cfg.B):
-            st = side[b % len(side)]
-            with torch.cuda.stream(st):
+        st_in.wait_stream(cur); st_out.wait_stream(cur)
+        with torch.cuda.stream(st_in):
+            for b in range(cfg.B):
                 sl = slice(b, b + 1)
-                dq_[sl].copy_(hq[sl], non_blocking=True); dk_[sl].copy_(hk[sl], non_blocking=True); dv_[sl].copy_(hv[sl], non_blocking=True)
-                lte.lte_scores(s1, c, dk_[sl], dv_[sl], z=z[sl])
-                lte.lte_select(s1, z[sl], idx=idx[sl], cnt=cnt[sl])
-                lte.lte_attn_prefill(s1, dq_[sl], dk_[sl], dv_[sl], idx[sl], cnt[sl], o=o[sl], lse=lse[sl])
+                dk_[sl].copy_(hk[sl], non_blocking=True); dv_[sl].copy_(hv[sl], non_blocking=True)
+                ev_kv[b].record(st_in)
+                dq_[sl].copy_(hq[sl], non_blocking=True)
+                ev_q[b].record(st_in)
+        for b in range(cfg.B):
+            sl = slice(b, b + 1)
+            cur.wait_event(ev_kv[b])
+            lte.lte_scores(s1, c, dk_[sl], dv_[sl], z=z[sl])
+            lte.lte_select(s1, z[sl], idx=idx[sl], cnt=cnt[sl])
+            cur.wait_event(ev_q[b])
+            lte.lte_attn_prefill(s1, dq_[sl], dk_[sl], dv_[sl], idx[sl], cnt[sl], o=o[sl], lse=lse[sl])
+            ev_done[b].record(cur)
+            with torch.cuda.stream(st_out):
+                st_out.wait_event(ev_done[b])
                 ho[sl].copy_(o[sl], non_blocking=True); hl[sl].copy_(lse[sl], non_blocking=True)
                 hi[sl].copy_(idx[sl], non_blocking=True); hc[sl].copy_(cnt[sl], non_blocking=True)
-        for st in side:
-            cur.wait_stream(st)
+        cur.wait_stream(st_out)
         return None
 
     barrier()
