@@ -67,7 +67,7 @@ template <int D> struct Smem {
 //   bar_s[b]  (commit)       S(t) is in TMEM buffer b = t & 1                     control -> softmax
 //   bar_p     (128 arrivals) P(t) is in shared memory, S buffer b is free         softmax -> control
 //   bar_pv    (commit)       PV(t) has completed                                   control -> softmax
-//   bar_g[b]  (128 arrivals) gathers issued before the top of tile t have landed   softmax -> control
+//   bar_gk[s], bar_gv[s] (128 arrivals, by cp.async completion) a gathered tile is in stage s   softmax -> control
 //   bar_k[s], bar_v[s]       TMA transaction barriers of the window tiles
 //   bar_kf[s], bar_vf[s]     (commit) the MMA that read stage s has completed          MMA lane -> load lane
 // S(t+1) and S(t+2) are computed while the softmax of tile t runs; loads run two to three tiles ahead.
@@ -94,11 +94,11 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const uint32_t bar_k0 = bar_q + 8;                         // 3 slots
     const uint32_t bar_v0 = bar_q + 32;                        // 3 slots
     const uint32_t bar_s0 = bar_q + 56;                        // 2 slots
-    const uint32_t bar_g0 = bar_q + 72;                        // 2 slots
     const uint32_t bar_p = bar_q + 88, bar_pv = bar_q + 96;
     const uint32_t bar_kf0 = bar_q + 104;                      // 3 slots: K stage free
     const uint32_t bar_vf0 = bar_q + 128;                      // 3 slots: V stage free
     const uint32_t tmem_slot = bar_q + 152;
+    const uint32_t bar_gk0 = bar_q + 160, bar_gv0 = bar_q + 184;   // 3 slots each: a gathered tile has landed in the stage
     volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(smem_raw + S::OFF_BAR + 152);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -112,7 +112,6 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const int j_start = max(i0 - W + 1, 0);
     const int n_win = (i_hi - j_start + 1 + BN - 1) / BN;
     const int32_t* id = idx + (size_t)bhk * R;
-    const int g_first = max(n_win - Smem<D>::KST, 0);        // first tile whose top may have gathers in flight
 
     if (tid == 0) {
         mbar_init(bar_q, 1);
@@ -124,7 +123,8 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         mbar_init(bar_s0, 1); mbar_init(bar_s0 + 8, 1);
         // every softmax thread arrives itself: one arrival per warp behind a __syncwarp() lengthened the hand-over of P
         // to the MMA warp and cost 3 % at d = 128, T = 32768
-        mbar_init(bar_g0, 128); mbar_init(bar_g0 + 8, 128);
+#pragma unroll
+        for (int s2 = 0; s2 < 3; ++s2) { mbar_init(bar_gk0 + 8 * s2, 128); mbar_init(bar_gv0 + 8 * s2, 128); }
         mbar_init(bar_p, 128); mbar_init(bar_pv, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -211,15 +211,15 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 const uint32_t va = sV + st * S::KVTILE;
                 v_desc[st] = (va >> 4) | ((S::ONES ? ((base + S::OFF_ONES - va) >> 4) : (8192u >> 4)) << 16);
             }
-            uint32_t k_par = 0, v_par = 0, g_waited = 0;       // TMA barrier parities (bit per stage); bar_g phases consumed
+            uint32_t k_par = 0, v_par = 0, gk_par = 0, gv_par = 0;   // barrier parities, a bit per stage (TMA tiles; gathered tiles)
             int ks = 0, vs = 0;                                // stage of the next S / PV operand
             int ts = 0;                                        // next S tile to issue
-            // gathers issued before the top of tile t have landed (the softmax warps signal from tile g_first on)
-            auto need_g = [&](int t) {
-                while ((int)g_waited <= t - g_first) { mbar_wait(bar_g0 + 8 * (g_waited & 1), (g_waited >> 1) & 1, 10); ++g_waited; }
-            };
             auto mma_s = [&]() {                               // S(ts) from K stage ks into S buffer ts & 1
                 if (ts < n_win) { mbar_wait(bar_k0 + 8 * ks, (k_par >> ks) & 1u, 2); k_par ^= 1u << ks; }
+                else {                                         // gathered rows: generic-proxy writes, made visible to the tensor core here
+                    mbar_wait(bar_gk0 + 8 * ks, (gk_par >> ks) & 1u, 10); gk_par ^= 1u << ks;
+                    fence_proxy_async();
+                }
                 tc_fence_after();
                 const uint32_t kb = k_lo + (uint32_t)ks * (S::KVTILE >> 4);
                 const uint32_t dcol = tmem + (ts & 1) * BN;
@@ -240,16 +240,13 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             mbar_wait(bar_q, 0, 1);
             PLM(16);
             mma_s();                                           // tile 0 is always a window tile
-            if (n_tiles > 1) {
-                if (n_win < 2) need_g(0);                      // tile 1 is a retained tile: the prologue gathers
-                mma_s();
-            }
+            if (n_tiles > 1) mma_s();
             for (int t = 0; t < n_tiles; ++t) {
                 // PV(t): everything but P is normally there long before
                 PLM(17);
                 PLM_TILE(t);
-                need_g(t);
                 if (t < n_win) { mbar_wait(bar_v0 + 8 * vs, (v_par >> vs) & 1u, 4); v_par ^= 1u << vs; }
+                else { mbar_wait(bar_gv0 + 8 * vs, (gv_par >> vs) & 1u, 11); gv_par ^= 1u << vs; fence_proxy_async(); }
                 PLM(18);
                 uint32_t vb = v_desc[0];
 #pragma unroll
@@ -334,8 +331,8 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         cp_async16(dst + off, src + c * 8, ok ? 16u : 0u);
                     }
                 }
+                cp_async_arrive((is_v ? bar_gv0 : bar_gk0) + 8 * st);   // this thread's share of the tile has landed
             }
-            cp_async_commit();
         };
         // prologue gathers: the first KST key tiles and VST value tiles (those that are retained tiles)
         if (n_win < KST) {
@@ -356,13 +353,6 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             int rk[4], rv[4];
             gather_rows(t + KST, rk);
             gather_rows(t + VST - 1, rv);
-            // gathers issued before this point have landed (all of them, or all but the latest value tile)
-            if (t >= g_first) {
-                if (VST == 3) cp_async_wait<1>(); else cp_async_wait<0>();
-                fence_proxy_async();
-                mbar_arrive(bar_g0 + 8 * ((t - g_first) & 1));
-            }
-
             // column range this row may see in the tile
             // rows of a warp are consecutive and both bounds grow with the row: its first / last row give the warp's
             // union range (columns any row sees) and intersection range (columns every row sees)
@@ -490,7 +480,7 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             mbar_arrive(bar_p);
             PLM(10);
             // value tile t+VST-1 goes into the stage of V(t-1), which PV(t-1) has finished reading
-            if (t > 0) gather_issue(t + VST - 1, true, rv); else cp_async_commit();
+            if (t > 0) gather_issue(t + VST - 1, true, rv);
             PLM(11);
         }
         mbar_wait(bar_pv, (n_tiles - 1) & 1, 5);
