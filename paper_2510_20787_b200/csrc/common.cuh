@@ -98,7 +98,10 @@ int launch_select(const Params& p, const float* z, int32_t* idx, int32_t* cnt, i
 int launch_prefill_simt(const Params& p, const void* q, const void* k, const void* v, const int32_t* idx,
                         const int32_t* cnt, void* o, float* lse, cudaStream_t st);
 int launch_prefill_tc_long(const Params& p, const void* q, const void* k, const void* v, const int32_t* idx,
-                           const int32_t* cnt, void* o, float* lse, cudaStream_t st);
+                           const int32_t* cnt, void* o, float* lse, void* ws, size_t ws_bytes, cudaStream_t st);
+size_t prefill_compact_bytes(const Params& p);
+int launch_prefill_compact(const Params& p, const void* k, const void* v, const int32_t* idx, const int32_t* cnt, void* kc, void* vc,
+                           cudaStream_t st);
 int prefill_long_status_fetch_and_clear();
 int launch_cache_init(const Params& p, const void* k, const void* v, const float* z, const int32_t* idx,
                       const int32_t* cnt, void* cache, cudaStream_t st);

@@ -8,7 +8,7 @@
 namespace lte {
 
 int launch_prefill_tc(const Params& p, const void* q, const void* k, const void* v, const int32_t* idx,
-                      const int32_t* cnt, void* o, float* lse, cudaStream_t st);
+                      const int32_t* cnt, void* o, float* lse, void* ws, size_t ws_bytes, cudaStream_t st);
 int prefill_status_fetch_and_clear();
 int decode_status_fetch_and_clear();
 int scores_status_fetch_and_clear();
@@ -98,7 +98,7 @@ CacheScorePlan cache_score_plan(const lte_shape* s, const lte_conv* c)
 }
 
 // scratch of lte_attn_prefill_chunk, sized for the longest local sequence (pool rows + full ring + chunk)
-struct ChunkPlan { size_t klin, vlin, z, zrank, zsrc, oldpos, idx, cnt, sub, total; };
+struct ChunkPlan { size_t klin, vlin, z, zrank, zsrc, oldpos, idx, cnt, sub, att, total; };
 ChunkPlan chunk_plan(const lte_shape* s, const lte_conv* c)
 {
     auto up = [](size_t x) { return (x + 255) / 256 * 256; };
@@ -119,6 +119,8 @@ ChunkPlan chunk_plan(const lte_shape* s, const lte_conv* c)
         lte_shape s2 = *s; s2.T = (int32_t)Tm;
         off += up(scores_stack_tc_workspace(make_params(&s2, c)));
     }
+    w.att = off;                                             // the attention's compacted retained rows
+    off += up(prefill_compact_bytes(make_params(s, c)));
     w.total = off;
     return w;
 }
@@ -169,6 +171,10 @@ size_t lte_workspace_bytes(int op, const lte_shape* s, const lte_conv* c)
     if (op == LTE_OP_DECODE && c && c->n_layers == 3) {
         if (check_shape(s, false) != LTE_OK) return 0;
         return cache_score_plan(s, c).total;
+    }
+    if (op == LTE_OP_PREFILL) {
+        if (check_shape(s, true) != LTE_OK) return 0;
+        return prefill_compact_bytes(make_params(s, nullptr));
     }
     if (op == LTE_OP_STATS) {
         if (check_shape(s, true) != LTE_OK) return 0;
@@ -223,13 +229,12 @@ int lte_select(const lte_shape* s, const float* z, int32_t* idx, int32_t* cnt, i
 int lte_attn_prefill(const lte_shape* s, const void* q, const void* k, const void* v, const int32_t* idx,
                      const int32_t* cnt, void* o, float* lse, void* ws, size_t ws_bytes, void* stream)
 {
-    (void)ws; (void)ws_bytes;
     int e = check_shape(s, true); if (e) return e;
     if (!q || !k || !v || !o || !lse || !cnt || (s->R > 0 && !idx)) return LTE_ERR_INVALID_ARG;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return LTE_ERR_INVALID_ARG;
     e = check_arch(); if (e) return e;
     Params p = make_params(s, nullptr);
-    if (s->dtype == LTE_BF16) return launch_prefill_tc(p, q, k, v, idx, cnt, o, lse, (cudaStream_t)stream);
+    if (s->dtype == LTE_BF16) return launch_prefill_tc(p, q, k, v, idx, cnt, o, lse, ws, ws_bytes, (cudaStream_t)stream);
     return launch_prefill_simt(p, q, k, v, idx, cnt, o, lse, (cudaStream_t)stream);
 }
 
@@ -304,7 +309,7 @@ int lte_attn_prefill_chunk(const lte_shape* s, const lte_conv* c, void* cache, i
     int32_t* oldpos = (int32_t*)(base + w.oldpos); int32_t* idx = (int32_t*)(base + w.idx); int32_t* cnt = (int32_t*)(base + w.cnt);
     e = launch_chunk_gather(p, cache, k, v, base + w.klin, base + w.vlin, zsrc, oldpos, n_past, R0, Wn, st); if (e) return e;
     if (p.stack) {
-        e = launch_scores_stack_tc(p, base + w.klin, base + w.vlin, z, nullptr, base + w.sub, w.total - w.sub, st);
+        e = launch_scores_stack_tc(p, base + w.klin, base + w.vlin, z, nullptr, base + w.sub, w.att - w.sub, st);
         if (e == LTE_ERR_UNSUPPORTED) e = launch_scores_stack(p, base + w.klin, base + w.vlin, z, nullptr, st);
     } else {
         e = launch_scores(p, base + w.klin, base + w.vlin, z, nullptr, st);
@@ -313,7 +318,7 @@ int lte_attn_prefill_chunk(const lte_shape* s, const lte_conv* c, void* cache, i
     e = launch_chunk_merge_z(p, z, zrank, zsrc, oldpos, n_past, R0, Wn, st); if (e) return e;
     e = launch_select(psel, zrank, idx, cnt, nullptr, st); if (e) return e;
     // the attention kernels take the chunk's q, o, lse as they are: query row r stands at position qoff + r
-    if (s->dtype == LTE_BF16) e = launch_prefill_tc(patt, q, base + w.klin, base + w.vlin, idx, cnt, o, lse, st);
+    if (s->dtype == LTE_BF16) e = launch_prefill_tc(patt, q, base + w.klin, base + w.vlin, idx, cnt, o, lse, base + w.att, w.total - w.att, st);
     else e = launch_prefill_simt(patt, q, base + w.klin, base + w.vlin, idx, cnt, o, lse, st);
     if (e) return e;
     return launch_chunk_commit(p, cache, base + w.klin, base + w.vlin, z, idx, cnt, oldpos, n_past, n_past + Tc, R0, Wn, st);

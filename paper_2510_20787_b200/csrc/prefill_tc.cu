@@ -587,12 +587,12 @@ int run(const Params& p, const void* q, const void* k, const void* v, const int3
 }  // namespace
 
 int launch_prefill_tc(const Params& p, const void* q, const void* k, const void* v, const int32_t* idx,
-                      const int32_t* cnt, void* o, float* lse, cudaStream_t st)
+                      const int32_t* cnt, void* o, float* lse, void* ws, size_t ws_bytes, cudaStream_t st)
 {
     switch (p.d) {
         case 64: return run<64>(p, q, k, v, idx, cnt, o, lse, st);
         // d = 128: ten and more key tiles per item; one CTA per item under the hardware scheduler is faster there
-        case 128: return launch_prefill_tc_long(p, q, k, v, idx, cnt, o, lse, st);
+        case 128: return launch_prefill_tc_long(p, q, k, v, idx, cnt, o, lse, ws, ws_bytes, st);
     }
     return launch_prefill_simt(p, q, k, v, idx, cnt, o, lse, st);   // d = 32: rows too narrow for the 128-byte swizzle
 }

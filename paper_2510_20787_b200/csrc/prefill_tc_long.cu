@@ -71,10 +71,12 @@ template <int D> struct Smem {
 //   bar_k[s], bar_v[s]       TMA transaction barriers of the window tiles
 //   bar_kf[s], bar_vf[s]     (commit) the MMA that read stage s has completed          MMA lane -> load lane
 // S(t+1) and S(t+2) are computed while the softmax of tile t runs; loads run two to three tiles ahead.
-template <int D>
+template <int D, bool compact>
 __global__ void __launch_bounds__(NTHREADS, 2)
 prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                  const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO, const __nv_bfloat16* __restrict__ kg,
+                  const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
+                  const __grid_constant__ CUtensorMap tmKc, const __grid_constant__ CUtensorMap tmVc,
+                  const __nv_bfloat16* __restrict__ kg,
                   const __nv_bfloat16* __restrict__ vg, const int32_t* __restrict__ idx,
                   const int32_t* __restrict__ cnt, __nv_bfloat16* __restrict__ o, float* __restrict__ lse, int Tlen,
                   int W, int R, float scale, int G, int qoff)
@@ -157,39 +159,35 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             mbar_expect_tx(bar_q, S::QTILE);
 #pragma unroll
             for (int sb = 0; sb < SUB; ++sb) tma_load_3d(sQ + sb * 16384, &tmQ, sb * 64, i0 - qoff, bh, bar_q);
+            // compact = 1: the retained rows were copied into contiguous tensors [B*H][R][d] beforehand (tmKc, tmVc), so the
+            // retained tiles are TMA boxes like the window tiles; otherwise the softmax warps gather them
+            const int n_load = compact ? n_tiles : n_win;
+            auto load_tile = [&](int t, bool is_v, int st) {
+                const uint32_t dst = (is_v ? sV : sK) + st * S::KVTILE;
+                const uint32_t bar = (is_v ? bar_v0 : bar_k0) + 8 * st;
+                const CUtensorMap* tm = t < n_win ? (is_v ? &tmV : &tmK) : (is_v ? &tmVc : &tmKc);
+                const int y = t < n_win ? j_start + t * BN : (t - n_win) * BN;
+                mbar_expect_tx(bar, S::KVTILE);
+#pragma unroll
+                for (int sb = 0; sb < SUB; ++sb) tma_load_3d(dst + sb * 8192, tm, sb * 64, y, bhk, bar);
+            };
             int ks = 0, vs = 0;                                // stage of the next K / V tile to load
             uint32_t kf_par = 0, vf_par = 0;                   // parity bit per stage of the "free" barriers
-            int tk = 0, tv = 0;                                // next window tile to load
-            int y = j_start;
-            for (; tk < KST && tk < n_win; ++tk, y += BN) {
-                mbar_expect_tx(bar_k0 + 8 * tk, S::KVTILE);
-#pragma unroll
-                for (int sb = 0; sb < SUB; ++sb) tma_load_3d(sK + tk * S::KVTILE + sb * 8192, &tmK, sb * 64, y, bhk, bar_k0 + 8 * tk);
-            }
-            y = j_start;
-            for (; tv < VST && tv < n_win; ++tv, y += BN) {
-                mbar_expect_tx(bar_v0 + 8 * tv, S::KVTILE);
-#pragma unroll
-                for (int sb = 0; sb < SUB; ++sb) tma_load_3d(sV + tv * S::KVTILE + sb * 8192, &tmV, sb * 64, y, bhk, bar_v0 + 8 * tv);
-            }
-            while (tk < n_win || tv < n_win) {
-                if (tk < n_win) {                              // K(tk) into the stage of K(tk - KST)
+            int tk = 0, tv = 0;                                // next tile to load
+            for (; tk < KST && tk < n_load; ++tk) load_tile(tk, false, tk);
+            for (; tv < VST && tv < n_load; ++tv) load_tile(tv, true, tv);
+            while (tk < n_load || tv < n_load) {
+                if (tk < n_load) {                             // K(tk) into the stage of K(tk - KST)
                     mbar_wait(bar_kf0 + 8 * ks, (kf_par >> ks) & 1u, 6);
                     kf_par ^= 1u << ks;
-                    mbar_expect_tx(bar_k0 + 8 * ks, S::KVTILE);
-#pragma unroll
-                    for (int sb = 0; sb < SUB; ++sb)
-                        tma_load_3d(sK + ks * S::KVTILE + sb * 8192, &tmK, sb * 64, j_start + tk * BN, bhk, bar_k0 + 8 * ks);
+                    load_tile(tk, false, ks);
                     ++tk;
                     ks = ks + 1 == KST ? 0 : ks + 1;
                 }
-                if (tv < n_win) {                              // V(tv) into the stage of V(tv - VST)
+                if (tv < n_load) {                             // V(tv) into the stage of V(tv - VST)
                     mbar_wait(bar_vf0 + 8 * vs, (vf_par >> vs) & 1u, 8);
                     vf_par ^= 1u << vs;
-                    mbar_expect_tx(bar_v0 + 8 * vs, S::KVTILE);
-#pragma unroll
-                    for (int sb = 0; sb < SUB; ++sb)
-                        tma_load_3d(sV + vs * S::KVTILE + sb * 8192, &tmV, sb * 64, j_start + tv * BN, bhk, bar_v0 + 8 * vs);
+                    load_tile(tv, true, vs);
                     ++tv;
                     vs = vs + 1 == VST ? 0 : vs + 1;
                 }
@@ -215,7 +213,7 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             int ks = 0, vs = 0;                                // stage of the next S / PV operand
             int ts = 0;                                        // next S tile to issue
             auto mma_s = [&]() {                               // S(ts) from K stage ks into S buffer ts & 1
-                if (ts < n_win) { mbar_wait(bar_k0 + 8 * ks, (k_par >> ks) & 1u, 2); k_par ^= 1u << ks; }
+                if (ts < n_win || compact) { mbar_wait(bar_k0 + 8 * ks, (k_par >> ks) & 1u, 2); k_par ^= 1u << ks; }
                 else {                                         // gathered rows: generic-proxy writes, made visible to the tensor core here
                     mbar_wait(bar_gk0 + 8 * ks, (gk_par >> ks) & 1u, 10); gk_par ^= 1u << ks;
                     fence_proxy_async();
@@ -245,7 +243,7 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 // PV(t): everything but P is normally there long before
                 PLM(17);
                 PLM_TILE(t);
-                if (t < n_win) { mbar_wait(bar_v0 + 8 * vs, (v_par >> vs) & 1u, 4); v_par ^= 1u << vs; }
+                if (t < n_win || compact) { mbar_wait(bar_v0 + 8 * vs, (v_par >> vs) & 1u, 4); v_par ^= 1u << vs; }
                 else { mbar_wait(bar_gv0 + 8 * vs, (gv_par >> vs) & 1u, 11); gv_par ^= 1u << vs; fence_proxy_async(); }
                 PLM(18);
                 uint32_t vb = v_desc[0];
@@ -313,11 +311,11 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 #pragma unroll
             for (int ps = 0; ps < 4; ++ps) {
                 const int e = (t - n_win) * BN + ps * 16 + g_row;
-                rows4[ps] = (t >= n_win && t < n_tiles && e < nv_max) ? id[e] : -1;
+                rows4[ps] = (!compact && t >= n_win && t < n_tiles && e < nv_max) ? id[e] : -1;
             }
         };
         auto gather_issue = [&](int t, bool is_v, const int (&rows4)[4]) {
-            if (t >= n_win && t < n_tiles) {
+            if (!compact && t >= n_win && t < n_tiles) {
                 const int st = is_v ? (t % VST) : (t % KST);
                 const uint32_t dst = (is_v ? sV : sK) + st * S::KVTILE;
 #pragma unroll
@@ -535,36 +533,88 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     if (warp == 4) tmem_dealloc(tmem, TMEM_COLS);
 }
 
+// Retained rows into contiguous tensors kc, vc [B*H][R][d] (list order; rows past the head's count are zero), so that the
+// attention kernels can fetch retained tiles as TMA boxes instead of gathering rows (Section 3.1.3: the retained keys
+// and values are compacted into a contiguous span when the cache is filled).  Block (32-row part, head).
+__global__ void prefill_compact_kernel(const uint4* __restrict__ k, const uint4* __restrict__ v, const int32_t* __restrict__ idx,
+                                       const int32_t* __restrict__ cnt, uint4* __restrict__ kc, uint4* __restrict__ vc, int Tlen,
+                                       int R, int pieces)
+{
+    pdl_launch_dependents();
+    pdl_wait();
+    const int bhk = blockIdx.y, n = cnt[bhk];
+    const int e_lo = blockIdx.x * 32, e_hi = min(e_lo + 32, R);
+    for (int x = e_lo * pieces + threadIdx.x; x < e_hi * pieces; x += blockDim.x) {
+        const int e = x / pieces, c = x - e * pieces;
+        uint4 a = make_uint4(0, 0, 0, 0), b = a;
+        if (e < n) {
+            const size_t src = ((size_t)bhk * Tlen + idx[(size_t)bhk * R + e]) * pieces + c;
+            a = k[src]; b = v[src];
+        }
+        kc[((size_t)bhk * R + e) * pieces + c] = a;
+        vc[((size_t)bhk * R + e) * pieces + c] = b;
+    }
+}
+
 template <int D>
 int run(const Params& p, const void* q, const void* k, const void* v, const int32_t* idx, const int32_t* cnt, void* o,
-        float* lse, cudaStream_t st)
+        float* lse, void* ws, size_t ws_bytes, cudaStream_t st)
 {
-    CUtensorMap tq, tk, tv, to;
+    CUtensorMap tq, tk, tv, to, tkc, tvc;
     const int BHK = p.B * p.H, BH = BHK * p.G;                 // key/value heads, query heads
     const int Tq = p.T - p.qoff;                               // query rows
     if (!make_map(&tq, q, BH, Tq, D, BM) || !make_map(&tk, k, BHK, p.T, D, BN) || !make_map(&tv, v, BHK, p.T, D, BN) ||
         !make_map(&to, o, BH, Tq, D, 32))
         return LTE_ERR_CUDA;
+    // with a workspace the retained rows are compacted first and every tile is a TMA box
+    const size_t half = prefill_compact_bytes(p) / 2;
+    const int compact = (ws != nullptr && half > 0 && ws_bytes >= 2 * half && ((uintptr_t)ws & 127u) == 0) ? 1 : 0;
+    tkc = tk; tvc = tv;
+    if (compact) {
+        char* kc = (char*)ws; char* vc = kc + half;
+        if (int e = launch_prefill_compact(p, k, v, idx, cnt, kc, vc, st)) return e;
+        if (!make_map(&tkc, kc, BHK, p.R, D, BN) || !make_map(&tvc, vc, BHK, p.R, D, BN)) return LTE_ERR_CUDA;
+    }
     static bool attr_done = false;
     if (!attr_done) {
-        if (cudaFuncSetAttribute(prefill_long_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::BYTES) !=
-            cudaSuccess)
+        if (cudaFuncSetAttribute(prefill_long_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::BYTES) != cudaSuccess ||
+            cudaFuncSetAttribute(prefill_long_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::BYTES) != cudaSuccess)
             return LTE_ERR_CUDA;
         attr_done = true;
     }
     dim3 grid((Tq + BM - 1) / BM, BH);
-    return cuda_status(launch_pdl(prefill_long_kernel<D>, grid, dim3(NTHREADS), Smem<D>::BYTES, st, tq, tk, tv, to, (const __nv_bfloat16*)k,
+    if (compact)
+        return cuda_status(launch_pdl(prefill_long_kernel<D, true>, grid, dim3(NTHREADS), Smem<D>::BYTES, st, tq, tk, tv, to, tkc, tvc, (const __nv_bfloat16*)k,
+                                                                 (const __nv_bfloat16*)v, idx, cnt, (__nv_bfloat16*)o,
+                                                                 lse, p.T, p.W, p.R, p.scale, p.G, p.qoff));
+    return cuda_status(launch_pdl(prefill_long_kernel<D, false>, grid, dim3(NTHREADS), Smem<D>::BYTES, st, tq, tk, tv, to, tkc, tvc, (const __nv_bfloat16*)k,
                                                                  (const __nv_bfloat16*)v, idx, cnt, (__nv_bfloat16*)o,
                                                                  lse, p.T, p.W, p.R, p.scale, p.G, p.qoff));
 }
 
 }  // namespace
 
+// bytes of the two compacted tensors (keys, then values), each a multiple of 128; 0 where there is nothing to compact
+size_t prefill_compact_bytes(const Params& p)
+{
+    if (p.dtype != LTE_BF16 || (p.d != 64 && p.d != 128) || p.R <= 0) return 0;
+    const size_t one = ((size_t)p.B * p.H * p.R * p.d * 2 + 127) / 128 * 128;
+    return 2 * one;
+}
+
+int launch_prefill_compact(const Params& p, const void* k, const void* v, const int32_t* idx, const int32_t* cnt, void* kc, void* vc,
+                           cudaStream_t st)
+{
+    dim3 grid((p.R + 31) / 32, p.B * p.H);
+    return cuda_status(launch_pdl(prefill_compact_kernel, grid, dim3(256), 0, st, (const uint4*)k, (const uint4*)v, idx, cnt, (uint4*)kc,
+                                  (uint4*)vc, p.T, p.R, p.d * 2 / 16));
+}
+
 int launch_prefill_tc_long(const Params& p, const void* q, const void* k, const void* v, const int32_t* idx,
-                           const int32_t* cnt, void* o, float* lse, cudaStream_t st)
+                           const int32_t* cnt, void* o, float* lse, void* ws, size_t ws_bytes, cudaStream_t st)
 {
     if (p.d != 128) return LTE_ERR_UNSUPPORTED;
-    return run<128>(p, q, k, v, idx, cnt, o, lse, st);
+    return run<128>(p, q, k, v, idx, cnt, o, lse, ws, ws_bytes, st);
 }
 
 #ifdef LTE_PROFILE

@@ -170,15 +170,21 @@ def lte_select(s, z, idx=None, cnt=None, ncand=None):
     return idx, cnt
 
 
-def lte_attn_prefill(s, q, k, v, idx, cnt, o=None, lse=None):
-    """q [B,H*group,T,d], k, v [B,H,T,d], retained list -> o [B,H*group,T,d], lse [B,H*group,T] fp32."""
+def lte_attn_prefill(s, q, k, v, idx, cnt, o=None, lse=None, ws=None):
+    """q [B,H*group,T,d], k, v [B,H,T,d], retained list -> o [B,H*group,T,d], lse [B,H*group,T] fp32.
+    ws: uint8 tensor of lte_workspace_bytes(OP_PREFILL, s) bytes (the retained rows are compacted into it and fetched
+    as tiles), allocated here when None; False: no workspace (the kernels gather the retained rows themselves)."""
     if o is None:
         o = torch.empty_like(q)
     if lse is None:
         lse = torch.empty((s.B, s.H * max(s.group, 1), s.T), dtype=torch.float32, device=q.device)
+    if ws is None:
+        need = lte_workspace_bytes(OP_PREFILL, s, None)
+        ws = torch.empty(need, dtype=torch.uint8, device=q.device) if need > 0 else False
+    wp, wn = (None, 0) if ws is False else (_ptr(ws), ws.numel())
     _check("lte_attn_prefill", lib().lte_attn_prefill(ctypes.addressof(s), _ptr(q), _ptr(k), _ptr(v),
                                                       _ptr(idx, torch.int32), _ptr(cnt, torch.int32), _ptr(o),
-                                                      _ptr(lse, torch.float32), None, 0, _stream()))
+                                                      _ptr(lse, torch.float32), wp, wn, _stream()))
     return o, lse
 
 
