@@ -106,6 +106,18 @@ def device_inputs(cfg, seed, torch, T=None, with_dO=False):
     return out
 
 
+_PREFILL_WS = {}
+
+
+def prefill_ws(torch, lte, s):
+    """The prefill attention's workspace (compacted retained rows) for a shape, allocated once."""
+    key = (s.B, s.H, s.R, s.d, s.dtype)
+    if key not in _PREFILL_WS:
+        need = lte.lte_workspace_bytes(lte.OP_PREFILL, s, None)
+        _PREFILL_WS[key] = torch.empty(need, dtype=torch.uint8, device="cuda") if need > 0 else False
+    return _PREFILL_WS[key]
+
+
 def timed(torch, fn, steps, warmup, flush, sub_events=0):
     """Run fn() warmup + steps times; returns per-step ms list and, if fn returns event lists, their deltas."""
     for _ in range(warmup):
@@ -209,14 +221,14 @@ def run_lte(args):
     def step():                               # the three calls as a user makes them: nothing between the launches
         lte.lte_scores(s, c, k, v, z=z)
         lte.lte_select(s, z, idx=idx, cnt=cnt)
-        lte.lte_attn_prefill(s, q, k, v, idx, cnt, o=o, lse=lse)
+        lte.lte_attn_prefill(s, q, k, v, idx, cnt, o=o, lse=lse, ws=prefill_ws(torch, lte, s))
         return None
 
     def step_marked():                        # the same step with an event after every launch (per-kernel durations)
         m = [ev()]
         lte.lte_scores(s, c, k, v, z=z); m.append(ev())
         lte.lte_select(s, z, idx=idx, cnt=cnt); m.append(ev())
-        lte.lte_attn_prefill(s, q, k, v, idx, cnt, o=o, lse=lse); m.append(ev())
+        lte.lte_attn_prefill(s, q, k, v, idx, cnt, o=o, lse=lse, ws=prefill_ws(torch, lte, s)); m.append(ev())
         return m
 
     def barrier():
@@ -286,7 +298,7 @@ def run_lte(args):
             lte.lte_scores(s1, c, dk_[sl], dv_[sl], z=z[sl])
             lte.lte_select(s1, z[sl], idx=idx[sl], cnt=cnt[sl])
             cur.wait_event(ev_q[b])
-            lte.lte_attn_prefill(s1, dq_[sl], dk_[sl], dv_[sl], idx[sl], cnt[sl], o=o[sl], lse=lse[sl])
+            lte.lte_attn_prefill(s1, dq_[sl], dk_[sl], dv_[sl], idx[sl], cnt[sl], o=o[sl], lse=lse[sl], ws=prefill_ws(torch, lte, s1))
             ev_done[b].record(cur)
             with torch.cuda.stream(st_out):
                 st_out.wait_event(ev_done[b])
@@ -324,9 +336,9 @@ def run_lte(args):
                        "parallelism": "replicas x%d (independent (batch, head) units)" % world},
             "e2e": {"value": tokens / (e2e_ms * 1e-3), "unit": "tokens/s", "ms_per_step": e2e_ms,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-            "gpu_launches": 3 * args.steps, "roofline": roof, "wall_s": t_wall,
+            "gpu_launches": 4 * args.steps, "roofline": roof, "wall_s": t_wall,
             "ms_per_step_marked": float(np.mean(ms_marked)),
-            "timing_note": "value: K steps of three back-to-back launches; roofline.kernel_ms: a second pass of K steps with an event after every launch"}
+            "timing_note": "value: K steps of three back-to-back calls (four launches: scores, select, compaction of the retained rows, attention); roofline.kernel_ms: a second pass of K steps with an event after every call (lte_attn_prefill = compaction + attention kernel)"}
     if rank == 0:
         line["clocks"] = clocks
 
@@ -407,7 +419,7 @@ def _extra_k(out, torch, lte, synth, pk, flush, n5):
 
         def one_shot():
             lte.lte_scores(s1, c, kc, vc, z=z1); lte.lte_select(s1, z1, idx=i1, cnt=c1)
-            lte.lte_attn_prefill(s1, qc, kc, vc, i1, c1, o=o, lse=lse)
+            lte.lte_attn_prefill(s1, qc, kc, vc, i1, c1, o=o, lse=lse, ws=prefill_ws(torch, lte, s1))
 
         ms1, _ = timed(torch, one_shot, n5, 3, flush)
         t = mid3(ms) * 1e-3
@@ -470,7 +482,7 @@ def _extra_s(out, torch, lte, synth, pk, flush, n5):
     s5 = lte.shape(cfg5.B, cfg5.H, cfg5.T, cfg5.d, cfg5.W, cfg5.R, lte.BF16)
     z5 = lte.lte_scores(s5, c, x5["k"], x5["v"])
     idx5, cnt5 = lte.lte_select(s5, z5)
-    o5, lse5 = lte.lte_attn_prefill(s5, x5["q"], x5["k"], x5["v"], idx5, cnt5)
+    o5, lse5 = lte.lte_attn_prefill(s5, x5["q"], x5["k"], x5["v"], idx5, cnt5, ws=prefill_ws(torch, lte, s5))
     ws5 = torch.empty(lte.lte_workspace_bytes(lte.OP_BWD, s5, c), dtype=torch.uint8, device="cuda")
     c1 = lte.conv(x5["w"])
     ws1 = torch.empty(lte.lte_workspace_bytes(lte.OP_BWD, s5, c1), dtype=torch.uint8, device="cuda")
@@ -541,10 +553,10 @@ def _extra_p(out, torch, lte, synth, pk, flush, n5):
     def step():
         lte.lte_scores(s, c, x["k"], x["v"], z=z)
         lte.lte_select(s, z, idx=idx, cnt=cnt)
-        lte.lte_attn_prefill(s, x["q"], x["k"], x["v"], idx, cnt, o=o, lse=lse)
+        lte.lte_attn_prefill(s, x["q"], x["k"], x["v"], idx, cnt, o=o, lse=lse, ws=prefill_ws(torch, lte, s))
 
     def f_attn():
-        lte.lte_attn_prefill(s, x["q"], x["k"], x["v"], idx, cnt, o=o, lse=lse)
+        lte.lte_attn_prefill(s, x["q"], x["k"], x["v"], idx, cnt, o=o, lse=lse, ws=prefill_ws(torch, lte, s))
 
     ms, _ = timed(torch, step, n5, 3, flush)
     ms_a, _ = timed(torch, f_attn, n5, 3, flush)
@@ -596,10 +608,10 @@ def _extra_p(out, torch, lte, synth, pk, flush, n5):
     def step_g():
         lte.lte_scores(sg, cg, kg, vg, z=zg)
         lte.lte_select(sg, zg, idx=idxg, cnt=cntg)
-        lte.lte_attn_prefill(sg, qg, kg, vg, idxg, cntg, o=og, lse=lseg)
+        lte.lte_attn_prefill(sg, qg, kg, vg, idxg, cntg, o=og, lse=lseg, ws=prefill_ws(torch, lte, sg))
 
     def attn_g():
-        lte.lte_attn_prefill(sg, qg, kg, vg, idxg, cntg, o=og, lse=lseg)
+        lte.lte_attn_prefill(sg, qg, kg, vg, idxg, cntg, o=og, lse=lseg, ws=prefill_ws(torch, lte, sg))
 
     tg, tag = mid3(timed(torch, step_g, n5, 3, flush)[0]) * 1e-3, mid3(timed(torch, attn_g, n5, 3, flush)[0]) * 1e-3
     flg = attn_flops(idxg, cntg, cfg.T, cfg.W, cfg.d, torch) * G
@@ -641,7 +653,7 @@ def _extra_c3(out, torch, lte, synth, pk, flush, n5):
     idx, cnt = lte.lte_select(s, z)
     o = torch.empty_like(x["q"]); lse = torch.empty((cfg.B, cfg.H, cfg.T), dtype=torch.float32, device="cuda")
     def f_attn():
-        lte.lte_attn_prefill(s, x["q"], x["k"], x["v"], idx, cnt, o=o, lse=lse)
+        lte.lte_attn_prefill(s, x["q"], x["k"], x["v"], idx, cnt, o=o, lse=lse, ws=prefill_ws(torch, lte, s))
 
     def f_scores():
         lte.lte_scores(s, c, x["k"], x["v"], z=z)
@@ -680,12 +692,12 @@ def _extra_c5(out, torch, lte, synth, pk, flush, n5):
     c = lte.conv(x["w"])
     z = lte.lte_scores(s, c, x["k"], x["v"])
     idx, cnt = lte.lte_select(s, z)
-    o, lse = lte.lte_attn_prefill(s, x["q"], x["k"], x["v"], idx, cnt)
+    o, lse = lte.lte_attn_prefill(s, x["q"], x["k"], x["v"], idx, cnt, ws=prefill_ws(torch, lte, s))
     ws = torch.empty(lte.lte_workspace_bytes(lte.OP_BWD, s, c), dtype=torch.uint8, device="cuda")
 
     def fwd():
         lte.lte_scores(s, c, x["k"], x["v"], z=z); lte.lte_select(s, z, idx=idx, cnt=cnt)
-        lte.lte_attn_prefill(s, x["q"], x["k"], x["v"], idx, cnt, o=o, lse=lse)
+        lte.lte_attn_prefill(s, x["q"], x["k"], x["v"], idx, cnt, o=o, lse=lse, ws=prefill_ws(torch, lte, s))
 
     def bwd():
         lte.lte_attn_bwd(s, c, x["q"], x["k"], x["v"], o, lse, x["dO"], z, idx, cnt, ws=ws)

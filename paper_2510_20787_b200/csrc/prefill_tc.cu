@@ -95,10 +95,14 @@ __device__ __forceinline__ int count_le(const int32_t* id, int n, int lim, int l
 //   bar_k[s], bar_v[s]       TMA transaction barriers of the window tiles (one phase per TMA use of the stage)
 //   bar_kf[s], bar_vf[s]     (commit) the MMA that read the stage's tile g has completed   phase g / stages   MMA -> load
 // S(g+1) and S(g+2) are computed while the softmax of tile g runs; loads run two to three tiles ahead, across items.
-template <int D>
+// COMPACT: the retained rows were copied into contiguous tensors [B*H][R][d] beforehand (tmKc, tmVc), so retained tiles are
+// TMA boxes like the window tiles and the softmax warps gather nothing (a compile-time variant: the gather code costs the
+// softmax loop instruction-cache room even where it does not run).
+template <int D, bool COMPACT>
 __global__ void __launch_bounds__(NTHREADS, 2)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                   const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
+                  const __grid_constant__ CUtensorMap tmKc, const __grid_constant__ CUtensorMap tmVc,
                   const __nv_bfloat16* __restrict__ kg,
                   const __nv_bfloat16* __restrict__ vg, const int32_t* __restrict__ idx,
                   const int32_t* __restrict__ cnt, float* __restrict__ lse, int Tlen,
@@ -170,25 +174,31 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 mbar_expect_tx(bar_q, S::QTILE);
 #pragma unroll
                 for (int sb = 0; sb < SUB; ++sb) tma_load_3d(sQ + sb * 16384, &tmQ, sb * 64, w.i0 - qoff, w.bh, bar_q);
-                // window tiles, each into its stage as soon as the MMA that read the stage's previous tile has completed
-                for (int t = 0; t < w.n_win; ++t) {
+            }
+            // tiles, each into its stage as soon as the MMA that read the stage's previous tile has completed
+            auto load_tiles = [&](int t_lo, int t_hi) {
+                for (int t = t_lo; t < t_hi; ++t) {
                     const uint32_t gg = g + t;
-                    const int y = w.j_start + t * BN;
+                    const bool win = t < w.n_win;
+                    const int y = win ? w.j_start + t * BN : (t - w.n_win) * BN;
                     const uint32_t ks = gg % KST, vs = gg % VST;
                     if (gg >= (uint32_t)KST) mbar_wait(bar_kf0 + 8 * ks, (gg / KST - 1) & 1u, 6);
                     mbar_expect_tx(bar_k0 + 8 * ks, S::KVTILE);
 #pragma unroll
                     for (int sb = 0; sb < SUB; ++sb)
-                        tma_load_3d(sK + ks * S::KVTILE + sb * 8192, &tmK, sb * 64, y, w.bhk, bar_k0 + 8 * ks);
+                        tma_load_3d(sK + ks * S::KVTILE + sb * 8192, win ? &tmK : &tmKc, sb * 64, y, w.bhk, bar_k0 + 8 * ks);
                     if (gg >= (uint32_t)VST) mbar_wait(bar_vf0 + 8 * vs, (gg / VST - 1) & 1u, 8);
                     mbar_expect_tx(bar_v0 + 8 * vs, S::KVTILE);
 #pragma unroll
                     for (int sb = 0; sb < SUB; ++sb)
-                        tma_load_3d(sV + vs * S::KVTILE + sb * 8192, &tmV, sb * 64, y, w.bhk, bar_v0 + 8 * vs);
+                        tma_load_3d(sV + vs * S::KVTILE + sb * 8192, win ? &tmV : &tmVc, sb * 64, y, w.bhk, bar_v0 + 8 * vs);
                 }
-            }
-            // the item's retained tiles also take tile numbers (counted after the loads are on their way)
-            g += w.n_win + (count_le(idx + (size_t)w.bhk * R, cnt[w.bhk], w.i_hi - W, lane) + BN - 1) / BN;
+            };
+            if (lane == 0) load_tiles(0, w.n_win);
+            // the item's retained tiles also take tile numbers (counted after the window loads are on their way)
+            const int n_ret_tiles = (count_le(idx + (size_t)w.bhk * R, cnt[w.bhk], w.i_hi - W, lane) + BN - 1) / BN;
+            if (COMPACT && lane == 0) load_tiles(w.n_win, w.n_win + n_ret_tiles);
+            g += w.n_win + n_ret_tiles;
         }
     } else if (warp == 4) {
         // ================================= MMA warp (lane 0 issues) =========================================
@@ -220,7 +230,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             };
             auto mma_s = [&]() {                           // S of the item's tile ts
                 const uint32_t gg = g + ts, ks = gg % KST;
-                if (ts < w.n_win) { mbar_wait(bar_k0 + 8 * ks, (k_par >> ks) & 1u, 2); k_par ^= 1u << ks; }
+                if (COMPACT || ts < w.n_win) { mbar_wait(bar_k0 + 8 * ks, (k_par >> ks) & 1u, 2); k_par ^= 1u << ks; }
                 else need_g(g + max(ts - (KST == 2 ? 1 : 2), 0));   // a gathered K tile: issued in tile ts - KST or in the item's prologue
                 tc_fence_after();
                 const uint32_t kb = k_lo + ks * (S::KVTILE >> 4);
@@ -246,8 +256,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             {
                 for (int t = 0; t < n_tiles; ++t) {
                     const uint32_t gg = g + t, vs = gg % VST;
-                    need_g(gg);
-                    if (t < w.n_win) { mbar_wait(bar_v0 + 8 * vs, (v_par >> vs) & 1u, 4); v_par ^= 1u << vs; }
+                    if (!COMPACT) need_g(gg);
+                    if (COMPACT || t < w.n_win) { mbar_wait(bar_v0 + 8 * vs, (v_par >> vs) & 1u, 4); v_par ^= 1u << vs; }
                     // value operand: the second 64-column group of B is the next sub-tile (d = 128) or the block of
                     // ones (d = 64, LBO = its distance from the value stage)
                     const uint32_t va = sV + vs * S::KVTILE;
@@ -357,30 +367,32 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             };
             // prologue gathers: the first KST key tiles and VST value tiles, where those are retained tiles.  Their
             // stages are free: every product of the previous item has completed (its last bar_s and bar_pv were awaited).
-            if (n_win < KST) {
+            if (!COMPACT && n_win < KST) {
                 int rows4[4];
                 for (int t = 0; t < KST; ++t) { gather_rows(t, rows4); gather_issue(t, false, rows4); }
                 for (int t = 0; t < VST; ++t) { gather_rows(t, rows4); gather_issue(t, true, rows4); }
             }
             float m_run = -INFINITY, l_run = 0.f;              // running max (log2 domain) and sum (sum only if !ONES)
-            bool gathered = n_win < KST;                       // some gather of this item may be in flight (warp-uniform)
+            bool gathered = !COMPACT && n_win < KST;           // some gather of this item may be in flight (warp-uniform)
 
             for (int t = 0; t < n_tiles; ++t) {
                 const uint32_t gg = g + t;
                 // row positions for this tile's two gathers, fetched first so their latency hides under the softmax
                 // (all of this tile's gather work sits behind warp-uniform tests: most tiles of a short list have none)
-                const bool k_gather = t + KST >= n_win && t + KST < n_tiles;
-                const bool v_gather = t > 0 && t + VST - 1 >= n_win && t + VST - 1 < n_tiles;
+                const bool k_gather = !COMPACT && t + KST >= n_win && t + KST < n_tiles;
+                const bool v_gather = !COMPACT && t > 0 && t + VST - 1 >= n_win && t + VST - 1 < n_tiles;
                 int rk[4], rv[4];
                 if (k_gather) gather_rows(t + KST, rk);
                 if (v_gather) gather_rows(t + VST - 1, rv);
-                // gathers issued before this point have landed (all of them, or all but the latest value tile)
-                if (gathered) {
-                    if (VST == 3) cp_async_wait<1>(); else cp_async_wait<0>();
-                    fence_proxy_async();
+                if (!COMPACT) {
+                    // gathers issued before this point have landed (all of them, or all but the latest value tile)
+                    if (gathered) {
+                        if (VST == 3) cp_async_wait<1>(); else cp_async_wait<0>();
+                        fence_proxy_async();
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_g0 + 8 * (gg & 1));
                 }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_g0 + 8 * (gg & 1));
 
                 // column range this row may see in the tile
                 int c_lo, c_hi;
@@ -419,7 +431,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 mbar_wait(bar_s0 + 8 * (gg & 1), (gg >> 1) & 1, 3);   // S is in TMEM buffer gg & 1
                 tc_fence_after();
                 if (k_gather) { gather_issue(t + KST, false, rk); gathered = true; }   // its stage held this tile's K, which S has finished reading
-                else cp_async_commit();
+                else if (!COMPACT) cp_async_commit();
                 const uint32_t s_col = (gg & 1) * BN;
                 uint32_t r[2][32];
 #pragma unroll
@@ -498,7 +510,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 if (lane == 0) mbar_arrive(bar_p);
                 // value tile t+VST-1 goes into the stage of tile t-1's V, which that PV has finished reading
                 if (v_gather) { gather_issue(t + VST - 1, true, rv); gathered = true; }
-                else cp_async_commit();
+                else if (!COMPACT) cp_async_commit();
             }
             mbar_wait(bar_pv, (g + n_tiles - 1) & 1, 5);
             tc_fence_after();
@@ -558,18 +570,27 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 
 template <int D>
 int run(const Params& p, const void* q, const void* k, const void* v, const int32_t* idx, const int32_t* cnt, void* o,
-        float* lse, cudaStream_t st)
+        float* lse, void* ws, size_t ws_bytes, cudaStream_t st)
 {
-    CUtensorMap tq, tk, tv, to;
+    CUtensorMap tq, tk, tv, to, tkc, tvc;
     const int BHK = p.B * p.H, BH = BHK * p.G;                 // key/value heads, query heads
     const int Tq = p.T - p.qoff;                               // query rows (the whole sequence unless a chunk is prefilled)
     if (!make_map(&tq, q, BH, Tq, D, BM) || !make_map(&tk, k, BHK, p.T, D, BN) || !make_map(&tv, v, BHK, p.T, D, BN) ||
         !make_map(&to, o, BH, Tq, D, 32))
         return LTE_ERR_CUDA;
+    // with a workspace the retained rows are compacted first and every tile is a TMA box
+    const size_t half = prefill_compact_bytes(p) / 2;
+    const bool compact = ws != nullptr && half > 0 && ws_bytes >= 2 * half && ((uintptr_t)ws & 127u) == 0;
+    tkc = tk; tvc = tv;
+    if (compact) {
+        char* kc = (char*)ws; char* vc = kc + half;
+        if (int e = launch_prefill_compact(p, k, v, idx, cnt, kc, vc, st)) return e;
+        if (!make_map(&tkc, kc, BHK, p.R, D, BN) || !make_map(&tvc, vc, BHK, p.R, D, BN)) return LTE_ERR_CUDA;
+    }
     static int slots = 0;                                      // resident CTAs: two per SM
     if (slots == 0) {
-        if (cudaFuncSetAttribute(prefill_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::BYTES) !=
-            cudaSuccess)
+        if (cudaFuncSetAttribute(prefill_tc_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::BYTES) != cudaSuccess ||
+            cudaFuncSetAttribute(prefill_tc_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::BYTES) != cudaSuccess)
             return LTE_ERR_CUDA;
         int dev = 0, sms = 0;
         if (cudaGetDevice(&dev) != cudaSuccess ||
@@ -579,9 +600,13 @@ int run(const Params& p, const void* q, const void* k, const void* v, const int3
     }
     const int n_qt = (Tq + BM - 1) / BM, n_items = n_qt * BH;
     const int grid = n_items < slots ? n_items : slots;
-    return cuda_status(launch_pdl(prefill_tc_kernel<D>, dim3(grid), dim3(NTHREADS), Smem<D>::BYTES, st, tq, tk, tv, to, (const __nv_bfloat16*)k,
-                                                                 (const __nv_bfloat16*)v, idx, cnt,
-                                                                 lse, p.T, p.W, p.R, p.scale, n_qt, BH, p.G, p.qoff));
+    if (compact)
+        return cuda_status(launch_pdl(prefill_tc_kernel<D, true>, dim3(grid), dim3(NTHREADS), Smem<D>::BYTES, st, tq, tk, tv, to, tkc, tvc,
+                                      (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, idx, cnt, lse, p.T, p.W, p.R, p.scale, n_qt,
+                                      BH, p.G, p.qoff));
+    return cuda_status(launch_pdl(prefill_tc_kernel<D, false>, dim3(grid), dim3(NTHREADS), Smem<D>::BYTES, st, tq, tk, tv, to, tkc, tvc,
+                                  (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, idx, cnt, lse, p.T, p.W, p.R, p.scale, n_qt, BH,
+                                  p.G, p.qoff));
 }
 
 }  // namespace
@@ -590,7 +615,7 @@ int launch_prefill_tc(const Params& p, const void* q, const void* k, const void*
                       const int32_t* cnt, void* o, float* lse, void* ws, size_t ws_bytes, cudaStream_t st)
 {
     switch (p.d) {
-        case 64: return run<64>(p, q, k, v, idx, cnt, o, lse, st);
+        case 64: return run<64>(p, q, k, v, idx, cnt, o, lse, ws, ws_bytes, st);
         // d = 128: ten and more key tiles per item; one CTA per item under the hardware scheduler is faster there
         case 128: return launch_prefill_tc_long(p, q, k, v, idx, cnt, o, lse, ws, ws_bytes, st);
     }

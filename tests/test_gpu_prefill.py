@@ -143,3 +143,25 @@ def test_caller_made_list_uniform_stride(dtype, d, T, W, R):
     torch.cuda.synchronize()
     o64, l64 = orc.attn_prefill(x["q"], x["k"], x["v"], idx, cnt, W)
     _assert_close(cfg, (o.float().cpu().numpy(), lse.cpu().numpy(), o64, l64))
+
+
+@pytest.mark.parametrize("d,T,W,R", [(64, 1100, 96, 200), (128, 900, 64, 130), (64, 300, 40, 0)])
+def test_compacted_and_gathered_retained_rows_agree(d, T, W, R):
+    """With a workspace the retained rows are compacted and fetched as tiles, without one they are gathered row by row:
+    two kernels variants, the same numbers (bit for bit: the products and their order are the same)."""
+    cfg = synth.Config("cmp", "bf16", 2, 3, d, T, W, R, 7, 0.1)
+    x = synth.make(cfg, 12)
+    s = shape_of(cfg)
+    c = lte.conv(torch.from_numpy(x["w"]).cuda())
+    q, k, v = (dev(x[t], "bf16") for t in "qkv")
+    z = lte.lte_scores(s, c, k, v)
+    idx, cnt = lte.lte_select(s, z)
+    need = lte.lte_workspace_bytes(lte.OP_PREFILL, s, None)
+    assert need == (0 if R == 0 else 2 * ((cfg.B * cfg.H * R * d * 2 + 127) // 128 * 128))
+    o1, l1 = lte.lte_attn_prefill(s, q, k, v, idx, cnt, ws=False)
+    o2, l2 = lte.lte_attn_prefill(s, q, k, v, idx, cnt)                      # allocates the workspace
+    ws = torch.empty(need + 128, dtype=torch.uint8, device="cuda")
+    o3, l3 = lte.lte_attn_prefill(s, q, k, v, idx, cnt, ws=ws[64:64 + max(need, 1)] if need else False)   # misaligned: falls back to gathering
+    torch.cuda.synchronize()
+    assert lte.lib().lte_device_status() == 0
+    assert torch.equal(o1, o2) and torch.equal(l1, l2) and torch.equal(o1, o3)
