@@ -464,8 +464,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 if (__any_sync(0xffffffffu, need)) {
                     // PV of the previous tile must be done before O is rescaled
                     if (t > 0) { mbar_wait(bar_pv, (gg - 1) & 1, 4); tc_fence_after(); }
-#pragma unroll
-                    for (int cb = 0; cb < D / 32 + (S::ONES ? 1 : 0); ++cb) {   // with ONES the row-sum columns are rescaled too
+#pragma unroll 1
+                    for (int cb = 0; cb < D / 32 + (S::ONES ? 1 : 0); ++cb) {   // with ONES the row-sum columns are rescaled too (rolled: rarely taken, and the loop is sensitive to its code size)
                         uint32_t q4[32];
                         tmem_ld32(tmem + lane_base + O_COL + cb * 32, q4);
                         tmem_wait_ld();

@@ -137,6 +137,23 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const uint32_t tmem = *tmem_slot_gen;
     pdl_launch_dependents();
     pdl_wait();                                                // everything above ran beside the previous kernel's tail
+    // Q and the first window tiles need nothing but the tile's coordinates: they are on their way before the list is looked at
+    const int n_early = min(n_win, Smem<D>::VST);
+    if (warp == 5 && lane == 0) {
+        mbar_expect_tx(bar_q, S::QTILE);
+#pragma unroll
+        for (int sb = 0; sb < SUB; ++sb) tma_load_3d(sQ + sb * 16384, &tmQ, sb * 64, i0 - qoff, bh, bar_q);
+        for (int t = 0; t < n_early; ++t) {
+            mbar_expect_tx(bar_k0 + 8 * t, S::KVTILE);
+            mbar_expect_tx(bar_v0 + 8 * t, S::KVTILE);
+#pragma unroll
+            for (int sb = 0; sb < SUB; ++sb) {
+                tma_load_3d(sK + t * S::KVTILE + sb * 8192, &tmK, sb * 64, j_start + t * BN, bhk, bar_k0 + 8 * t);
+                tma_load_3d(sV + t * S::KVTILE + sb * 8192, &tmV, sb * 64, j_start + t * BN, bhk, bar_v0 + 8 * t);
+            }
+        }
+    }
+    __syncwarp();
     const int n_ret = cnt[bhk];
 
     if (warp >= 4) {
@@ -156,9 +173,6 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         if (warp == 5 && lane == 0) {
             // ---- load lane: Q, then the window tiles, each into its stage as soon as the MMA that read the
             //      stage's previous tile has completed (bar_kf / bar_vf, one phase per use of a stage)
-            mbar_expect_tx(bar_q, S::QTILE);
-#pragma unroll
-            for (int sb = 0; sb < SUB; ++sb) tma_load_3d(sQ + sb * 16384, &tmQ, sb * 64, i0 - qoff, bh, bar_q);
             // compact = 1: the retained rows were copied into contiguous tensors [B*H][R][d] beforehand (tmKc, tmVc), so the
             // retained tiles are TMA boxes like the window tiles; otherwise the softmax warps gather them
             const int n_load = compact ? n_tiles : n_win;
@@ -173,7 +187,7 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             };
             int ks = 0, vs = 0;                                // stage of the next K / V tile to load
             uint32_t kf_par = 0, vf_par = 0;                   // parity bit per stage of the "free" barriers
-            int tk = 0, tv = 0;                                // next tile to load
+            int tk = n_early, tv = n_early;                    // next tile to load (the first ones are already on their way)
             for (; tk < KST && tk < n_load; ++tk) load_tile(tk, false, tk);
             for (; tv < VST && tv < n_load; ++tv) load_tile(tv, true, tv);
             while (tk < n_load || tv < n_load) {
@@ -424,8 +438,8 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             if (__any_sync(0xffffffffu, need)) {
                 // PV(t-1) must be done before O is rescaled
                 if (t > 0) { mbar_wait(bar_pv, (t - 1) & 1, 4); tc_fence_after(); }
-#pragma unroll
-                for (int cb = 0; cb < D / 32 + (S::ONES ? 1 : 0); ++cb) {   // with ONES the row-sum columns are rescaled too
+#pragma unroll 1
+                for (int cb = 0; cb < D / 32 + (S::ONES ? 1 : 0); ++cb) {   // (rolled: rarely taken, and the softmax loop is sensitive to its code size)   // with ONES the row-sum columns are rescaled too
                     uint32_t q4[32];
                     tmem_ld32(tmem + lane_base + O_COL + cb * 32, q4);
                     tmem_wait_ld();
