@@ -66,7 +66,8 @@ template <int D> struct Smem {
 // They meet on mbarriers:
 //   bar_s[b]  (commit)       S(t) is in TMEM buffer b = t & 1                     control -> softmax
 //   bar_p     (128 arrivals) P(t) is in shared memory, S buffer b is free         softmax -> control
-//   bar_pv    (commit)       PV(t) has completed                                   control -> softmax
+//   bar_pv[b] (commit)       PV(t) has completed, b = t & 1 (a barrier per parity: a waiter can then never find it two
+//                            phases ahead, so the softmax threads wait on it only where they need the product)   control -> softmax
 //   bar_gk[s], bar_gv[s] (128 arrivals, by cp.async completion) a gathered tile is in stage s   softmax -> control
 //   bar_k[s], bar_v[s]       TMA transaction barriers of the window tiles
 //   bar_kf[s], bar_vf[s]     (commit) the MMA that read stage s has completed          MMA lane -> load lane
@@ -96,7 +97,7 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const uint32_t bar_k0 = bar_q + 8;                         // 3 slots
     const uint32_t bar_v0 = bar_q + 32;                        // 3 slots
     const uint32_t bar_s0 = bar_q + 56;                        // 2 slots
-    const uint32_t bar_p = bar_q + 88, bar_pv = bar_q + 96;
+    const uint32_t bar_p0 = bar_q + 88, bar_p1 = bar_q + 216, bar_pv0 = bar_q + 96, bar_pv1 = bar_q + 208;   // per tile parity
     const uint32_t bar_kf0 = bar_q + 104;                      // 3 slots: K stage free
     const uint32_t bar_vf0 = bar_q + 128;                      // 3 slots: V stage free
     const uint32_t tmem_slot = bar_q + 152;
@@ -127,7 +128,7 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         // to the MMA warp and cost 3 % at d = 128, T = 32768
 #pragma unroll
         for (int s2 = 0; s2 < 3; ++s2) { mbar_init(bar_gk0 + 8 * s2, 128); mbar_init(bar_gv0 + 8 * s2, 128); }
-        mbar_init(bar_p, 128); mbar_init(bar_pv, 1);
+        mbar_init(bar_p0, 128); mbar_init(bar_p1, 128); mbar_init(bar_pv0, 1); mbar_init(bar_pv1, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 4) tmem_alloc(tmem_slot, TMEM_COLS);
@@ -263,14 +264,14 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 uint32_t vb = v_desc[0];
 #pragma unroll
                 for (int st = 1; st < VST; ++st) vb = vs == st ? v_desc[st] : vb;
-                mbar_wait(bar_p, t & 1, 7);
+                mbar_wait((t & 1) ? bar_p1 : bar_p0, (t >> 1) & 1, 7);
                 PLM(19);
                 tc_fence_after();
                 if (lane == 0) {
 #pragma unroll
                     for (int kk = 0; kk < BN / 16; ++kk)
                         umma_ts(tmem + O_COL, tmem + (t & 1) * BN + kk * 8, desc64(vb + kk * 128, HI), IDESC_O, (t > 0 || kk > 0) ? 1u : 0u);
-                    umma_commit(bar_pv);
+                    umma_commit((t & 1) ? bar_pv1 : bar_pv0);
                     umma_commit(bar_vf0 + 8 * vs);             // the V stage is free once PV(t) has completed
                 }
                 __syncwarp();
@@ -437,7 +438,7 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             else if (m_tile > m_run + 8.f) { alpha = fast_exp2(m_run - m_tile); m_run = m_tile; need = true; }
             if (__any_sync(0xffffffffu, need)) {
                 // PV(t-1) must be done before O is rescaled
-                if (t > 0) { mbar_wait(bar_pv, (t - 1) & 1, 4); tc_fence_after(); }
+                if (t > 0) { mbar_wait(((t - 1) & 1) ? bar_pv1 : bar_pv0, ((t - 1) >> 1) & 1, 4); tc_fence_after(); }
 #pragma unroll 1
                 for (int cb = 0; cb < D / 32 + (S::ONES ? 1 : 0); ++cb) {   // (rolled: rarely taken, and the softmax loop is sensitive to its code size)   // with ONES the row-sum columns are rescaled too
                     uint32_t q4[32];
@@ -486,16 +487,16 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             tmem_wait_st();
             tc_fence_before();                                 // our TMEM accesses are ordered before the arrive
             PLM(9);
-            // PV(t-1) has normally completed long ago; the wait sits before the arrive so that the barrier cannot
-            // run two phases ahead of this thread
-            if (t > 0) mbar_wait(bar_pv, (t - 1) & 1, 4);
-            mbar_arrive(bar_p);
+            // (P and PV barriers come in pairs by tile parity: the MMA warp consumes P(t) before it issues S(t+2), which the
+            // softmax needs before it can post P(t+2) on the same barrier, so no barrier runs two phases ahead of a waiter)
+            if (!compact && t > 0) mbar_wait(((t - 1) & 1) ? bar_pv1 : bar_pv0, ((t - 1) >> 1) & 1, 4);   // (the value gather below needs PV(t-1) done)
+            mbar_arrive((t & 1) ? bar_p1 : bar_p0);
             PLM(10);
             // value tile t+VST-1 goes into the stage of V(t-1), which PV(t-1) has finished reading
             if (t > 0) gather_issue(t + VST - 1, true, rv);
             PLM(11);
         }
-        mbar_wait(bar_pv, (n_tiles - 1) & 1, 5);
+        mbar_wait(((n_tiles - 1) & 1) ? bar_pv1 : bar_pv0, ((n_tiles - 1) >> 1) & 1, 5);
         PLM_TILE(0);
         PLM(12);
         tc_fence_after();
