@@ -32,7 +32,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu captures (profiles/),
 # keyed by kernel family (profiles/prefill_tc_kernel_C2.md, profiles/decode_tc_kernel_C4.md).
-NCU_TRAFFIC_BYTES = {"prefill_attn_C2": 114.8e6, "decode_C4": 142.9e6}
+NCU_TRAFFIC_BYTES = {"prefill_attn_C2": 119.4e6, "decode_C4": 142.9e6}
 
 
 def peaks():
