@@ -60,8 +60,6 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                  const float* __restrict__ lse, const int32_t* __restrict__ idx, const int32_t* __restrict__ cnt,
                  __nv_bfloat16* __restrict__ dq, float* __restrict__ delta, int Tlen, int W, int R, float scale, int G)
 {
-    pdl_launch_dependents();
-    pdl_wait();                                                // see launch_pdl: earlier kernels of the stream have completed
     using S = SmemQ<D>;
     constexpr int SUB = S::SUB;
     constexpr bool DB = S::DB;
@@ -84,7 +82,6 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     const int j_start = max(i0 - W + 1, 0);
     const int n_win = (i_hi - j_start + 1 + BN - 1) / BN;
     const int32_t* id = idx + (size_t)bhk * R;
-    const int n_ret = cnt[bhk];
 
     if (tid == 0) {
         mbar_init(bar_q, 1);
@@ -100,20 +97,13 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot_gen;
+    pdl_launch_dependents();
+    pdl_wait();                                                // everything above ran beside the previous kernel's tail (see launch_pdl)
+    const int n_ret = cnt[bhk];
 
     if (warp == 4) {
         // =================================== control warp (one lane) ========================================
-        int nv_max = 0;
-        {
-            const int lim = i_hi - W;
-            for (int e0 = 0; e0 < n_ret; e0 += 32) {
-                const int e = e0 + lane < n_ret ? id[e0 + lane] : 0x7fffffff;
-                const unsigned bal = __ballot_sync(0xffffffffu, e <= lim);
-                nv_max += __popc(bal);
-                if (bal != 0xffffffffu) break;
-            }
-        }
-        const int n_tiles = n_win + (nv_max + BN - 1) / BN;
+        int n_tiles = n_win;                                   // + the retained tiles, counted once the first loads are on their way
         // The whole warp walks the loop and waits on the barriers; only the TMA / tcgen05 instructions are guarded by the
         // lane test, so that addresses and descriptors are computed in convergent code (cheaper to issue).
         const bool leader = lane == 0;
@@ -172,6 +162,18 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                 if (D == 64) tma_load_3d(sDS, &tmO, 0, i0, bh, bar_q);
             }
             for (int t = 0; t < NS && t < n_win; ++t) { tma_kv(t, false); tma_kv(t, true); }
+            {
+                // retained entries visible to the tile's last row (idx ascending => a prefix): read while the loads fly
+                int nv_max = 0;
+                const int lim = i_hi - W;
+                for (int e0 = 0; e0 < n_ret; e0 += 32) {
+                    const int e = e0 + lane < n_ret ? id[e0 + lane] : 0x7fffffff;
+                    const unsigned bal = __ballot_sync(0xffffffffu, e <= lim);
+                    nv_max += __popc(bal);
+                    if (bal != 0xffffffffu) break;
+                }
+                n_tiles = n_win + (nv_max + BN - 1) / BN;
+            }
             bwait(bar_q, 0, 1);                                // (tile 0 is always a window tile: no gather to wait for)
             wait_kv(0);
             tc_fence_after();
