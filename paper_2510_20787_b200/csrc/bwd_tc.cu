@@ -456,8 +456,6 @@ bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                   float* __restrict__ dk_ret, float* __restrict__ dv_ret, float* __restrict__ dr_ret, int n_wt, int Tlen,
                   int W, int R, float scale, int G)
 {
-    pdl_launch_dependents();
-    pdl_wait();                                                // see launch_pdl: earlier kernels of the stream have completed
     using S = SmemK<D>;
     constexpr int SUB = S::SUB;
     constexpr uint32_t DP_COL = 64, DV_COL = 128, DK_COL = 128 + D;
@@ -472,28 +470,6 @@ bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     const bool is_ret = lin < tot_ret;
     const int bh = is_ret ? lin / n_rt : (lin - tot_ret) / n_wt;
     const int tile = is_ret ? lin % n_rt : (lin - tot_ret) % n_wt;
-    const int n_ret = cnt[bh];
-    const int32_t* id = idx + (size_t)bh * R;
-    const int j0 = is_ret ? 0 : tile * 128;                    // window tile: first key
-    const int e0 = is_ret ? tile * 128 : 0;                    // retained tile: first list entry
-    if (is_ret && e0 >= n_ret) return;                         // nothing retained in this slice of the list
-
-    // query blocks that can see the tile
-    int ib_start, n_blk;
-    if (!is_ret) {
-        ib_start = j0;
-        const int i_end = min(Tlen - 1, j0 + 127 + W - 1);
-        n_blk = (i_end - ib_start) / 64 + 1;
-    } else {
-        const int first = id[e0] + W;                          // the oldest entry's first far query
-        ib_start = (first / 64) * 64;
-        n_blk = first <= Tlen - 1 ? (Tlen - 1 - ib_start) / 64 + 1 : 0;
-    }
-    // grouped queries: the G query heads of this key/value head walk the same query blocks one after the other and
-    // accumulate into the same dK, dV; walk step t is block t % n_pos of query head bh G + t / n_pos
-    const int n_pos = n_blk;
-    n_blk *= G;
-
     const uint32_t sK = base + S::OFF_K, sV = base + S::OFF_V, sQ = base + S::OFF_Q, sDO = base + S::OFF_DO;
     const uint32_t sPT = base + S::OFF_PT, sDST = base + S::OFF_DST;
     float* s_col = reinterpret_cast<float*>(smem_raw + S::OFF_COL);
@@ -513,6 +489,32 @@ bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot_gen;
+    pdl_launch_dependents();
+    pdl_wait();                                                // everything above ran beside the previous kernel's tail (see launch_pdl)
+    const int n_ret = cnt[bh];
+    const int32_t* id = idx + (size_t)bh * R;
+    const int j0 = is_ret ? 0 : tile * 128;                    // window tile: first key
+    const int e0 = is_ret ? tile * 128 : 0;                    // retained tile: first list entry
+    if (is_ret && e0 >= n_ret) {                               // nothing retained in this slice of the list
+        if (warp == 4) tmem_dealloc(tmem, S::TMEM_COLS);
+        return;
+    }
+
+    // query blocks that can see the tile
+    int ib_start, n_blk;
+    if (!is_ret) {
+        ib_start = j0;
+        const int i_end = min(Tlen - 1, j0 + 127 + W - 1);
+        n_blk = (i_end - ib_start) / 64 + 1;
+    } else {
+        const int first = id[e0] + W;                          // the oldest entry's first far query
+        ib_start = (first / 64) * 64;
+        n_blk = first <= Tlen - 1 ? (Tlen - 1 - ib_start) / 64 + 1 : 0;
+    }
+    // grouped queries: the G query heads of this key/value head walk the same query blocks one after the other and
+    // accumulate into the same dK, dV; walk step t is block t % n_pos of query head bh G + t / n_pos
+    const int n_pos = n_blk;
+    n_blk *= G;
 
     if (warp == 4) {
         // (the whole warp walks the loop and waits; only the TMA / tcgen05 instructions are guarded by the lane test)
