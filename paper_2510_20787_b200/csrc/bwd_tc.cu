@@ -434,14 +434,20 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 // ================================================ dkv kernel =====================================================
 template <int D> struct SmemK {
     static constexpr int SUB = D / 64;
+    // d = 128 runs one CTA per SM and has the TMEM columns for two S^T / dP^T buffers: block t+2's products are issued
+    // while the key threads work on block t+1, which takes one more stage of query blocks in flight
+    static constexpr bool DB = D == 128;
+    static constexpr int NSTK = DB ? 4 : 3;
     static constexpr int KTILE = 128 * D * 2, QBLK = 64 * D * 2;
-    static constexpr int OFF_K = 0, OFF_V = KTILE, OFF_Q = 2 * KTILE, OFF_DO = OFF_Q + NST * QBLK;
-    static constexpr int OFF_PT = OFF_DO + NST * QBLK;         // [128][64] bf16
+    static constexpr int OFF_K = 0, OFF_V = KTILE, OFF_Q = 2 * KTILE, OFF_DO = OFF_Q + NSTK * QBLK;
+    static constexpr int OFF_PT = OFF_DO + NSTK * QBLK;        // [128][64] bf16
     static constexpr int OFF_DST = OFF_PT + 128 * 64 * 2;      // [128][64] bf16
     static constexpr int OFF_COL = OFF_DST + 128 * 64 * 2;     // L2[64], delta[64] of the current query block
     static constexpr int OFF_BAR = OFF_COL + 512;
     static constexpr int BYTES = OFF_BAR + 128;
-    static constexpr uint32_t TMEM_COLS = D == 64 ? 256 : 512; // S^T [0,64) dP^T [64,128) dV [128,128+D) dK [128+D,128+2D)
+    // d = 64: S^T [0,64) dP^T [64,128) dV [128,192) dK [192,256); d = 128: S^T, dP^T of even blocks [0,128), of odd blocks
+    // [128,256), dV [256,384), dK [384,512)
+    static constexpr uint32_t TMEM_COLS = D == 64 ? 256 : 512;
 };
 
 template <int D, bool F32OUT>
@@ -458,7 +464,9 @@ bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
 {
     using S = SmemK<D>;
     constexpr int SUB = S::SUB;
-    constexpr uint32_t DP_COL = 64, DV_COL = 128, DK_COL = 128 + D;
+    constexpr bool DB = S::DB;
+    constexpr int NSTK = S::NSTK;
+    constexpr uint32_t DP_COL = 64, DV_COL = DB ? 256 : 128, DK_COL = DV_COL + D;
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     const uint32_t base = smem_u32(smem_raw);
     if ((base & 1023u) != 0) { if (threadIdx.x == 0) atomicExch(&g_bwd_status, 9); return; }
@@ -473,15 +481,15 @@ bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     const uint32_t sK = base + S::OFF_K, sV = base + S::OFF_V, sQ = base + S::OFF_Q, sDO = base + S::OFF_DO;
     const uint32_t sPT = base + S::OFF_PT, sDST = base + S::OFF_DST;
     float* s_col = reinterpret_cast<float*>(smem_raw + S::OFF_COL);
-    const uint32_t bar_kv = base + S::OFF_BAR, bar_q0 = bar_kv + 8, bar_s = bar_kv + 32, bar_g = bar_kv + 40;
-    const uint32_t bar_p = bar_kv + 48, bar_pv = bar_kv + 56, tmem_slot = bar_kv + 64;
-    volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(smem_raw + S::OFF_BAR + 64);
+    const uint32_t bar_kv = base + S::OFF_BAR, bar_q0 = bar_kv + 8, bar_s0 = bar_kv + 40, bar_g = bar_kv + 56;
+    const uint32_t bar_p = bar_kv + 64, bar_pv = bar_kv + 72, tmem_slot = bar_kv + 80;
+    volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(smem_raw + S::OFF_BAR + 80);
 
     if (tid == 0) {
         mbar_init(bar_kv, 1);
 #pragma unroll
-        for (int s2 = 0; s2 < NST; ++s2) mbar_init(bar_q0 + 8 * s2, 1);
-        mbar_init(bar_s, 1); mbar_init(bar_g, 128); mbar_init(bar_p, 128); mbar_init(bar_pv, 1);
+        for (int s2 = 0; s2 < NSTK; ++s2) mbar_init(bar_q0 + 8 * s2, 1);
+        mbar_init(bar_s0, 1); mbar_init(bar_s0 + 8, 1); mbar_init(bar_g, 128); mbar_init(bar_p, 128); mbar_init(bar_pv, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 4) tmem_alloc(tmem_slot, S::TMEM_COLS);
@@ -527,7 +535,7 @@ bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
             const uint32_t qmn_lo = desc_lo(sQ, 8192), domn_lo = desc_lo(sDO, 8192);
             uint32_t q_phase = 0;
             auto tma_blk = [&](int t) {
-                const int st = t % NST;
+                const int st = t % NSTK;
                 const uint32_t bar = bar_q0 + 8 * st;
                 const int y = ib_start + (t % n_pos) * 64, bhq = bh * G + t / n_pos;
                 if (leader) {
@@ -540,21 +548,22 @@ bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                 }
             };
             auto wait_blk = [&](int t) {
-                const int st = t % NST;
+                const int st = t % NSTK;
                 bwait(bar_q0 + 8 * st, (q_phase >> st) & 1u, 2); q_phase ^= 1u << st;
             };
             auto mma_s_dp = [&](int t) {
-                const uint32_t so = (uint32_t)(t % NST) * (S::QBLK >> 4);
+                const uint32_t so = (uint32_t)(t % NSTK) * (S::QBLK >> 4);
+                const uint32_t tb = tmem + (DB ? (uint32_t)(t & 1) * 128u : 0u);
                 if (leader) {
 #pragma unroll
                     for (int kk = 0; kk < D / 16; ++kk)
-                        umma(tmem, desc64(k_lo + (kk >> 2) * 1024 + (kk & 3) * 2, kDescHi),
+                        umma(tb, desc64(k_lo + (kk >> 2) * 1024 + (kk & 3) * 2, kDescHi),
                              desc64(q_lo + so + (kk >> 2) * 512 + (kk & 3) * 2, kDescHi), IDESC_S, kk > 0);
 #pragma unroll
                     for (int kk = 0; kk < D / 16; ++kk)
-                        umma(tmem + DP_COL, desc64(v_lo + (kk >> 2) * 1024 + (kk & 3) * 2, kDescHi),
+                        umma(tb + DP_COL, desc64(v_lo + (kk >> 2) * 1024 + (kk & 3) * 2, kDescHi),
                              desc64(do_lo + so + (kk >> 2) * 512 + (kk & 3) * 2, kDescHi), IDESC_S, kk > 0);
-                    umma_commit(bar_s);
+                    umma_commit(DB ? bar_s0 + 8 * (t & 1) : bar_s0);
                 }
                 __syncwarp();
             };
@@ -566,19 +575,22 @@ bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                     tma_load_3d(sV + sb * 16384, &tmV, sb * 64, j0, bh, bar_kv);
                 }
             }
-            for (int t = 0; t < NST && t < n_blk; ++t) tma_blk(t);
+            for (int t = 0; t < NSTK && t < n_blk; ++t) tma_blk(t);
             if (!is_ret) bwait(bar_kv, 0, 1); else bwait(bar_g, 0, 10);   // the tile's own K/V rows are in shared memory
             wait_blk(0);
             tc_fence_after();
             mma_s_dp(0);
+            if (DB && n_blk > 1) { wait_blk(1); mma_s_dp(1); }
             for (int t = 0; t < n_blk; ++t) {
                 bwait(bar_p, t & 1, 7);                        // P^T(t), dS^T(t) are in shared memory
                 tc_fence_after();
-                // the next block's S^T, dP^T first: the key threads wait for those, while dV, dK of this block are only
-                // needed before the operand buffers are rewritten a block later
-                if (t + 1 < n_blk) { wait_blk(t + 1); mma_s_dp(t + 1); }
+                // one buffer: the next block's S^T, dP^T first (the key threads wait for those, while dV, dK of this block
+                // are only needed before the operand buffers are rewritten a block later); two buffers: the next block's
+                // products are already there, so dV, dK go first and block t+2's products take the buffer of block t,
+                // which the key threads have read out
+                if (!DB && t + 1 < n_blk) { wait_blk(t + 1); mma_s_dp(t + 1); }
                 {
-                    const uint32_t so = (uint32_t)(t % NST) * (S::QBLK >> 4);
+                    const uint32_t so = (uint32_t)(t % NSTK) * (S::QBLK >> 4);
                     if (leader) {
 #pragma unroll
                         for (int kk = 0; kk < 4; ++kk)
@@ -592,9 +604,10 @@ bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                     }
                     __syncwarp();
                 }
+                if (DB && t + 2 < n_blk) { wait_blk(t + 2); mma_s_dp(t + 2); }
                 // the accumulations of block t-1 have completed (the key threads waited for them before producing
-                // block t's operands): its stage can take block t-1+NST
-                if (t >= 1 && t - 1 + NST < n_blk) tma_blk(t - 1 + NST);
+                // block t's operands): its stage can take block t-1+NSTK
+                if (t >= 1 && t - 1 + NSTK < n_blk) tma_blk(t - 1 + NSTK);
             }
         }
     } else {
@@ -618,19 +631,23 @@ bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         const float c2 = scale * kLog2e;
         const uint32_t lane_base = ((uint32_t)(warp * 32)) << 16;
         // per-column constants of the next block, fetched one block ahead: thread c < 64 holds -L2, thread 64 + c
-        // -delta scale (the forms the fused multiply-adds below take)
+        // -delta scale (the forms the fused multiply-adds below take).  The fetch returns the value as loaded and the
+        // factor is applied a block later, where it is stored: arithmetic placed right behind the load would hold the
+        // warp (which issues in order) for the whole latency of the load.
+        const float* col_src = tid < 64 ? lse : delta;
+        const float col_mul = tid < 64 ? -kLog2e : -scale;
         auto col_fetch = [&](int t) -> float {
             if (t >= n_blk) return 0.f;
             const int i = ib_start + (t % n_pos) * 64 + (tid & 63);
-            if (i >= Tlen) return tid < 64 ? -INFINITY : 0.f;                   // -L2 = -inf makes P = 0
+            if (i >= Tlen) return tid < 64 ? INFINITY : 0.f;                    // -L2 = -inf makes P = 0
             const size_t bhq = (size_t)bh * G + t / n_pos;
-            return tid < 64 ? -lse[bhq * Tlen + i] * kLog2e : -delta[bhq * Tlen + i] * scale;
+            return col_src[bhq * Tlen + i];
         };
         float col_next = col_fetch(0);
 
         for (int t = 0; t < n_blk; ++t) {
             group_sync();                                      // everyone is done with the previous block's constants
-            s_col[tid] = col_next;
+            s_col[tid] = col_next * col_mul;
             col_next = col_fetch(t + 1);
             group_sync();
             const int ib = ib_start + (t % n_pos) * 64;
@@ -640,16 +657,18 @@ bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
             else { c_lo = pos + W - ib; c_hi = Tlen - 1 - ib; }
             const int u_lo = __reduce_min_sync(0xffffffffu, c_lo), u_hi = __reduce_max_sync(0xffffffffu, c_hi);
 
-            bwait(bar_s, t & 1, 3);                            // S^T(t), dP^T(t) are in TMEM
+            if (DB) bwait(bar_s0 + 8 * (t & 1), (t >> 1) & 1, 3);   // S^T(t), dP^T(t) are in TMEM
+            else bwait(bar_s0, t & 1, 3);
             tc_fence_after();
+            const uint32_t tb = tmem + lane_base + (DB ? (uint32_t)(t & 1) * 128u : 0u);
             uint32_t pp[32], pd[32];                           // P^T and dS^T rows as 64 bf16 each
 #pragma unroll
             for (int cb = 0; cb < 2; ++cb) {
                 const bool act = cb * 32 <= u_hi && cb * 32 + 31 >= u_lo;
                 if (act) {
                     uint32_t rs[32], rp[32];
-                    tmem_ld32(tmem + lane_base + cb * 32, rs);
-                    tmem_ld32(tmem + lane_base + DP_COL + cb * 32, rp);
+                    tmem_ld32(tb + cb * 32, rs);
+                    tmem_ld32(tb + DP_COL + cb * 32, rp);
                     tmem_wait_ld();
 #pragma unroll
                     for (int c = 0; c < 32; c += 4) {
