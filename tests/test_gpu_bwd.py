@@ -66,3 +66,11 @@ def test_deterministic():
     b = _bwd(cfg, seed=1)
     for n in a:
         assert np.array_equal(a[n][0], b[n][0])
+
+
+@pytest.mark.parametrize("d,T,W,R", [(128, 9000, 64, 200), (64, 4500, 100, 130)])
+def test_long_sequence_two_retained_tiles(d, T, W, R):
+    # thousands of tokens: a retained tile walks many query blocks (the double-buffered products at d = 128 and the
+    # stage ring wrap many times), and the list spans two tiles, the second one partly filled
+    cfg = synth.Config("bwdlong", "bf16", 1, 2, d, T, W, R, 7, 0.05)
+    _assert(cfg, _bwd(cfg, seed=3))
