@@ -304,13 +304,18 @@ int lte_attn_bwd(const lte_shape* s, const lte_conv* c,
  * allocator-locked region, or a host that must not call cudaMalloc because that call synchronises the device
  * and would stall every other stream.  Such callers cannot create the workspace lte_attn_bwd asks for.
  *
- * Same arguments, results and errors as lte_attn_bwd, minus `ws` / `ws_bytes`: the scratch is a fixed array of
- * LTE_STATIC_SCRATCH_BYTES inside the library (each GPU that loads the library holds it until the process
- * ends).  The call itself performs no cudaMalloc / cudaFree and uses no allocating library routine.
+ * Same arguments and results as lte_attn_bwd, minus `ws` / `ws_bytes` (grouped queries included); the scorer must be
+ * the single layer (the three-layer stack answers LTE_ERR_UNSUPPORTED here: its scratch does not fit).  The scratch is a
+ * fixed array of LTE_STATIC_SCRATCH_BYTES inside the library; each GPU on which the library's code gets loaded holds
+ * it until the process ends.  The call itself performs no cudaMalloc / cudaFree and uses no allocating library routine.
  *   - Shapes whose scratch need (lte_workspace_bytes(LTE_OP_BWD, ...) for flags = LTE_BWD_CNN_INPUT_GRAD; less
  *     without that flag) exceeds LTE_STATIC_SCRATCH_BYTES are rejected with LTE_ERR_WORKSPACE; nothing is launched.
  *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with that device
- *     current).  Make that first call outside any stream capture.
+ *     current).  Under CUDA's lazy loading that look-up is also the moment the driver loads this part of the library
+ *     onto the device and sets the array aside, which takes device memory once and may synchronise the device; a
+ *     device whose memory is already spent answers LTE_ERR_CUDA.  So make that first call at start-up, before the
+ *     memory pool is frozen and outside any stream capture; later calls on that device touch no memory management at all.
+ *     cudaDeviceReset() invalidates the looked-up address: do not call this entry point on a device after resetting it.
  *   - All calls on a device share the one array, which still holds whatever the previous call left there.  The
  *     backward kernels write every scratch value before reading it, so no clearing is needed, but two calls that
  *     overlap on the GPU (different streams) would race on it: issue them on one stream, or serialise them.

@@ -429,7 +429,6 @@ int lte_attn_bwd_static(const lte_shape* s, const lte_conv* c, const void* q, co
     if (!q || !k || !v || !o || !lse || !dO || !z || !cnt || (s->R > 0 && !idx) || !dq || !dk || !dv || !dw)
         return LTE_ERR_INVALID_ARG;
     if (flags & ~LTE_BWD_CNN_INPUT_GRAD) return LTE_ERR_INVALID_ARG;
-    if (s->group > 1) return LTE_ERR_UNSUPPORTED;
     Params p = make_params(s, c);
     if (bwd_workspace_bytes(p, flags) > (size_t)LTE_STATIC_SCRATCH_BYTES) return LTE_ERR_WORKSPACE;   /* too large for the fixed array */
     e = check_arch(); if (e) return e;

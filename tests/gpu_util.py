@@ -61,3 +61,42 @@ def check_idx(idx_gpu, cnt_gpu, z64, W, R, sink=0, tau=0.5):
 def rel_l2(a, b):
     a = np.asarray(a, np.float64); b = np.asarray(b, np.float64)
     return float(np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-30))
+
+
+def assert_grad_close(name, got, want, tol, idx=None, cnt=None, block=128):
+    """Gradient comparison at three granularities, each with the same relative-L2 bound: the whole tensor; for a
+    [B,H,T,d] tensor every block of `block` consecutive rows of every (b,h); and, given a retained list, the rows
+    idx[b,h,:cnt[b,h]] of every (b,h) on their own (Eq. 6 reads exactly those rows of dV, and a wrong head's worth of
+    them moves the whole-tensor norm by far less than the bound).  For other tensors with a leading head axis
+    ([H,...]) the per-head slices are compared.  A slice whose reference norm is below 1e-3 of the tensor's RMS slice
+    norm is compared against that floor instead (a relative error on an all-but-zero slice says nothing)."""
+    a = np.asarray(got, np.float64); b = np.asarray(want, np.float64)
+    assert a.shape == b.shape, (name, a.shape, b.shape)
+    assert np.all(np.isfinite(a)), name
+    whole = rel_l2(a, b)
+    assert whole <= tol, (name, "whole tensor", whole)
+    if a.ndim == 4:
+        B, H, T, d = a.shape
+        nb = (T + block - 1) // block
+        pad = nb * block - T
+        ap = np.pad(a, ((0, 0), (0, 0), (0, pad), (0, 0))).reshape(B, H, nb, block * d)
+        bp = np.pad(b, ((0, 0), (0, 0), (0, pad), (0, 0))).reshape(B, H, nb, block * d)
+        num = np.linalg.norm(ap - bp, axis=-1); den = np.linalg.norm(bp, axis=-1)
+        floor = 1e-3 * np.sqrt(np.mean(den ** 2)) + 1e-30
+        rel = num / np.maximum(den, floor)
+        worst = np.unravel_index(np.argmax(rel), rel.shape)
+        assert rel[worst] <= tol, (name, "(b, h, row block)", worst, float(rel[worst]))
+        if idx is not None:
+            for bb in range(B):
+                for h in range(H):
+                    rows = idx[bb, h, :cnt[bb, h]]
+                    if len(rows) == 0:
+                        continue
+                    r = rel_l2(a[bb, h, rows], b[bb, h, rows])
+                    assert r <= tol, (name, "retained rows of (b, h)", bb, h, r)
+    elif a.ndim >= 2:
+        num = np.linalg.norm((a - b).reshape(a.shape[0], -1), axis=-1); den = np.linalg.norm(b.reshape(a.shape[0], -1), axis=-1)
+        floor = 1e-3 * np.sqrt(np.mean(den ** 2)) + 1e-30
+        rel = num / np.maximum(den, floor)
+        assert np.max(rel) <= tol, (name, "head", int(np.argmax(rel)), float(np.max(rel)))
+    return whole

@@ -129,6 +129,12 @@ def test_chunk_dtypes_sinks_groups(kw, plan, scale, group):
     _compare(_cfg(**kw), plan, seed=1, scale=scale, group=group)
 
 
+def test_serving_shape_chunk_on_a_big_cache():
+    """The "serving-like" chunk of the benchmark: a 512-token chunk on a W = 768, R = 512 cache with sink tokens,
+    after a prompt, followed by decode steps."""
+    _compare(_cfg(B=1, H=2, W=768, R=512, sink=4), [("prefill", 2000), ("chunk", 512), ("decode", 4)], seed=2)
+
+
 def test_wrong_token_count_is_reported_and_leaves_the_cache_alone():
     cfg = _cfg(B=1, H=2)
     x = synth.make(cfg, 0, T=120)

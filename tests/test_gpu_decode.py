@@ -171,3 +171,12 @@ def test_config4_full_batch_sampled_sequences():
             want = pidx[a, h, :pcnt[a, h]]
             assert np.array_equal(pools[b * cfg.H + h], want)
     assert all(n == Ttot for n in ns)
+
+
+@pytest.mark.parametrize("d", [64, 128])
+def test_serving_shape_single_group(d):
+    """The paper-like serving shape of the benchmark (W = 768, R = 512, 4 sink tokens), one query head per key/value
+    head: 1,280 cache rows per head, far beyond the tensor-core kernel's 256, so the row-looping step kernel runs."""
+    cfg = synth.Config("serve", "bf16", 1, 2, d, 2100, 768, 512, 7, 0.05, sink=4)
+    _assert(cfg, _decode_run(cfg, cfg.T, 40, seed=5), cfg.T + 40)
+    assert lte.lte_device_status() == 0

@@ -77,6 +77,14 @@ def test_config3_sampled_queries():
     _assert_close(cfg, _pipeline(cfg, seed=0, qpos=qpos))
 
 
+def test_serving_shape_with_sink():
+    """The paper-like serving shape of the benchmark: W = 768, R = 512, 4 sink tokens (window of six key tiles, a list
+    that is not full on every head because the sink entries take slots)."""
+    cfg = synth.Config("serve", "bf16", 1, 2, 64, 4096, 768, 512, 7, 0.05, sink=4)
+    _assert_close(cfg, _pipeline(cfg, seed=3))
+    _assert_close(cfg.with_(d=128), _pipeline(cfg.with_(d=128, T=2500), seed=3))
+
+
 def test_config5_forward():
     cfg = synth.CONFIGS["C5"]
     _assert_close(cfg, _pipeline(cfg, seed=0, batch=[0, 7]))

@@ -139,3 +139,36 @@ def test_rope_is_a_rotation_of_channel_pairs_and_inverts():
     np.testing.assert_allclose(np.linalg.norm(y, axis=-1), np.linalg.norm(x, axis=-1), rtol=1e-12)
     np.testing.assert_allclose(orc.rope(y, cos, sin, pos0=11, inverse=True), x, atol=1e-12)
     np.testing.assert_allclose(orc.rope(x[..., :1, :], cos, sin, pos0=0), x[..., :1, :], atol=0)
+
+
+@pytest.mark.parametrize("tau0", [0, 1, 2])
+def test_stack_single_tap_reads_one_hand_worked_position(tau0):
+    """Tap order inside a layer (Appendix A: kernel 3, dilation 2, three layers; cross-correlation, tap 0 = the oldest
+    input).  With only tap tau0 non-zero in every layer, layer l's output at time t reads its input at t - (2 - tau0) * 2
+    and nothing else, so after three layers and the deferral of the logit by 6 the logit of token j reads exactly the
+    input at j - 6 (tau0 = 0), j (tau0 = 1) or j + 6 (tau0 = 2): worked out by hand from those numbers, not from the
+    oracle's index expression.  A tap order taken the other way round swaps the first and the last case.  The value is
+    pinned too: through one channel with unit weights it is Swish applied three times to that input."""
+    B, H, T, d = 1, 2, 40, 8
+    ch = [2 * d, d, d // 2, d // 4]
+    k, v = _rand((B, H, T, d), 50), _rand((B, H, T, d), 51)
+    wl = [np.zeros((H, ch[l + 1], 3, ch[l])) for l in range(3)]
+    c_in = 3                                              # a key channel
+    wl[0][:, 1, tau0, c_in] = 1.0                         # input channel 3 -> hidden channel 1
+    wl[1][:, 2, tau0, 1] = 1.0                            # hidden 1 -> hidden 2
+    wl[2][:, 0, tau0, 2] = 1.0                            # hidden 2 -> hidden 0
+    wout = np.zeros((H, ch[3])); wout[:, 0] = 1.0
+    z = orc.scores_stack(k, v, wl, [None] * 3, wout, None, 3, 2)
+    src = {0: -6, 1: 0, 2: 6}[tau0]
+    sw = lambda a: a / (1.0 + np.exp(-a))
+    for j in range(T - 6):
+        p = j + src
+        # left of time 0 the input is zero, and so is every hidden activation there: the logit is Swish^3(0) = 0
+        want = sw(sw(sw(k[0, :, p, c_in]))) if p >= 0 else np.zeros(H)
+        np.testing.assert_allclose(z[0, :, j], want, atol=1e-14)
+    # support, by perturbation: exactly one input position moves the logit of token j
+    j = 20
+    for p in range(T):
+        k2 = k.copy(); k2[0, :, p, c_in] += 1.0
+        z2 = orc.scores_stack(k2, v, wl, [None] * 3, wout, None, 3, 2)
+        assert (not np.allclose(z2[0, :, j], z[0, :, j])) == (p == j + src), (tau0, p)
