@@ -45,11 +45,13 @@ def test_static_scratch_backward_matches_oracle_and_workspace_backward_twice_in_
         want = lte.lte_attn_bwd(*args)
         outs = tuple(torch.empty_like(t) for t in want)          # caller-owned outputs: the call allocates nothing
         torch.cuda.synchronize()
-        free0, alloc0, resv0 = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+        # requests made to the caller's allocator so far (a counter: it never goes down when something is freed)
+        nreq = lambda: torch.cuda.memory_stats()["allocation.all.allocated"]
+        free0, req0, resv0 = torch.cuda.mem_get_info()[0], nreq(), torch.cuda.memory_reserved()
         got = lte.lte_attn_bwd_static(*args, outs=outs)
         torch.cuda.synchronize()
-        free1, alloc1, resv1 = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
-        assert (alloc1, resv1) == (alloc0, resv0), "the caller's allocator was used"
+        free1, req1, resv1 = torch.cuda.mem_get_info()[0], nreq(), torch.cuda.memory_reserved()
+        assert (req1, resv1) == (req0, resv0), "the caller's allocator was used"
         if n > 0:                                                 # the first call on a device may load the library's module
             assert free1 == free0, "device memory was taken or given back during the call"
         idx_n, cnt_n = args[9].cpu().numpy(), args[10].cpu().numpy()
