@@ -30,9 +30,41 @@ import numpy as np  # noqa: E402
 METRIC = "LTE attn prefill tokens/s & % bf16 TC peak; decode step us & % HBM BW"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu captures (profiles/),
-# keyed by kernel family (profiles/prefill_tc_kernel_C2.md, profiles/decode_tc_kernel_C4.md).
-NCU_TRAFFIC_BYTES = {"prefill_attn_C2": 119.4e6, "decode_C4": 142.9e6}
+WORKLOAD = "C2 bf16 prefill: B=4 H=16 d=64 T=4096 W=128 R=128 K=7 per GPU, scores+select+attention"
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "ncu_traffic.json")
+
+
+def bench_config(world):
+    """The `config` object of the bench line (both arms print the same one: the reference arm times this workload too)."""
+    return {"workload": WORKLOAD, "l2": "flushed between timed steps (256 MB write)",
+            "parallelism": "replicas x%d (independent (batch, head) units)" % world}
+
+
+def sources_digest(files):
+    """sha256 over the named kernel sources (paths relative to the package's csrc/), in the given order."""
+    import hashlib
+    h = hashlib.sha256()
+    for f in files:
+        with open(os.path.join(ROOT, "paper_2510_20787_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()
+
+
+def ncu_traffic(key):
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch of a kernel, from the record of its last ncu capture
+    (profiles/ncu_traffic.json: bytes, the commit the capture was taken at, and a digest of the kernel's sources at that
+    commit).  The figure is reported only while the sources still have that digest; after a change to the kernel it is
+    None until the kernel is captured again.  Returns (bytes or None, provenance dict)."""
+    try:
+        rec = json.load(open(TRAFFIC_FILE))[key]
+    except (OSError, KeyError, ValueError):
+        return None, {"capture": None}
+    try:
+        current = sources_digest(rec["sources"])
+    except OSError:
+        current = None
+    prov = {"capture_commit": rec.get("commit"), "summary": rec.get("summary"), "sources_unchanged": current == rec.get("sources_sha256")}
+    return (float(rec["dram_bytes_per_launch"]) if prov["sources_unchanged"] else None), prov
 
 
 def peaks():
@@ -190,7 +222,7 @@ def run_lte(args):
     dist = None
     if world > 1:
         import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        dist.init_process_group(args.backend, device_id=torch.device("cuda", local))
     lte.lib()
     pk = peaks()
     if args.section and args.skip_main:
@@ -322,7 +354,8 @@ def run_lte(args):
     attn_s = k_ms[2] * 1e-3
     roof = {"bound": "hbm", "kernel": "lte_attn_prefill", "achieved": attn_bytes / attn_s / 1e9,
             "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": attn_bytes / attn_s / 1e9 / pk["hbm_gbs"],
-            "traffic": NCU_TRAFFIC_BYTES["prefill_attn_C2"], "peak_source": pk["source"],
+            "traffic": ncu_traffic("prefill_attn_C2")[0], "traffic_capture": ncu_traffic("prefill_attn_C2")[1],
+            "peak_source": pk["source"],
             "algorithmic_bytes": attn_bytes, "algorithmic_flops": flops,
             "tensor_tflops": flops / attn_s / 1e12, "tensor_frac": flops / attn_s / 1e12 / pk["bf16_tflops"],
             "kernel_ms": {"lte_scores": float(k_ms[0]), "lte_select": float(k_ms[1]), "lte_attn_prefill": float(k_ms[2])},
@@ -331,9 +364,7 @@ def run_lte(args):
     line = {"metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": "C2 bf16 prefill: B=4 H=16 d=64 T=4096 W=128 R=128 K=7 per GPU, "
-                                   "scores+select+attention", "l2": "flushed between timed steps (256 MB write)",
-                       "parallelism": "replicas x%d (independent (batch, head) units)" % world},
+            "config": bench_config(world),
             "e2e": {"value": tokens / (e2e_ms * 1e-3), "unit": "tokens/s", "ms_per_step": e2e_ms,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
             "gpu_launches": 4 * args.steps, "roofline": roof, "wall_s": t_wall,
@@ -757,7 +788,7 @@ def _extra_c4(out, torch, lte, synth, pk, flush, n5):
     out["C4_decode"] = {"us_per_step": us, "us_per_step_python_launches": us_eager, "steps_timed": len(evs),
                         "timing": "CUDA graph of the 248 steps, middle 3 of 5 replays", "algorithmic_bytes_per_step": by,
                         "hbm_gbs": by / (us * 1e-6) / 1e9, "hbm_frac": by / (us * 1e-6) / 1e9 / pk["hbm_gbs"],
-                        "traffic": NCU_TRAFFIC_BYTES["decode_C4"],
+                        "traffic": ncu_traffic("decode_C4")[0], "traffic_capture": ncu_traffic("decode_C4")[1],
                         "note": "the 138 MB cache is about the size of L2: see the ncu DRAM bytes in profiles/"}
 
 
@@ -792,24 +823,91 @@ def run_reference(args):
     cfg = synth.CONFIGS["C2"]
     x = synth.make(cfg, 0)
     x = {n: np.asarray(a, np.float64) for n, a in x.items()}
-    for _ in range(min(args.warmup, 3)):
+    for _ in range(args.warmup):
         oracle_step(orc, x, cfg)
-    steps = min(args.steps, 20)
+    steps = args.steps
     t0 = time.time()
     for _ in range(steps):
         oracle_step(orc, x, cfg)
     dt = (time.time() - t0) / steps
     val = cfg.B * cfg.T / dt
-    sample = "each step = the full C2 batch once (B=4, 16384 tokens); %d steps timed" % steps
+    sample = "each step = the full C2 batch once (B=4, 16384 tokens) on rank 0's host cores; %d steps timed" % steps
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": val, "unit": "tokens/s", "n_gpus": args.gpus,
-        "steps": steps, "warmup": min(args.warmup, 3), "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "steps": steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": "C2 bf16 prefill: B=4 H=16 d=64 T=4096 W=128 R=128 K=7, scores+select+attention"},
+        "config": bench_config(max(args.gpus, 1)),
+        "host_note": "the oracle runs on rank 0's host cores only (OpenMP over (batch, head)); no GPU, no L2 flush",
         "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": orc.num_threads(), "kind": "oracle",
                          "sample": sample},
         "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0}))
+
+
+TRAFFIC_SOURCES = {
+    "prefill_attn_C2": ["prefill_tc.cu", "prefill_tc_long.cu", "tc_common.cuh", "tma_util.cuh", "common.cuh"],
+    "decode_C4": ["decode_tc.cu", "tc_common.cuh", "tma_util.cuh", "common.cuh"],
+}
+
+
+def record_traffic(spec):
+    """--record-traffic KEY=BYTES[,SUMMARY]: write the DRAM bytes per launch read off an ncu capture of the kernel behind
+    KEY into profiles/ncu_traffic.json, with the current commit and the digest of the kernel's sources, so that a later
+    bench line can tell whether the figure still belongs to the kernel it times.  Run it on the tree the capture used."""
+    key, _, rest = spec.partition("=")
+    val, _, summary = rest.partition(",")
+    try:
+        commit = subprocess.check_output(["git", "-C", ROOT, "rev-parse", "--short", "HEAD"], text=True).strip()
+        if subprocess.check_output(["git", "-C", ROOT, "status", "--porcelain", "--", "paper_2510_20787_b200/csrc"], text=True).strip():
+            commit += "+uncommitted"
+    except (OSError, subprocess.CalledProcessError):
+        commit = None
+    try:
+        rec = json.load(open(TRAFFIC_FILE))
+    except (OSError, ValueError):
+        rec = {}
+    rec[key] = {"dram_bytes_per_launch": float(val), "commit": commit, "summary": summary or None,
+                "sources": TRAFFIC_SOURCES[key], "sources_sha256": sources_digest(TRAFFIC_SOURCES[key])}
+    with open(TRAFFIC_FILE, "w") as f:
+        json.dump(rec, f, indent=1, sort_keys=True)
+        f.write("\n")
+    print(json.dumps(rec[key]))
+
+
+def free_port():
+    import socket
+    with socket.socket() as so:
+        so.bind(("127.0.0.1", 0))
+        return so.getsockname()[1]
+
+
+def spawn_ranks(n, argv):
+    """`python bench.py --gpus N` outside a launcher: start N local ranks of this same command under
+    torch.distributed.run (one process per GPU, rendezvous on 127.0.0.1) and return their exit code.  Inside a launcher
+    (RANK / WORLD_SIZE in the environment) nothing is spawned and None is returned."""
+    if n <= 1 or "RANK" in os.environ or "WORLD_SIZE" in os.environ:
+        return None
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(n),
+           "--master-addr", "127.0.0.1", "--master-port", str(free_port()), os.path.abspath(__file__)] + list(argv)
+    return subprocess.call(cmd)
+
+
+def run_rank_selftest(args):
+    """The rank plumbing alone (process group, barrier, max over ranks, whole-job rate) on the given backend: what N > 1
+    adds to the single-GPU run.  Used by the CPU test with gloo; rank r pretends its step took 1 + r ms."""
+    import torch
+    import torch.distributed as dist
+    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1:
+        dist.init_process_group(args.backend)
+    dev = "cuda" if args.backend == "nccl" else "cpu"
+    if world > 1:
+        dist.barrier()
+    ms = max_over_ranks(1.0 + rank, dist if world > 1 else None, dev)
+    if world > 1:
+        dist.barrier(); dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps({"selftest": "ranks", "n_gpus": world, "ms_per_step": ms, "value": whole_job_rate(1000, world, ms)}))
 
 
 def main():
@@ -822,10 +920,23 @@ def main():
     ap.add_argument("--section", default=None, choices=["C3", "C4", "C5", "P", "S", "K"],
                     help="time only this extra section (long prefill / decode / forward+backward) after the main loop")
     ap.add_argument("--skip-main", action="store_true", help="with --section: skip the main C2 loop")
+    ap.add_argument("--backend", default="nccl", choices=["nccl", "gloo"], help="process-group backend for N > 1")
+    ap.add_argument("--selftest-ranks", action="store_true", help="run only the rank plumbing (barrier, max over ranks)")
+    ap.add_argument("--record-traffic", default=None, metavar="KEY=BYTES[,SUMMARY]",
+                    help="no benchmark: store an ncu DRAM-bytes figure with its provenance (see record_traffic)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
-    if args.impl == "reference":
-        run_reference(args)
+    if args.record_traffic:
+        record_traffic(args.record_traffic)
+        return
+    if args.impl == "reference" and not args.selftest_ranks:
+        run_reference(args)                   # host only: rank 0 works, nothing to spawn
+        return
+    rc = spawn_ranks(args.gpus, sys.argv[1:])
+    if rc is not None:
+        sys.exit(rc)
+    if args.selftest_ranks:
+        run_rank_selftest(args)
     else:
         run_lte(args)
 

@@ -34,6 +34,46 @@ def test_slowest_rank_sets_the_time_and_rate_is_the_aggregate():
         assert abs(rate - 2 * 1000 / 2e-3) < 1e-6
 
 
+def test_bench_starts_its_own_ranks():
+    """`python bench.py --gpus 2` outside a launcher starts two local ranks itself (the same start-up function the GPU
+    run goes through); here with the gloo backend and only the rank plumbing, so that it runs without a GPU."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--backend", "gloo", "--selftest-ranks"],
+                       capture_output=True, text=True, env=env, timeout=300)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [json.loads(l) for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1, r.stdout                               # rank 0 alone prints
+    assert lines[0]["n_gpus"] == 2 and lines[0]["ms_per_step"] == 2.0 and abs(lines[0]["value"] - 2 * 1000 / 2e-3) < 1e-6
+
+
+def test_inside_a_launcher_nothing_is_spawned(monkeypatch):
+    sys.path.insert(0, ROOT)
+    import bench
+    monkeypatch.setenv("RANK", "0"); monkeypatch.setenv("WORLD_SIZE", "2")
+    assert bench.spawn_ranks(2, []) is None
+    monkeypatch.delenv("RANK"); monkeypatch.delenv("WORLD_SIZE")
+    assert bench.spawn_ranks(1, []) is None
+
+
+def test_traffic_figure_is_dropped_when_the_kernel_sources_changed(tmp_path, monkeypatch):
+    import json
+    sys.path.insert(0, ROOT)
+    import bench
+    f = tmp_path / "t.json"
+    monkeypatch.setattr(bench, "TRAFFIC_FILE", str(f))
+    assert bench.ncu_traffic("prefill_attn_C2")[0] is None          # no record at all
+    src = bench.TRAFFIC_SOURCES["prefill_attn_C2"]
+    f.write_text(json.dumps({"prefill_attn_C2": {"dram_bytes_per_launch": 1.5e8, "commit": "abc", "summary": "x.md", "sources": src,
+                                                 "sources_sha256": bench.sources_digest(src)}}))
+    val, prov = bench.ncu_traffic("prefill_attn_C2")
+    assert val == 1.5e8 and prov["sources_unchanged"] and prov["capture_commit"] == "abc"
+    f.write_text(json.dumps({"prefill_attn_C2": {"dram_bytes_per_launch": 1.5e8, "commit": "abc", "summary": "x.md", "sources": src,
+                                                 "sources_sha256": "0" * 64}}))
+    assert bench.ncu_traffic("prefill_attn_C2") == (None, {"capture_commit": "abc", "summary": "x.md", "sources_unchanged": False})
+
+
 def test_single_rank_is_a_no_op():
     sys.path.insert(0, ROOT)
     import bench
