@@ -4,9 +4,16 @@
  * C ABI.  Every tensor pointer is a DEVICE pointer owned by the caller, contiguous with the
  * last index fastest and 16-byte aligned; `lte_shape` / `lte_conv` themselves are HOST structs
  * (their `w` / `bias` members are device pointers).  Unless a function says otherwise the
- * library allocates nothing, keeps no global state, and every call is asynchronous on `stream`
- * (a cudaStream_t passed as void*; NULL = the legacy default stream).  Scratch memory is the
- * caller's: ask lte_workspace_bytes() and pass at least that many bytes.
+ * library allocates nothing and every call is asynchronous on `stream` (a cudaStream_t passed as
+ * void*; NULL = the legacy default stream).  Scratch memory is the caller's: ask
+ * lte_workspace_bytes() and pass at least that many bytes.
+ *
+ * State the library keeps between calls, all of it per device and none of it results: (1) on the
+ * host, a small table per device ordinal, filled on first use under a mutex (SM count, the raised
+ * dynamic-shared-memory limits of its kernels, one symbol address), so any number of host threads
+ * may call into the library on any devices; (2) on each device, one status record per kernel
+ * family (see lte_device_status) and the fixed scratch array of lte_attn_bwd_static.  Calls act
+ * on the device that is current when they are made.
  *
  * Return value: LTE_OK (0) or a negative lte_status; nothing throws or aborts across the ABI.
  * Host-side validation happens before anything is launched.
@@ -83,11 +90,19 @@ typedef enum lte_op {
 size_t lte_workspace_bytes(int op, const lte_shape* s, const lte_conv* c);
 
 /*
- * Sticky device-side status of the current device: LTE_OK, or LTE_ERR_DEVICE_STATUS if a kernel since the
- * last call gave up on a bounded wait (its outputs are then undefined).  Synchronous (a 4-byte copy from
- * the device, ordered after previously launched work on the legacy default stream's rules); reading clears it.
+ * Sticky device-side status of the current device: LTE_OK, or LTE_ERR_DEVICE_STATUS if, since the last call of this
+ * function, a kernel gave up on a bounded wait (the outputs of that launch are undefined) or found its input state other
+ * than the call said (lte_attn_prefill_chunk, lte_cache_score_unrope describe their cases).  The record is per DEVICE
+ * (one word per kernel family), not per cache, workspace or stream: with several caches or streams in flight it tells
+ * that something went wrong on the device, not whose launch it was; synchronise and check after the call you care
+ * about.  Only the launch that recorded an anomaly is affected: launches made after it, before or after the status is
+ * read, wait and run normally.  Synchronous (small copies from the device, ordered after previously launched work by
+ * the legacy default stream's rules); reading clears the record.
  */
 int lte_device_status(void);
+
+/* Diagnostic (no GPU is touched): initialisations the library's per-device host table has run for ordinal `dev`: 1. */
+int lte_selftest_per_device(int dev);
 
 /* Static text for a status code. */
 const char* lte_strerror(int status);
@@ -101,7 +116,8 @@ const char* lte_strerror(int status);
  *   z         out  [B,H,T] fp32
  *   r_or_null out  [B,H,T] fp32 sigmoid(z) (0 where z = -inf), or NULL
  *   ws, ws_bytes   device scratch, used by the three-layer stack only (see lte_conv); may be NULL, 0
- * Errors: INVALID_ARG (NULL, even K, n_layers != 1, dilation != 1, d not in {32,64,128}).
+ * Errors: INVALID_ARG (NULL or misaligned pointer, K even or > 13, W < K); UNSUPPORTED (n_layers other than 1 or 3,
+ * a dilation or kernel other than (1, K) for one layer or (2, 3) for the stack, d not in {32,64,128}, the stack at d = 128).
  */
 int lte_scores(const lte_shape* s, const lte_conv* c, const void* k, const void* v,
                float* z, float* r_or_null, void* ws, size_t ws_bytes, void* stream);

@@ -435,12 +435,9 @@ bwd_tail_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __rest
 // the resident-block slots as well as possible (ties: fewer, larger blocks).  Returns the chunks per sequence.
 inline int tail_chunks(const Params& p, int* rows_out)
 {
-    static int slots = 0;
-    if (slots == 0) {
-        int dev = 0, sms = 148;
-        if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        slots = 2 * sms;
-    }
+    int sms = 148;
+    device_sm_count(&sms);
+    const int slots = 2 * sms;
     const int lo = (p.T + TAIL_MAX_ROWS - 1) / TAIL_MAX_ROWS, hi = (p.T + TAIL_MIN_ROWS - 1) / TAIL_MIN_ROWS;
     int best = lo;
     double best_eff = -1.0;

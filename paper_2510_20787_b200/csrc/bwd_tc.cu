@@ -23,7 +23,7 @@
 
 namespace lte {
 
-__device__ int g_bwd_status = 0;
+__device__ StatusWord g_bwd_status = LTE_STATUS_INIT;
 
 namespace {
 
@@ -67,7 +67,7 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     constexpr uint32_t DP_COL = BN, DQ_COL = DB ? 4 * BN : 2 * BN;
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     const uint32_t base = smem_u32(smem_raw);
-    if ((base & 1023u) != 0) { if (threadIdx.x == 0) atomicExch(&g_bwd_status, 9); return; }
+    if ((base & 1023u) != 0) { if (threadIdx.x == 0) atomicExch(&g_bwd_status.code, 9); return; }
     const uint32_t sQ = base + S::OFF_Q, sDO = base + S::OFF_DO, sK = base + S::OFF_K, sV = base + S::OFF_V;
     const uint32_t sDS = base + S::OFF_DS;
     const uint32_t bar_q = base + S::OFF_BAR, bar_k0 = bar_q + 8, bar_v0 = bar_q + 40, bar_s0 = bar_q + 72;   // 4, 4, 2 slots
@@ -469,7 +469,7 @@ bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     constexpr uint32_t DP_COL = 64, DV_COL = DB ? 256 : 128, DK_COL = DV_COL + D;
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     const uint32_t base = smem_u32(smem_raw);
-    if ((base & 1023u) != 0) { if (threadIdx.x == 0) atomicExch(&g_bwd_status, 9); return; }
+    if ((base & 1023u) != 0) { if (threadIdx.x == 0) atomicExch(&g_bwd_status.code, 9); return; }
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     // the retained tiles walk many more query blocks than the window tiles: they take the lowest block numbers so
     // that they start first and do not form the tail of the launch
@@ -860,12 +860,9 @@ int launch_bwd_dq_tc(const Params& p, const void* q, const void* k, const void* 
     dim3 grid((p.T + BM - 1) / BM, BH);
 #define LTE_GO(D)                                                                                                  \
     do {                                                                                                           \
-        static bool attr_done = false;                                                                             \
-        if (!attr_done) {                                                                                          \
-            if (cudaFuncSetAttribute(bwd_dq_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,      \
-                                     SmemQ<D>::BYTES) != cudaSuccess) return LTE_ERR_CUDA;                         \
-            attr_done = true;                                                                                      \
-        }                                                                                                          \
+        static PerDeviceOnce attr;                                                                                 \
+        if (int e = attr.run([] { return cudaFuncSetAttribute(bwd_dq_tc_kernel<D>,                                 \
+                cudaFuncAttributeMaxDynamicSharedMemorySize, SmemQ<D>::BYTES); })) return e;                       \
         launch_pdl(bwd_dq_tc_kernel<D>, grid, dim3(NTHREADS), SmemQ<D>::BYTES, st,                            \
             tq, tdo, to, tdq, tk, tv, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (const __nv_bfloat16*)o,        \
             (const __nv_bfloat16*)dO, lse, idx, cnt, (__nv_bfloat16*)dq, delta, p.T, p.W, p.R, p.scale, p.G);      \
@@ -900,12 +897,9 @@ int launch_bwd_dkv_tc(const Params& p, const void* q, const void* k, const void*
     dim3 grid(n_wt + n_rt, BH);
 #define LTE_GO(D, F)                                                                                               \
     do {                                                                                                           \
-        static bool attr_done = false;                                                                             \
-        if (!attr_done) {                                                                                          \
-            if (cudaFuncSetAttribute(bwd_dkv_tc_kernel<D, F>, cudaFuncAttributeMaxDynamicSharedMemorySize,          \
-                                     SmemK<D>::BYTES) != cudaSuccess) return LTE_ERR_CUDA;                         \
-            attr_done = true;                                                                                      \
-        }                                                                                                          \
+        static PerDeviceOnce attr;                                                                                 \
+        if (int e = attr.run([] { return cudaFuncSetAttribute(bwd_dkv_tc_kernel<D, F>,                             \
+                cudaFuncAttributeMaxDynamicSharedMemorySize, SmemK<D>::BYTES); })) return e;                       \
         launch_pdl(bwd_dkv_tc_kernel<D, F>, grid, dim3(NTHREADS), SmemK<D>::BYTES, st,                              \
             tk, tv, tq, tdo, tdk, tdv, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, lse, delta, idx, cnt,     \
             (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, dk32, dv32, dz, dk_ret, dv_ret, dr_ret, n_wt, p.T, p.W, p.R,   \
@@ -929,12 +923,6 @@ int launch_bwd_dkv_tc(const Params& p, const void* q, const void* k, const void*
     return cuda_status(cudaGetLastError());
 }
 
-int bwd_status_fetch_and_clear()
-{
-    int h = 0, zero = 0;
-    if (cudaMemcpyFromSymbol(&h, g_bwd_status, sizeof(int)) != cudaSuccess) return -1;
-    if (h != 0) cudaMemcpyToSymbol(g_bwd_status, &zero, sizeof(int));
-    return h;
-}
+int bwd_status_fetch_and_clear() { return status_fetch_and_clear(g_bwd_status); }
 
 }  // namespace lte

@@ -15,7 +15,7 @@
 
 namespace lte {
 
-__device__ int g_chunk_status = 0;            // 0 = fine; 31: the cache does not hold n_past tokens
+__device__ StatusWord g_chunk_status = LTE_STATUS_INIT;   // report only; 31: the cache does not hold n_past tokens
 
 namespace {
 
@@ -26,11 +26,13 @@ constexpr int kRowsPerBlock = 128;
 
 // Block (part, (b,h)): rows [part 128, part 128 + 128) of the local sequence: pool rows, ring rows (time order) and the
 // chunk's rows of k, v.  Part 0 also copies the logits of the pool and the ring into zsrc [R0 + Wn] and the pool's
-// positions into oldpos [R].
+// positions into oldpos [R], and writes gate[b,h] = 1 if the head's cache holds n0 tokens as the call said, else 0 (the
+// head's cache is then left alone by the commit of this same call; the flag lives in the call's scratch, so it says
+// nothing about any other call).
 __global__ void chunk_gather_kernel(const unsigned char* __restrict__ cache, CacheLayout L, const unsigned char* __restrict__ kc,
                                     const unsigned char* __restrict__ vc, unsigned char* __restrict__ klin,
                                     unsigned char* __restrict__ vlin, float* __restrict__ zsrc, int32_t* __restrict__ oldpos,
-                                    int D, int W, int R, int n0, int R0, int Wn, int Tloc)
+                                    int32_t* __restrict__ gate, int D, int W, int R, int n0, int R0, int Wn, int Tloc)
 {
     const int bh = blockIdx.y;
     const unsigned char* blk = cache + L.header + (size_t)bh * L.stride;
@@ -39,7 +41,11 @@ __global__ void chunk_gather_kernel(const unsigned char* __restrict__ cache, Cac
     const float* zc = reinterpret_cast<const float*>(blk + L.off_z);
     const int32_t* pidx = reinterpret_cast<const int32_t*>(blk + L.off_pidx);
     const int32_t* meta = reinterpret_cast<const int32_t*>(blk + L.off_meta);
-    if (meta[0] != n0) { if (threadIdx.x == 0) atomicExch(&g_chunk_status, 31); return; }
+    if (meta[0] != n0) {
+        if (threadIdx.x == 0) { atomicExch(&g_chunk_status.code, 31); if (blockIdx.x == 0) gate[bh] = 0; }
+        return;
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) gate[bh] = 1;
     const int cnt = meta[1];
     const int pieces = D * (int)L.esz / 16;                    // 16-byte pieces per row
     uint4* kd = reinterpret_cast<uint4*>(klin) + (size_t)bh * Tloc * pieces;
@@ -114,11 +120,11 @@ __global__ void chunk_merge_z_kernel(float* __restrict__ z, float* __restrict__ 
 __global__ void chunk_commit_kernel(unsigned char* __restrict__ cache, CacheLayout L, const unsigned char* __restrict__ klin,
                                     const unsigned char* __restrict__ vlin, const float* __restrict__ z,
                                     const int32_t* __restrict__ idx, const int32_t* __restrict__ cntp,
-                                    const int32_t* __restrict__ oldpos, int D, int W, int R, int n0, int n1, int R0, int Wn,
-                                    int Tloc, int half)
+                                    const int32_t* __restrict__ oldpos, const int32_t* __restrict__ gate, int D, int W, int R,
+                                    int n0, int n1, int R0, int Wn, int Tloc, int half)
 {
-    if (*reinterpret_cast<volatile int*>(&g_chunk_status) != 0) return;   // the gather found another state: leave the cache alone
     const int bh = blockIdx.y;
+    if (gate[bh] == 0) return;                                 // this call's gather found another state: leave the cache alone
     unsigned char* blk = cache + L.header + (size_t)bh * L.stride;
     uint4* Kc = reinterpret_cast<uint4*>(blk + L.off_k);
     uint4* Vc = reinterpret_cast<uint4*>(blk + L.off_v);
@@ -161,22 +167,16 @@ __global__ void chunk_commit_kernel(unsigned char* __restrict__ cache, CacheLayo
 
 }  // namespace
 
-int chunk_status_fetch_and_clear()
-{
-    int h = 0, zero = 0;
-    if (cudaMemcpyFromSymbol(&h, g_chunk_status, sizeof(int)) != cudaSuccess) return -1;
-    if (h != 0) cudaMemcpyToSymbol(g_chunk_status, &zero, sizeof(int));
-    return h;
-}
+int chunk_status_fetch_and_clear() { return status_fetch_and_clear(g_chunk_status); }
 
 // p.T = local length; the launchers run on one stream in the order gather, (scores), merge, (select, attention), commit
 int launch_chunk_gather(const Params& p, const void* cache, const void* k, const void* v, void* klin, void* vlin, float* zsrc,
-                        int32_t* oldpos, int n0, int R0, int Wn, cudaStream_t st)
+                        int32_t* oldpos, int32_t* gate, int n0, int R0, int Wn, cudaStream_t st)
 {
     const CacheLayout L = cache_layout(p.d, p.W, p.R, p.dtype);
     dim3 grid((p.T + kRowsPerBlock - 1) / kRowsPerBlock, p.B * p.H);
     chunk_gather_kernel<<<grid, 256, 0, st>>>((const unsigned char*)cache, L, (const unsigned char*)k, (const unsigned char*)v,
-                                              (unsigned char*)klin, (unsigned char*)vlin, zsrc, oldpos, p.d, p.W, p.R, n0, R0, Wn, p.T);
+                                              (unsigned char*)klin, (unsigned char*)vlin, zsrc, oldpos, gate, p.d, p.W, p.R, n0, R0, Wn, p.T);
     return cuda_status(cudaGetLastError());
 }
 
@@ -189,12 +189,13 @@ int launch_chunk_merge_z(const Params& p, float* z, float* zrank, const float* z
 }
 
 int launch_chunk_commit(const Params& p, void* cache, const void* klin, const void* vlin, const float* z, const int32_t* idx,
-                        const int32_t* cnt, const int32_t* oldpos, int n0, int n1, int R0, int Wn, cudaStream_t st)
+                        const int32_t* cnt, const int32_t* oldpos, const int32_t* gate, int n0, int n1, int R0, int Wn,
+                        cudaStream_t st)
 {
     const CacheLayout L = cache_layout(p.d, p.W, p.R, p.dtype);
     dim3 grid((p.W + p.R + kRowsPerBlock - 1) / kRowsPerBlock, p.B * p.H);
     chunk_commit_kernel<<<grid, 256, 0, st>>>((unsigned char*)cache, L, (const unsigned char*)klin, (const unsigned char*)vlin, z,
-                                                   idx, cnt, oldpos, p.d, p.W, p.R, n0, n1, R0, Wn, p.T, p.half);
+                                                   idx, cnt, oldpos, gate, p.d, p.W, p.R, n0, n1, R0, Wn, p.T, p.half);
     return cuda_status(cudaGetLastError());
 }
 

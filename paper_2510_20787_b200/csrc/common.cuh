@@ -5,6 +5,8 @@
 #include <math.h>
 #include <stdint.h>
 
+#include <mutex>
+
 #include "lte.h"
 
 namespace lte {
@@ -109,11 +111,12 @@ int launch_ring_linearize(const Params& p, const void* cache, void* klin, void* 
                           int rope_len, cudaStream_t st);
 int launch_ring_scatter_z(const Params& p, void* cache, const float* zlin, cudaStream_t st);
 int launch_chunk_gather(const Params& p, const void* cache, const void* k, const void* v, void* klin, void* vlin, float* zsrc,
-                        int32_t* oldpos, int n0, int R0, int Wn, cudaStream_t st);
+                        int32_t* oldpos, int32_t* gate, int n0, int R0, int Wn, cudaStream_t st);
 int launch_chunk_merge_z(const Params& p, float* z, float* zrank, const float* zsrc, const int32_t* oldpos, int n0, int R0, int Wn,
                          cudaStream_t st);
 int launch_chunk_commit(const Params& p, void* cache, const void* klin, const void* vlin, const float* z, const int32_t* idx,
-                        const int32_t* cnt, const int32_t* oldpos, int n0, int n1, int R0, int Wn, cudaStream_t st);
+                        const int32_t* cnt, const int32_t* oldpos, const int32_t* gate, int n0, int n1, int R0, int Wn,
+                        cudaStream_t st);
 int chunk_status_fetch_and_clear();
 int launch_sparsity_stats(const Params& p, const float* z, const float* lambda, float* count, float* penalty, float* part, float tau,
                           cudaStream_t st);
@@ -128,6 +131,62 @@ int launch_bwd(const Params& p, const void* q, const void* k, const void* v, con
                cudaStream_t st);
 
 inline int cuda_status(cudaError_t e) { return e == cudaSuccess ? LTE_OK : LTE_ERR_CUDA; }
+
+// Device-side status of one kernel family (a __device__ variable per family, so one per device).
+//   code        sticky report for the host: 0, or the code of the first anomaly since lte_device_status() last read it
+//               (a bounded wait that gave up, a cache in another state than the call said, ...).  Never read by kernels.
+//   abort_grid  grid id of the launch whose bounded wait gave up last (~0 = none): only the waits of that same launch
+//               look at it, to end the lost launch quickly.  A later launch has another grid id and waits normally.
+struct StatusWord { int code; int pad; unsigned long long abort_grid; };
+#define LTE_STATUS_INIT {0, 0, ~0ull}
+template <typename Sym> inline int status_fetch_and_clear(const Sym& sym)
+{
+    StatusWord h;
+    if (cudaMemcpyFromSymbol(&h, sym, sizeof(h)) != cudaSuccess) return -1;
+    if (h.code != 0 || h.abort_grid != ~0ull) {
+        const StatusWord z = LTE_STATUS_INIT;
+        if (cudaMemcpyToSymbol(sym, &z, sizeof(z)) != cudaSuccess) return -1;
+    }
+    return h.code;
+}
+
+// Host-side facts that belong to a device, not to the process: looked up (or applied) once per device ordinal, under a
+// mutex, by whichever thread gets there first with that device current.  `init` returns an lte_status; a failed init
+// is retried by the next call.
+constexpr int kMaxDevices = 64;
+template <typename T> class PerDevice {
+public:
+    template <typename F> int get(T* out, F&& init)
+    {
+        int dev = -1;
+        if (cudaGetDevice(&dev) != cudaSuccess) return LTE_ERR_CUDA;
+        return get_for(dev, out, init);
+    }
+    template <typename F> int get_for(int dev, T* out, F&& init)
+    {
+        if (dev < 0 || dev >= kMaxDevices) return LTE_ERR_UNSUPPORTED;
+        std::lock_guard<std::mutex> lock(mu_);
+        if (!have_[dev]) {
+            const int e = init(&val_[dev]);
+            if (e != LTE_OK) return e;
+            have_[dev] = true;
+        }
+        if (out) *out = val_[dev];
+        return LTE_OK;
+    }
+private:
+    std::mutex mu_;
+    bool have_[kMaxDevices] = {};
+    T val_[kMaxDevices] = {};
+};
+// cudaFuncSetAttribute(MaxDynamicSharedMemorySize) and the like: once per device.  `f` returns a cudaError_t.
+class PerDeviceOnce {
+public:
+    template <typename F> int run(F&& f) { return t_.get(nullptr, [&](char*) { return cuda_status(f()); }); }
+private:
+    PerDevice<char> t_;
+};
+int device_sm_count(int* n_sm);       // SM count of the current device
 
 // Programmatic dependent launch: a kernel launched through launch_pdl may become resident while its predecessor in the
 // stream is still running, and does its set-up (barriers, tensor memory, index arithmetic) there.  It must execute

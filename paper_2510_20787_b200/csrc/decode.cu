@@ -287,7 +287,7 @@ __global__ void __launch_bounds__(DT) decode_kernel(unsigned char* __restrict__ 
 // key buffer is refilled with head i+1's keys, and after the PV pass the value buffer is refilled likewise, so
 // the loads of the next head run under the softmax / PV / write-back of the current one.  Everything is computed
 // out of shared memory; only the rows that change go back to HBM.  Used when a block fits (it does at W+R = 256).
-__device__ int g_decode_status = 0;
+__device__ StatusWord g_decode_status = LTE_STATUS_INIT;   // report only: no wait polls it
 #ifdef LTE_PROFILE
 __device__ long long g_dprof[64];
 #define DPROF(slot) do { if (blockIdx.x == 7 && threadIdx.x == 96 && it == 2) g_dprof[slot] = clock64(); } while (0)
@@ -415,7 +415,7 @@ __global__ void __launch_bounds__(DT) decode_bulk_kernel(unsigned char* __restri
         }
         __syncthreads();
         if (s_flag) {                                           // bounded wait ran out: give up, outputs undefined
-            if (tid == 0) atomicExch(&g_decode_status, 1);
+            if (tid == 0) atomicExch(&g_decode_status.code, 1);
             return;
         }
         DPROF(1);
@@ -664,13 +664,7 @@ __global__ void cache_init_kernel(unsigned char* __restrict__ cache, CacheLayout
 
 }  // namespace
 
-int decode_status_fetch_and_clear()
-{
-    int h = 0, zero = 0;
-    if (cudaMemcpyFromSymbol(&h, g_decode_status, sizeof(int)) != cudaSuccess) return -1;
-    if (h != 0) cudaMemcpyToSymbol(g_decode_status, &zero, sizeof(int));
-    return h;
-}
+int decode_status_fetch_and_clear() { return status_fetch_and_clear(g_decode_status); }
 
 int launch_cache_init(const Params& p, const void* k, const void* v, const float* z, const int32_t* idx,
                       const int32_t* cnt, void* cache, cudaStream_t st)
@@ -725,7 +719,7 @@ __global__ void ring_linearize_kernel(const unsigned char* __restrict__ cache, C
                     // inverse rotation: (x1, x2) -> (x1 cos + x2 sin, x2 cos - x1 sin)
                     kx = from_f<T>(c < hd ? a * co + b * si : a * co - b * si);
                 } else if (c == 0) {
-                    atomicExch(&g_decode_status, 32);              // the tables do not reach this position: key left rotated
+                    atomicExch(&g_decode_status.code, 32);              // the tables do not reach this position: key left rotated
                 }
             }
         }
@@ -1092,25 +1086,17 @@ static int launch_decode_step(const Params& p, void* cache, const void* q1, cons
     const BulkSmem bp = bulk_smem_plan(L, p.W, p.R);
     const size_t bulk_smem = bp.total;
     const bool bulk = bulk_smem <= 73 * 1024 && p.K <= 2 * (DT / 32);   // three blocks per SM still fit
-    static int n_sm = 0;
-    if (bulk && n_sm == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-            return LTE_ERR_CUDA;
-    }
+    int n_sm = 0;
+    if (int e = device_sm_count(&n_sm)) return e;
     // persistent grid: every CTA walks `per_cta` consecutive heads; all CTAs are resident (3 per SM)
     const int BH = p.B * p.H;
     const int per_cta = bulk ? (BH + 3 * n_sm - 1) / (3 * n_sm) : 1;
     const int n_cta = bulk ? (BH + per_cta - 1) / per_cta : BH;
 #define LTE_BULK(T, D)                                                                                            \
     do {                                                                                                          \
-        static bool attr_done = false;                                                                            \
-        if (!attr_done) {                                                                                         \
-            if (cudaFuncSetAttribute(decode_bulk_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,        \
-                                     73 * 1024) != cudaSuccess) return LTE_ERR_CUDA;                              \
-            attr_done = true;                                                                                     \
-        }                                                                                                         \
+        static PerDeviceOnce attr;                                                                                \
+        if (int e = attr.run([] { return cudaFuncSetAttribute(decode_bulk_kernel<T, D>,                           \
+                cudaFuncAttributeMaxDynamicSharedMemorySize, 73 * 1024); })) return e;                            \
         decode_bulk_kernel<T, D><<<n_cta, DT, bulk_smem, st>>>((unsigned char*)cache, L, (const T*)q1,             \
             (const T*)k1, (const T*)v1, (T*)o1, lse1, p.w, p.bias, BH, per_cta, p.H, p.W, p.R, p.sink, p.K,        \
             p.zthr, p.scale, p.G);                                                                                     \
@@ -1169,12 +1155,8 @@ int launch_decode(const Params& p, void* cache, const void* q1, const void* k1, 
     const size_t att_smem = sizeof(float) * ((size_t)ATT_Q * (p.W + p.R) + (size_t)(DT / 32) * ATT_Q * p.d);
     // blocks per key/value head (a cluster): more than one only while there are fewer blocks than SMs and a share keeps 256 rows
     // (with 256 heads of 1280 rows, two blocks per head measured 41 us per step against 29 us for one)
-    static int n_sm_att = 0;
-    if (n_sm_att == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n_sm_att, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-            return LTE_ERR_CUDA;
-    }
+    int n_sm_att = 0;
+    if (int e = device_sm_count(&n_sm_att)) return e;
     int nsplit = 1;
     while (nsplit < 8 && p.B * p.H * nsplit < n_sm_att && (p.W + p.R) / (2 * nsplit) >= 256) nsplit *= 2;
     cudaLaunchConfig_t acfg = {};
@@ -1185,13 +1167,10 @@ int launch_decode(const Params& p, void* cache, const void* q1, const void* k1, 
     acfg.attrs = aattr; acfg.numAttrs = 1;
 #define LTE_ATT(T, D)                                                                                                  \
     do {                                                                                                               \
-        static bool attr_done = false;                                                                                 \
-        if (!attr_done) {                                                                                              \
-            if (cudaFuncSetAttribute(decode_attend_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,           \
-                                     (int)(sizeof(float) * ((size_t)ATT_Q * MAX_ROWS + (DT / 32) * ATT_Q * 128))) != cudaSuccess) \
-                return LTE_ERR_CUDA;                                                                                   \
-            attr_done = true;                                                                                          \
-        }                                                                                                              \
+        static PerDeviceOnce attr;                                                                                     \
+        if (int e = attr.run([] { return cudaFuncSetAttribute(decode_attend_kernel<T, D>,                              \
+                cudaFuncAttributeMaxDynamicSharedMemorySize,                                                           \
+                (int)(sizeof(float) * ((size_t)ATT_Q * MAX_ROWS + (DT / 32) * ATT_Q * 128))); })) return e;            \
         if (cudaLaunchKernelEx(&acfg, decode_attend_kernel<T, D>, (unsigned char*)cache, L, (const T*)q1, (T*)o1, lse1,        \
                                p.W, p.G, p.scale, 0, (const T*)k1, (const T*)v1, p.w, p.bias, p.H, p.R, p.sink, ps.K,    \
                                p.zthr) != cudaSuccess) return LTE_ERR_CUDA;                                             \

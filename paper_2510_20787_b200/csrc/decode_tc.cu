@@ -16,7 +16,7 @@
 
 namespace lte {
 
-__device__ int g_decode_tc_status = 0;
+__device__ StatusWord g_decode_tc_status = LTE_STATUS_INIT;
 
 namespace {
 
@@ -59,7 +59,7 @@ __global__ void __launch_bounds__(NTHR) decode_tc_kernel(unsigned char* __restri
     extern __shared__ __align__(1024) unsigned char dsm[];
     const Plan P = plan_of(L);
     const uint32_t base = smem_u32(dsm);
-    if ((base & 1023u) != 0) { if (threadIdx.x == 0) atomicExch(&g_decode_tc_status, 9); return; }
+    if ((base & 1023u) != 0) { if (threadIdx.x == 0) atomicExch(&g_decode_tc_status.code, 9); return; }
     const uint32_t sK = base, sV = base + P.off_v, sT = base + P.off_tail, sQ = base + P.off_q, sP = base + P.off_p;
     const uint32_t bar_k = base + P.off_bar, bar_v = bar_k + 8, bar_t0 = bar_k + 16;     // bar_t0, bar_t0 + 8
     const uint32_t bar_q = bar_k + 32, bar_s = bar_k + 40, bar_p = bar_k + 48, bar_o = bar_k + 56, tmem_slot = bar_k + 64;
@@ -339,16 +339,10 @@ int launch_decode_tc(const Params& p, void* cache, const void* q1, const void* k
     const CacheLayout L = cache_layout(p.d, p.W, p.R, p.dtype);
     if (!L.swz || p.K > 16) return LTE_ERR_UNSUPPORTED;
     const Plan P = plan_of(L);
-    static int n_sm = 0;
-    static bool attr_done = false;
-    if (!attr_done) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
-            cudaFuncSetAttribute(decode_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 80 * 1024) != cudaSuccess)
-            return LTE_ERR_CUDA;
-        attr_done = true;
-    }
+    static PerDeviceOnce attr;
+    if (int e = attr.run([] { return cudaFuncSetAttribute(decode_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 80 * 1024); })) return e;
+    int n_sm = 0;
+    if (int e = device_sm_count(&n_sm)) return e;
     if (P.total > 80 * 1024) return LTE_ERR_UNSUPPORTED;
     const int BH = p.B * p.H;
     const int slots = 3 * n_sm;                                // three CTAs per SM
@@ -359,12 +353,6 @@ int launch_decode_tc(const Params& p, void* cache, const void* q1, const void* k
                                                    p.w, p.bias, BH, per_cta, p.H, p.W, p.R, p.sink, p.K, p.zthr, p.scale, p.G));
 }
 
-int decode_tc_status_fetch_and_clear()
-{
-    int h = 0, zero = 0;
-    if (cudaMemcpyFromSymbol(&h, g_decode_tc_status, sizeof(int)) != cudaSuccess) return -1;
-    if (h != 0) cudaMemcpyToSymbol(g_decode_tc_status, &zero, sizeof(int));
-    return h;
-}
+int decode_tc_status_fetch_and_clear() { return status_fetch_and_clear(g_decode_tc_status); }
 
 }  // namespace lte

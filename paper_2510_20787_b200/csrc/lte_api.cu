@@ -1,7 +1,7 @@
 // C-ABI entry points of liblte: argument validation and dispatch.  No torch types, no allocation.
 #include <math.h>
 
-#include <mutex>
+#include <atomic>
 
 #include "common.cuh"
 
@@ -16,6 +16,18 @@ int stack_tc_status_fetch_and_clear();
 int stack_bwd_tc_status_fetch_and_clear();
 int bwd_status_fetch_and_clear();
 int decode_tc_status_fetch_and_clear();
+
+// SM count of the current device, looked up once per device
+int device_sm_count(int* n_sm)
+{
+    static PerDevice<int> table;
+    return table.get(n_sm, [](int* out) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(out, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || *out <= 0)
+            return (int)LTE_ERR_CUDA;
+        return (int)LTE_OK;
+    });
+}
 
 namespace {
 
@@ -98,7 +110,7 @@ CacheScorePlan cache_score_plan(const lte_shape* s, const lte_conv* c)
 }
 
 // scratch of lte_attn_prefill_chunk, sized for the longest local sequence (pool rows + full ring + chunk)
-struct ChunkPlan { size_t klin, vlin, z, zrank, zsrc, oldpos, idx, cnt, sub, att, total; };
+struct ChunkPlan { size_t klin, vlin, z, zrank, zsrc, oldpos, idx, cnt, gate, sub, att, total; };
 ChunkPlan chunk_plan(const lte_shape* s, const lte_conv* c)
 {
     auto up = [](size_t x) { return (x + 255) / 256 * 256; };
@@ -114,6 +126,7 @@ ChunkPlan chunk_plan(const lte_shape* s, const lte_conv* c)
     w.oldpos = off; off += up(bhk * (size_t)(s->R > 0 ? s->R : 1) * 4);
     w.idx = off; off += up(bhk * (size_t)(s->R > 0 ? s->R : 1) * 4);
     w.cnt = off; off += up(bhk * 4);
+    w.gate = off; off += up(bhk * 4);                        // per head: the cache held n_past tokens (written by every call's gather)
     w.sub = off;
     if (c && c->n_layers == 3) {
         lte_shape s2 = *s; s2.T = (int32_t)Tm;
@@ -307,7 +320,8 @@ int lte_attn_prefill_chunk(const lte_shape* s, const lte_conv* c, void* cache, i
     Params patt = p; patt.qoff = qoff;                       // the queries are the chunk's: positions qoff .. Tloc-1
     float* z = (float*)(base + w.z); float* zrank = (float*)(base + w.zrank); float* zsrc = (float*)(base + w.zsrc);
     int32_t* oldpos = (int32_t*)(base + w.oldpos); int32_t* idx = (int32_t*)(base + w.idx); int32_t* cnt = (int32_t*)(base + w.cnt);
-    e = launch_chunk_gather(p, cache, k, v, base + w.klin, base + w.vlin, zsrc, oldpos, n_past, R0, Wn, st); if (e) return e;
+    int32_t* gate = (int32_t*)(base + w.gate);
+    e = launch_chunk_gather(p, cache, k, v, base + w.klin, base + w.vlin, zsrc, oldpos, gate, n_past, R0, Wn, st); if (e) return e;
     if (p.stack) {
         e = launch_scores_stack_tc(p, base + w.klin, base + w.vlin, z, nullptr, base + w.sub, w.att - w.sub, st);
         if (e == LTE_ERR_UNSUPPORTED) e = launch_scores_stack(p, base + w.klin, base + w.vlin, z, nullptr, st);
@@ -321,7 +335,7 @@ int lte_attn_prefill_chunk(const lte_shape* s, const lte_conv* c, void* cache, i
     if (s->dtype == LTE_BF16) e = launch_prefill_tc(patt, q, base + w.klin, base + w.vlin, idx, cnt, o, lse, base + w.att, w.total - w.att, st);
     else e = launch_prefill_simt(patt, q, base + w.klin, base + w.vlin, idx, cnt, o, lse, st);
     if (e) return e;
-    return launch_chunk_commit(p, cache, base + w.klin, base + w.vlin, z, idx, cnt, oldpos, n_past, n_past + Tc, R0, Wn, st);
+    return launch_chunk_commit(p, cache, base + w.klin, base + w.vlin, z, idx, cnt, oldpos, gate, n_past, n_past + Tc, R0, Wn, st);
 }
 
 int lte_attn_decode(const lte_shape* s, const lte_conv* c, void* cache, const void* q1, const void* k1,
@@ -401,23 +415,31 @@ int lte_attn_bwd(const lte_shape* s, const lte_conv* c, const void* q, const voi
 static __device__ __align__(256) unsigned char g_bwd_static_scratch[LTE_STATIC_SCRATCH_BYTES];
 
 namespace {
-std::mutex g_static_mu;
-void* g_static_ptr[64] = {nullptr};          /* resolved device address of the array, per device ordinal */
-
-/* Device address of the scratch array on the current device (resolved on first use), or NULL on failure. */
+/* Device address of the scratch array on the current device (resolved on first use, per device ordinal), or NULL. */
 void* static_scratch_for_current_device()
 {
-    int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
-    std::lock_guard<std::mutex> lock(g_static_mu);
-    if (!g_static_ptr[dev]) {
-        void* p = nullptr;
-        if (cudaGetSymbolAddress(&p, g_bwd_static_scratch) != cudaSuccess) return nullptr;
-        g_static_ptr[dev] = p;
-    }
-    return g_static_ptr[dev];
+    static PerDevice<void*> table;
+    void* p = nullptr;
+    const int e = table.get(&p, [](void** out) {
+        return cuda_status(cudaGetSymbolAddress(out, g_bwd_static_scratch));
+    });
+    return e == LTE_OK ? p : nullptr;
 }
 }  // namespace
+
+/* Diagnostic for the per-device table every launcher keeps its once-per-device facts in (SM count, raised shared-memory
+ * limits, symbol addresses): looks `dev` up in a table of its own and returns how many times the table has run the
+ * initialiser for that device so far: 1, however many threads ask at once.  Touches no GPU. */
+int lte_selftest_per_device(int dev)
+{
+    static PerDevice<int> table;
+    static std::atomic<int> inits[kMaxDevices];
+    if (dev < 0 || dev >= kMaxDevices) return LTE_ERR_INVALID_ARG;
+    int v = 0;
+    const int e = table.get_for(dev, &v, [dev](int* out) { *out = dev + 1000; inits[dev].fetch_add(1); return (int)LTE_OK; });
+    if (e != LTE_OK || v != dev + 1000) return LTE_ERR_DEVICE_STATUS;
+    return inits[dev].load();
+}
 
 int lte_attn_bwd_static(const lte_shape* s, const lte_conv* c, const void* q, const void* k, const void* v,
                         const void* o, const float* lse, const void* dO, const float* z, const int32_t* idx,

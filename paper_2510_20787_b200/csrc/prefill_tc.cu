@@ -21,7 +21,7 @@
 
 namespace lte {
 
-__device__ int g_prefill_status = 0;          // 0 = fine; otherwise the code of the wait that gave up
+__device__ StatusWord g_prefill_status = LTE_STATUS_INIT;         // 0 = fine; otherwise the code of the wait that gave up
 
 namespace {
 
@@ -116,7 +116,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     const uint32_t base = smem_u32(smem_raw);
     if ((base & 1023u) != 0) {                                 // the swizzled tiles need 1024-byte alignment
-        if (threadIdx.x == 0) atomicExch(&g_prefill_status, 9);
+        if (threadIdx.x == 0) atomicExch(&g_prefill_status.code, 9);
         return;
     }
     const uint32_t sQ = base + S::OFF_Q, sK = base + S::OFF_K, sV = base + S::OFF_V;
@@ -587,17 +587,14 @@ int run(const Params& p, const void* q, const void* k, const void* v, const int3
         if (int e = launch_prefill_compact(p, k, v, idx, cnt, kc, vc, st)) return e;
         if (!make_map(&tkc, kc, BHK, p.R, D, BN) || !make_map(&tvc, vc, BHK, p.R, D, BN)) return LTE_ERR_CUDA;
     }
-    static int slots = 0;                                      // resident CTAs: two per SM
-    if (slots == 0) {
-        if (cudaFuncSetAttribute(prefill_tc_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::BYTES) != cudaSuccess ||
-            cudaFuncSetAttribute(prefill_tc_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::BYTES) != cudaSuccess)
-            return LTE_ERR_CUDA;
-        int dev = 0, sms = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
-            return LTE_ERR_CUDA;
-        slots = 2 * sms;
-    }
+    static PerDeviceOnce attr;
+    if (int e = attr.run([] {
+            const cudaError_t a = cudaFuncSetAttribute(prefill_tc_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::BYTES);
+            return a != cudaSuccess ? a : cudaFuncSetAttribute(prefill_tc_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::BYTES);
+        })) return e;
+    int sms = 0;
+    if (int e = device_sm_count(&sms)) return e;
+    const int slots = 2 * sms;                                 // resident CTAs: two per SM
     const int n_qt = (Tq + BM - 1) / BM, n_items = n_qt * BH;
     const int grid = n_items < slots ? n_items : slots;
     if (compact)
@@ -625,10 +622,7 @@ int launch_prefill_tc(const Params& p, const void* q, const void* k, const void*
 
 int prefill_status_fetch_and_clear()
 {
-    int h = 0, zero = 0;
-    if (cudaMemcpyFromSymbol(&h, g_prefill_status, sizeof(int)) != cudaSuccess) return -1;
-    if (h != 0) cudaMemcpyToSymbol(g_prefill_status, &zero, sizeof(int));
-    const int h2 = prefill_long_status_fetch_and_clear();
+    const int h = status_fetch_and_clear(g_prefill_status), h2 = prefill_long_status_fetch_and_clear();
     return h != 0 ? h : h2;
 }
 

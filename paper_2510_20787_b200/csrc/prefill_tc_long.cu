@@ -11,7 +11,7 @@
 
 namespace lte {
 
-__device__ int g_prefill_long_status = 0;     // 0 = fine; otherwise the code of the wait that gave up
+__device__ StatusWord g_prefill_long_status = LTE_STATUS_INIT; // 0 = fine; otherwise the code of the wait that gave up
 
 
 #ifdef LTE_PROFILE
@@ -89,7 +89,7 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     const uint32_t base = smem_u32(smem_raw);
     if ((base & 1023u) != 0) {                                 // the swizzled tiles need 1024-byte alignment
-        if (threadIdx.x == 0) atomicExch(&g_prefill_long_status, 9);
+        if (threadIdx.x == 0) atomicExch(&g_prefill_long_status.code, 9);
         return;
     }
     const uint32_t sQ = base + S::OFF_Q, sK = base + S::OFF_K, sV = base + S::OFF_V;
@@ -590,13 +590,11 @@ int run(const Params& p, const void* q, const void* k, const void* v, const int3
         if (int e = launch_prefill_compact(p, k, v, idx, cnt, kc, vc, st)) return e;
         if (!make_map(&tkc, kc, BHK, p.R, D, BN) || !make_map(&tvc, vc, BHK, p.R, D, BN)) return LTE_ERR_CUDA;
     }
-    static bool attr_done = false;
-    if (!attr_done) {
-        if (cudaFuncSetAttribute(prefill_long_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::BYTES) != cudaSuccess ||
-            cudaFuncSetAttribute(prefill_long_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::BYTES) != cudaSuccess)
-            return LTE_ERR_CUDA;
-        attr_done = true;
-    }
+    static PerDeviceOnce attr;
+    if (int e = attr.run([] {
+            const cudaError_t a = cudaFuncSetAttribute(prefill_long_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::BYTES);
+            return a != cudaSuccess ? a : cudaFuncSetAttribute(prefill_long_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::BYTES);
+        })) return e;
     dim3 grid((Tq + BM - 1) / BM, BH);
     if (compact)
         return cuda_status(launch_pdl(prefill_long_kernel<D, true>, grid, dim3(NTHREADS), Smem<D>::BYTES, st, tq, tk, tv, to, tkc, tvc, (const __nv_bfloat16*)k,
@@ -640,12 +638,6 @@ extern "C" void lte_plprof_read(unsigned long long* out, int clear)
 }
 #endif
 
-int prefill_long_status_fetch_and_clear()
-{
-    int h = 0, zero = 0;
-    if (cudaMemcpyFromSymbol(&h, g_prefill_long_status, sizeof(int)) != cudaSuccess) return -1;
-    if (h != 0) cudaMemcpyToSymbol(g_prefill_long_status, &zero, sizeof(int));
-    return h;
-}
+int prefill_long_status_fetch_and_clear() { return status_fetch_and_clear(g_prefill_long_status); }
 
 }  // namespace lte

@@ -8,6 +8,9 @@
 #include "tc_common.cuh"
 
 namespace lte {
+
+__device__ StatusWord g_scores_status = LTE_STATUS_INIT;
+
 namespace {
 
 constexpr int NT = 128;
@@ -131,7 +134,7 @@ __global__ void __launch_bounds__(NT + 64) scores_tc_kernel(const __grid_constan
                                                        const __grid_constant__ CUtensorMap tmV,
                                                        const float* __restrict__ w, const float* __restrict__ bias,
                                                        float* __restrict__ z, float* __restrict__ r, int H, int Tlen,
-                                                       int n_flat, int* __restrict__ status)
+                                                       int n_flat)
 {
     using C = ScoresTc<D, K>;
     constexpr int HALF = K / 2;
@@ -151,7 +154,7 @@ __global__ void __launch_bounds__(NT + 64) scores_tc_kernel(const __grid_constan
     const int n_tiles = f_end - f_begin;
     if (n_tiles <= 0) return;
 
-    if ((tile0 & 1023u) != 0) { if (tid == 0) atomicExch(status, 8); return; }
+    if ((tile0 & 1023u) != 0) { if (tid == 0) atomicExch(&g_scores_status.code, 8); return; }
     const uint32_t bar_free0 = tmem_slot + 8;            // 2 barriers: accumulator buffer taken out of TMEM (128 arrivals)
     const uint32_t bar_b = bar_free0 + 16;               // B rebuilt for the next head (128 arrivals)
     if (tid == 0) {
@@ -175,7 +178,7 @@ __global__ void __launch_bounds__(NT + 64) scores_tc_kernel(const __grid_constan
             int fb = f_begin / n_all, ft = f_begin - fb * n_all;      // (head, row tile) of the next tile to load
             for (int i = 0; i < n_tiles; ++i) {
                 // the stage is free once the MMAs of the tile that used it have completed
-                if (i >= NSTAGE) mbar_wait_s(bar_mma0 + 8 * ((i - NSTAGE) & 1), ((i - NSTAGE) >> 1) & 1, 3, status);
+                if (i >= NSTAGE) mbar_wait_s(bar_mma0 + 8 * ((i - NSTAGE) & 1), ((i - NSTAGE) >> 1) & 1, 3, &g_scores_status);
                 const uint32_t dst = tile0 + (i % NSTAGE) * C::STAGE, bar = bar_ld0 + 8 * (i % NSTAGE);
                 const int y = ft * TJ - HALF;
                 mbar_expect_tx(bar, C::STAGE);
@@ -197,9 +200,9 @@ __global__ void __launch_bounds__(NT + 64) scores_tc_kernel(const __grid_constan
             int ft = f_begin % n_all, n_heads = 0;
             bool new_head = true;
             for (int i = 0; i < n_tiles; ++i) {
-                if (new_head) { mbar_wait_s(bar_b, n_heads & 1, 5, status); ++n_heads; }   // B of this head is ready
-                mbar_wait_s(bar_ld0 + 8 * (i % NSTAGE), (i / NSTAGE) & 1, 7, status);
-                if (i >= 2) mbar_wait_s(bar_free0 + 8 * (i & 1), ((i - 2) >> 1) & 1, 4, status);   // its accumulator buffer is free
+                if (new_head) { mbar_wait_s(bar_b, n_heads & 1, 5, &g_scores_status); ++n_heads; }   // B of this head is ready
+                mbar_wait_s(bar_ld0 + 8 * (i % NSTAGE), (i / NSTAGE) & 1, 7, &g_scores_status);
+                if (i >= 2) mbar_wait_s(bar_free0 + 8 * (i & 1), ((i - 2) >> 1) & 1, 4, &g_scores_status);   // its accumulator buffer is free
                 tc_fence_after();
                 const uint32_t a_lo = a_lo0 + (uint32_t)(i % NSTAGE) * (C::STAGE >> 4);
                 const uint32_t dcol = tmem + (i & 1) * C::ACC_COLS;
@@ -274,7 +277,7 @@ __global__ void __launch_bounds__(NT + 64) scores_tc_kernel(const __grid_constan
                 mbar_arrive(bar_b);
             }
             SPROF(4 * i);
-            mbar_wait_s(bar_mma0 + 8 * (i & 1), (i >> 1) & 1, 6, status);
+            mbar_wait_s(bar_mma0 + 8 * (i & 1), (i >> 1) & 1, 6, &g_scores_status);
             tc_fence_after();
             SPROF(4 * i + 1);
             {
@@ -329,8 +332,6 @@ __global__ void __launch_bounds__(NT + 64) scores_tc_kernel(const __grid_constan
     if (warp == 4) tmem_dealloc(tmem, TMEM_COLS);
 }
 
-__device__ int g_scores_status = 0;
-
 template <int D, int K>
 int run_tma(const Params& p, const void* k, const void* v, float* z, float* r, cudaStream_t st)
 {
@@ -338,17 +339,10 @@ int run_tma(const Params& p, const void* k, const void* v, float* z, float* r, c
     constexpr int TJ = NT - (K - 1);
     CUtensorMap tk, tv;
     if (!make_map(&tk, k, p.B * p.H, p.T, D, NT) || !make_map(&tv, v, p.B * p.H, p.T, D, NT)) return LTE_ERR_CUDA;
-    static bool attr_done = false;
-    static int* status_ptr = nullptr;
-    static int n_sm = 0;
-    if (!attr_done) {
-        int dev = 0;
-        if (cudaFuncSetAttribute(scores_tc_kernel<D, K>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::BYTES) != cudaSuccess ||
-            cudaGetSymbolAddress((void**)&status_ptr, g_scores_status) != cudaSuccess || cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-            return LTE_ERR_CUDA;
-        attr_done = true;
-    }
+    static PerDeviceOnce attr;
+    if (int e = attr.run([] { return cudaFuncSetAttribute(scores_tc_kernel<D, K>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::BYTES); })) return e;
+    int n_sm = 0;
+    if (int e = device_sm_count(&n_sm)) return e;
     // one wave of CTAs (two per SM at d = 64, one at d = 128) shares the flat list of (head, row tile) pairs evenly
     const int n_all = (p.T + TJ - 1) / TJ, BH = p.B * p.H;
     const long long n_flat = (long long)n_all * BH;
@@ -356,7 +350,7 @@ int run_tma(const Params& p, const void* k, const void* v, float* z, float* r, c
     const int slots = n_sm * (D == 64 ? 2 : 1);
     const int n_cta = (int)(n_flat < slots ? n_flat : slots);
     if (launch_pdl(scores_tc_kernel<D, K>, dim3(n_cta), dim3(NT + 64), C::BYTES, st, tk, tv, p.w, p.bias, z, r, p.H, p.T,
-                   (int)n_flat, status_ptr) != cudaSuccess)
+                   (int)n_flat) != cudaSuccess)
         return LTE_ERR_CUDA;
     return cuda_status(cudaGetLastError());
 }
@@ -405,13 +399,7 @@ int by_d(const Params& p, const void* k, const void* v, float* z, float* r, cuda
 
 }  // namespace
 
-int scores_status_fetch_and_clear()
-{
-    int h = 0, zero = 0;
-    if (cudaMemcpyFromSymbol(&h, g_scores_status, sizeof(int)) != cudaSuccess) return -1;
-    if (h != 0) cudaMemcpyToSymbol(g_scores_status, &zero, sizeof(int));
-    return h;
-}
+int scores_status_fetch_and_clear() { return status_fetch_and_clear(g_scores_status); }
 
 int launch_scores(const Params& p, const void* k, const void* v, float* z, float* r, cudaStream_t st)
 {

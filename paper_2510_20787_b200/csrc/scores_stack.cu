@@ -177,14 +177,11 @@ template <typename T, int D>
 int run_stack(const Params& p, const void* k, const void* v, float* z, float* r, cudaStream_t st)
 {
     using P = StackPlan<D>;
-    static bool attr_done = false;
-    if (!attr_done) {
-        if (cudaFuncSetAttribute(scores_stack_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P::BYTES) != cudaSuccess)
-            return LTE_ERR_CUDA;
-        attr_done = true;
-    }
-    int dev = 0, sms = 148;
-    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    static PerDeviceOnce attr;
+    if (int e = attr.run([] { return cudaFuncSetAttribute(scores_stack_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P::BYTES); }))
+        return e;
+    int sms = 148;
+    device_sm_count(&sms);
     const int BH = p.B * p.H, n_tiles = (p.T + SK_TR - 1) / SK_TR;
     // a CTA keeps one head's parameters in shared memory (one CTA per SM): split every (b,h) into about SMs / (B H) chunks
     int chunks = sms / BH;

@@ -393,21 +393,15 @@ int launch_stack_bwd(const Params& p, const void* k, const void* v, const float*
     dim3 grid(chunks, p.B * p.H);
     cudaError_t e;
     if (p.dtype == LTE_BF16) {
-        static bool done = false;
-        if (!done) {
-            if (cudaFuncSetAttribute(stack_bwd_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SB_BYTES) != cudaSuccess)
-                return LTE_ERR_CUDA;
-            done = true;
-        }
+        static PerDeviceOnce attr;
+        if (int e2 = attr.run([] { return cudaFuncSetAttribute(stack_bwd_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SB_BYTES); }))
+            return e2;
         e = launch_pdl(stack_bwd_kernel<__nv_bfloat16>, grid, dim3(SB_NT), SB_BYTES, st, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v,
                        p.w, p.bias, dz, (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, (float*)part, p.H, p.T, per, input_grad ? 1 : 0);
     } else {
-        static bool done = false;
-        if (!done) {
-            if (cudaFuncSetAttribute(stack_bwd_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SB_BYTES) != cudaSuccess)
-                return LTE_ERR_CUDA;
-            done = true;
-        }
+        static PerDeviceOnce attr;
+        if (int e2 = attr.run([] { return cudaFuncSetAttribute(stack_bwd_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SB_BYTES); }))
+            return e2;
         e = launch_pdl(stack_bwd_kernel<float>, grid, dim3(SB_NT), SB_BYTES, st, (const float*)k, (const float*)v, p.w, p.bias, dz,
                        (float*)dk, (float*)dv, (float*)part, p.H, p.T, per, input_grad ? 1 : 0);
     }

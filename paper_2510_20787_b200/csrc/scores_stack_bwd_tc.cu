@@ -18,7 +18,7 @@
 
 namespace lte {
 
-__device__ int g_stack_bwd_status = 0;
+__device__ StatusWord g_stack_bwd_status = LTE_STATUS_INIT;
 
 namespace {
 
@@ -62,9 +62,9 @@ __device__ __forceinline__ void bwait(uint32_t bar, uint32_t parity, int code) {
         asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
                      : "=r"(ok) : "r"(bar), "r"(parity), "r"(20000u) : "memory");
         if (ok) return;
-        if ((i & 255u) == 255u && *reinterpret_cast<volatile int*>(&g_stack_bwd_status) != 0) return;
+        if ((i & 255u) == 255u && launch_aborted(&g_stack_bwd_status)) return;   // another wait of this launch has given up
     }
-    atomicExch(&g_stack_bwd_status, code);
+    wait_gave_up(&g_stack_bwd_status, code);
 }
 __device__ __forceinline__ void tmem_ld16b(uint32_t taddr, uint32_t (&r)[16]) {
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 "
@@ -128,7 +128,7 @@ stack_bwd_tc_kernel(const __nv_bfloat16* __restrict__ kg, const __nv_bfloat16* _
     pdl_wait();
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     const uint32_t base = smem_u32(smem_raw);
-    if ((base & 127u) != 0) { if (threadIdx.x == 0) atomicExch(&g_stack_bwd_status, 9); return; }
+    if ((base & 127u) != 0) { if (threadIdx.x == 0) atomicExch(&g_stack_bwd_status.code, 9); return; }
     const uint32_t sW = base + BO_W, sX = base + BO_X, sH0 = base + BO_H0, sH1 = base + BO_H1;
     const uint32_t sD0 = base + BO_D0, sD1 = base + BO_D1, sD2 = base + BO_D2;
     const uint32_t sF0 = sW, sF1 = sF0 + BI_F0, sF2 = sF1 + BI_F1, sT0 = sF2 + BI_F2, sT1 = sT0 + BI_T0, sT2 = sT1 + BI_T1;
@@ -588,13 +588,7 @@ int bt_chunks(const Params& p)
 
 }  // namespace
 
-int stack_bwd_tc_status_fetch_and_clear()
-{
-    int h = 0, zero = 0;
-    if (cudaMemcpyFromSymbol(&h, g_stack_bwd_status, sizeof(int)) != cudaSuccess) return -1;
-    if (h != 0) cudaMemcpyToSymbol(g_stack_bwd_status, &zero, sizeof(int));
-    return h;
-}
+int stack_bwd_tc_status_fetch_and_clear() { return status_fetch_and_clear(g_stack_bwd_status); }
 
 // scratch: the weight image, then one packed partial gradient per CTA; 0 where the tensor-core path does not apply
 size_t stack_bwd_tc_workspace(const Params& p)
@@ -607,11 +601,8 @@ int launch_stack_bwd_tc(const Params& p, const void* k, const void* v, const flo
                         float* dbias, bool input_grad, void* ws, cudaStream_t st)
 {
     if (p.dtype != LTE_BF16 || p.d != 64) return LTE_ERR_UNSUPPORTED;
-    static bool done = false;
-    if (!done) {
-        if (cudaFuncSetAttribute(stack_bwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, BT_SMEM) != cudaSuccess) return LTE_ERR_CUDA;
-        done = true;
-    }
+    static PerDeviceOnce attr;
+    if (int e = attr.run([] { return cudaFuncSetAttribute(stack_bwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, BT_SMEM); })) return e;
     uint8_t* img = (uint8_t*)ws;
     float* part = (float*)((char*)ws + ((size_t)p.H * BI_HEAD + 255) / 256 * 256);
     if (launch_pdl(stack_bwd_image_kernel, dim3(p.H, 32), dim3(256), 0, st, p.w, p.bias, img, p.H) != cudaSuccess) return LTE_ERR_CUDA;

@@ -24,7 +24,7 @@
 
 namespace lte {
 
-__device__ int g_stack_tc_status = 0;
+__device__ StatusWord g_stack_tc_status = LTE_STATUS_INIT;
 #ifdef LTE_PROFILE
 __device__ long long g_stprof[64];
 #define STP(i) do { if (blockIdx.x == 3 && it == 5 && lane == 0) g_stprof[i] = clock64(); } while (0)
@@ -78,9 +78,9 @@ __device__ __forceinline__ void swait(uint32_t bar, uint32_t parity, int code) {
         asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
                      : "=r"(ok) : "r"(bar), "r"(parity), "r"(20000u) : "memory");
         if (ok) return;
-        if ((i & 255u) == 255u && *reinterpret_cast<volatile int*>(&g_stack_tc_status) != 0) return;
+        if ((i & 255u) == 255u && launch_aborted(&g_stack_tc_status)) return;   // another wait of this launch has given up
     }
-    atomicExch(&g_stack_tc_status, code);
+    wait_gave_up(&g_stack_tc_status, code);
 }
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
@@ -167,7 +167,7 @@ scores_stack_tc_kernel(const __nv_bfloat16* __restrict__ kg, const __nv_bfloat16
     pdl_wait();                                                // the weight image is written by the preceding kernel
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     const uint32_t base = smem_u32(smem_raw);
-    if ((base & 127u) != 0) { if (threadIdx.x == 0) atomicExch(&g_stack_tc_status, 9); return; }
+    if ((base & 127u) != 0) { if (threadIdx.x == 0) atomicExch(&g_stack_tc_status.code, 9); return; }
     const uint32_t sRing = base + OFF_RING, sX = base + OFF_X, sH0 = base + OFF_HID, sH1 = base + OFF_HID, sW1 = base + OFF_W1, sW2 = base + OFF_W2;
     const float* par = reinterpret_cast<const float*>(smem_raw + OFF_PAR);
     const uint32_t bar0 = base + OFF_BAR;
@@ -511,13 +511,7 @@ scores_stack_tc_kernel(const __nv_bfloat16* __restrict__ kg, const __nv_bfloat16
 
 }  // namespace
 
-int stack_tc_status_fetch_and_clear()
-{
-    int h = 0, zero = 0;
-    if (cudaMemcpyFromSymbol(&h, g_stack_tc_status, sizeof(int)) != cudaSuccess) return -1;
-    if (h != 0) cudaMemcpyToSymbol(g_stack_tc_status, &zero, sizeof(int));
-    return h;
-}
+int stack_tc_status_fetch_and_clear() { return status_fetch_and_clear(g_stack_tc_status); }
 
 // Workspace of the tensor-core stack scorer (the split weight image), 0 where that path does not apply.
 size_t scores_stack_tc_workspace(const Params& p)
@@ -532,15 +526,10 @@ int launch_scores_stack_tc(const Params& p, const void* k, const void* v, float*
 {
     const size_t need = scores_stack_tc_workspace(p);
     if (need == 0 || !ws || ws_bytes < need || ((uintptr_t)ws & 127u) != 0) return LTE_ERR_UNSUPPORTED;
-    static bool attr_done = false;
-    static int n_sm = 0;
-    if (!attr_done) {
-        int dev = 0;
-        if (cudaFuncSetAttribute(scores_stack_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ST_SMEM) != cudaSuccess ||
-            cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-            return LTE_ERR_CUDA;
-        attr_done = true;
-    }
+    static PerDeviceOnce attr;
+    if (int e = attr.run([] { return cudaFuncSetAttribute(scores_stack_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ST_SMEM); })) return e;
+    int n_sm = 0;
+    if (int e = device_sm_count(&n_sm)) return e;
     const int BH = p.B * p.H;
     if (launch_pdl(stack_image_kernel, dim3(p.H, 32), dim3(256), 0, st, p.w, p.bias, (uint8_t*)ws, p.H) != cudaSuccess) return LTE_ERR_CUDA;
     const int n_t = (p.T - ST_HALF + ST_VALID - 1) / ST_VALID;

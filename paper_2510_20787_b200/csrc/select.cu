@@ -186,12 +186,9 @@ int launch_select(const Params& p, const float* z, int32_t* idx, int32_t* cnt, i
     const size_t key_bytes = (size_t)N * 4;
     constexpr size_t kCacheMax = 200 * 1024;              // keys of up to 51200 positions stay on chip
     if (key_bytes <= kCacheMax) {
-        static bool attr_done = false;
-        if (!attr_done) {
-            if (cudaFuncSetAttribute(select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCacheMax) != cudaSuccess)
-                return LTE_ERR_CUDA;
-            attr_done = true;
-        }
+        static PerDeviceOnce attr;
+        if (int e = attr.run([] { return cudaFuncSetAttribute(select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCacheMax); }))
+            return e;
         select_kernel<true><<<p.B * p.H, threads, key_bytes, st>>>(z, idx, cnt, ncand, p.T, p.W, p.R, p.sink, p.zthr);
     } else {
         select_kernel<false><<<p.B * p.H, threads, 0, st>>>(z, idx, cnt, ncand, p.T, p.W, p.R, p.sink, p.zthr);

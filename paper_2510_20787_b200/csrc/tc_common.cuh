@@ -30,14 +30,29 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
                  : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait: gives up after kSpinLimit polls, records `code`, and lets the kernel run on to its end.
-__device__ __forceinline__ void mbar_wait_s(uint32_t bar, uint32_t parity, int code, int* status) {
-    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+// Bounded wait: gives up after kSpinLimit polls, records `code` in the family's status word, and lets the kernel run on
+// to its end.  Once a wait of a launch has given up, that launch is lost, and its other waits stop early so that it ends
+// quickly; they recognise their own launch by its grid id, so a later launch waits normally even while the report
+// is still unread (see StatusWord in common.cuh).
+__device__ __forceinline__ unsigned long long grid_id() {
+    unsigned long long g;
+    asm volatile("mov.u64 %0, %%gridid;" : "=l"(g));
+    return g;
+}
+__device__ __forceinline__ bool launch_aborted(const StatusWord* st) {
+    return *reinterpret_cast<const volatile unsigned long long*>(&st->abort_grid) == grid_id();
+}
+__device__ __forceinline__ void wait_gave_up(StatusWord* st, int code) {
+    atomicExch(&st->code, code);
+    atomicExch(&st->abort_grid, grid_id());
+}
+template <uint32_t LIMIT = kSpinLimit>
+__device__ __forceinline__ void mbar_wait_s(uint32_t bar, uint32_t parity, int code, StatusWord* st) {
+    for (uint32_t i = 0; i < LIMIT; ++i) {
         if (mbar_try_wait(bar, parity)) return;
-        // once any wait has given up, the launch is lost: stop waiting everywhere so it ends quickly
-        if ((i & 1023u) == 1023u && *reinterpret_cast<volatile int*>(status) != 0) return;
+        if ((i & 1023u) == 1023u && launch_aborted(st)) return;
     }
-    atomicExch(status, code);
+    wait_gave_up(st, code);
 }
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, int x, int y, int z, uint32_t bar) {
     asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"

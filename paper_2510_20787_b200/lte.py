@@ -20,7 +20,7 @@ BWD_CNN_INPUT_GRAD = 1
 
 EXPORTS = ["lte_device_status", "lte_workspace_bytes", "lte_strerror", "lte_scores", "lte_select", "lte_cache_score", "lte_attn_prefill",
            "lte_cache_bytes", "lte_cache_init", "lte_attn_decode", "lte_attn_prefill_chunk", "lte_attn_bwd", "lte_attn_bwd_static",
-           "lte_sparsity_stats", "lte_lambda_update", "lte_cache_score_unrope"]
+           "lte_sparsity_stats", "lte_lambda_update", "lte_cache_score_unrope", "lte_selftest_per_device"]
 STATIC_SCRATCH_BYTES = 8 << 20
 
 
@@ -70,6 +70,7 @@ def lib():
         L.lte_attn_prefill_chunk.argtypes = [vp] * 3 + [ctypes.c_int32] + [vp] * 6 + [ctypes.c_size_t, vp]
         L.lte_attn_bwd.argtypes = [vp] * 17 + [ctypes.c_uint32, vp, ctypes.c_size_t, vp]
         L.lte_attn_bwd_static.argtypes = [vp] * 17 + [ctypes.c_uint32, vp]
+        L.lte_selftest_per_device.argtypes = [ctypes.c_int]
         for name in EXPORTS:
             if name not in ("lte_strerror", "lte_workspace_bytes", "lte_cache_bytes", "lte_device_status"):
                 getattr(L, name).restype = ctypes.c_int

@@ -166,3 +166,26 @@ def test_unrope_scoring_host_side():
     assert L.lte_cache_score_unrope(a(s), a(stack), fake, fake, fake, 0, fake, 1 << 30, None) == -1
     assert L.lte_cache_score_unrope(a(s), a(stack), fake, fake, fake, 100, fake, 16, None) == -3
     assert L.lte_cache_score_unrope(a(s), a(lte.LteConv(1, 7, 1, 256, 0)), fake, fake, fake, 100, fake, 1 << 30, None) == -2
+
+
+def test_per_device_table_initialises_once_per_device_under_threads():
+    """The launchers keep their once-per-device facts (SM count, raised shared-memory limits, symbol addresses) in a
+    table indexed by device ordinal and guarded by a mutex.  Two threads that ask for the same ordinals at the same time
+    (ctypes releases the interpreter lock around the calls) must see exactly one initialisation per ordinal."""
+    import threading
+    L = lte.lib()
+    errs = []
+
+    def worker():
+        for n in range(3000):
+            for dev in (0, 1, 5, 63):
+                if L.lte_selftest_per_device(dev) != 1:
+                    errs.append(dev)
+
+    ts = [threading.Thread(target=worker) for _ in range(2)]
+    for t in ts:
+        t.start()
+    for t in ts:
+        t.join()
+    assert not errs
+    assert L.lte_selftest_per_device(64) == -1 and L.lte_selftest_per_device(-1) == -1

@@ -151,3 +151,28 @@ def test_wrong_token_count_is_reported_and_leaves_the_cache_alone():
     assert lte.lib().lte_device_status() != 0
     assert torch.equal(before, cache)
     assert lte.lib().lte_device_status() == 0               # the status is cleared by reading it
+
+
+def test_a_reported_mismatch_does_not_stop_the_next_call_from_committing():
+    """A call that named the wrong token count is reported and leaves the cache alone; a correct call made after it,
+    with the report still unread, must advance the cache as if nothing had happened (the report word is not a gate)."""
+    cfg = _cfg(B=1, H=2)
+    x = synth.make(cfg, 0, T=120)
+    c = lte.conv(torch.from_numpy(x["w"]).cuda())
+    q, k, v = (dev(x[t], cfg.dtype) for t in "qkv")
+    s = shape_of(cfg, T=80)
+    z = lte.lte_scores(s, c, k[:, :, :80].contiguous(), v[:, :, :80].contiguous())
+    idx, cnt = lte.lte_select(s, z)
+    cache = lte.lte_cache_init(s, c, k[:, :, :80].contiguous(), v[:, :, :80].contiguous(), z, idx, cnt)
+    good = cache.clone()
+    s2 = shape_of(cfg, T=40)
+    qc, kc, vc = (t[:, :, 80:].contiguous() for t in (q, k, v))
+    lte.lte_attn_prefill_chunk(s2, c, cache, 79, qc, kc, vc)                  # wrong count: reported, cache untouched
+    o1, l1 = lte.lte_attn_prefill_chunk(s2, c, cache, 80, qc, kc, vc)         # right count, report still unread
+    o2, l2 = lte.lte_attn_prefill_chunk(s2, c, good, 80, qc, kc, vc)          # the same call on an untouched copy
+    torch.cuda.synchronize()
+    assert torch.equal(cache, good) and torch.equal(o1, o2) and torch.equal(l1, l2)
+    _, ns = _read_pool(cache, cfg, cfg.B)
+    assert all(n == 120 for n in ns)
+    assert lte.lib().lte_device_status() != 0                                 # the first call's report is still there
+    assert lte.lib().lte_device_status() == 0

@@ -173,3 +173,15 @@ def test_compacted_and_gathered_retained_rows_agree(d, T, W, R):
     torch.cuda.synchronize()
     assert lte.lib().lte_device_status() == 0
     assert torch.equal(o1, o2) and torch.equal(l1, l2) and torch.equal(o1, o3)
+
+
+def test_second_device_after_the_first():
+    """A process that drives two GPUs: the tiny fp32 configuration and a tensor-core shape on device 0, then on device 1
+    (raised shared-memory limits, SM count and status words are per device).  Skipped unless two devices are visible."""
+    if torch.cuda.device_count() < 2:
+        pytest.skip("needs two visible devices")
+    for dev_id in (0, 1):
+        with torch.cuda.device(dev_id):
+            for cfg in (synth.CONFIGS["C1"], synth.Config("dev", "bf16", 1, 2, 64, 700, 64, 48, 7, 0.1)):
+                _assert_close(cfg, _pipeline(cfg, seed=0))
+            assert lte.lte_device_status() == 0
