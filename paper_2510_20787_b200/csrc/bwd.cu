@@ -19,7 +19,8 @@ int launch_bwd_dq_tc(const Params& p, const void* q, const void* k, const void* 
 size_t bwd_tc_ret_bytes(const Params& p);
 int launch_bwd_dkv_tc(const Params& p, const void* q, const void* k, const void* v, const float* lse, const void* dO,
                       const float* delta, const float* z, const int32_t* idx, const int32_t* cnt, const float* lambda,
-                      void* dk, void* dv, float* dk32, float* dv32, float* dz, void* ret_ws, bool f32out, cudaStream_t st);
+                      void* dk, void* dv, float* dk32, float* dv32, float* dz, void* ret_ws, bool f32out, bool merge_here,
+                      cudaStream_t st);
 
 namespace {
 
@@ -308,18 +309,26 @@ __global__ void __launch_bounds__(256) bwd_finish_inplace_kernel(const float* __
     }
 }
 
-// Tensor-core path, K = 5 or 7: one pass over the rows of k, v, dk, dv does both scorer jobs.  A block takes `rows`
+// Tensor-core path, K = 5 or 7: one pass over the rows of k, v, dk, dv finishes the backward.  It first turns Eq. 6's inner
+// products into logit gradients for the block's positions (and the taps around them): dr = the window share the dk/dv kernel
+// wrote + the far-query share of a retained key (+ lambda where the token passes the threshold, Eq. 7), dz = dr r (1 - r);
+// the retained keys' far-query shares of dk, dv (fp32, one row per list entry) are added onto their rows in the same
+// pass, so that a retained row is rounded once.  Then both scorer jobs:  A block takes `rows`
 // consecutive positions of one (b,h); a thread owns 4 channels of x = [k ; v] for every row it visits, so its
 // K x 4 scorer weights stay in registers, and walks the block's rows: dw partials acc[t][c] += dz[p - t + half] x[p][c],
 // and (FINISH) the scorer's input gradient sum_t dz[p - t + half] w[h,t,c] added onto the bf16 dk, dv rows in place.
 // The partials of the threads that own the same channels are added in a fixed order (a tree over the row slots
 // through shared memory).
+__device__ __forceinline__ bool isv_of(int cg, int D) { return cg >= D / 4; }
 constexpr int TAIL_MIN_ROWS = 256, TAIL_MAX_ROWS = 1024;   // rows per block are chosen per launch to fill whole waves
 template <int D, int K, bool FINISH>
 __global__ void __launch_bounds__(256, 2)
-bwd_tail_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v, const float* __restrict__ dz,
-                const float* __restrict__ w, __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv,
-                float* __restrict__ part_w, float* __restrict__ part_b, int B, int H, int Tlen, int nchunk, int rows)
+bwd_tail_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v, const float* __restrict__ dr_win,
+                const float* __restrict__ z, const float* __restrict__ lambda, const int32_t* __restrict__ idx,
+                const int32_t* __restrict__ cnt, const float* __restrict__ dk_ret, const float* __restrict__ dv_ret,
+                const float* __restrict__ dr_ret, const float* __restrict__ w, __nv_bfloat16* __restrict__ dk,
+                __nv_bfloat16* __restrict__ dv, float* __restrict__ part_w, float* __restrict__ part_b, int B, int H, int Tlen,
+                int R, float zthr, int nchunk, int rows)
 {
     pdl_launch_dependents();
     pdl_wait();                                                // see launch_pdl: earlier kernels of the stream have completed
@@ -329,17 +338,39 @@ bwd_tail_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __rest
     const int NDZ = (rows + K - 1 + 3) & ~3;
     extern __shared__ float sm[];
     float* dzs = sm;                                // dz[p0-half .. p0+rows-1+half]
-    float* red = dzs + NDZ;                         // [RPP/2][K][2D]
+    int* ent = reinterpret_cast<int*>(dzs + NDZ);   // list entry of the same positions, or -1
+    float* red = dzs + 2 * NDZ;                     // [RPP/2][K][2D]
     const int h = blockIdx.y;
     const int b = blockIdx.x / nchunk, ch = blockIdx.x % nchunk;
     const int bh = b * H + h;
     const int p0 = ch * rows;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    for (int a = tid; a < rows + K - 1; a += 256) ent[a] = -1;
+    __syncthreads();
+    {
+        const int n_ret = cnt[bh];
+        const int32_t* id = idx + (size_t)bh * R;
+        for (int e = tid; e < n_ret; e += 256) {
+            const int a = id[e] - (p0 - half);
+            if (a >= 0 && a < rows + K - 1) ent[a] = e;
+        }
+    }
+    __syncthreads();
     for (int a = tid; a < rows + K - 1; a += 256) {
         const int j = p0 - half + a;
-        dzs[a] = (j >= 0 && j + half <= Tlen - 1) ? dz[(size_t)bh * Tlen + j] : 0.f;
+        float g = 0.f;
+        if (j >= 0 && j + half <= Tlen - 1) {       // scored tokens only
+            float dr = dr_win[(size_t)bh * Tlen + j];
+            if (ent[a] >= 0) dr += dr_ret[(size_t)bh * R + ent[a]];
+            const float zz = z[(size_t)bh * Tlen + j];
+            const float r = 1.f / (1.f + expf(-zz));
+            if (lambda && zz > zthr) dr += lambda[h];
+            g = dr * r * (1.f - r);
+        }
+        dzs[a] = g;
     }
     const int cg = tid % TPR, r0 = tid / TPR;       // channel group: x channels [4 cg, 4 cg + 4); row slot
+    const float* gret = isv_of(cg, D) ? dv_ret : dk_ret;
     const bool isv = cg >= D / 4;
     const int cc = (cg % (D / 4)) * 4;              // first of this thread's 4 channels within k or v
     const __nv_bfloat16* src = isv ? v : k;
@@ -368,7 +399,8 @@ bwd_tail_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __rest
             const int p = min(p0 + rb + u * RPP, Tlen - 1);
             const size_t a0 = ((size_t)bh * Tlen + p) * D + cc;
             ux[u] = *reinterpret_cast<const uint2*>(src + a0);
-            if (FINISH) ug[u] = *reinterpret_cast<const uint2*>(gdst + a0);
+            ug[u] = make_uint2(0u, 0u);
+            if (FINISH || ent[min(rb + u * RPP, rows - 1) + half] >= 0) ug[u] = *reinterpret_cast<const uint2*>(gdst + a0);
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) {
@@ -383,12 +415,19 @@ bwd_tail_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __rest
             for (int t = 0; t < K; ++t)
 #pragma unroll
                 for (int e = 0; e < 4; ++e) acc[t][e] = fmaf(g[t], x[e], acc[t][e]);
-            if (FINISH) {
+            const int er = ent[rl + half];                   // retained: its far-query share is added here
+            if (FINISH || er >= 0) {
                 float gi[4] = {0.f, 0.f, 0.f, 0.f};
+                if (FINISH) {
 #pragma unroll
-                for (int t = 0; t < K; ++t)
+                    for (int t = 0; t < K; ++t)
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) gi[e] = fmaf(g[t], wr[t][e], gi[e]);
+                        for (int e = 0; e < 4; ++e) gi[e] = fmaf(g[t], wr[t][e], gi[e]);
+                }
+                if (er >= 0) {
+                    const float4 f4 = *reinterpret_cast<const float4*>(gret + ((size_t)bh * R + er) * D + cc);
+                    gi[0] += f4.x; gi[1] += f4.y; gi[2] += f4.z; gi[3] += f4.w;
+                }
                 __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(ug[u].x << 16) + gi[0], __uint_as_float(ug[u].x & 0xffff0000u) + gi[1]);
                 __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(ug[u].y << 16) + gi[2], __uint_as_float(ug[u].y & 0xffff0000u) + gi[3]);
                 *reinterpret_cast<uint2*>(gdst + ((size_t)bh * Tlen + p) * D + cc) =
@@ -453,17 +492,23 @@ inline int tail_chunks(const Params& p, int* rows_out)
 }
 
 template <int D, int K>
-int run_tail(const Params& p, const void* k, const void* v, const float* dz, void* dk, void* dv, float* part_w,
-             float* part_b, bool finish, int nchunk, int rows, cudaStream_t st)
+int run_tail(const Params& p, const void* k, const void* v, const float* dr_win, const float* z, const float* lambda,
+             const int32_t* idx, const int32_t* cnt, const float* ret_ws, void* dk, void* dv, float* part_w, float* part_b,
+             bool finish, int nchunk, int rows, cudaStream_t st)
 {
-    const size_t sm = (size_t)(((rows + K - 1 + 3) & ~3) + (256 / (2 * D / 4) / 2) * K * 2 * D) * sizeof(float);
+    const size_t sm = (size_t)(2 * ((rows + K - 1 + 3) & ~3) + (256 / (2 * D / 4) / 2) * K * 2 * D) * sizeof(float);
     dim3 grid(p.B * nchunk, p.H);
+    // the retained tiles' scratch: dk_ret, dv_ret [B,H,R,d], dr_ret [B,H,R] (layout of launch_bwd_dkv_tc)
+    const size_t n = (size_t)p.B * p.H * (p.R > 0 ? p.R : 1);
+    const float* dk_ret = ret_ws; const float* dv_ret = dk_ret + n * D; const float* dr_ret = dv_ret + n * D;
     if (finish)
-        launch_pdl(bwd_tail_kernel<D, K, true>, grid, dim3(256), sm, st, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, dz, p.w,
-                                                          (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, part_w, part_b, p.B, p.H, p.T, nchunk, rows);
+        launch_pdl(bwd_tail_kernel<D, K, true>, grid, dim3(256), sm, st, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, dr_win, z,
+                   lambda, idx, cnt, dk_ret, dv_ret, dr_ret, p.w, (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, part_w, part_b, p.B, p.H,
+                   p.T, p.R, p.zthr, nchunk, rows);
     else
-        launch_pdl(bwd_tail_kernel<D, K, false>, grid, dim3(256), sm, st, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, dz, p.w,
-                                                           (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, part_w, part_b, p.B, p.H, p.T, nchunk, rows);
+        launch_pdl(bwd_tail_kernel<D, K, false>, grid, dim3(256), sm, st, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, dr_win, z,
+                   lambda, idx, cnt, dk_ret, dv_ret, dr_ret, p.w, (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, part_w, part_b, p.B, p.H,
+                   p.T, p.R, p.zthr, nchunk, rows);
     return cuda_status(cudaGetLastError());
 }
 
@@ -521,8 +566,10 @@ int run(const Params& p, const void* q, const void* k, const void* v, const void
                                                    idx, cnt, (T*)dq, delta, p.T, p.W, p.R, p.scale, p.G);
     }
     if constexpr (sizeof(T) == 2 && (D == 64 || D == 128)) {
+        // K = 5 or 7 with the single layer: the last pass (bwd_tail_kernel) also merges the retained shares and forms dz
+        const bool tail_merges = !p.stack && (p.K == 5 || p.K == 7);
         const int e = launch_bwd_dkv_tc(p, q, k, v, lse, dO, delta, z, idx, cnt, lambda, dk, dv, dk32, dv32, dz, base + w.ret,
-                                        false, st);
+                                        false, !tail_merges, st);
         if (e != LTE_OK) return e;
     } else if (f32) {
         bwd_dkv_kernel<T, D, true><<<grid, 128, 0, st>>>((const T*)q, (const T*)k, (const T*)v, (const T*)dO, lse, delta,
@@ -543,8 +590,9 @@ int run(const Params& p, const void* q, const void* k, const void* v, const void
         if (p.K == 5 || p.K == 7) {                   // fused pass: dw partials and the scorer's input gradient
             int rows = 0;
             const int nch = tail_chunks(p, &rows);
-            const int e = p.K == 7 ? run_tail<D, 7>(p, k, v, dz, dk, dv, part_w, part_b, f32, nch, rows, st)
-                                   : run_tail<D, 5>(p, k, v, dz, dk, dv, part_w, part_b, f32, nch, rows, st);
+            const float* rw = (const float*)(base + w.ret);
+            const int e = p.K == 7 ? run_tail<D, 7>(p, k, v, dz, z, lambda, idx, cnt, rw, dk, dv, part_w, part_b, f32, nch, rows, st)
+                                   : run_tail<D, 5>(p, k, v, dz, z, lambda, idx, cnt, rw, dk, dv, part_w, part_b, f32, nch, rows, st);
             if (e != LTE_OK) return e;
             launch_pdl(bwd_conv_reduce_kernel, gr, dim3(256), 0, st, part_w, part_b, dw, dbias, p.B * nch, per_head);
             return cuda_status(cudaGetLastError());

@@ -881,7 +881,8 @@ size_t bwd_tc_ret_bytes(const Params& p)
 
 int launch_bwd_dkv_tc(const Params& p, const void* q, const void* k, const void* v, const float* lse, const void* dO,
                       const float* delta, const float* z, const int32_t* idx, const int32_t* cnt, const float* lambda,
-                      void* dk, void* dv, float* dk32, float* dv32, float* dz, void* ret_ws, bool f32out, cudaStream_t st)
+                      void* dk, void* dv, float* dk32, float* dv32, float* dz, void* ret_ws, bool f32out, bool merge_here,
+                      cudaStream_t st)
 {
     const int BH = p.B * p.H;
     CUtensorMap tk, tv, tq, tdo, tdk, tdv;
@@ -909,6 +910,8 @@ int launch_bwd_dkv_tc(const Params& p, const void* q, const void* k, const void*
     else if (p.d == 128) { if (f32out) LTE_GO(128, true); else LTE_GO(128, false); }
     else return LTE_ERR_UNSUPPORTED;
 #undef LTE_GO
+    // merge_here = false: the caller's last pass adds the retained shares and turns dr into dz itself
+    if (!merge_here) return cuda_status(cudaGetLastError());
     if (p.R > 0) {
         dim3 gm(p.R, BH);
         if (f32out)

@@ -43,7 +43,7 @@ __device__ __forceinline__ bool launch_aborted(const StatusWord* st) {
     return *reinterpret_cast<const volatile unsigned long long*>(&st->abort_grid) == grid_id();
 }
 __device__ __forceinline__ void wait_gave_up(StatusWord* st, int code) {
-    atomicExch(&st->code, code);
+    atomicCAS(&st->code, 0, code);                              // the first anomaly since the host last read the word stays
     atomicExch(&st->abort_grid, grid_id());
 }
 template <uint32_t LIMIT = kSpinLimit>

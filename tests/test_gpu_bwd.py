@@ -88,3 +88,20 @@ def test_long_prefill_shape_four_retained_tiles():
     res = _bwd(cfg, seed=4)
     assert np.all(res["_list"][1] == 512)
     _assert(cfg, res)
+
+
+@pytest.mark.parametrize("B,H,T,W,R,sink", [
+    (1, 1, 100, 64, 20, 0),         # a single ragged tile
+    (2, 3, 129, 64, 200, 0),        # second tile of one row; list longer than the sequence allows
+    (3, 5, 1000, 33, 300, 2),       # several list chunks per tile, sink tokens, a window that is no multiple of anything
+    (7, 23, 640, 64, 64, 0),        # more (head, tile) pairs than SMs: a thread block's run crosses heads and starts inside one
+    (2, 2, 520, 7, 40, 0),          # the narrowest window the scorer allows
+    (2, 2, 700, 9, 0, 0),           # no list at all
+    (1, 2, 4100, 64, 700, 0),       # eleven list chunks: the chunk ring wraps inside an item
+])
+def test_short_window_shapes(B, H, T, W, R, sink):
+    """bf16, d = 64, windows of at most one key tile (the training shape's regime): ragged tiles, lists longer than a tile,
+    more (head, tile) pairs than SMs, sink tokens, no list at all."""
+    cfg = synth.Config("fused", "bf16", B, H, 64, T, W, R, 7, 0.1, sink=sink)
+    _assert(cfg, _bwd(cfg, seed=9, lam=np.linspace(0.0, 0.5, H), scale=0.0))
+    assert lte.lte_device_status() == 0
