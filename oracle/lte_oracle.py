@@ -272,3 +272,61 @@ def attn_bwd(q, k, v, dO, z, idx, cnt, w, W, scale=None, tau=0.5, lam=None,
                             _p(q), _p(k), _p(v), _p(dO), _p(z), _p(idx), _p(cnt), _p(w), _p(lam),
                             _p(dq), _p(dk), _p(dv), _p(dw), _p(db), _p(dz))
     return dict(dq=dq, dk=dk, dv=dv, dw=dw, dbias=db, dz=dz)
+
+
+# ---- training-free selection rules of the ablation (Section 4, last paragraph) ---------------------------------
+RULE_LEARNED, RULE_UNIFORM, RULE_ACCUM_ATTN = 0, 1, 2
+
+
+def select_uniform(B, H, T, W, R, sink=0):
+    """"Unif.+SWA": out-of-window tokens retained at a uniform stride.  Eligible positions are 0 .. E-1 with
+    E = max(T - W, 0).  Sink positions j < sink come first and count against R; the n = R - #sink remaining slots
+    go to the positions sink, sink + stride, sink + 2 stride, ... < E with the smallest stride that fits:
+    stride = max(1, ceil((E - sink) / n)).  The same list for every head.  -> idx [B,H,R] ascending (-1 unused), cnt."""
+    E = max(T - W, 0)
+    keep = list(range(min(sink, E, max(R, 0))))
+    n = max(R, 0) - len(keep)
+    rest = E - min(sink, E)
+    if n > 0 and rest > 0:
+        stride = max(1, -(-rest // n))
+        keep += list(range(sink, E, stride))
+    idx = np.full((B, H, max(R, 0)), -1, np.int32)
+    cnt = np.full((B, H), len(keep), np.int32)
+    idx[:, :, :len(keep)] = np.asarray(keep, np.int32)
+    return idx, cnt
+
+
+def attn_colsum(q, k, idx, cnt, W, scale=None):
+    """Accumulated attention of every key: a[b,h,j] = sum over the queries i that attend j (window i-W < j <= i, or j in
+    the list and j <= i-W) of P_ij, P = the softmax weights of lte_attn_prefill over those sets.  The ranking quantity of
+    the accumulated-attention eviction heuristics the ablation compares with.  -> a [B,H,T]."""
+    q, k = _f64(q), _f64(k)
+    B, H, T, d = q.shape
+    scale = 1.0 / np.sqrt(d) if scale is None else float(scale)
+    a = np.zeros((B, H, T), np.float64)
+    for b in range(B):
+        for h in range(H):
+            kept = [int(j) for j in idx[b, h, :cnt[b, h]]]
+            for i in range(T):
+                js = [j for j in kept if j <= i - W] + list(range(max(i - W + 1, 0), i + 1))
+                s = np.array([scale * float(q[b, h, i] @ k[b, h, j]) for j in js])
+                p = np.exp(s - s.max())
+                p /= p.sum()
+                for j, pj in zip(js, p):
+                    a[b, h, j] += pj
+    return a
+
+
+def select_rule(rule, score, T, W, R, sink=0, tau=0.5, B=None, H=None):
+    """lte_select with a rule: RULE_LEARNED = select(score = z, threshold tau); RULE_UNIFORM = select_uniform (score
+    unused); RULE_ACCUM_ATTN: every out-of-window token is a candidate, the R with the largest accumulated attention
+    stay (sink first, ties to the older token): select() without a threshold."""
+    if rule == RULE_UNIFORM:
+        if score is not None:
+            B, H = np.asarray(score).shape[:2]
+        return select_uniform(B, H, T, W, R, sink)
+    if rule == RULE_ACCUM_ATTN:
+        idx, cnt, _ = select(score, W, R, sink, tau=0.0)
+        return idx, cnt
+    idx, cnt, _ = select(score, W, R, sink, tau)
+    return idx, cnt
