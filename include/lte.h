@@ -138,6 +138,33 @@ int lte_select(const lte_shape* s, const float* z, int32_t* idx, int32_t* cnt,
                int32_t* ncand_or_null, void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * The same list interface for the training-free rules the paper's ablation compares with (Section 4, last paragraph:
+ * "Unif.+SWA retains out-of-window tokens at a uniform stride"; an eviction heuristic based on accumulated attention):
+ *   LTE_RULE_LEARNED     lte_select (score = z).
+ *   LTE_RULE_UNIFORM     score is ignored (may be NULL).  Eligible positions are 0 .. E-1, E = max(T - W, 0).  The sink
+ *                        positions j < sink come first and count against R; the n = R - #sink remaining slots go to
+ *                        sink, sink + stride, sink + 2 stride, ... < E with stride = max(1, ceil((E - sink) / n)), the
+ *                        smallest stride that fits.  Every head gets the same list; ncand = E.
+ *   LTE_RULE_ACCUM_ATTN  score = a [B,H,T] fp32, the accumulated attention of lte_attn_colsum (or any non-negative
+ *                        importance): every position j <= T-1-W is a candidate (no threshold; s->tau is ignored), the R
+ *                        largest stay, sink first, ties to the older token.
+ * idx, cnt, ncand_or_null as for lte_select.  Errors: INVALID_ARG (unknown rule, NULL score where one is read).
+ */
+enum { LTE_RULE_LEARNED = 0, LTE_RULE_UNIFORM = 1, LTE_RULE_ACCUM_ATTN = 2 };
+int lte_select_rule(const lte_shape* s, int rule, const float* score, int32_t* idx, int32_t* cnt, int32_t* ncand_or_null,
+                    void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Accumulated attention of every key under the attention lte_attn_prefill computed (Section 2.2 / Section 4: the quantity
+ * eviction heuristics rank by): a[b,h,j] = sum over the queries i with j in A_i, and over the query heads of the group,
+ * of exp(scale q_i.k_j - lse_i).  lse is lte_attn_prefill's output for the same q, k, idx, cnt.  The sum of a over j is
+ * T * group per head.  A plain fp32 kernel (one warp per key), deterministic; not part of the learned rule's hot path.
+ *   q in [B,H*group,T,d], k in [B,H,T,d] of s->dtype;  lse in [B,H*group,T];  a out [B,H,T] fp32
+ */
+int lte_attn_colsum(const lte_shape* s, const void* q, const void* k, const float* lse, const int32_t* idx, const int32_t* cnt,
+                    float* a, void* stream);
+
+/*
  * Prefill attention (Section 3.1.3, "Cached prefilling and decoding"): query i attends over
  * A_i = {max(0,i-W+1) .. i}  U  {j in idx[b,h,:cnt] : j <= i-W}:
  *   o_i = softmax_{j in A_i}(scale * q_i.k_j) v_j,   lse_i = log sum_{j in A_i} exp(scale * q_i.k_j).

@@ -97,6 +97,9 @@ int launch_stack_bwd(const Params& p, const void* k, const void* v, const float*
 int launch_scores_stack_tc(const Params& p, const void* k, const void* v, float* z, float* r, void* ws, size_t ws_bytes,
                            cudaStream_t st);
 int launch_select(const Params& p, const float* z, int32_t* idx, int32_t* cnt, int32_t* ncand, cudaStream_t st);
+int launch_select_uniform(const Params& p, int32_t* idx, int32_t* cnt, int32_t* ncand, cudaStream_t st);
+int launch_colsum(const Params& p, const void* q, const void* k, const float* lse, const int32_t* idx, const int32_t* cnt,
+                  float* a, cudaStream_t st);
 int launch_prefill_simt(const Params& p, const void* q, const void* k, const void* v, const int32_t* idx,
                         const int32_t* cnt, void* o, float* lse, cudaStream_t st);
 int launch_prefill_tc_long(const Params& p, const void* q, const void* k, const void* v, const int32_t* idx,

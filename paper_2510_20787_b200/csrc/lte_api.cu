@@ -239,6 +239,36 @@ int lte_select(const lte_shape* s, const float* z, int32_t* idx, int32_t* cnt, i
     return launch_select(make_params(s, nullptr), z, idx, cnt, ncand_or_null, (cudaStream_t)stream);
 }
 
+int lte_select_rule(const lte_shape* s, int rule, const float* score, int32_t* idx, int32_t* cnt, int32_t* ncand_or_null,
+                    void* ws, size_t ws_bytes, void* stream)
+{
+    if (rule == LTE_RULE_LEARNED) return lte_select(s, score, idx, cnt, ncand_or_null, ws, ws_bytes, stream);
+    int e = check_shape(s, true); if (e) return e;
+    if (!cnt || (s->R > 0 && !idx)) return LTE_ERR_INVALID_ARG;
+    if (s->T - s->W > (1 << 24)) return LTE_ERR_UNSUPPORTED;
+    if (rule == LTE_RULE_UNIFORM) {
+        e = check_arch(); if (e) return e;
+        return launch_select_uniform(make_params(s, nullptr), idx, cnt, ncand_or_null, (cudaStream_t)stream);
+    }
+    if (rule == LTE_RULE_ACCUM_ATTN) {                       // the learned rule's ranking without its threshold
+        if (!score) return LTE_ERR_INVALID_ARG;
+        e = check_arch(); if (e) return e;
+        Params p = make_params(s, nullptr);
+        p.zthr = -INFINITY;
+        return launch_select(p, score, idx, cnt, ncand_or_null, (cudaStream_t)stream);
+    }
+    return LTE_ERR_INVALID_ARG;
+}
+
+int lte_attn_colsum(const lte_shape* s, const void* q, const void* k, const float* lse, const int32_t* idx, const int32_t* cnt,
+                    float* a, void* stream)
+{
+    int e = check_shape(s, true); if (e) return e;
+    if (!q || !k || !lse || !cnt || (s->R > 0 && !idx) || !a) return LTE_ERR_INVALID_ARG;
+    e = check_arch(); if (e) return e;
+    return launch_colsum(make_params(s, nullptr), q, k, lse, idx, cnt, a, (cudaStream_t)stream);
+}
+
 int lte_attn_prefill(const lte_shape* s, const void* q, const void* k, const void* v, const int32_t* idx,
                      const int32_t* cnt, void* o, float* lse, void* ws, size_t ws_bytes, void* stream)
 {

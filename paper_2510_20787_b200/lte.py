@@ -20,7 +20,7 @@ BWD_CNN_INPUT_GRAD = 1
 
 EXPORTS = ["lte_device_status", "lte_workspace_bytes", "lte_strerror", "lte_scores", "lte_select", "lte_cache_score", "lte_attn_prefill",
            "lte_cache_bytes", "lte_cache_init", "lte_attn_decode", "lte_attn_prefill_chunk", "lte_attn_bwd", "lte_attn_bwd_static",
-           "lte_sparsity_stats", "lte_lambda_update", "lte_cache_score_unrope", "lte_selftest_per_device"]
+           "lte_sparsity_stats", "lte_lambda_update", "lte_cache_score_unrope", "lte_selftest_per_device", "lte_select_rule", "lte_attn_colsum"]
 STATIC_SCRATCH_BYTES = 8 << 20
 
 
@@ -71,6 +71,8 @@ def lib():
         L.lte_attn_bwd.argtypes = [vp] * 17 + [ctypes.c_uint32, vp, ctypes.c_size_t, vp]
         L.lte_attn_bwd_static.argtypes = [vp] * 17 + [ctypes.c_uint32, vp]
         L.lte_selftest_per_device.argtypes = [ctypes.c_int]
+        L.lte_select_rule.argtypes = [vp, ctypes.c_int] + [vp] * 5 + [ctypes.c_size_t, vp]
+        L.lte_attn_colsum.argtypes = [vp] * 8
         for name in EXPORTS:
             if name not in ("lte_strerror", "lte_workspace_bytes", "lte_cache_bytes", "lte_device_status"):
                 getattr(L, name).restype = ctypes.c_int
@@ -169,6 +171,31 @@ def lte_select(s, z, idx=None, cnt=None, ncand=None):
     _check("lte_select", lib().lte_select(ctypes.addressof(s), _ptr(z, torch.float32), _ptr(idx, torch.int32),
                                           _ptr(cnt, torch.int32), _ptr(ncand, torch.int32), None, 0, _stream()))
     return idx, cnt
+
+
+RULE_LEARNED, RULE_UNIFORM, RULE_ACCUM_ATTN = 0, 1, 2
+
+
+def lte_select_rule(s, rule, score=None, idx=None, cnt=None, ncand=None, device=None):
+    """lte_select under one of the rules: RULE_LEARNED (score = z), RULE_UNIFORM (no score), RULE_ACCUM_ATTN (score = the
+    accumulated attention of lte_attn_colsum)."""
+    dev = score.device if score is not None else (device or torch.device("cuda"))
+    if idx is None:
+        idx = torch.empty((s.B, s.H, s.R), dtype=torch.int32, device=dev)
+    if cnt is None:
+        cnt = torch.empty((s.B, s.H), dtype=torch.int32, device=dev)
+    _check("lte_select_rule", lib().lte_select_rule(ctypes.addressof(s), int(rule), _ptr(score, torch.float32), _ptr(idx, torch.int32),
+                                                    _ptr(cnt, torch.int32), _ptr(ncand, torch.int32), None, 0, _stream()))
+    return idx, cnt
+
+
+def lte_attn_colsum(s, q, k, lse, idx, cnt, a=None):
+    """Accumulated attention a [B,H,T] fp32 of every key under the attention lte_attn_prefill ran with this list."""
+    if a is None:
+        a = torch.empty((s.B, s.H, s.T), dtype=torch.float32, device=q.device)
+    _check("lte_attn_colsum", lib().lte_attn_colsum(ctypes.addressof(s), _ptr(q), _ptr(k), _ptr(lse, torch.float32),
+                                                    _ptr(idx, torch.int32), _ptr(cnt, torch.int32), _ptr(a, torch.float32), _stream()))
+    return a
 
 
 def lte_attn_prefill(s, q, k, v, idx, cnt, o=None, lse=None, ws=None):

@@ -189,3 +189,14 @@ def test_per_device_table_initialises_once_per_device_under_threads():
         t.join()
     assert not errs
     assert L.lte_selftest_per_device(64) == -1 and L.lte_selftest_per_device(-1) == -1
+
+
+def test_selection_rules_host_side():
+    L = lte.lib()
+    s = lte.shape(1, 1, 64, 64, 8, 4, lte.BF16)
+    p = ctypes.addressof(s)
+    assert L.lte_select_rule(p, 7, 256, 256, 256, None, None, 0, None) == -1            # unknown rule
+    assert L.lte_select_rule(p, lte.RULE_ACCUM_ATTN, None, 256, 256, None, None, 0, None) == -1   # this rule reads a score
+    assert L.lte_select_rule(p, lte.RULE_UNIFORM, None, 256, None, None, None, 0, None) == -1     # cnt is required
+    assert L.lte_select_rule(p, lte.RULE_LEARNED, None, 256, 256, None, None, 0, None) == -1      # lte_select's own check
+    assert L.lte_attn_colsum(p, None, 256, 256, 256, 256, 256, None) == -1
