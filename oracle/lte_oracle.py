@@ -330,3 +330,36 @@ def select_rule(rule, score, T, W, R, sink=0, tau=0.5, B=None, H=None):
         return idx, cnt
     idx, cnt, _ = select(score, W, R, sink, tau)
     return idx, cnt
+
+
+def stream_intervals(z, n0, n1, W, R, pool_idx, pool_cnt, sink=0, tau=0.5):
+    """The streaming rule of Section 3.1.3 (decoding paragraph: a token leaving the window is appended while the pool has
+    room, else it replaces the lowest-scoring entry iff it scores strictly higher) applied token by token while a chunk
+    [n0, n1) arrives on top of a pool, written as visibility intervals: entry j is in the pool for the queries
+    enter <= i < leave.  One (b,h): z [>= n1 - W] logits of the whole sequence, pool_idx[:pool_cnt] the pool before the
+    chunk (entries of the pool before the chunk get enter = n0).  Sink tokens are never evicted; among equal lowest
+    scores the youngest goes.  -> list of (position, enter, leave) in order of entering; leave = n1 for the survivors."""
+    thr = logit(tau)
+    pool = [int(j) for j in pool_idx[:pool_cnt]]
+    rec = {j: [j, n0, n1] for j in pool}
+    order = list(pool)
+    for n in range(n0, n1):
+        p = n - W
+        if p < 0 or R <= 0 or p in rec or not (p < sink or z[p] > thr):
+            continue
+        if len(pool) < R:
+            pool.append(p)
+        elif p >= sink:
+            cand = [j for j in pool if j >= sink]
+            if not cand:
+                continue
+            worst = min(cand, key=lambda j: (z[j], -j))
+            if not z[p] > z[worst]:
+                continue
+            rec[worst][2] = n
+            pool[pool.index(worst)] = p
+        else:
+            continue
+        rec[p] = [p, n, n1]
+        order.append(p)
+    return [tuple(rec[j]) for j in order]

@@ -100,3 +100,25 @@ def test_arbitrary_pool_against_dense_masked_attention():
         oref, lref, _ = dense_attention(q[0, h], k[0, h], v[0, h], M, 0.3)
         np.testing.assert_allclose(o[0, h], oref[n0:], atol=1e-12)
         np.testing.assert_allclose(lse[0, h], lref[n0:], atol=1e-12)
+
+
+def test_streaming_intervals_reproduce_the_token_by_token_pool_with_a_binding_cap():
+    """The streaming reading of a chunk, written as visibility intervals [enter, leave) per entry (the form the GPU path
+    consumes), against the token-by-token simulation: at every query of the chunk the entries whose interval contains
+    it are exactly the simulation's pool at that step (read off as the final pool of the simulation stopped there).
+    The cap binds (R far below the number of candidates), so entries do leave inside the chunk."""
+    rng = np.random.default_rng(5)
+    T, d, W, R, sink, n0 = 90, 4, 6, 5, 1, 40
+    q, k, v = (rng.standard_normal((1, 1, T, d)) for _ in range(3))
+    z = rng.standard_normal((1, 1, T)); z[0, 0, 50] = z[0, 0, 44]                    # an exact tie among candidates
+    p_idx, p_cnt, _ = orc.select(z[:, :, :n0], W, R, sink)
+    iv = orc.stream_intervals(z[0, 0], n0, T, W, R, p_idx[0, 0], int(p_cnt[0, 0]), sink)
+    left_inside = [e for e in iv if e[2] < T]
+    assert len(left_inside) >= 3                                                     # the cap does bind inside the chunk
+    for i in range(n0, T):
+        _, _, pool_i, cnt_i = orc.stream(q[:, :, :i + 1], k[:, :, :i + 1], v[:, :, :i + 1], z[:, :, :i + 1], W, R, sink)
+        want = set(int(j) for j in pool_i[0, 0, :cnt_i[0, 0]])
+        got = set(j for j, a, b in iv if a <= i < b)
+        assert got == want, (i, sorted(got), sorted(want))
+    # an entry is seen from the query that pushes it out of the window (position + W), or from the chunk's start
+    assert all(a == max(j + W, n0) for j, a, b in iv)
