@@ -83,7 +83,7 @@ typedef struct lte_conv {
  */
 
 typedef enum lte_op {
-    LTE_OP_SCORES = 0, LTE_OP_SELECT = 1, LTE_OP_PREFILL = 2, LTE_OP_DECODE = 3, LTE_OP_BWD = 4, LTE_OP_CHUNK = 5, LTE_OP_STATS = 6
+    LTE_OP_SCORES = 0, LTE_OP_SELECT = 1, LTE_OP_PREFILL = 2, LTE_OP_DECODE = 3, LTE_OP_BWD = 4, LTE_OP_CHUNK = 5, LTE_OP_STATS = 6, LTE_OP_CHUNK_STREAM = 7
 } lte_op;
 
 /* Bytes of caller-supplied scratch the given entry point needs for this shape (0 if none). */
@@ -283,6 +283,23 @@ int lte_cache_score_unrope(const lte_shape* s, const lte_conv* c, void* cache, c
 int lte_attn_prefill_chunk(const lte_shape* s, const lte_conv* c, void* cache, int32_t n_past,
                            const void* q, const void* k, const void* v, void* o, float* lse,
                            void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * The same with a choice of reading (flags = 0: lte_attn_prefill_chunk).  LTE_CHUNK_STREAMING: the streaming reading
+ * (Section 3.1.3, decoding paragraph, applied token by token inside the chunk): query i of the chunk sees its window and
+ * the pool as the replace-the-lowest rule has left it after the token i - W was offered, i.e. exactly what T calls of
+ * lte_attn_decode compute, also where the cap R binds: an entry that a later token of the same chunk pushes out is still
+ * seen by the queries before that token's.  The cache afterwards is the same under both readings.
+ * The pool is walked token by token (one warp per head) and the attention runs row by row on the fp32 ALUs for every
+ * dtype (the tiled tensor-core kernels take a list prefix per query, not an interval per entry): exact, and several
+ * times slower than the chunk-end reading.
+ *   ws   device scratch of lte_workspace_bytes(LTE_OP_CHUNK_STREAM, s, c) bytes, 256-byte aligned
+ * Errors: as lte_attn_prefill_chunk; INVALID_ARG for unknown flags; UNSUPPORTED for R > 4096 with the flag.
+ */
+#define LTE_CHUNK_STREAMING 1u
+int lte_attn_prefill_chunk_ex(const lte_shape* s, const lte_conv* c, void* cache, int32_t n_past,
+                              const void* q, const void* k, const void* v, void* o, float* lse, uint32_t flags,
+                              void* ws, size_t ws_bytes, void* stream);
 
 /*
  * Training-side statistics of the scorer (Section 3.1.2, Eq. 7, and the retention count that Algorithm 1 steers):

@@ -165,7 +165,92 @@ __global__ void chunk_commit_kernel(unsigned char* __restrict__ cache, CacheLayo
     if (threadIdx.x == 0) { meta[0] = n1; meta[1] = cnt; }
 }
 
+// The streaming reading (Section 3.1.3, decoding paragraph, applied inside a chunk): one warp per (b,h) walks the chunk's
+// queries in order and applies the replace-the-lowest rule to the token each query pushes out of its window (local row
+// rq - W).  Out: the list of every entry that is in the pool at some query of the chunk (local rows, in order of
+// entering = ascending; the pool the cache held comes first), for each the query row from which it is gone (`leave`,
+// INT_MAX for the survivors), and the survivors as the new pool (idx, cnt; ascending local rows).  zrank holds the logits
+// of the local sequence with sink tokens at +inf; keep iff zrank > zthr.
+__global__ void __launch_bounds__(32) chunk_stream_kernel(const float* __restrict__ zrank, const int32_t* __restrict__ oldpos,
+                                                          int32_t* __restrict__ ulist, int32_t* __restrict__ leave,
+                                                          int32_t* __restrict__ ucnt, int32_t* __restrict__ idx,
+                                                          int32_t* __restrict__ cnt, int R, int W, int Tloc, int ucap, int n0,
+                                                          int R0, int Wn, float zthr)
+{
+    extern __shared__ int sm_i[];
+    float* pz = reinterpret_cast<float*>(sm_i);                // [R] logit of pool entry
+    int* ppos = sm_i + R;                                       // [R] position (for the tie rule: the youngest of equals goes)
+    int* pu = sm_i + 2 * R;                                     // [R] its index in the entry list
+    const int bh = blockIdx.x, lane = threadIdx.x;
+    const float* zr = zrank + (size_t)bh * Tloc;
+    const int32_t* op = oldpos + (size_t)bh * R;
+    int32_t* ul = ulist + (size_t)bh * ucap;
+    int32_t* lv = leave + (size_t)bh * ucap;
+    int n_pool = 0;
+    if (R0 > 0) {                                              // the pool the cache holds: local rows [0, its count)
+        for (int e = lane; e < R; e += 32) {
+            const bool ok = op[e] >= 0;
+            if (ok) { pz[e] = zr[e]; ppos[e] = op[e]; pu[e] = e; ul[e] = e; lv[e] = 0x7fffffff; }
+            n_pool += ok ? 1 : 0;                              // valid slots are the first ones
+        }
+        n_pool = __reduce_add_sync(0xffffffffu, n_pool);
+    }
+    int n_u = n_pool;
+    __syncwarp();
+    const int Tc = Tloc - R0 - Wn;
+    for (int t = 0; t < Tc; ++t) {
+        const int rq = R0 + Wn + t, r = rq - W;                // the query's row; the row it pushes out of its window
+        if (r < R0 || R <= 0) continue;
+        const float zc = zr[r];
+        if (!(zc > zthr)) continue;
+        const int pos = n0 - Wn + (r - R0);
+        if (n_pool < R) {
+            if (lane == 0) { pz[n_pool] = zc; ppos[n_pool] = pos; pu[n_pool] = n_u; ul[n_u] = r; lv[n_u] = 0x7fffffff; }
+            ++n_pool; ++n_u;
+        } else {
+            // the lowest logit; among equals the youngest
+            float wz = INFINITY; int wp = -1, wi = -1;
+            for (int e = lane; e < R; e += 32) {
+                const float ze = pz[e]; const int pe = ppos[e];
+                if (ze < wz || (ze == wz && pe > wp)) { wz = ze; wp = pe; wi = e; }
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const float oz = __shfl_xor_sync(0xffffffffu, wz, o);
+                const int opp = __shfl_xor_sync(0xffffffffu, wp, o), oi = __shfl_xor_sync(0xffffffffu, wi, o);
+                if (oz < wz || (oz == wz && opp > wp)) { wz = oz; wp = opp; wi = oi; }
+            }
+            if (wi >= 0 && zc > wz) {                            // strictly better: the entry is gone from this query on
+                if (lane == 0) { lv[pu[wi]] = rq; pz[wi] = zc; ppos[wi] = pos; pu[wi] = n_u; ul[n_u] = r; lv[n_u] = 0x7fffffff; }
+                ++n_u;
+            }
+        }
+        __syncwarp();
+    }
+    __syncwarp();
+    // the survivors, in list order (ascending local rows), are the new pool
+    int n_out = 0;
+    for (int e0 = 0; e0 < n_u; e0 += 32) {
+        const int e = e0 + lane;
+        const bool keep = e < n_u && lv[e] == 0x7fffffff;
+        const unsigned bal = __ballot_sync(0xffffffffu, keep);
+        if (keep) idx[(size_t)bh * R + n_out + __popc(bal & ((1u << lane) - 1u))] = ul[e];
+        n_out += __popc(bal);
+    }
+    for (int e = n_out + lane; e < R; e += 32) idx[(size_t)bh * R + e] = -1;
+    if (lane == 0) { cnt[bh] = n_out; ucnt[bh] = n_u; }
+}
+
 }  // namespace
+
+int launch_chunk_stream(const Params& p, const float* zrank, const int32_t* oldpos, int32_t* ulist, int32_t* leave, int32_t* ucnt,
+                        int32_t* idx, int32_t* cnt, int ucap, int n0, int R0, int Wn, cudaStream_t st)
+{
+    const size_t smem = (size_t)(p.R > 0 ? p.R : 1) * 12;
+    if (smem > 48 * 1024) return LTE_ERR_UNSUPPORTED;           // pools of up to 4096 entries
+    chunk_stream_kernel<<<p.B * p.H, 32, smem, st>>>(zrank, oldpos, ulist, leave, ucnt, idx, cnt, p.R, p.W, p.T, ucap, n0, R0, Wn, p.zthr);
+    return cuda_status(cudaGetLastError());
+}
 
 int chunk_status_fetch_and_clear() { return status_fetch_and_clear(g_chunk_status); }
 

@@ -110,8 +110,8 @@ CacheScorePlan cache_score_plan(const lte_shape* s, const lte_conv* c)
 }
 
 // scratch of lte_attn_prefill_chunk, sized for the longest local sequence (pool rows + full ring + chunk)
-struct ChunkPlan { size_t klin, vlin, z, zrank, zsrc, oldpos, idx, cnt, gate, sub, att, total; };
-ChunkPlan chunk_plan(const lte_shape* s, const lte_conv* c)
+struct ChunkPlan { size_t klin, vlin, z, zrank, zsrc, oldpos, idx, cnt, gate, ulist, leave, ucnt, sub, att, total; int ucap; };
+ChunkPlan chunk_plan(const lte_shape* s, const lte_conv* c, bool streaming = false)
 {
     auto up = [](size_t x) { return (x + 255) / 256 * 256; };
     ChunkPlan w;
@@ -127,6 +127,15 @@ ChunkPlan chunk_plan(const lte_shape* s, const lte_conv* c)
     w.idx = off; off += up(bhk * (size_t)(s->R > 0 ? s->R : 1) * 4);
     w.cnt = off; off += up(bhk * 4);
     w.gate = off; off += up(bhk * 4);                        // per head: the cache held n_past tokens (written by every call's gather)
+    // streaming reading: every entry that is in the pool at some query of the chunk (at most the old pool plus one per
+    // token that leaves the window), and the query from which each is gone
+    w.ucap = s->R + s->T;
+    w.ulist = w.leave = w.ucnt = off;
+    if (streaming) {
+        w.ulist = off; off += up(bhk * (size_t)w.ucap * 4);
+        w.leave = off; off += up(bhk * (size_t)w.ucap * 4);
+        w.ucnt = off; off += up(bhk * 4);
+    }
     w.sub = off;
     if (c && c->n_layers == 3) {
         lte_shape s2 = *s; s2.T = (int32_t)Tm;
@@ -193,10 +202,10 @@ size_t lte_workspace_bytes(int op, const lte_shape* s, const lte_conv* c)
         if (check_shape(s, true) != LTE_OK) return 0;
         return ((size_t)s->B * s->H * 2 * sizeof(float) + 255) / 256 * 256;
     }
-    if (op == LTE_OP_CHUNK) {
+    if (op == LTE_OP_CHUNK || op == LTE_OP_CHUNK_STREAM) {
         if (check_shape(s, true) != LTE_OK || !c) return 0;
         if ((double)s->B * s->H * (s->group > 1 ? s->group : 1) * ((double)s->R + s->W + s->T) * s->d > 2.0e10) return 0;
-        return chunk_plan(s, c).total;
+        return chunk_plan(s, c, op == LTE_OP_CHUNK_STREAM).total;
     }
     if (op == LTE_OP_SCORES && c && c->n_layers == 3) {
         if (check_shape(s, true) != LTE_OK) return 0;
@@ -330,13 +339,22 @@ int lte_cache_score_unrope(const lte_shape* s, const lte_conv* c, void* cache, c
 int lte_attn_prefill_chunk(const lte_shape* s, const lte_conv* c, void* cache, int32_t n_past, const void* q, const void* k,
                            const void* v, void* o, float* lse, void* ws, size_t ws_bytes, void* stream)
 {
+    return lte_attn_prefill_chunk_ex(s, c, cache, n_past, q, k, v, o, lse, 0u, ws, ws_bytes, stream);
+}
+
+int lte_attn_prefill_chunk_ex(const lte_shape* s, const lte_conv* c, void* cache, int32_t n_past, const void* q, const void* k,
+                              const void* v, void* o, float* lse, uint32_t flags, void* ws, size_t ws_bytes, void* stream)
+{
     int e = check_shape(s, true); if (e) return e;
+    if (flags & ~LTE_CHUNK_STREAMING) return LTE_ERR_INVALID_ARG;
+    const bool streaming = (flags & LTE_CHUNK_STREAMING) != 0;
+    if (streaming && s->R > 4096) return LTE_ERR_UNSUPPORTED;
     e = check_conv_or_stack(s, c); if (e) return e;
     if (!cache || !q || !k || !v || !o || !lse || n_past < 0) return LTE_ERR_INVALID_ARG;
     if (!aligned16(cache) || !aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return LTE_ERR_INVALID_ARG;
     const size_t G = s->group > 1 ? s->group : 1, bhq = (size_t)s->B * s->H * G;
     if ((double)bhq * ((double)s->R + s->W + s->T) * s->d > 2.0e10 || (double)n_past + s->T > 2.0e9) return LTE_ERR_UNSUPPORTED;
-    const ChunkPlan w = chunk_plan(s, c);
+    const ChunkPlan w = chunk_plan(s, c, streaming);
     if (!ws || ((uintptr_t)ws & 255u) != 0 || ws_bytes < w.total) return LTE_ERR_WORKSPACE;
     e = check_arch(); if (e) return e;
     cudaStream_t st = (cudaStream_t)stream;
@@ -360,10 +378,20 @@ int lte_attn_prefill_chunk(const lte_shape* s, const lte_conv* c, void* cache, i
     }
     if (e) return e;
     e = launch_chunk_merge_z(p, z, zrank, zsrc, oldpos, n_past, R0, Wn, st); if (e) return e;
-    e = launch_select(psel, zrank, idx, cnt, nullptr, st); if (e) return e;
-    // the attention kernels take the chunk's q, o, lse as they are: query row r stands at position qoff + r
-    if (s->dtype == LTE_BF16) e = launch_prefill_tc(patt, q, base + w.klin, base + w.vlin, idx, cnt, o, lse, base + w.att, w.total - w.att, st);
-    else e = launch_prefill_simt(patt, q, base + w.klin, base + w.vlin, idx, cnt, o, lse, st);
+    if (streaming) {
+        // token by token: the pool every query sees is the streaming rule's at that query.  The entries that are in the
+        // pool at some query, each with the query from which it is gone, feed the row-by-row attention kernel (the tiled
+        // tensor-core kernels know prefixes of a list only); the survivors are the new pool.
+        int32_t* ulist = (int32_t*)(base + w.ulist); int32_t* leave = (int32_t*)(base + w.leave); int32_t* ucnt = (int32_t*)(base + w.ucnt);
+        e = launch_chunk_stream(psel, zrank, oldpos, ulist, leave, ucnt, idx, cnt, w.ucap, n_past, R0, Wn, st); if (e) return e;
+        Params pu = patt; pu.R = w.ucap;                      // the entry list's row length
+        e = launch_prefill_simt(pu, q, base + w.klin, base + w.vlin, ulist, ucnt, o, lse, st, leave);
+    } else {
+        e = launch_select(psel, zrank, idx, cnt, nullptr, st); if (e) return e;
+        // the attention kernels take the chunk's q, o, lse as they are: query row r stands at position qoff + r
+        if (s->dtype == LTE_BF16) e = launch_prefill_tc(patt, q, base + w.klin, base + w.vlin, idx, cnt, o, lse, base + w.att, w.total - w.att, st);
+        else e = launch_prefill_simt(patt, q, base + w.klin, base + w.vlin, idx, cnt, o, lse, st);
+    }
     if (e) return e;
     return launch_chunk_commit(p, cache, base + w.klin, base + w.vlin, z, idx, cnt, oldpos, gate, n_past, n_past + Tc, R0, Wn, st);
 }

@@ -2,6 +2,8 @@
 // One warp per query; the d channels are spread over the lanes, keys are visited one by one
 // (retained entries already out of the query's window first, then the window), online softmax.
 // This is the reference-precision path for fp32 tensors; bf16 tensors use the tensor-core kernel.
+// With `leave` (the streaming reading of a chunked prefill) list entry a is visible to query i only while i < leave[a]:
+// the entry was pushed out of the pool by a better token at that query.
 #include "common.cuh"
 
 namespace lte {
@@ -11,7 +13,8 @@ template <typename T, int D>
 __global__ void __launch_bounds__(128) prefill_simt_kernel(const T* __restrict__ q, const T* __restrict__ k,
                                                            const T* __restrict__ v, const int32_t* __restrict__ idx,
                                                            const int32_t* __restrict__ cnt, T* __restrict__ o,
-                                                           float* __restrict__ lse, int Tlen, int W, int R, float scale, int G, int qoff)
+                                                           float* __restrict__ lse, int Tlen, int W, int R, float scale, int G, int qoff,
+                                                           const int32_t* __restrict__ leave)
 {
     constexpr int C = D / 32;                  // channels per lane
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -24,6 +27,7 @@ __global__ void __launch_bounds__(128) prefill_simt_kernel(const T* __restrict__
     for (int c = 0; c < C; ++c) { qv[c] = to_f(q[base + lane + 32 * c]) * scale; acc[c] = 0.f; }
     float m = -INFINITY, l = 0.f;
     const int32_t* id = idx + (size_t)bhk * R;
+    const int32_t* lv = leave ? leave + (size_t)bhk * R : nullptr;
     const int n_ret = cnt[bhk];
     const int lo = i - W + 1 > 0 ? i - W + 1 : 0;
     // number of retained entries visible to this query: idx ascending => a prefix
@@ -36,6 +40,7 @@ __global__ void __launch_bounds__(128) prefill_simt_kernel(const T* __restrict__
     }
     const int total = nvis + (i - lo + 1);
     for (int a = 0; a < total; ++a) {
+        if (lv && a < nvis && lv[a] <= i) continue;                 // no longer in the pool at this query
         const int j = a < nvis ? id[a] : lo + (a - nvis);
         const T* kr = k + kbase + (size_t)j * D;
         const T* vr = v + kbase + (size_t)j * D;
@@ -58,12 +63,12 @@ __global__ void __launch_bounds__(128) prefill_simt_kernel(const T* __restrict__
 
 template <typename T>
 int run(const Params& p, const void* q, const void* k, const void* v, const int32_t* idx, const int32_t* cnt,
-        void* o, float* lse, cudaStream_t st)
+        void* o, float* lse, const int32_t* leave, cudaStream_t st)
 {
     dim3 grid((p.T - p.qoff + 3) / 4, p.B * p.H * p.G);
 #define LTE_GO(D)                                                                                          \
     prefill_simt_kernel<T, D><<<grid, 128, 0, st>>>((const T*)q, (const T*)k, (const T*)v, idx, cnt, (T*)o, \
-                                                    lse, p.T, p.W, p.R, p.scale, p.G, p.qoff)
+                                                    lse, p.T, p.W, p.R, p.scale, p.G, p.qoff, leave)
     switch (p.d) {
         case 32: LTE_GO(32); break;
         case 64: LTE_GO(64); break;
@@ -77,10 +82,10 @@ int run(const Params& p, const void* q, const void* k, const void* v, const int3
 }  // namespace
 
 int launch_prefill_simt(const Params& p, const void* q, const void* k, const void* v, const int32_t* idx,
-                        const int32_t* cnt, void* o, float* lse, cudaStream_t st)
+                        const int32_t* cnt, void* o, float* lse, cudaStream_t st, const int32_t* leave)
 {
-    return p.dtype == LTE_BF16 ? run<__nv_bfloat16>(p, q, k, v, idx, cnt, o, lse, st)
-                               : run<float>(p, q, k, v, idx, cnt, o, lse, st);
+    return p.dtype == LTE_BF16 ? run<__nv_bfloat16>(p, q, k, v, idx, cnt, o, lse, leave, st)
+                               : run<float>(p, q, k, v, idx, cnt, o, lse, leave, st);
 }
 
 }  // namespace lte

@@ -15,12 +15,13 @@ LIB_PATH = os.path.join(_HERE, "liblte.so")
 _lib = None
 
 F32, BF16 = 0, 1
-OP_SCORES, OP_SELECT, OP_PREFILL, OP_DECODE, OP_BWD, OP_CHUNK, OP_STATS = range(7)
+OP_SCORES, OP_SELECT, OP_PREFILL, OP_DECODE, OP_BWD, OP_CHUNK, OP_STATS, OP_CHUNK_STREAM = range(8)
+CHUNK_STREAMING = 1
 BWD_CNN_INPUT_GRAD = 1
 
 EXPORTS = ["lte_device_status", "lte_workspace_bytes", "lte_strerror", "lte_scores", "lte_select", "lte_cache_score", "lte_attn_prefill",
            "lte_cache_bytes", "lte_cache_init", "lte_attn_decode", "lte_attn_prefill_chunk", "lte_attn_bwd", "lte_attn_bwd_static",
-           "lte_sparsity_stats", "lte_lambda_update", "lte_cache_score_unrope", "lte_selftest_per_device", "lte_select_rule", "lte_attn_colsum"]
+           "lte_sparsity_stats", "lte_lambda_update", "lte_cache_score_unrope", "lte_selftest_per_device", "lte_select_rule", "lte_attn_colsum", "lte_attn_prefill_chunk_ex"]
 STATIC_SCRATCH_BYTES = 8 << 20
 
 
@@ -68,6 +69,7 @@ def lib():
         L.lte_sparsity_stats.argtypes = [vp] * 6 + [ctypes.c_size_t, vp]
         L.lte_lambda_update.argtypes = [ctypes.c_int32, vp, vp, vp, ctypes.c_int64, vp]
         L.lte_attn_prefill_chunk.argtypes = [vp] * 3 + [ctypes.c_int32] + [vp] * 6 + [ctypes.c_size_t, vp]
+        L.lte_attn_prefill_chunk_ex.argtypes = [vp] * 3 + [ctypes.c_int32] + [vp] * 5 + [ctypes.c_uint32, vp, ctypes.c_size_t, vp]
         L.lte_attn_bwd.argtypes = [vp] * 17 + [ctypes.c_uint32, vp, ctypes.c_size_t, vp]
         L.lte_attn_bwd_static.argtypes = [vp] * 17 + [ctypes.c_uint32, vp]
         L.lte_selftest_per_device.argtypes = [ctypes.c_int]
@@ -243,20 +245,21 @@ def lte_attn_decode(s, c, cache, q1, k1, v1, o1=None, lse1=None):
     return o1, lse1
 
 
-def lte_attn_prefill_chunk(s, c, cache, n_past, q, k, v, o=None, lse=None, ws=None):
+def lte_attn_prefill_chunk(s, c, cache, n_past, q, k, v, o=None, lse=None, ws=None, streaming=False):
     """Chunked prefill on top of a cache that holds n_past tokens: q [B,H*group,T,d], k, v [B,H,T,d] (T = s.T new
     tokens) -> o, lse of the chunk's queries; the cache is advanced to n_past + T tokens in place.  ws: uint8 tensor of
-    lte_workspace_bytes(OP_CHUNK, s, c) bytes, allocated here when None."""
+    lte_workspace_bytes(OP_CHUNK or OP_CHUNK_STREAM, s, c) bytes, allocated here when None.  streaming=True: the
+    token-by-token reading (what decode steps compute, also where the cap binds)."""
     if o is None:
         o = torch.empty_like(q)
     if lse is None:
         lse = torch.empty((s.B, s.H * max(s.group, 1), s.T), dtype=torch.float32, device=q.device)
     if ws is None:
-        ws = torch.empty(max(lte_workspace_bytes(OP_CHUNK, s, c), 256), dtype=torch.uint8, device=q.device)
-    _check("lte_attn_prefill_chunk", lib().lte_attn_prefill_chunk(ctypes.addressof(s), ctypes.addressof(c), _ptr(cache),
-                                                                  ctypes.c_int32(int(n_past)), _ptr(q), _ptr(k), _ptr(v),
-                                                                  _ptr(o), _ptr(lse, torch.float32), _ptr(ws), ws.numel(),
-                                                                  _stream()))
+        ws = torch.empty(max(lte_workspace_bytes(OP_CHUNK_STREAM if streaming else OP_CHUNK, s, c), 256), dtype=torch.uint8, device=q.device)
+    _check("lte_attn_prefill_chunk", lib().lte_attn_prefill_chunk_ex(ctypes.addressof(s), ctypes.addressof(c), _ptr(cache),
+                                                                     ctypes.c_int32(int(n_past)), _ptr(q), _ptr(k), _ptr(v),
+                                                                     _ptr(o), _ptr(lse, torch.float32), CHUNK_STREAMING if streaming else 0,
+                                                                     _ptr(ws), ws.numel(), _stream()))
     return o, lse
 
 

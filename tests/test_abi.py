@@ -200,3 +200,18 @@ def test_selection_rules_host_side():
     assert L.lte_select_rule(p, lte.RULE_UNIFORM, None, 256, None, None, None, 0, None) == -1     # cnt is required
     assert L.lte_select_rule(p, lte.RULE_LEARNED, None, 256, 256, None, None, 0, None) == -1      # lte_select's own check
     assert L.lte_attn_colsum(p, None, 256, 256, 256, 256, 256, None) == -1
+
+
+def test_streaming_chunk_host_side():
+    L = lte.lib()
+    s = lte.shape(1, 2, 64, 64, 16, 8, lte.BF16)
+    c = lte.LteConv(1, 7, 1, 256, 0)
+    ps, pc = ctypes.addressof(s), ctypes.addressof(c)
+    need0 = lte.lte_workspace_bytes(lte.OP_CHUNK, s, c)
+    need1 = lte.lte_workspace_bytes(lte.OP_CHUNK_STREAM, s, c)
+    assert need1 > need0 > 0 and need1 % 256 == 0            # the entry list and its leave times come on top
+    args = (ps, pc, 256, 0, 256, 256, 256, 256, 256)
+    assert L.lte_attn_prefill_chunk_ex(*args, 2, 256, need1, None) == -1          # unknown flag
+    assert L.lte_attn_prefill_chunk_ex(*args, lte.CHUNK_STREAMING, 256, need0, None) == -3   # the streaming scratch is larger
+    big = lte.shape(1, 2, 64, 64, 16, 5000, lte.BF16)
+    assert L.lte_attn_prefill_chunk_ex(ctypes.addressof(big), pc, 256, 0, 256, 256, 256, 256, 256, lte.CHUNK_STREAMING, 256, 1 << 40, None) == -2

@@ -18,7 +18,7 @@ def _cfg(dtype="bf16", B=2, H=3, d=64, W=32, R=24, K=7, sink=0):
     return synth.Config("chunk", dtype, B, H, d, 0, W, R, K, 0.05 if dtype == "bf16" else 0.1, sink=sink)
 
 
-def _run(cfg, plan, seed=0, scale=0.0, group=1):
+def _run(cfg, plan, seed=0, scale=0.0, group=1, streaming=False):
     """plan: list of ("prefill", n) (first only), ("decode", n), ("chunk", n).  Returns per-phase GPU outputs and the
     final cache; every phase continues the same sequence."""
     Ttot = sum(n for _, n in plan)
@@ -52,7 +52,7 @@ def _run(cfg, plan, seed=0, scale=0.0, group=1):
             outs.append((np.stack(oo, axis=2), np.stack(ll, axis=2)))
         else:
             o, l = lte.lte_attn_prefill_chunk(s, c, cache, n, q[:, :, n:n + m].contiguous(), k[:, :, n:n + m].contiguous(),
-                                              v[:, :, n:n + m].contiguous())
+                                              v[:, :, n:n + m].contiguous(), streaming=streaming)
             outs.append((o.float().cpu().numpy(), l.cpu().numpy()))
         n += m
     torch.cuda.synchronize()
@@ -60,7 +60,7 @@ def _run(cfg, plan, seed=0, scale=0.0, group=1):
     return x, outs, cache
 
 
-def _oracle(cfg, x, plan, scale=0.0, group=1):
+def _oracle(cfg, x, plan, scale=0.0, group=1, streaming=False):
     """The same plan on the oracle: decode steps by the token-by-token simulation (its pool at any time is the one-shot
     list of the prefix), chunks by prefill_chunk on top of that pool."""
     sc = None if scale == 0.0 else scale
@@ -71,7 +71,7 @@ def _oracle(cfg, x, plan, scale=0.0, group=1):
     for kind, m in plan:
         if kind == "prefill":
             outs.append(None)
-        elif kind == "decode":
+        elif kind == "decode" or streaming:                        # the streaming reading of a chunk IS the token-by-token simulation
             o, l, _, _ = orc.stream(x["q"][:, :, :n + m], kq[:, :, :n + m], vq[:, :, :n + m], zq[:, :, :n + m], cfg.W, cfg.R, cfg.sink, scale=sc, n_from=n)
             outs.append((o, l))
         else:
@@ -87,9 +87,9 @@ def _oracle(cfg, x, plan, scale=0.0, group=1):
     return outs, f_idx, f_cnt, n
 
 
-def _compare(cfg, plan, seed=0, scale=0.0, group=1):
-    x, got, cache = _run(cfg, plan, seed, scale, group)
-    want, f_idx, f_cnt, n = _oracle(cfg, x, plan, scale, group)
+def _compare(cfg, plan, seed=0, scale=0.0, group=1, streaming=False):
+    x, got, cache = _run(cfg, plan, seed, scale, group, streaming)
+    want, f_idx, f_cnt, n = _oracle(cfg, x, plan, scale, group, streaming)
     for (kind, m), g, w in zip(plan, got, want):
         if g is None:
             continue
@@ -176,3 +176,32 @@ def test_a_reported_mismatch_does_not_stop_the_next_call_from_committing():
     assert all(n == 120 for n in ns)
     assert lte.lib().lte_device_status() != 0                                 # the first call's report is still there
     assert lte.lib().lte_device_status() == 0
+
+
+@pytest.mark.parametrize("kw,plan,group", [
+    (dict(), [("prefill", 200), ("chunk", 150), ("decode", 12)], 1),
+    (dict(), [("prefill", 0), ("chunk", 100), ("chunk", 60), ("decode", 5)], 1),
+    (dict(), [("prefill", 33), ("chunk", 5), ("chunk", 1), ("chunk", 300), ("decode", 4)], 1),
+    (dict(sink=3, W=16, R=9), [("prefill", 40), ("decode", 7), ("chunk", 220)], 1),
+    (dict(dtype="f32", d=32, W=16, R=8, K=5, B=1, H=2), [("prefill", 60), ("chunk", 90), ("decode", 6)], 1),
+    (dict(d=128, W=40, R=30, B=1, H=2), [("prefill", 150), ("chunk", 140)], 1),
+    (dict(W=64, R=40, B=1, H=2), [("prefill", 300), ("chunk", 260), ("decode", 3)], 3),
+    (dict(W=32, R=0), [("prefill", 50), ("chunk", 90)], 1),
+])
+def test_streaming_reading_equals_token_by_token_decoding_with_a_binding_cap(kw, plan, group):
+    """LTE_CHUNK_STREAMING: every chunk query sees the pool the replace-the-lowest rule holds at that query, so a chunk
+    equals as many decode steps, also where the cap binds (about half of all tokens pass the threshold here and the
+    budgets are small: entries are pushed out inside the chunk)."""
+    _compare(_cfg(**kw), plan, seed=3, group=group, streaming=True)
+
+
+def test_the_two_readings_differ_where_the_cap_binds_and_leave_the_same_cache():
+    cfg = _cfg(B=1, H=2)
+    plan = [("prefill", 200), ("chunk", 150)]
+    x, a, cache_a = _run(cfg, plan, seed=3)
+    _, b, cache_b = _run(cfg, plan, seed=3, streaming=True)
+    assert np.max(np.abs(a[1][0] - b[1][0])) > 5e-2                  # an early query sees entries that leave later in the chunk
+    pa, na = _read_pool(cache_a, cfg, cfg.B); pb, nb = _read_pool(cache_b, cfg, cfg.B)
+    assert na == nb and all(np.array_equal(u, v) for u, v in zip(pa, pb))
+    # the last query of the chunk sees the final pool under both readings
+    assert np.max(np.abs(a[1][0][:, :, -1] - b[1][0][:, :, -1])) <= 2e-2
