@@ -20,10 +20,8 @@ __device__ long long g_selprof[16];
 #endif
 
 // key of position j: 0xFFFFFFFF for sink positions, the monotone image of z_j for candidates (z_j > zthr), 0 otherwise.
-// The logit is read past L1: in the fused path other SMs wrote it during the same launch.
-__device__ __forceinline__ uint32_t select_key_of(const float* zz, int j, int sink, float zthr) {
+__device__ __forceinline__ uint32_t select_key_from(float z, int j, int sink, float zthr) {
     if (j < sink) return 0xFFFFFFFFu;
-    const float z = __ldcg(zz + j);
     return z > zthr ? order_key(z) : 0u;
 }
 
@@ -39,9 +37,22 @@ __device__ __forceinline__ void select_group(const float* __restrict__ zz, int32
     const int N = T - W > 0 ? T - W : 0;
     const int p0 = tid * KPT;
 
+    // A thread's KPT consecutive logits are one run of memory: 16-byte loads through L1 where the run is aligned (a thread's
+    // loads then touch each 32-byte sector once: scalar loads past L1 made this phase 17 us of 36 at 32K positions per head)
     uint32_t key[KPT];
+    if (KPT % 4 == 0 && (reinterpret_cast<uintptr_t>(zz + p0) & 15u) == 0 && p0 + KPT <= T) {
 #pragma unroll
-    for (int i = 0; i < KPT; ++i) key[i] = p0 + i < N ? select_key_of(zz, p0 + i, sink, zthr) : 0u;
+        for (int i = 0; i < KPT; i += 4) {
+            const float4 z4 = __ldg(reinterpret_cast<const float4*>(zz + p0 + i));
+            key[i] = p0 + i < N ? select_key_from(z4.x, p0 + i, sink, zthr) : 0u;
+            key[i + 1] = p0 + i + 1 < N ? select_key_from(z4.y, p0 + i + 1, sink, zthr) : 0u;
+            key[i + 2] = p0 + i + 2 < N ? select_key_from(z4.z, p0 + i + 2, sink, zthr) : 0u;
+            key[i + 3] = p0 + i + 3 < N ? select_key_from(z4.w, p0 + i + 3, sink, zthr) : 0u;
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < KPT; ++i) key[i] = p0 + i < N ? select_key_from(__ldg(zz + p0 + i), p0 + i, sink, zthr) : 0u;
+    }
     // block-wide sum of a per-thread count, one barrier per call and no atomics: every warp leaves its sum in one of two
     // alternating rows of partials, and after the barrier every warp adds the row up itself.  A row is rewritten two calls
     // later, when every warp has passed the barrier of the call in between and so has finished reading it.
