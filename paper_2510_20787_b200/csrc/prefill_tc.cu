@@ -23,6 +23,23 @@ namespace lte {
 
 __device__ StatusWord g_prefill_status = LTE_STATUS_INIT;         // 0 = fine; otherwise the code of the wait that gave up
 
+// -DLTE_PROFILE: cycle counters of the row threads' phases (lane 0 of warp 0 of every CTA), added up over all CTAs;
+// PP(c) charges the time since the previous mark to phase c.  The product build does not define it.
+#ifdef LTE_PROFILE
+__device__ unsigned long long g_pprof[16];
+__device__ unsigned long long g_pprof_cta[1024 * 2];           // per CTA: globaltimer at kernel entry and at the end of the row loop
+#define PP_DECL long long pp_t = clock64(); long long pp_a[16] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0}
+#define PP(c) do { const long long pp_n = clock64(); pp_a[c] += pp_n - pp_t; pp_t = pp_n; } while (0)
+#define PP_COUNT(c, n) do { pp_a[c] += (n); } while (0)
+#define PP_FLUSH() do { if (warp == 0 && lane == 0) { _Pragma("unroll") for (int pp_i = 0; pp_i < 16; ++pp_i) atomicAdd(&g_pprof[pp_i], (unsigned long long)pp_a[pp_i]); \
+    unsigned long long gt; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt)); if (blockIdx.x < 1024) g_pprof_cta[blockIdx.x * 2 + 1] = gt; } } while (0)
+#else
+#define PP_DECL
+#define PP(c)
+#define PP_COUNT(c, n)
+#define PP_FLUSH()
+#endif
+
 namespace {
 
 constexpr int BM = 128, BN = 64, NTHREADS = 192;
@@ -43,8 +60,7 @@ template <int D> struct Smem {
     // more 64-column group, LBO away from the value tile.
     static constexpr bool ONES = D == 64;
     static constexpr int OFF_ONES = OFF_V + VST * KVTILE;     // [64][64] bf16 ones (8 KB), d = 64 only
-    static constexpr int OFF_OST = OFF_ONES + (ONES ? BN * 128 : 0);   // output staging: a [32][64] bf16 slab per softmax warp
-    static constexpr int OFF_BAR = OFF_OST + 4 * 4096;        // mbarriers, tmem slot
+    static constexpr int OFF_BAR = OFF_ONES + (ONES ? BN * 128 : 0);   // mbarriers, tmem slot
     static constexpr int BYTES = OFF_BAR + 256;
     static constexpr uint32_t TMEM_COLS = 256;                // S0: [0,64)  S1: [64,128)  O: [128, 128+D) (+16 row-sum columns)
 };
@@ -101,14 +117,17 @@ __device__ __forceinline__ int count_le(const int32_t* id, int n, int lim, int l
 template <int D, bool COMPACT>
 __global__ void __launch_bounds__(NTHREADS, 2)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                  const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
+                  const __grid_constant__ CUtensorMap tmV,
                   const __grid_constant__ CUtensorMap tmKc, const __grid_constant__ CUtensorMap tmVc,
                   const __nv_bfloat16* __restrict__ kg,
-                  const __nv_bfloat16* __restrict__ vg, const int32_t* __restrict__ idx,
+                  const __nv_bfloat16* __restrict__ vg, __nv_bfloat16* __restrict__ og, const int32_t* __restrict__ idx,
                   const int32_t* __restrict__ cnt, float* __restrict__ lse, int Tlen,
                   int W, int R, float scale, int n_qt, int n_bh, int G, int qoff)
 {
     const int n_items = n_qt * n_bh;
+#ifdef LTE_PROFILE
+    if (threadIdx.x == 0 && blockIdx.x < 1024) { unsigned long long gt; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt)); g_pprof_cta[blockIdx.x * 2] = gt; }
+#endif
     using S = Smem<D>;
     constexpr int SUB = S::SUB, KST = S::KST, VST = S::VST;
     constexpr uint32_t TMEM_COLS = S::TMEM_COLS;
@@ -299,6 +318,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             }
         };
         prefetch_list(blockIdx.x);
+        PP_DECL;
         for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++it) {
             const Item w = decode_item(item, n_qt, n_bh, Tlen, W, G, qoff);
             const int bh = w.bh, bhk = w.bhk, n_win = w.n_win, j_start = w.j_start;
@@ -337,6 +357,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             const int n_tiles = n_win + (nv_max + BN - 1) / BN;
             const int nvis_first = __shfl_sync(0xffffffffu, nvis, 0), nvis_last = __shfl_sync(0xffffffffu, nvis, 31);
             prefetch_list(item + gridDim.x);
+            PP(0); PP_COUNT(14, 1); PP_COUNT(15, n_tiles);
 
             // gather of one retained tile (t = its number within the item): 8 lanes per row copy its 16-byte chunks
             // (coalesced reads, conflict-free swizzled writes); rows past the visible prefix are zero-filled
@@ -428,8 +449,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     const uint32_t below_a = a >= 32 ? 0xffffffffu : ((1u << a) - 1u);
                     vm[cb] = b2 > a ? (below_b & ~below_a) : 0u;
                 }
+                PP(1);
                 mbar_wait(bar_s0 + 8 * (gg & 1), (gg >> 1) & 1, 3);   // S is in TMEM buffer gg & 1
                 tc_fence_after();
+                PP(2);
                 if (k_gather) { gather_issue(t + KST, false, rk); gathered = true; }   // its stage held this tile's K, which S has finished reading
                 else if (!COMPACT) cp_async_commit();
                 const uint32_t s_col = (gg & 1) * BN;
@@ -438,6 +461,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 for (int cb = 0; cb < 2; ++cb)
                     if (act[cb]) tmem_ld32(tmem + lane_base + s_col + cb * 32, r[cb]);
                 tmem_wait_ld();
+                PP(3);
                 float mr[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // row max of the raw logits, 4 chains
 #pragma unroll
                 for (int cb = 0; cb < 2; ++cb) {
@@ -477,6 +501,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     l_run *= alpha;
                 }
                 const float neg_m = m_run == -INFINITY ? 0.f : -m_run;
+                PP(4);
                 float ls[4] = {0.f, 0.f, 0.f, 0.f};
                 uint32_t pk[32];                               // the row of P as 64 bf16, two per word
 #pragma unroll
@@ -497,6 +522,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     }
                 }
                 l_run += (ls[0] + ls[1]) + (ls[2] + ls[3]);
+                PP(5);
                 // P goes back into TMEM, over the first 32 columns of the S buffer it was computed from (this thread has
                 // all of its row in registers), and feeds the PV product as the A operand: no trip through shared memory
                 tmem_st32(tmem + lane_base + s_col, pk);
@@ -505,15 +531,19 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 // PV of the previous tile has normally completed long ago.  Every phase of bar_pv is awaited in turn (a
                 // parity test is only meaningful for the current or the previous phase), and before the arrive: after
                 // it the barrier could run ahead of this thread.  At t = 0 the item's epilogue has awaited it.
+                PP(6);
                 if (t > 0) mbar_wait(bar_pv, (gg - 1) & 1, 4);
+                PP(7);
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_p);
                 // value tile t+VST-1 goes into the stage of tile t-1's V, which that PV has finished reading
                 if (v_gather) { gather_issue(t + VST - 1, true, rv); gathered = true; }
                 else if (!COMPACT) cp_async_commit();
             }
+            PP(1);
             mbar_wait(bar_pv, (g + n_tiles - 1) & 1, 5);
             tc_fence_after();
+            PP(8);
 
             // ---- epilogue: O / l -> bf16, logsumexp ------------------------------------------------------
             if (S::ONES) {                                     // the row sum is column D of the accumulator
@@ -523,9 +553,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 l_run = __uint_as_float(q1);
             }
             const float inv = 1.f / l_run;
-            // the normalised rows go through a swizzled shared-memory slab per warp and leave as one tile store per
-            // 64 columns (rows past the end of the sequence are clipped by the tensor map)
-            const uint32_t slab = base + S::OFF_OST + warp * 4096;
+            // a normalised row is D * 2 contiguous bytes of the output (whole 128-byte lines, and the rows of a warp are
+            // consecutive): each thread stores its own row with 16-byte stores, no staging in shared memory
+            __nv_bfloat16* orow = og + ((size_t)bh * (Tlen - qoff) + (i - qoff)) * D;
 #pragma unroll
             for (int sb = 0; sb < SUB; ++sb) {
                 uint32_t ow[32];                               // 64 columns of the row as bf16 pairs
@@ -545,23 +575,18 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar_of);        // the accumulator may take the next item
                 }
-                if (lane == 0) bulk_wait_read0();              // the slab's previous store has been read out
-                __syncwarp();
+                PP(9);
+                if (i < Tlen) {
 #pragma unroll
-                for (int ch = 0; ch < 8; ++ch)
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(slab + lane * 128 + ((ch ^ (lane & 7)) << 4)),
-                                 "r"(ow[4 * ch]), "r"(ow[4 * ch + 1]), "r"(ow[4 * ch + 2]), "r"(ow[4 * ch + 3]) : "memory");
-                fence_proxy_async();
-                __syncwarp();
-                if (lane == 0 && w.i0 + warp * 32 < Tlen) {
-                    tma_store_3d(&tmO, slab, sb * 64, w.i0 - qoff + warp * 32, bh);
-                    bulk_commit();
+                    for (int ch = 0; ch < 8; ++ch)
+                        *reinterpret_cast<uint4*>(orow + sb * 64 + ch * 8) = make_uint4(ow[4 * ch], ow[4 * ch + 1], ow[4 * ch + 2], ow[4 * ch + 3]);
                 }
             }
             if (i < Tlen) lse[(size_t)bh * (Tlen - qoff) + (i - qoff)] = m_run * 0.6931471805599453f + logf(l_run);
             g += n_tiles;
+            PP(11);
         }
-        if (lane == 0) bulk_wait_read0();                      // this warp's tile stores have read their slab
+        PP_FLUSH();
     }
     tc_fence_before();
     __syncthreads();
@@ -572,12 +597,10 @@ template <int D>
 int run(const Params& p, const void* q, const void* k, const void* v, const int32_t* idx, const int32_t* cnt, void* o,
         float* lse, void* ws, size_t ws_bytes, cudaStream_t st)
 {
-    CUtensorMap tq, tk, tv, to, tkc, tvc;
+    CUtensorMap tq, tk, tv, tkc, tvc;
     const int BHK = p.B * p.H, BH = BHK * p.G;                 // key/value heads, query heads
     const int Tq = p.T - p.qoff;                               // query rows (the whole sequence unless a chunk is prefilled)
-    if (!make_map(&tq, q, BH, Tq, D, BM) || !make_map(&tk, k, BHK, p.T, D, BN) || !make_map(&tv, v, BHK, p.T, D, BN) ||
-        !make_map(&to, o, BH, Tq, D, 32))
-        return LTE_ERR_CUDA;
+    if (!make_map(&tq, q, BH, Tq, D, BM) || !make_map(&tk, k, BHK, p.T, D, BN) || !make_map(&tv, v, BHK, p.T, D, BN)) return LTE_ERR_CUDA;
     // with a workspace the retained rows are compacted first and every tile is a TMA box
     const size_t half = prefill_compact_bytes(p) / 2;
     const bool compact = ws != nullptr && half > 0 && ws_bytes >= 2 * half && ((uintptr_t)ws & 127u) == 0;
@@ -598,11 +621,11 @@ int run(const Params& p, const void* q, const void* k, const void* v, const int3
     const int n_qt = (Tq + BM - 1) / BM, n_items = n_qt * BH;
     const int grid = n_items < slots ? n_items : slots;
     if (compact)
-        return cuda_status(launch_pdl(prefill_tc_kernel<D, true>, dim3(grid), dim3(NTHREADS), Smem<D>::BYTES, st, tq, tk, tv, to, tkc, tvc,
-                                      (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, idx, cnt, lse, p.T, p.W, p.R, p.scale, n_qt,
+        return cuda_status(launch_pdl(prefill_tc_kernel<D, true>, dim3(grid), dim3(NTHREADS), Smem<D>::BYTES, st, tq, tk, tv, tkc, tvc,
+                                      (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (__nv_bfloat16*)o, idx, cnt, lse, p.T, p.W, p.R, p.scale, n_qt,
                                       BH, p.G, p.qoff));
-    return cuda_status(launch_pdl(prefill_tc_kernel<D, false>, dim3(grid), dim3(NTHREADS), Smem<D>::BYTES, st, tq, tk, tv, to, tkc, tvc,
-                                  (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, idx, cnt, lse, p.T, p.W, p.R, p.scale, n_qt, BH,
+    return cuda_status(launch_pdl(prefill_tc_kernel<D, false>, dim3(grid), dim3(NTHREADS), Smem<D>::BYTES, st, tq, tk, tv, tkc, tvc,
+                                  (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (__nv_bfloat16*)o, idx, cnt, lse, p.T, p.W, p.R, p.scale, n_qt, BH,
                                   p.G, p.qoff));
 }
 
@@ -619,6 +642,19 @@ int launch_prefill_tc(const Params& p, const void* q, const void* k, const void*
     return launch_prefill_simt(p, q, k, v, idx, cnt, o, lse, st);   // d = 32: rows too narrow for the 128-byte swizzle
 }
 
+
+#ifdef LTE_PROFILE
+extern "C" int lte_pprof_read(unsigned long long* out, int clear)
+{
+    if (cudaMemcpyFromSymbol(out, g_pprof, sizeof(unsigned long long) * 16) != cudaSuccess) return -1;
+    if (clear) { unsigned long long z[16] = {}; cudaMemcpyToSymbol(g_pprof, z, sizeof(z)); }
+    return 0;
+}
+extern "C" int lte_pprof_cta_read(unsigned long long* out)
+{
+    return cudaMemcpyFromSymbol(out, g_pprof_cta, sizeof(unsigned long long) * 2048) == cudaSuccess ? 0 : -1;
+}
+#endif
 
 int prefill_status_fetch_and_clear()
 {
