@@ -1,6 +1,5 @@
 // Capped selection of one (b,h) by a group of threads that keep their keys in registers (Section 3.1.3, "Capped
-// capacity"): shared by the select kernel (a whole block) and by the scorer kernel, whose CTA that completes a head's
-// last logits selects that head on the spot.
+// capacity"): the body of the select kernel, written for any group of whole warps with a barrier of its own.
 //
 // Thread `tid` of `nthr` owns KPT consecutive positions.  The R-th largest key is found by bisection on its 32 bits:
 // each step counts the keys >= a candidate value (compares in registers, a warp reduction, one group barrier), so
