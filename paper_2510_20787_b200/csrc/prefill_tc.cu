@@ -502,6 +502,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 }
                 const float neg_m = m_run == -INFINITY ? 0.f : -m_run;
                 PP(4);
+                const uint64_t c2_2 = pack2(c2, c2), neg_m2 = pack2(neg_m, neg_m);
                 float ls[4] = {0.f, 0.f, 0.f, 0.f};
                 uint32_t pk[32];                               // the row of P as 64 bf16, two per word
 #pragma unroll
@@ -510,8 +511,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 #pragma unroll
                         for (int c = 0; c < 32; c += 2) {
                             // masked entries hold -inf: fma gives -inf and exp2(-inf) = 0
-                            const float p0 = fast_exp2(fmaf(__uint_as_float(r[cb][c]), c2, neg_m));
-                            const float p1 = fast_exp2(fmaf(__uint_as_float(r[cb][c + 1]), c2, neg_m));
+                            float x0, x1;                      // two columns per packed fp32 instruction
+                            unpack2(fma2(pack2(__uint_as_float(r[cb][c]), __uint_as_float(r[cb][c + 1])), c2_2, neg_m2), x0, x1);
+                            const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
                             if (!S::ONES) ls[(c >> 1) & 3] += p0 + p1;   // with ONES the tensor core sums the rounded probabilities
                             __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
                             pk[cb * 16 + (c >> 1)] = *reinterpret_cast<uint32_t*>(&h);
