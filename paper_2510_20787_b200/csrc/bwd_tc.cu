@@ -335,6 +335,7 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             tc_fence_after();
             const uint32_t sbuf = DB ? (uint32_t)(t & 1) * (2 * BN) : 0u;
             uint32_t pk[32];                                   // dS row as 64 bf16
+            const uint64_t c2_2 = pack2(c2, c2), nl2_2 = pack2(-L2, -L2), scale_2 = pack2(scale, scale), ndls_2 = pack2(-dl * scale, -dl * scale);
 #pragma unroll
             for (int cb = 0; cb < 2; ++cb) {
                 const bool act = cb * 32 <= u_hi && cb * 32 + 31 >= u_lo;
@@ -343,15 +344,18 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     tmem_ld32(tmem + lane_base + sbuf + cb * 32, rs);
                     tmem_ld32(tmem + lane_base + sbuf + DP_COL + cb * 32, rp);
                     tmem_wait_ld();
+                    // validity bits of this row's 32 columns; the arithmetic runs on packed fp32 pairs
+                    const int a = min(max(c_lo - cb * 32, 0), 32), b2 = min(max(c_hi - cb * 32 + 1, 0), 32);
+                    const uint32_t below_b = b2 >= 32 ? 0xffffffffu : ((1u << b2) - 1u);
+                    const uint32_t below_a = a >= 32 ? 0xffffffffu : ((1u << a) - 1u);
+                    const uint32_t vm = b2 > a ? (below_b & ~below_a) : 0u;
 #pragma unroll
                     for (int c = 0; c < 32; c += 2) {
-                        const int col = cb * 32 + c;
-                        float d0 = 0.f, d1 = 0.f;
-                        if (col >= c_lo && col <= c_hi)
-                            d0 = fast_exp2(fmaf(__uint_as_float(rs[c]), c2, -L2)) * (__uint_as_float(rp[c]) - dl) * scale;
-                        if (col + 1 >= c_lo && col + 1 <= c_hi)
-                            d1 = fast_exp2(fmaf(__uint_as_float(rs[c + 1]), c2, -L2)) * (__uint_as_float(rp[c + 1]) - dl) * scale;
-                        __nv_bfloat162 h = __floats2bfloat162_rn(d0, d1);
+                        float x0, x1, d0, d1;
+                        unpack2(fma2(pack2(__uint_as_float(rs[c]), __uint_as_float(rs[c + 1])), c2_2, nl2_2), x0, x1);
+                        const uint64_t g2 = fma2(pack2(__uint_as_float(rp[c]), __uint_as_float(rp[c + 1])), scale_2, ndls_2);   // (dP - delta) scale
+                        unpack2(mul2(pack2(fast_exp2(x0), fast_exp2(x1)), g2), d0, d1);
+                        __nv_bfloat162 h = __floats2bfloat162_rn((vm & (1u << c)) ? d0 : 0.f, (vm & (2u << c)) ? d1 : 0.f);
                         pk[cb * 16 + (c >> 1)] = *reinterpret_cast<uint32_t*>(&h);
                     }
                 } else {
@@ -662,6 +666,7 @@ bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
             tc_fence_after();
             const uint32_t tb = tmem + lane_base + (DB ? (uint32_t)(t & 1) * 128u : 0u);
             uint32_t pp[32], pd[32];                           // P^T and dS^T rows as 64 bf16 each
+            const uint64_t c2_2 = pack2(c2, c2), scale_2 = pack2(scale, scale);
 #pragma unroll
             for (int cb = 0; cb < 2; ++cb) {
                 const bool act = cb * 32 <= u_hi && cb * 32 + 31 >= u_lo;
@@ -669,20 +674,24 @@ bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                     uint32_t rs[32], rp[32];
                     tmem_ld32(tb + cb * 32, rs);
                     tmem_ld32(tb + DP_COL + cb * 32, rp);
+                    const int a = min(max(c_lo - cb * 32, 0), 32), b2 = min(max(c_hi - cb * 32 + 1, 0), 32);
+                    const uint32_t below_b = b2 >= 32 ? 0xffffffffu : ((1u << b2) - 1u);
+                    const uint32_t below_a = a >= 32 ? 0xffffffffu : ((1u << a) - 1u);
+                    const uint32_t vm = b2 > a ? (below_b & ~below_a) : 0u;   // validity bits of this row's 32 columns
                     tmem_wait_ld();
 #pragma unroll
                     for (int c = 0; c < 32; c += 4) {
                         const int col = cb * 32 + c;
                         const float4 l4 = *reinterpret_cast<const float4*>(&s_col[col]);
                         const float4 d4 = *reinterpret_cast<const float4*>(&s_col[64 + col]);
-                        const float lv[4] = {l4.x, l4.y, l4.z, l4.w}, dvv[4] = {d4.x, d4.y, d4.z, d4.w};
-                        float p[4], ds[4];
+                        // packed fp32 pairs: exponent arguments, (dP scale - delta scale), their product with P
+                        float x[4], p[4], ds[4];
+                        unpack2(fma2(pack2(__uint_as_float(rs[c]), __uint_as_float(rs[c + 1])), c2_2, pack2(l4.x, l4.y)), x[0], x[1]);
+                        unpack2(fma2(pack2(__uint_as_float(rs[c + 2]), __uint_as_float(rs[c + 3])), c2_2, pack2(l4.z, l4.w)), x[2], x[3]);
 #pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            const bool ok = col + u >= c_lo && col + u <= c_hi;
-                            p[u] = ok ? fast_exp2(fmaf(__uint_as_float(rs[c + u]), c2, lv[u])) : 0.f;
-                            ds[u] = p[u] * fmaf(__uint_as_float(rp[c + u]), scale, dvv[u]);
-                        }
+                        for (int u = 0; u < 4; ++u) p[u] = (vm & (1u << (c + u))) ? fast_exp2(x[u]) : 0.f;
+                        unpack2(mul2(pack2(p[0], p[1]), fma2(pack2(__uint_as_float(rp[c]), __uint_as_float(rp[c + 1])), scale_2, pack2(d4.x, d4.y))), ds[0], ds[1]);
+                        unpack2(mul2(pack2(p[2], p[3]), fma2(pack2(__uint_as_float(rp[c + 2]), __uint_as_float(rp[c + 3])), scale_2, pack2(d4.z, d4.w))), ds[2], ds[3]);
                         __nv_bfloat162 h0 = __floats2bfloat162_rn(p[0], p[1]), h1 = __floats2bfloat162_rn(p[2], p[3]);
                         __nv_bfloat162 g0 = __floats2bfloat162_rn(ds[0], ds[1]), g1 = __floats2bfloat162_rn(ds[2], ds[3]);
                         pp[cb * 16 + (c >> 1)] = *reinterpret_cast<uint32_t*>(&h0);
