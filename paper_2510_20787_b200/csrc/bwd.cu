@@ -10,6 +10,7 @@
 //               the scorer's share sum_t dz[p-t+half] w[h,t,c] is added to the fp32 dk, dv before the one rounding.
 // Workspace: delta, dz [B,H,T] fp32; dw/dbias partials; fp32 dk, dv [B,H,T,d] when the flag is set.
 #include "common.cuh"
+#include "tc_common.cuh"
 
 namespace lte {
 
@@ -375,20 +376,21 @@ bwd_tail_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __rest
     const int cc = (cg % (D / 4)) * 4;              // first of this thread's 4 channels within k or v
     const __nv_bfloat16* src = isv ? v : k;
     __nv_bfloat16* gdst = isv ? dv : dk;
-    float wr[K][4];                                 // this thread's scorer weights
+    // the multiply-adds run on packed fp32 pairs (channels 0,1 and 2,3 of the thread's four): the loop is bound by
+    // instruction issue, not by memory
+    using tc::pack2; using tc::unpack2; using tc::fma2;
+    uint64_t wr2[K][2];                             // this thread's scorer weights
     if (FINISH) {
 #pragma unroll
         for (int t = 0; t < K; ++t) {
             const float4 w4 = *reinterpret_cast<const float4*>(&w[((size_t)h * K + t) * 2 * D + cg * 4]);
-            wr[t][0] = w4.x; wr[t][1] = w4.y; wr[t][2] = w4.z; wr[t][3] = w4.w;
+            wr2[t][0] = pack2(w4.x, w4.y); wr2[t][1] = pack2(w4.z, w4.w);
         }
     }
     __syncthreads();
-    float acc[K][4];
+    uint64_t acc2[K][2];
 #pragma unroll
-    for (int t = 0; t < K; ++t)
-#pragma unroll
-        for (int e = 0; e < 4; ++e) acc[t][e] = 0.f;
+    for (int t = 0; t < K; ++t) acc2[t][0] = acc2[t][1] = pack2(0.f, 0.f);
     // U rows per batch: all of a batch's loads are issued before any of its arithmetic (row indices are clamped so
     // that every load is legal; rows past the end are skipped afterwards)
     constexpr int U = 8;
@@ -406,23 +408,21 @@ bwd_tail_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __rest
         for (int u = 0; u < U; ++u) {
             const int rl = rb + u * RPP, p = p0 + rl;
             if (rl >= rows || p >= Tlen) continue;
-            float x[4], g[K];
-            x[0] = __uint_as_float(ux[u].x << 16); x[1] = __uint_as_float(ux[u].x & 0xffff0000u);
-            x[2] = __uint_as_float(ux[u].y << 16); x[3] = __uint_as_float(ux[u].y & 0xffff0000u);
+            uint64_t g2[K];
+            const uint64_t x01 = pack2(__uint_as_float(ux[u].x << 16), __uint_as_float(ux[u].x & 0xffff0000u));
+            const uint64_t x23 = pack2(__uint_as_float(ux[u].y << 16), __uint_as_float(ux[u].y & 0xffff0000u));
 #pragma unroll
-            for (int t = 0; t < K; ++t) g[t] = dzs[rl - t + 2 * half];      // dz[p - t + half]
+            for (int t = 0; t < K; ++t) { const float g = dzs[rl - t + 2 * half]; g2[t] = pack2(g, g); }   // dz[p - t + half]
 #pragma unroll
-            for (int t = 0; t < K; ++t)
-#pragma unroll
-                for (int e = 0; e < 4; ++e) acc[t][e] = fmaf(g[t], x[e], acc[t][e]);
+            for (int t = 0; t < K; ++t) { acc2[t][0] = fma2(g2[t], x01, acc2[t][0]); acc2[t][1] = fma2(g2[t], x23, acc2[t][1]); }
             const int er = ent[rl + half];                   // retained: its far-query share is added here
             if (FINISH || er >= 0) {
                 float gi[4] = {0.f, 0.f, 0.f, 0.f};
                 if (FINISH) {
+                    uint64_t gi01 = pack2(0.f, 0.f), gi23 = gi01;
 #pragma unroll
-                    for (int t = 0; t < K; ++t)
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) gi[e] = fmaf(g[t], wr[t][e], gi[e]);
+                    for (int t = 0; t < K; ++t) { gi01 = fma2(g2[t], wr2[t][0], gi01); gi23 = fma2(g2[t], wr2[t][1], gi23); }
+                    unpack2(gi01, gi[0], gi[1]); unpack2(gi23, gi[2], gi[3]);
                 }
                 if (er >= 0) {
                     const float4 f4 = *reinterpret_cast<const float4*>(gret + ((size_t)bh * R + er) * D + cc);
@@ -435,6 +435,9 @@ bwd_tail_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __rest
             }
         }
     }
+    float acc[K][4];
+#pragma unroll
+    for (int t = 0; t < K; ++t) { unpack2(acc2[t][0], acc[t][0], acc[t][1]); unpack2(acc2[t][1], acc[t][2], acc[t][3]); }
     // ---- add the partials of the row slots: slots [step, 2 step) hand their sums to slots [0, step) ---------
 #pragma unroll
     for (int step = RPP / 2; step >= 1; step >>= 1) {
