@@ -13,7 +13,7 @@ namespace lte {
 
 #ifdef LTE_PROFILE
 __device__ long long g_selprof[16];
-#define SELP(i) do { if (blockIdx.x == 0 && tid == 0) g_selprof[i] = clock64(); } while (0)
+#define SELP(i) do { if (blockIdx.x == 0 && tid == 0) { g_selprof[i] = clock64(); if ((i) == 0 || (i) == 6) { unsigned long long gt; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt)); g_selprof[(i) == 0 ? 10 : 11] = (long long)gt; } } } while (0)
 #else
 #define SELP(i) do {} while (0)
 #endif
