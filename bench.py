@@ -463,10 +463,24 @@ def _extra_k(out, torch, lte, synth, pk, flush, n5):
             lte.lte_attn_prefill(s1, qc, kc, vc, i1, c1, o=o, lse=lse, ws=prefill_ws(torch, lte, s1))
 
         ms1, _ = timed(torch, one_shot, n5, 3, flush)
+        # the streaming reading of the same chunk (exact under a binding cap; row-by-row attention on the fp32 ALUs)
+        ws_s = torch.empty(lte.lte_workspace_bytes(lte.OP_CHUNK_STREAM, sc, c), dtype=torch.uint8, device="cuda")
+        ms_s = []
+        for it in range(2 + n5):
+            cache.copy_(cache0)
+            flush()
+            e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+            e0.record()
+            lte.lte_attn_prefill_chunk(sc, c, cache, cfg.T, qc, kc, vc, o=o, lse=lse, ws=ws_s, streaming=True)
+            e1.record(); torch.cuda.synchronize()
+            if it >= 2:
+                ms_s.append(e0.elapsed_time(e1))
+        del ws_s
         t = mid3(ms) * 1e-3
         res[tag] = {"workload": "B=%d H=%d d=%d, cache after %d tokens (W=%d, R=%d), chunk of %d tokens" % (cfg.B, cfg.H, cfg.d, cfg.T, cfg.W, cfg.R, Tc),
                     "chunk_ms": t * 1e3, "tokens_per_s": cfg.B * Tc / t, "local_rows": cfg.R + cfg.W + Tc,
                     "one_shot_prefill_of_a_prompt_of_the_chunks_length_ms": mid3(ms1),
+                    "streaming_reading_chunk_ms": mid3(ms_s),
                     "workspace_bytes": int(ws.numel())}
         del x, cache, cache0, ws, o, lse, qc, kc, vc
     out["K_chunked_prefill"] = res
