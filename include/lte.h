@@ -77,7 +77,7 @@ typedef struct lte_conv {
  * aligned; it receives the weights split into bf16 pieces, rebuilt by every call) the stack runs on the tensor cores
  * with exact products and fp32 accumulation; without the workspace, and for every other accepted shape, on the fp32
  * ALUs.  Both agree with an fp64 evaluation to about 1e-5 at |z| of a few units.
- * lte_attn_bwd takes the stack for d = 64: dw and dbias then have the packed layouts of w and bias above.
+ * lte_attn_bwd takes the stack for d = 64 and d = 32: dw and dbias then have the packed layouts of w and bias above.
  * lte_cache_init and lte_attn_decode take the stack for d = 32 or 64 and W >= 20; the step then scores nothing and
  * lte_cache_score has to be called periodically.  lte_attn_bwd_static takes the single layer only.
  */

@@ -449,8 +449,8 @@ int lte_attn_bwd(const lte_shape* s, const lte_conv* c, const void* q, const voi
                  uint32_t flags, void* ws, size_t ws_bytes, void* stream)
 {
     int e = check_shape(s, true); if (e) return e;
-    if (c && c->w && c->n_layers == 3) {                   // the paper's stack: d = 64, gradients packed like the parameters
-        if (c->kernel != 3 || c->dilation != 2 || s->d != 64) return LTE_ERR_UNSUPPORTED;
+    if (c && c->w && c->n_layers == 3) {                   // the paper's stack: d = 64 or 32, gradients packed like the parameters
+        if (c->kernel != 3 || c->dilation != 2 || (s->d != 64 && s->d != 32)) return LTE_ERR_UNSUPPORTED;
         if (s->W < 7 || !aligned16(c->w)) return LTE_ERR_INVALID_ARG;
     } else {
         e = check_conv(s, c); if (e) return e;

@@ -1,4 +1,4 @@
-// Backward of the paper's scorer stack (Section 3.1.1's module under the gradient of Section 3.1.2), d = 64, fp32 on
+// Backward of the paper's scorer stack (Section 3.1.1's module under the gradient of Section 3.1.2), d = 64 or 32, fp32 on
 // the ordinary ALUs: given dL/dz per token (the straight-through surrogate has already produced it), the gradients of
 // the three conv layers' weights and biases and of the output map, and optionally the gradient into k and v.
 //
@@ -17,24 +17,32 @@ namespace lte {
 namespace {
 
 constexpr int SB_NT = 256, SB_TR = 32;
-constexpr int SB_C0 = 128, SB_C1 = 64, SB_C2 = 32, SB_C3 = 16;
 // rows of a tile: x from a-12, h0 from a-8, h1 from a-4, h2 from a; all end at a + TR + 12
 constexpr int SB_RX = SB_TR + 24, SB_R0 = SB_TR + 20, SB_R1 = SB_TR + 16, SB_R2 = SB_TR + 12;
-constexpr int SB_SX = SB_C0 + 4, SB_S0 = SB_C1 + 4, SB_S1 = SB_C2 + 4, SB_S2 = SB_C3 + 4;   // row strides (floats)
-constexpr int SB_W0 = 3 * SB_C0 * (SB_C1 + 4), SB_W1 = 3 * SB_C1 * (SB_C2 + 4), SB_W2 = 3 * SB_C2 * (SB_C3 + 4);
-constexpr int SB_OFF_W0 = 0, SB_OFF_W1 = SB_OFF_W0 + SB_W0, SB_OFF_W2 = SB_OFF_W1 + SB_W1, SB_OFF_P = SB_OFF_W2 + SB_W2;
-constexpr int SB_OFF_X = SB_OFF_P + 144;                       // parameters: b0[64] b1[32] b2[16] wout[16] bout
-constexpr int SB_OFF_H0 = SB_OFF_X + SB_RX * SB_SX, SB_OFF_D0 = SB_OFF_H0 + SB_R0 * SB_S0;
-constexpr int SB_OFF_H1 = SB_OFF_D0 + SB_R0 * SB_S0, SB_OFF_D1 = SB_OFF_H1 + SB_R1 * SB_S1;
-constexpr int SB_OFF_H2 = SB_OFF_D1 + SB_R1 * SB_S1, SB_OFF_D2 = SB_OFF_H2 + SB_R2 * SB_S2;
-constexpr int SB_OFF_DZ = SB_OFF_D2 + SB_R2 * SB_S2;           // delta3 of the tile's rows [SB_R2]
-constexpr int SB_FLOATS = SB_OFF_DZ + ((SB_R2 + 3) & ~3);
-constexpr size_t SB_BYTES = (size_t)SB_FLOATS * sizeof(float);
-static_assert(SB_BYTES <= 232448, "shared memory");
-// packed gradient layout of one head (floats): wl0 [64][3][128] | wl1 [32][3][64] | wl2 [16][3][32] | wout [16] | b0 | b1 | b2 | bout
-constexpr int SB_G0 = SB_C1 * 3 * SB_C0, SB_G1 = SB_C2 * 3 * SB_C1, SB_G2 = SB_C3 * 3 * SB_C2;
-constexpr int SB_PART = SB_G0 + SB_G1 + SB_G2 + SB_C3 + SB_C1 + SB_C2 + SB_C3 + 1;   // 32,385
-constexpr int SB_PART_PAD = (SB_PART + 31) & ~31;
+// Channel plan 2d -> d -> d/2 -> d/4 -> 1 and everything that follows from it (d = 64 or 32).
+template <int D> struct SBL {
+    static constexpr int C0 = 2 * D, C1 = D, C2 = D / 2, C3 = D / 4;
+    static constexpr int SX = C0 + 4, S0 = C1 + 4, S1 = C2 + 4, S2 = C3 + 4;   // row strides (floats)
+    static constexpr int W0 = 3 * C0 * (C1 + 4), W1 = 3 * C1 * (C2 + 4), W2 = 3 * C2 * (C3 + 4);
+    static constexpr int OFF_W0 = 0, OFF_W1 = OFF_W0 + W0, OFF_W2 = OFF_W1 + W1, OFF_P = OFF_W2 + W2;
+    // parameters: b0[C1] b1[C2] b2[C3] wout[C3] bout; the same thread numbers own their gradients
+    static constexpr int P1 = C1, P2 = P1 + C2, P3 = P2 + C3, P4 = P3 + C3, NP = P4 + 1, NP_PAD = (NP + 15) & ~15;
+    static constexpr int OFF_X = OFF_P + NP_PAD;
+    static constexpr int OFF_H0 = OFF_X + SB_RX * SX, OFF_D0 = OFF_H0 + SB_R0 * S0;
+    static constexpr int OFF_H1 = OFF_D0 + SB_R0 * S0, OFF_D1 = OFF_H1 + SB_R1 * S1;
+    static constexpr int OFF_H2 = OFF_D1 + SB_R1 * S1, OFF_D2 = OFF_H2 + SB_R2 * S2;
+    static constexpr int OFF_DZ = OFF_D2 + SB_R2 * S2;         // delta3 of the tile's rows [SB_R2]
+    static constexpr int FLOATS = OFF_DZ + ((SB_R2 + 3) & ~3);
+    static constexpr size_t BYTES = (size_t)FLOATS * sizeof(float);
+    static_assert(BYTES <= 232448, "shared memory");
+    // packed gradient layout of one head (floats): wl0 [C1][3][C0] | wl1 [C2][3][C1] | wl2 [C3][3][C2] | wout [C3] | b0 | b1 | b2 | bout
+    static constexpr int G0 = C1 * 3 * C0, G1 = C2 * 3 * C1, G2 = C3 * 3 * C2;
+    static constexpr int PART = G0 + G1 + G2 + C3 + C1 + C2 + C3 + 1;   // 32,385 at d = 64
+    static constexpr int PART_PAD = (PART + 31) & ~31;
+    // input channels per thread in the weight-gradient products (a thread owns 4 outputs x CB inputs x 3 taps)
+    static constexpr int CB0 = D == 64 ? 8 : 2, CB1 = D == 64 ? 2 : 1, CB2 = 1;
+    static_assert((C1 / 4) * (C0 / CB0) <= SB_NT && (C2 / 4) * (C1 / CB1) <= SB_NT && (C3 / 4) * (C2 / CB2) <= SB_NT, "threads");
+};
 
 // Forward layer: out[r][o] = Swish(y), sp[r][o] = Swish'(y), y = bias[o] + sum_{tau, c} w[tau][c][o] in[r + 2 tau][c];
 // out row r is at time t_out0 + r (zero, with zero derivative, at negative times); in row 0 is at time t_out0 - 4.
@@ -166,7 +174,7 @@ __device__ __forceinline__ void sb_wgrad(float (&acc)[3][4][CB], const float* __
     }
 }
 
-template <typename T>
+template <typename T, int D>
 __global__ void __launch_bounds__(SB_NT, 1)
 stack_bwd_kernel(const T* __restrict__ k, const T* __restrict__ v, const float* __restrict__ wpack,
                  const float* __restrict__ bpack, const float* __restrict__ dz, T* __restrict__ dk, T* __restrict__ dv,
@@ -175,52 +183,53 @@ stack_bwd_kernel(const T* __restrict__ k, const T* __restrict__ v, const float* 
     extern __shared__ __align__(16) float sm[];
     pdl_launch_dependents();
     pdl_wait();
-    constexpr int D = 64;
+    using L = SBL<D>;
     const int bh = blockIdx.y, h = bh % H, tid = threadIdx.x;
     const int n_tiles = (Tlen + SB_TR - 1) / SB_TR;
     const int tile_begin = blockIdx.x * tiles_per_cta, tile_end = min(tile_begin + tiles_per_cta, n_tiles);
-    float* my_part = part + ((size_t)bh * gridDim.x + blockIdx.x) * SB_PART_PAD;
+    float* my_part = part + ((size_t)bh * gridDim.x + blockIdx.x) * L::PART_PAD;
 
     // ---- this head's parameters: weights as [tap][c_in][c_out + 4] ----
-    const float* g0 = wpack + (size_t)h * SB_G0;
-    const float* g1 = wpack + (size_t)H * SB_G0 + (size_t)h * SB_G1;
-    const float* g2 = wpack + (size_t)H * (SB_G0 + SB_G1) + (size_t)h * SB_G2;
-    const float* go = wpack + (size_t)H * (SB_G0 + SB_G1 + SB_G2) + (size_t)h * SB_C3;
-    for (int e = tid; e < SB_G0; e += SB_NT) {                 // e = (o * 3 + tau) * C0 + c
-        const int c = e % SB_C0, ot = e / SB_C0, tau = ot % 3, o = ot / 3;
-        sm[SB_OFF_W0 + (tau * SB_C0 + c) * (SB_C1 + 4) + o] = g0[e];
+    const float* g0 = wpack + (size_t)h * L::G0;
+    const float* g1 = wpack + (size_t)H * L::G0 + (size_t)h * L::G1;
+    const float* g2 = wpack + (size_t)H * (L::G0 + L::G1) + (size_t)h * L::G2;
+    const float* go = wpack + (size_t)H * (L::G0 + L::G1 + L::G2) + (size_t)h * L::C3;
+    for (int e = tid; e < L::G0; e += SB_NT) {                 // e = (o * 3 + tau) * C0 + c
+        const int c = e % L::C0, ot = e / L::C0, tau = ot % 3, o = ot / 3;
+        sm[L::OFF_W0 + (tau * L::C0 + c) * (L::C1 + 4) + o] = g0[e];
     }
-    for (int e = tid; e < SB_G1; e += SB_NT) {
-        const int c = e % SB_C1, ot = e / SB_C1, tau = ot % 3, o = ot / 3;
-        sm[SB_OFF_W1 + (tau * SB_C1 + c) * (SB_C2 + 4) + o] = g1[e];
+    for (int e = tid; e < L::G1; e += SB_NT) {
+        const int c = e % L::C1, ot = e / L::C1, tau = ot % 3, o = ot / 3;
+        sm[L::OFF_W1 + (tau * L::C1 + c) * (L::C2 + 4) + o] = g1[e];
     }
-    for (int e = tid; e < SB_G2; e += SB_NT) {
-        const int c = e % SB_C2, ot = e / SB_C2, tau = ot % 3, o = ot / 3;
-        sm[SB_OFF_W2 + (tau * SB_C2 + c) * (SB_C3 + 4) + o] = g2[e];
+    for (int e = tid; e < L::G2; e += SB_NT) {
+        const int c = e % L::C2, ot = e / L::C2, tau = ot % 3, o = ot / 3;
+        sm[L::OFF_W2 + (tau * L::C2 + c) * (L::C3 + 4) + o] = g2[e];
     }
-    for (int e = tid; e < 144; e += SB_NT) {
+    for (int e = tid; e < L::NP; e += SB_NT) {
         float b = 0.f;
-        if (e < 64) b = bpack ? bpack[(size_t)h * 64 + e] : 0.f;
-        else if (e < 96) b = bpack ? bpack[(size_t)H * 64 + (size_t)h * 32 + (e - 64)] : 0.f;
-        else if (e < 112) b = bpack ? bpack[(size_t)H * 96 + (size_t)h * 16 + (e - 96)] : 0.f;
-        else if (e < 128) b = go[e - 112];
-        else if (e == 128) b = bpack ? bpack[(size_t)H * 112 + h] : 0.f;
-        sm[SB_OFF_P + e] = b;
+        if (e < L::P1) b = bpack ? bpack[(size_t)h * L::C1 + e] : 0.f;
+        else if (e < L::P2) b = bpack ? bpack[(size_t)H * L::C1 + (size_t)h * L::C2 + (e - L::P1)] : 0.f;
+        else if (e < L::P3) b = bpack ? bpack[(size_t)H * (L::C1 + L::C2) + (size_t)h * L::C3 + (e - L::P2)] : 0.f;
+        else if (e < L::P4) b = go[e - L::P3];
+        else b = bpack ? bpack[(size_t)H * (L::C1 + L::C2 + L::C3) + h] : 0.f;
+        sm[L::OFF_P + e] = b;
     }
-    const float* sb0 = sm + SB_OFF_P, *sb1 = sm + SB_OFF_P + 64, *sb2 = sm + SB_OFF_P + 96, *swo = sm + SB_OFF_P + 112;
+    const float* sb0 = sm + L::OFF_P, *sb1 = sm + L::OFF_P + L::P1, *sb2 = sm + L::OFF_P + L::P2, *swo = sm + L::OFF_P + L::P3;
 
     // gradient accumulators of this CTA (registers, across its tiles)
-    float a0[3][4][8], a1[3][4][2], a2[3][4][1];
+    float a0[3][4][L::CB0], a1[3][4][L::CB1], a2[3][4][L::CB2];
 #pragma unroll
     for (int t = 0; t < 3; ++t)
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
 #pragma unroll
-            for (int c = 0; c < 8; ++c) a0[t][j][c] = 0.f;
-            a1[t][j][0] = a1[t][j][1] = 0.f;
+            for (int c = 0; c < L::CB0; ++c) a0[t][j][c] = 0.f;
+#pragma unroll
+            for (int c = 0; c < L::CB1; ++c) a1[t][j][c] = 0.f;
             a2[t][j][0] = 0.f;
         }
-    float small = 0.f;                                         // thread < 64: db0; < 96: db1; < 112: db2; < 128: dwout; 128: dbout
+    float small = 0.f;                                         // thread < P1: db0; < P2: db1; < P3: db2; < P4: dwout; P4: dbout
 
     const T* kk = k + (size_t)bh * Tlen * D;
     const T* vv = v + (size_t)bh * Tlen * D;
@@ -229,8 +238,8 @@ stack_bwd_kernel(const T* __restrict__ k, const T* __restrict__ v, const float* 
         const int a = tile * SB_TR;                            // the tile owns times a .. a + TR - 1
         __syncthreads();                                       // the previous tile's readers are done (and the parameters are in)
         // ---- input rows a-12 .. a+TR+11 (zero outside [0, T)) and delta3[t] = dz[t - 6] for the rows a .. a+TR+11 ----
-        for (int e = tid; e < SB_RX * (SB_C0 / 4); e += SB_NT) {
-            const int r = e / (SB_C0 / 4), c4 = (e % (SB_C0 / 4)) * 4;
+        for (int e = tid; e < SB_RX * (L::C0 / 4); e += SB_NT) {
+            const int r = e / (L::C0 / 4), c4 = (e % (L::C0 / 4)) * 4;
             const int t = a - 12 + r;
             float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
             if (t >= 0 && t < Tlen) {
@@ -243,54 +252,54 @@ stack_bwd_kernel(const T* __restrict__ k, const T* __restrict__ v, const float* 
                     x = *reinterpret_cast<const float4*>(src);
                 }
             }
-            *reinterpret_cast<float4*>(&sm[SB_OFF_X + r * SB_SX + c4]) = x;
+            *reinterpret_cast<float4*>(&sm[L::OFF_X + r * L::SX + c4]) = x;
         }
         if (tid < SB_R2) {
             const int t = a + tid;
-            sm[SB_OFF_DZ + tid] = (t >= 6 && t < Tlen) ? dzz[t - 6] : 0.f;   // the caller's dz is zero where the logit is undefined
+            sm[L::OFF_DZ + tid] = (t >= 6 && t < Tlen) ? dzz[t - 6] : 0.f;   // the caller's dz is zero where the logit is undefined
         }
         __syncthreads();
         // ---- forward, keeping activations and Swish' ----
-        sb_forward<SB_C0, SB_C1, SB_R0, SB_SX, SB_S0>(sm + SB_OFF_X, sm + SB_OFF_H0, sm + SB_OFF_D0, sm + SB_OFF_W0, sb0, a - 8);
+        sb_forward<L::C0, L::C1, SB_R0, L::SX, L::S0>(sm + L::OFF_X, sm + L::OFF_H0, sm + L::OFF_D0, sm + L::OFF_W0, sb0, a - 8);
         __syncthreads();
-        sb_forward<SB_C1, SB_C2, SB_R1, SB_S0, SB_S1>(sm + SB_OFF_H0, sm + SB_OFF_H1, sm + SB_OFF_D1, sm + SB_OFF_W1, sb1, a - 4);
+        sb_forward<L::C1, L::C2, SB_R1, L::S0, L::S1>(sm + L::OFF_H0, sm + L::OFF_H1, sm + L::OFF_D1, sm + L::OFF_W1, sb1, a - 4);
         __syncthreads();
-        sb_forward<SB_C2, SB_C3, SB_R2, SB_S1, SB_S2>(sm + SB_OFF_H1, sm + SB_OFF_H2, sm + SB_OFF_D2, sm + SB_OFF_W2, sb2, a);
+        sb_forward<L::C2, L::C3, SB_R2, L::S1, L::S2>(sm + L::OFF_H1, sm + L::OFF_H2, sm + L::OFF_D2, sm + L::OFF_W2, sb2, a);
         __syncthreads();
         // ---- output map: dwout, dbout over the tile's own times; delta2 = delta3 wout Swish'(y2) in place ----
-        if (tid >= 112 && tid <= 128) {
+        if (tid >= L::P3 && tid <= L::P4) {
             for (int t = 0; t < SB_TR; ++t) {
-                const float d3 = sm[SB_OFF_DZ + t];
-                small += tid == 128 ? d3 : d3 * sm[SB_OFF_H2 + t * SB_S2 + (tid - 112)];
+                const float d3 = sm[L::OFF_DZ + t];
+                small += tid == L::P4 ? d3 : d3 * sm[L::OFF_H2 + t * L::S2 + (tid - L::P3)];
             }
         }
         __syncthreads();
-        for (int e = tid; e < SB_R2 * SB_C3; e += SB_NT) {
-            const int r = e / SB_C3, c = e % SB_C3;
-            sm[SB_OFF_D2 + r * SB_S2 + c] *= sm[SB_OFF_DZ + r] * swo[c];
+        for (int e = tid; e < SB_R2 * L::C3; e += SB_NT) {
+            const int r = e / L::C3, c = e % L::C3;
+            sm[L::OFF_D2 + r * L::S2 + c] *= sm[L::OFF_DZ + r] * swo[c];
         }
         __syncthreads();
         // ---- layer 2: weight gradient (delta2 x h1), bias, then delta1 into the Swish' buffer of layer 1 (rows from a) ----
-        sb_wgrad<SB_C3, SB_C2, 1, SB_S2, SB_S1>(a2, sm + SB_OFF_D2, sm + SB_OFF_H1);
-        if (tid >= 96 && tid < 112)
-            for (int t = 0; t < SB_TR; ++t) small += sm[SB_OFF_D2 + t * SB_S2 + (tid - 96)];
-        sb_transposed<SB_C3, SB_C2, SB_TR + 8, SB_S2>(sm + SB_OFF_D2, sm + SB_OFF_W2,
-                                                      [&](int r, int c, float g) { sm[SB_OFF_D1 + (r + 4) * SB_S1 + c] *= g; });
+        sb_wgrad<L::C3, L::C2, L::CB2, L::S2, L::S1>(a2, sm + L::OFF_D2, sm + L::OFF_H1);
+        if (tid >= L::P2 && tid < L::P3)
+            for (int t = 0; t < SB_TR; ++t) small += sm[L::OFF_D2 + t * L::S2 + (tid - L::P2)];
+        sb_transposed<L::C3, L::C2, SB_TR + 8, L::S2>(sm + L::OFF_D2, sm + L::OFF_W2,
+                                                      [&](int r, int c, float g) { sm[L::OFF_D1 + (r + 4) * L::S1 + c] *= g; });
         __syncthreads();
         // ---- layer 1 ----
-        sb_wgrad<SB_C2, SB_C1, 2, SB_S1, SB_S0>(a1, sm + SB_OFF_D1 + 4 * SB_S1, sm + SB_OFF_H0 + 4 * SB_S0);
-        if (tid >= 64 && tid < 96)
-            for (int t = 0; t < SB_TR; ++t) small += sm[SB_OFF_D1 + (t + 4) * SB_S1 + (tid - 64)];
-        sb_transposed<SB_C2, SB_C1, SB_TR + 4, SB_S1>(sm + SB_OFF_D1 + 4 * SB_S1, sm + SB_OFF_W1,
-                                                      [&](int r, int c, float g) { sm[SB_OFF_D0 + (r + 8) * SB_S0 + c] *= g; });
+        sb_wgrad<L::C2, L::C1, L::CB1, L::S1, L::S0>(a1, sm + L::OFF_D1 + 4 * L::S1, sm + L::OFF_H0 + 4 * L::S0);
+        if (tid >= L::P1 && tid < L::P2)
+            for (int t = 0; t < SB_TR; ++t) small += sm[L::OFF_D1 + (t + 4) * L::S1 + (tid - L::P1)];
+        sb_transposed<L::C2, L::C1, SB_TR + 4, L::S1>(sm + L::OFF_D1 + 4 * L::S1, sm + L::OFF_W1,
+                                                      [&](int r, int c, float g) { sm[L::OFF_D0 + (r + 8) * L::S0 + c] *= g; });
         __syncthreads();
         // ---- layer 0 ----
-        sb_wgrad<SB_C1, SB_C0, 8, SB_S0, SB_SX>(a0, sm + SB_OFF_D0 + 8 * SB_S0, sm + SB_OFF_X + 8 * SB_SX);
-        if (tid < 64)
-            for (int t = 0; t < SB_TR; ++t) small += sm[SB_OFF_D0 + (t + 8) * SB_S0 + tid];
+        sb_wgrad<L::C1, L::C0, L::CB0, L::S0, L::SX>(a0, sm + L::OFF_D0 + 8 * L::S0, sm + L::OFF_X + 8 * L::SX);
+        if (tid < L::P1)
+            for (int t = 0; t < SB_TR; ++t) small += sm[L::OFF_D0 + (t + 8) * L::S0 + tid];
         if (input_grad) {
             // the gradient into the inputs: channels [0, 64) into dk, [64, 128) into dv, added to what the attention left there
-            sb_transposed<SB_C1, SB_C0, SB_TR, SB_S0>(sm + SB_OFF_D0 + 8 * SB_S0, sm + SB_OFF_W0, [&](int r, int c, float g) {
+            sb_transposed<L::C1, L::C0, SB_TR, L::S0>(sm + L::OFF_D0 + 8 * L::S0, sm + L::OFF_W0, [&](int r, int c, float g) {
                 const int t = a + r;
                 if (t < Tlen) {
                     T* dst = (c < D ? dk : dv) + ((size_t)bh * Tlen + t) * D + (c < D ? c : c - D);
@@ -299,65 +308,77 @@ stack_bwd_kernel(const T* __restrict__ k, const T* __restrict__ v, const float* 
             });
         }
     }
-    // ---- this CTA's partial sums, in the packed layout of the parameters ----
+    // ---- this CTA's partial sums, in the packed layout of the parameters (thread -> block as in sb_wgrad) ----
     {
-        const int cb = tid % 16, ob = tid / 16;                // layer 0: 16 blocks of 4 outputs x 16 blocks of 8 inputs
+        constexpr int NCB = L::C0 / L::CB0;                    // layer 0: blocks of 4 outputs x CB0 inputs
+        if (tid < (L::C1 / 4) * NCB) {
+            const int cb = tid % NCB, ob = tid / NCB;
 #pragma unroll
-        for (int tau = 0; tau < 3; ++tau)
+            for (int tau = 0; tau < 3; ++tau)
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
+                for (int j = 0; j < 4; ++j)
 #pragma unroll
-                for (int cc = 0; cc < 8; ++cc) my_part[((4 * ob + j) * 3 + tau) * SB_C0 + cb * 8 + cc] = a0[tau][j][cc];
+                    for (int cc = 0; cc < L::CB0; ++cc) my_part[((4 * ob + j) * 3 + tau) * L::C0 + cb * L::CB0 + cc] = a0[tau][j][cc];
+        }
     }
     {
-        const int cb = tid % 32, ob = tid / 32;                // layer 1: 8 x 32 blocks of 4 x 2
+        constexpr int NCB = L::C1 / L::CB1;                    // layer 1
+        if (tid < (L::C2 / 4) * NCB) {
+            const int cb = tid % NCB, ob = tid / NCB;
 #pragma unroll
-        for (int tau = 0; tau < 3; ++tau)
+            for (int tau = 0; tau < 3; ++tau)
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
+                for (int j = 0; j < 4; ++j)
 #pragma unroll
-                for (int cc = 0; cc < 2; ++cc) my_part[SB_G0 + ((4 * ob + j) * 3 + tau) * SB_C1 + cb * 2 + cc] = a1[tau][j][cc];
-    }
-    if (tid < 128) {
-        const int cb = tid % 32, ob = tid / 32;                // layer 2: 4 x 32 blocks of 4 x 1
-#pragma unroll
-        for (int tau = 0; tau < 3; ++tau)
-#pragma unroll
-            for (int j = 0; j < 4; ++j) my_part[SB_G0 + SB_G1 + ((4 * ob + j) * 3 + tau) * SB_C2 + cb] = a2[tau][j][0];
+                    for (int cc = 0; cc < L::CB1; ++cc) my_part[L::G0 + ((4 * ob + j) * 3 + tau) * L::C1 + cb * L::CB1 + cc] = a1[tau][j][cc];
+        }
     }
     {
-        // wout [16] | b0 [64] | b1 [32] | b2 [16] | bout
-        float* sp = my_part + SB_G0 + SB_G1 + SB_G2;
-        if (tid < 64) sp[16 + tid] = small;
-        else if (tid < 96) sp[16 + 64 + (tid - 64)] = small;
-        else if (tid < 112) sp[16 + 96 + (tid - 96)] = small;
-        else if (tid < 128) sp[tid - 112] = small;
-        else if (tid == 128) sp[16 + 112] = small;
+        constexpr int NCB = L::C2 / L::CB2;                    // layer 2
+        if (tid < (L::C3 / 4) * NCB) {
+            const int cb = tid % NCB, ob = tid / NCB;
+#pragma unroll
+            for (int tau = 0; tau < 3; ++tau)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) my_part[L::G0 + L::G1 + ((4 * ob + j) * 3 + tau) * L::C2 + cb] = a2[tau][j][0];
+        }
+    }
+    {
+        // wout [C3] | b0 [C1] | b1 [C2] | b2 [C3] | bout
+        float* sp = my_part + L::G0 + L::G1 + L::G2;
+        if (tid < L::P1) sp[L::C3 + tid] = small;
+        else if (tid < L::P2) sp[L::C3 + L::C1 + (tid - L::P1)] = small;
+        else if (tid < L::P3) sp[L::C3 + L::C1 + L::C2 + (tid - L::P2)] = small;
+        else if (tid < L::P4) sp[tid - L::P3] = small;
+        else if (tid == L::P4) sp[L::C3 + L::C1 + L::C2 + L::C3] = small;
     }
 }
 
 // dw = wl0 | wl1 | wl2 | wout (every tensor over all heads), dbias = bl0 | bl1 | bl2 | bout: sums of the partials of a head's
 // CTAs (all batch elements, all row chunks) in a fixed order.
+template <int D>
 __global__ void stack_bwd_reduce_kernel(const float* __restrict__ part, float* __restrict__ dw, float* __restrict__ dbias,
                                         int B, int H, int chunks)
 {
+    using L = SBL<D>;
     pdl_launch_dependents();
     pdl_wait();
     const int h = blockIdx.y, e = blockIdx.x * blockDim.x + threadIdx.x;
-    if (e >= SB_PART) return;
+    if (e >= L::PART) return;
     float t = 0.f;
     for (int b = 0; b < B; ++b)
-        for (int ch = 0; ch < chunks; ++ch) t += part[(((size_t)b * H + h) * chunks + ch) * SB_PART_PAD + e];
-    if (e < SB_G0) dw[(size_t)h * SB_G0 + e] = t;
-    else if (e < SB_G0 + SB_G1) dw[(size_t)H * SB_G0 + (size_t)h * SB_G1 + (e - SB_G0)] = t;
-    else if (e < SB_G0 + SB_G1 + SB_G2) dw[(size_t)H * (SB_G0 + SB_G1) + (size_t)h * SB_G2 + (e - SB_G0 - SB_G1)] = t;
-    else if (e < SB_G0 + SB_G1 + SB_G2 + 16) dw[(size_t)H * (SB_G0 + SB_G1 + SB_G2) + (size_t)h * 16 + (e - SB_G0 - SB_G1 - SB_G2)] = t;
+        for (int ch = 0; ch < chunks; ++ch) t += part[(((size_t)b * H + h) * chunks + ch) * L::PART_PAD + e];
+    constexpr int GW = L::G0 + L::G1 + L::G2;
+    if (e < L::G0) dw[(size_t)h * L::G0 + e] = t;
+    else if (e < L::G0 + L::G1) dw[(size_t)H * L::G0 + (size_t)h * L::G1 + (e - L::G0)] = t;
+    else if (e < GW) dw[(size_t)H * (L::G0 + L::G1) + (size_t)h * L::G2 + (e - L::G0 - L::G1)] = t;
+    else if (e < GW + L::C3) dw[(size_t)H * GW + (size_t)h * L::C3 + (e - GW)] = t;
     else if (dbias) {
-        const int f = e - (SB_G0 + SB_G1 + SB_G2 + 16);        // b0 [64] | b1 [32] | b2 [16] | bout
-        if (f < 64) dbias[(size_t)h * 64 + f] = t;
-        else if (f < 96) dbias[(size_t)H * 64 + (size_t)h * 32 + (f - 64)] = t;
-        else if (f < 112) dbias[(size_t)H * 96 + (size_t)h * 16 + (f - 96)] = t;
-        else dbias[(size_t)H * 112 + h] = t;
+        const int f = e - (GW + L::C3);                        // b0 [C1] | b1 [C2] | b2 [C3] | bout
+        if (f < L::P1) dbias[(size_t)h * L::C1 + f] = t;
+        else if (f < L::P2) dbias[(size_t)H * L::C1 + (size_t)h * L::C2 + (f - L::P1)] = t;
+        else if (f < L::P3) dbias[(size_t)H * (L::C1 + L::C2) + (size_t)h * L::C3 + (f - L::P2)] = t;
+        else dbias[(size_t)H * (L::C1 + L::C2 + L::C3) + h] = t;
     }
 }
 
@@ -378,38 +399,46 @@ int stack_bwd_chunks(const Params& p)
 // Scratch of the stack's backward: one packed partial gradient per CTA.
 size_t stack_bwd_workspace(const Params& p)
 {
-    if (p.d != 64) return 0;
-    return (size_t)p.B * p.H * stack_bwd_chunks(p) * SB_PART_PAD * sizeof(float);
+    if (p.d != 64 && p.d != 32) return 0;
+    const int pad = p.d == 64 ? SBL<64>::PART_PAD : SBL<32>::PART_PAD;
+    return (size_t)p.B * p.H * stack_bwd_chunks(p) * pad * sizeof(float);
 }
+
+namespace {
+template <typename T, int D>
+int run_stack_bwd(const Params& p, const void* k, const void* v, const float* dz, void* dk, void* dv, float* dw, float* dbias,
+                  bool input_grad, void* part, cudaStream_t st)
+{
+    using L = SBL<D>;
+    const int chunks = stack_bwd_chunks(p);
+    const int n_tiles = (p.T + SB_TR - 1) / SB_TR, per = (n_tiles + chunks - 1) / chunks;
+    dim3 grid(chunks, p.B * p.H);
+    static PerDeviceOnce attr;
+    if (int e2 = attr.run([] { return cudaFuncSetAttribute(stack_bwd_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L::BYTES); }))
+        return e2;
+    if (launch_pdl(stack_bwd_kernel<T, D>, grid, dim3(SB_NT), L::BYTES, st, (const T*)k, (const T*)v, p.w, p.bias, dz, (T*)dk, (T*)dv,
+                   (float*)part, p.H, p.T, per, input_grad ? 1 : 0) != cudaSuccess)
+        return LTE_ERR_CUDA;
+    if (launch_pdl(stack_bwd_reduce_kernel<D>, dim3((L::PART + 255) / 256, p.H), dim3(256), 0, st, (const float*)part, dw, dbias, p.B,
+                   p.H, chunks) != cudaSuccess)
+        return LTE_ERR_CUDA;
+    return cuda_status(cudaGetLastError());
+}
+}  // namespace
 
 // dz [B,H,T] fp32 (zero where the logit is undefined) -> dw, dbias (packed like the parameters; dbias may be null) and,
 // with input_grad, dk += , dv += the gradient into the scorer's inputs.  part: stack_bwd_workspace(p) bytes.
 int launch_stack_bwd(const Params& p, const void* k, const void* v, const float* dz, void* dk, void* dv, float* dw,
                      float* dbias, bool input_grad, void* part, cudaStream_t st)
 {
-    if (p.d != 64) return LTE_ERR_UNSUPPORTED;
-    const int chunks = stack_bwd_chunks(p);
-    const int n_tiles = (p.T + SB_TR - 1) / SB_TR, per = (n_tiles + chunks - 1) / chunks;
-    dim3 grid(chunks, p.B * p.H);
-    cudaError_t e;
-    if (p.dtype == LTE_BF16) {
-        static PerDeviceOnce attr;
-        if (int e2 = attr.run([] { return cudaFuncSetAttribute(stack_bwd_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SB_BYTES); }))
-            return e2;
-        e = launch_pdl(stack_bwd_kernel<__nv_bfloat16>, grid, dim3(SB_NT), SB_BYTES, st, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v,
-                       p.w, p.bias, dz, (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, (float*)part, p.H, p.T, per, input_grad ? 1 : 0);
-    } else {
-        static PerDeviceOnce attr;
-        if (int e2 = attr.run([] { return cudaFuncSetAttribute(stack_bwd_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SB_BYTES); }))
-            return e2;
-        e = launch_pdl(stack_bwd_kernel<float>, grid, dim3(SB_NT), SB_BYTES, st, (const float*)k, (const float*)v, p.w, p.bias, dz,
-                       (float*)dk, (float*)dv, (float*)part, p.H, p.T, per, input_grad ? 1 : 0);
-    }
-    if (e != cudaSuccess) return LTE_ERR_CUDA;
-    if (launch_pdl(stack_bwd_reduce_kernel, dim3((SB_PART + 255) / 256, p.H), dim3(256), 0, st, (const float*)part, dw, dbias, p.B,
-                   p.H, chunks) != cudaSuccess)
-        return LTE_ERR_CUDA;
-    return cuda_status(cudaGetLastError());
+    const bool bf = p.dtype == LTE_BF16;
+    if (p.d == 64)
+        return bf ? run_stack_bwd<__nv_bfloat16, 64>(p, k, v, dz, dk, dv, dw, dbias, input_grad, part, st)
+                  : run_stack_bwd<float, 64>(p, k, v, dz, dk, dv, dw, dbias, input_grad, part, st);
+    if (p.d == 32)
+        return bf ? run_stack_bwd<__nv_bfloat16, 32>(p, k, v, dz, dk, dv, dw, dbias, input_grad, part, st)
+                  : run_stack_bwd<float, 32>(p, k, v, dz, dk, dv, dw, dbias, input_grad, part, st);
+    return LTE_ERR_UNSUPPORTED;
 }
 
 }  // namespace lte

@@ -232,13 +232,15 @@ def _rel(a, b):
     return float(np.linalg.norm(np.asarray(a, np.float64) - b) / (np.linalg.norm(b) + 1e-30))
 
 
-@pytest.mark.parametrize("dtype,T,W,R,bias,in_grad,B,H", [("bf16", 200, 16, 12, True, True, 2, 2), ("bf16", 333, 24, 40, False, True, 2, 2),
-                                                          ("f32", 150, 16, 10, True, True, 2, 2), ("bf16", 260, 32, 16, True, False, 2, 2),
-                                                          ("bf16", 2048, 64, 64, True, True, 5, 8), ("bf16", 700, 64, 32, True, True, 40, 8)])
-def test_stack_backward(dtype, T, W, R, bias, in_grad, B, H):
+@pytest.mark.parametrize("dtype,T,W,R,bias,in_grad,B,H,d", [("bf16", 200, 16, 12, True, True, 2, 2, 64), ("bf16", 333, 24, 40, False, True, 2, 2, 64),
+                                                            ("f32", 150, 16, 10, True, True, 2, 2, 64), ("bf16", 260, 32, 16, True, False, 2, 2, 64),
+                                                            ("bf16", 2048, 64, 64, True, True, 5, 8, 64), ("bf16", 700, 64, 32, True, True, 40, 8, 64),
+                                                            ("f32", 150, 16, 10, True, True, 2, 2, 32), ("bf16", 333, 24, 40, True, True, 2, 3, 32),
+                                                            ("f32", 700, 32, 16, False, False, 3, 2, 32)])
+def test_stack_backward(dtype, T, W, R, bias, in_grad, B, H, d):
     """dq, dk, dv and the gradients of every parameter of the stack against the oracle: the attention backward and the
-    straight-through surrogate give dz, the stack's backward (pinned by finite differences on the CPU) the rest."""
-    d = 64
+    straight-through surrogate give dz, the stack's backward (pinned by finite differences on the CPU) the rest.  d = 32 takes
+    the fp32 kernels for the attention part and for the stack."""
     cfg = synth.Config("stackbwd", dtype, B, H, d, T, W, R, 7, 0.1)   # the last two: several tiles per thread block
     x = synth.make(cfg, 8, with_dO=True)
     wl, wout, bl, bout = _stack_params(cfg.H, d, 8, bias)
