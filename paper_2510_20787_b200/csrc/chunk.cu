@@ -198,34 +198,52 @@ __global__ void __launch_bounds__(32) chunk_stream_kernel(const float* __restric
     int n_u = n_pool;
     __syncwarp();
     const int Tc = Tloc - R0 - Wn;
-    for (int t = 0; t < Tc; ++t) {
-        const int rq = R0 + Wn + t, r = rq - W;                // the query's row; the row it pushes out of its window
-        if (r < R0 || R <= 0) continue;
-        const float zc = zr[r];
-        if (!(zc > zthr)) continue;
-        const int pos = n0 - Wn + (r - R0);
-        if (n_pool < R) {
-            if (lane == 0) { pz[n_pool] = zc; ppos[n_pool] = pos; pu[n_pool] = n_u; ul[n_u] = r; lv[n_u] = 0x7fffffff; }
-            ++n_pool; ++n_u;
-        } else {
-            // the lowest logit; among equals the youngest
-            float wz = INFINITY; int wp = -1, wi = -1;
-            for (int e = lane; e < R; e += 32) {
-                const float ze = pz[e]; const int pe = ppos[e];
-                if (ze < wz || (ze == wz && pe > wp)) { wz = ze; wp = pe; wi = e; }
-            }
+    // The lowest entry of a full pool only ever rises (a replacement puts a higher logit in its place), so a token at or
+    // below it can be dropped without looking at the pool again: the lowest entry is searched once after every
+    // replacement, and 32 tokens at a time are tested against it with one ballot.
+    bool worst_known = false;
+    float wz = INFINITY; int wp = -1, wi = -1;
+    auto find_worst = [&]() {                                  // the lowest logit; among equals the youngest
+        wz = INFINITY; wp = -1; wi = -1;
+        for (int e = lane; e < R; e += 32) {
+            const float ze = pz[e]; const int pe = ppos[e];
+            if (ze < wz || (ze == wz && pe > wp)) { wz = ze; wp = pe; wi = e; }
+        }
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                const float oz = __shfl_xor_sync(0xffffffffu, wz, o);
-                const int opp = __shfl_xor_sync(0xffffffffu, wp, o), oi = __shfl_xor_sync(0xffffffffu, wi, o);
-                if (oz < wz || (oz == wz && opp > wp)) { wz = oz; wp = opp; wi = oi; }
+        for (int o = 16; o > 0; o >>= 1) {
+            const float oz = __shfl_xor_sync(0xffffffffu, wz, o);
+            const int opp = __shfl_xor_sync(0xffffffffu, wp, o), oi = __shfl_xor_sync(0xffffffffu, wi, o);
+            if (oz < wz || (oz == wz && opp > wp)) { wz = oz; wp = opp; wi = oi; }
+        }
+        worst_known = true;
+    };
+    for (int t0 = 0; t0 < Tc && R > 0; t0 += 32) {
+        // lane l: the token that query t0 + l pushes out of its window (local row rq - W), if it passes the threshold
+        const int my_rq = R0 + Wn + t0 + lane, my_r = my_rq - W;
+        const float my_z = (t0 + lane < Tc && my_r >= R0) ? zr[my_r] : -INFINITY;
+        unsigned todo = __ballot_sync(0xffffffffu, my_z > zthr);
+        if (worst_known) todo &= __ballot_sync(0xffffffffu, my_z > wz);
+        while (todo != 0u) {
+            const int l = __ffs(todo) - 1;
+            todo &= todo - 1u;
+            const float zc = __shfl_sync(0xffffffffu, my_z, l);
+            const int rq = R0 + Wn + t0 + l, r = rq - W;
+            const int pos = n0 - Wn + (r - R0);
+            if (n_pool < R) {
+                if (lane == 0) { pz[n_pool] = zc; ppos[n_pool] = pos; pu[n_pool] = n_u; ul[n_u] = r; lv[n_u] = 0x7fffffff; }
+                ++n_pool; ++n_u;
+                __syncwarp();
+                continue;
             }
+            if (!worst_known) find_worst();
             if (wi >= 0 && zc > wz) {                            // strictly better: the entry is gone from this query on
                 if (lane == 0) { lv[pu[wi]] = rq; pz[wi] = zc; ppos[wi] = pos; pu[wi] = n_u; ul[n_u] = r; lv[n_u] = 0x7fffffff; }
                 ++n_u;
+                __syncwarp();
+                find_worst();
             }
+            todo &= __ballot_sync(0xffffffffu, my_z > wz);      // the later tokens of the batch against the new lowest entry
         }
-        __syncwarp();
     }
     __syncwarp();
     // the survivors, in list order (ascending local rows), are the new pool

@@ -8,7 +8,8 @@
 namespace lte {
 
 int launch_prefill_tc(const Params& p, const void* q, const void* k, const void* v, const int32_t* idx,
-                      const int32_t* cnt, void* o, float* lse, void* ws, size_t ws_bytes, cudaStream_t st);
+                      const int32_t* cnt, void* o, float* lse, void* ws, size_t ws_bytes, cudaStream_t st,
+                      const int32_t* leave = nullptr);
 int prefill_status_fetch_and_clear();
 int decode_status_fetch_and_clear();
 int scores_status_fetch_and_clear();
@@ -141,8 +142,12 @@ ChunkPlan chunk_plan(const lte_shape* s, const lte_conv* c, bool streaming = fal
         lte_shape s2 = *s; s2.T = (int32_t)Tm;
         off += up(scores_stack_tc_workspace(make_params(&s2, c)));
     }
-    w.att = off;                                             // the attention's compacted retained rows
-    off += up(prefill_compact_bytes(make_params(s, c)));
+    w.att = off;                                             // the attention's compacted retained rows (streaming: of the entry list)
+    {
+        Params pa = make_params(s, c);
+        if (streaming) pa.R = w.ucap;
+        off += up(prefill_compact_bytes(pa));
+    }
     w.total = off;
     return w;
 }
@@ -385,7 +390,9 @@ int lte_attn_prefill_chunk_ex(const lte_shape* s, const lte_conv* c, void* cache
         int32_t* ulist = (int32_t*)(base + w.ulist); int32_t* leave = (int32_t*)(base + w.leave); int32_t* ucnt = (int32_t*)(base + w.ucnt);
         e = launch_chunk_stream(psel, zrank, oldpos, ulist, leave, ucnt, idx, cnt, w.ucap, n_past, R0, Wn, st); if (e) return e;
         Params pu = patt; pu.R = w.ucap;                      // the entry list's row length
-        e = launch_prefill_simt(pu, q, base + w.klin, base + w.vlin, ulist, ucnt, o, lse, st, leave);
+        // bf16: the tiled kernel with the leave times as one more mask on its retained tiles (d = 64), else row by row
+        if (s->dtype == LTE_BF16) e = launch_prefill_tc(pu, q, base + w.klin, base + w.vlin, ulist, ucnt, o, lse, base + w.att, w.total - w.att, st, leave);
+        else e = launch_prefill_simt(pu, q, base + w.klin, base + w.vlin, ulist, ucnt, o, lse, st, leave);
     } else {
         e = launch_select(psel, zrank, idx, cnt, nullptr, st); if (e) return e;
         // the attention kernels take the chunk's q, o, lse as they are: query row r stands at position qoff + r

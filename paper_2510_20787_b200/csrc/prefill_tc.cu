@@ -61,7 +61,8 @@ template <int D> struct Smem {
     static constexpr bool ONES = D == 64;
     static constexpr int OFF_ONES = OFF_V + VST * KVTILE;     // [64][64] bf16 ones (8 KB), d = 64 only
     static constexpr int OFF_BAR = OFF_ONES + (ONES ? BN * 128 : 0);   // mbarriers, tmem slot
-    static constexpr int BYTES = OFF_BAR + 256;
+    static constexpr int OFF_LV = OFF_BAR + 256;              // STREAM: the leave times of a retained tile, [4 warps][64]
+    static constexpr int BYTES = OFF_LV + 4 * 64 * 4;
     static constexpr uint32_t TMEM_COLS = 256;                // S0: [0,64)  S1: [64,128)  O: [128, 128+D) (+16 row-sum columns)
 };
 
@@ -114,14 +115,16 @@ __device__ __forceinline__ int count_le(const int32_t* id, int n, int lim, int l
 // COMPACT: the retained rows were copied into contiguous tensors [B*H][R][d] beforehand (tmKc, tmVc), so retained tiles are
 // TMA boxes like the window tiles and the softmax warps gather nothing (a compile-time variant: the gather code costs the
 // softmax loop instruction-cache room even where it does not run).
-template <int D, bool COMPACT>
+// STREAM (with COMPACT): the list is every entry that is retained at some query of a chunk, and entry e is gone from query
+// leave[e] on (the streaming reading of a chunk): retained tiles take one more mask, leave > query position.
+template <int D, bool COMPACT, bool STREAM>
 __global__ void __launch_bounds__(NTHREADS, 2)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                   const __grid_constant__ CUtensorMap tmV,
                   const __grid_constant__ CUtensorMap tmKc, const __grid_constant__ CUtensorMap tmVc,
                   const __nv_bfloat16* __restrict__ kg,
                   const __nv_bfloat16* __restrict__ vg, __nv_bfloat16* __restrict__ og, const int32_t* __restrict__ idx,
-                  const int32_t* __restrict__ cnt, float* __restrict__ lse, int Tlen,
+                  const int32_t* __restrict__ cnt, const int32_t* __restrict__ leave, float* __restrict__ lse, int Tlen,
                   int W, int R, float scale, int n_qt, int n_bh, int G, int qoff)
 {
     const int n_items = n_qt * n_bh;
@@ -449,6 +452,29 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     const uint32_t below_a = a >= 32 ? 0xffffffffu : ((1u << a) - 1u);
                     vm[cb] = b2 > a ? (below_b & ~below_a) : 0u;
                 }
+                if (STREAM && t >= n_win) {
+                    // the tile's 64 leave times go through a per-warp scratch (two coalesced loads), then every row tests
+                    // them against its own position; the chunks take the masked path
+                    int* slv = reinterpret_cast<int*>(smem_raw + S::OFF_LV) + warp * 64;
+                    const int e0 = (t - n_win) * BN;
+                    const int32_t* lvp = leave + (size_t)bhk * R;
+                    __syncwarp();                              // the previous tile's readers are done
+                    slv[lane] = e0 + lane < R ? lvp[e0 + lane] : 0;
+                    slv[32 + lane] = e0 + 32 + lane < R ? lvp[e0 + 32 + lane] : 0;
+                    __syncwarp();
+#pragma unroll
+                    for (int cb = 0; cb < 2; ++cb) {
+                        uint32_t m = 0;
+#pragma unroll
+                        for (int c = 0; c < 32; c += 4) {
+                            const int4 l4 = *reinterpret_cast<const int4*>(&slv[cb * 32 + c]);
+                            m |= (l4.x > i ? 1u : 0u) << c; m |= (l4.y > i ? 2u : 0u) << c;
+                            m |= (l4.z > i ? 4u : 0u) << c; m |= (l4.w > i ? 8u : 0u) << c;
+                        }
+                        vm[cb] &= m;
+                        full[cb] = false;
+                    }
+                }
                 PP(1);
                 mbar_wait(bar_s0 + 8 * (gg & 1), (gg >> 1) & 1, 3);   // S is in TMEM buffer gg & 1
                 tc_fence_after();
@@ -597,7 +623,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 
 template <int D>
 int run(const Params& p, const void* q, const void* k, const void* v, const int32_t* idx, const int32_t* cnt, void* o,
-        float* lse, void* ws, size_t ws_bytes, cudaStream_t st)
+        float* lse, void* ws, size_t ws_bytes, cudaStream_t st, const int32_t* leave)
 {
     CUtensorMap tq, tk, tv, tkc, tvc;
     const int BHK = p.B * p.H, BH = BHK * p.G;                 // key/value heads, query heads
@@ -614,33 +640,44 @@ int run(const Params& p, const void* q, const void* k, const void* v, const int3
     }
     static PerDeviceOnce attr;
     if (int e = attr.run([] {
-            const cudaError_t a = cudaFuncSetAttribute(prefill_tc_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::BYTES);
-            return a != cudaSuccess ? a : cudaFuncSetAttribute(prefill_tc_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::BYTES);
+            cudaError_t a = cudaFuncSetAttribute(prefill_tc_kernel<D, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::BYTES);
+            if (a == cudaSuccess) a = cudaFuncSetAttribute(prefill_tc_kernel<D, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::BYTES);
+            return a != cudaSuccess ? a : cudaFuncSetAttribute(prefill_tc_kernel<D, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::BYTES);
         })) return e;
     int sms = 0;
     if (int e = device_sm_count(&sms)) return e;
     const int slots = 2 * sms;                                 // resident CTAs: two per SM
     const int n_qt = (Tq + BM - 1) / BM, n_items = n_qt * BH;
     const int grid = n_items < slots ? n_items : slots;
+    if (leave != nullptr) {
+        if (!compact) return LTE_ERR_UNSUPPORTED;             // the streaming variant takes compacted rows only
+        return cuda_status(launch_pdl(prefill_tc_kernel<D, true, true>, dim3(grid), dim3(NTHREADS), Smem<D>::BYTES, st, tq, tk, tv, tkc, tvc,
+                                      (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (__nv_bfloat16*)o, idx, cnt, leave, lse, p.T, p.W, p.R,
+                                      p.scale, n_qt, BH, p.G, p.qoff));
+    }
     if (compact)
-        return cuda_status(launch_pdl(prefill_tc_kernel<D, true>, dim3(grid), dim3(NTHREADS), Smem<D>::BYTES, st, tq, tk, tv, tkc, tvc,
-                                      (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (__nv_bfloat16*)o, idx, cnt, lse, p.T, p.W, p.R, p.scale, n_qt,
-                                      BH, p.G, p.qoff));
-    return cuda_status(launch_pdl(prefill_tc_kernel<D, false>, dim3(grid), dim3(NTHREADS), Smem<D>::BYTES, st, tq, tk, tv, tkc, tvc,
-                                  (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (__nv_bfloat16*)o, idx, cnt, lse, p.T, p.W, p.R, p.scale, n_qt, BH,
-                                  p.G, p.qoff));
+        return cuda_status(launch_pdl(prefill_tc_kernel<D, true, false>, dim3(grid), dim3(NTHREADS), Smem<D>::BYTES, st, tq, tk, tv, tkc, tvc,
+                                      (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (__nv_bfloat16*)o, idx, cnt, leave, lse, p.T, p.W, p.R,
+                                      p.scale, n_qt, BH, p.G, p.qoff));
+    return cuda_status(launch_pdl(prefill_tc_kernel<D, false, false>, dim3(grid), dim3(NTHREADS), Smem<D>::BYTES, st, tq, tk, tv, tkc, tvc,
+                                  (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (__nv_bfloat16*)o, idx, cnt, leave, lse, p.T, p.W, p.R,
+                                  p.scale, n_qt, BH, p.G, p.qoff));
 }
 
 }  // namespace
 
+// leave: null, or the streaming reading's per-entry leave times (d = 64 with a workspace: the tiled kernel; otherwise the
+// row-by-row kernel)
 int launch_prefill_tc(const Params& p, const void* q, const void* k, const void* v, const int32_t* idx,
-                      const int32_t* cnt, void* o, float* lse, void* ws, size_t ws_bytes, cudaStream_t st)
+                      const int32_t* cnt, void* o, float* lse, void* ws, size_t ws_bytes, cudaStream_t st, const int32_t* leave)
 {
-    switch (p.d) {
-        case 64: return run<64>(p, q, k, v, idx, cnt, o, lse, ws, ws_bytes, st);
-        // d = 128: ten and more key tiles per item; one CTA per item under the hardware scheduler is faster there
-        case 128: return launch_prefill_tc_long(p, q, k, v, idx, cnt, o, lse, ws, ws_bytes, st);
+    if (p.d == 64) {
+        const int e = run<64>(p, q, k, v, idx, cnt, o, lse, ws, ws_bytes, st, leave);
+        if (e != LTE_ERR_UNSUPPORTED || leave == nullptr) return e;
     }
+    if (leave != nullptr) return launch_prefill_simt(p, q, k, v, idx, cnt, o, lse, st, leave);
+    // d = 128: ten and more key tiles per item; one CTA per item under the hardware scheduler is faster there
+    if (p.d == 128) return launch_prefill_tc_long(p, q, k, v, idx, cnt, o, lse, ws, ws_bytes, st);
     return launch_prefill_simt(p, q, k, v, idx, cnt, o, lse, st);   // d = 32: rows too narrow for the 128-byte swizzle
 }
 

@@ -135,6 +135,16 @@ def test_serving_shape_chunk_on_a_big_cache():
     _compare(_cfg(B=1, H=2, W=768, R=512, sink=4), [("prefill", 2000), ("chunk", 512), ("decode", 4)], seed=2)
 
 
+@pytest.mark.parametrize("kw,plan", [
+    (dict(B=1, H=2, W=768, R=512, sink=4), [("prefill", 2000), ("chunk", 512), ("decode", 4)]),   # the benchmark's serving-like chunk
+    (dict(B=1, H=2, W=128, R=128), [("prefill", 1500), ("chunk", 1200)]),                          # the C2 window and budget: several retained tiles
+])
+def test_streaming_reading_at_the_benchmark_shapes(kw, plan):
+    """The streaming reading on the tiled tensor-core kernel (bf16, d = 64): retained tiles of the entry list with the leave
+    times as one more mask; equal to token-by-token decoding."""
+    _compare(_cfg(**kw), plan, seed=2, streaming=True)
+
+
 def test_wrong_token_count_is_reported_and_leaves_the_cache_alone():
     cfg = _cfg(B=1, H=2)
     x = synth.make(cfg, 0, T=120)
