@@ -291,9 +291,9 @@ int lte_attn_prefill_chunk(const lte_shape* s, const lte_conv* c, void* cache, i
  * lte_attn_decode compute, also where the cap R binds: an entry that a later token of the same chunk pushes out is still
  * seen by the queries before that token's.  The cache afterwards is the same under both readings.
  * The pool is walked token by token (one warp per head), which gives every entry that is retained at some query of the
- * chunk and the query from which it is gone.  bf16 with d = 64: the tiled tensor-core kernel attends over that entry list
- * with the leave times as one more mask on its retained tiles (about twice the time of the chunk-end reading); other
- * shapes and dtypes: row by row on the fp32 ALUs (exact as well, but tens of times slower).
+ * chunk and the query from which it is gone.  bf16 with d = 64 or 128: the tiled tensor-core kernels attend over that entry
+ * list with the leave times as one more mask on their retained tiles (about twice the time of the chunk-end reading);
+ * fp32 and d = 32: row by row on the fp32 ALUs (exact as well, but tens of times slower).
  *   ws   device scratch of lte_workspace_bytes(LTE_OP_CHUNK_STREAM, s, c) bytes, 256-byte aligned
  * Errors: as lte_attn_prefill_chunk; INVALID_ARG for unknown flags; UNSUPPORTED for R > 4096 with the flag.
  */

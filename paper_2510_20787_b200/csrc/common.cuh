@@ -105,7 +105,8 @@ int launch_prefill_simt(const Params& p, const void* q, const void* k, const voi
 int launch_chunk_stream(const Params& p, const float* zrank, const int32_t* oldpos, int32_t* ulist, int32_t* leave, int32_t* ucnt,
                         int32_t* idx, int32_t* cnt, int ucap, int n0, int R0, int Wn, cudaStream_t st);
 int launch_prefill_tc_long(const Params& p, const void* q, const void* k, const void* v, const int32_t* idx,
-                           const int32_t* cnt, void* o, float* lse, void* ws, size_t ws_bytes, cudaStream_t st);
+                           const int32_t* cnt, void* o, float* lse, void* ws, size_t ws_bytes, cudaStream_t st,
+                           const int32_t* leave = nullptr);
 size_t prefill_compact_bytes(const Params& p);
 int launch_prefill_compact(const Params& p, const void* k, const void* v, const int32_t* idx, const int32_t* cnt, void* kc, void* vc,
                            cudaStream_t st);

@@ -666,8 +666,8 @@ int run(const Params& p, const void* q, const void* k, const void* v, const int3
 
 }  // namespace
 
-// leave: null, or the streaming reading's per-entry leave times (d = 64 with a workspace: the tiled kernel; otherwise the
-// row-by-row kernel)
+// leave: null, or the streaming reading's per-entry leave times (d = 64 or 128 with a workspace: the tiled kernels; otherwise
+// the row-by-row kernel)
 int launch_prefill_tc(const Params& p, const void* q, const void* k, const void* v, const int32_t* idx,
                       const int32_t* cnt, void* o, float* lse, void* ws, size_t ws_bytes, cudaStream_t st, const int32_t* leave)
 {
@@ -675,7 +675,13 @@ int launch_prefill_tc(const Params& p, const void* q, const void* k, const void*
         const int e = run<64>(p, q, k, v, idx, cnt, o, lse, ws, ws_bytes, st, leave);
         if (e != LTE_ERR_UNSUPPORTED || leave == nullptr) return e;
     }
-    if (leave != nullptr) return launch_prefill_simt(p, q, k, v, idx, cnt, o, lse, st, leave);
+    if (leave != nullptr) {
+        if (p.d == 128) {
+            const int e = launch_prefill_tc_long(p, q, k, v, idx, cnt, o, lse, ws, ws_bytes, st, leave);
+            if (e != LTE_ERR_UNSUPPORTED) return e;
+        }
+        return launch_prefill_simt(p, q, k, v, idx, cnt, o, lse, st, leave);
+    }
     // d = 128: ten and more key tiles per item; one CTA per item under the hardware scheduler is faster there
     if (p.d == 128) return launch_prefill_tc_long(p, q, k, v, idx, cnt, o, lse, ws, ws_bytes, st);
     return launch_prefill_simt(p, q, k, v, idx, cnt, o, lse, st);   // d = 32: rows too narrow for the 128-byte swizzle

@@ -72,15 +72,17 @@ template <int D> struct Smem {
 //   bar_k[s], bar_v[s]       TMA transaction barriers of the window tiles
 //   bar_kf[s], bar_vf[s]     (commit) the MMA that read stage s has completed          MMA lane -> load lane
 // S(t+1) and S(t+2) are computed while the softmax of tile t runs; loads run two to three tiles ahead.
-template <int D, bool compact>
+// STREAM (with compact): the list is every entry retained at some query of a chunk and entry e is gone from query leave[e] on
+// (the streaming reading of a chunk): retained tiles take one more mask, leave > query position.
+template <int D, bool compact, bool STREAM>
 __global__ void __launch_bounds__(NTHREADS, 2)
 prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                   const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
                   const __grid_constant__ CUtensorMap tmKc, const __grid_constant__ CUtensorMap tmVc,
                   const __nv_bfloat16* __restrict__ kg,
                   const __nv_bfloat16* __restrict__ vg, const int32_t* __restrict__ idx,
-                  const int32_t* __restrict__ cnt, __nv_bfloat16* __restrict__ o, float* __restrict__ lse, int Tlen,
-                  int W, int R, float scale, int G, int qoff)
+                  const int32_t* __restrict__ cnt, const int32_t* __restrict__ leave, __nv_bfloat16* __restrict__ o,
+                  float* __restrict__ lse, int Tlen, int W, int R, float scale, int G, int qoff)
 {
     using S = Smem<D>;
     constexpr int SUB = S::SUB, KST = S::KST, VST = S::VST;
@@ -399,6 +401,21 @@ prefill_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     vm[cb] = b2 > a ? (below_b & ~below_a) : 0u;
                 }
             }
+            if (STREAM && t >= n_win) {
+                // the tile's 64 leave times, two per lane, are passed round the warp and tested against this row's position
+                // (shared memory has no room for a scratch at two CTAs per SM); the chunks take the masked path
+                const int e0 = (t - n_win) * BN;
+                const int32_t* lvp = leave + (size_t)bhk * R;
+                const int l0 = e0 + lane < R ? lvp[e0 + lane] : 0, l1 = e0 + 32 + lane < R ? lvp[e0 + 32 + lane] : 0;
+                uint32_t m0 = 0, m1 = 0;
+#pragma unroll
+                for (int c = 0; c < 32; ++c) {
+                    m0 |= (__shfl_sync(0xffffffffu, l0, c) > i ? 1u : 0u) << c;
+                    m1 |= (__shfl_sync(0xffffffffu, l1, c) > i ? 1u : 0u) << c;
+                }
+                vm[0] &= m0; vm[1] &= m1;
+                full[0] = full[1] = false;
+            }
             PLM(2);
             mbar_wait(bar_s0 + 8 * (t & 1), (t >> 1) & 1, 3);  // S(t) is in TMEM buffer t & 1
             tc_fence_after();
@@ -573,7 +590,7 @@ __global__ void prefill_compact_kernel(const uint4* __restrict__ k, const uint4*
 
 template <int D>
 int run(const Params& p, const void* q, const void* k, const void* v, const int32_t* idx, const int32_t* cnt, void* o,
-        float* lse, void* ws, size_t ws_bytes, cudaStream_t st)
+        float* lse, void* ws, size_t ws_bytes, cudaStream_t st, const int32_t* leave)
 {
     CUtensorMap tq, tk, tv, to, tkc, tvc;
     const int BHK = p.B * p.H, BH = BHK * p.G;                 // key/value heads, query heads
@@ -592,17 +609,24 @@ int run(const Params& p, const void* q, const void* k, const void* v, const int3
     }
     static PerDeviceOnce attr;
     if (int e = attr.run([] {
-            const cudaError_t a = cudaFuncSetAttribute(prefill_long_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::BYTES);
-            return a != cudaSuccess ? a : cudaFuncSetAttribute(prefill_long_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::BYTES);
+            cudaError_t a = cudaFuncSetAttribute(prefill_long_kernel<D, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::BYTES);
+            if (a == cudaSuccess) a = cudaFuncSetAttribute(prefill_long_kernel<D, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::BYTES);
+            return a != cudaSuccess ? a : cudaFuncSetAttribute(prefill_long_kernel<D, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::BYTES);
         })) return e;
     dim3 grid((Tq + BM - 1) / BM, BH);
+    if (leave != nullptr) {
+        if (!compact) return LTE_ERR_UNSUPPORTED;             // the streaming variant takes compacted rows only
+        return cuda_status(launch_pdl(prefill_long_kernel<D, true, true>, grid, dim3(NTHREADS), Smem<D>::BYTES, st, tq, tk, tv, to, tkc, tvc,
+                                      (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, idx, cnt, leave, (__nv_bfloat16*)o, lse, p.T, p.W, p.R,
+                                      p.scale, p.G, p.qoff));
+    }
     if (compact)
-        return cuda_status(launch_pdl(prefill_long_kernel<D, true>, grid, dim3(NTHREADS), Smem<D>::BYTES, st, tq, tk, tv, to, tkc, tvc, (const __nv_bfloat16*)k,
-                                                                 (const __nv_bfloat16*)v, idx, cnt, (__nv_bfloat16*)o,
-                                                                 lse, p.T, p.W, p.R, p.scale, p.G, p.qoff));
-    return cuda_status(launch_pdl(prefill_long_kernel<D, false>, grid, dim3(NTHREADS), Smem<D>::BYTES, st, tq, tk, tv, to, tkc, tvc, (const __nv_bfloat16*)k,
-                                                                 (const __nv_bfloat16*)v, idx, cnt, (__nv_bfloat16*)o,
-                                                                 lse, p.T, p.W, p.R, p.scale, p.G, p.qoff));
+        return cuda_status(launch_pdl(prefill_long_kernel<D, true, false>, grid, dim3(NTHREADS), Smem<D>::BYTES, st, tq, tk, tv, to, tkc, tvc,
+                                      (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, idx, cnt, leave, (__nv_bfloat16*)o, lse, p.T, p.W, p.R,
+                                      p.scale, p.G, p.qoff));
+    return cuda_status(launch_pdl(prefill_long_kernel<D, false, false>, grid, dim3(NTHREADS), Smem<D>::BYTES, st, tq, tk, tv, to, tkc, tvc,
+                                  (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, idx, cnt, leave, (__nv_bfloat16*)o, lse, p.T, p.W, p.R,
+                                  p.scale, p.G, p.qoff));
 }
 
 }  // namespace
@@ -624,10 +648,10 @@ int launch_prefill_compact(const Params& p, const void* k, const void* v, const 
 }
 
 int launch_prefill_tc_long(const Params& p, const void* q, const void* k, const void* v, const int32_t* idx,
-                           const int32_t* cnt, void* o, float* lse, void* ws, size_t ws_bytes, cudaStream_t st)
+                           const int32_t* cnt, void* o, float* lse, void* ws, size_t ws_bytes, cudaStream_t st, const int32_t* leave)
 {
     if (p.d != 128) return LTE_ERR_UNSUPPORTED;
-    return run<128>(p, q, k, v, idx, cnt, o, lse, ws, ws_bytes, st);
+    return run<128>(p, q, k, v, idx, cnt, o, lse, ws, ws_bytes, st, leave);
 }
 
 #ifdef LTE_PROFILE
