@@ -31,6 +31,24 @@ def test_library_follows_the_oracle_over_a_long_run():
     assert (lam.numpy() == 0).any() and step == 399
 
 
+def test_moving_average_weights_the_new_sample_by_a_hand_computed():
+    """Algorithm 1's average with the new sample weighted by a = 2 / (1 + u/2) (the reading taken): u = 6 gives a = 1/2,
+    so from 0 the counts 8, 4, 10 give 4, 4, 7 by hand; the listing's weights the other way round would give the same
+    numbers here only by accident of a = 1/2, so u = 2 (a = 1: the average IS the last count) is checked as well."""
+    lam = torch.full((1,), 0.5, dtype=torch.float32); cbar = torch.zeros(1, dtype=torch.float32)
+    cfg = lte.LteLambdaCfg(6, 512.0, 2.0, 0.95, 1e-9, 1.0)
+    seen = []
+    for step, cnt in enumerate([8.0, 4.0, 10.0], start=1):
+        lte.lte_lambda_update(lam, cbar, torch.tensor([cnt], dtype=torch.float64), step, cfg)
+        seen.append(float(cbar[0]))
+    assert seen == [4.0, 4.0, 7.0]
+    cbar.zero_()
+    cfg2 = lte.LteLambdaCfg(2, 512.0, 2.0, 0.95, 1e-9, 1.0)
+    for step, cnt in enumerate([8.0, 4.0, 10.0], start=1):
+        lte.lte_lambda_update(lam, cbar, torch.tensor([cnt], dtype=torch.float64), step, cfg2)
+        assert float(cbar[0]) == cnt
+
+
 def test_defaults_and_argument_checks():
     L = lte.lib()
     lam = (ctypes.c_float * 2)(0.5, 0.0); cbar = (ctypes.c_float * 2)(600.0, 600.0); cnt = (ctypes.c_float * 2)(600.0, 600.0)
