@@ -100,9 +100,9 @@ def test_three_layer_stack_and_groups_host_side():
     short = lte.shape(4, 16, 4096, 64, 16, 8, lte.BF16)
     assert L.lte_cache_score(a(short), a(stack), fake, fake, 1 << 30, None) == -1
     assert L.lte_attn_decode(a(short), a(stack), fake, fake, fake, fake, fake, fake, None) == -1
-    # the stack's backward: d = 64 only; negative group counts are rejected everywhere
-    s32 = lte.shape(1, 2, 128, 32, 16, 8, lte.BF16)
-    args = [a(s32), a(stack)] + [fake] * 9 + [None] + [fake] * 4 + [None, 0, fake, 1 << 30, None]
+    # the stack's backward: d = 64 and d = 32 only; negative group counts are rejected everywhere
+    s128 = lte.shape(1, 2, 128, 128, 16, 8, lte.BF16)
+    args = [a(s128), a(stack)] + [fake] * 9 + [None] + [fake] * 4 + [None, 0, fake, 1 << 30, None]
     assert L.lte_attn_bwd(*args) == -2
     neg = lte.shape(1, 2, 128, 64, 16, 8, lte.BF16, group=-1)
     assert L.lte_attn_prefill(a(neg), fake, fake, fake, fake, fake, fake, fake, None, 0, None) == -1
