@@ -72,7 +72,8 @@ def test_select_exact_on_ties_and_ranks():
     # lte_select alone on hand-made logits with many exact ties: must equal the oracle bit for bit.
     rng = np.random.default_rng(0)
     for T, W, R, sink in [(50, 7, 5, 0), (4096, 128, 128, 0), (3000, 1, 2999, 3), (9000, 500, 1, 0), (40000, 512, 512, 4),
-                          (20001, 100, 77, 2), (65000, 64, 4000, 0)]:   # the last three: a cluster of blocks per head
+                          (20001, 100, 77, 2), (65000, 64, 4000, 0),   # these three and the next: a cluster of blocks per head
+                          (16512, 128, 0, 0), (20000, 100, 25000, 1), (16384 + 64, 64, 3, 0)]:   # no budget; budget above the candidates; smallest N
         z = (np.round(rng.standard_normal((2, 3, T)) * 4) / 4).astype(np.float32)
         z[0, 0] = 1.0                      # all equal and positive: oldest R win
         z[0, 1] = -1.0                     # nothing passes
