@@ -175,8 +175,8 @@ int lte_attn_colsum(const lte_shape* s, const void* q, const void* k, const floa
  *   idx, cnt in   as written by lte_select (idx ascending; entries >= cnt ignored)
  *   o        out  [B,H*group,T,d] of s->dtype
  *   lse      out  [B,H*group,T] fp32 (natural log)
- *   ws       optional device scratch of lte_workspace_bytes(LTE_OP_PREFILL, s, NULL) bytes, 128-byte aligned (bf16 with
- *            d = 64 or 128): the retained rows idx[:cnt] of k and v are first copied into it as contiguous tensors
+ *   ws       optional device scratch of lte_workspace_bytes(LTE_OP_PREFILL, s, NULL) bytes, 128-byte aligned (bf16, any
+ *            supported d): the retained rows idx[:cnt] of k and v are first copied into it as contiguous tensors
  *            [B*H][R][d] (the compaction of Section 3.1.3), and the attention kernel then fetches retained tiles as whole
  *            boxes like the window tiles.  NULL (or too small, or misaligned): the kernel gathers the retained rows itself,
  *            row by row (slower; same results).

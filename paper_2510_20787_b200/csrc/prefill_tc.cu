@@ -125,7 +125,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                   const __nv_bfloat16* __restrict__ kg,
                   const __nv_bfloat16* __restrict__ vg, __nv_bfloat16* __restrict__ og, const int32_t* __restrict__ idx,
                   const int32_t* __restrict__ cnt, const int32_t* __restrict__ leave, float* __restrict__ lse, int Tlen,
-                  int W, int R, float scale, int n_qt, int n_bh, int G, int qoff)
+                  int W, int R, float scale, int n_qt, int n_bh, int G, int qoff, int dg)
 {
     const int n_items = n_qt * n_bh;
 #ifdef LTE_PROFILE
@@ -379,11 +379,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     for (int ps = 0; ps < 4; ++ps) {
                         const int row = ps * 16 + g_row;
                         const bool ok = rows4[ps] >= 0;
-                        const __nv_bfloat16* src = (is_v ? vg : kg) + ((size_t)bhk * Tlen + (ok ? rows4[ps] : 0)) * D;
+                        const __nv_bfloat16* src = (is_v ? vg : kg) + ((size_t)bhk * Tlen + (ok ? rows4[ps] : 0)) * dg;
 #pragma unroll
                         for (int c = g_sub; c < D / 8; c += 8) {
                             const uint32_t off = (c >> 3) * 8192 + row * 128 + (((c & 7) ^ (row & 7)) << 4);
-                            cp_async16(dst + off, src + c * 8, ok ? 16u : 0u);
+                            const bool real = ok && c * 8 < dg;    // columns past the head dimension are zero-filled
+                            cp_async16(dst + off, src + (real ? c * 8 : 0), real ? 16u : 0u);
                         }
                     }
                 }
@@ -583,7 +584,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             const float inv = 1.f / l_run;
             // a normalised row is D * 2 contiguous bytes of the output (whole 128-byte lines, and the rows of a warp are
             // consecutive): each thread stores its own row with 16-byte stores, no staging in shared memory
-            __nv_bfloat16* orow = og + ((size_t)bh * (Tlen - qoff) + (i - qoff)) * D;
+            __nv_bfloat16* orow = og + ((size_t)bh * (Tlen - qoff) + (i - qoff)) * dg;
 #pragma unroll
             for (int sb = 0; sb < SUB; ++sb) {
                 uint32_t ow[32];                               // 64 columns of the row as bf16 pairs
@@ -607,7 +608,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 if (i < Tlen) {
 #pragma unroll
                     for (int ch = 0; ch < 8; ++ch)
-                        *reinterpret_cast<uint4*>(orow + sb * 64 + ch * 8) = make_uint4(ow[4 * ch], ow[4 * ch + 1], ow[4 * ch + 2], ow[4 * ch + 3]);
+                        if (sb * 64 + ch * 8 < dg)
+                            *reinterpret_cast<uint4*>(orow + sb * 64 + ch * 8) = make_uint4(ow[4 * ch], ow[4 * ch + 1], ow[4 * ch + 2], ow[4 * ch + 3]);
                 }
             }
             if (i < Tlen) lse[(size_t)bh * (Tlen - qoff) + (i - qoff)] = m_run * 0.6931471805599453f + logf(l_run);
@@ -628,7 +630,10 @@ int run(const Params& p, const void* q, const void* k, const void* v, const int3
     CUtensorMap tq, tk, tv, tkc, tvc;
     const int BHK = p.B * p.H, BH = BHK * p.G;                 // key/value heads, query heads
     const int Tq = p.T - p.qoff;                               // query rows (the whole sequence unless a chunk is prefilled)
-    if (!make_map(&tq, q, BH, Tq, D, BM) || !make_map(&tk, k, BHK, p.T, D, BN) || !make_map(&tv, v, BHK, p.T, D, BN)) return LTE_ERR_CUDA;
+    // head dimension in memory: D, or half of it (d = 32 runs the d = 64 kernel: the tensor maps' 64-column boxes reach past
+    // the 32 columns a row has and the copy engine fills the rest of every tile row with zeros, which change no product)
+    const int dg = p.d;
+    if (!make_map(&tq, q, BH, Tq, dg, BM) || !make_map(&tk, k, BHK, p.T, dg, BN) || !make_map(&tv, v, BHK, p.T, dg, BN)) return LTE_ERR_CUDA;
     // with a workspace the retained rows are compacted first and every tile is a TMA box
     const size_t half = prefill_compact_bytes(p) / 2;
     const bool compact = ws != nullptr && half > 0 && ws_bytes >= 2 * half && ((uintptr_t)ws & 127u) == 0;
@@ -636,7 +641,7 @@ int run(const Params& p, const void* q, const void* k, const void* v, const int3
     if (compact) {
         char* kc = (char*)ws; char* vc = kc + half;
         if (int e = launch_prefill_compact(p, k, v, idx, cnt, kc, vc, st)) return e;
-        if (!make_map(&tkc, kc, BHK, p.R, D, BN) || !make_map(&tvc, vc, BHK, p.R, D, BN)) return LTE_ERR_CUDA;
+        if (!make_map(&tkc, kc, BHK, p.R, dg, BN) || !make_map(&tvc, vc, BHK, p.R, dg, BN)) return LTE_ERR_CUDA;
     }
     static PerDeviceOnce attr;
     if (int e = attr.run([] {
@@ -653,15 +658,15 @@ int run(const Params& p, const void* q, const void* k, const void* v, const int3
         if (!compact) return LTE_ERR_UNSUPPORTED;             // the streaming variant takes compacted rows only
         return cuda_status(launch_pdl(prefill_tc_kernel<D, true, true>, dim3(grid), dim3(NTHREADS), Smem<D>::BYTES, st, tq, tk, tv, tkc, tvc,
                                       (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (__nv_bfloat16*)o, idx, cnt, leave, lse, p.T, p.W, p.R,
-                                      p.scale, n_qt, BH, p.G, p.qoff));
+                                      p.scale, n_qt, BH, p.G, p.qoff, dg));
     }
     if (compact)
         return cuda_status(launch_pdl(prefill_tc_kernel<D, true, false>, dim3(grid), dim3(NTHREADS), Smem<D>::BYTES, st, tq, tk, tv, tkc, tvc,
                                       (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (__nv_bfloat16*)o, idx, cnt, leave, lse, p.T, p.W, p.R,
-                                      p.scale, n_qt, BH, p.G, p.qoff));
+                                      p.scale, n_qt, BH, p.G, p.qoff, dg));
     return cuda_status(launch_pdl(prefill_tc_kernel<D, false, false>, dim3(grid), dim3(NTHREADS), Smem<D>::BYTES, st, tq, tk, tv, tkc, tvc,
                                   (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (__nv_bfloat16*)o, idx, cnt, leave, lse, p.T, p.W, p.R,
-                                  p.scale, n_qt, BH, p.G, p.qoff));
+                                  p.scale, n_qt, BH, p.G, p.qoff, dg));
 }
 
 }  // namespace
@@ -671,7 +676,7 @@ int run(const Params& p, const void* q, const void* k, const void* v, const int3
 int launch_prefill_tc(const Params& p, const void* q, const void* k, const void* v, const int32_t* idx,
                       const int32_t* cnt, void* o, float* lse, void* ws, size_t ws_bytes, cudaStream_t st, const int32_t* leave)
 {
-    if (p.d == 64) {
+    if (p.d == 64 || p.d == 32) {
         const int e = run<64>(p, q, k, v, idx, cnt, o, lse, ws, ws_bytes, st, leave);
         if (e != LTE_ERR_UNSUPPORTED || leave == nullptr) return e;
     }
@@ -684,7 +689,7 @@ int launch_prefill_tc(const Params& p, const void* q, const void* k, const void*
     }
     // d = 128: ten and more key tiles per item; one CTA per item under the hardware scheduler is faster there
     if (p.d == 128) return launch_prefill_tc_long(p, q, k, v, idx, cnt, o, lse, ws, ws_bytes, st);
-    return launch_prefill_simt(p, q, k, v, idx, cnt, o, lse, st);   // d = 32: rows too narrow for the 128-byte swizzle
+    return launch_prefill_simt(p, q, k, v, idx, cnt, o, lse, st);
 }
 
 

@@ -634,7 +634,7 @@ int run(const Params& p, const void* q, const void* k, const void* v, const int3
 // bytes of the two compacted tensors (keys, then values), each a multiple of 128; 0 where there is nothing to compact
 size_t prefill_compact_bytes(const Params& p)
 {
-    if (p.dtype != LTE_BF16 || (p.d != 64 && p.d != 128) || p.R <= 0) return 0;
+    if (p.dtype != LTE_BF16 || (p.d != 32 && p.d != 64 && p.d != 128) || p.R <= 0) return 0;
     const size_t one = ((size_t)p.B * p.H * p.R * p.d * 2 + 127) / 128 * 128;
     return 2 * one;
 }

@@ -153,7 +153,7 @@ def test_caller_made_list_uniform_stride(dtype, d, T, W, R):
     _assert_close(cfg, (o.float().cpu().numpy(), lse.cpu().numpy(), o64, l64))
 
 
-@pytest.mark.parametrize("d,T,W,R", [(64, 1100, 96, 200), (128, 900, 64, 130), (64, 300, 40, 0)])
+@pytest.mark.parametrize("d,T,W,R", [(64, 1100, 96, 200), (128, 900, 64, 130), (64, 300, 40, 0), (32, 700, 48, 90)])
 def test_compacted_and_gathered_retained_rows_agree(d, T, W, R):
     """With a workspace the retained rows are compacted and fetched as tiles, without one they are gathered row by row:
     two kernels variants, the same numbers (bit for bit: the products and their order are the same)."""
