@@ -73,7 +73,7 @@ typedef struct lte_conv {
  *   w    = wl0 [H, d, 3, 2d] | wl1 [H, d/2, 3, d] | wl2 [H, d/4, 3, d/2] | wout [H, d/4]    (one fp32 buffer, 16-byte aligned;
  *          wl[o][tau][c] multiplies channel c of the input at time t - (2 - tau) * 2)
  *   bias = bl0 [H, d] | bl1 [H, d/2] | bl2 [H, d/4] | bout [H], or NULL for zero.
- * With bf16 inputs, d = 64, T > 12 and a workspace of lte_workspace_bytes(LTE_OP_SCORES, s, c) bytes (128-byte
+ * With bf16 inputs, d = 64 or 32, T > 12 and a workspace of lte_workspace_bytes(LTE_OP_SCORES, s, c) bytes (128-byte
  * aligned; it receives the weights split into bf16 pieces, rebuilt by every call) the stack runs on the tensor cores
  * with exact products and fp32 accumulation; without the workspace, and for every other accepted shape, on the fp32
  * ALUs.  Both agree with an fp64 evaluation to about 1e-5 at |z| of a few units.

@@ -111,42 +111,51 @@ __device__ __forceinline__ void split3(float a, float b, uint32_t& hi, uint32_t&
 
 // ---- weight image -------------------------------------------------------------------------------------------------
 // blockIdx.x = head, the blocks along y share its elements.  wpack = wl0 | wl1 | wl2 | wout with wl[l] [H][c_out][3][c_in]; bpack = bl0 | bl1 | bl2 | bout or null.
-__global__ void stack_image_kernel(const float* __restrict__ wpack, const float* __restrict__ bpack, uint8_t* __restrict__ img, int H)
+// dg = the head dimension of the data, 64 or 32.  d = 32 runs the d = 64 kernel on a padded problem: channels [dg, 64) of the
+// key and value halves of the input, and the upper half of every hidden layer, carry zero weights (and zero biases, so the
+// padded activations are Swish(0) = 0); the image below is the d = 64 layout with those zeros written in.
+__global__ void stack_image_kernel(const float* __restrict__ wpack, const float* __restrict__ bpack, uint8_t* __restrict__ img, int H, int dg)
 {
     pdl_launch_dependents();
     pdl_wait();
     const int h = blockIdx.x, tid = blockIdx.y * blockDim.x + threadIdx.x, nthr = gridDim.y * blockDim.x;
     uint8_t* out = img + (size_t)h * IMG_HEAD;
-    const float* g0 = wpack + (size_t)h * ST_C1 * 3 * ST_C0;
-    const float* g1 = wpack + (size_t)H * ST_C1 * 3 * ST_C0 + (size_t)h * ST_C2 * 3 * ST_C1;
-    const float* g2 = wpack + (size_t)H * (ST_C1 * 3 * ST_C0 + ST_C2 * 3 * ST_C1) + (size_t)h * ST_C3 * 3 * ST_C2;
-    const float* go = wpack + (size_t)H * (ST_C1 * 3 * ST_C0 + ST_C2 * 3 * ST_C1 + ST_C3 * 3 * ST_C2) + (size_t)h * ST_C3;
+    const int c0 = 2 * dg, c1 = dg, c2 = dg / 2, c3 = dg / 4;   // the real channel plan
+    const float* g0 = wpack + (size_t)h * c1 * 3 * c0;
+    const float* g1 = wpack + (size_t)H * c1 * 3 * c0 + (size_t)h * c2 * 3 * c1;
+    const float* g2 = wpack + (size_t)H * (c1 * 3 * c0 + c2 * 3 * c1) + (size_t)h * c3 * 3 * c2;
+    const float* go = wpack + (size_t)H * (c1 * 3 * c0 + c2 * 3 * c1 + c3 * 3 * c2) + (size_t)h * c3;
     auto piece = [](float w, int s) -> __nv_bfloat16 {
         __nv_bfloat16 p = __float2bfloat16_rn(w);
         for (int i = 0; i < s; ++i) { w -= __bfloat162float(p); p = __float2bfloat16_rn(w); }
         return p;
     };
-    auto fill = [&](uint8_t* dst, const float* g, int cin, int cout) {
-        // dst [tap][chunk cin/8][n = piece * cout + o][8] ; g [o][tap][cin]
+    // padded dims cin x cout, real dims cin_r x cout_r; split: the input channels are two halves (key, value), each with its
+    // real channels first
+    auto fill = [&](uint8_t* dst, const float* g, int cin, int cout, int cin_r, int cout_r, bool split) {
+        // dst [tap][chunk cin/8][n = piece * cout + o][8] ; g [o][tap][cin_r]
         const int n_el = 3 * cin * 3 * cout;
         __nv_bfloat16* d = reinterpret_cast<__nv_bfloat16*>(dst);
         for (int e = tid; e < n_el; e += nthr) {
             const int k8 = e & 7, n = (e >> 3) % (3 * cout), rest = (e >> 3) / (3 * cout), c = rest % (cin / 8), tau = rest / (cin / 8);
-            const int s = n / cout, o = n % cout;
-            d[e] = piece(g[((size_t)o * 3 + tau) * cin + c * 8 + k8], s);
+            const int s = n / cout, o = n % cout, ch = c * 8 + k8;
+            int cr;
+            if (split) { const int half = cin / 2, hr = cin_r / 2; cr = ch % half < hr ? (ch / half) * hr + ch % half : -1; }
+            else cr = ch < cin_r ? ch : -1;
+            d[e] = (o < cout_r && cr >= 0) ? piece(g[((size_t)o * 3 + tau) * cin_r + cr], s) : __float2bfloat16_rn(0.f);
         }
     };
-    fill(out, g0, ST_C0, ST_C1);
-    fill(out + IMG_W0, g1, ST_C1, ST_C2);
-    fill(out + IMG_W0 + IMG_W1, g2, ST_C2, ST_C3);
+    fill(out, g0, ST_C0, ST_C1, c0, c1, true);
+    fill(out + IMG_W0, g1, ST_C1, ST_C2, c1, c2, false);
+    fill(out + IMG_W0 + IMG_W1, g2, ST_C2, ST_C3, c2, c3, false);
     float* par = reinterpret_cast<float*>(out + IMG_W0 + IMG_W1 + IMG_W2);
     for (int e = tid; e < IMG_PAR / 4; e += nthr) {
         float x = 0.f;
-        if (e < 64) x = bpack ? bpack[(size_t)h * 64 + e] : 0.f;
-        else if (e < 96) x = bpack ? bpack[(size_t)H * 64 + (size_t)h * 32 + (e - 64)] : 0.f;
-        else if (e < 112) x = bpack ? bpack[(size_t)H * 96 + (size_t)h * 16 + (e - 96)] : 0.f;
-        else if (e < 128) x = go[e - 112];
-        else if (e == 128) x = bpack ? bpack[(size_t)H * 112 + h] : 0.f;
+        if (e < 64) x = (bpack && e < c1) ? bpack[(size_t)h * c1 + e] : 0.f;
+        else if (e < 96) x = (bpack && e - 64 < c2) ? bpack[(size_t)H * c1 + (size_t)h * c2 + (e - 64)] : 0.f;
+        else if (e < 112) x = (bpack && e - 96 < c3) ? bpack[(size_t)H * (c1 + c2) + (size_t)h * c3 + (e - 96)] : 0.f;
+        else if (e < 128) x = e - 112 < c3 ? go[e - 112] : 0.f;
+        else if (e == 128) x = bpack ? bpack[(size_t)H * (c1 + c2 + c3) + h] : 0.f;
         par[e] = x;
     }
 }
@@ -161,7 +170,7 @@ __device__ __forceinline__ StackWork stack_work(int f, int n_t, int B, int H) {
 __global__ void __launch_bounds__(ST_THREADS, 1)
 scores_stack_tc_kernel(const __nv_bfloat16* __restrict__ kg, const __nv_bfloat16* __restrict__ vg,
                        const uint8_t* __restrict__ img, float* __restrict__ z, float* __restrict__ r_out, int B, int H,
-                       int Tlen, int n_t, int n_flat, int per_cta)
+                       int Tlen, int n_t, int n_flat, int per_cta, int dg)
 {
     pdl_launch_dependents();
     pdl_wait();                                                // the weight image is written by the preceding kernel
@@ -209,8 +218,8 @@ scores_stack_tc_kernel(const __nv_bfloat16* __restrict__ kg, const __nv_bfloat16
         // rows and one of 4 chunks, so a quarter warp writes 128 contiguous bytes and reads full 32-byte sectors.  Rows
         // outside [0, T) are zero-filled.  (Tensor-map copies with 16-byte boxes needed about 3,600 cycles per tile.)
         auto load_x = [&](const StackWork& w) {
-            const __nv_bfloat16* kb = kg + (size_t)w.bh * Tlen * ST_D;
-            const __nv_bfloat16* vb = vg + (size_t)w.bh * Tlen * ST_D;
+            const __nv_bfloat16* kb = kg + (size_t)w.bh * Tlen * dg;
+            const __nv_bfloat16* vb = vg + (size_t)w.bh * Tlen * dg;
             const int t0 = w.tb - 12, r_in = lane & 7, cq = lane >> 3;
 #pragma unroll 1
             for (int rb = 0; rb < (ST_XROWS + 7) / 8; ++rb) {
@@ -220,8 +229,9 @@ scores_stack_tc_kernel(const __nv_bfloat16* __restrict__ kg, const __nv_bfloat16
 #pragma unroll
                     for (int cg = 0; cg < 4; ++cg) {
                         const int c = cg * 4 + cq;
-                        const __nv_bfloat16* src = (cg < 2 ? kb : vb) + (size_t)(ok ? t : 0) * ST_D + (c & 7) * 8;
-                        cp_async16(sX + c * ST_COL + r * 16, src, ok ? 16u : 0u);
+                        const bool real = ok && (c & 7) * 8 < dg;   // channels past the head dimension are zero-filled
+                        const __nv_bfloat16* src = (cg < 2 ? kb : vb) + (size_t)(real ? t : 0) * dg + (real ? (c & 7) * 8 : 0);
+                        cp_async16(sX + c * ST_COL + r * 16, src, real ? 16u : 0u);
                     }
                 }
             }
@@ -516,7 +526,7 @@ int stack_tc_status_fetch_and_clear() { return status_fetch_and_clear(g_stack_tc
 // Workspace of the tensor-core stack scorer (the split weight image), 0 where that path does not apply.
 size_t scores_stack_tc_workspace(const Params& p)
 {
-    if (p.dtype != LTE_BF16 || p.d != ST_D || p.T <= 2 * ST_HALF) return 0;
+    if (p.dtype != LTE_BF16 || (p.d != ST_D && p.d != 32) || p.T <= 2 * ST_HALF) return 0;
     return (size_t)p.H * IMG_HEAD;
 }
 
@@ -531,7 +541,7 @@ int launch_scores_stack_tc(const Params& p, const void* k, const void* v, float*
     int n_sm = 0;
     if (int e = device_sm_count(&n_sm)) return e;
     const int BH = p.B * p.H;
-    if (launch_pdl(stack_image_kernel, dim3(p.H, 32), dim3(256), 0, st, p.w, p.bias, (uint8_t*)ws, p.H) != cudaSuccess) return LTE_ERR_CUDA;
+    if (launch_pdl(stack_image_kernel, dim3(p.H, 32), dim3(256), 0, st, p.w, p.bias, (uint8_t*)ws, p.H, p.d) != cudaSuccess) return LTE_ERR_CUDA;
     const int n_t = (p.T - ST_HALF + ST_VALID - 1) / ST_VALID;
     const long long n_flat = (long long)BH * n_t;
     if (n_flat > 0x7fffffffLL) return LTE_ERR_UNSUPPORTED;
@@ -539,7 +549,7 @@ int launch_scores_stack_tc(const Params& p, const void* k, const void* v, float*
     const int per = (int)((n_flat + grid - 1) / grid);
     const int n_cta = (int)((n_flat + per - 1) / per);
     if (launch_pdl(scores_stack_tc_kernel, dim3(n_cta), dim3(ST_THREADS), ST_SMEM, st, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (const uint8_t*)ws, z, r, p.B, p.H,
-                   p.T, n_t, (int)n_flat, per) != cudaSuccess)
+                   p.T, n_t, (int)n_flat, per, p.d) != cudaSuccess)
         return LTE_ERR_CUDA;
     return cuda_status(cudaGetLastError());
 }

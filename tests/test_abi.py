@@ -86,7 +86,7 @@ def test_three_layer_stack_and_groups_host_side():
     s = lte.shape(4, 16, 4096, 64, 128, 128, lte.BF16)
     assert lte.lte_workspace_bytes(lte.OP_SCORES, s, stack) == 16 * 194176            # the split weight image per head
     assert lte.lte_workspace_bytes(lte.OP_SCORES, lte.shape(4, 16, 4096, 64, 128, 128, lte.F32), stack) == 0
-    assert lte.lte_workspace_bytes(lte.OP_SCORES, lte.shape(4, 16, 4096, 32, 128, 128, lte.BF16), stack) == 0
+    assert lte.lte_workspace_bytes(lte.OP_SCORES, lte.shape(4, 16, 4096, 32, 128, 128, lte.BF16), stack) == 16 * 194176   # d = 32 takes the same image (zero channels)
     dec = lte.lte_workspace_bytes(lte.OP_DECODE, s, stack)                             # ring copy (k, v), its logits, the image
     assert dec >= 2 * 4 * 16 * 128 * 64 * 2 + 4 * 16 * 128 * 4 + 16 * 194176
     assert lte.lte_workspace_bytes(lte.OP_DECODE, s, single) == 0

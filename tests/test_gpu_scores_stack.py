@@ -45,15 +45,16 @@ def test_stack_logits_and_selection(dtype, d, T, W, R, bias):
     check_idx(idx.cpu().numpy(), cnt.cpu().numpy(), z64, W, R, 0, 0.5)
 
 
-@pytest.mark.parametrize("B,H,T,bias", [(1, 1, 13, True), (2, 2, 126, False), (1, 2, 127, True), (2, 1, 246, True), (1, 3, 247, False),
-                                        (3, 20, 500, True), (4, 16, 4096, True)])
-def test_stack_tensor_core_path(B, H, T, bias):
-    """bf16, d = 64 with a workspace: the tensor-core kernel (three-way split operands).  Tile edges (120 logits per
-    tile), several heads per thread block and several thread blocks per head; the same call without a workspace runs
-    the fp32 kernel, and both have to agree with the oracle."""
-    cfg = synth.Config("stack", "bf16", B, H, 64, T, 8, 12, 7, 0.1)
+@pytest.mark.parametrize("B,H,T,bias,d", [(1, 1, 13, True, 64), (2, 2, 126, False, 64), (1, 2, 127, True, 64), (2, 1, 246, True, 64),
+                                          (1, 3, 247, False, 64), (3, 20, 500, True, 64), (4, 16, 4096, True, 64),
+                                          (2, 3, 300, True, 32), (1, 2, 127, False, 32), (4, 16, 2048, True, 32)])
+def test_stack_tensor_core_path(B, H, T, bias, d):
+    """bf16, d = 64 or 32 with a workspace: the tensor-core kernel (three-way split operands; d = 32 as the d = 64 problem
+    with zero channels).  Tile edges (120 logits per tile), several heads per thread block and several thread blocks per
+    head; the same call without a workspace runs the fp32 kernel, and both have to agree with the oracle."""
+    cfg = synth.Config("stack", "bf16", B, H, d, T, 8, 12, 7, 0.1)
     x = synth.make(cfg, 5)
-    wl, wout, bl, bout = _stack_params(H, 64, 5, bias)
+    wl, wout, bl, bout = _stack_params(H, d, 5, bias)
     z64 = orc.scores_stack(x["k"], x["v"], wl, bl, wout, bout)
     s = shape_of(cfg, B=B)
     t = lambda a: None if a is None else torch.from_numpy(a).cuda()
