@@ -134,8 +134,10 @@ __global__ void __launch_bounds__(NT + 64) scores_tc_kernel(const __grid_constan
                                                        const __grid_constant__ CUtensorMap tmV,
                                                        const float* __restrict__ w, const float* __restrict__ bias,
                                                        float* __restrict__ z, float* __restrict__ r, int H, int Tlen,
-                                                       int n_flat)
+                                                       int n_flat, int dg)
 {
+    // dg = the head dimension in memory: D, or D / 2 = 32 for the d = 64 kernel on d = 32 data (the tensor maps then fill
+    // the upper half of every tile row with zeros, and B carries zeros in the same columns)
     using C = ScoresTc<D, K>;
     constexpr int HALF = K / 2;
     constexpr int TJ = NT - (K - 1);
@@ -242,8 +244,9 @@ __global__ void __launch_bounds__(NT + 64) scores_tc_kernel(const __grid_constan
                 for (int q = 0; q < NCH; ++q) {
                     const int e = tid + q * NT, n = e / (2 * D / 8), c8 = e % (2 * D / 8);
                     wf[q][0] = wf[q][1] = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (n < 3 * K) {
-                        const float4* src = reinterpret_cast<const float4*>(w + ((size_t)h * K + n % K) * 2 * D + c8 * 8);
+                    const int part = c8 / (D / 8), cin = (c8 % (D / 8)) * 8;   // key or value half; channel within it
+                    if (n < 3 * K && cin < dg) {
+                        const float4* src = reinterpret_cast<const float4*>(w + ((size_t)h * K + n % K) * 2 * dg + part * dg + cin);
                         wf[q][0] = src[0]; wf[q][1] = src[1];
                     }
                 }
@@ -333,12 +336,12 @@ __global__ void __launch_bounds__(NT + 64) scores_tc_kernel(const __grid_constan
 }
 
 template <int D, int K>
-int run_tma(const Params& p, const void* k, const void* v, float* z, float* r, cudaStream_t st)
+int run_tma(const Params& p, const void* k, const void* v, float* z, float* r, cudaStream_t st, int dg = D)
 {
     using C = ScoresTc<D, K>;
     constexpr int TJ = NT - (K - 1);
     CUtensorMap tk, tv;
-    if (!make_map(&tk, k, p.B * p.H, p.T, D, NT) || !make_map(&tv, v, p.B * p.H, p.T, D, NT)) return LTE_ERR_CUDA;
+    if (!make_map(&tk, k, p.B * p.H, p.T, dg, NT) || !make_map(&tv, v, p.B * p.H, p.T, dg, NT)) return LTE_ERR_CUDA;
     static PerDeviceOnce attr;
     if (int e = attr.run([] { return cudaFuncSetAttribute(scores_tc_kernel<D, K>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::BYTES); })) return e;
     int n_sm = 0;
@@ -350,7 +353,7 @@ int run_tma(const Params& p, const void* k, const void* v, float* z, float* r, c
     const int slots = n_sm * (D == 64 ? 2 : 1);
     const int n_cta = (int)(n_flat < slots ? n_flat : slots);
     if (launch_pdl(scores_tc_kernel<D, K>, dim3(n_cta), dim3(NT + 64), C::BYTES, st, tk, tv, p.w, p.bias, z, r, p.H, p.T,
-                   (int)n_flat) != cudaSuccess)
+                   (int)n_flat, dg) != cudaSuccess)
         return LTE_ERR_CUDA;
     return cuda_status(cudaGetLastError());
 }
@@ -368,6 +371,7 @@ template <typename T, int D, int K>
 int pick(const Params& p, const void* k, const void* v, float* z, float* r, cudaStream_t st)
 {
     if constexpr (sizeof(T) == 2 && (D == 64 || D == 128)) return run_tma<D, K>(p, k, v, z, r, st);
+    else if constexpr (sizeof(T) == 2 && D == 32) return run_tma<64, K>(p, k, v, z, r, st, 32);   // zero-filled tile columns
     else return run<T, D, K>(p, k, v, z, r, st);
 }
 

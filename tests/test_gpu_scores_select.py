@@ -48,6 +48,7 @@ def test_config1_scores_and_list():
 @pytest.mark.parametrize("d,K,T,W,R,sink", [
     (32, 1, 1, 1, 1, 0), (32, 3, 7, 3, 2, 0), (64, 5, 123, 16, 8, 2), (128, 7, 130, 9, 200, 0),
     (64, 7, 517, 40, 0, 0), (32, 13, 1000, 64, 33, 4), (64, 9, 300, 400, 16, 0), (128, 11, 259, 11, 5, 7),
+    (32, 7, 4000, 128, 128, 0), (32, 5, 777, 40, 30, 2),     # bf16: the d = 64 tensor-core kernel on zero-filled tile columns
 ])
 def test_odd_shapes(dtype, d, K, T, W, R, sink):
     cfg = synth.Config("odd", dtype, 2, 3, d, T, W, R, K, 0.1, sink=sink)
