@@ -534,7 +534,7 @@ WsPlan plan(const Params& p, uint32_t flags)
         w.part_b = off; off += up((size_t)p.H * p.B * w.nchunk * 4);
     }
     w.dk32 = w.dv32 = 0;
-    const bool tc_path = p.dtype == LTE_BF16 && (p.d == 64 || p.d == 128);
+    const bool tc_path = p.dtype == LTE_BF16 && (p.d == 32 || p.d == 64 || p.d == 128);
     if ((flags & LTE_BWD_CNN_INPUT_GRAD) && !tc_path && !p.stack) {
         w.dk32 = off; off += up(bht * p.d * 4);
         w.dv32 = off; off += up(bht * p.d * 4);
@@ -561,14 +561,14 @@ int run(const Params& p, const void* q, const void* k, const void* v, const void
     const bool want_in = flags & LTE_BWD_CNN_INPUT_GRAD;
     const bool f32 = want_in && !p.stack;             // the stack's backward adds its input gradient to dk, dv in place
     dim3 grid((p.T + 3) / 4, p.B * p.H), gridq((p.T + 3) / 4, p.B * p.H * p.G);
-    if constexpr (sizeof(T) == 2 && (D == 64 || D == 128)) {
+    if constexpr (sizeof(T) == 2 && (D == 32 || D == 64 || D == 128)) {
         const int e = launch_bwd_dq_tc(p, q, k, v, o, lse, dO, idx, cnt, dq, delta, st);
         if (e != LTE_OK) return e;
     } else {
         bwd_dq_kernel<T, D><<<gridq, 128, 0, st>>>((const T*)q, (const T*)k, (const T*)v, (const T*)o, (const T*)dO, lse,
                                                    idx, cnt, (T*)dq, delta, p.T, p.W, p.R, p.scale, p.G);
     }
-    if constexpr (sizeof(T) == 2 && (D == 64 || D == 128)) {
+    if constexpr (sizeof(T) == 2 && (D == 32 || D == 64 || D == 128)) {
         // K = 5 or 7 with the single layer: the last pass (bwd_tail_kernel) also merges the retained shares and forms dz
         const bool tail_merges = !p.stack && (p.K == 5 || p.K == 7);
         const int e = launch_bwd_dkv_tc(p, q, k, v, lse, dO, delta, z, idx, cnt, lambda, dk, dv, dk32, dv32, dz, base + w.ret,
@@ -589,7 +589,7 @@ int run(const Params& p, const void* q, const void* k, const void* v, const void
     }
     const int per_head = p.K * 2 * D;
     dim3 gr((per_head + 255) / 256, p.H);
-    if constexpr (sizeof(T) == 2 && (D == 64 || D == 128)) {
+    if constexpr (sizeof(T) == 2 && (D == 32 || D == 64 || D == 128)) {
         if (p.K == 5 || p.K == 7) {                   // fused pass: dw partials and the scorer's input gradient
             int rows = 0;
             const int nch = tail_chunks(p, &rows);
@@ -606,7 +606,7 @@ int run(const Params& p, const void* q, const void* k, const void* v, const void
         (const T*)k, (const T*)v, dz, part_w, part_b, p.B, p.H, p.T, D, p.K, w.nchunk);
     bwd_conv_reduce_kernel<<<gr, 256, 0, st>>>(part_w, part_b, dw, dbias, p.B * w.nchunk, per_head);
     if (f32) {
-        if constexpr (sizeof(T) == 2 && (D == 64 || D == 128)) {
+        if constexpr (sizeof(T) == 2 && (D == 32 || D == 64 || D == 128)) {
             constexpr int ROWS = 4 * (256 / (D / 8));
             dim3 gf((p.T + ROWS - 1) / ROWS, p.B * p.H);
             const size_t sm = (size_t)(p.K * 2 * D + ROWS + p.K - 1) * sizeof(float);

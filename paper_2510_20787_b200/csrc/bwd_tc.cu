@@ -58,8 +58,10 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                  const __nv_bfloat16* __restrict__ kg, const __nv_bfloat16* __restrict__ vg,
                  const __nv_bfloat16* __restrict__ og, const __nv_bfloat16* __restrict__ dog,
                  const float* __restrict__ lse, const int32_t* __restrict__ idx, const int32_t* __restrict__ cnt,
-                 __nv_bfloat16* __restrict__ dq, float* __restrict__ delta, int Tlen, int W, int R, float scale, int G)
+                 __nv_bfloat16* __restrict__ dq, float* __restrict__ delta, int Tlen, int W, int R, float scale, int G, int dg)
 {
+    // dg = the head dimension in memory: D, or 32 for the d = 64 kernel on d = 32 data (the tensor maps then fill the upper
+    // half of every tile row with zeros on the way in and clip it on the way out; the gathers zero-fill the same columns)
     using S = SmemQ<D>;
     constexpr int SUB = S::SUB;
     constexpr bool DB = S::DB;
@@ -295,11 +297,12 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                 for (int ps = 0; ps < 4; ++ps) {
                     const int row = ps * 16 + g_row;
                     const bool ok = rows4[ps] >= 0;
-                    const __nv_bfloat16* src = (is_v ? vg : kg) + ((size_t)bhk * Tlen + (ok ? rows4[ps] : 0)) * D;
+                    const __nv_bfloat16* src = (is_v ? vg : kg) + ((size_t)bhk * Tlen + (ok ? rows4[ps] : 0)) * dg;
 #pragma unroll
                     for (int c = g_sub; c < D / 8; c += 8) {
                         const uint32_t off = (c >> 3) * 8192 + row * 128 + (((c & 7) ^ (row & 7)) << 4);
-                        cp_async16(dst + off, src + c * 8, ok ? 16u : 0u);
+                        const bool real = ok && c * 8 < dg;
+                        cp_async16(dst + off, src + (real ? c * 8 : 0), real ? 16u : 0u);
                     }
                 }
             }
@@ -464,7 +467,7 @@ bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                   const int32_t* __restrict__ cnt, __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv,
                   float* __restrict__ dk32, float* __restrict__ dv32, float* __restrict__ dr_win,
                   float* __restrict__ dk_ret, float* __restrict__ dv_ret, float* __restrict__ dr_ret, int n_wt, int Tlen,
-                  int W, int R, float scale, int G)
+                  int W, int R, float scale, int G, int dg)
 {
     using S = SmemK<D>;
     constexpr int SUB = S::SUB;
@@ -619,13 +622,13 @@ bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         const int pos = is_ret ? (e0 + tid < n_ret ? id[e0 + tid] : -1) : (j0 + tid < Tlen ? j0 + tid : -1);
         if (is_ret) {
             // this tile's K / V rows, gathered once (zero rows past the end of the list)
-            const size_t rowoff = ((size_t)bh * Tlen + (pos >= 0 ? pos : 0)) * D;
-            const uint32_t nb = pos >= 0 ? 16u : 0u;
+            const size_t rowoff = ((size_t)bh * Tlen + (pos >= 0 ? pos : 0)) * dg;   // dg: the head dimension in memory (see the dq kernel)
 #pragma unroll
             for (int c = 0; c < D / 8; ++c) {
                 const uint32_t off = (c >> 3) * 16384 + tid * 128 + (((c & 7) ^ (tid & 7)) << 4);
-                cp_async16(sK + off, kg + rowoff + c * 8, nb);
-                cp_async16(sV + off, vg + rowoff + c * 8, nb);
+                const bool real = pos >= 0 && c * 8 < dg;
+                cp_async16(sK + off, kg + rowoff + (real ? c * 8 : 0), real ? 16u : 0u);
+                cp_async16(sV + off, vg + rowoff + (real ? c * 8 : 0), real ? 16u : 0u);
             }
             cp_async_commit();
             cp_async_wait<0>();
@@ -722,7 +725,7 @@ bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         // ---- epilogue: dV, dK rows and Eq. 6's <v_j, dV_j> ------------------------------------------------------
         float dr = 0.f;
         const bool live = pos >= 0;
-        const size_t orow = is_ret ? ((size_t)bh * R + e0 + tid) * D : ((size_t)bh * Tlen + (live ? pos : 0)) * D;
+        const size_t orow = is_ret ? ((size_t)bh * R + e0 + tid) * dg : ((size_t)bh * Tlen + (live ? pos : 0)) * dg;
 #pragma unroll
         for (int half2 = 0; half2 < 2; ++half2) {              // 0: dV, 1: dK
 #pragma unroll
@@ -750,7 +753,7 @@ bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                         }
                     }
                 }
-                if (live && (is_ret || F32OUT || D != 64)) {
+                if (live && cb * 32 < dg && (is_ret || F32OUT || D != 64)) {
                     if (is_ret || F32OUT) {
                         float* dst = (is_ret ? (half2 ? dk_ret : dv_ret) : (half2 ? dk32 : dv32)) + orow + cb * 32;
 #pragma unroll
@@ -874,9 +877,9 @@ int launch_bwd_dq_tc(const Params& p, const void* q, const void* k, const void* 
                 cudaFuncAttributeMaxDynamicSharedMemorySize, SmemQ<D>::BYTES); })) return e;                       \
         launch_pdl(bwd_dq_tc_kernel<D>, grid, dim3(NTHREADS), SmemQ<D>::BYTES, st,                            \
             tq, tdo, to, tdq, tk, tv, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (const __nv_bfloat16*)o,        \
-            (const __nv_bfloat16*)dO, lse, idx, cnt, (__nv_bfloat16*)dq, delta, p.T, p.W, p.R, p.scale, p.G);      \
+            (const __nv_bfloat16*)dO, lse, idx, cnt, (__nv_bfloat16*)dq, delta, p.T, p.W, p.R, p.scale, p.G, p.d); \
     } while (0)
-    if (p.d == 64) LTE_GO(64); else if (p.d == 128) LTE_GO(128); else return LTE_ERR_UNSUPPORTED;
+    if (p.d == 64 || p.d == 32) LTE_GO(64); else if (p.d == 128) LTE_GO(128); else return LTE_ERR_UNSUPPORTED;
 #undef LTE_GO
     return cuda_status(cudaGetLastError());
 }
@@ -913,9 +916,9 @@ int launch_bwd_dkv_tc(const Params& p, const void* q, const void* k, const void*
         launch_pdl(bwd_dkv_tc_kernel<D, F>, grid, dim3(NTHREADS), SmemK<D>::BYTES, st,                              \
             tk, tv, tq, tdo, tdk, tdv, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, lse, delta, idx, cnt,     \
             (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, dk32, dv32, dz, dk_ret, dv_ret, dr_ret, n_wt, p.T, p.W, p.R,   \
-            p.scale, p.G);                                                                                         \
+            p.scale, p.G, p.d);                                                                                    \
     } while (0)
-    if (p.d == 64) { if (f32out) LTE_GO(64, true); else LTE_GO(64, false); }
+    if (p.d == 64 || p.d == 32) { if (f32out) LTE_GO(64, true); else LTE_GO(64, false); }
     else if (p.d == 128) { if (f32out) LTE_GO(128, true); else LTE_GO(128, false); }
     else return LTE_ERR_UNSUPPORTED;
 #undef LTE_GO

@@ -47,7 +47,8 @@ def _assert(cfg, res):
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("d,K,T,W,R,sink", [(32, 5, 128, 16, 8, 0), (64, 7, 300, 40, 25, 2), (128, 3, 130, 9, 200, 0),
-                                            (64, 7, 260, 300, 10, 0), (32, 1, 50, 4, 0, 0), (64, 13, 777, 64, 64, 0)])
+                                            (64, 7, 260, 300, 10, 0), (32, 1, 50, 4, 0, 0), (64, 13, 777, 64, 64, 0),
+                                            (32, 7, 900, 64, 150, 1), (32, 9, 700, 100, 40, 0)])   # bf16 d = 32: the d = 64 tensor-core kernels on zero-filled columns
 @pytest.mark.parametrize("flags", [0, 1])
 def test_small_shapes(dtype, d, K, T, W, R, sink, flags):
     cfg = synth.Config("bwd", dtype, 2, 3, d, T, W, R, K, 0.1, sink=sink, qk_unit=(dtype == "f32"))
