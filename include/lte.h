@@ -66,7 +66,7 @@ typedef struct lte_conv {
     const float* bias;             /* device, [H] fp32, or NULL for zero                                    */
 } lte_conv;
 /*
- * n_layers = 3 (accepted by lte_scores only; d = 32 or 64): the scorer of Section 3.1.1 with the hyper-parameters of
+ * n_layers = 3 (d = 32 or 64; which calls take it is said below): the scorer of Section 3.1.1 with the hyper-parameters of
  * Appendix A: three grouped conv layers of kernel = 3, dilation = 2, channels 2d -> d -> d/2 -> d/4, Swish after each,
  * then a per-head linear map to the logit; receptive field 13, the logit of token j is the output at time j + 6
  * (z_j = -inf for j > T-1-6).  Every layer's input is zero at negative times, hidden activations included.
@@ -291,9 +291,9 @@ int lte_attn_prefill_chunk(const lte_shape* s, const lte_conv* c, void* cache, i
  * lte_attn_decode compute, also where the cap R binds: an entry that a later token of the same chunk pushes out is still
  * seen by the queries before that token's.  The cache afterwards is the same under both readings.
  * The pool is walked token by token (one warp per head), which gives every entry that is retained at some query of the
- * chunk and the query from which it is gone.  bf16 with d = 64 or 128: the tiled tensor-core kernels attend over that entry
- * list with the leave times as one more mask on their retained tiles (about twice the time of the chunk-end reading);
- * fp32 and d = 32: row by row on the fp32 ALUs (exact as well, but tens of times slower).
+ * chunk and the query from which it is gone.  bf16: the tiled tensor-core kernels attend over that entry list with the
+ * leave times as one more mask on their retained tiles (about twice the time of the chunk-end reading); fp32: row by
+ * row on the fp32 ALUs (exact as well, but tens of times slower).
  *   ws   device scratch of lte_workspace_bytes(LTE_OP_CHUNK_STREAM, s, c) bytes, 256-byte aligned
  * Errors: as lte_attn_prefill_chunk; INVALID_ARG for unknown flags; UNSUPPORTED for R > 4096 with the flag.
  */

@@ -139,6 +139,7 @@ def test_serving_shape_chunk_on_a_big_cache():
     (dict(B=1, H=2, W=768, R=512, sink=4), [("prefill", 2000), ("chunk", 512), ("decode", 4)]),   # the benchmark's serving-like chunk
     (dict(B=1, H=2, W=128, R=128), [("prefill", 1500), ("chunk", 1200)]),                          # the C2 window and budget: several retained tiles
     (dict(B=1, H=2, d=128, W=96, R=70), [("prefill", 700), ("chunk", 900), ("decode", 3)]),        # d = 128: the other tiled kernel
+    (dict(B=2, H=2, d=32, W=48, R=40), [("prefill", 300), ("chunk", 500), ("decode", 3)]),         # d = 32: the d = 64 kernel on zero-filled columns
 ])
 def test_streaming_reading_at_the_benchmark_shapes(kw, plan):
     """The streaming reading on the tiled tensor-core kernel (bf16, d = 64): retained tiles of the entry list with the leave
